@@ -1,0 +1,231 @@
+/*
+ * mx.h -- C ABI of the Microscaling (MX) hot path for NVIDIA B200 (sm_100a).
+ *
+ * The library implements, as hand-written CUDA kernels, the three operations
+ * the MX paper (arXiv 2310.10537) defines:
+ *
+ *   mx_quantize    Section 3, Algorithm 1: scalar floats -> MX blocks
+ *   mx_dequantize  Section 2: v_i = X * P_i, NaN if X is NaN
+ *   mx_gemm        Section 4.1 ("Compute Flow"): dot products of two MX operands,
+ *                  scalar-float (FP32) output
+ *
+ * An MX block is k = 32 elements P_i that share one E8M0 scale X = 2^(byte-127)
+ * (Section 2, Table 1).  Element formats: FP8 E4M3 / E5M2, FP6 E3M2 / E2M3,
+ * FP4 E2M1 and INT8 (Table 1).
+ *
+ * Conventions common to every entry point
+ *   - All data pointers are DEVICE pointers unless the function name ends in
+ *     "_host".  The caller allocates and frees every buffer; the library
+ *     allocates no device memory.  Shapes and sizes are passed by value or as
+ *     HOST arrays.
+ *   - Calls are asynchronous on opts->stream (a cudaStream_t passed as void*;
+ *     NULL = the legacy default stream).  The "_host" variants synchronise the
+ *     stream before they return.
+ *   - Return value: MX_OK (0) or a negative mx_status_t.  Nothing throws,
+ *     aborts or traps.  mx_strerror() gives a static description;
+ *     mx_last_cuda_error() gives the text of the CUDA error behind the last
+ *     MX_ERR_CUDA on the calling thread.
+ *   - If the CUDA driver or a GPU is missing every compute entry point returns
+ *     MX_ERR_CUDA.  There is no CPU fallback.
+ */
+#ifndef MX_H_
+#define MX_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+/* Element data formats (Table 1).  INT8 is two's complement with value n/64. */
+typedef enum {
+  MX_E4M3 = 0, /* FP8, 4 exponent / 3 mantissa bits, max normal 448     */
+  MX_E5M2 = 1, /* FP8, 5 / 2, max normal 57344                           */
+  MX_E3M2 = 2, /* FP6, 3 / 2, max normal 28                              */
+  MX_E2M3 = 3, /* FP6, 2 / 3, max normal 7.5                             */
+  MX_E2M1 = 4, /* FP4, 2 / 1, max normal 6                               */
+  MX_INT8 = 5  /* 1 sign + 1 integer + 6 fraction bits, max 127/64       */
+} mx_fmt_t;
+
+/* Rounding of V_i / X onto the element grid (Algorithm 1, line 4).
+ * Section 4.3 uses round-half-to-even for inference, Section 4.5
+ * round-half-away-from-zero for training. */
+typedef enum { MX_RNE = 0, MX_RHAZ = 1 } mx_round_t;
+
+/* Scalar float type of the unquantized tensor. */
+typedef enum { MX_F32 = 0, MX_BF16 = 1 } mx_dtype_t;
+
+/* Where the scale byte of (row, kblock) lives.  Section 2 leaves the layout of
+ * a block free; this library keeps scales in their own tensor.
+ *   LINEAR   : scales[row * kblocks + kblock]
+ *   SWIZZLED : 512-byte chunks of 128 rows x 4 kblocks, the unit one
+ *              shared-memory -> tensor-memory copy feeds to the block-scaled
+ *              MMA.  See mx_scale_offset().  Padding bytes are written as 0. */
+typedef enum { MX_SCALES_LINEAR = 0, MX_SCALES_SWIZZLED = 1 } mx_scale_layout_t;
+
+typedef enum {
+  MX_OK = 0,
+  MX_ERR_NULL = -1,        /* a required pointer is NULL                     */
+  MX_ERR_SHAPE = -2,       /* bad ndim / axis / extent (see each function)   */
+  MX_ERR_FMT = -3,         /* enum value out of range                        */
+  MX_ERR_ALIGN = -4,       /* a pointer is not aligned as required           */
+  MX_ERR_UNSUPPORTED = -5, /* valid request this build does not implement    */
+  MX_ERR_CUDA = -6,        /* CUDA runtime / driver error                    */
+  MX_ERR_TIMEOUT = -7,     /* a bounded device-side wait gave up             */
+  MX_ERR_WORKSPACE = -8    /* caller-supplied workspace is too small         */
+} mx_status_t;
+
+/* Optional arguments.  A NULL pointer means
+ * { MX_F32, MX_SCALES_SWIZZLED, NULL stream, check_status = 0 }. */
+typedef struct {
+  int32_t dtype;        /* mx_dtype_t of the float tensor (input of quantize,
+                           output of dequantize); ignored by mx_gemm          */
+  int32_t scale_layout; /* mx_scale_layout_t of every scale tensor in the call */
+  void* stream;         /* cudaStream_t                                        */
+  int32_t check_status; /* mx_gemm: nonzero = synchronise the stream and return
+                           MX_ERR_TIMEOUT if a device-side wait expired        */
+} mx_opts_t;
+
+/* ------------------------------------------------------------------------- */
+/* Size and index helpers (host only, no CUDA calls)                         */
+/* ------------------------------------------------------------------------- */
+
+/* Bits per element code: 8, 6 or 4; 0 for an invalid format. */
+int mx_fmt_bits(mx_fmt_t fmt);
+
+/* Bytes of the packed element tensor produced by mx_quantize for a float tensor
+ * of shape[ndim] quantized along `axis`: numel * bits / 8.  0 on bad arguments
+ * (including shape[axis] % 32 != 0). */
+size_t mx_elems_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt);
+
+/* Bytes of the scale tensor for the same call.  rows = numel / shape[axis],
+ * kblocks = shape[axis] / 32.  LINEAR: rows * kblocks.
+ * SWIZZLED: ceil(rows/128) * ceil(kblocks/4) * 512.  0 on bad arguments. */
+size_t mx_scales_bytes(const int64_t* shape, int ndim, int axis, mx_scale_layout_t layout);
+
+/* Byte offset of the scale of (row, kblock) inside a scale tensor of
+ * rows x kblocks.  SWIZZLED:
+ *   ((row/128) * ceil(kblocks/4) + kblock/4) * 512
+ *     + (row%32)*16 + ((row%128)/32)*4 + kblock%4
+ * Returns (size_t)-1 on out-of-range arguments. */
+size_t mx_scale_offset(int64_t row, int64_t kblock, int64_t rows, int64_t kblocks,
+                       mx_scale_layout_t layout);
+
+const char* mx_strerror(int status);
+const char* mx_last_cuda_error(void);
+
+/* ------------------------------------------------------------------------- */
+/* mx_quantize -- Algorithm 1 (Section 3)                                    */
+/* ------------------------------------------------------------------------- */
+/*
+ * in         contiguous row-major float tensor of shape[ndim] (opts->dtype),
+ *            16-byte aligned.  View it as [outer, L, inner] with
+ *            L = shape[axis]; L must be a multiple of 32.
+ * axis       the axis the scale is shared along (Section 3, last paragraph:
+ *            normally the reduction dimension of the matmul that consumes the
+ *            tensor).  Block (o, j, b) is in[o, 32b .. 32b+31, j].
+ * elems_out  packed element codes, ALWAYS with the quantization axis innermost
+ *            ("K-major"): logical [outer*inner, L], output row o*inner + j.
+ *            For axis == ndim-1 nothing moves; for a 2-D [K x N] tensor with
+ *            axis == 0 the result is the [N x K] operand that dgrad / wgrad
+ *            need (Section 3: quantizing and transposing do not commute, so
+ *            this is a separate tensor; Section 4.1).
+ *            Codes form a little-endian bit stream along a row: code i occupies
+ *            bits [w*i, w*i + w), w = 8 / 6 / 4.  16-byte aligned,
+ *            mx_elems_bytes() long.
+ * scales_out one E8M0 byte per block, mx_scales_bytes() long, layout
+ *            opts->scale_layout; every byte of the buffer is written.
+ *            16-byte aligned.
+ *
+ * Per block: inputs whose FP32 exponent field is 0 count as signed zero
+ * (Section 3, note on subnormals); shared_exp = floor(log2(max|V_i|)) -
+ * emax_elem, clamped to [-127, 127]; an all-zero block gets scale byte 0x00; a
+ * block holding Inf or NaN gets scale byte 0xFF (X = NaN) and zero codes;
+ * P_i = V_i / X rounded (rounding) to the element grid, subnormals included,
+ * and saturated to +-max normal with the sign kept (Algorithm 1 line 4 and its
+ * note).  Results that round to zero keep their sign bit in the FP formats.
+ *
+ * Errors: MX_ERR_NULL, MX_ERR_SHAPE (ndim < 1 or > 8, axis out of range,
+ * shape[axis] % 32 != 0, an extent < 0), MX_ERR_FMT, MX_ERR_ALIGN,
+ * MX_ERR_CUDA.  A tensor with zero elements is a successful no-op.
+ */
+int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out,
+                const int64_t* shape, int ndim, int axis,
+                mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts);
+
+/* ------------------------------------------------------------------------- */
+/* mx_dequantize -- Section 2 value semantics                                */
+/* ------------------------------------------------------------------------- */
+/*
+ * elems, scales  an MX tensor as mx_quantize writes it (K-major).
+ * shape, ndim    logical float shape of that K-major tensor; axis must be
+ *                ndim-1 (anything else: MX_ERR_UNSUPPORTED).
+ * out            contiguous float tensor of that shape (opts->dtype), 16-byte
+ *                aligned.
+ * v = decode(P) * 2^(byte-127); scale byte 0xFF -> NaN for the whole block;
+ * element codes that encode NaN / Inf (E4M3 0x7F/0xFF; E5M2 0x7C-0x7F and
+ * 0xFC-0xFF) decode to NaN / +-Inf; |v| beyond the FP32 range -> +-Inf (the
+ * paper leaves that case implementation-defined).  BF16 output rounds to nearest even.
+ */
+int mx_dequantize(const void* elems, const uint8_t* scales, void* out,
+                  const int64_t* shape, int ndim, int axis,
+                  mx_fmt_t fmt, const mx_opts_t* opts);
+
+/* ------------------------------------------------------------------------- */
+/* mx_gemm -- dot products of MX operands (Section 4.1)                      */
+/* ------------------------------------------------------------------------- */
+/*
+ * A   packed [M x K] codes, K-major (fmtA);  sA its scales, rows = M.
+ * B   packed [N x K] codes, K-major (fmtB);  sB its scales, rows = N.
+ *     Scales must be in MX_SCALES_SWIZZLED layout with kblocks = K / 32.
+ * C   FP32 row-major [M x N], overwritten:
+ *       C[m,n] = sum over K-blocks b of X_A[m,b] * X_B[n,b] *
+ *                sum_{i<32} P_A[m,32b+i] * P_B[n,32b+i]
+ *     accumulated in FP32 on the tensor cores.
+ * Requirements: M, N multiples of 128, K a multiple of 128; A, B 128-byte
+ * aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
+ * (the block-scaled tensor-core instruction has no integer element type).
+ * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN,
+ * MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT (only with
+ * opts->check_status).
+ */
+int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, float* C,
+            int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+            const mx_opts_t* opts);
+
+/* ------------------------------------------------------------------------- */
+/* Host-buffer variants                                                      */
+/* ------------------------------------------------------------------------- */
+/*
+ * Same operations with HOST input and output buffers (pinned memory gives the
+ * best copy rate, pageable memory works).  The caller supplies a DEVICE
+ * workspace of at least mx_*_host_workspace_bytes(); the call copies the
+ * inputs to it, runs the device entry point above, copies the results back and
+ * synchronises opts->stream.  Additional error: MX_ERR_WORKSPACE.
+ */
+size_t mx_quantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis,
+                                        mx_fmt_t fmt, const mx_opts_t* opts);
+int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                     const int64_t* shape, int ndim, int axis,
+                     mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts,
+                     void* workspace_dev, size_t workspace_bytes);
+
+size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis,
+                                          mx_fmt_t fmt, const mx_opts_t* opts);
+int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                       const int64_t* shape, int ndim, int axis,
+                       mx_fmt_t fmt, const mx_opts_t* opts,
+                       void* workspace_dev, size_t workspace_bytes);
+
+size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K,
+                                    mx_fmt_t fmtA, mx_fmt_t fmtB);
+int mx_gemm_host(const void* A_host, const uint8_t* sA_host,
+                 const void* B_host, const uint8_t* sB_host, float* C_host,
+                 int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                 const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* MX_H_ */
