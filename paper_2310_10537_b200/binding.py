@@ -1,0 +1,233 @@
+"""ctypes binding of ``libmx_b200.so`` (the C ABI declared in ``include/mx.h``).
+
+Argument marshalling only: every function takes torch tensors (or raw
+pointers), passes ``data_ptr()`` and the current CUDA stream to the C entry point
+of the same name and raises :class:`MxError` on a nonzero status.  PyTorch owns
+the memory; all arithmetic runs in the library's CUDA kernels.  If the shared
+library is missing the import of this module fails -- there is no fallback.
+"""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Sequence, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+LIB_PATH = os.path.join(_HERE, "libmx_b200.so")
+
+# enums of include/mx.h
+MX_E4M3, MX_E5M2, MX_E3M2, MX_E2M3, MX_E2M1, MX_INT8 = range(6)
+FORMATS = {"e4m3": MX_E4M3, "e5m2": MX_E5M2, "e3m2": MX_E3M2, "e2m3": MX_E2M3,
+           "e2m1": MX_E2M1, "int8": MX_INT8}
+MX_RNE, MX_RHAZ = 0, 1
+MX_F32, MX_BF16 = 0, 1
+MX_SCALES_LINEAR, MX_SCALES_SWIZZLED = 0, 1
+MX_OK = 0
+MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN = -1, -2, -3, -4
+MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, -8
+
+EXPORTS = [
+    "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
+    "mx_last_cuda_error", "mx_quantize", "mx_dequantize", "mx_gemm",
+    "mx_quantize_host_workspace_bytes", "mx_quantize_host",
+    "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
+    "mx_gemm_host_workspace_bytes", "mx_gemm_host",
+]
+
+
+class mx_opts_t(ctypes.Structure):
+    _fields_ = [("dtype", ctypes.c_int32), ("scale_layout", ctypes.c_int32),
+                ("stream", ctypes.c_void_p), ("check_status", ctypes.c_int32)]
+
+
+class MxError(RuntimeError):
+    def __init__(self, status: int, where: str):
+        self.status = status
+        msg = _lib.mx_strerror(status).decode()
+        if status == MX_ERR_CUDA:
+            msg += ": " + _lib.mx_last_cuda_error().decode()
+        super().__init__(f"{where}: {msg} ({status})")
+
+
+def _load() -> ctypes.CDLL:
+    if not os.path.exists(LIB_PATH):
+        raise ImportError(
+            f"{LIB_PATH} is missing: build it with `python -m paper_2310_10537_b200.build` "
+            "(the library has no CPU or PyTorch fallback)")
+    lib = ctypes.CDLL(LIB_PATH)
+    vp, i64p, u8p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_void_p
+    ci, i64, sz = ctypes.c_int, ctypes.c_int64, ctypes.c_size_t
+    op = ctypes.POINTER(mx_opts_t)
+    lib.mx_fmt_bits.argtypes = [ci]
+    lib.mx_elems_bytes.argtypes = [i64p, ci, ci, ci]
+    lib.mx_elems_bytes.restype = sz
+    lib.mx_scales_bytes.argtypes = [i64p, ci, ci, ci]
+    lib.mx_scales_bytes.restype = sz
+    lib.mx_scale_offset.argtypes = [i64, i64, i64, i64, ci]
+    lib.mx_scale_offset.restype = sz
+    lib.mx_strerror.argtypes = [ci]
+    lib.mx_strerror.restype = ctypes.c_char_p
+    lib.mx_last_cuda_error.restype = ctypes.c_char_p
+    lib.mx_quantize.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op]
+    lib.mx_dequantize.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op]
+    lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
+    lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
+    lib.mx_quantize_host_workspace_bytes.restype = sz
+    lib.mx_quantize_host.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op, vp, sz]
+    lib.mx_dequantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
+    lib.mx_dequantize_host_workspace_bytes.restype = sz
+    lib.mx_dequantize_host.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op, vp, sz]
+    lib.mx_gemm_host_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
+    lib.mx_gemm_host_workspace_bytes.restype = sz
+    lib.mx_gemm_host.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op, vp, sz]
+    return lib
+
+
+_lib = _load()
+
+
+def lib() -> ctypes.CDLL:
+    """The loaded C library (for callers that pass raw pointers)."""
+    return _lib
+
+
+def _shape_arr(shape: Sequence[int]):
+    return (ctypes.c_int64 * len(shape))(*[int(s) for s in shape])
+
+
+def _dtype_code(dt: torch.dtype) -> int:
+    if dt == torch.float32:
+        return MX_F32
+    if dt == torch.bfloat16:
+        return MX_BF16
+    raise TypeError(f"unsupported float dtype {dt}")
+
+
+def _opts(dtype: int, layout: int, check: bool = False, stream: Optional[int] = None) -> mx_opts_t:
+    if stream is None:
+        stream = torch.cuda.current_stream().cuda_stream
+    return mx_opts_t(dtype, layout, ctypes.c_void_p(stream), 1 if check else 0)
+
+
+def _check(status: int, where: str) -> None:
+    if status != MX_OK:
+        raise MxError(status, where)
+
+
+def mx_fmt_bits(fmt: int) -> int:
+    return _lib.mx_fmt_bits(fmt)
+
+
+def mx_elems_bytes(shape: Sequence[int], axis: int, fmt: int) -> int:
+    return int(_lib.mx_elems_bytes(_shape_arr(shape), len(shape), axis, fmt))
+
+
+def mx_scales_bytes(shape: Sequence[int], axis: int, layout: int = MX_SCALES_SWIZZLED) -> int:
+    return int(_lib.mx_scales_bytes(_shape_arr(shape), len(shape), axis, layout))
+
+
+def mx_scale_offset(row: int, kblock: int, rows: int, kblocks: int,
+                    layout: int = MX_SCALES_SWIZZLED) -> int:
+    return int(_lib.mx_scale_offset(row, kblock, rows, kblocks, layout))
+
+
+def mx_quantize(x: torch.Tensor, axis: int, fmt: int, rounding: int = MX_RNE,
+                layout: int = MX_SCALES_SWIZZLED,
+                out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None
+                ) -> Tuple[torch.Tensor, torch.Tensor]:
+    """Quantize a contiguous CUDA tensor along ``axis`` (Algorithm 1).
+
+    Returns (elems, scales) as flat uint8 tensors; the packed tensor has the
+    quantization axis innermost.  ``out`` lets the caller reuse buffers."""
+    assert x.is_cuda and x.is_contiguous()
+    axis %= x.dim()
+    shape = list(x.shape)
+    if out is None:
+        elems = torch.empty(mx_elems_bytes(shape, axis, fmt), dtype=torch.uint8, device=x.device)
+        scales = torch.empty(mx_scales_bytes(shape, axis, layout), dtype=torch.uint8, device=x.device)
+    else:
+        elems, scales = out
+    o = _opts(_dtype_code(x.dtype), layout)
+    _check(_lib.mx_quantize(x.data_ptr(), elems.data_ptr(), scales.data_ptr(), _shape_arr(shape),
+                            len(shape), axis, fmt, rounding, ctypes.byref(o)), "mx_quantize")
+    return elems, scales
+
+
+def mx_dequantize(elems: torch.Tensor, scales: torch.Tensor, shape: Sequence[int], fmt: int,
+                  dtype: torch.dtype = torch.float32, layout: int = MX_SCALES_SWIZZLED,
+                  out: Optional[torch.Tensor] = None) -> torch.Tensor:
+    """Dequantize a packed MX tensor of logical shape ``shape`` (blocks along the last axis)."""
+    assert elems.is_cuda and scales.is_cuda
+    shape = list(shape)
+    if out is None:
+        out = torch.empty(shape, dtype=dtype, device=elems.device)
+    o = _opts(_dtype_code(out.dtype), layout)
+    _check(_lib.mx_dequantize(elems.data_ptr(), scales.data_ptr(), out.data_ptr(),
+                              _shape_arr(shape), len(shape), len(shape) - 1, fmt,
+                              ctypes.byref(o)), "mx_dequantize")
+    return out
+
+
+def mx_gemm(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
+            M: int, N: int, K: int, fmtA: int, fmtB: int,
+            out: Optional[torch.Tensor] = None, check_status: bool = False) -> torch.Tensor:
+    """C[M,N] = A[M,K] . B[N,K]^T on MX operands (swizzled scales), FP32 output."""
+    assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
+    if out is None:
+        out = torch.empty((M, N), dtype=torch.float32, device=A.device)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    _check(_lib.mx_gemm(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(), out.data_ptr(),
+                        M, N, K, fmtA, fmtB, ctypes.byref(o)), "mx_gemm")
+    return out
+
+
+# ---- host-buffer variants: tensors live in (pinned) host memory ----------------
+
+def mx_quantize_host_workspace_bytes(shape, axis, fmt, dtype, layout=MX_SCALES_SWIZZLED) -> int:
+    o = _opts(_dtype_code(dtype), layout, stream=0)
+    return int(_lib.mx_quantize_host_workspace_bytes(_shape_arr(shape), len(shape), axis, fmt,
+                                                     ctypes.byref(o)))
+
+
+def mx_quantize_host(x: torch.Tensor, elems: torch.Tensor, scales: torch.Tensor, axis: int,
+                     fmt: int, rounding: int, workspace: torch.Tensor,
+                     layout: int = MX_SCALES_SWIZZLED) -> None:
+    assert not x.is_cuda and not elems.is_cuda and not scales.is_cuda and workspace.is_cuda
+    shape = list(x.shape)
+    o = _opts(_dtype_code(x.dtype), layout)
+    _check(_lib.mx_quantize_host(x.data_ptr(), elems.data_ptr(), scales.data_ptr(),
+                                 _shape_arr(shape), len(shape), axis % len(shape), fmt, rounding,
+                                 ctypes.byref(o), workspace.data_ptr(), workspace.numel()),
+           "mx_quantize_host")
+
+
+def mx_dequantize_host_workspace_bytes(shape, fmt, dtype, layout=MX_SCALES_SWIZZLED) -> int:
+    o = _opts(_dtype_code(dtype), layout, stream=0)
+    return int(_lib.mx_dequantize_host_workspace_bytes(_shape_arr(shape), len(shape),
+                                                       len(shape) - 1, fmt, ctypes.byref(o)))
+
+
+def mx_dequantize_host(elems: torch.Tensor, scales: torch.Tensor, out: torch.Tensor, fmt: int,
+                       workspace: torch.Tensor, layout: int = MX_SCALES_SWIZZLED) -> None:
+    assert not elems.is_cuda and not scales.is_cuda and not out.is_cuda and workspace.is_cuda
+    shape = list(out.shape)
+    o = _opts(_dtype_code(out.dtype), layout)
+    _check(_lib.mx_dequantize_host(elems.data_ptr(), scales.data_ptr(), out.data_ptr(),
+                                   _shape_arr(shape), len(shape), len(shape) - 1, fmt,
+                                   ctypes.byref(o), workspace.data_ptr(), workspace.numel()),
+           "mx_dequantize_host")
+
+
+def mx_gemm_host_workspace_bytes(M: int, N: int, K: int, fmtA: int, fmtB: int) -> int:
+    return int(_lib.mx_gemm_host_workspace_bytes(M, N, K, fmtA, fmtB))
+
+
+def mx_gemm_host(A, sA, B, sB, C, M: int, N: int, K: int, fmtA: int, fmtB: int,
+                 workspace: torch.Tensor) -> None:
+    assert not A.is_cuda and not C.is_cuda and workspace.is_cuda
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED)
+    _check(_lib.mx_gemm_host(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
+                             C.data_ptr(), M, N, K, fmtA, fmtB, ctypes.byref(o),
+                             workspace.data_ptr(), workspace.numel()), "mx_gemm_host")

@@ -1,0 +1,271 @@
+// C ABI of the library (declared in include/mx.h): argument validation, size
+// helpers, kernel dispatch and the host-buffer variants.  No arithmetic of the
+// method lives here.
+#include <cuda_runtime.h>
+
+#include <cstdio>
+#include <cstring>
+
+#include "mx.h"
+#include "mx_launch.h"
+
+namespace {
+
+thread_local char g_cuda_error[256] = "";
+
+int fail_cuda(cudaError_t e) {
+  std::snprintf(g_cuda_error, sizeof(g_cuda_error), "%s: %s", cudaGetErrorName(e),
+                cudaGetErrorString(e));
+  return MX_ERR_CUDA;
+}
+
+bool fmt_ok(int f) { return f >= MX_E4M3 && f <= MX_INT8; }
+int fmt_bits(int f) {
+  switch (f) {
+    case MX_E4M3: case MX_E5M2: case MX_INT8: return 8;
+    case MX_E3M2: case MX_E2M3: return 6;
+    case MX_E2M1: return 4;
+    default: return 0;
+  }
+}
+
+struct View {
+  int64_t outer, L, inner, numel, rows, kblocks;
+};
+
+// [outer, L, inner] view of shape[ndim] around `axis`; false on a bad shape.
+bool make_view(const int64_t* shape, int ndim, int axis, View* v) {
+  if (!shape || ndim < 1 || ndim > 8 || axis < 0 || axis >= ndim) return false;
+  v->outer = v->inner = 1;
+  for (int i = 0; i < ndim; ++i) {
+    if (shape[i] < 0) return false;
+    if (i < axis) v->outer *= shape[i];
+    if (i > axis) v->inner *= shape[i];
+  }
+  v->L = shape[axis];
+  if (v->L % 32 != 0) return false;
+  v->numel = v->outer * v->L * v->inner;
+  v->rows = v->outer * v->inner;
+  v->kblocks = v->L / 32;
+  return true;
+}
+
+size_t scales_bytes(int64_t rows, int64_t kblocks, int layout) {
+  if (layout == MX_SCALES_LINEAR) return (size_t)(rows * kblocks);
+  return (size_t)(((rows + 127) / 128) * ((kblocks + 3) / 4) * 512);
+}
+
+struct Opts {
+  int dtype, layout, check;
+  cudaStream_t stream;
+};
+bool read_opts(const mx_opts_t* o, Opts* out) {
+  out->dtype = o ? o->dtype : MX_F32;
+  out->layout = o ? o->scale_layout : MX_SCALES_SWIZZLED;
+  out->stream = o ? (cudaStream_t)o->stream : nullptr;
+  out->check = o ? o->check_status : 0;
+  return (out->dtype == MX_F32 || out->dtype == MX_BF16) &&
+         (out->layout == MX_SCALES_LINEAR || out->layout == MX_SCALES_SWIZZLED);
+}
+
+// SM count of the current device, cached per device ordinal.
+int sm_count(cudaError_t* err) {
+  static int cache[64] = {0};
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return 0;
+  if (dev >= 0 && dev < 64 && cache[dev]) return cache[dev];
+  int n = 0;
+  *err = cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+  if (*err != cudaSuccess) return 0;
+  if (dev >= 0 && dev < 64) cache[dev] = n;
+  return n;
+}
+
+size_t align_up(size_t x, size_t a) { return (x + a - 1) / a * a; }
+
+}  // namespace
+
+extern "C" {
+
+int mx_fmt_bits(mx_fmt_t fmt) { return fmt_bits((int)fmt); }
+
+size_t mx_elems_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt) {
+  View v;
+  if (!fmt_ok((int)fmt) || !make_view(shape, ndim, axis, &v)) return 0;
+  return (size_t)(v.numel / 8 * fmt_bits((int)fmt));
+}
+
+size_t mx_scales_bytes(const int64_t* shape, int ndim, int axis, mx_scale_layout_t layout) {
+  View v;
+  if ((layout != MX_SCALES_LINEAR && layout != MX_SCALES_SWIZZLED) ||
+      !make_view(shape, ndim, axis, &v))
+    return 0;
+  return scales_bytes(v.rows, v.kblocks, (int)layout);
+}
+
+size_t mx_scale_offset(int64_t row, int64_t kblock, int64_t rows, int64_t kblocks,
+                       mx_scale_layout_t layout) {
+  if (row < 0 || row >= rows || kblock < 0 || kblock >= kblocks) return (size_t)-1;
+  if (layout == MX_SCALES_LINEAR) return (size_t)(row * kblocks + kblock);
+  if (layout != MX_SCALES_SWIZZLED) return (size_t)-1;
+  const int64_t kchunks = (kblocks + 3) / 4;
+  return (size_t)(((row / 128) * kchunks + kblock / 4) * 512 + (row % 32) * 16 +
+                  ((row % 128) / 32) * 4 + kblock % 4);
+}
+
+const char* mx_strerror(int status) {
+  switch (status) {
+    case MX_OK: return "ok";
+    case MX_ERR_NULL: return "a required pointer is NULL";
+    case MX_ERR_SHAPE: return "bad shape, axis or extent";
+    case MX_ERR_FMT: return "enum value out of range";
+    case MX_ERR_ALIGN: return "pointer not aligned as required";
+    case MX_ERR_UNSUPPORTED: return "request not supported by this build";
+    case MX_ERR_CUDA: return "CUDA error (see mx_last_cuda_error)";
+    case MX_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+    case MX_ERR_WORKSPACE: return "workspace too small";
+    default: return "unknown status";
+  }
+}
+
+const char* mx_last_cuda_error(void) { return g_cuda_error; }
+
+int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int64_t* shape,
+                int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts) {
+  Opts o;
+  View v;
+  if (!shape) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || (rounding != MX_RNE && rounding != MX_RHAZ) || !read_opts(opts, &o))
+    return MX_ERR_FMT;
+  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (v.numel == 0) return MX_OK;
+  if (!in || !elems_out || !scales_out) return MX_ERR_NULL;
+  if ((uintptr_t)in % 16 || (uintptr_t)elems_out % 16 || (uintptr_t)scales_out % 16)
+    return MX_ERR_ALIGN;
+  if (v.numel / 8 >= (int64_t)1 << 31 || v.rows >= (int64_t)1 << 31 || v.inner >= (int64_t)1 << 31)
+    return MX_ERR_UNSUPPORTED;
+  cudaError_t e;
+  mx::QuantizeArgs a;
+  a.in = in; a.elems = (uint8_t*)elems_out; a.scales = scales_out;
+  a.outer = v.outer; a.L = v.L; a.inner = v.inner; a.numel = v.numel;
+  a.fmt = (int)fmt; a.rounding = (int)rounding; a.dtype = o.dtype; a.layout = o.layout;
+  a.stream = o.stream;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  // The swizzled tensor has padding when rows % 128 or kblocks % 4 is nonzero:
+  // zero the buffer first so that every byte is defined.
+  if (o.layout == MX_SCALES_SWIZZLED && (v.rows % 128 != 0 || v.kblocks % 4 != 0)) {
+    e = cudaMemsetAsync(scales_out, 0, scales_bytes(v.rows, v.kblocks, o.layout), o.stream);
+    if (e != cudaSuccess) return fail_cuda(e);
+  }
+  e = mx::launch_quantize(a);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+int mx_dequantize(const void* elems, const uint8_t* scales, void* out, const int64_t* shape,
+                  int ndim, int axis, mx_fmt_t fmt, const mx_opts_t* opts) {
+  Opts o;
+  View v;
+  if (!shape) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (axis != ndim - 1) return MX_ERR_UNSUPPORTED;
+  if (v.numel == 0) return MX_OK;
+  if (!elems || !scales || !out) return MX_ERR_NULL;
+  if ((uintptr_t)elems % 16 || (uintptr_t)scales % 16 || (uintptr_t)out % 16) return MX_ERR_ALIGN;
+  if (v.numel / 8 >= (int64_t)1 << 31) return MX_ERR_UNSUPPORTED;
+  cudaError_t e;
+  mx::DequantizeArgs a;
+  a.elems = (const uint8_t*)elems; a.scales = scales; a.out = out;
+  a.rows = v.rows; a.L = v.L; a.fmt = (int)fmt; a.dtype = o.dtype; a.layout = o.layout;
+  a.stream = o.stream;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = mx::launch_dequantize(a);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+// ---------------------------------------------------------------------------
+// Host-buffer variants: copy in, run the device entry point, copy out, sync.
+// ---------------------------------------------------------------------------
+
+size_t mx_quantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                                        const mx_opts_t* opts) {
+  Opts o;
+  View v;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o) || !make_view(shape, ndim, axis, &v)) return 0;
+  const size_t in_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
+  return align_up(in_b, 256) + align_up((size_t)v.numel / 8 * fmt_bits((int)fmt), 256) +
+         align_up(scales_bytes(v.rows, v.kblocks, o.layout), 256);
+}
+
+int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                     const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
+                     const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  Opts o;
+  View v;
+  if (!shape) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (v.numel == 0) return MX_OK;
+  if (!in_host || !elems_out_host || !scales_out_host || !workspace_dev) return MX_ERR_NULL;
+  if ((uintptr_t)workspace_dev % 256) return MX_ERR_ALIGN;
+  if (workspace_bytes < mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts))
+    return MX_ERR_WORKSPACE;
+  const size_t in_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
+  const size_t el_b = (size_t)v.numel / 8 * fmt_bits((int)fmt);
+  const size_t sc_b = scales_bytes(v.rows, v.kblocks, o.layout);
+  char* d_in = (char*)workspace_dev;
+  char* d_el = d_in + align_up(in_b, 256);
+  char* d_sc = d_el + align_up(el_b, 256);
+  cudaError_t e = cudaMemcpyAsync(d_in, in_host, in_b, cudaMemcpyHostToDevice, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  const int rc = mx_quantize(d_in, d_el, (uint8_t*)d_sc, shape, ndim, axis, fmt, rounding, opts);
+  if (rc != MX_OK) return rc;
+  e = cudaMemcpyAsync(elems_out_host, d_el, el_b, cudaMemcpyDeviceToHost, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = cudaMemcpyAsync(scales_out_host, d_sc, sc_b, cudaMemcpyDeviceToHost, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = cudaStreamSynchronize(o.stream);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                                          const mx_opts_t* opts) {
+  return mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts);
+}
+
+int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                       const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                       const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  Opts o;
+  View v;
+  if (!shape) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (axis != ndim - 1) return MX_ERR_UNSUPPORTED;
+  if (v.numel == 0) return MX_OK;
+  if (!elems_host || !scales_host || !out_host || !workspace_dev) return MX_ERR_NULL;
+  if ((uintptr_t)workspace_dev % 256) return MX_ERR_ALIGN;
+  if (workspace_bytes < mx_dequantize_host_workspace_bytes(shape, ndim, axis, fmt, opts))
+    return MX_ERR_WORKSPACE;
+  const size_t out_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
+  const size_t el_b = (size_t)v.numel / 8 * fmt_bits((int)fmt);
+  const size_t sc_b = scales_bytes(v.rows, v.kblocks, o.layout);
+  char* d_out = (char*)workspace_dev;
+  char* d_el = d_out + align_up(out_b, 256);
+  char* d_sc = d_el + align_up(el_b, 256);
+  cudaError_t e = cudaMemcpyAsync(d_el, elems_host, el_b, cudaMemcpyHostToDevice, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = cudaMemcpyAsync(d_sc, scales_host, sc_b, cudaMemcpyHostToDevice, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  const int rc = mx_dequantize(d_el, (const uint8_t*)d_sc, d_out, shape, ndim, axis, fmt, opts);
+  if (rc != MX_OK) return rc;
+  e = cudaMemcpyAsync(out_host, d_out, out_b, cudaMemcpyDeviceToHost, o.stream);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = cudaStreamSynchronize(o.stream);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+}  // extern "C"

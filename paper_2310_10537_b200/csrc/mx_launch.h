@@ -1,0 +1,49 @@
+// Internal interface between the C ABI (mx_api.cu) and the kernel files.
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include "mx.h"
+
+namespace mx {
+
+struct QuantizeArgs {
+  const void* in;
+  uint8_t* elems;
+  uint8_t* scales;
+  int64_t outer, L, inner;  // input viewed as [outer, L, inner], blocks along L
+  int64_t numel;
+  int fmt, rounding, dtype, layout;
+  int sm_count;
+  cudaStream_t stream;
+};
+cudaError_t launch_quantize(const QuantizeArgs& a);
+
+struct DequantizeArgs {
+  const uint8_t* elems;
+  const uint8_t* scales;
+  void* out;
+  int64_t rows, L;
+  int fmt, dtype, layout;
+  int sm_count;
+  cudaStream_t stream;
+};
+cudaError_t launch_dequantize(const DequantizeArgs& a);
+
+struct GemmArgs {
+  const void* A;
+  const uint8_t* sA;
+  const void* B;
+  const uint8_t* sB;
+  float* C;
+  int64_t M, N, K;
+  int fmtA, fmtB;
+  int sm_count;
+  uint32_t* status;  // device word: 0 = ok, else first bounded wait that gave up
+  cudaStream_t stream;
+};
+// Returns MX_OK or a negative mx_status_t; fills *cuda_err on MX_ERR_CUDA.
+int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err);
+
+}  // namespace mx

@@ -1,0 +1,78 @@
+"""CPU-only checks of the C ABI: the library loads, exports every symbol the
+public header declares, its size / index helpers agree with the oracle's own
+restatement of the layouts, and argument validation returns the documented
+status codes without touching a GPU."""
+import ctypes
+import os
+import re
+
+import numpy as np
+
+import oracle as O
+import paper_2310_10537_b200 as mx
+
+ROOT = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+
+
+def _declared_functions():
+    text = open(os.path.join(ROOT, "include", "mx.h")).read()
+    text = re.sub(r"/\*.*?\*/", "", text, flags=re.S)
+    return sorted(set(re.findall(r"\b(mx_[a-z0-9_]+)\s*\(", text)))
+
+
+def test_library_exports_every_declared_symbol():
+    names = _declared_functions()
+    assert "mx_quantize" in names and "mx_gemm" in names and len(names) >= 15
+    lib = ctypes.CDLL(mx.LIB_PATH)
+    for n in names:
+        assert hasattr(lib, n), n
+    assert sorted(mx.EXPORTS) == names
+
+
+def test_helpers_match_oracle_layouts():
+    for fmt in range(6):
+        assert mx.mx_fmt_bits(fmt) == O.fmt_bits(fmt)
+        assert mx.mx_elems_bytes([3, 64, 5], 1, fmt) == 3 * 64 * 5 * O.fmt_bits(fmt) // 8
+    assert mx.mx_fmt_bits(6) == 0
+    for rows, kb in ((1, 1), (128, 4), (200, 7), (257, 9)):
+        for layout in (0, 1):
+            assert mx.mx_scales_bytes([rows, kb * 32], 1, layout) == O.scales_bytes(rows, kb, layout)
+            for r in range(0, rows, 13):
+                for k in range(kb):
+                    assert mx.mx_scale_offset(r, k, rows, kb, layout) == O.scale_offset(r, k, rows, kb, layout)
+    assert mx.mx_scale_offset(5, 0, 5, 1, 1) == ctypes.c_size_t(-1).value
+    assert mx.mx_elems_bytes([4, 33], 1, 0) == 0
+    assert mx.mx_scales_bytes([4, 64], 2, 0) == 0
+
+
+def test_argument_validation_without_gpu():
+    lib = mx.lib()
+    shape = (ctypes.c_int64 * 2)(4, 64)
+    buf = np.zeros(4096, np.uint8)
+    p = buf.ctypes.data + (-buf.ctypes.data) % 64
+    o = mx.binding.mx_opts_t(mx.MX_F32, mx.MX_SCALES_LINEAR, None, 0)
+    q = lib.mx_quantize
+    assert q(None, p, p, shape, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_NULL
+    assert q(p, p, p, None, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_NULL
+    assert q(p, p, p, shape, 2, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
+    assert q(p, p, p, shape, 0, 0, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
+    assert q(p, p, p, shape, 2, 0, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE  # 4 % 32 != 0
+    assert q(p, p, p, shape, 2, 1, 6, 0, ctypes.byref(o)) == mx.MX_ERR_FMT
+    assert q(p, p, p, shape, 2, 1, 0, 2, ctypes.byref(o)) == mx.MX_ERR_FMT
+    assert q(p + 4, p, p, shape, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_ALIGN
+    bad = mx.binding.mx_opts_t(7, 0, None, 0)
+    assert q(p, p, p, shape, 2, 1, 0, 0, ctypes.byref(bad)) == mx.MX_ERR_FMT
+    empty = (ctypes.c_int64 * 2)(0, 64)
+    assert q(None, None, None, empty, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_OK
+    d = lib.mx_dequantize
+    assert d(p, p, p, shape, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
+    shape3 = (ctypes.c_int64 * 2)(64, 4)
+    assert d(p, p, p, shape3, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_UNSUPPORTED
+    assert d(p, None, p, shape, 2, 1, 0, ctypes.byref(o)) == mx.MX_ERR_NULL
+    g = lib.mx_gemm
+    assert g(p, p, p, p, p, 100, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert g(p, p, p, p, p, 128, 128, 64, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert g(p, p, p, p, p, 128, 128, 128, 5, 0, None) == mx.MX_ERR_UNSUPPORTED
+    assert g(p, p, p, p, p, 128, 128, 128, 0, 9, None) == mx.MX_ERR_FMT
+    assert g(None, p, p, p, p, 128, 128, 128, 0, 0, None) == mx.MX_ERR_NULL
+    assert lib.mx_strerror(mx.MX_ERR_ALIGN) and lib.mx_strerror(-99)

@@ -1,0 +1,231 @@
+"""GPU parity: mx_quantize / mx_dequantize through the C ABI against the CPU
+oracle, byte for byte, on the same seeded inputs."""
+import ctypes
+
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2310_10537_b200 as mx
+from paper_2310_10537_b200 import inputs
+from gpu_util import Guarded, to_oracle_input
+
+pytestmark = pytest.mark.gpu
+
+FMTS = list(range(6))
+DTYPES = [torch.float32, torch.bfloat16]
+
+
+def _quantize_guarded(x, axis, fmt, rounding, layout):
+    shape = list(x.shape)
+    ge = Guarded(mx.mx_elems_bytes(shape, axis, fmt))
+    gs = Guarded(mx.mx_scales_bytes(shape, axis, layout))
+    mx.mx_quantize(x, axis, fmt, rounding, layout, out=(ge.view, gs.view))
+    torch.cuda.synchronize()
+    ge.check()
+    gs.check()
+    return ge.view, gs.view
+
+
+def _assert_same_bytes(got: torch.Tensor, want: np.ndarray, what):
+    got = got.cpu().numpy()
+    assert got.shape == want.shape, what
+    if not (got == want).all():
+        bad = np.flatnonzero(got != want)
+        raise AssertionError(f"{what}: {bad.size} bytes differ, first at {bad[0]}: "
+                             f"got {got[bad[0]]:#x} want {want[bad[0]]:#x}")
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_last_axis_adversarial_bit_exact(fmt, dtype):
+    # 200 rows x 51 blocks: several CTA tiles, a ragged tail, padding in the swizzled scales
+    x = inputs.adversarial("cuda", rows=200, cols=1632, dtype=dtype, seed=11 + fmt)
+    xin = to_oracle_input(x)
+    for rounding in (mx.MX_RNE, mx.MX_RHAZ):
+        for layout in (mx.MX_SCALES_LINEAR, mx.MX_SCALES_SWIZZLED):
+            e, s = _quantize_guarded(x, 1, fmt, rounding, layout)
+            we, ws = O.quantize(xin, 1, fmt, rounding, layout)
+            _assert_same_bytes(e, we, ("elems", fmt, dtype, rounding, layout))
+            _assert_same_bytes(s, ws, ("scales", fmt, dtype, rounding, layout))
+            e2, s2 = _quantize_guarded(x, 1, fmt, rounding, layout)  # same bytes on a second run
+            assert torch.equal(e, e2) and torch.equal(s, s2)
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("inner", [1000, 1002, 999])
+def test_strided_axis_adversarial_bit_exact(fmt, dtype, inner):
+    # blocks along axis 0 of a [352 x inner] tensor (11 blocks deep); inner picks the
+    # 4-, 2- or 1-column variant of the kernel
+    x = inputs.adversarial("cuda", rows=inner, cols=352, dtype=dtype, seed=5 + fmt).t().contiguous()
+    assert list(x.shape) == [352, inner]
+    xin = to_oracle_input(x)
+    rounding = mx.MX_RHAZ if (fmt + inner) % 2 else mx.MX_RNE
+    for layout in (mx.MX_SCALES_LINEAR, mx.MX_SCALES_SWIZZLED):
+        e, s = _quantize_guarded(x, 0, fmt, rounding, layout)
+        we, ws = O.quantize(xin, 0, fmt, rounding, layout)
+        _assert_same_bytes(e, we, ("elems", fmt, dtype, inner, layout))
+        _assert_same_bytes(s, ws, ("scales", fmt, dtype, inner, layout))
+
+
+@pytest.mark.parametrize("fmt", [mx.MX_E4M3, mx.MX_E3M2, mx.MX_E2M1, mx.MX_INT8])
+def test_middle_axis_of_3d_tensor(fmt):
+    x = inputs.adversarial("cuda", rows=3 * 40, cols=64, dtype=torch.float32, seed=3)
+    x = x.view(3, 40, 64).transpose(1, 2).contiguous()  # [3, 64, 40], blocks along axis 1
+    xin = to_oracle_input(x)
+    e, s = _quantize_guarded(x, 1, fmt, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+    we, ws = O.quantize(xin, 1, fmt, mx.MX_RNE, O.SWIZZLED)
+    _assert_same_bytes(e, we, "elems")
+    _assert_same_bytes(s, ws, "scales")
+    # negative axis and a last-axis call on a 3-D tensor
+    y = x.transpose(1, 2).contiguous()
+    e, s = _quantize_guarded(y, -1, fmt, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
+    we, ws = O.quantize(to_oracle_input(y), 2, fmt, O.RHAZ, O.LINEAR)
+    _assert_same_bytes(e, we, "elems")
+    _assert_same_bytes(s, ws, "scales")
+
+
+def test_worked_blocks_on_device():
+    """The hand-worked W1 / W4 / W5 blocks straight through the kernel."""
+    v = torch.zeros(32, device="cuda")
+    v[:6] = torch.tensor([100, 1, -0.75, 0.3, 0.001, -1e-30])
+    e, s = mx.mx_quantize(v.view(1, 32), 1, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_LINEAR)
+    assert e[:6].tolist() == [0x7C, 0x48, 0xC4, 0x3A, 0x02, 0x80] and s.tolist() == [0x7D]
+    e, s = mx.mx_quantize(v.view(1, 32), 1, mx.MX_E4M3, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
+    assert e[0].item() == 0x7D
+    w4 = [6, 5, 4, 3.5, 3, 2.5, 2, 1.75, 1.5, 1.25, 1, 0.75, 0.5, 0.25, 0.2, 0, -0.25, -6, 7]
+    v = torch.zeros(32, device="cuda")
+    v[:len(w4)] = torch.tensor(w4)
+    e, s = mx.mx_quantize(v.view(1, 32), 1, mx.MX_E2M1, mx.MX_RNE, mx.MX_SCALES_LINEAR)
+    assert e[:10].tolist() == [0x67, 0x66, 0x45, 0x44, 0x23, 0x22, 0x01, 0x00, 0xF8, 0x07]
+    assert s.tolist() == [0x7F]
+    v = torch.zeros(32, device="cuda")
+    v[:7] = torch.tensor([1.5, -1.5, 1.9921875, 0.0078125, -0.0078125, 0.0234375, 1])
+    e, _ = mx.mx_quantize(v.view(1, 32), 1, mx.MX_INT8, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
+    assert e[:7].tolist() == [0x60, 0xA0, 0x7F, 0x01, 0xFF, 0x02, 0x40]
+    # FP6 bit order: codes 1..8 of E2M3 are the values 0.125 .. 1.0
+    v = torch.zeros(32, device="cuda")
+    v[:8] = torch.arange(1, 9, device="cuda") * 0.125
+    v[31] = 4.0  # pins the scale at 2^0
+    e, s = mx.mx_quantize(v.view(1, 32), 1, mx.MX_E2M3, mx.MX_RNE, mx.MX_SCALES_LINEAR)
+    assert s.tolist() == [0x7F] and e[:6].tolist() == [0x81, 0x30, 0x10, 0x85, 0x71, 0x20]
+
+
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_dequantize_every_code_and_scale(fmt, dtype):
+    rows, L = 130, 32 * 37
+    rng = np.random.default_rng(100 + fmt)
+    nbytes = rows * L * O.fmt_bits(fmt) // 8
+    elems = rng.integers(0, 256, nbytes, dtype=np.uint8)
+    out_dt = O.BF16 if dtype == torch.bfloat16 else O.F32
+    for layout in (O.LINEAR, O.SWIZZLED):
+        scales = rng.integers(0, 256, O.scales_bytes(rows, L // 32, layout), dtype=np.uint8)
+        scales[:64] = np.tile(np.array([0, 1, 254, 255, 127, 2, 253, 126], np.uint8), 8)
+        want = O.dequantize(elems, scales, rows, L, fmt, out_dt, layout)
+        g = Guarded(rows * L * (2 if dtype == torch.bfloat16 else 4))
+        out = g.view.view(dtype).view(rows, L)
+        mx.mx_dequantize(torch.from_numpy(elems).cuda(), torch.from_numpy(scales).cuda(),
+                         [rows, L], fmt, dtype, layout, out=out)
+        torch.cuda.synchronize()
+        g.check()
+        if dtype == torch.bfloat16:
+            got = out.view(torch.int16).cpu().numpy().view(np.uint16)
+        else:
+            got = out.view(torch.int32).cpu().numpy().view(np.uint32)
+            want = want.view(np.uint32)
+        assert (got == want).all(), (fmt, dtype, layout, int((got != want).sum()))
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_quantize_dequantize_round_trip_is_fixed_point(fmt):
+    x = inputs.adversarial("cuda", rows=64, cols=512, dtype=torch.float32, seed=77, nonfinite=False)
+    e, s = mx.mx_quantize(x, 1, fmt, layout=mx.MX_SCALES_LINEAR)
+    d = mx.mx_dequantize(e, s, [64, 512], fmt, torch.float32, mx.MX_SCALES_LINEAR)
+    e2, s2 = mx.mx_quantize(d, 1, fmt, layout=mx.MX_SCALES_LINEAR)
+    # Q(D(Q(V))) == Q(V) for every block whose elements all dequantize to normal FP32
+    # numbers (with a scale near 2^-127 they become FP32 subnormals, which Algorithm 1 flushes)
+    keep = s >= 32
+    assert int(keep.sum()) > 500
+    assert torch.equal(s[keep], s2[keep])
+    bpb = 32 * mx.mx_fmt_bits(fmt) // 8
+    assert torch.equal(e.view(-1, bpb)[keep], e2.view(-1, bpb)[keep])
+
+
+def test_empty_and_error_paths_on_device():
+    x = torch.empty((0, 64), device="cuda")
+    e, s = mx.mx_quantize(x, 1, mx.MX_E4M3)
+    assert e.numel() == 0 and s.numel() == 0
+    with pytest.raises(mx.MxError) as ei:
+        mx.mx_quantize(torch.zeros((4, 48), device="cuda"), 1, mx.MX_E4M3,
+                       out=(torch.zeros(256, dtype=torch.uint8, device="cuda"),
+                            torch.zeros(512, dtype=torch.uint8, device="cuda")))
+    assert ei.value.status == mx.MX_ERR_SHAPE
+    buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    shape = (ctypes.c_int64 * 2)(4, 64)
+    rc = mx.lib().mx_quantize(buf.data_ptr() + 4, buf.data_ptr() + 2048, buf.data_ptr() + 3072,
+                              shape, 2, 1, 0, 0, None)
+    assert rc == mx.MX_ERR_ALIGN
+
+
+def test_host_buffer_entry_points():
+    x = inputs.adversarial("cpu", rows=64, cols=256, dtype=torch.bfloat16, seed=2).pin_memory()
+    shape = [64, 256]
+    for fmt in (mx.MX_E4M3, mx.MX_E2M3, mx.MX_E2M1):
+        elems = torch.empty(mx.mx_elems_bytes(shape, 1, fmt), dtype=torch.uint8).pin_memory()
+        scales = torch.empty(mx.mx_scales_bytes(shape, 1), dtype=torch.uint8).pin_memory()
+        ws = torch.empty(mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, torch.bfloat16),
+                         dtype=torch.uint8, device="cuda")
+        mx.mx_quantize_host(x, elems, scales, 1, fmt, mx.MX_RNE, ws)
+        we, ws_ = O.quantize(to_oracle_input(x), 1, fmt, O.RNE, O.SWIZZLED)
+        assert (elems.numpy() == we).all() and (scales.numpy() == ws_).all()
+        out = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
+        ws2 = torch.empty(mx.mx_dequantize_host_workspace_bytes(shape, fmt, torch.bfloat16),
+                          dtype=torch.uint8, device="cuda")
+        mx.mx_dequantize_host(elems, scales, out, fmt, ws2)
+        want = O.dequantize(we, ws_, 64, 256, fmt, O.BF16, O.SWIZZLED)
+        assert (out.view(torch.int16).numpy().view(np.uint16) == want).all()
+        with pytest.raises(mx.MxError) as ei:
+            mx.mx_quantize_host(x, elems, scales, 1, fmt, mx.MX_RNE, ws[:256])
+        assert ei.value.status == mx.MX_ERR_WORKSPACE
+
+
+@pytest.mark.parametrize("fmt", FMTS)
+def test_config2_full_size_sweep(fmt):
+    """The 8192 x 8192 BF16 sweep tensor in the launch configuration the benchmark
+    times: quantize, then dequantize back to BF16.  E4M3 is compared on the whole
+    tensor, the other formats on 512 sampled rows (rows are independent)."""
+    T = inputs.config2("cuda")
+    rows, cols = T.shape
+    if fmt == mx.MX_E4M3:
+        sel = np.arange(rows)
+    else:
+        sel = np.sort(np.random.default_rng(fmt).choice(rows, 512, replace=False))
+    sel_t = torch.from_numpy(sel).cuda()
+    Tin = to_oracle_input(T[sel_t].contiguous())
+    w = O.fmt_bits(fmt)
+    for rounding in (mx.MX_RNE, mx.MX_RHAZ):
+        e, s = mx.mx_quantize(T, 1, fmt, rounding, mx.MX_SCALES_LINEAR)
+        d = mx.mx_dequantize(e, s, [rows, cols], fmt, torch.bfloat16, mx.MX_SCALES_LINEAR)
+        we, ws = O.quantize(Tin, 1, fmt, rounding, O.LINEAR)
+        ge = e.view(rows, cols * w // 8)[sel_t].cpu().numpy().reshape(-1)
+        gs = s.view(rows, cols // 32)[sel_t].cpu().numpy().reshape(-1)
+        assert (ge == we).all() and (gs == ws).all(), (fmt, rounding)
+        wd = O.dequantize(we, ws, sel.size, cols, fmt, O.BF16, O.LINEAR)
+        gd = d[sel_t].view(torch.int16).cpu().numpy().view(np.uint16)
+        assert (gd == wd).all(), (fmt, rounding)
+        if rounding == mx.MX_RNE:
+            # swizzled scales hold the same bytes in the other order
+            e2, s2 = mx.mx_quantize(T, 1, fmt, rounding, mx.MX_SCALES_SWIZZLED)
+            assert torch.equal(e, e2)
+            r = torch.arange(rows, device="cuda").view(-1, 1)
+            k = torch.arange(cols // 32, device="cuda").view(1, -1)
+            off = ((r // 128) * ((cols // 32 + 3) // 4) + k // 4) * 512 + (r % 32) * 16 + ((r % 128) // 32) * 4 + k % 4
+            assert torch.equal(s2[off.reshape(-1)], s)
+    # structure of the workload: the zero and tiny blocks are really there
+    if fmt == mx.MX_E4M3:
+        sb = s.cpu().numpy()
+        assert 0.0005 < (sb == 0).mean() < 0.002
+        assert 0.0005 < ((sb > 0) & (sb < 40)).mean() < 0.002
