@@ -24,7 +24,8 @@
  *   - Return value: MX_OK (0) or a negative mx_status_t.  Nothing throws,
  *     aborts or traps.  mx_strerror() gives a static description;
  *     mx_last_cuda_error() gives the text of the CUDA error behind the last
- *     MX_ERR_CUDA on the calling thread.
+ *     MX_ERR_CUDA (or which device-side wait expired, after MX_ERR_TIMEOUT) on
+ *     the calling thread.
  *   - If the CUDA driver or a GPU is missing every compute entry point returns
  *     MX_ERR_CUDA.  There is no CPU fallback.
  */
@@ -183,7 +184,7 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out,
  *       C[m,n] = sum over K-blocks b of X_A[m,b] * X_B[n,b] *
  *                sum_{i<32} P_A[m,32b+i] * P_B[n,32b+i]
  *     accumulated in FP32 on the tensor cores.
- * Requirements: M, N multiples of 128, K a multiple of 128; A, B 128-byte
+ * Requirements: M, N multiples of 128, K a nonzero multiple of 128; A, B 32-byte
  * aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
  * (the block-scaled tensor-core instruction has no integer element type).
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN,

@@ -46,7 +46,7 @@ class MxError(RuntimeError):
     def __init__(self, status: int, where: str):
         self.status = status
         msg = _lib.mx_strerror(status).decode()
-        if status == MX_ERR_CUDA:
+        if status in (MX_ERR_CUDA, MX_ERR_TIMEOUT):
             msg += ": " + _lib.mx_last_cuda_error().decode()
         super().__init__(f"{where}: {msg} ({status})")
 

@@ -268,4 +268,97 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 
+// ---------------------------------------------------------------------------
+// GEMM
+// ---------------------------------------------------------------------------
+
+static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
+                         const float* C, int64_t M, int64_t N, int64_t K, int fmtA, int fmtB) {
+  if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
+  if (!fmt_ok(fmtA) || !fmt_ok(fmtB)) return MX_ERR_FMT;
+  if (fmtA == MX_INT8 || fmtB == MX_INT8) return MX_ERR_UNSUPPORTED;
+  if (M < 0 || N < 0 || K < 128 || M % 128 || N % 128 || K % 128) return MX_ERR_SHAPE;
+  if (M >= ((int64_t)1 << 31) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return MX_ERR_SHAPE;
+  return MX_OK;
+}
+
+int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, float* C,
+            int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
+  Opts o;
+  int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB);
+  if (rc != MX_OK) return rc;
+  if (!read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.layout != MX_SCALES_SWIZZLED) return MX_ERR_UNSUPPORTED;
+  if ((uintptr_t)A % 32 || (uintptr_t)B % 32 || (uintptr_t)sA % 16 || (uintptr_t)sB % 16 ||
+      (uintptr_t)C % 16)
+    return MX_ERR_ALIGN;
+  if (M == 0 || N == 0) return MX_OK;
+  cudaError_t e;
+  mx::GemmArgs a;
+  a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C;
+  a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
+  a.stream = o.stream;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  rc = mx::launch_gemm(a, &e);
+  if (rc != MX_OK) return rc == MX_ERR_CUDA ? fail_cuda(e) : rc;
+  if (o.check) {
+    unsigned int st = 0;
+    rc = mx::gemm_status(o.stream, &st, &e);
+    if (rc != MX_OK) return fail_cuda(e);
+    if (st != 0) {
+      std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u gave up "
+                    "(1 producer/stage empty, 2 MMA/stage full, 3 MMA/accumulator free, "
+                    "4 epilogue/accumulator full)", st);
+      return MX_ERR_TIMEOUT;
+    }
+  }
+  return MX_OK;
+}
+
+size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {
+  if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || M < 0 || N < 0 || K < 0 || K % 32) return 0;
+  return align_up((size_t)(M * K / 8 * fmt_bits((int)fmtA)), 256) +
+         align_up(scales_bytes(M, K / 32, MX_SCALES_SWIZZLED), 256) +
+         align_up((size_t)(N * K / 8 * fmt_bits((int)fmtB)), 256) +
+         align_up(scales_bytes(N, K / 32, MX_SCALES_SWIZZLED), 256) +
+         align_up((size_t)(M * N) * 4, 256);
+}
+
+int mx_gemm_host(const void* A_host, const uint8_t* sA_host, const void* B_host,
+                 const uint8_t* sB_host, float* C_host, int64_t M, int64_t N, int64_t K,
+                 mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts, void* workspace_dev,
+                 size_t workspace_bytes) {
+  Opts o;
+  int rc = gemm_validate(A_host, sA_host, B_host, sB_host, C_host, M, N, K, (int)fmtA, (int)fmtB);
+  if (rc != MX_OK) return rc;
+  if (!read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!workspace_dev) return MX_ERR_NULL;
+  if ((uintptr_t)workspace_dev % 256) return MX_ERR_ALIGN;
+  if (workspace_bytes < mx_gemm_host_workspace_bytes(M, N, K, fmtA, fmtB)) return MX_ERR_WORKSPACE;
+  if (M == 0 || N == 0) return MX_OK;
+  const size_t a_b = (size_t)(M * K / 8 * fmt_bits((int)fmtA));
+  const size_t sa_b = scales_bytes(M, K / 32, MX_SCALES_SWIZZLED);
+  const size_t b_b = (size_t)(N * K / 8 * fmt_bits((int)fmtB));
+  const size_t sb_b = scales_bytes(N, K / 32, MX_SCALES_SWIZZLED);
+  const size_t c_b = (size_t)(M * N) * 4;
+  char* dA = (char*)workspace_dev;
+  char* dsA = dA + align_up(a_b, 256);
+  char* dB = dsA + align_up(sa_b, 256);
+  char* dsB = dB + align_up(b_b, 256);
+  char* dC = dsB + align_up(sb_b, 256);
+  cudaError_t e;
+  if ((e = cudaMemcpyAsync(dA, A_host, a_b, cudaMemcpyHostToDevice, o.stream)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dsA, sA_host, sa_b, cudaMemcpyHostToDevice, o.stream)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dB, B_host, b_b, cudaMemcpyHostToDevice, o.stream)) != cudaSuccess ||
+      (e = cudaMemcpyAsync(dsB, sB_host, sb_b, cudaMemcpyHostToDevice, o.stream)) != cudaSuccess)
+    return fail_cuda(e);
+  rc = mx_gemm(dA, (const uint8_t*)dsA, dB, (const uint8_t*)dsB, (float*)dC, M, N, K, fmtA, fmtB, opts);
+  if (rc != MX_OK) return rc;
+  if ((e = cudaMemcpyAsync(C_host, dC, c_b, cudaMemcpyDeviceToHost, o.stream)) != cudaSuccess)
+    return fail_cuda(e);
+  e = cudaStreamSynchronize(o.stream);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
 }  // extern "C"

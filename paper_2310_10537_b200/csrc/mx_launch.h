@@ -40,10 +40,12 @@ struct GemmArgs {
   int64_t M, N, K;
   int fmtA, fmtB;
   int sm_count;
-  uint32_t* status;  // device word: 0 = ok, else first bounded wait that gave up
   cudaStream_t stream;
 };
 // Returns MX_OK or a negative mx_status_t; fills *cuda_err on MX_ERR_CUDA.
 int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err);
+// Synchronises the stream, then reads and clears the per-device status word that a
+// bounded device-side wait sets when it gives up (0 = every wait completed).
+int gemm_status(cudaStream_t stream, unsigned int* status, cudaError_t* cuda_err);
 
 }  // namespace mx

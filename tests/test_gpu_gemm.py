@@ -1,0 +1,279 @@
+"""GPU parity: mx_gemm through the C ABI against the CPU oracle.
+
+Bound for every checked output (FP32 accumulation on the tensor cores against the
+FP64 dot product of the same dequantized values):
+    |C_gpu - C64| <= 1e-5 * sum_k |a_k| * |b_k|
+Exactly representable cases must match exactly."""
+import numpy as np
+import pytest
+import torch
+
+import oracle as O
+import paper_2310_10537_b200 as mx
+from paper_2310_10537_b200 import inputs
+from gpu_util import Guarded, to_oracle_input
+
+pytestmark = pytest.mark.gpu
+TOL = 1e-5
+FP = [mx.MX_E4M3, mx.MX_E5M2, mx.MX_E3M2, mx.MX_E2M3, mx.MX_E2M1]
+
+
+def _gemm_guarded(ea, sa, eb, sb, M, N, K, fa, fb):
+    g = Guarded(M * N * 4)
+    out = g.view.view(torch.float32).view(M, N)
+    mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=out, check_status=True)
+    torch.cuda.synchronize()
+    g.check()
+    return out
+
+
+def _check_bound(C, C64, S, what):
+    C = C.astype(np.float64)
+    err = np.abs(C - C64)
+    bound = TOL * S
+    ok = (err <= bound) | (np.isnan(C) & np.isnan(C64))
+    if not ok.all():
+        i = np.flatnonzero(~ok.reshape(-1))[0]
+        raise AssertionError(f"{what}: {int((~ok).sum())} of {ok.size} outputs beyond 1e-5*S; first "
+                             f"flat index {i}: got {C.reshape(-1)[i]!r} want {C64.reshape(-1)[i]!r} "
+                             f"S {S.reshape(-1)[i]!r}")
+    return float(np.nanmax(err / np.maximum(S, 1e-300)))
+
+
+def _packed_from_codes(codes: np.ndarray, fmt: int) -> torch.Tensor:
+    return torch.from_numpy(O.pack_codes(codes.reshape(-1), fmt)).cuda()
+
+
+def _swizzle_scales(sc: np.ndarray) -> np.ndarray:
+    rows, kb = sc.shape
+    out = np.zeros(O.scales_bytes(rows, kb, O.SWIZZLED), np.uint8)
+    for r in range(rows):
+        for k in range(kb):
+            out[O.scale_offset(r, k, rows, kb, O.SWIZZLED)] = sc[r, k]
+    return out
+
+
+ONE = {mx.MX_E4M3: 0x38, mx.MX_E5M2: 0x3C, mx.MX_E3M2: 0x0C, mx.MX_E2M3: 0x08, mx.MX_E2M1: 0x2}
+
+
+@pytest.mark.parametrize("fa,fb", [(0, 0), (1, 1), (2, 3), (3, 2), (4, 4), (0, 4), (4, 0), (2, 0)])
+@pytest.mark.parametrize("N", [256, 384])
+def test_scale_identification_exact(fa, fb, N):
+    """Every element is 1.0 and every (row, K-block) has its own power-of-two scale, so each
+    output is an exact sum that names the scale pairs the hardware applied: this pins the
+    operand tile layout, the swizzled scale layout and the per-MMA scale selection."""
+    M, K = 256, 1024
+    kb = K // 32
+    rng = np.random.default_rng(fa * 7 + fb + N)
+    for f in (fa, fb):
+        assert O.decode_element(ONE[f], f) == 1.0
+    a_codes = np.full((M, K), ONE[fa], np.uint8)
+    b_codes = np.full((N, K), ONE[fb], np.uint8)
+    # exponents within +-3: every partial sum fits FP32's 24 bits, so the result is exact
+    sa = (127 + rng.integers(-3, 4, (M, kb))).astype(np.uint8)
+    sb = (127 + rng.integers(-3, 4, (N, kb))).astype(np.uint8)
+    sa_sw, sb_sw = _swizzle_scales(sa), _swizzle_scales(sb)
+    ea, eb = O.pack_codes(a_codes.reshape(-1), fa), O.pack_codes(b_codes.reshape(-1), fb)
+    C = _gemm_guarded(torch.from_numpy(ea).cuda(), torch.from_numpy(sa_sw).cuda(),
+                      torch.from_numpy(eb).cuda(), torch.from_numpy(sb_sw).cuda(), M, N, K, fa, fb)
+    C64, _ = O.gemm(ea, sa_sw, eb, sb_sw, M, N, K, fa, fb)
+    want = 32.0 * (2.0 ** (sa.astype(np.float64) - 127)) @ (2.0 ** (sb.astype(np.float64) - 127)).T
+    assert (C64 == want).all()
+    assert (C.cpu().numpy().astype(np.float64) == C64).all()
+
+
+def test_element_position_probe_exact():
+    """One nonzero element per row of A at a row-dependent K position against a B whose entries
+    encode their K position: checks that element k of A meets element k of B for every k,
+    across swizzle atoms, MMA K-slices and pipeline stages."""
+    M = N = 128
+    K = 512
+    fa = fb = mx.MX_E4M3
+    a_codes = np.zeros((M, K), np.uint8)
+    for m in range(M):
+        a_codes[m, (37 * m + 11) % K] = 0x38  # 1.0
+    # B[n, k] = small integers that identify (n, k): value (k % 7 + 1) * sign(n)
+    vals = np.array([[(k % 7 + 1) * (1 if (n + k) % 3 else -1) for k in range(K)] for n in range(N)], np.float32)
+    b_codes = np.array([[O.encode_element(float(v), fb) for v in row] for row in vals], np.uint8)
+    sa = np.full((M, K // 32), 127, np.uint8)
+    sb = np.full((N, K // 32), 127, np.uint8)
+    ea, eb = O.pack_codes(a_codes.reshape(-1), fa), O.pack_codes(b_codes.reshape(-1), fb)
+    C = _gemm_guarded(torch.from_numpy(ea).cuda(), torch.from_numpy(_swizzle_scales(sa)).cuda(),
+                      torch.from_numpy(eb).cuda(), torch.from_numpy(_swizzle_scales(sb)).cuda(),
+                      M, N, K, fa, fb).cpu().numpy()
+    want = np.array([[vals[n, (37 * m + 11) % K] for n in range(N)] for m in range(M)], np.float32)
+    assert (C == want).all()
+
+
+def test_config1_full_matrix():
+    d = inputs.config1("cuda")
+    A, B = d["A"], d["B"]
+    M, K = A.shape
+    N = B.shape[1]
+    ea, sa = mx.mx_quantize(A, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(B, 0, mx.MX_E4M3)
+    # operands are bit-exact against the oracle, so both sides multiply the same values
+    wea, wsa = O.quantize(to_oracle_input(A), 1, O.E4M3)
+    web, wsb = O.quantize(to_oracle_input(B), 0, O.E4M3)
+    assert (ea.cpu().numpy() == wea).all() and (sa.cpu().numpy() == wsa).all()
+    assert (eb.cpu().numpy() == web).all() and (sb.cpu().numpy() == wsb).all()
+    C = _gemm_guarded(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3)
+    C64, S = O.gemm(wea, wsa, web, wsb, M, N, K, O.E4M3, O.E4M3)
+    worst = _check_bound(C.cpu().numpy(), C64, S, "config 1")
+    assert worst <= TOL
+    # second launch gives the same bits (no order-dependent accumulation between launches)
+    C2 = _gemm_guarded(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3)
+    assert torch.equal(C, C2)
+
+
+@pytest.mark.parametrize("fa,fb", [(0, 0), (1, 0), (2, 3), (3, 3), (4, 4), (0, 4), (4, 1), (2, 2)])
+@pytest.mark.parametrize("shape", [(128, 128, 128), (256, 384, 640), (384, 512, 1024)])
+def test_all_format_pairs_small(fa, fb, shape):
+    M, N, K = shape
+    g = torch.Generator(device="cuda").manual_seed(M + N + K + fa * 11 + fb)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.05
+    A.view(M, K // 32, 32)[::5, 1] = 0.0  # zero blocks contribute exactly nothing
+    ea, sa = mx.mx_quantize(A, 1, fa, mx.MX_RHAZ)
+    eb, sb = mx.mx_quantize(B, 1, fb, mx.MX_RNE)
+    C = _gemm_guarded(ea, sa, eb, sb, M, N, K, fa, fb).cpu().numpy()
+    C64, S = O.gemm(ea.cpu().numpy(), sa.cpu().numpy(), eb.cpu().numpy(), sb.cpu().numpy(), M, N, K, fa, fb)
+    _check_bound(C, C64, S, (fa, fb, shape))
+
+
+def test_long_k_accumulation_and_extreme_scales():
+    M = N = 256
+    K = 8192
+    g = torch.Generator(device="cuda").manual_seed(99)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    # rows with very large and very small magnitudes: scale bytes far from 127
+    A[:8] *= 2.0 ** 60
+    A[8:16] *= 2.0 ** -60
+    B[:8] *= 2.0 ** 40
+    B[8:16] *= 2.0 ** -50
+    for fa, fb in ((mx.MX_E4M3, mx.MX_E4M3), (mx.MX_E4M3, mx.MX_E2M1)):
+        ea, sa = mx.mx_quantize(A, 1, fa)
+        eb, sb = mx.mx_quantize(B, 1, fb)
+        C = _gemm_guarded(ea, sa, eb, sb, M, N, K, fa, fb).cpu().numpy()
+        C64, S = O.gemm(ea.cpu().numpy(), sa.cpu().numpy(), eb.cpu().numpy(), sb.cpu().numpy(), M, N, K, fa, fb)
+        worst = _check_bound(C, C64, S, ("long K", fa, fb))
+        print("long-K worst |err|/S:", worst)
+
+
+def test_nan_scale_poisons_row_and_gemm_errors():
+    M = N = 128
+    K = 256
+    g = torch.Generator(device="cuda").manual_seed(5)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    A[3, 40] = float("inf")   # block (3, 1) gets scale 0xFF
+    B[7, 200] = float("nan")  # block (7, 6) gets scale 0xFF
+    ea, sa = mx.mx_quantize(A, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(B, 1, mx.MX_E4M3)
+    C = _gemm_guarded(ea, sa, eb, sb, M, N, K, 0, 0).cpu().numpy()
+    C64, S = O.gemm(ea.cpu().numpy(), sa.cpu().numpy(), eb.cpu().numpy(), sb.cpu().numpy(), M, N, K, 0, 0)
+    assert np.isnan(C64[3]).all() and np.isnan(C64[:, 7]).all()
+    assert np.isnan(C[3]).all() and np.isnan(C[:, 7]).all()
+    fin = ~np.isnan(C64)
+    assert not np.isnan(C[fin]).any()
+    _check_bound(np.where(fin, C, 0), np.where(fin, C64, 0), np.where(fin, S, 0), "finite part")
+    with pytest.raises(mx.MxError) as ei:
+        mx.mx_gemm(ea, sa, eb, sb, 100, N, K, 0, 0)
+    assert ei.value.status == mx.MX_ERR_SHAPE
+    with pytest.raises(mx.MxError) as ei:
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_INT8, 0)
+    assert ei.value.status == mx.MX_ERR_UNSUPPORTED
+
+
+def _sample_positions(M, N, rng, full_rows=2, full_cols=2, tile=128):
+    ms, ns = [], []
+    for r in rng.choice(M, full_rows, replace=False):
+        ms += [r] * N
+        ns += list(range(N))
+    for c in rng.choice(N, full_cols, replace=False):
+        ms += list(range(M))
+        ns += [c] * M
+    tm, tn = M // tile, N // tile
+    gm, gn = np.meshgrid(np.arange(tm), np.arange(tn), indexing="ij")
+    ms += list((gm * tile + rng.integers(0, tile, gm.shape)).reshape(-1))
+    ns += list((gn * tile + rng.integers(0, tile, gn.shape)).reshape(-1))
+    ms += [0, 0, M - 1, M - 1]
+    ns += [0, N - 1, 0, N - 1]
+    return np.array(ms, np.int64), np.array(ns, np.int64)
+
+
+def _full_size_check(name, ea, sa, eb, sb, M, N, K, fa, fb, seed):
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    rng = np.random.default_rng(seed)
+    ms, ns = _sample_positions(M, N, rng)
+    hea, hsa, heb, hsb = (t.cpu().numpy() for t in (ea, sa, eb, sb))
+    c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].cpu().numpy()
+    worst = _check_bound(got, c64, s, name + " sampled")
+    # whole matrix against an FP64 library product of the oracle-dequantized operands
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    rows_per = max(128, (1 << 27) // N // 128 * 128)
+    bad = 0
+    for r0 in range(0, M, rows_per):
+        r1 = min(M, r0 + rows_per)
+        c64f = da[r0:r1] @ db.T
+        sf = da[r0:r1].abs() @ db.abs().T
+        bad += int(((C[r0:r1].double() - c64f).abs() > TOL * sf).sum())
+    assert bad == 0, f"{name}: {bad} outputs of the full matrix beyond the bound"
+    print(name, "worst sampled |err|/S:", worst)
+
+
+def test_config3_full_size():
+    d = inputs.config3("cuda")
+    X, W = d["X"], d["W"]
+    M, K = X.shape
+    N = W.shape[1]
+    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(W, 0, mx.MX_E4M3)
+    _full_size_check("config 3", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, 3)
+
+
+def test_config4_training_step():
+    d = inputs.config4("cuda")
+    X, W, dY = d["X"], d["W"], d["dY"]
+    n = X.shape[0]
+    act, wt, rnd = mx.MX_E3M2, mx.MX_E2M3, mx.MX_RHAZ
+    # forward Y = X W: A = Q(X, axis 1), B = Q(W, axis 0) -> [N x K]
+    _full_size_check("config 4 fwd", *mx.mx_quantize(X, 1, act, rnd), *mx.mx_quantize(W, 0, wt, rnd),
+                     n, n, n, act, wt, 41)
+    # dgrad dX = dY W^T: A = Q(dY, axis 1), B = Q(W, axis 1)
+    _full_size_check("config 4 dgrad", *mx.mx_quantize(dY, 1, act, rnd), *mx.mx_quantize(W, 1, wt, rnd),
+                     n, n, n, act, wt, 42)
+    # wgrad dW = X^T dY: A = Q(X, axis 0), B = Q(dY, axis 0)
+    _full_size_check("config 4 wgrad", *mx.mx_quantize(X, 0, act, rnd), *mx.mx_quantize(dY, 0, act, rnd),
+                     n, n, n, act, act, 43)
+
+
+def test_config5_full_size():
+    d = inputs.config5("cuda")
+    W, X = d["W"], d["X"]
+    M, K = X.shape
+    N = W.shape[1]
+    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(W, 0, mx.MX_E2M1)
+    del d, W, X
+    _full_size_check("config 5", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, 5)
+
+
+def test_host_buffer_gemm():
+    M, N, K = 128, 256, 256
+    g = torch.Generator(device="cuda").manual_seed(8)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    ea, sa = mx.mx_quantize(A, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(B, 1, mx.MX_E2M1)
+    ref = mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1)
+    hC = torch.empty((M, N), dtype=torch.float32).pin_memory()
+    ws = torch.empty(mx.mx_gemm_host_workspace_bytes(M, N, K, mx.MX_E4M3, mx.MX_E2M1),
+                     dtype=torch.uint8, device="cuda")
+    mx.mx_gemm_host(ea.cpu().pin_memory(), sa.cpu().pin_memory(), eb.cpu().pin_memory(),
+                    sb.cpu().pin_memory(), hC, M, N, K, mx.MX_E4M3, mx.MX_E2M1, ws)
+    assert torch.equal(hC, ref.cpu())

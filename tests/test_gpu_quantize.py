@@ -19,6 +19,7 @@ DTYPES = [torch.float32, torch.bfloat16]
 
 def _quantize_guarded(x, axis, fmt, rounding, layout):
     shape = list(x.shape)
+    axis %= len(shape)
     ge = Guarded(mx.mx_elems_bytes(shape, axis, fmt))
     gs = Guarded(mx.mx_scales_bytes(shape, axis, layout))
     mx.mx_quantize(x, axis, fmt, rounding, layout, out=(ge.view, gs.view))
