@@ -1,0 +1,441 @@
+#!/usr/bin/env python
+"""Benchmark of the MX hot path on B200: quantize / dequantize GB/s and block-scaled
+GEMM TFLOP/s on seeded synthetic tensors shaped like the paper's transformer
+workloads (arXiv 2310.10537).
+
+One step = one pass of the whole hot path:
+  sweep   the 8192 x 8192 BF16 tensor of the quantize/dequantize sweep, cast to each of
+          the six MX formats (blocks along the last axis, scales in the layout the
+          GEMM reads) and dequantized back to BF16                      [12 launches]
+  ffn     the FFN up-projection: quantize X[8192 x 4096] along its contiguous axis,
+          W[4096 x 16384] along its strided axis (transposing requantize), then the
+          MXFP8 block-scaled GEMM 8192 x 16384 x 4096 with FP32 output  [3 launches]
+`value` is the algorithmic GB/s of the sweep (the configuration the quantize metric is
+quoted on); the GEMM and the other phases are reported beside it in the same line.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+Under torchrun every rank runs the same step on its own GPU (weak scaling, no
+exchange: MX blocks are independent) and rank 0 prints one JSON line.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+FMT_NAMES = ["e4m3", "e5m2", "e3m2", "e2m3", "e2m1", "int8"]
+FMT_BITS = [8, 8, 6, 6, 4, 8]
+SWEEP_ROWS, SWEEP_COLS = 8192, 8192
+FFN_TOKENS, FFN_IN, FFN_OUT = 8192, 4096, 16384
+
+
+def algorithmic_bytes(numel: int, in_bytes: int, bits: int) -> float:
+    """Bytes a quantize (or dequantize) pass must move: float tensor + codes + one scale per 32."""
+    return numel * (in_bytes + bits / 8.0 + 1.0 / 32.0)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
+                 "--format=csv,noheader,nounits", "-lms", "20"],
+                stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        time.sleep(0.25)
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx_, power, reasons = [], [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for line in out.strip().splitlines():
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) < 7:
+                continue
+            try:
+                sm.append(float(parts[0]))
+                mx_.append(float(parts[1]))
+                power.append(float(parts[2]))
+            except ValueError:
+                continue
+            for n, v in zip(names, parts[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(n)
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
+        busy = [s for s, p in zip(sm, power) if p > 0.5 * max(power)] or sm
+        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx_), "samples": len(sm),
+                "power_w_max": max(power), "reasons": sorted(reasons)}
+
+
+# --------------------------------------------------------------------------------------
+# our arm: the CUDA library through its Python binding
+# --------------------------------------------------------------------------------------
+
+class Workload:
+    def __init__(self, torch, mx, inputs, device, seed_offset: int):
+        self.torch, self.mx = torch, mx
+        T = inputs.config2(device, SWEEP_ROWS, SWEEP_COLS, seed=2002 + seed_offset)
+        self.T = [T, T.clone()]  # two copies, read alternately: no launch re-reads what L2 still holds
+        shape = [SWEEP_ROWS, SWEEP_COLS]
+        u8 = dict(dtype=torch.uint8, device=device)
+        self.sweep = []
+        for fmt in range(6):
+            e = torch.empty(mx.mx_elems_bytes(shape, 1, fmt), **u8)
+            s = torch.empty(mx.mx_scales_bytes(shape, 1), **u8)
+            d = torch.empty(shape, dtype=torch.bfloat16, device=device)
+            self.sweep.append((e, s, d))
+        f = inputs.config3(device, FFN_TOKENS, FFN_IN, FFN_OUT, seed=3003 + seed_offset)
+        self.X, self.W = f["X"], f["W"]
+        self.ea = torch.empty(mx.mx_elems_bytes([FFN_TOKENS, FFN_IN], 1, mx.MX_E4M3), **u8)
+        self.sa = torch.empty(mx.mx_scales_bytes([FFN_TOKENS, FFN_IN], 1), **u8)
+        self.eb = torch.empty(mx.mx_elems_bytes([FFN_IN, FFN_OUT], 0, mx.MX_E4M3), **u8)
+        self.sb = torch.empty(mx.mx_scales_bytes([FFN_IN, FFN_OUT], 0), **u8)
+        self.C = torch.empty((FFN_TOKENS, FFN_OUT), dtype=torch.float32, device=device)
+        self.flush_buf = torch.empty(256 << 20, **u8)  # > L2 (126 MB)
+        n = SWEEP_ROWS * SWEEP_COLS
+        self.bytes_q = [algorithmic_bytes(n, 2, b) for b in FMT_BITS]
+        self.bytes_sweep = 2.0 * sum(self.bytes_q)
+        self.bytes_qx = algorithmic_bytes(FFN_TOKENS * FFN_IN, 2, 8)
+        self.bytes_qw = algorithmic_bytes(FFN_IN * FFN_OUT, 2, 8)
+        self.flops = 2.0 * FFN_TOKENS * FFN_OUT * FFN_IN
+        self.launches_per_step = 15
+
+    def flush_l2(self):
+        self.flush_buf.zero_()
+
+    def step(self, ev=None):
+        """One pass of the hot path.  ev: list of 8 CUDA events bracketing the phases."""
+        torch, mx = self.torch, self.mx
+        rec = (lambda i: ev[i].record()) if ev is not None else (lambda i: None)
+        rec(0)
+        for fmt in range(6):                                   # a1-a4: float -> MX, last axis
+            e, s, _ = self.sweep[fmt]
+            mx.mx_quantize(self.T[fmt & 1], 1, fmt, mx.MX_RNE, mx.MX_SCALES_SWIZZLED, out=(e, s))
+        rec(1)
+        for fmt in range(6):                                   # a6: MX -> BF16
+            e, s, d = self.sweep[fmt]
+            mx.mx_dequantize(e, s, [SWEEP_ROWS, SWEEP_COLS], fmt, torch.bfloat16,
+                             mx.MX_SCALES_SWIZZLED, out=d)
+        rec(2)
+        self.flush_l2()
+        rec(3)
+        mx.mx_quantize(self.X, 1, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_SWIZZLED, out=(self.ea, self.sa))
+        rec(4)
+        mx.mx_quantize(self.W, 0, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_SWIZZLED, out=(self.eb, self.sb))  # a5
+        rec(5)
+        self.flush_l2()
+        rec(6)
+        mx.mx_gemm(self.ea, self.sa, self.eb, self.sb, FFN_TOKENS, FFN_OUT, FFN_IN,       # a7-a9
+                   mx.MX_E4M3, mx.MX_E4M3, out=self.C)
+        rec(7)
+
+
+def run_e2e(torch, mx, inputs, steps: int, warmup: int):
+    """The sweep through the host-buffer entry points: pinned host tensors in, pinned host
+    results out, every copy inside the timed region."""
+    T = inputs.config2("cpu", 2048, SWEEP_COLS, seed=2002).pin_memory()  # a quarter of the sweep tensor
+    rows, cols = T.shape
+    shape = [rows, cols]
+    n = rows * cols
+    bufs = []
+    ws_bytes = 0
+    for fmt in range(6):
+        e = torch.empty(mx.mx_elems_bytes(shape, 1, fmt), dtype=torch.uint8).pin_memory()
+        s = torch.empty(mx.mx_scales_bytes(shape, 1), dtype=torch.uint8).pin_memory()
+        bufs.append((e, s))
+        ws_bytes = max(ws_bytes, mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, torch.bfloat16))
+    out = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
+    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+    h2d = d2h = 0
+
+    def one():
+        nonlocal h2d, d2h
+        h2d = d2h = 0
+        for fmt in range(6):
+            e, s = bufs[fmt]
+            mx.mx_quantize_host(T, e, s, 1, fmt, mx.MX_RNE, ws)
+            h2d += T.numel() * 2
+            d2h += e.numel() + s.numel()
+            mx.mx_dequantize_host(e, s, out, fmt, ws)
+            h2d += e.numel() + s.numel()
+            d2h += out.numel() * 2
+
+    for _ in range(max(1, warmup)):
+        one()
+    torch.cuda.synchronize()
+    t0 = time.perf_counter()
+    for _ in range(steps):
+        one()
+    torch.cuda.synchronize()
+    dt = (time.perf_counter() - t0) / steps
+    total_bytes = 2.0 * sum(algorithmic_bytes(n, 2, b) for b in FMT_BITS)
+    return {"value": total_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
+            "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3,
+            "workload": f"sweep on a {rows}x{cols} BF16 slice via mx_quantize_host / mx_dequantize_host "
+                        "(pinned host buffers, copies timed)"}
+
+
+def run_cpu_baseline(rows: int = 2048, seconds_target: float = 15.0):
+    """The oracle, as it stands, on the host cores: the same sweep on `rows` rows of the tensor."""
+    import numpy as np
+    import torch
+
+    import oracle as O
+    from paper_2310_10537_b200 import inputs
+    T = inputs.config2("cpu", rows, SWEEP_COLS, seed=2002)
+    x = T.view(torch.int16).numpy().view(np.uint16)
+    n = rows * SWEEP_COLS
+    t0 = time.perf_counter()
+    total = 0.0
+    for fmt in range(6):
+        e, s = O.quantize(x, 1, fmt, O.RNE, O.SWIZZLED)
+        O.dequantize(e, s, rows, SWEEP_COLS, fmt, O.BF16, O.SWIZZLED)
+        total += 2 * algorithmic_bytes(n, 2, FMT_BITS[fmt])
+        if time.perf_counter() - t0 > 4 * seconds_target:
+            break
+    dt = time.perf_counter() - t0
+    return {"value": total / dt / 1e9, "unit": "GB/s", "cores": O.threads(), "kind": "oracle",
+            "sample": f"quantize+dequantize sweep, 6 formats, {rows}x{SWEEP_COLS} BF16 slice of the "
+                      f"sweep tensor, {dt:.1f} s"}, dt
+
+
+def main_ours(args, rank, world, local_rank):
+    import torch
+
+    import paper_2310_10537_b200 as mx
+    from paper_2310_10537_b200 import inputs
+
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        import torch.distributed as dist
+        dist.init_process_group("nccl", device_id=dev)
+    peaks = measured_peaks()
+    w = Workload(torch, mx, inputs, dev, seed_offset=rank)
+
+    def barrier():
+        if world > 1:
+            import torch.distributed as dist
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        w.step()
+    barrier()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(args.steps)]
+    t_begin = torch.cuda.Event(enable_timing=True)
+    t_end = torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_begin.record()
+    for i in range(args.steps):
+        w.step(evs[i])
+    t_end.record()
+    barrier()
+    clocks = sampler.stop() if sampler else None
+
+    def phase(a, b):
+        return sum(e[a].elapsed_time(e[b]) for e in evs) / args.steps  # ms per step
+
+    ms = {"quantize_sweep": phase(0, 1), "dequantize_sweep": phase(1, 2), "quantize_x": phase(3, 4),
+          "quantize_w_strided": phase(4, 5), "gemm": phase(6, 7)}
+    ms_step = t_begin.elapsed_time(t_end) / args.steps
+    t = torch.tensor([ms_step, ms["quantize_sweep"] + ms["dequantize_sweep"], ms["gemm"],
+                      ms["quantize_sweep"]], dtype=torch.float64, device=dev)
+    if world > 1:
+        import torch.distributed as dist
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_step_max, ms_sweep_max, ms_gemm_max, ms_q_max = t.tolist()
+    if rank != 0:
+        return
+
+    value = world * w.bytes_sweep / (ms_sweep_max * 1e-3) / 1e9
+    gemm_tflops = world * w.flops / (ms_gemm_max * 1e-3) / 1e12
+    q_gbs = sum(w.bytes_q) / (ms["quantize_sweep"] * 1e-3) / 1e9
+    fp8_peak = 2.0 * peaks["bf16_tflops"]
+    line = {
+        "metric": "mx_quantize_dequantize_GBps",
+        "value": value,
+        "unit": "GB/s",
+        "n_gpus": world,
+        "steps": args.steps,
+        "warmup": max(args.warmup, 3),
+        "ms_per_step": ms_step_max,
+        "higher_is_better": True,
+        "scaling": "weak",
+        "vs_baseline": None,
+        "dtype": "bf16->mx (fp8/fp6/fp4/int8 codes, e8m0 scales); gemm mxfp8 x mxfp8 -> f32",
+        "data": "synthetic",
+        "config": {
+            "workload": "configs[1] quantize/dequantize sweep, BF16 8192x8192 Student-t(3)x4 with zero and "
+                        "1e-30 blocks, six formats, k=32 along the last axis; plus configs[2] FFN "
+                        "up-projection (quantize X, transposing quantize W, MXFP8 GEMM 8192x16384x4096)",
+            "l2": "inputs larger than L2 and read from alternating copies; 256 MB L2 flush before the FFN "
+                  "quantizes and before the GEMM (outside the phase timers)",
+            "rounding": "nearest-even", "scale_layout": "swizzled",
+        },
+        "phases_ms": ms,
+        "gemm": {"metric": "mx_gemm_TFLOPs", "value": gemm_tflops, "unit": "TFLOP/s",
+                 "workload": "configs[2] MXFP8 E4M3 8192x16384x4096, FP32 out",
+                 "ms": ms_gemm_max},
+        "quantize_x_GBps": w.bytes_qx / (ms["quantize_x"] * 1e-3) / 1e9,
+        "quantize_w_strided_GBps": w.bytes_qw / (ms["quantize_w_strided"] * 1e-3) / 1e9,
+        "dequantize_sweep_GBps": sum(w.bytes_q) / (ms["dequantize_sweep"] * 1e-3) / 1e9,
+        "roofline": {
+            "kernel": "quantize_lastaxis_kernel (six format instances, BF16 in, swizzled scales)",
+            "bound": "hbm", "achieved": q_gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+            "frac": q_gbs / peaks["hbm_gbs"], "peak_source": peaks["source"],
+            "traffic": NCU_TRAFFIC.get("quantize"),
+        },
+        "roofline_gemm": {
+            "kernel": "mx_gemm_kernel<256>", "bound": "tensor", "achieved": gemm_tflops / world,
+            "peak": fp8_peak, "unit": "TFLOP/s", "frac": gemm_tflops / world / fp8_peak,
+            "peak_source": f"2 x {peaks['source']} BF16 burst (nominal FP8:BF16 ratio)",
+            "frac_of_sustained": gemm_tflops / world / (2.0 * peaks["bf16_tflops_sustained"]),
+            "traffic": NCU_TRAFFIC.get("gemm"),
+        },
+        "gpu_launches": w.launches_per_step * args.steps,
+        "clocks": clocks,
+    }
+    if world == 1:
+        line["e2e"] = run_e2e(torch, mx, inputs, max(2, min(args.steps, 5)), 1)
+        cpu, _ = run_cpu_baseline(rows=SWEEP_ROWS)
+        line["cpu_baseline"] = cpu
+    else:
+        line["e2e"] = None
+    print(json.dumps(line))
+
+
+# DRAM bytes per launch from the committed ncu captures (profiles/), filled in when a
+# capture exists; None = not captured.
+NCU_TRAFFIC = {"quantize": None, "gemm": None}
+
+
+def main_reference(args, rank, world):
+    """The reference arm: the CPU oracle on the same metric, on a bounded sample per step."""
+    if rank != 0:
+        return
+    times, total = [], None
+    for i in range(max(args.warmup, 1) + args.steps):
+        res, dt = run_cpu_baseline(rows=2048)
+        if i >= max(args.warmup, 1):
+            times.append(dt)
+            total = res
+    ms = 1e3 * sum(times) / len(times)
+    # value over the timed steps
+    rows = 2048
+    nbytes = 2.0 * sum(algorithmic_bytes(rows * SWEEP_COLS, 2, b) for b in FMT_BITS)
+    value = nbytes / (ms * 1e-3) / 1e9
+    line = {
+        "impl": "reference", "metric": "mx_quantize_dequantize_GBps", "value": value, "unit": "GB/s",
+        "n_gpus": world, "steps": args.steps, "warmup": max(args.warmup, 1), "ms_per_step": ms,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64/int (CPU oracle)",
+        "data": "synthetic",
+        "config": {"workload": "configs[1] quantize/dequantize sweep; each step a 2048x8192 BF16 slice, "
+                               "six formats, on the host cores"},
+        "cpu_baseline": {"value": value, "unit": "GB/s", "cores": total["cores"], "kind": "oracle",
+                         "sample": total["sample"]},
+        "e2e": {"value": value, "unit": "GB/s", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main_case(args):
+    """A few launches of one kernel on a small case, for profiler captures (prints no bench line)."""
+    import torch
+
+    import paper_2310_10537_b200 as mx
+    from paper_2310_10537_b200 import inputs
+    torch.cuda.set_device(0)
+    reps = 3
+    if args.case in ("quantize", "dequantize"):
+        T = inputs.config2("cuda", SWEEP_ROWS, SWEEP_COLS)
+        fmt = mx.FORMATS[args.fmt]
+        e, s = mx.mx_quantize(T, 1, fmt)
+        d = torch.empty_like(T)
+        for _ in range(reps):
+            if args.case == "quantize":
+                mx.mx_quantize(T, 1, fmt, out=(e, s))
+            else:
+                mx.mx_dequantize(e, s, list(T.shape), fmt, torch.bfloat16, out=d)
+    elif args.case == "quantize_strided":
+        W = inputs.config3("cuda")["W"]
+        fmt = mx.FORMATS[args.fmt]
+        for _ in range(reps):
+            mx.mx_quantize(W, 0, fmt)
+    elif args.case == "gemm":
+        n = 4096
+        d = inputs.config4("cuda", n)
+        fmt = mx.FORMATS[args.fmt]
+        ea, sa = mx.mx_quantize(d["X"], 1, fmt)
+        eb, sb = mx.mx_quantize(d["W"], 0, fmt)
+        C = torch.empty((n, n), dtype=torch.float32, device="cuda")
+        for _ in range(reps):
+            mx.mx_gemm(ea, sa, eb, sb, n, n, n, fmt, fmt, out=C, check_status=True)
+    torch.cuda.synchronize()
+    print(json.dumps({"case": args.case, "fmt": args.fmt, "launches": reps}))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm"],
+                    default="step", help="'step' = the benchmark; the others run three launches of one "
+                                         "kernel on a small case for a profiler capture")
+    ap.add_argument("--fmt", choices=FMT_NAMES, default="e4m3")
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=100)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    args = ap.parse_args()
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.case != "step":
+        main_case(args)
+    elif args.impl == "reference":
+        main_reference(args, rank, world)
+    else:
+        main_ours(args, rank, world, local_rank)
+
+
+if __name__ == "__main__":
+    main()
