@@ -2,7 +2,7 @@
 // every element of a block is NaN when the scale X is NaN.
 //
 // A pure stream bound by HBM bandwidth: bits/8 + 1/32 bytes read and 2 or 4
-// bytes written per element.  8 elements per thread, 4 lanes per MX block.
+// bytes written per element.
 #include <cuda_fp16.h>
 
 #include "mx_device.cuh"
@@ -11,6 +11,9 @@
 namespace mx {
 
 constexpr int kDqThreads = 256;
+#ifndef MX_DQ_CAP
+#define MX_DQ_CAP 0  // CTAs per SM the grid is capped at (0 = one CTA per 256 units, no loop)
+#endif
 
 // Two codes -> two FP32 values (exact: every element value fits FP16).
 // pair = code0 | code1 << 8  (FP4: code0 | code1 << 4 in the low byte).
@@ -36,32 +39,49 @@ __device__ __forceinline__ void decode_pair(uint32_t pair, float& a, float& b) {
   b = f.y;
 }
 
+// A thread produces 64 bytes of output: a whole block as BF16 (32 elements) or half
+// a block as FP32 (16 elements), written with two 256-bit stores.
 template <int FMT, int DTYPE, int LAYOUT, bool ALIGNED32>
 __global__ void __launch_bounds__(kDqThreads)
 dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__ scales,
-                  void* __restrict__ out, uint32_t n_chunks, uint32_t kblocks, FastDiv kb_div) {
+                  void* __restrict__ out, uint32_t n_units, uint32_t kblocks, FastDiv kb_div) {
   constexpr int bits = FmtTraits<FMT>::bits;
-  for (uint32_t c = blockIdx.x * kDqThreads + threadIdx.x; c < n_chunks;
-       c += gridDim.x * kDqThreads) {
-    // 8 codes as four byte pairs
-    uint32_t pair[4];
-    if (bits == 8) {
-      const uint2 w = __ldg(reinterpret_cast<const uint2*>(elems + (size_t)c * 8));
-      pair[0] = w.x & 0xFFFF; pair[1] = w.x >> 16; pair[2] = w.y & 0xFFFF; pair[3] = w.y >> 16;
-    } else if (bits == 4) {
-      const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(elems + (size_t)c * 4));
+  constexpr int kElems = DTYPE == MX_BF16 ? 32 : 16;
+  constexpr int kLanes = kBlock / kElems;
+  constexpr int kInBytes = kElems * bits / 8;  // 32/24/16 or 16/12/8
+  constexpr int kWords = kInBytes / 4;
+  for (uint32_t unit = blockIdx.x * kDqThreads + threadIdx.x; unit < n_units;
+       unit += gridDim.x * kDqThreads) {
+    uint32_t w[kWords];
+    const uint8_t* src = elems + (size_t)unit * kInBytes;
+    if (kInBytes == 32) {
+      if (ALIGNED32) {
+        uint32_t t[8];
+        ld_stream_32(src, t);
 #pragma unroll
-      for (int i = 0; i < 4; ++i) pair[i] = (w >> (8 * i)) & 0xFF;
-    } else {
-      const uint16_t* p = reinterpret_cast<const uint16_t*>(elems + (size_t)c * 6);
-      const uint64_t w = (uint64_t)__ldg(p) | ((uint64_t)__ldg(p + 1) << 16) | ((uint64_t)__ldg(p + 2) << 32);
-#pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const uint32_t q = (uint32_t)(w >> (12 * i)) & 0xFFFu;  // two 6-bit codes
-        pair[i] = (q & 0x3F) | ((q & 0xFC0) << 2);
+        for (int i = 0; i < 8; ++i) w[i % kWords] = t[i];
+      } else {
+        const uint4 a = ld_stream_16(src), b = ld_stream_16(src + 16);
+        w[0] = a.x; w[1] = a.y; w[2] = a.z; w[3] = a.w;
+        w[4 % kWords] = b.x; w[5 % kWords] = b.y; w[6 % kWords] = b.z; w[7 % kWords] = b.w;
       }
+    } else if (kInBytes == 16) {
+      const uint4 a = ld_stream_16(src);
+      w[0] = a.x; w[1] = a.y; w[2 % kWords] = a.z; w[3 % kWords] = a.w;
+    } else if (kInBytes == 8) {
+      const uint2 a = __ldg(reinterpret_cast<const uint2*>(src));
+      w[0] = a.x; w[1] = a.y;
+    } else if (kInBytes == 24) {  // 8-byte aligned
+#pragma unroll
+      for (int i = 0; i < 3; ++i) {
+        const uint2 a = __ldg(reinterpret_cast<const uint2*>(src) + i);
+        w[(2 * i) % kWords] = a.x; w[(2 * i + 1) % kWords] = a.y;
+      }
+    } else {  // 12 bytes, 4-byte aligned
+#pragma unroll
+      for (int i = 0; i < 3; ++i) w[i % kWords] = __ldg(reinterpret_cast<const uint32_t*>(src) + i);
     }
-    const uint32_t blk = c >> 2;
+    const uint32_t blk = unit / kLanes;
     size_t off;
     if (LAYOUT == MX_SCALES_LINEAR) {
       off = blk;
@@ -72,54 +92,71 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
     const uint32_t sb = __ldg(scales + off);
     // X = 2^(sb - 127); sb = 0 is the FP32 subnormal 2^-127, sb = 255 is NaN
     const float X = __uint_as_float(sb == 0 ? 0x00400000u : (sb == 255 ? 0x7FC00000u : sb << 23));
-    uint32_t r[8];
+    uint32_t r[kElems];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
+    for (int i = 0; i < kElems / 2; ++i) {
+      uint32_t pair;  // code(2i) | code(2i+1) << 8   (4-bit: both in the low byte)
+      if (bits == 8) {
+        pair = (w[i / 2] >> (16 * (i & 1))) & 0xFFFFu;
+      } else if (bits == 4) {
+        pair = (w[i / 4] >> (8 * (i & 3))) & 0xFFu;
+      } else {
+        const int bit = 12 * i;  // two 6-bit codes at bit offset 12 i of the stream
+        uint32_t q = w[bit / 32] >> (bit % 32);
+        if (bit % 32 > 20) q |= w[(bit / 32 + 1) % kWords] << (32 - bit % 32);
+        q &= 0xFFFu;
+        pair = (q & 0x3Fu) | ((q & 0xFC0u) << 2);
+      }
       float a, b;
-      decode_pair<FMT>(pair[i], a, b);
+      decode_pair<FMT>(pair, a, b);
       a *= X;  // exact unless it overflows to Inf
       b *= X;
       r[2 * i] = (a != a) ? 0x7FC00000u : __float_as_uint(a);
       r[2 * i + 1] = (b != b) ? 0x7FC00000u : __float_as_uint(b);
     }
+    char* dst = reinterpret_cast<char*>(out) + (size_t)unit * 64;
+    uint32_t o[16];
     if (DTYPE == MX_F32) {
-      if (ALIGNED32) {
-        st_32(reinterpret_cast<char*>(out) + (size_t)c * 32, r);
-      } else {
-        uint4* o = reinterpret_cast<uint4*>(out) + (size_t)c * 2;
-        o[0] = make_uint4(r[0], r[1], r[2], r[3]);
-        o[1] = make_uint4(r[4], r[5], r[6], r[7]);
-      }
-    } else {
-      uint32_t w[4];
 #pragma unroll
-      for (int i = 0; i < 4; ++i) {
-        const float lo = __uint_as_float(r[2 * i]), hi = __uint_as_float(r[2 * i + 1]);
+      for (int i = 0; i < 16; ++i) o[i] = r[i % kElems];
+    } else {
+#pragma unroll
+      for (int i = 0; i < 16; ++i) {
+        const float lo = __uint_as_float(r[(2 * i) % kElems]), hi = __uint_as_float(r[(2 * i + 1) % kElems]);
         uint32_t pk;
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));  // round to nearest even
         if (lo != lo) pk = (pk & 0xFFFF0000u) | 0x7FC0u;
         if (hi != hi) pk = (pk & 0x0000FFFFu) | 0x7FC00000u;
-        w[i] = pk;
+        o[i] = pk;
       }
-      reinterpret_cast<uint4*>(out)[c] = make_uint4(w[0], w[1], w[2], w[3]);
+    }
+    if (ALIGNED32) {
+      const uint32_t o0[8] = {o[0], o[1], o[2], o[3], o[4], o[5], o[6], o[7]};
+      const uint32_t o1[8] = {o[8], o[9], o[10], o[11], o[12], o[13], o[14], o[15]};
+      st_32(dst, o0);
+      st_32(dst + 32, o1);
+    } else {
+#pragma unroll
+      for (int j = 0; j < 4; ++j)
+        reinterpret_cast<uint4*>(dst)[j] = make_uint4(o[4 * j], o[4 * j + 1], o[4 * j + 2], o[4 * j + 3]);
     }
   }
 }
 
 template <int FMT, int DTYPE, int LAYOUT>
 static cudaError_t launch_dq(const DequantizeArgs& a) {
-  const uint32_t n_chunks = (uint32_t)(a.rows * a.L / 8);
+  constexpr int kElems = DTYPE == MX_BF16 ? 32 : 16;
+  const uint32_t n_units = (uint32_t)(a.rows * a.L / kElems);
   const uint32_t kblocks = (uint32_t)(a.L / kBlock);
-  uint32_t grid = (n_chunks + kDqThreads - 1) / kDqThreads;
-  const uint32_t cap = (uint32_t)a.sm_count * 32;
-  if (grid > cap) grid = cap;
   const FastDiv kd = make_fastdiv(kblocks);
-  if (DTYPE == MX_F32 && (uintptr_t)a.out % 32 == 0)
-    dequantize_kernel<FMT, DTYPE, LAYOUT, true><<<grid, kDqThreads, 0, a.stream>>>(
-        a.elems, a.scales, a.out, n_chunks, kblocks, kd);
-  else
-    dequantize_kernel<FMT, DTYPE, LAYOUT, false><<<grid, kDqThreads, 0, a.stream>>>(
-        a.elems, a.scales, a.out, n_chunks, kblocks, kd);
+  const bool al32 = (uintptr_t)a.out % 32 == 0 && (uintptr_t)a.elems % 32 == 0;
+  auto kernel = al32 ? dequantize_kernel<FMT, DTYPE, LAYOUT, true> : dequantize_kernel<FMT, DTYPE, LAYOUT, false>;
+  uint32_t grid = (n_units + kDqThreads - 1) / kDqThreads;
+#if MX_DQ_CAP > 0
+  const uint32_t cap = (uint32_t)a.sm_count * MX_DQ_CAP;
+  if (grid > cap) grid = cap;
+#endif
+  kernel<<<grid, kDqThreads, 0, a.stream>>>(a.elems, a.scales, a.out, n_units, kblocks, kd);
   return cudaGetLastError();
 }
 

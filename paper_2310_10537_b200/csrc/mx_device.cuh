@@ -125,9 +125,11 @@ __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
     asm("{ .reg .b8 t; cvt.rn.satfinite.e2m1x2.f32 t, %1, %2; mov.b16 %0, {t, 0}; }"
         : "=h"(p) : "f"(hi), "f"(lo));
   } else {  // INT8: value n/64, inputs already multiplied by 64; saturate at +-127
-    const int a = __float2int_rn(fminf(fmaxf(lo, -127.0f), 127.0f));
-    const int b = __float2int_rn(fminf(fmaxf(hi, -127.0f), 127.0f));
-    p = (uint16_t)((a & 0xFF) | ((b & 0xFF) << 8));
+    // x + 1.5 * 2^23 rounds x to an integer (nearest even) in the low mantissa bits, as two's
+    // complement for negative x: no float-to-int conversion needed.
+    const float a = fminf(fmaxf(lo, -127.0f), 127.0f) + 12582912.0f;
+    const float b = fminf(fmaxf(hi, -127.0f), 127.0f) + 12582912.0f;
+    p = (uint16_t)((__float_as_uint(a) & 0xFFu) | ((__float_as_uint(b) & 0xFFu) << 8));
   }
   return p;
 }

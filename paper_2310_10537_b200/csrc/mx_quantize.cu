@@ -15,92 +15,173 @@
 namespace mx {
 
 constexpr int kThreads = 256;
+#ifndef MX_Q_U
+#define MX_Q_U 1      // 64-byte units per thread and loop iteration
+#endif
+#ifndef MX_Q_CAP
+#define MX_Q_CAP 0     // CTAs per SM the grid is capped at (0 = no cap, -1 = resident CTAs)
+#endif
+#ifndef MX_Q_MINB
+#define MX_Q_MINB 4   // resident CTAs per SM the register allocation must allow
+#endif
 
 // ---------------------------------------------------------------------------
 // Contiguous axis
 // ---------------------------------------------------------------------------
 
-// Load 8 consecutive elements as FP32 values.  chunk = index of the 8-element
-// group.  ALIGNED32: the FP32 tensor base is 32-byte aligned (256-bit load).
+// A thread owns 64 bytes of input: one whole block of BF16 (32 elements) or half
+// a block of FP32 (16 elements, the other half in the neighbouring lane).  It
+// reads them with two 256-bit loads (four 128-bit loads when the tensor is only
+// 16-byte aligned), so a block needs at most one shuffle, the scale is computed
+// once per 64 bytes, and the codes leave as one 32 / 16-byte store.
+template <int DTYPE> struct LastAxis {
+  static constexpr int kElems = DTYPE == MX_BF16 ? 32 : 16;  // elements per thread
+  static constexpr int kLanes = kBlock / kElems;             // lanes per MX block
+};
+
 template <int DTYPE, bool ALIGNED32>
-__device__ __forceinline__ void load8(const void* in, size_t chunk, float (&v)[8]) {
-  if (DTYPE == MX_BF16) {
-    const uint4 w = ld_stream_16(reinterpret_cast<const uint4*>(in) + chunk);
-    const uint32_t u[4] = {w.x, w.y, w.z, w.w};
+__device__ __forceinline__ void load_unit(const void* in, size_t unit,
+                                          float (&v)[LastAxis<DTYPE>::kElems]) {
+  uint32_t w[16];
+  const char* p = reinterpret_cast<const char*>(in) + unit * 64;
+  if (ALIGNED32) {
+    uint32_t a[8], b[8];
+    ld_stream_32(p, a);
+    ld_stream_32(p + 32, b);
 #pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      v[2 * i] = __uint_as_float(u[i] << 16);  // BF16 widens exactly
-      v[2 * i + 1] = __uint_as_float(u[i] & 0xFFFF0000u);
-    }
-  } else if (ALIGNED32) {
-    uint32_t u[8];
-    ld_stream_32(reinterpret_cast<const char*>(in) + chunk * 32, u);
-#pragma unroll
-    for (int i = 0; i < 8; ++i) v[i] = __uint_as_float(u[i]);
+    for (int i = 0; i < 8; ++i) { w[i] = a[i]; w[8 + i] = b[i]; }
   } else {
-    const uint4* p = reinterpret_cast<const uint4*>(in) + chunk * 2;
-    const uint4 a = __ldg(p), b = __ldg(p + 1);
-    v[0] = __uint_as_float(a.x); v[1] = __uint_as_float(a.y);
-    v[2] = __uint_as_float(a.z); v[3] = __uint_as_float(a.w);
-    v[4] = __uint_as_float(b.x); v[5] = __uint_as_float(b.y);
-    v[6] = __uint_as_float(b.z); v[7] = __uint_as_float(b.w);
+#pragma unroll
+    for (int j = 0; j < 4; ++j) {
+      const uint4 q = ld_stream_16(p + 16 * j);
+      w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
+    }
+  }
+  if (DTYPE == MX_BF16) {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) {
+      v[(2 * i) % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i] << 16);  // BF16 widens exactly
+      v[(2 * i + 1) % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i] & 0xFFFF0000u);
+    }
+  } else {
+#pragma unroll
+    for (int i = 0; i < 16; ++i) v[i % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i]);
   }
 }
 
-// U chunks of 8 elements per thread per iteration, all loads issued before any
-// arithmetic so that U * 16 (BF16) or U * 32 (FP32) bytes per thread are in flight.
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, bool ALIGNED32, int U>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kThreads, MX_Q_MINB)
 quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
-                         uint8_t* __restrict__ scales, uint32_t n_chunks, uint32_t kblocks,
-                         FastDiv kb_div) {
+                         uint8_t* __restrict__ scales, uint32_t n_units, uint32_t kblocks,
+                         FastDiv kb_div, uint32_t scale_words) {
   constexpr int bits = FmtTraits<FMT>::bits;
-  const uint32_t lane4 = threadIdx.x & 3u;  // position of this thread's 8 elements in the block
+  constexpr int kElems = LastAxis<DTYPE>::kElems;
+  constexpr int kLanes = LastAxis<DTYPE>::kLanes;
+  constexpr int kOutBytes = kElems * bits / 8;  // 32/24/16 (BF16) or 16/12/8 (FP32) per thread
+  const uint32_t lane = threadIdx.x & 31u;
   const uint32_t span = kThreads * U;
-  for (uint32_t base = blockIdx.x * span; base < n_chunks; base += gridDim.x * span) {
-    float v[U][8];
+  for (uint32_t base = blockIdx.x * span; base < n_units; base += gridDim.x * span) {
+    float v[U][kElems];
     bool ok[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const uint32_t c = base + u * kThreads + threadIdx.x;
-      ok[u] = c < n_chunks;  // whole groups of 4 lanes are in or out: n_chunks % 4 == 0
+      const uint32_t unit = base + u * kThreads + threadIdx.x;
+      ok[u] = unit < n_units;  // groups of 4 blocks are in or out together: n_units * kLanes % 4 == 0 or tail
       if (ok[u]) {
-        load8<DTYPE, ALIGNED32>(in, c, v[u]);
+        load_unit<DTYPE, ALIGNED32>(in, unit, v[u]);
       } else {
 #pragma unroll
-        for (int i = 0; i < 8; ++i) v[u][i] = 0.0f;
+        for (int i = 0; i < kElems; ++i) v[u][i] = 0.0f;
       }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
-      const uint32_t c = base + u * kThreads + threadIdx.x;
-      // Line 1 of Algorithm 1: max |V_i| over the block (8 local values, 4 lanes).
+      const uint32_t unit = base + u * kThreads + threadIdx.x;
+      // Line 1 of Algorithm 1: max |V_i| over the block
       float amax = absmax_nan(v[u][0], v[u][1]);
 #pragma unroll
-      for (int i = 2; i < 8; ++i) amax = absmax_nan(amax, v[u][i]);
-      amax = absmax_nan(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
-      amax = absmax_nan(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 2));
+      for (int i = 2; i < kElems; ++i) amax = absmax_nan(amax, v[u][i]);
+      if (kLanes == 2) amax = absmax_nan(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
       const BlockScale s = block_scale<FMT>(amax);
       // Lines 3-5: P_i = quantize(V_i / X)
-      uint32_t lo, hi;
-      cast8<FMT, ROUND>(v[u], s, lo, hi);
-      if (bits == 6) {
-        // 4 lanes hold 6 bytes each; lanes 0..2 of the group store 8 bytes each.
-        const uint64_t mine = (uint64_t)lo | ((uint64_t)hi << 32);
-        const uint32_t nlo = __shfl_down_sync(0xFFFFFFFFu, lo, 1);
-        const uint32_t nhi = __shfl_down_sync(0xFFFFFFFFu, hi, 1);
-        const uint64_t next = (uint64_t)nlo | ((uint64_t)nhi << 32);
-        const uint64_t q = (mine >> (16 * lane4)) | (next << (48 - 16 * lane4));
-        if (ok[u] && lane4 < 3) {
-          uint8_t* dst = elems + (size_t)(c >> 2) * 24 + lane4 * 8;
-          *reinterpret_cast<uint2*>(dst) = make_uint2((uint32_t)q, (uint32_t)(q >> 32));
-        }
-      } else if (ok[u]) {
-        if (bits == 8) *reinterpret_cast<uint2*>(elems + (size_t)c * 8) = make_uint2(lo, hi);
-        else *reinterpret_cast<uint32_t*>(elems + (size_t)c * 4) = lo;
+      uint32_t w[kElems / 4];  // 8-bit: all words; 6-bit: 3 of every 4; 4-bit: every other
+#pragma unroll
+      for (int g = 0; g < kElems / 8; ++g) {
+        float x[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) x[i] = v[u][8 * g + i];
+        cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
       }
-      if (ok[u] && lane4 == 0) {
-        const uint32_t blk = c >> 2;
+      uint8_t* dst = elems + (size_t)unit * kOutBytes;
+      if (bits == 8) {
+        if (kElems == 32) {
+          if (ok[u]) {
+            if (ALIGNED32) {
+              const uint32_t o[8] = {w[0], w[1], w[2], w[3], w[4 % (kElems / 4)], w[5 % (kElems / 4)],
+                                     w[6 % (kElems / 4)], w[7 % (kElems / 4)]};
+              st_32(dst, o);
+            } else {
+              reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+              reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4 % (kElems / 4)], w[5 % (kElems / 4)],
+                                                            w[6 % (kElems / 4)], w[7 % (kElems / 4)]);
+            }
+          }
+        } else if (ok[u]) {
+          *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[1], w[2], w[3]);
+        }
+      } else if (bits == 4) {
+        if (kElems == 32) {
+          if (ok[u]) *reinterpret_cast<uint4*>(dst) = make_uint4(w[0], w[2], w[4 % (kElems / 4)], w[6 % (kElems / 4)]);
+        } else if (ok[u]) {
+          *reinterpret_cast<uint2*>(dst) = make_uint2(w[0], w[2]);
+        }
+      } else {
+        // 6-bit: each group of 8 codes is 48 bits (lo 32 + hi 16)
+        const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
+        const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
+        if (kElems == 32) {
+          const uint64_t g2 = (uint64_t)w[4 % (kElems / 4)] | ((uint64_t)w[5 % (kElems / 4)] << 32);
+          const uint64_t g3 = (uint64_t)w[6 % (kElems / 4)] | ((uint64_t)w[7 % (kElems / 4)] << 32);
+          const uint64_t q0 = g0 | (g1 << 48), q1 = (g1 >> 16) | (g2 << 32), q2 = (g2 >> 32) | (g3 << 16);
+          if (ok[u]) {
+            uint2* d2 = reinterpret_cast<uint2*>(dst);  // 24-byte blocks are 8-byte aligned
+            d2[0] = make_uint2((uint32_t)q0, (uint32_t)(q0 >> 32));
+            d2[1] = make_uint2((uint32_t)q1, (uint32_t)(q1 >> 32));
+            d2[2] = make_uint2((uint32_t)q2, (uint32_t)(q2 >> 32));
+          }
+        } else {
+          // 12 bytes per lane, 24 per block: the even lane stores bytes 0..15, the odd lane 16..23
+          const uint32_t t0 = (uint32_t)g0, t1 = (uint32_t)(g0 >> 32) | ((uint32_t)g1 << 16),
+                         t2 = (uint32_t)(g1 >> 16);
+          const uint32_t n0 = __shfl_down_sync(0xFFFFFFFFu, t0, 1);
+          if (ok[u]) {
+            uint8_t* blk = elems + (size_t)(unit >> 1) * 24;
+            if ((lane & 1u) == 0) {
+              reinterpret_cast<uint2*>(blk)[0] = make_uint2(t0, t1);
+              reinterpret_cast<uint2*>(blk)[1] = make_uint2(t2, n0);
+            } else {
+              reinterpret_cast<uint2*>(blk)[2] = make_uint2(t1, t2);
+            }
+          }
+        }
+      }
+      // scale bytes: four consecutive blocks of a row share one 32-bit word
+      const uint32_t blk = unit / kLanes;
+      if (scale_words) {
+        uint32_t word = s.byte << (8 * (blk & 3u));
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, kLanes);
+        word |= __shfl_xor_sync(0xFFFFFFFFu, word, 2 * kLanes);
+        if (ok[u] && (lane & (4 * kLanes - 1)) == 0) {
+          size_t off;
+          if (LAYOUT == MX_SCALES_LINEAR) {
+            off = blk;
+          } else {
+            const uint32_t row = fastdiv(blk, kb_div);
+            off = scale_offset<LAYOUT>(row, blk - row * kblocks, kblocks);
+          }
+          *reinterpret_cast<uint32_t*>(scales + off) = word;
+        }
+      } else if (ok[u] && (lane & (kLanes - 1)) == 0) {
         size_t off;
         if (LAYOUT == MX_SCALES_LINEAR) {
           off = blk;
@@ -211,24 +292,45 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
 // Host-side dispatch
 // ---------------------------------------------------------------------------
 
-template <int FMT, int ROUND, int DTYPE, int LAYOUT>
-static cudaError_t launch_lastaxis(const QuantizeArgs& a) {
-  constexpr int U = 4;
-  const uint32_t n_chunks = (uint32_t)(a.numel / 8);
+// Resident CTAs per SM of a kernel (queried once per instantiation): persistent grids are sized
+// to exactly fill the machine so that no partial wave trails the launch.
+template <typename K>
+static int resident_ctas(K kernel, int threads) {
+  int n = 0;
+  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1) n = 1;
+  return n;
+}
+
+template <int FMT, int ROUND, int DTYPE, int LAYOUT, bool AL32>
+static cudaError_t launch_lastaxis_al(const QuantizeArgs& a) {
+  constexpr int U = MX_Q_U;
+  constexpr int kElems = LastAxis<DTYPE>::kElems;
+  const uint32_t n_units = (uint32_t)(a.numel / kElems);
+  const uint32_t n_blocks = (uint32_t)(a.numel / kBlock);
   const uint32_t kblocks = (uint32_t)(a.L / kBlock);
   const uint32_t span = kThreads * U;
-  uint32_t grid = (n_chunks + span - 1) / span;
-  const uint32_t cap = (uint32_t)a.sm_count * 8;
+  auto kernel = quantize_lastaxis_kernel<FMT, ROUND, DTYPE, LAYOUT, AL32, U>;
+  uint32_t grid = (n_units + span - 1) / span;
+#if MX_Q_CAP > 0
+  const uint32_t cap = (uint32_t)a.sm_count * MX_Q_CAP;
   if (grid > cap) grid = cap;
+#elif MX_Q_CAP < 0
+  static const int per_sm = resident_ctas(kernel, kThreads);
+  const uint32_t cap = (uint32_t)(a.sm_count * per_sm);
+  if (grid > cap) grid = cap;
+#endif
   const FastDiv kd = make_fastdiv(kblocks);
-  const bool al32 = DTYPE == MX_F32 && ((uintptr_t)a.in % 32 == 0);
-  if (al32)
-    quantize_lastaxis_kernel<FMT, ROUND, DTYPE, LAYOUT, true, U><<<grid, kThreads, 0, a.stream>>>(
-        a.in, a.elems, a.scales, n_chunks, kblocks, kd);
-  else
-    quantize_lastaxis_kernel<FMT, ROUND, DTYPE, LAYOUT, false, U><<<grid, kThreads, 0, a.stream>>>(
-        a.in, a.elems, a.scales, n_chunks, kblocks, kd);
+  // one 32-bit store per four scale bytes when groups of four never straddle a row or the end
+  const uint32_t scale_words = LAYOUT == MX_SCALES_LINEAR ? (n_blocks % 4 == 0) : (kblocks % 4 == 0);
+  kernel<<<grid, kThreads, 0, a.stream>>>(a.in, a.elems, a.scales, n_units, kblocks, kd, scale_words);
   return cudaGetLastError();
+}
+
+template <int FMT, int ROUND, int DTYPE, int LAYOUT>
+static cudaError_t launch_lastaxis(const QuantizeArgs& a) {
+  if ((uintptr_t)a.in % 32 == 0 && (uintptr_t)a.elems % 32 == 0)
+    return launch_lastaxis_al<FMT, ROUND, DTYPE, LAYOUT, true>(a);
+  return launch_lastaxis_al<FMT, ROUND, DTYPE, LAYOUT, false>(a);
 }
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
