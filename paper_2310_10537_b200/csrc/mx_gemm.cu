@@ -49,10 +49,12 @@ __device__ unsigned int g_gemm_status;
 
 template <int BN>
 struct Cfg {
-  static_assert(BN == 128 || BN == 256, "tile width");
-  static constexpr int kStages = BN == 256 ? 4 : 6;
+  static_assert(BN == 128 || BN == 192 || BN == 256, "tile width");
+  static constexpr int kStages = BN == 256 ? 4 : (BN == 192 ? 5 : 6);
   static constexpr int kAccStages = BN == 256 ? 1 : 2;
-  static constexpr int kSfbChunks = BN / 128;             // 512-byte scale chunks of B per stage
+  // 512-byte scale chunks (128 rows each) of B per stage; a 192-wide tile starts on a
+  // 64-row boundary and always lies inside two consecutive chunks
+  static constexpr int kSfbChunks = BN == 128 ? 1 : 2;
   static constexpr int kSfCols = 4 + 4 * kSfbChunks;       // TMEM columns of scales per stage
   static constexpr int kSfCol0 = kAccStages * BN;          // first scale column
   static constexpr uint32_t kABytes = BM * BK;             // one byte per element in shared memory
@@ -215,7 +217,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tiles_m = M / BM, tiles_n = N / BN, num_tiles = tiles_m * tiles_n;
+  const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
+  const uint32_t n_chunks128 = N / 128;  // scale chunks of B along N
   const uint32_t k_chunks = K / BK;
 
   if (threadIdx.x == 0) {
@@ -257,7 +260,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             break;
           }
           const uint32_t fb = full_bar(stage);
-          mbar_arrive_expect_tx(fb, tx_bytes);
+          // a ragged last tile (BN = 192) may reach past the last scale chunk of B
+          const uint32_t sfb_first = tc.tn * BN / 128;
+          const uint32_t sfb_have = min((uint32_t)cfg::kSfbChunks, n_chunks128 - sfb_first);
+          mbar_arrive_expect_tx(fb, tx_bytes - 512u * (cfg::kSfbChunks - sfb_have));
           tma_load_2d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BK),
                       (int)(tc.tm * BM), fb);
           tma_load_2d(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, (int)(kc * BK),
@@ -266,8 +272,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           bulk_load(sf, sA + ((size_t)tc.tm * k_chunks + kc) * 512, 512, fb);
 #pragma unroll
           for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
-            bulk_load(sf + 512 + 512 * j,
-                      sB + ((size_t)(tc.tn * cfg::kSfbChunks + j) * k_chunks + kc) * 512, 512, fb);
+            if (j < sfb_have)
+              bulk_load(sf + 512 + 512 * j, sB + ((size_t)(sfb_first + j) * k_chunks + kc) * 512, 512, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -288,6 +294,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
         tc_fence_after();
         const uint32_t d_tmem = tmem_base + acc * BN;
+        // scales of row n of the tile sit in column (n0 % 128 + n) / 32 of the copied chunks
+        const uint32_t sfb_col = 4 + ((tile_coord(t, tiles_m, tiles_n, group_m).tn * BN) % 128) / 32;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
             raise_abort(abort_flag, ST_MMA_WAIT_FULL);
@@ -307,7 +315,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           for (uint32_t k = 0; k < BK / kMmaK; ++k) {
             // byte k of each 32-bit scale column belongs to MX block k of this stage
             const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
-            tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4,
+            tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + sfb_col,
                    (kc | k) != 0 ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
@@ -331,23 +339,29 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t row = tc.tm * BM + quarter * 32 + lane;
       float* crow = C + (size_t)row * N + (size_t)tc.tn * BN;
       const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * BN;
-#pragma unroll 1
-      for (uint32_t c0 = 0; c0 < BN; c0 += 32) {
-        uint32_t r[32];
-        tc_ld32(taddr + c0, r);
+      const uint32_t valid_cols = min((uint32_t)BN, N - tc.tn * BN);  // multiple of 64
+      // two register buffers: the load of chunk j+1 is in flight while chunk j is stored
+      uint32_t r[2][32];
+      tc_ld32(taddr, r[0]);
+#pragma unroll
+      for (uint32_t j = 0; j < BN / 32; ++j) {
         tc_wait_ld();
-        if (c_aligned32) {
+        if (j + 1 < BN / 32) tc_ld32(taddr + 32 * (j + 1), r[(j + 1) & 1]);
+        const uint32_t c0 = 32 * j;
+        if (c0 < valid_cols) {
+          if (c_aligned32) {
 #pragma unroll
-          for (int i = 0; i < 4; ++i)
-            asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(crow + c0 + 8 * i),
-                         "r"(r[8 * i]), "r"(r[8 * i + 1]), "r"(r[8 * i + 2]), "r"(r[8 * i + 3]),
-                         "r"(r[8 * i + 4]), "r"(r[8 * i + 5]), "r"(r[8 * i + 6]), "r"(r[8 * i + 7])
-                         : "memory");
-        } else {
+            for (int i = 0; i < 4; ++i)
+              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(crow + c0 + 8 * i),
+                           "r"(r[j & 1][8 * i]), "r"(r[j & 1][8 * i + 1]), "r"(r[j & 1][8 * i + 2]),
+                           "r"(r[j & 1][8 * i + 3]), "r"(r[j & 1][8 * i + 4]), "r"(r[j & 1][8 * i + 5]),
+                           "r"(r[j & 1][8 * i + 6]), "r"(r[j & 1][8 * i + 7]) : "memory");
+          } else {
 #pragma unroll
-          for (int i = 0; i < 8; ++i)
-            *reinterpret_cast<uint4*>(crow + c0 + 4 * i) =
-                make_uint4(r[4 * i], r[4 * i + 1], r[4 * i + 2], r[4 * i + 3]);
+            for (int i = 0; i < 8; ++i)
+              *reinterpret_cast<uint4*>(crow + c0 + 4 * i) =
+                  make_uint4(r[j & 1][4 * i], r[j & 1][4 * i + 1], r[j & 1][4 * i + 2], r[j & 1][4 * i + 3]);
+          }
         }
       }
       tc_fence_before();
@@ -430,7 +444,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)(a.M / BM) * (uint32_t)(a.N / BN);
+  const uint32_t tiles = (uint32_t)(a.M / BM) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
   const uint32_t group_m = 16;
   // Bytes the producer's copies report to a stage's mbarrier: the tensor-map copies count the
@@ -450,7 +464,14 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   EncodeTiledFn fn = encode_fn(cuda_err);
   if (!fn) return MX_ERR_CUDA;
-  const int bn = (a.N % 256 == 0) ? 256 : 128;
+#ifdef MX_GEMM_BN
+  const int bn = MX_GEMM_BN;
+#else
+  // 256-wide tiles move the fewest operand bytes through shared memory per flop; problems with
+  // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
+  const int64_t tiles256 = (a.M / BM) * ((a.N + 255) / 256);
+  const int bn = tiles256 >= a.sm_count ? 256 : 128;
+#endif
   CUtensorMap ma, mb;
   if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, BM) ||
       !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, (uint32_t)bn)) {
@@ -460,7 +481,8 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   // a_format [7,10), b_format [10,13), K-major A and B, scale format E8M0 (bit 23), M = 128
   const uint32_t idesc = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23) |
                          ((uint32_t)(BM >> 4) << 24);
-  *cuda_err = bn == 256 ? launch_bn<256>(a, ma, mb, idesc) : launch_bn<128>(a, ma, mb, idesc);
+  *cuda_err = bn == 256 ? launch_bn<256>(a, ma, mb, idesc)
+              : bn == 192 ? launch_bn<192>(a, ma, mb, idesc) : launch_bn<128>(a, ma, mb, idesc);
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
 }
 
