@@ -54,7 +54,7 @@ class MxError(RuntimeError):
 def _load() -> ctypes.CDLL:
     if not os.path.exists(LIB_PATH):
         raise ImportError(
-            f"{LIB_PATH} is missing: build it with `python -m paper_2310_10537_b200.build` "
+            f"{LIB_PATH} is missing: build it with `python paper_2310_10537_b200/build.py` "
             "(the library has no CPU or PyTorch fallback)")
     lib = ctypes.CDLL(LIB_PATH)
     vp, i64p, u8p = ctypes.c_void_p, ctypes.POINTER(ctypes.c_int64), ctypes.c_void_p
