@@ -326,7 +326,7 @@ def main_ours(args, rank, world, local_rank):
             "traffic": NCU_TRAFFIC.get("quantize"),
         },
         "roofline_gemm": {
-            "kernel": "mx_gemm_kernel<256>", "bound": "tensor", "achieved": gemm_tflops / world,
+            "kernel": "mx_gemm_pair_kernel (two-CTA 256x256 tiles, tcgen05 cta_group::2)", "bound": "tensor", "achieved": gemm_tflops / world,
             "peak": fp8_peak, "unit": "TFLOP/s", "frac": gemm_tflops / world / fp8_peak,
             "peak_source": f"2 x {peaks['source']} BF16 burst (nominal FP8:BF16 ratio)",
             "frac_of_sustained": gemm_tflops / world / (2.0 * peaks["bf16_tflops_sustained"]),

@@ -14,7 +14,8 @@
 //             512-byte swizzled scale chunks -> shared-memory ring
 //   warp 1    MMA issuer: scales shared -> tensor memory (tcgen05.cp), four
 //             MMAs per stage, tcgen05.commit releases the stage / the accumulator
-//   warps 2-5 epilogue: tensor memory -> registers -> FP32 C
+//   warps 2-9 epilogue: tensor memory -> registers (the accumulator is released as soon as
+//             it is in registers) -> FP32 C, overlapping the next tile's MMAs
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status
 // word, raises a CTA-wide abort flag and every role falls through to the common
 // exit, where tensor memory is released.
@@ -32,7 +33,7 @@ namespace {
 constexpr int BM = 128;         // rows of C per tile (= MMA M, one TMEM lane per row)
 constexpr int BK = 128;         // K elements per pipeline stage: 4 MX blocks, 4 MMAs
 constexpr int kMmaK = 32;       // K of one kind::mxf8f6f4 MMA = the MX block size
-constexpr int kThreads = 192;   // 6 warps
+constexpr int kThreads = 320;   // 10 warps: producer, MMA issuer, 8 epilogue warps
 constexpr int kTmemCols = 512;  // whole tensor memory of the SM (one CTA per SM)
 constexpr long long kSpinLimit = 2000000000LL;  // cycles (~1 s) before a wait gives up
 
@@ -47,14 +48,21 @@ enum : unsigned int {
 // First failure of any GEMM launch on this device since the last check (0 = none).
 __device__ unsigned int g_gemm_status;
 
+// Epilogue staging in shared memory: chunks of 32 rows x 16 columns of FP32 per warp.
+constexpr uint32_t kEpiChunkCols = 16;
+constexpr uint32_t kEpiChunkBytes = 32 * kEpiChunkCols * 4;
+#ifndef MX_EPI_BUFS
+#define MX_EPI_BUFS 1
+#endif
+constexpr uint32_t kEpiBufs = MX_EPI_BUFS;                        // staging chunks per warp
+constexpr uint32_t kEpiBytes = 8 * kEpiBufs * kEpiChunkBytes;     // eight epilogue warps
+
 template <int BN>
 struct Cfg {
-  static_assert(BN == 128 || BN == 192 || BN == 256, "tile width");
-  static constexpr int kStages = BN == 256 ? 4 : (BN == 192 ? 5 : 6);
+  static_assert(BN == 128 || BN == 256, "tile width");
+  static constexpr int kStages = BN == 256 ? 4 : 6;
   static constexpr int kAccStages = BN == 256 ? 1 : 2;
-  // 512-byte scale chunks (128 rows each) of B per stage; a 192-wide tile starts on a
-  // 64-row boundary and always lies inside two consecutive chunks
-  static constexpr int kSfbChunks = BN == 128 ? 1 : 2;
+  static constexpr int kSfbChunks = BN / 128;  // 512-byte scale chunks (128 rows each) of B per stage
   static constexpr int kSfCols = 4 + 4 * kSfbChunks;       // TMEM columns of scales per stage
   static constexpr int kSfCol0 = kAccStages * BN;          // first scale column
   static constexpr uint32_t kABytes = BM * BK;             // one byte per element in shared memory
@@ -62,12 +70,14 @@ struct Cfg {
   static constexpr uint32_t kSfBytes = 512 * (1 + kSfbChunks);
   static constexpr uint32_t kOffA = 0;
   static constexpr uint32_t kOffB = kOffA + kStages * kABytes;
-  static constexpr uint32_t kOffSf = kOffB + kStages * kBBytes;
+  static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;   // 1024-byte aligned
+  static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
   // barriers: full[S], empty[S], acc_full[A], acc_empty[A]; then tmem slot + abort flag
   static constexpr uint32_t kNumBars = 2 * kStages + 2 * kAccStages;
   static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;  // + alignment slack
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
+  static_assert(kSmemBytes <= 232448, "shared memory budget");
 };
 
 // ---- PTX wrappers ------------------------------------------------------------
@@ -105,17 +115,15 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
     }
   }
 }
-__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y,
+// Every copy of a stage (A tile, B tile, A scales, B scales) goes through a rank-3 tensor map, so
+// that lanes 0..3 of the producer warp can issue all four with ONE warp instruction, each lane
+// with its own map, coordinates and destination: issuing them one after the other from a single
+// thread costs more than the 512 clocks a stage's MMAs take.
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
                                             uint32_t bar) {
   asm volatile(
-      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
-}
-__device__ __forceinline__ void bulk_load(uint32_t dst, const void* src, uint32_t bytes,
-                                          uint32_t bar) {
-  asm volatile(
-      "cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
-      ::"r"(dst), "l"(src), "r"(bytes), "r"(bar) : "memory");
+      "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
@@ -175,6 +183,57 @@ __device__ __forceinline__ uint64_t scale_desc(uint32_t saddr) {
   return lo | (hi << 32);
 }
 
+// ---- epilogue: registers -> shared memory -> TMA store ---------------------------
+// A thread holds one row of the accumulator, so direct global stores would touch 32
+// different lines per warp instruction and crowd the L1 data path that also feeds the
+// tensor core from shared memory.  Instead each warp stages 32 rows x 16 columns (2 KB,
+// 64-byte rows in the 64-byte TMA swizzle, conflict-free 16-byte stores) and one lane
+// hands the chunk to the TMA engine, which writes full lines and clips at the tensor edge.
+
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, int x, int y, uint32_t src) {
+  asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%1, %2}], [%3];"
+               ::"l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(src) : "memory");
+  asm volatile("cp.async.bulk.commit_group;" ::: "memory");
+}
+template <int N>
+__device__ __forceinline__ void bulk_wait_read() {
+  asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
+}
+__device__ __forceinline__ void bulk_wait_all() {
+  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
+}
+
+// r[j][i] = column 32 j + i of this thread's row (row0 + lane) starting at column col0 of C.
+template <uint32_t kLoads>
+__device__ __forceinline__ void store_rows(const uint32_t (&r)[kLoads][32], uint32_t stage_smem,
+                                           const CUtensorMap* tmap_c, int col0, int row0,
+                                           uint32_t valid_cols, uint32_t lane) {
+  if (lane == 0) bulk_wait_read<0>();  // chunks of the previous tile have left shared memory
+  __syncwarp();
+#pragma unroll
+  for (uint32_t q = 0; q < kLoads * 2; ++q) {
+    if (q * kEpiChunkCols < valid_cols) {
+      const uint32_t buf = q % kEpiBufs;
+      if (q >= kEpiBufs) {
+        if (lane == 0) bulk_wait_read<(int)kEpiBufs - 1>();
+        __syncwarp();
+      }
+      const uint32_t base = stage_smem + buf * kEpiChunkBytes + lane * 64;
+#pragma unroll
+      for (uint32_t c = 0; c < 4; ++c) {
+        const uint32_t* v = &r[q / 2][(q % 2) * 16 + 4 * c];
+        asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                     ::"r"(base + ((c ^ ((lane >> 1) & 3u)) << 4)), "r"(v[0]), "r"(v[1]), "r"(v[2]), "r"(v[3])
+                     : "memory");
+      }
+      asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+      __syncwarp();
+      if (lane == 0)
+        tma_store_2d(tmap_c, col0 + (int)(q * kEpiChunkCols), row0, stage_smem + buf * kEpiChunkBytes);
+    }
+  }
+}
+
 struct TileCoord {
   uint32_t tm, tn;
 };
@@ -200,9 +259,10 @@ __device__ __forceinline__ void raise_abort(volatile uint32_t* abort_flag, unsig
 template <int BN>
 __global__ void __launch_bounds__(kThreads, 1)
 mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const uint8_t* __restrict__ sA, const uint8_t* __restrict__ sB,
-               float* __restrict__ C, uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t c_aligned32, uint32_t tx_bytes) {
+               const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
+               const __grid_constant__ CUtensorMap tmap_c,
+               uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
+               uint32_t group_m, uint32_t tx_bytes) {
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -218,7 +278,6 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
-  const uint32_t n_chunks128 = N / 128;  // scale chunks of B along N
   const uint32_t k_chunks = K / BK;
 
   if (threadIdx.x == 0) {
@@ -228,13 +287,14 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
     for (uint32_t a = 0; a < cfg::kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
-      mbar_init(acc_empty_bar(a), 4);  // one arrival per epilogue warp
+      mbar_init(acc_empty_bar(a), 8);  // one arrival per epilogue warp
     }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_a)) : "memory");
     asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_b)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_c)) : "memory");
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
@@ -248,32 +308,32 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    if (lane == 0) {
+    // lanes 0..3 issue the four copies of a stage together (see tma_load_3d)
+    if (lane < 4) {
+      const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
+      const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
+                                                                                         : cfg::kOffSf + 512u;
+      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : lane == 1 ? cfg::kBBytes : cfg::kSfBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        // operands: (k, row, 0); scales: (0, k chunk, 128-row group).  Rows or groups past the end
+        // of B on a ragged last tile are zero-filled by the copy.
+        const int cy_fixed = lane == 0 ? (int)(tc.tm * BM) : (int)(tc.tn * BN);
+        const int cz = lane == 2 ? (int)tc.tm : lane == 3 ? (int)(tc.tn * BN / 128) : 0;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             ok = false;
-            break;
           }
+          if (!__all_sync(0xFu, ok)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
-          // a ragged last tile (BN = 192) may reach past the last scale chunk of B
-          const uint32_t sfb_first = tc.tn * BN / 128;
-          const uint32_t sfb_have = min((uint32_t)cfg::kSfbChunks, n_chunks128 - sfb_first);
-          mbar_arrive_expect_tx(fb, tx_bytes - 512u * (cfg::kSfbChunks - sfb_have));
-          tma_load_2d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BK),
-                      (int)(tc.tm * BM), fb);
-          tma_load_2d(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, (int)(kc * BK),
-                      (int)(tc.tn * BN), fb);
-          const uint32_t sf = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
-          bulk_load(sf, sA + ((size_t)tc.tm * k_chunks + kc) * 512, 512, fb);
-#pragma unroll
-          for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
-            if (j < sfb_have)
-              bulk_load(sf + 512 + 512 * j, sB + ((size_t)(sfb_first + j) * k_chunks + kc) * 512, 512, fb);
+          if (lane == 0) mbar_arrive_expect_tx(fb, tx_bytes);
+          __syncwarp(0xFu);
+          const int cx = lane < 2 ? (int)(kc * BK) : 0;
+          const int cy = lane < 2 ? cy_fixed : (int)kc;
+          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -305,10 +365,12 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           tc_fence_after();
           const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          tc_cp_scales(sf_tmem, scale_desc(sf_smem));
+          {
+            tc_cp_scales(sf_tmem, scale_desc(sf_smem));
 #pragma unroll
-          for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
-            tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
+            for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
+              tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
+          }
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
 #pragma unroll
@@ -327,7 +389,11 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     }
   } else {
     // -------------------------------- epilogue --------------------------------
-    const uint32_t quarter = warp & 3u;  // TMEM lanes this warp may read: 32*quarter .. +31
+    // Two warps per TMEM lane quarter, each taking half of the tile's columns into registers;
+    // the accumulator is handed back before the global stores are issued.
+    const uint32_t quarter = warp & 3u;           // TMEM lanes this warp may read: 32*quarter .. +31
+    const uint32_t half = (warp - 2u) >> 2;       // 0: columns [0, BN/2), 1: [BN/2, BN)
+    constexpr uint32_t kHalf = BN / 2, kLoads = kHalf / 32;
     uint32_t acc = 0, acc_phase = 0;
     for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
@@ -336,39 +402,21 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         break;
       }
       tc_fence_after();
-      const uint32_t row = tc.tm * BM + quarter * 32 + lane;
-      float* crow = C + (size_t)row * N + (size_t)tc.tn * BN;
-      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * BN;
-      const uint32_t valid_cols = min((uint32_t)BN, N - tc.tn * BN);  // multiple of 64
-      // two register buffers: the load of chunk j+1 is in flight while chunk j is stored
-      uint32_t r[2][32];
-      tc_ld32(taddr, r[0]);
+      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * BN + half * kHalf;
+      const uint32_t col0 = tc.tn * BN + half * kHalf;
+      const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;  // multiple of 32
+      uint32_t r[kLoads][32];
 #pragma unroll
-      for (uint32_t j = 0; j < BN / 32; ++j) {
-        tc_wait_ld();
-        if (j + 1 < BN / 32) tc_ld32(taddr + 32 * (j + 1), r[(j + 1) & 1]);
-        const uint32_t c0 = 32 * j;
-        if (c0 < valid_cols) {
-          if (c_aligned32) {
-#pragma unroll
-            for (int i = 0; i < 4; ++i)
-              asm volatile("st.global.v8.b32 [%0], {%1,%2,%3,%4,%5,%6,%7,%8};" ::"l"(crow + c0 + 8 * i),
-                           "r"(r[j & 1][8 * i]), "r"(r[j & 1][8 * i + 1]), "r"(r[j & 1][8 * i + 2]),
-                           "r"(r[j & 1][8 * i + 3]), "r"(r[j & 1][8 * i + 4]), "r"(r[j & 1][8 * i + 5]),
-                           "r"(r[j & 1][8 * i + 6]), "r"(r[j & 1][8 * i + 7]) : "memory");
-          } else {
-#pragma unroll
-            for (int i = 0; i < 8; ++i)
-              *reinterpret_cast<uint4*>(crow + c0 + 4 * i) =
-                  make_uint4(r[j & 1][4 * i], r[j & 1][4 * i + 1], r[j & 1][4 * i + 2], r[j & 1][4 * i + 3]);
-          }
-        }
-      }
+      for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
+      tc_wait_ld();
       tc_fence_before();
       __syncwarp();
-      if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+      if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // the MMA issuer may overwrite the accumulator
+      store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                         (int)col0, (int)(tc.tm * BM + quarter * 32), valid_cols, lane);
       if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
+    if (lane == 0) bulk_wait_all();  // this warp's stores have completed
   }
 
   // common exit: every role arrives here, also after an abort
@@ -377,6 +425,249 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)kTmemCols) : "memory");
+  }
+}
+
+
+// ============================================================================
+// Two-CTA variant: a cluster of two CTAs (two SMs) computes one 256 x 256 tile
+// with tcgen05.mma.cta_group::2.  CTA r of the pair stages rows 128r.. of the A
+// tile and rows 128r.. of the B tile, so each SM moves half of B through its
+// shared memory per flop compared with the one-CTA kernel.  The even CTA (the
+// leader) issues every MMA; its accumulator rows 0..127 live in its own tensor
+// memory, rows 128..255 in the peer's.
+//   - both producers copy with the mbarrier of the LEADER as completion target
+//     (cp.async.bulk.tensor ... .cta_group::2), the leader alone arms it with the
+//     byte count of both CTAs;
+//   - tcgen05.commit with a two-CTA mask releases a stage / publishes the
+//     accumulator in both CTAs;
+//   - the epilogue warps of both CTAs arrive on the leader's accumulator-empty
+//     barrier.
+// No load is multicast: each CTA fetches what it needs itself (the B scales are
+// fetched by both).
+// ============================================================================
+
+struct Cfg2 {
+  static constexpr int BN = 256;
+#ifndef MX_PAIR_STAGES
+#define MX_PAIR_STAGES 6
+#endif
+  static constexpr int kStages = MX_PAIR_STAGES;
+  static constexpr int kSfCols = 12;          // 4 (A) + 8 (B, all 256 rows) per stage
+  static constexpr int kSfCol0 = BN;          // single accumulator stage
+  static constexpr uint32_t kABytes = 128 * BK;   // this CTA's 128 rows of A
+  static constexpr uint32_t kBBytes = 128 * BK;   // this CTA's 128 rows of B
+  static constexpr uint32_t kSfBytes = 512 + 1024;
+  static constexpr uint32_t kOffA = 0;
+  static constexpr uint32_t kOffB = kOffA + kStages * kABytes;
+  static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;
+  static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
+  static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
+  static constexpr uint32_t kNumBars = 2 * kStages + 2;
+  static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
+  static_assert(kSmemBytes <= 232448, "shared memory budget");
+  static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
+};
+
+constexpr uint32_t kPeerMask = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address
+
+__device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
+                                                 int z, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+__device__ __forceinline__ void tc_cp_scales_pair(uint32_t taddr, uint64_t sdesc) {
+  asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
+}
+__device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                            uint32_t idesc, uint32_t sfa_tmem, uint32_t sfb_tmem,
+                                            uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf8f6f4.block_scale.scale_vec::1X [%0], %1, %2, %3, [%4], [%5], p;\n\t"
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
+        "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
+}
+__device__ __forceinline__ void cluster_sync() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
+                    const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
+                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair) {
+  using cfg = Cfg2;
+  constexpr int BN = cfg::BN;
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t bar0 = smem_base + cfg::kOffBar;
+  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (cfg::kStages + s); };
+  const uint32_t acc_full_bar = bar0 + 8 * (2 * cfg::kStages);
+  const uint32_t acc_empty_bar = bar0 + 8 * (2 * cfg::kStages + 1);
+  volatile uint32_t* tmem_slot =
+      reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  uint32_t rank;
+  asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
+  const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
+  const uint32_t k_chunks = K / BK;
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < cfg::kStages; ++s) {
+      mbar_init(full_bar(s), 1);   // used in the leader only: its producer's arrive + all bytes
+      mbar_init(empty_bar(s), 1);  // one tcgen05.commit per use, delivered to both CTAs
+    }
+    mbar_init(acc_full_bar, 1);
+    mbar_init(acc_empty_bar, 16);  // eight epilogue warps in each CTA (the leader's barrier is used)
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_a)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_b)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_sa)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_sb)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_c)) : "memory");
+  }
+  if (warp == 1) {  // the same warp in both CTAs: the allocation is collective over the pair
+    asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();  // the peer's barriers exist before anything is signalled remotely
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------- TMA producer (both CTAs) -------------------------
+    if (lane < 4) {
+      const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
+      const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
+                                                                                         : cfg::kOffSf + 512u;
+      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : lane == 1 ? cfg::kBBytes : cfg::kSfBytes;
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        // this CTA's 128 rows of A and of B (B rows may lie past N on a ragged tile: zero fill);
+        // its own A scales and the B scales of all 256 columns
+        const int cy_fixed = lane == 0 ? (int)(tc.tm * 256 + rank * 128) : (int)(tc.tn * BN + rank * 128);
+        const int cz = lane == 2 ? (int)(tc.tm * 2 + rank) : lane == 3 ? (int)(tc.tn * 2) : 0;
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+            raise_abort(abort_flag, ST_PRODUCER_WAIT);
+            ok = false;
+          }
+          if (!__all_sync(0xFu, ok)) { ok = false; break; }
+          const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
+          if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
+          __syncwarp(0xFu);
+          const int cx = lane < 2 ? (int)(kc * BK) : 0;
+          const int cy = lane < 2 ? cy_fixed : (int)kc;
+          tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 1) {
+    // --------------------------- MMA issuer (leader) ---------------------------
+    if (lane == 0 && rank == 0) {
+      uint32_t stage = 0, phase = 0, acc_phase = 0;
+      bool ok = true;
+      for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+        if (!mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag)) {
+          raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+          break;
+        }
+        tc_fence_after();
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+            raise_abort(abort_flag, ST_MMA_WAIT_FULL);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+          const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
+          tc_cp_scales_pair(sf_tmem, scale_desc(sf_smem));
+          tc_cp_scales_pair(sf_tmem + 4, scale_desc(sf_smem + 512));
+          tc_cp_scales_pair(sf_tmem + 8, scale_desc(sf_smem + 1024));
+          const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
+          const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
+#pragma unroll
+          for (uint32_t k = 0; k < BK / kMmaK; ++k) {
+            const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
+            tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4,
+                        (kc | k) != 0 ? 1u : 0u);
+          }
+          tc_commit_pair(empty_bar(stage));
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit_pair(acc_full_bar);
+        acc_phase ^= 1u;
+      }
+    }
+  } else {
+    // ---------------------------- epilogue (both CTAs) ----------------------------
+    const uint32_t quarter = warp & 3u;
+    const uint32_t half = (warp - 2u) >> 2;
+    constexpr uint32_t kHalf = BN / 2, kLoads = kHalf / 32;
+    uint32_t acc_phase = 0;
+    for (uint32_t t = pair; t < num_tiles; t += num_pairs) {
+      const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+      if (!mbar_wait(acc_full_bar, acc_phase, abort_flag)) {
+        if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + half * kHalf;
+      const uint32_t col0 = tc.tn * BN + half * kHalf;
+      const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;
+      uint32_t r[kLoads][32];
+#pragma unroll
+      for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
+      tc_wait_ld();
+      tc_fence_before();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
+      store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                         (int)col0, (int)(tc.tm * 256 + rank * 128 + quarter * 32), valid_cols, lane);
+      acc_phase ^= 1u;
+    }
+    if (lane == 0) bulk_wait_all();
+  }
+
+  // common exit: both CTAs of the pair leave together, then the pair's tensor memory is freed
+  tc_fence_before();
+  __syncthreads();
+  cluster_sync();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"((uint32_t)kTmemCols) : "memory");
   }
 }
@@ -400,6 +691,11 @@ EncodeTiledFn encode_fn(cudaError_t* err) {
   return fn;
 }
 
+EncodeTiledFn encode_fn_cached() {
+  cudaError_t e;
+  return encode_fn(&e);
+}
+
 int fmt_bits(int f) { return f == MX_E2M1 ? 4 : ((f == MX_E3M2 || f == MX_E2M3) ? 6 : 8); }
 
 // Format field of the instruction descriptor.
@@ -421,18 +717,51 @@ bool make_operand_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int f
   const CUtensorMapDataType dt = bits == 8 ? CU_TENSOR_MAP_DATA_TYPE_UINT8
                                  : bits == 6 ? CU_TENSOR_MAP_DATA_TYPE_16U6_ALIGN16B
                                              : CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN16B;
-  const cuuint64_t dims[2] = {K, rows};
-  const cuuint64_t strides[1] = {K * (uint64_t)bits / 8};
-  const cuuint32_t box[2] = {(cuuint32_t)BK, box_rows};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, dt, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+  const cuuint64_t pitch = K * (uint64_t)bits / 8;
+  const cuuint64_t dims[3] = {K, rows, 1};
+  const cuuint64_t strides[2] = {pitch, pitch * rows};
+  const cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor map over a swizzled scale tensor seen as [row groups of 128][K chunks][128 words]:
+// one 512-byte chunk per (row group, K chunk); the box takes `groups` consecutive row groups.
+bool make_scale_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
+                    uint32_t groups) {
+  const uint64_t k_chunks = K / BK;
+  const cuuint64_t dims[3] = {128, k_chunks, rows / 128};
+  const cuuint64_t strides[2] = {512, 512 * k_chunks};
+  const cuuint32_t box[3] = {128, 1, groups};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Tensor map of the FP32 output [M x N]: box = 16 columns x 32 rows in the 64-byte swizzle the
+// epilogue writes its staging chunks in.
+bool make_c_map(EncodeTiledFn fn, CUtensorMap* map, float* C, uint64_t M, uint64_t N) {
+  const cuuint64_t dims[2] = {N, M};
+  const cuuint64_t strides[1] = {N * 4};
+  const cuuint32_t box[2] = {kEpiChunkCols, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
 template <int BN>
 cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb,
                       uint32_t idesc_base) {
+  CUtensorMap mc, msa, msb;
+  EncodeTiledFn fn = encode_fn_cached();
+  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) ||
+      !make_scale_map(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1) ||
+      !make_scale_map(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, Cfg<BN>::kSfbChunks))
+    return cudaErrorInvalidValue;
   using cfg = Cfg<BN>;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -452,9 +781,38 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   const uint32_t tx_bytes = (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8) +
                             cfg::kSfBytes;
   mx_gemm_kernel<BN><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
-      ma, mb, a.sA, a.sB, a.C, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
-      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, (uint32_t)((uintptr_t)a.C % 32 == 0),
-      tx_bytes);
+      ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
+      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes);
+  return cudaGetLastError();
+}
+
+cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn, uint32_t idesc_base) {
+  using cfg = Cfg2;
+  CUtensorMap ma, mb, msa, msb, mc;
+  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) ||
+      !make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, 128) ||
+      !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, 128) ||
+      !make_scale_map(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1) ||
+      !make_scale_map(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, 2))
+    return cudaErrorInvalidValue;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(mx_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                             (int)cfg::kSmemBytes);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint32_t tiles = (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
+  const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
+  // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
+  const uint32_t tx_pair = 2u * (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 128 * BK * fmt_bits(a.fmtB) / 8 +
+                                           (int)cfg::kSfBytes);
+  const uint32_t idesc = idesc_base | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+  mx_gemm_pair_kernel<<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
+      ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair);
   return cudaGetLastError();
 }
 
@@ -472,6 +830,17 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   const int64_t tiles256 = (a.M / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
 #endif
+#ifndef MX_GEMM_NO_PAIR
+  // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
+#ifndef MX_GEMM_PAIR_MIN_TILES
+#define MX_GEMM_PAIR_MIN_TILES (a.sm_count / 2)
+#endif
+  if (a.M % 256 == 0 && (a.M / 256) * ((a.N + 255) / 256) >= MX_GEMM_PAIR_MIN_TILES) {
+    const uint32_t idesc2 = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23);
+    *cuda_err = launch_pair(a, fn, idesc2);
+    return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
+  }
+#endif
   CUtensorMap ma, mb;
   if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, BM) ||
       !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, (uint32_t)bn)) {
@@ -481,8 +850,7 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   // a_format [7,10), b_format [10,13), K-major A and B, scale format E8M0 (bit 23), M = 128
   const uint32_t idesc = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23) |
                          ((uint32_t)(BM >> 4) << 24);
-  *cuda_err = bn == 256 ? launch_bn<256>(a, ma, mb, idesc)
-              : bn == 192 ? launch_bn<192>(a, ma, mb, idesc) : launch_bn<128>(a, ma, mb, idesc);
+  *cuda_err = bn == 256 ? launch_bn<256>(a, ma, mb, idesc) : launch_bn<128>(a, ma, mb, idesc);
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
 }
 
@@ -501,3 +869,4 @@ int gemm_status(cudaStream_t stream, unsigned int* out, cudaError_t* cuda_err) {
 }
 
 }  // namespace mx
+

@@ -226,6 +226,37 @@ def _full_size_check(name, ea, sa, eb, sb, M, N, K, fa, fb, seed):
     print(name, "worst sampled |err|/S:", worst)
 
 
+@pytest.mark.parametrize("shape,fa,fb", [
+    ((4736, 8192, 256), 0, 0),    # M = 37 x 128: the one-CTA 128 x 256 kernel
+    ((4736, 8320, 384), 3, 4),    # ... with a ragged last tile (N = 65 x 128)
+    ((2048, 9600, 384), 0, 2),    # M % 256 == 0: the two-CTA 256 x 256 kernel, ragged N
+    ((256, 256 * 74, 128), 1, 0),  # two-CTA kernel, one tile per pair, a single K stage
+])
+def test_kernel_variants_whole_matrix(shape, fa, fb):
+    """Shapes that select each GEMM kernel variant; the whole output is checked against an
+    FP64 library product of the oracle-dequantized operands and sampled against the oracle."""
+    M, N, K = shape
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.02
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    g_out = Guarded(M * N * 4)
+    C = g_out.view.view(torch.float32).view(M, N)
+    mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy() for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    bad = int(((C.double() - da @ db.T).abs() > TOL * (da.abs() @ db.abs().T)).sum())
+    assert bad == 0, f"{shape}: {bad} outputs beyond the bound"
+    rng = np.random.default_rng(M)
+    ms, ns = rng.integers(0, M, 2000), rng.integers(0, N, 2000)
+    c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    _check_bound(C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].cpu().numpy(), c64, s, shape)
+
+
 def test_config3_full_size():
     d = inputs.config3("cuda")
     X, W = d["X"], d["W"]
