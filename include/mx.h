@@ -212,6 +212,36 @@ int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_
                      mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts,
                      void* workspace_dev, size_t workspace_bytes);
 
+/*
+ * mx_quantize_host_static -- mx_quantize_host without a caller-supplied workspace.
+ * (The paper has no counterpart: this is a deployment convenience of this library.)
+ *
+ * Some callers of mx_quantize_host cannot provide its device workspace because they are not
+ * allowed to allocate device memory at all: a plug-in inside a host application that has
+ * handed every free byte of the GPU to its own memory pool and forbids further allocations,
+ * or a latency-critical loop that must never enter cudaMalloc (which may synchronise the
+ * device).  For them the staging area lives in a fixed array inside the library,
+ * MX_STATIC_SCRATCH_BYTES long, which every GPU that loads the library holds from module
+ * load until the process exits.  This call allocates nothing: no cudaMalloc, no cudaFree,
+ * no allocating library routine.
+ *
+ * Arguments, results and errors are those of mx_quantize_host (host input, host outputs, the
+ * stream is synchronised before returning).  A request whose staging need
+ * (mx_quantize_host_workspace_bytes) exceeds MX_STATIC_SCRATCH_BYTES is rejected with
+ * MX_ERR_WORKSPACE and nothing is launched.
+ *
+ * The first call on a device looks up the device address of the array (once per device, with
+ * that device current); make that first call outside any stream capture.  All calls on a
+ * device share the one array and it keeps the bytes of the previous call: the routine
+ * rewrites every byte it later reads back (including the padding of the swizzled scale
+ * tensor), but two calls that overlap on the GPU -- from two threads or two streams -- race
+ * on it and must be serialised by the caller.
+ */
+#define MX_STATIC_SCRATCH_BYTES (16u * 1024u * 1024u)
+int mx_quantize_host_static(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                            const int64_t* shape, int ndim, int axis,
+                            mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts);
+
 size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis,
                                           mx_fmt_t fmt, const mx_opts_t* opts);
 int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void* out_host,

@@ -31,7 +31,7 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_dequantize", "mx_gemm",
-    "mx_quantize_host_workspace_bytes", "mx_quantize_host",
+    "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
 ]
@@ -76,6 +76,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
     lib.mx_quantize_host.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op, vp, sz]
+    lib.mx_quantize_host_static.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op]
     lib.mx_dequantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_dequantize_host_workspace_bytes.restype = sz
     lib.mx_dequantize_host.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op, vp, sz]
@@ -201,6 +202,22 @@ def mx_quantize_host(x: torch.Tensor, elems: torch.Tensor, scales: torch.Tensor,
                                  _shape_arr(shape), len(shape), axis % len(shape), fmt, rounding,
                                  ctypes.byref(o), workspace.data_ptr(), workspace.numel()),
            "mx_quantize_host")
+
+
+MX_STATIC_SCRATCH_BYTES = 16 * 1024 * 1024
+
+
+def mx_quantize_host_static(x: torch.Tensor, elems: torch.Tensor, scales: torch.Tensor, axis: int,
+                            fmt: int, rounding: int, layout: int = MX_SCALES_SWIZZLED) -> None:
+    """mx_quantize_host for callers that may not allocate device memory: the staging area is a
+    fixed array inside the library (MX_STATIC_SCRATCH_BYTES), so no workspace is passed.  Calls
+    on one device share that array and must not overlap."""
+    assert not x.is_cuda and not elems.is_cuda and not scales.is_cuda
+    shape = list(x.shape)
+    o = _opts(_dtype_code(x.dtype), layout)
+    _check(_lib.mx_quantize_host_static(x.data_ptr(), elems.data_ptr(), scales.data_ptr(),
+                                        _shape_arr(shape), len(shape), axis % len(shape), fmt,
+                                        rounding, ctypes.byref(o)), "mx_quantize_host_static")
 
 
 def mx_dequantize_host_workspace_bytes(shape, fmt, dtype, layout=MX_SCALES_SWIZZLED) -> int:

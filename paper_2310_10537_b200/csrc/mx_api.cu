@@ -231,6 +231,56 @@ int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 
+// ---------------------------------------------------------------------------
+// Host-buffer quantize for callers that may not allocate device memory
+// ---------------------------------------------------------------------------
+
+}  // extern "C"
+
+namespace {
+
+// Staging area of mx_quantize_host_static.  In host code this name is only a handle for the
+// symbol, not a device address: the address is looked up once per device below.
+static __device__ __align__(256) unsigned char g_static_scratch[MX_STATIC_SCRATCH_BYTES];
+
+// Device address of g_static_scratch on the current device (cached per device ordinal).
+void* static_scratch_address(cudaError_t* err) {
+  static void* cache[64] = {nullptr};
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess) return nullptr;
+  if (dev >= 0 && dev < 64 && cache[dev]) return cache[dev];
+  void* p = nullptr;
+  *err = cudaGetSymbolAddress(&p, g_static_scratch);
+  if (*err != cudaSuccess) return nullptr;
+  if (dev >= 0 && dev < 64) cache[dev] = p;
+  return p;
+}
+
+}  // namespace
+
+extern "C" {
+
+int mx_quantize_host_static(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                            const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                            mx_round_t rounding, const mx_opts_t* opts) {
+  // size check first: an oversized request is refused before anything touches the device
+  Opts o;
+  View v;
+  if (!shape) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts) > MX_STATIC_SCRATCH_BYTES)
+    return MX_ERR_WORKSPACE;
+  cudaError_t e;
+  void* scratch = static_scratch_address(&e);
+  if (!scratch) return fail_cuda(e);
+  // mx_quantize_host copies the input in, zeroes the scale padding where there is any, runs
+  // the kernel and copies exactly the produced bytes out: nothing stale is ever read back.
+  return mx_quantize_host(in_host, elems_out_host, scales_out_host, shape, ndim, axis, fmt, rounding,
+                          opts, scratch, MX_STATIC_SCRATCH_BYTES);
+}
+
 size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
                                           const mx_opts_t* opts) {
   return mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts);
