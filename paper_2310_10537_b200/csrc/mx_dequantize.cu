@@ -92,6 +92,16 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
     const uint32_t sb = __ldg(scales + off);
     // X = 2^(sb - 127); sb = 0 is the FP32 subnormal 2^-127, sb = 255 is NaN
     const float X = __uint_as_float(sb == 0 ? 0x00400000u : (sb == 255 ? 0x7FC00000u : sb << 23));
+    // Special values are rare and are decided once per thread: a NaN scale makes the whole
+    // block NaN; only the FP8 formats have element codes for NaN (and E5M2 for Inf).
+    bool special = sb == 255;
+    if (FMT == MX_E4M3) {  // 0x7F / 0xFF: low seven bits all ones
+#pragma unroll
+      for (int i = 0; i < kWords; ++i) special |= (((w[i] & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u) != 0;
+    } else if (FMT == MX_E5M2) {  // exponent field 31
+#pragma unroll
+      for (int i = 0; i < kWords; ++i) special |= (((w[i] & 0x7C7C7C7Cu) + 0x04040404u) & 0x80808080u) != 0;
+    }
     uint32_t r[kElems];
 #pragma unroll
     for (int i = 0; i < kElems / 2; ++i) {
@@ -109,10 +119,15 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
       }
       float a, b;
       decode_pair<FMT>(pair, a, b);
-      a *= X;  // exact unless it overflows to Inf
-      b *= X;
-      r[2 * i] = (a != a) ? 0x7FC00000u : __float_as_uint(a);
-      r[2 * i + 1] = (b != b) ? 0x7FC00000u : __float_as_uint(b);
+      r[2 * i] = __float_as_uint(a * X);  // exact unless it overflows to Inf
+      r[2 * i + 1] = __float_as_uint(b * X);
+    }
+    if (special) {  // canonical quiet NaN wherever the value is NaN
+#pragma unroll
+      for (int i = 0; i < kElems; ++i) {
+        const float f = __uint_as_float(r[i]);
+        if (f != f) r[i] = 0x7FC00000u;
+      }
     }
     char* dst = reinterpret_cast<char*>(out) + (size_t)unit * 64;
     uint32_t o[16];
@@ -125,9 +140,15 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
         const float lo = __uint_as_float(r[(2 * i) % kElems]), hi = __uint_as_float(r[(2 * i + 1) % kElems]);
         uint32_t pk;
         asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));  // round to nearest even
-        if (lo != lo) pk = (pk & 0xFFFF0000u) | 0x7FC0u;
-        if (hi != hi) pk = (pk & 0x0000FFFFu) | 0x7FC00000u;
         o[i] = pk;
+      }
+      if (special) {  // the packed conversion returns 0x7FFF for NaN: make it the canonical 0x7FC0
+#pragma unroll
+        for (int i = 0; i < 16; ++i) {
+          const float lo = __uint_as_float(r[(2 * i) % kElems]), hi = __uint_as_float(r[(2 * i + 1) % kElems]);
+          if (lo != lo) o[i] = (o[i] & 0xFFFF0000u) | 0x7FC0u;
+          if (hi != hi) o[i] = (o[i] & 0x0000FFFFu) | 0x7FC00000u;
+        }
       }
     }
     if (ALIGNED32) {

@@ -70,6 +70,25 @@ __device__ __forceinline__ float absmax_nan(float a, float b) {
   return d;
 }
 
+// The same on two packed BF16 values per operand (the result's halves carry arbitrary signs).
+__device__ __forceinline__ uint32_t absmax_nan_bf16x2(uint32_t a, uint32_t b) {
+  uint32_t d;
+  asm("max.NaN.xorsign.abs.bf16x2 %0, %1, %2;" : "=r"(d) : "r"(a), "r"(b));
+  return d;
+}
+// A float whose magnitude bits are the larger magnitude of the two BF16 halves of m.
+__device__ __forceinline__ float bf16x2_halves_max(uint32_t m) {
+  const uint32_t lo = (m << 16) & 0x7FFF0000u, hi = m & 0x7FFF0000u;
+  return __uint_as_float(lo > hi ? lo : hi);  // magnitudes order like unsigned integers; NaN stays on top
+}
+
+// min(|x|, bound) with the sign of x (bound > 0): one instruction.
+__device__ __forceinline__ float clamp_abs(float x, float bound) {
+  float d;
+  asm("min.xorsign.abs.f32 %0, %1, %2;" : "=f"(d) : "f"(x), "f"(bound));
+  return d;
+}
+
 // Per-block scalars derived from the block maximum.
 struct BlockScale {
   uint32_t byte;  // E8M0 scale byte: 0xFF for a block with Inf/NaN
@@ -127,8 +146,8 @@ __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
   } else {  // INT8: value n/64, inputs already multiplied by 64; saturate at +-127
     // x + 1.5 * 2^23 rounds x to an integer (nearest even) in the low mantissa bits, as two's
     // complement for negative x: no float-to-int conversion needed.
-    const float a = fminf(fmaxf(lo, -127.0f), 127.0f) + 12582912.0f;
-    const float b = fminf(fmaxf(hi, -127.0f), 127.0f) + 12582912.0f;
+    const float a = clamp_abs(lo, 127.0f) + 12582912.0f;
+    const float b = clamp_abs(hi, 127.0f) + 12582912.0f;
     p = (uint16_t)((__float_as_uint(a) & 0xFFu) | ((__float_as_uint(b) & 0xFFu) << 8));
   }
   return p;

@@ -39,10 +39,9 @@ template <int DTYPE> struct LastAxis {
   static constexpr int kLanes = kBlock / kElems;             // lanes per MX block
 };
 
-template <int DTYPE, bool ALIGNED32>
-__device__ __forceinline__ void load_unit(const void* in, size_t unit,
-                                          float (&v)[LastAxis<DTYPE>::kElems]) {
-  uint32_t w[16];
+// Raw 64 bytes of a unit as sixteen 32-bit words.
+template <bool ALIGNED32>
+__device__ __forceinline__ void load_unit(const void* in, size_t unit, uint32_t (&w)[16]) {
   const char* p = reinterpret_cast<const char*>(in) + unit * 64;
   if (ALIGNED32) {
     uint32_t a[8], b[8];
@@ -57,15 +56,42 @@ __device__ __forceinline__ void load_unit(const void* in, size_t unit,
       w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
     }
   }
+}
+
+// max |V_i| over the unit as a balanced tree (short dependency chains), on packed BF16 pairs
+// where the input is BF16.
+template <int DTYPE>
+__device__ __forceinline__ float unit_amax(const uint32_t (&w)[16]) {
+  if constexpr (DTYPE == MX_BF16) {
+    uint32_t m[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m[i] = absmax_nan_bf16x2(w[2 * i], w[2 * i + 1]);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m[i] = absmax_nan_bf16x2(m[2 * i], m[2 * i + 1]);
+    m[0] = absmax_nan_bf16x2(absmax_nan_bf16x2(m[0], m[1]), absmax_nan_bf16x2(m[2], m[3]));
+    return bf16x2_halves_max(m[0]);
+  } else {
+    float m[8];
+#pragma unroll
+    for (int i = 0; i < 8; ++i) m[i] = absmax_nan(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
+#pragma unroll
+    for (int i = 0; i < 4; ++i) m[i] = absmax_nan(m[2 * i], m[2 * i + 1]);
+    return absmax_nan(absmax_nan(m[0], m[1]), absmax_nan(m[2], m[3]));
+  }
+}
+
+// Elements 8g .. 8g+7 of the unit as FP32 values.
+template <int DTYPE>
+__device__ __forceinline__ void unit_group(const uint32_t (&w)[16], int g, float (&x)[8]) {
   if (DTYPE == MX_BF16) {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) {
-      v[(2 * i) % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i] << 16);  // BF16 widens exactly
-      v[(2 * i + 1) % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i] & 0xFFFF0000u);
+    for (int i = 0; i < 4; ++i) {
+      x[2 * i] = __uint_as_float(w[4 * g + i] << 16);  // BF16 widens exactly
+      x[2 * i + 1] = __uint_as_float(w[4 * g + i] & 0xFFFF0000u);
     }
   } else {
 #pragma unroll
-    for (int i = 0; i < 16; ++i) v[i % LastAxis<DTYPE>::kElems] = __uint_as_float(w[i]);
+    for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(w[(8 * g + i) % 16]);
   }
 }
 
@@ -81,26 +107,24 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t span = kThreads * U;
   for (uint32_t base = blockIdx.x * span; base < n_units; base += gridDim.x * span) {
-    float v[U][kElems];
+    uint32_t raw[U][16];
     bool ok[U];
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const uint32_t unit = base + u * kThreads + threadIdx.x;
       ok[u] = unit < n_units;  // groups of 4 blocks are in or out together: n_units * kLanes % 4 == 0 or tail
       if (ok[u]) {
-        load_unit<DTYPE, ALIGNED32>(in, unit, v[u]);
+        load_unit<ALIGNED32>(in, unit, raw[u]);
       } else {
 #pragma unroll
-        for (int i = 0; i < kElems; ++i) v[u][i] = 0.0f;
+        for (int i = 0; i < 16; ++i) raw[u][i] = 0u;
       }
     }
 #pragma unroll
     for (int u = 0; u < U; ++u) {
       const uint32_t unit = base + u * kThreads + threadIdx.x;
       // Line 1 of Algorithm 1: max |V_i| over the block
-      float amax = absmax_nan(v[u][0], v[u][1]);
-#pragma unroll
-      for (int i = 2; i < kElems; ++i) amax = absmax_nan(amax, v[u][i]);
+      float amax = unit_amax<DTYPE>(raw[u]);
       if (kLanes == 2) amax = absmax_nan(amax, __shfl_xor_sync(0xFFFFFFFFu, amax, 1));
       const BlockScale s = block_scale<FMT>(amax);
       // Lines 3-5: P_i = quantize(V_i / X)
@@ -108,8 +132,7 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
 #pragma unroll
       for (int g = 0; g < kElems / 8; ++g) {
         float x[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = v[u][8 * g + i];
+        unit_group<DTYPE>(raw[u], g, x);
         cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
       }
       uint8_t* dst = elems + (size_t)unit * kOutBytes;
@@ -199,18 +222,46 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
 // Strided axis
 // ---------------------------------------------------------------------------
 
-// Tensor viewed as [outer, L, inner], blocks along L.  A thread owns COLS
-// adjacent columns (inner positions) and walks KB_PER_THREAD consecutive blocks;
-// a warp therefore reads 32*COLS consecutive elements of each input row.
-// Output row = o * inner + column, block axis innermost.
+// Tensor viewed as [outer, L, inner], blocks along L.  A thread owns COLS adjacent
+// columns (inner positions) and walks kb_per_thread consecutive blocks; a warp therefore
+// reads 32*COLS consecutive elements of each input row.  The 32 rows of a block stay in
+// registers in their packed input form (8 bytes per row for the wide variants: four BF16
+// or two FP32 columns), so a block of every column is complete in one thread: no shared
+// memory, no shuffles.  Output row = o * inner + column, block axis innermost.
+#ifndef MX_QT_THREADS
+#define MX_QT_THREADS 128
+#endif
+constexpr int kStridedThreads = MX_QT_THREADS;
+
+template <int DTYPE, int COLS> struct StridedRow {
+  static constexpr int kBytes = COLS * (DTYPE == MX_BF16 ? 2 : 4);   // bytes loaded per row: 8, 4 or 2
+  static constexpr int kWords = kBytes >= 4 ? kBytes / 4 : 1;
+};
+
+// Element (row k, column c) of the packed rows as an FP32 value.
+template <int DTYPE, int COLS>
+__device__ __forceinline__ float strided_elem(const uint32_t (&raw)[kBlock][StridedRow<DTYPE, COLS>::kWords],
+                                              int k, int c) {
+  if (DTYPE == MX_BF16) {
+    const uint32_t w = raw[k][(c / 2) % StridedRow<DTYPE, COLS>::kWords];
+    return __uint_as_float((c & 1) ? (w & 0xFFFF0000u) : (w << 16));
+  }
+  return __uint_as_float(raw[k][c % StridedRow<DTYPE, COLS>::kWords]);
+}
+
+#ifndef MX_QT_MINB
+#define MX_QT_MINB 4
+#endif
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
-__global__ void __launch_bounds__(kThreads)
+__global__ void __launch_bounds__(kStridedThreads, MX_QT_MINB)
 quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
                         uint8_t* __restrict__ scales, uint32_t outer, uint32_t L,
                         uint32_t inner, uint32_t kb_per_thread) {
   constexpr int bits = FmtTraits<FMT>::bits;
+  constexpr int kWords = StridedRow<DTYPE, COLS>::kWords;
+  constexpr int kRowBytes = StridedRow<DTYPE, COLS>::kBytes;
   const uint32_t kblocks = L / kBlock;
-  const uint32_t col0 = (blockIdx.x * kThreads + threadIdx.x) * COLS;
+  const uint32_t col0 = (blockIdx.x * kStridedThreads + threadIdx.x) * COLS;
   if (col0 >= inner) return;  // no warp-level exchange in this kernel
   const uint32_t kb_begin = blockIdx.y * kb_per_thread;
   const uint32_t kb_end = min(kb_begin + kb_per_thread, kblocks);
@@ -220,42 +271,55 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
 
   for (uint32_t o = blockIdx.z; o < outer; o += gridDim.z)
   for (uint32_t kb = kb_begin; kb < kb_end; ++kb) {
-    const char* src = reinterpret_cast<const char*>(in) + ((size_t)o * L * inner + col0) * esz;
-    // 32 input rows x COLS columns, every load issued before the arithmetic
-    float v[COLS][kBlock];
-    const char* p = src + (size_t)kb * kBlock * row_pitch;
+    const char* p = reinterpret_cast<const char*>(in) + ((size_t)o * L * inner + col0) * esz +
+                    (size_t)kb * kBlock * row_pitch;
+    // 32 input rows, every load issued before the arithmetic
+    uint32_t raw[kBlock][kWords];
 #pragma unroll
     for (int k = 0; k < kBlock; ++k) {
       const char* q = p + (size_t)k * row_pitch;
-      if (DTYPE == MX_BF16) {
-        if (COLS == 4) {
-          const uint2 w = __ldg(reinterpret_cast<const uint2*>(q));
-          v[0][k] = __uint_as_float(w.x << 16); v[1 % COLS][k] = __uint_as_float(w.x & 0xFFFF0000u);
-          v[2 % COLS][k] = __uint_as_float(w.y << 16); v[3 % COLS][k] = __uint_as_float(w.y & 0xFFFF0000u);
-        } else if (COLS == 2) {
-          const uint32_t w = __ldg(reinterpret_cast<const uint32_t*>(q));
-          v[0][k] = __uint_as_float(w << 16); v[1 % COLS][k] = __uint_as_float(w & 0xFFFF0000u);
-        } else {
-          v[0][k] = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(q)) << 16);
-        }
+      if (kRowBytes == 8) {
+        const uint2 w = __ldg(reinterpret_cast<const uint2*>(q));
+        raw[k][0] = w.x; raw[k][1 % kWords] = w.y;
+      } else if (kRowBytes == 4) {
+        raw[k][0] = __ldg(reinterpret_cast<const uint32_t*>(q));
       } else {
-        if (COLS == 4) {
-          const float4 w = __ldg(reinterpret_cast<const float4*>(q));
-          v[0][k] = w.x; v[1 % COLS][k] = w.y; v[2 % COLS][k] = w.z; v[3 % COLS][k] = w.w;
-        } else if (COLS == 2) {
-          const float2 w = __ldg(reinterpret_cast<const float2*>(q));
-          v[0][k] = w.x; v[1 % COLS][k] = w.y;
-        } else {
-          v[0][k] = __ldg(reinterpret_cast<const float*>(q));
-        }
+        raw[k][0] = (uint32_t)__ldg(reinterpret_cast<const uint16_t*>(q));
+      }
+    }
+    // Line 1 of Algorithm 1 for every column: balanced trees over the 32 rows, on packed
+    // BF16 pairs where the input is BF16 (two columns per operation)
+    float amax[COLS];
+    if (DTYPE == MX_BF16) {
+#pragma unroll
+      for (int wi = 0; wi < kWords; ++wi) {
+        uint32_t m[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m[i] = absmax_nan_bf16x2(raw[2 * i][wi], raw[2 * i + 1][wi]);
+#pragma unroll
+        for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+          for (int i = 0; i < n; ++i) m[i] = absmax_nan_bf16x2(m[2 * i], m[2 * i + 1]);
+        amax[(2 * wi) % COLS] = __uint_as_float((m[0] << 16) & 0x7FFF0000u);
+        if (COLS > 1) amax[(2 * wi + 1) % COLS] = __uint_as_float(m[0] & 0x7FFF0000u);
+      }
+    } else {
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) {
+        float m[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i)
+          m[i] = absmax_nan(__uint_as_float(raw[2 * i][c % kWords]), __uint_as_float(raw[2 * i + 1][c % kWords]));
+#pragma unroll
+        for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+          for (int i = 0; i < n; ++i) m[i] = absmax_nan(m[2 * i], m[2 * i + 1]);
+        amax[c] = m[0];
       }
     }
 #pragma unroll
     for (int c = 0; c < COLS; ++c) {
-      float amax = absmax_nan(v[c][0], v[c][1]);
-#pragma unroll
-      for (int k = 2; k < kBlock; ++k) amax = absmax_nan(amax, v[c][k]);
-      const BlockScale s = block_scale<FMT>(amax);
+      const BlockScale s = block_scale<FMT>(amax[c]);
       const uint32_t row = o * inner + col0 + c;
       uint8_t* dst = elems + (size_t)row * out_row_bytes + (size_t)kb * (kBlock * bits / 8);
       uint32_t w[8];
@@ -263,7 +327,7 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
       for (int g = 0; g < 4; ++g) {
         float x[8];
 #pragma unroll
-        for (int i = 0; i < 8; ++i) x[i] = v[c][g * 8 + i];
+        for (int i = 0; i < 8; ++i) x[i] = strided_elem<DTYPE, COLS>(raw, g * 8 + i, c);
         cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
       }
       if (bits == 8) {
@@ -285,6 +349,150 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
       }
       scales[scale_offset<LAYOUT>(row, kb, kblocks)] = (uint8_t)s.byte;
     }
+  }
+}
+
+// Staged variant of the same kernel for the common case (kblocks % 4 == 0, output rows 16-byte
+// aligned): a thread still owns COLS columns, but it walks four consecutive blocks, parks their
+// codes in shared memory, and the warp then writes every output row's 128 / 96 / 64-byte run with
+// coalesced 16-byte stores.  Without this each lane writes its own row and the L2 sees two (8-bit),
+// three (6-bit) or one (4-bit) partial-sector request per block and row, which is what bounded the
+// direct version.  Each warp has a private staging area, so only __syncwarp is needed.
+constexpr int kStagedThreads = 64;
+
+template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
+__global__ void __launch_bounds__(kStagedThreads, 6)
+quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
+                               uint8_t* __restrict__ scales, uint32_t outer, uint32_t L,
+                               uint32_t inner) {
+  constexpr int bits = FmtTraits<FMT>::bits;
+  constexpr int kWords = StridedRow<DTYPE, COLS>::kWords;
+  constexpr uint32_t kBpb = kBlock * bits / 8;                     // bytes of one block's codes
+  constexpr uint32_t kSeg = 4 * kBpb;                              // four blocks: 128 / 96 / 64
+  constexpr uint32_t kPitch = kSeg + (bits == 6 ? 8 : 16);         // conflict-free lane stride
+  constexpr uint32_t kRows = 32 * COLS;                            // output rows per warp
+  extern __shared__ __align__(16) uint8_t staging[];
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  uint8_t* area = staging + warp * (kRows * kPitch);
+  const uint32_t kblocks = L / kBlock;
+  const uint32_t warp_col0 = (blockIdx.x * kStagedThreads + warp * 32) * COLS;  // first column of the warp
+  if (warp_col0 >= inner) return;                                  // whole warp out of range
+  const uint32_t col0 = warp_col0 + lane * COLS;
+  const bool lane_ok = col0 < inner;                               // inner % COLS == 0: all or none of its columns
+  const size_t esz = DTYPE == MX_BF16 ? 2 : 4;
+  const size_t row_pitch = (size_t)inner * esz;
+  const size_t out_row_bytes = (size_t)L * bits / 8;
+  const uint32_t rows_here = min(kRows, (inner - warp_col0));      // valid output rows of this warp
+
+  for (uint32_t o = blockIdx.z; o < outer; o += gridDim.z) {
+    const uint32_t kb0 = blockIdx.y * 4;
+    uint32_t scale_word[COLS];
+#pragma unroll
+    for (int c = 0; c < COLS; ++c) scale_word[c] = 0;
+#pragma unroll 1
+    for (uint32_t j = 0; j < 4; ++j) {
+      const uint32_t kb = kb0 + j;
+      uint32_t raw[kBlock][kWords];
+      if (lane_ok) {
+        const char* p = reinterpret_cast<const char*>(in) + ((size_t)o * L * inner + col0) * esz +
+                        (size_t)kb * kBlock * row_pitch;
+#pragma unroll
+        for (int k = 0; k < kBlock; ++k) {
+          const uint2 w = __ldg(reinterpret_cast<const uint2*>(p + (size_t)k * row_pitch));
+          raw[k][0] = w.x; raw[k][1 % kWords] = w.y;
+        }
+      } else {
+#pragma unroll
+        for (int k = 0; k < kBlock; ++k) { raw[k][0] = 0; raw[k][1 % kWords] = 0; }
+      }
+      float amax[COLS];
+      if (DTYPE == MX_BF16) {
+#pragma unroll
+        for (int wi = 0; wi < kWords; ++wi) {
+          uint32_t m[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i) m[i] = absmax_nan_bf16x2(raw[2 * i][wi], raw[2 * i + 1][wi]);
+#pragma unroll
+          for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+            for (int i = 0; i < n; ++i) m[i] = absmax_nan_bf16x2(m[2 * i], m[2 * i + 1]);
+          amax[(2 * wi) % COLS] = __uint_as_float((m[0] << 16) & 0x7FFF0000u);
+          amax[(2 * wi + 1) % COLS] = __uint_as_float(m[0] & 0x7FFF0000u);
+        }
+      } else {
+#pragma unroll
+        for (int c = 0; c < COLS; ++c) {
+          float m[16];
+#pragma unroll
+          for (int i = 0; i < 16; ++i)
+            m[i] = absmax_nan(__uint_as_float(raw[2 * i][c % kWords]), __uint_as_float(raw[2 * i + 1][c % kWords]));
+#pragma unroll
+          for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+            for (int i = 0; i < n; ++i) m[i] = absmax_nan(m[2 * i], m[2 * i + 1]);
+          amax[c] = m[0];
+        }
+      }
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) {
+        const BlockScale s = block_scale<FMT>(amax[c]);
+        scale_word[c] |= s.byte << (8 * j);
+        uint32_t w[8];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = strided_elem<DTYPE, COLS>(raw, g * 8 + i, c);
+          cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
+        }
+        // staging row of (lane, c) is c * 32 + lane: consecutive lanes are one pitch apart
+        uint8_t* dst = area + (c * 32 + lane) * kPitch + j * kBpb;
+        if (bits == 8) {
+          reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        } else if (bits == 4) {
+          reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[2], w[4], w[6]);
+        } else {
+          const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
+          const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
+          const uint64_t g2 = (uint64_t)w[4] | ((uint64_t)w[5] << 32);
+          const uint64_t g3 = (uint64_t)w[6] | ((uint64_t)w[7] << 32);
+          const uint64_t q0 = g0 | (g1 << 48), q1 = (g1 >> 16) | (g2 << 32), q2 = (g2 >> 32) | (g3 << 16);
+          uint2* d2 = reinterpret_cast<uint2*>(dst);  // 8-byte aligned: pitch and 24 j are multiples of 8
+          d2[0] = make_uint2((uint32_t)q0, (uint32_t)(q0 >> 32));
+          d2[1] = make_uint2((uint32_t)q1, (uint32_t)(q1 >> 32));
+          d2[2] = make_uint2((uint32_t)q2, (uint32_t)(q2 >> 32));
+        }
+      }
+    }
+    if (lane_ok) {
+#pragma unroll
+      for (int c = 0; c < COLS; ++c) {  // four scale bytes of a row are one aligned word in both layouts
+        const uint32_t row = o * inner + col0 + c;
+        *reinterpret_cast<uint32_t*>(scales + scale_offset<LAYOUT>(row, kb0, kblocks)) = scale_word[c];
+      }
+    }
+    __syncwarp();
+    // write-out: 16-byte chunks, consecutive lanes on consecutive chunks of one output row
+    constexpr uint32_t kChunks = kSeg / 16;
+    for (uint32_t i = lane; i < kRows * kChunks; i += 32) {
+      const uint32_t r = i / kChunks, ch = i - r * kChunks;      // staging row, chunk in the row
+      const uint32_t c = r >> 5, owner = r & 31;                  // column of the owning lane
+      const uint32_t col = owner * COLS + c;                      // column offset inside the warp
+      if (col < rows_here) {
+        const uint8_t* src = area + r * kPitch + ch * 16;
+        uint4 v;
+        if (bits == 6) {
+          const uint2 a = reinterpret_cast<const uint2*>(src)[0], b = reinterpret_cast<const uint2*>(src)[1];
+          v = make_uint4(a.x, a.y, b.x, b.y);
+        } else {
+          v = *reinterpret_cast<const uint4*>(src);
+        }
+        uint8_t* g = elems + (size_t)(o * inner + warp_col0 + col) * out_row_bytes + (size_t)kb0 * kBpb + ch * 16;
+        *reinterpret_cast<uint4*>(g) = v;
+      }
+    }
+    __syncwarp();
   }
 }
 
@@ -337,10 +545,16 @@ template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
 static cudaError_t launch_strided_cols(const QuantizeArgs& a) {
   const uint32_t kblocks = (uint32_t)(a.L / kBlock);
   const uint32_t threads_x = (uint32_t)((a.inner + COLS - 1) / COLS);
-  const uint32_t kb_per_thread = kblocks < 4 ? kblocks : 4;
-  dim3 grid((threads_x + kThreads - 1) / kThreads, (kblocks + kb_per_thread - 1) / kb_per_thread,
-            (uint32_t)(a.outer < 65535 ? a.outer : 65535));
-  quantize_strided_kernel<FMT, ROUND, DTYPE, LAYOUT, COLS><<<grid, kThreads, 0, a.stream>>>(
+  const uint32_t grid_x = (threads_x + kStridedThreads - 1) / kStridedThreads;
+  // consecutive blocks of a column are written by the same thread (their codes are adjacent in
+  // the output row); fewer per thread when the grid would otherwise not fill the machine
+  uint32_t kb_per_thread = kblocks < 4 ? kblocks : 4;
+  const uint64_t outer_eff = a.outer < 65535 ? (uint64_t)a.outer : 65535;
+  while (kb_per_thread > 1 &&
+         (uint64_t)grid_x * ((kblocks + kb_per_thread - 1) / kb_per_thread) * outer_eff < (uint64_t)a.sm_count * 16)
+    kb_per_thread >>= 1;
+  dim3 grid(grid_x, (kblocks + kb_per_thread - 1) / kb_per_thread, (uint32_t)outer_eff);
+  quantize_strided_kernel<FMT, ROUND, DTYPE, LAYOUT, COLS><<<grid, kStridedThreads, 0, a.stream>>>(
       a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner, kb_per_thread);
   return cudaGetLastError();
 }
@@ -348,9 +562,30 @@ static cudaError_t launch_strided_cols(const QuantizeArgs& a) {
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
 static cudaError_t launch_strided(const QuantizeArgs& a) {
   // widest column group whose loads stay aligned: 8 bytes per row and thread
-  const int wide = DTYPE == MX_BF16 ? 4 : 2;
-  if (a.inner % wide == 0 && (uintptr_t)a.in % 8 == 0)
-    return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, (DTYPE == MX_BF16 ? 4 : 2)>(a);
+  constexpr int kWide = DTYPE == MX_BF16 ? 4 : 2;
+  constexpr int bits = FmtTraits<FMT>::bits;
+  const uint32_t kblocks = (uint32_t)(a.L / kBlock);
+  const bool wide = a.inner % kWide == 0 && (uintptr_t)a.in % 8 == 0;
+  // 6- and 4-bit codes go through the staged kernel (their per-lane stores would be partial
+  // sectors); 8-bit codes are whole 32-byte sectors per lane already and are faster direct
+  const bool staged = bits != 8 && wide && kblocks % 4 == 0 && (a.L * bits / 8) % 16 == 0 && (uintptr_t)a.elems % 16 == 0 &&
+                      (uintptr_t)a.scales % 4 == 0;
+  if (staged) {
+    constexpr uint32_t kPitch = 4 * kBlock * bits / 8 + (bits == 6 ? 8 : 16);
+    constexpr uint32_t smem = (kStagedThreads / 32) * 32 * kWide * kPitch;
+    static_assert(smem <= 48 * 1024, "staging fits the default shared-memory limit");
+    const uint32_t threads_x = (uint32_t)(a.inner / kWide);
+    dim3 grid((threads_x + kStagedThreads - 1) / kStagedThreads, kblocks / 4,
+              (uint32_t)(a.outer < 65535 ? a.outer : 65535));
+    quantize_strided_staged_kernel<FMT, ROUND, DTYPE, LAYOUT, kWide><<<grid, kStagedThreads, smem, a.stream>>>(
+        a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner);
+    return cudaGetLastError();
+  }
+#ifdef MX_QT_BF16_COLS
+  if (DTYPE == MX_BF16 && a.inner % MX_QT_BF16_COLS == 0 && (uintptr_t)a.in % 4 == 0)
+    return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, (DTYPE == MX_BF16 ? MX_QT_BF16_COLS : kWide)>(a);
+#endif
+  if (wide) return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, kWide>(a);
   return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, 1>(a);
 }
 
