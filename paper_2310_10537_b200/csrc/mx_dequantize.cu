@@ -39,6 +39,43 @@ __device__ __forceinline__ void decode_pair(uint32_t pair, float& a, float& b) {
   b = f.y;
 }
 
+
+// ---- conversion-free decode -----------------------------------------------------
+// Element code e of the thread's packed words, moved to the top of a 32-bit word (sign at bit 31).
+template <int BITS, int KWORDS>
+__device__ __forceinline__ uint32_t code_at_top(const uint32_t (&w)[KWORDS], int e) {
+  const int pos = BITS * e, wi = pos / 32, off = pos % 32;
+  if (off + BITS <= 32) return off + BITS == 32 ? w[wi] : w[wi] << (32 - BITS - off);
+  return __funnelshift_r(w[wi], w[(wi + 1) % KWORDS], off) << (32 - BITS);  // 6-bit code across two words
+}
+
+// Value of the code whose bits sit at the top of t, times fix = 2^(127 - bias) ... returned
+// WITHOUT that factor: the caller multiplies by fix and by the block scale (both exact).
+// The magnitude bits are dropped into an FP32 exponent/mantissa field: for normal codes that is
+// the value / 2^(127 - bias), and for the format's subnormal codes it is an FP32 subnormal with
+// the same meaning, which the multiply then normalises -- no special cases.  NaN / Inf codes of
+// the FP8 formats are NOT handled here (the caller tests for them once per thread).
+template <int FMT>
+__device__ __forceinline__ float raw_value(uint32_t t) {
+  if (FMT == MX_INT8) {
+    const int n = (int)t >> 24;                                         // two's complement byte
+    return __uint_as_float(0x4B400000u + (uint32_t)n) - 12582912.0f;    // exact int -> float
+  }
+  constexpr int W = FmtTraits<FMT>::bits;
+  constexpr int MSHIFT = (FMT == MX_E4M3 || FMT == MX_E2M3) ? 20 : (FMT == MX_E2M1 ? 22 : 21);
+  constexpr uint32_t MASK = ((1u << (W - 1)) - 1u) << MSHIFT;
+  constexpr int SH = (32 - W) - MSHIFT;
+  return __uint_as_float((t & 0x80000000u) | ((t >> SH) & MASK));
+}
+template <int FMT>
+__device__ __forceinline__ float bias_fix() {  // 2^(127 - bias); INT8: 2^-6
+  return FMT == MX_E4M3 ? 1.329227995784916e36f      // 2^120
+       : FMT == MX_E5M2 ? 5.192296858534828e33f      // 2^112
+       : FMT == MX_E3M2 ? 2.1267647932558654e37f     // 2^124
+       : FMT == MX_INT8 ? 0.015625f
+                        : 8.507059173023462e37f;     // 2^126 (E2M3, E2M1)
+}
+
 // A thread produces 64 bytes of output: a whole block as BF16 (32 elements) or half
 // a block as FP32 (16 elements), written with two 256-bit stores.
 template <int FMT, int DTYPE, int LAYOUT, bool ALIGNED32>
@@ -92,9 +129,10 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
     const uint32_t sb = __ldg(scales + off);
     // X = 2^(sb - 127); sb = 0 is the FP32 subnormal 2^-127, sb = 255 is NaN
     const float X = __uint_as_float(sb == 0 ? 0x00400000u : (sb == 255 ? 0x7FC00000u : sb << 23));
-    // Special values are rare and are decided once per thread: a NaN scale makes the whole
-    // block NaN; only the FP8 formats have element codes for NaN (and E5M2 for Inf).
-    bool special = sb == 255;
+    // Special cases are rare and decided once per thread: a NaN scale, element codes for NaN / Inf
+    // (FP8 formats only), and scales so small that results can be FP32 subnormals (which BF16
+    // output would have to round).  Everything else takes the conversion-free path below.
+    bool special = sb == 255 || sb < 24;
     if (FMT == MX_E4M3) {  // 0x7F / 0xFF: low seven bits all ones
 #pragma unroll
       for (int i = 0; i < kWords; ++i) special |= (((w[i] & 0x7F7F7F7Fu) + 0x01010101u) & 0x80808080u) != 0;
@@ -102,52 +140,57 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
 #pragma unroll
       for (int i = 0; i < kWords; ++i) special |= (((w[i] & 0x7C7C7C7Cu) + 0x04040404u) & 0x80808080u) != 0;
     }
-    uint32_t r[kElems];
-#pragma unroll
-    for (int i = 0; i < kElems / 2; ++i) {
-      uint32_t pair;  // code(2i) | code(2i+1) << 8   (4-bit: both in the low byte)
-      if (bits == 8) {
-        pair = (w[i / 2] >> (16 * (i & 1))) & 0xFFFFu;
-      } else if (bits == 4) {
-        pair = (w[i / 4] >> (8 * (i & 3))) & 0xFFu;
-      } else {
-        const int bit = 12 * i;  // two 6-bit codes at bit offset 12 i of the stream
-        uint32_t q = w[bit / 32] >> (bit % 32);
-        if (bit % 32 > 20) q |= w[(bit / 32 + 1) % kWords] << (32 - bit % 32);
-        q &= 0xFFFu;
-        pair = (q & 0x3Fu) | ((q & 0xFC0u) << 2);
-      }
-      float a, b;
-      decode_pair<FMT>(pair, a, b);
-      r[2 * i] = __float_as_uint(a * X);  // exact unless it overflows to Inf
-      r[2 * i + 1] = __float_as_uint(b * X);
-    }
-    if (special) {  // canonical quiet NaN wherever the value is NaN
-#pragma unroll
-      for (int i = 0; i < kElems; ++i) {
-        const float f = __uint_as_float(r[i]);
-        if (f != f) r[i] = 0x7FC00000u;
-      }
-    }
     char* dst = reinterpret_cast<char*>(out) + (size_t)unit * 64;
     uint32_t o[16];
-    if (DTYPE == MX_F32) {
+    if (!special) {
+      const float fix = bias_fix<FMT>();
+      uint32_t r[kElems];
 #pragma unroll
-      for (int i = 0; i < 16; ++i) o[i] = r[i % kElems];
-    } else {
+      for (int e = 0; e < kElems; ++e)
+        r[e] = __float_as_uint(raw_value<FMT>(code_at_top<bits, kWords>(w, e)) * fix * X);  // both products exact
+      if (DTYPE == MX_F32) {
 #pragma unroll
-      for (int i = 0; i < 16; ++i) {
-        const float lo = __uint_as_float(r[(2 * i) % kElems]), hi = __uint_as_float(r[(2 * i + 1) % kElems]);
-        uint32_t pk;
-        asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));  // round to nearest even
-        o[i] = pk;
+        for (int i = 0; i < 16; ++i) o[i] = r[i % kElems];
+      } else {
+        // at most 7 significant bits and no FP32 subnormals here: the upper half IS the BF16 value
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o[i] = __byte_perm(r[(2 * i) % kElems], r[(2 * i + 1) % kElems], 0x7632);
       }
-      if (special) {  // the packed conversion returns 0x7FFF for NaN: make it the canonical 0x7FC0
+    } else {
+      uint32_t r[kElems];
+#pragma unroll
+      for (int i = 0; i < kElems / 2; ++i) {
+        uint32_t pair;  // code(2i) | code(2i+1) << 8   (4-bit: both in the low byte)
+        if (bits == 8) {
+          pair = (w[i / 2] >> (16 * (i & 1))) & 0xFFFFu;
+        } else if (bits == 4) {
+          pair = (w[i / 4] >> (8 * (i & 3))) & 0xFFu;
+        } else {
+          const int bit = 12 * i;  // two 6-bit codes at bit offset 12 i of the stream
+          uint32_t q = w[bit / 32] >> (bit % 32);
+          if (bit % 32 > 20) q |= w[(bit / 32 + 1) % kWords] << (32 - bit % 32);
+          q &= 0xFFFu;
+          pair = (q & 0x3Fu) | ((q & 0xFC0u) << 2);
+        }
+        float a, b;
+        decode_pair<FMT>(pair, a, b);
+        a *= X;  // exact unless it overflows to Inf
+        b *= X;
+        r[2 * i] = (a != a) ? 0x7FC00000u : __float_as_uint(a);  // canonical quiet NaN
+        r[2 * i + 1] = (b != b) ? 0x7FC00000u : __float_as_uint(b);
+      }
+      if (DTYPE == MX_F32) {
+#pragma unroll
+        for (int i = 0; i < 16; ++i) o[i] = r[i % kElems];
+      } else {
 #pragma unroll
         for (int i = 0; i < 16; ++i) {
           const float lo = __uint_as_float(r[(2 * i) % kElems]), hi = __uint_as_float(r[(2 * i + 1) % kElems]);
-          if (lo != lo) o[i] = (o[i] & 0xFFFF0000u) | 0x7FC0u;
-          if (hi != hi) o[i] = (o[i] & 0x0000FFFFu) | 0x7FC00000u;
+          uint32_t pk;
+          asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(hi), "f"(lo));  // round to nearest even
+          if (lo != lo) pk = (pk & 0xFFFF0000u) | 0x7FC0u;   // the packed conversion gives 0x7FFF for NaN
+          if (hi != hi) pk = (pk & 0x0000FFFFu) | 0x7FC00000u;
+          o[i] = pk;
         }
       }
     }
