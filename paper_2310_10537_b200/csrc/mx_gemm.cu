@@ -448,17 +448,25 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // fetched by both).
 // ============================================================================
 
+// F4 = both operands FP4 E2M1: kind::mxf4 takes them densely packed (two codes per byte, K = 64 per
+// MMA, two MX blocks and therefore two scales per row and instruction: scale_vec::2X), which doubles
+// the MACs per operand byte and per tensor-core cycle.  A stage then holds 256 K-elements.
+template <bool F4>
 struct Cfg2 {
   static constexpr int BN = 256;
 #ifndef MX_PAIR_STAGES
 #define MX_PAIR_STAGES 6
 #endif
-  static constexpr int kStages = MX_PAIR_STAGES;
-  static constexpr int kSfCols = 12;          // 4 (A) + 8 (B, all 256 rows) per stage
-  static constexpr int kSfCol0 = BN;          // single accumulator stage
-  static constexpr uint32_t kABytes = 128 * BK;   // this CTA's 128 rows of A
-  static constexpr uint32_t kBBytes = 128 * BK;   // this CTA's 128 rows of B
-  static constexpr uint32_t kSfBytes = 512 + 1024;
+  static constexpr int kStages = F4 ? MX_PAIR_STAGES - 1 : MX_PAIR_STAGES;
+  static constexpr int kBKe = F4 ? 256 : 128;           // K elements per stage (128-byte operand rows)
+  static constexpr int kKChunks = kBKe / 128;           // 512-byte scale chunks (4 MX blocks) along K per stage
+  static constexpr int kSfColsA = 4 * kKChunks;         // TMEM columns: this CTA's 128 rows of A
+  static constexpr int kSfCols = kSfColsA + 8 * kKChunks;  // ... plus all 256 rows of B
+  static constexpr int kSfCol0 = BN;                    // single accumulator stage
+  static constexpr uint32_t kABytes = 128 * 128;        // this CTA's 128 rows of A, 128 bytes each
+  static constexpr uint32_t kBBytes = 128 * 128;        // this CTA's 128 rows of B
+  static constexpr uint32_t kSfABytes = 512 * kKChunks;
+  static constexpr uint32_t kSfBytes = kSfABytes + 1024 * kKChunks;
   static constexpr uint32_t kOffA = 0;
   static constexpr uint32_t kOffB = kOffA + kStages * kABytes;
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;
@@ -497,6 +505,17 @@ __device__ __forceinline__ void tc_mma_pair(uint32_t d_tmem, uint64_t adesc, uin
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
         "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void tc_mma_pair_f4(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                               uint32_t idesc, uint32_t sfa_tmem, uint32_t sfb_tmem,
+                                               uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %6, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::mxf4.block_scale.scale_vec::2X [%0], %1, %2, %3, [%4], [%5], p;\n\t"
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
+        "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
 }
@@ -505,13 +524,15 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
+template <bool F4>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
                     uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair) {
-  using cfg = Cfg2;
+  using cfg = Cfg2<F4>;
   constexpr int BN = cfg::BN;
+  constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -529,7 +550,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
-  const uint32_t k_chunks = K / BK;
+  const uint32_t k_chunks = K / BKe;
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
@@ -563,7 +584,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     if (lane < 4) {
       const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
       const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
-                                                                                         : cfg::kOffSf + 512u;
+                                                                                         : cfg::kOffSf + cfg::kSfABytes;
       const uint32_t dst_stride = lane == 0 ? cfg::kABytes : lane == 1 ? cfg::kBBytes : cfg::kSfBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
@@ -582,8 +603,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
           __syncwarp(0xFu);
-          const int cx = lane < 2 ? (int)(kc * BK) : 0;
-          const int cy = lane < 2 ? cy_fixed : (int)kc;
+          const int cx = lane < 2 ? (int)(kc * BKe) : 0;
+          const int cy = lane < 2 ? cy_fixed : (int)(kc * cfg::kKChunks);
           tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -613,16 +634,31 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           tc_fence_after();
           const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          tc_cp_scales_pair(sf_tmem, scale_desc(sf_smem));
-          tc_cp_scales_pair(sf_tmem + 4, scale_desc(sf_smem + 512));
-          tc_cp_scales_pair(sf_tmem + 8, scale_desc(sf_smem + 1024));
+          // scale chunks -> TMEM.  A: K chunk c at columns 4c.  B: the box is [row group][K chunk],
+          // and the MMA wants the columns of one K chunk together: group g, chunk c -> 8c + 4g.
+#pragma unroll
+          for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
+            tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
+#pragma unroll
+            for (uint32_t g = 0; g < 2; ++g)
+              tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
+                                scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+          }
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
 #pragma unroll
-          for (uint32_t k = 0; k < BK / kMmaK; ++k) {
-            const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
-            tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4,
-                        (kc | k) != 0 ? 1u : 0u);
+          for (uint32_t k = 0; k < 4; ++k) {  // every MMA advances 32 bytes along the 128-byte rows
+            if (F4) {
+              // K = 64: blocks 2k and 2k+1 of the stage = bytes (2k % 4, +1) of K chunk k / 2
+              const uint32_t sf_id = 2 * (k & 1);
+              const uint32_t idesc = idesc_base | (sf_id << 4) | (sf_id << 29);
+              tc_mma_pair_f4(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem + 4 * (k >> 1),
+                             sf_tmem + cfg::kSfColsA + 8 * (k >> 1), (kc | k) != 0 ? 1u : 0u);
+            } else {
+              const uint32_t idesc = idesc_base | (k << 4) | (k << 29);  // byte k of the scale columns
+              tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + cfg::kSfColsA,
+                          (kc | k) != 0 ? 1u : 0u);
+            }
           }
           tc_commit_pair(empty_bar(stage));
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
@@ -786,21 +822,51 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   return cudaGetLastError();
 }
 
-cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn, uint32_t idesc_base) {
-  using cfg = Cfg2;
+// Dense FP4 operand map for kind::mxf4: two codes per byte in shared memory as in global memory.
+bool make_f4_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K) {
+  const cuuint64_t pitch = K / 2;
+  const cuuint64_t dims[3] = {K, rows, 1};
+  const cuuint64_t strides[2] = {pitch, pitch * rows};
+  const cuuint32_t box[3] = {256, 128, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN8B, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// Scale map whose box also spans `kchunks` K chunks: [row groups][K chunks][128 words].
+bool make_scale_map_k(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
+                      uint32_t groups, uint32_t kchunks) {
+  const uint64_t k_chunks = K / BK;
+  const cuuint64_t dims[3] = {128, k_chunks, rows / 128};
+  const cuuint64_t strides[2] = {512, 512 * k_chunks};
+  const cuuint32_t box[3] = {128, kchunks, groups};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <bool F4>
+cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
+  using cfg = Cfg2<F4>;
   CUtensorMap ma, mb, msa, msb, mc;
-  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) ||
-      !make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, 128) ||
-      !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, 128) ||
-      !make_scale_map(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1) ||
-      !make_scale_map(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, 2))
-    return cudaErrorInvalidValue;
+  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) &&
+            make_scale_map_k(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1, cfg::kKChunks) &&
+            make_scale_map_k(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, 2, cfg::kKChunks);
+  if (F4)
+    ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)a.M, (uint64_t)a.K) &&
+         make_f4_map(fn, &mb, a.B, (uint64_t)a.N, (uint64_t)a.K);
+  else
+    ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, 128) &&
+         make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, 128);
+  if (!ok) return cudaErrorInvalidValue;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(mx_gemm_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(mx_gemm_pair_kernel<F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -808,10 +874,14 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn, uint32_t idesc_base
   const uint32_t tiles = (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
   const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
-  const uint32_t tx_pair = 2u * (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 128 * BK * fmt_bits(a.fmtB) / 8 +
-                                           (int)cfg::kSfBytes);
-  const uint32_t idesc = idesc_base | ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-  mx_gemm_pair_kernel<<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
+  const uint32_t op_bytes = F4 ? 2u * 128u * 128u
+                               : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 128 * BK * fmt_bits(a.fmtB) / 8);
+  const uint32_t tx_pair = 2u * (op_bytes + cfg::kSfBytes);
+  // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code()
+  const uint32_t fa = F4 ? 1u : mma_fmt_code(a.fmtA), fb = F4 ? 1u : mma_fmt_code(a.fmtB);
+  const uint32_t idesc = (fa << 7) | (fb << 10) | (1u << 23) | ((uint32_t)(256 >> 3) << 17) |
+                         ((uint32_t)(256 >> 4) << 24);
+  mx_gemm_pair_kernel<F4><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair);
   return cudaGetLastError();
 }
@@ -836,8 +906,9 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
 #define MX_GEMM_PAIR_MIN_TILES (a.sm_count / 2)
 #endif
   if (a.M % 256 == 0 && (a.M / 256) * ((a.N + 255) / 256) >= MX_GEMM_PAIR_MIN_TILES) {
-    const uint32_t idesc2 = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23);
-    *cuda_err = launch_pair(a, fn, idesc2);
+    // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
+    const bool f4 = a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
+    *cuda_err = f4 ? launch_pair<true>(a, fn) : launch_pair<false>(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
 #endif

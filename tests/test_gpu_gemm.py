@@ -82,6 +82,30 @@ def test_scale_identification_exact(fa, fb, N):
     assert (C.cpu().numpy().astype(np.float64) == C64).all()
 
 
+@pytest.mark.parametrize("fa,fb,K", [(0, 0, 1024), (4, 4, 1024), (4, 4, 768), (2, 4, 512)])
+def test_scale_identification_two_cta_kernels(fa, fb, K):
+    """The same exact probe at a shape that selects the two-CTA kernels: E4M3 x E4M3 and FP6 x FP4 on
+    kind::mxf8f6f4, FP4 x FP4 on kind::mxf4 (K % 256 == 0: two scales per row and MMA) and FP4 x FP4
+    with K % 256 != 0 (falls back to kind::mxf8f6f4)."""
+    M, N = 512, 256 * 37
+    kb = K // 32
+    rng = np.random.default_rng(fa * 7 + fb + K)
+    a_codes = np.full((M, K), ONE[fa], np.uint8)
+    b_codes = np.full((N, K), ONE[fb], np.uint8)
+    sa = (127 + rng.integers(-3, 4, (M, kb))).astype(np.uint8)
+    sb = (127 + rng.integers(-3, 4, (N, kb))).astype(np.uint8)
+    sa_sw, sb_sw = _swizzle_scales(sa), _swizzle_scales(sb)
+    ea, eb = O.pack_codes(a_codes.reshape(-1), fa), O.pack_codes(b_codes.reshape(-1), fb)
+    C = _gemm_guarded(torch.from_numpy(ea).cuda(), torch.from_numpy(sa_sw).cuda(),
+                      torch.from_numpy(eb).cuda(), torch.from_numpy(sb_sw).cuda(), M, N, K, fa, fb)
+    want = 32.0 * (2.0 ** (sa.astype(np.float64) - 127)) @ (2.0 ** (sb.astype(np.float64) - 127)).T
+    assert (C.cpu().numpy().astype(np.float64) == want).all()
+    ms = rng.integers(0, M, 500)
+    ns = rng.integers(0, N, 500)
+    c64, _ = O.gemm_samples(ea, sa_sw, eb, sb_sw, M, N, K, fa, fb, ms, ns)
+    assert (c64 == want[ms, ns]).all()
+
+
 def test_element_position_probe_exact():
     """One nonzero element per row of A at a row-dependent K position against a B whose entries
     encode their K position: checks that element k of A meets element k of B for every k,
@@ -231,6 +255,9 @@ def _full_size_check(name, ea, sa, eb, sb, M, N, K, fa, fb, seed):
     ((4736, 8320, 384), 3, 4),    # ... with a ragged last tile (N = 65 x 128)
     ((2048, 9600, 384), 0, 2),    # M % 256 == 0: the two-CTA 256 x 256 kernel, ragged N
     ((256, 256 * 74, 128), 1, 0),  # two-CTA kernel, one tile per pair, a single K stage
+    ((2048, 9600, 512), 4, 4),    # FP4 x FP4 on kind::mxf4 (K % 256 == 0), ragged N
+    ((256, 256 * 74, 256), 4, 4),  # kind::mxf4, a single K stage
+    ((1024, 4864, 640), 4, 4),    # FP4 x FP4 with K % 256 != 0: kind::mxf8f6f4
 ])
 def test_kernel_variants_whole_matrix(shape, fa, fb):
     """Shapes that select each GEMM kernel variant; the whole output is checked against an
