@@ -211,6 +211,64 @@ def run_e2e(torch, mx, inputs, steps: int, warmup: int):
                         "(pinned host buffers, copies timed)"}
 
 
+def run_extras(torch, mx, inputs):
+    """The other benchmark configurations, outside the timed step: the FP4-weight x FP8-activation
+    GEMM (16384 x 28672 x 8192), the same shape with both operands FP4 (kind::mxf4), and the
+    MXFP6 training step of one 4096^3 linear layer (six quantizes, three GEMMs)."""
+    def timed(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(reps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps * 1e-3
+
+    out = {}
+    d = inputs.config5("cuda")
+    W, X = d["W"], d["X"]
+    M, K = X.shape
+    N = W.shape[1]
+    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(W, 0, mx.MX_E2M1)
+    t_qw = timed(lambda: mx.mx_quantize(W, 0, mx.MX_E2M1, out=(eb, sb)), 5)
+    t_qx = timed(lambda: mx.mx_quantize(X, 1, mx.MX_E4M3, out=(ea, sa)), 5)
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    t = timed(lambda: mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, out=C), 5)
+    out["config5_mxfp4_weights_x_mxfp8_activations"] = {
+        "gemm_TFLOPs": 2.0 * M * N * K / t / 1e12, "gemm_ms": t * 1e3,
+        "quantize_w_strided_GBps": algorithmic_bytes(K * N, 2, 4) / t_qw / 1e9,
+        "quantize_x_GBps": algorithmic_bytes(M * K, 2, 8) / t_qx / 1e9}
+    ea4, sa4 = mx.mx_quantize(X, 1, mx.MX_E2M1)
+    t4 = timed(lambda: mx.mx_gemm(ea4, sa4, eb, sb, M, N, K, mx.MX_E2M1, mx.MX_E2M1, out=C), 5)
+    out["mxfp4_x_mxfp4_same_shape_kind_mxf4"] = {"gemm_TFLOPs": 2.0 * M * N * K / t4 / 1e12, "gemm_ms": t4 * 1e3}
+    del d, W, X, C, ea, sa, eb, sb, ea4, sa4
+    torch.cuda.empty_cache()
+    d = inputs.config4("cuda")
+    Xc, Wc, dY = d["X"], d["W"], d["dY"]
+    n = Xc.shape[0]
+    act, wt, rnd = mx.MX_E3M2, mx.MX_E2M3, mx.MX_RHAZ
+    Y = torch.empty((n, n), dtype=torch.float32, device="cuda")
+
+    def train_step():
+        xa = mx.mx_quantize(Xc, 1, act, rnd)
+        wb = mx.mx_quantize(Wc, 0, wt, rnd)
+        mx.mx_gemm(*xa, *wb, n, n, n, act, wt, out=Y)            # Y = X W
+        ga = mx.mx_quantize(dY, 1, act, rnd)
+        wb2 = mx.mx_quantize(Wc, 1, wt, rnd)
+        mx.mx_gemm(*ga, *wb2, n, n, n, act, wt, out=Y)           # dX = dY W^T
+        xt = mx.mx_quantize(Xc, 0, act, rnd)
+        gt = mx.mx_quantize(dY, 0, act, rnd)
+        mx.mx_gemm(*xt, *gt, n, n, n, act, act, out=Y)           # dW = X^T dY
+
+    ts = timed(train_step, 10)
+    out["config4_mxfp6_training_step"] = {"ms": ts * 1e3, "gemm_TFLOPs_if_all_time_were_gemm": 3 * 2.0 * n ** 3 / ts / 1e12,
+                                          "launches": 9}
+    return out
+
+
 def run_cpu_baseline(rows: int = 2048, seconds_target: float = 15.0):
     """The oracle, as it stands, on the host cores: the same sweep on `rows` rows of the tensor."""
     import numpy as np
@@ -339,6 +397,9 @@ def main_ours(args, rank, world, local_rank):
         line["e2e"] = run_e2e(torch, mx, inputs, max(2, min(args.steps, 5)), 1)
         cpu, _ = run_cpu_baseline(rows=SWEEP_ROWS)
         line["cpu_baseline"] = cpu
+        del w
+        torch.cuda.empty_cache()
+        line["other_configs"] = run_extras(torch, mx, inputs)
     else:
         line["e2e"] = None
     print(json.dumps(line))
