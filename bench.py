@@ -263,9 +263,19 @@ def run_extras(torch, mx, inputs):
         gt = mx.mx_quantize(dY, 0, act, rnd)
         mx.mx_gemm(*xt, *gt, n, n, n, act, act, out=Y)           # dW = X^T dY
 
+    def train_step_fused():  # each tensor is read once: both of its MX tensors come from one pass
+        (xa, xt) = mx.mx_quantize_dual(Xc, act, rnd)
+        (wb2, wb) = mx.mx_quantize_dual(Wc, wt, rnd)
+        (ga, gt) = mx.mx_quantize_dual(dY, act, rnd)
+        mx.mx_gemm(*xa, *wb, n, n, n, act, wt, out=Y)
+        mx.mx_gemm(*ga, *wb2, n, n, n, act, wt, out=Y)
+        mx.mx_gemm(*xt, *gt, n, n, n, act, act, out=Y)
+
     ts = timed(train_step, 10)
-    out["config4_mxfp6_training_step"] = {"ms": ts * 1e3, "gemm_TFLOPs_if_all_time_were_gemm": 3 * 2.0 * n ** 3 / ts / 1e12,
-                                          "launches": 9}
+    tf = timed(train_step_fused, 10)
+    out["config4_mxfp6_training_step"] = {
+        "ms_six_quantizes_three_gemms": ts * 1e3, "ms_three_dual_quantizes_three_gemms": tf * 1e3,
+        "gemm_flops_per_step": 3 * 2.0 * n ** 3}
     return out
 
 

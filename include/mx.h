@@ -155,6 +155,23 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out,
                 const int64_t* shape, int ndim, int axis,
                 mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts);
 
+/*
+ * mx_quantize_dual -- both MX tensors of a 2-D tensor in one pass (Sections 3 and 4.1)
+ *
+ * The training flow of Section 4.1 needs every matmul input quantized along its own reduction
+ * axis: X enters Y = X W with blocks along its rows and dW = X^T dY with blocks along its columns,
+ * and by Section 3 those are two different MX tensors.  This call reads in[R x C] once and writes
+ *   elems_row / scales_row : exactly what mx_quantize(in, axis = 1) writes  ([R x C], K = C)
+ *   elems_col / scales_col : exactly what mx_quantize(in, axis = 0) writes  ([C x R], K = R)
+ * with the same format, rounding, dtype and scale layout for both.
+ * Requirements: R a multiple of 128; C a multiple of 128 (BF16) or 64 (FP32); all pointers
+ * 16-byte aligned.  Other shapes: MX_ERR_UNSUPPORTED (call mx_quantize twice instead).
+ * Errors otherwise as mx_quantize.
+ */
+int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row,
+                     void* elems_col, uint8_t* scales_col, int64_t R, int64_t C,
+                     mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts);
+
 /* ------------------------------------------------------------------------- */
 /* mx_dequantize -- Section 2 value semantics                                */
 /* ------------------------------------------------------------------------- */

@@ -30,7 +30,7 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
-    "mx_last_cuda_error", "mx_quantize", "mx_dequantize", "mx_gemm",
+    "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -71,6 +71,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_strerror.restype = ctypes.c_char_p
     lib.mx_last_cuda_error.restype = ctypes.c_char_p
     lib.mx_quantize.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op]
+    lib.mx_quantize_dual.argtypes = [vp, vp, u8p, vp, u8p, i64, i64, ci, ci, op]
     lib.mx_dequantize.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op]
     lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
@@ -154,6 +155,26 @@ def mx_quantize(x: torch.Tensor, axis: int, fmt: int, rounding: int = MX_RNE,
     _check(_lib.mx_quantize(x.data_ptr(), elems.data_ptr(), scales.data_ptr(), _shape_arr(shape),
                             len(shape), axis, fmt, rounding, ctypes.byref(o)), "mx_quantize")
     return elems, scales
+
+
+def mx_quantize_dual(x: torch.Tensor, fmt: int, rounding: int = MX_RNE, layout: int = MX_SCALES_SWIZZLED,
+                     out=None):
+    """Both MX tensors of a contiguous 2-D CUDA tensor in one pass: returns
+    ((elems_row, scales_row), (elems_col, scales_col)) = (mx_quantize(x, 1), mx_quantize(x, 0))."""
+    assert x.is_cuda and x.is_contiguous() and x.dim() == 2
+    R, C = x.shape
+    if out is None:
+        u8 = dict(dtype=torch.uint8, device=x.device)
+        er = torch.empty(mx_elems_bytes([R, C], 1, fmt), **u8)
+        sr = torch.empty(mx_scales_bytes([R, C], 1, layout), **u8)
+        ec = torch.empty(mx_elems_bytes([R, C], 0, fmt), **u8)
+        sc = torch.empty(mx_scales_bytes([R, C], 0, layout), **u8)
+    else:
+        (er, sr), (ec, sc) = out
+    o = _opts(_dtype_code(x.dtype), layout)
+    _check(_lib.mx_quantize_dual(x.data_ptr(), er.data_ptr(), sr.data_ptr(), ec.data_ptr(), sc.data_ptr(),
+                                 R, C, fmt, rounding, ctypes.byref(o)), "mx_quantize_dual")
+    return (er, sr), (ec, sc)
 
 
 def mx_dequantize(elems: torch.Tensor, scales: torch.Tensor, shape: Sequence[int], fmt: int,

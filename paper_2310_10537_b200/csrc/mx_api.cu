@@ -163,6 +163,40 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 
+int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void* elems_col,
+                     uint8_t* scales_col, int64_t R, int64_t C, mx_fmt_t fmt, mx_round_t rounding,
+                     const mx_opts_t* opts) {
+  Opts o;
+  if (!fmt_ok((int)fmt) || (rounding != MX_RNE && rounding != MX_RHAZ) || !read_opts(opts, &o))
+    return MX_ERR_FMT;
+  if (R < 0 || C < 0 || R % 32 || C % 32) return MX_ERR_SHAPE;
+  if (R == 0 || C == 0) return MX_OK;
+  if (!in || !elems_row || !scales_row || !elems_col || !scales_col) return MX_ERR_NULL;
+  if ((uintptr_t)in % 16 || (uintptr_t)elems_row % 16 || (uintptr_t)scales_row % 16 ||
+      (uintptr_t)elems_col % 16 || (uintptr_t)scales_col % 16)
+    return MX_ERR_ALIGN;
+  const int64_t strip = o.dtype == MX_BF16 ? 128 : 64;
+  if (R % 128 || C % strip || R >= ((int64_t)1 << 31) || C >= ((int64_t)1 << 31)) return MX_ERR_UNSUPPORTED;
+  mx::DualArgs a;
+  a.in = in;
+  a.elems_row = (uint8_t*)elems_row; a.scales_row = scales_row;
+  a.elems_col = (uint8_t*)elems_col; a.scales_col = scales_col;
+  a.R = R; a.C = C; a.fmt = (int)fmt; a.rounding = (int)rounding; a.dtype = o.dtype; a.layout = o.layout;
+  a.stream = o.stream;
+  cudaError_t e;
+  // swizzled scale tensors have padding when kblocks % 4 != 0 (rows are multiples of 128 here)
+  if (o.layout == MX_SCALES_SWIZZLED && (C / 32) % 4 != 0) {
+    e = cudaMemsetAsync(scales_row, 0, scales_bytes(R, C / 32, o.layout), o.stream);
+    if (e != cudaSuccess) return fail_cuda(e);
+  }
+  if (o.layout == MX_SCALES_SWIZZLED && C % 128 != 0) {  // rows of the [C x R] scale tensor
+    e = cudaMemsetAsync(scales_col, 0, scales_bytes(C, R / 32, o.layout), o.stream);
+    if (e != cudaSuccess) return fail_cuda(e);
+  }
+  e = mx::launch_quantize_dual(a);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
 int mx_dequantize(const void* elems, const uint8_t* scales, void* out, const int64_t* shape,
                   int ndim, int axis, mx_fmt_t fmt, const mx_opts_t* opts) {
   Opts o;

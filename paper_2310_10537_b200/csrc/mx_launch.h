@@ -20,6 +20,16 @@ struct QuantizeArgs {
 };
 cudaError_t launch_quantize(const QuantizeArgs& a);
 
+struct DualArgs {
+  const void* in;
+  uint8_t *elems_row, *scales_row;  // blocks along the contiguous axis: [R x C]
+  uint8_t *elems_col, *scales_col;  // blocks along axis 0: [C x R]
+  int64_t R, C;
+  int fmt, rounding, dtype, layout;
+  cudaStream_t stream;
+};
+cudaError_t launch_quantize_dual(const DualArgs& a);
+
 struct DequantizeArgs {
   const uint8_t* elems;
   const uint8_t* scales;

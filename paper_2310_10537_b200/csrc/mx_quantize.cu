@@ -11,6 +11,7 @@
 // Both are bound by HBM bandwidth: in_bytes + bits/8 + 1/32 bytes per element.
 #include "mx_device.cuh"
 #include "mx_launch.h"
+#include "mx_quantize_common.cuh"
 
 namespace mx {
 
@@ -55,43 +56,6 @@ __device__ __forceinline__ void load_unit(const void* in, size_t unit, uint32_t 
       const uint4 q = ld_stream_16(p + 16 * j);
       w[4 * j] = q.x; w[4 * j + 1] = q.y; w[4 * j + 2] = q.z; w[4 * j + 3] = q.w;
     }
-  }
-}
-
-// max |V_i| over the unit as a balanced tree (short dependency chains), on packed BF16 pairs
-// where the input is BF16.
-template <int DTYPE>
-__device__ __forceinline__ float unit_amax(const uint32_t (&w)[16]) {
-  if constexpr (DTYPE == MX_BF16) {
-    uint32_t m[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) m[i] = absmax_nan_bf16x2(w[2 * i], w[2 * i + 1]);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) m[i] = absmax_nan_bf16x2(m[2 * i], m[2 * i + 1]);
-    m[0] = absmax_nan_bf16x2(absmax_nan_bf16x2(m[0], m[1]), absmax_nan_bf16x2(m[2], m[3]));
-    return bf16x2_halves_max(m[0]);
-  } else {
-    float m[8];
-#pragma unroll
-    for (int i = 0; i < 8; ++i) m[i] = absmax_nan(__uint_as_float(w[2 * i]), __uint_as_float(w[2 * i + 1]));
-#pragma unroll
-    for (int i = 0; i < 4; ++i) m[i] = absmax_nan(m[2 * i], m[2 * i + 1]);
-    return absmax_nan(absmax_nan(m[0], m[1]), absmax_nan(m[2], m[3]));
-  }
-}
-
-// Elements 8g .. 8g+7 of the unit as FP32 values.
-template <int DTYPE>
-__device__ __forceinline__ void unit_group(const uint32_t (&w)[16], int g, float (&x)[8]) {
-  if (DTYPE == MX_BF16) {
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-      x[2 * i] = __uint_as_float(w[4 * g + i] << 16);  // BF16 widens exactly
-      x[2 * i + 1] = __uint_as_float(w[4 * g + i] & 0xFFFF0000u);
-    }
-  } else {
-#pragma unroll
-    for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(w[(8 * g + i) % 16]);
   }
 }
 
@@ -232,22 +196,6 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
 #define MX_QT_THREADS 128
 #endif
 constexpr int kStridedThreads = MX_QT_THREADS;
-
-template <int DTYPE, int COLS> struct StridedRow {
-  static constexpr int kBytes = COLS * (DTYPE == MX_BF16 ? 2 : 4);   // bytes loaded per row: 8, 4 or 2
-  static constexpr int kWords = kBytes >= 4 ? kBytes / 4 : 1;
-};
-
-// Element (row k, column c) of the packed rows as an FP32 value.
-template <int DTYPE, int COLS>
-__device__ __forceinline__ float strided_elem(const uint32_t (&raw)[kBlock][StridedRow<DTYPE, COLS>::kWords],
-                                              int k, int c) {
-  if (DTYPE == MX_BF16) {
-    const uint32_t w = raw[k][(c / 2) % StridedRow<DTYPE, COLS>::kWords];
-    return __uint_as_float((c & 1) ? (w & 0xFFFF0000u) : (w << 16));
-  }
-  return __uint_as_float(raw[k][c % StridedRow<DTYPE, COLS>::kWords]);
-}
 
 #ifndef MX_QT_MINB
 #define MX_QT_MINB 4

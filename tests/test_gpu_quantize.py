@@ -88,6 +88,33 @@ def test_middle_axis_of_3d_tensor(fmt):
     _assert_same_bytes(s, ws, "scales")
 
 
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("fmt", FMTS)
+def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype):
+    """mx_quantize_dual reads the tensor once and must write exactly the two tensors that
+    quantizing along axis 1 and along axis 0 give (checked against the oracle, not against
+    mx_quantize)."""
+    R, C = (384, 320) if dtype == torch.float32 else (256, 384)
+    x = inputs.adversarial("cuda", rows=R, cols=C, dtype=dtype, seed=41 + fmt)
+    xin = to_oracle_input(x)
+    for rounding, layout in ((mx.MX_RNE, mx.MX_SCALES_SWIZZLED), (mx.MX_RHAZ, mx.MX_SCALES_LINEAR)):
+        g = [Guarded(mx.mx_elems_bytes([R, C], 1, fmt)), Guarded(mx.mx_scales_bytes([R, C], 1, layout)),
+             Guarded(mx.mx_elems_bytes([R, C], 0, fmt)), Guarded(mx.mx_scales_bytes([R, C], 0, layout))]
+        mx.mx_quantize_dual(x, fmt, rounding, layout, out=((g[0].view, g[1].view), (g[2].view, g[3].view)))
+        torch.cuda.synchronize()
+        for gg in g:
+            gg.check()
+        wer, wsr = O.quantize(xin, 1, fmt, rounding, layout)
+        wec, wsc = O.quantize(xin, 0, fmt, rounding, layout)
+        _assert_same_bytes(g[0].view, wer, ("row elems", fmt, dtype, layout))
+        _assert_same_bytes(g[1].view, wsr, ("row scales", fmt, dtype, layout))
+        _assert_same_bytes(g[2].view, wec, ("col elems", fmt, dtype, layout))
+        _assert_same_bytes(g[3].view, wsc, ("col scales", fmt, dtype, layout))
+    with pytest.raises(mx.MxError) as ei:
+        mx.mx_quantize_dual(torch.zeros((96, 128), dtype=dtype, device="cuda"), fmt)
+    assert ei.value.status == mx.MX_ERR_UNSUPPORTED
+
+
 def test_worked_blocks_on_device():
     """The hand-worked W1 / W4 / W5 blocks straight through the kernel."""
     v = torch.zeros(32, device="cuda")
