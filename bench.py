@@ -54,6 +54,25 @@ def measured_peaks():
             "source": "fallback"}
 
 
+def max_over_ranks(values, device, world: int):
+    """Element-wise maximum of a list of floats over all ranks (the slowest rank sets the job's
+    time).  With one rank it is the identity; otherwise an all-reduce on the process group that
+    is already initialised (NCCL on GPUs, gloo in the CPU tests)."""
+    import torch
+    if world <= 1:
+        return [float(v) for v in values]
+    import torch.distributed as dist
+    t = torch.tensor([float(v) for v in values], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return t.tolist()
+
+
+def job_throughput(units_per_rank: float, world: int, slowest_seconds: float) -> float:
+    """Whole-job throughput under weak scaling: every rank processes `units_per_rank` of its own
+    shard (MX blocks are independent, so ranks exchange nothing) in the time of the slowest rank."""
+    return world * units_per_rank / slowest_seconds
+
+
 class ClockSampler:
     """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
 
@@ -346,17 +365,13 @@ def main_ours(args, rank, world, local_rank):
     ms = {"quantize_sweep": phase(0, 1), "dequantize_sweep": phase(1, 2), "quantize_x": phase(3, 4),
           "quantize_w_strided": phase(4, 5), "gemm": phase(6, 7)}
     ms_step = t_begin.elapsed_time(t_end) / args.steps
-    t = torch.tensor([ms_step, ms["quantize_sweep"] + ms["dequantize_sweep"], ms["gemm"],
-                      ms["quantize_sweep"]], dtype=torch.float64, device=dev)
-    if world > 1:
-        import torch.distributed as dist
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    ms_step_max, ms_sweep_max, ms_gemm_max, ms_q_max = t.tolist()
+    ms_step_max, ms_sweep_max, ms_gemm_max, ms_q_max = max_over_ranks(
+        [ms_step, ms["quantize_sweep"] + ms["dequantize_sweep"], ms["gemm"], ms["quantize_sweep"]], dev, world)
     if rank != 0:
         return
 
-    value = world * w.bytes_sweep / (ms_sweep_max * 1e-3) / 1e9
-    gemm_tflops = world * w.flops / (ms_gemm_max * 1e-3) / 1e12
+    value = job_throughput(w.bytes_sweep, world, ms_sweep_max * 1e-3) / 1e9
+    gemm_tflops = job_throughput(w.flops, world, ms_gemm_max * 1e-3) / 1e12
     q_gbs = sum(w.bytes_q) / (ms["quantize_sweep"] * 1e-3) / 1e9
     fp8_peak = 2.0 * peaks["bf16_tflops"]
     line = {
