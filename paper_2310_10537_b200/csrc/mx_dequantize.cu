@@ -11,9 +11,6 @@
 namespace mx {
 
 constexpr int kDqThreads = 256;
-#ifndef MX_DQ_CAP
-#define MX_DQ_CAP 0  // CTAs per SM the grid is capped at (0 = one CTA per 256 units, no loop)
-#endif
 
 // Two codes -> two FP32 values (exact: every element value fits FP16).
 // pair = code0 | code1 << 8  (FP4: code0 | code1 << 4 in the low byte).
@@ -215,11 +212,7 @@ static cudaError_t launch_dq(const DequantizeArgs& a) {
   const FastDiv kd = make_fastdiv(kblocks);
   const bool al32 = (uintptr_t)a.out % 32 == 0 && (uintptr_t)a.elems % 32 == 0;
   auto kernel = al32 ? dequantize_kernel<FMT, DTYPE, LAYOUT, true> : dequantize_kernel<FMT, DTYPE, LAYOUT, false>;
-  uint32_t grid = (n_units + kDqThreads - 1) / kDqThreads;
-#if MX_DQ_CAP > 0
-  const uint32_t cap = (uint32_t)a.sm_count * MX_DQ_CAP;
-  if (grid > cap) grid = cap;
-#endif
+  const uint32_t grid = (n_units + kDqThreads - 1) / kDqThreads;  // one CTA per 256 units, no loop
   kernel<<<grid, kDqThreads, 0, a.stream>>>(a.elems, a.scales, a.out, n_units, kblocks, kd);
   return cudaGetLastError();
 }

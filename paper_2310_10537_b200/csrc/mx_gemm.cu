@@ -51,10 +51,7 @@ __device__ unsigned int g_gemm_status;
 // Epilogue staging in shared memory: chunks of 32 rows x 16 columns of FP32 per warp.
 constexpr uint32_t kEpiChunkCols = 16;
 constexpr uint32_t kEpiChunkBytes = 32 * kEpiChunkCols * 4;
-#ifndef MX_EPI_BUFS
-#define MX_EPI_BUFS 1
-#endif
-constexpr uint32_t kEpiBufs = MX_EPI_BUFS;                        // staging chunks per warp
+constexpr uint32_t kEpiBufs = 1;                                   // staging chunks per warp
 constexpr uint32_t kEpiBytes = 8 * kEpiBufs * kEpiChunkBytes;     // eight epilogue warps
 
 template <int BN>
@@ -454,10 +451,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 template <bool F4>
 struct Cfg2 {
   static constexpr int BN = 256;
-#ifndef MX_PAIR_STAGES
-#define MX_PAIR_STAGES 6
-#endif
-  static constexpr int kStages = F4 ? MX_PAIR_STAGES - 1 : MX_PAIR_STAGES;
+  static constexpr int kStages = F4 ? 5 : 6;
   static constexpr int kBKe = F4 ? 256 : 128;           // K elements per stage (128-byte operand rows)
   static constexpr int kKChunks = kBKe / 128;           // 512-byte scale chunks (4 MX blocks) along K per stage
   static constexpr int kSfColsA = 4 * kKChunks;         // TMEM columns: this CTA's 128 rows of A
@@ -892,26 +886,17 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   EncodeTiledFn fn = encode_fn(cuda_err);
   if (!fn) return MX_ERR_CUDA;
-#ifdef MX_GEMM_BN
-  const int bn = MX_GEMM_BN;
-#else
   // 256-wide tiles move the fewest operand bytes through shared memory per flop; problems with
   // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
   const int64_t tiles256 = (a.M / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
-#endif
-#ifndef MX_GEMM_NO_PAIR
   // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
-#ifndef MX_GEMM_PAIR_MIN_TILES
-#define MX_GEMM_PAIR_MIN_TILES (a.sm_count / 2)
-#endif
-  if (a.M % 256 == 0 && (a.M / 256) * ((a.N + 255) / 256) >= MX_GEMM_PAIR_MIN_TILES) {
+  if (a.M % 256 == 0 && (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
     const bool f4 = a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
     *cuda_err = f4 ? launch_pair<true>(a, fn) : launch_pair<false>(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
-#endif
   CUtensorMap ma, mb;
   if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, BM) ||
       !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, (uint32_t)bn)) {

@@ -16,15 +16,8 @@
 namespace mx {
 
 constexpr int kThreads = 256;
-#ifndef MX_Q_U
-#define MX_Q_U 1      // 64-byte units per thread and loop iteration
-#endif
-#ifndef MX_Q_CAP
-#define MX_Q_CAP 0     // CTAs per SM the grid is capped at (0 = no cap, -1 = resident CTAs)
-#endif
-#ifndef MX_Q_MINB
-#define MX_Q_MINB 4   // resident CTAs per SM the register allocation must allow
-#endif
+constexpr int kUnitsPerThread = 1;  // 64-byte units per thread (more only lowered occupancy)
+constexpr int kMinCtasPerSm = 4;    // resident CTAs per SM the register allocation must allow
 
 // ---------------------------------------------------------------------------
 // Contiguous axis
@@ -60,7 +53,7 @@ __device__ __forceinline__ void load_unit(const void* in, size_t unit, uint32_t 
 }
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, bool ALIGNED32, int U>
-__global__ void __launch_bounds__(kThreads, MX_Q_MINB)
+__global__ void __launch_bounds__(kThreads, kMinCtasPerSm)
 quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
                          uint8_t* __restrict__ scales, uint32_t n_units, uint32_t kblocks,
                          FastDiv kb_div, uint32_t scale_words) {
@@ -192,16 +185,10 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
 // registers in their packed input form (8 bytes per row for the wide variants: four BF16
 // or two FP32 columns), so a block of every column is complete in one thread: no shared
 // memory, no shuffles.  Output row = o * inner + column, block axis innermost.
-#ifndef MX_QT_THREADS
-#define MX_QT_THREADS 128
-#endif
-constexpr int kStridedThreads = MX_QT_THREADS;
+constexpr int kStridedThreads = 128;
 
-#ifndef MX_QT_MINB
-#define MX_QT_MINB 4
-#endif
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
-__global__ void __launch_bounds__(kStridedThreads, MX_QT_MINB)
+__global__ void __launch_bounds__(kStridedThreads, 4)
 quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
                         uint8_t* __restrict__ scales, uint32_t outer, uint32_t L,
                         uint32_t inner, uint32_t kb_per_thread) {
@@ -448,33 +435,18 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
 // Host-side dispatch
 // ---------------------------------------------------------------------------
 
-// Resident CTAs per SM of a kernel (queried once per instantiation): persistent grids are sized
-// to exactly fill the machine so that no partial wave trails the launch.
-template <typename K>
-static int resident_ctas(K kernel, int threads) {
-  int n = 0;
-  if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&n, kernel, threads, 0) != cudaSuccess || n < 1) n = 1;
-  return n;
-}
-
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, bool AL32>
 static cudaError_t launch_lastaxis_al(const QuantizeArgs& a) {
-  constexpr int U = MX_Q_U;
+  constexpr int U = kUnitsPerThread;
   constexpr int kElems = LastAxis<DTYPE>::kElems;
   const uint32_t n_units = (uint32_t)(a.numel / kElems);
   const uint32_t n_blocks = (uint32_t)(a.numel / kBlock);
   const uint32_t kblocks = (uint32_t)(a.L / kBlock);
   const uint32_t span = kThreads * U;
   auto kernel = quantize_lastaxis_kernel<FMT, ROUND, DTYPE, LAYOUT, AL32, U>;
-  uint32_t grid = (n_units + span - 1) / span;
-#if MX_Q_CAP > 0
-  const uint32_t cap = (uint32_t)a.sm_count * MX_Q_CAP;
-  if (grid > cap) grid = cap;
-#elif MX_Q_CAP < 0
-  static const int per_sm = resident_ctas(kernel, kThreads);
-  const uint32_t cap = (uint32_t)(a.sm_count * per_sm);
-  if (grid > cap) grid = cap;
-#endif
+  // one CTA per 256 units, no grid-stride loop: in steady state the block scheduler's natural
+  // desynchronisation of CTAs beat a persistent grid by 5-10 %
+  const uint32_t grid = (n_units + span - 1) / span;
   const FastDiv kd = make_fastdiv(kblocks);
   // one 32-bit store per four scale bytes when groups of four never straddle a row or the end
   const uint32_t scale_words = LAYOUT == MX_SCALES_LINEAR ? (n_blocks % 4 == 0) : (kblocks % 4 == 0);
@@ -529,10 +501,6 @@ static cudaError_t launch_strided(const QuantizeArgs& a) {
         a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner);
     return cudaGetLastError();
   }
-#ifdef MX_QT_BF16_COLS
-  if (DTYPE == MX_BF16 && a.inner % MX_QT_BF16_COLS == 0 && (uintptr_t)a.in % 4 == 0)
-    return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, (DTYPE == MX_BF16 ? MX_QT_BF16_COLS : kWide)>(a);
-#endif
   if (wide) return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, kWide>(a);
   return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, 1>(a);
 }
