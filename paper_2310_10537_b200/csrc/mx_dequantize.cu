@@ -84,6 +84,7 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
   constexpr int kLanes = kBlock / kElems;
   constexpr int kInBytes = kElems * bits / 8;  // 32/24/16 or 16/12/8
   constexpr int kWords = kInBytes / 4;
+  pdl_prologue();
   for (uint32_t unit = blockIdx.x * kDqThreads + threadIdx.x; unit < n_units;
        unit += gridDim.x * kDqThreads) {
     uint32_t w[kWords];
@@ -213,8 +214,7 @@ static cudaError_t launch_dq(const DequantizeArgs& a) {
   const bool al32 = (uintptr_t)a.out % 32 == 0 && (uintptr_t)a.elems % 32 == 0;
   auto kernel = al32 ? dequantize_kernel<FMT, DTYPE, LAYOUT, true> : dequantize_kernel<FMT, DTYPE, LAYOUT, false>;
   const uint32_t grid = (n_units + kDqThreads - 1) / kDqThreads;  // one CTA per 256 units, no loop
-  kernel<<<grid, kDqThreads, 0, a.stream>>>(a.elems, a.scales, a.out, n_units, kblocks, kd);
-  return cudaGetLastError();
+  return launch_pdl(kernel, dim3(grid), dim3(kDqThreads), 0, a.stream, a.elems, a.scales, a.out, n_units, kblocks, kd);
 }
 
 template <int FMT>

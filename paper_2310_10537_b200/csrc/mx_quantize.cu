@@ -63,6 +63,7 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
   constexpr int kOutBytes = kElems * bits / 8;  // 32/24/16 (BF16) or 16/12/8 (FP32) per thread
   const uint32_t lane = threadIdx.x & 31u;
   const uint32_t span = kThreads * U;
+  pdl_prologue();
   for (uint32_t base = blockIdx.x * span; base < n_units; base += gridDim.x * span) {
     uint32_t raw[U][16];
     bool ok[U];
@@ -197,6 +198,7 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
   constexpr int kRowBytes = StridedRow<DTYPE, COLS>::kBytes;
   const uint32_t kblocks = L / kBlock;
   const uint32_t col0 = (blockIdx.x * kStridedThreads + threadIdx.x) * COLS;
+  pdl_prologue();
   if (col0 >= inner) return;  // no warp-level exchange in this kernel
   const uint32_t kb_begin = blockIdx.y * kb_per_thread;
   const uint32_t kb_end = min(kb_begin + kb_per_thread, kblocks);
@@ -311,6 +313,7 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
   uint8_t* area = staging + warp * (kRows * kPitch);
   const uint32_t kblocks = L / kBlock;
   const uint32_t warp_col0 = (blockIdx.x * kStagedThreads + warp * 32) * COLS;  // first column of the warp
+  pdl_prologue();
   if (warp_col0 >= inner) return;                                  // whole warp out of range
   const uint32_t col0 = warp_col0 + lane * COLS;
   const bool lane_ok = col0 < inner;                               // inner % COLS == 0: all or none of its columns
@@ -450,8 +453,8 @@ static cudaError_t launch_lastaxis_al(const QuantizeArgs& a) {
   const FastDiv kd = make_fastdiv(kblocks);
   // one 32-bit store per four scale bytes when groups of four never straddle a row or the end
   const uint32_t scale_words = LAYOUT == MX_SCALES_LINEAR ? (n_blocks % 4 == 0) : (kblocks % 4 == 0);
-  kernel<<<grid, kThreads, 0, a.stream>>>(a.in, a.elems, a.scales, n_units, kblocks, kd, scale_words);
-  return cudaGetLastError();
+  return launch_pdl(kernel, dim3(grid), dim3(kThreads), 0, a.stream, a.in, a.elems, a.scales, n_units, kblocks, kd,
+                    scale_words);
 }
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
@@ -474,9 +477,9 @@ static cudaError_t launch_strided_cols(const QuantizeArgs& a) {
          (uint64_t)grid_x * ((kblocks + kb_per_thread - 1) / kb_per_thread) * outer_eff < (uint64_t)a.sm_count * 16)
     kb_per_thread >>= 1;
   dim3 grid(grid_x, (kblocks + kb_per_thread - 1) / kb_per_thread, (uint32_t)outer_eff);
-  quantize_strided_kernel<FMT, ROUND, DTYPE, LAYOUT, COLS><<<grid, kStridedThreads, 0, a.stream>>>(
-      a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner, kb_per_thread);
-  return cudaGetLastError();
+  return launch_pdl(quantize_strided_kernel<FMT, ROUND, DTYPE, LAYOUT, COLS>, grid, dim3(kStridedThreads), 0,
+                    a.stream, a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner,
+                    kb_per_thread);
 }
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
@@ -497,9 +500,9 @@ static cudaError_t launch_strided(const QuantizeArgs& a) {
     const uint32_t threads_x = (uint32_t)(a.inner / kWide);
     dim3 grid((threads_x + kStagedThreads - 1) / kStagedThreads, kblocks / 4,
               (uint32_t)(a.outer < 65535 ? a.outer : 65535));
-    quantize_strided_staged_kernel<FMT, ROUND, DTYPE, LAYOUT, kWide><<<grid, kStagedThreads, smem, a.stream>>>(
-        a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L, (uint32_t)a.inner);
-    return cudaGetLastError();
+    return launch_pdl(quantize_strided_staged_kernel<FMT, ROUND, DTYPE, LAYOUT, kWide>, grid,
+                      dim3(kStagedThreads), smem, a.stream, a.in, a.elems, a.scales, (uint32_t)a.outer,
+                      (uint32_t)a.L, (uint32_t)a.inner);
   }
   if (wide) return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, kWide>(a);
   return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, 1>(a);

@@ -52,6 +52,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   uint8_t* sarea = tarea + 32 * kTPitch;
   const uint32_t strip = blockIdx.x * (kDualThreads / 32) + warp;   // column strip of 32*COLS columns
   const uint32_t warp_col0 = strip * 32 * COLS;
+  pdl_prologue();
   if (warp_col0 >= C) return;
   const uint32_t col0 = warp_col0 + lane * COLS;
   const size_t esz = DTYPE == MX_BF16 ? 2 : 4;
@@ -196,9 +197,9 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
   static_assert(cfg::kSmem <= 48 * 1024, "fits the default shared-memory limit");
   const uint32_t strips = (uint32_t)(a.C / (32 * cfg::COLS));
   dim3 grid((strips + kDualThreads / 32 - 1) / (kDualThreads / 32), (uint32_t)(a.R / 128));
-  quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT><<<grid, kDualThreads, cfg::kSmem, a.stream>>>(
-      a.in, a.elems_row, a.scales_row, a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C);
-  return cudaGetLastError();
+  return launch_pdl(quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT>, grid, dim3(kDualThreads), cfg::kSmem,
+                    a.stream, a.in, a.elems_row, a.scales_row, a.elems_col, a.scales_col, (uint32_t)a.R,
+                    (uint32_t)a.C);
 }
 
 template <int FMT, int ROUND>
