@@ -212,6 +212,16 @@ int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, 
             int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
             const mx_opts_t* opts);
 
+/*
+ * mx_gemm with the result stored as BF16, the scalar-float format the paper keeps
+ * tensors in between MX operations (Section 6.2).  C is BF16 row-major [M x N]; each
+ * dot product is accumulated in FP32 exactly as in mx_gemm and rounded to nearest even
+ * once, in the epilogue.  Requirements and errors are those of mx_gemm.
+ */
+int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                 int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                 const mx_opts_t* opts);
+
 /* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */
 /* ------------------------------------------------------------------------- */

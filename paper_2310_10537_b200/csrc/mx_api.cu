@@ -357,7 +357,7 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
 // ---------------------------------------------------------------------------
 
 static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
-                         const float* C, int64_t M, int64_t N, int64_t K, int fmtA, int fmtB) {
+                         const void* C, int64_t M, int64_t N, int64_t K, int fmtA, int fmtB) {
   if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
   if (!fmt_ok(fmtA) || !fmt_ok(fmtB)) return MX_ERR_FMT;
   if (fmtA == MX_INT8 || fmtB == MX_INT8) return MX_ERR_UNSUPPORTED;
@@ -366,8 +366,9 @@ static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const 
   return MX_OK;
 }
 
-int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, float* C,
-            int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
+static int gemm_device(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                       int c_bf16, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                       const mx_opts_t* opts) {
   Opts o;
   int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB);
   if (rc != MX_OK) return rc;
@@ -379,7 +380,7 @@ int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, 
   if (M == 0 || N == 0) return MX_OK;
   cudaError_t e;
   mx::GemmArgs a;
-  a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C;
+  a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
   a.sm_count = sm_count(&e);
@@ -398,6 +399,17 @@ int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, 
     }
   }
   return MX_OK;
+}
+
+int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, float* C,
+            int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
+  return gemm_device(A, sA, B, sB, C, 0, M, N, K, fmtA, fmtB, opts);
+}
+
+int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                 int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                 const mx_opts_t* opts) {
+  return gemm_device(A, sA, B, sB, C, 1, M, N, K, fmtA, fmtB, opts);
 }
 
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {

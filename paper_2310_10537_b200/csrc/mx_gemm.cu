@@ -201,12 +201,42 @@ __device__ __forceinline__ void bulk_wait_all() {
 }
 
 // r[j][i] = column 32 j + i of this thread's row (row0 + lane) starting at column col0 of C.
+// A staging chunk is 32 rows x 64 bytes: 16 FP32 columns, or 32 BF16 columns (each FP32
+// accumulator rounded to nearest even).
 template <uint32_t kLoads>
 __device__ __forceinline__ void store_rows(const uint32_t (&r)[kLoads][32], uint32_t stage_smem,
                                            const CUtensorMap* tmap_c, int col0, int row0,
-                                           uint32_t valid_cols, uint32_t lane) {
+                                           uint32_t valid_cols, uint32_t lane, uint32_t c_bf16) {
   if (lane == 0) bulk_wait_read<0>();  // chunks of the previous tile have left shared memory
   __syncwarp();
+  if (c_bf16) {
+#pragma unroll
+    for (uint32_t q = 0; q < kLoads; ++q) {
+      if (q * 32u < valid_cols) {
+        const uint32_t buf = q % kEpiBufs;
+        if (q >= kEpiBufs) {
+          if (lane == 0) bulk_wait_read<(int)kEpiBufs - 1>();
+          __syncwarp();
+        }
+        const uint32_t base = stage_smem + buf * kEpiChunkBytes + lane * 64;
+#pragma unroll
+        for (uint32_t c = 0; c < 4; ++c) {
+          uint32_t w[4];
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i)
+            asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(w[i])
+                : "f"(__uint_as_float(r[q][8 * c + 2 * i + 1])), "f"(__uint_as_float(r[q][8 * c + 2 * i])));
+          asm volatile("st.shared.v4.b32 [%0], {%1, %2, %3, %4};"
+                       ::"r"(base + ((c ^ ((lane >> 1) & 3u)) << 4)), "r"(w[0]), "r"(w[1]), "r"(w[2]), "r"(w[3])
+                       : "memory");
+        }
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) tma_store_2d(tmap_c, col0 + (int)(q * 32u), row0, stage_smem + buf * kEpiChunkBytes);
+      }
+    }
+    return;
+  }
 #pragma unroll
   for (uint32_t q = 0; q < kLoads * 2; ++q) {
     if (q * kEpiChunkCols < valid_cols) {
@@ -259,7 +289,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                const __grid_constant__ CUtensorMap tmap_c,
                uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t tx_bytes) {
+               uint32_t group_m, uint32_t tx_bytes, uint32_t c_bf16) {
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -410,7 +440,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // the MMA issuer may overwrite the accumulator
       store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)(tc.tm * BM + quarter * 32), valid_cols, lane);
+                         (int)col0, (int)(tc.tm * BM + quarter * 32), valid_cols, lane, c_bf16);
       if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) bulk_wait_all();  // this warp's stores have completed
@@ -523,7 +553,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
-                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair) {
+                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, uint32_t c_bf16) {
   using cfg = Cfg2<F4>;
   constexpr int BN = cfg::BN;
   constexpr int BKe = cfg::kBKe;
@@ -685,7 +715,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
       store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)(tc.tm * 256 + rank * 128 + quarter * 32), valid_cols, lane);
+                         (int)col0, (int)(tc.tm * 256 + rank * 128 + quarter * 32), valid_cols, lane, c_bf16);
       acc_phase ^= 1u;
     }
     if (lane == 0) bulk_wait_all();
@@ -771,15 +801,15 @@ bool make_scale_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-// Tensor map of the FP32 output [M x N]: box = 16 columns x 32 rows in the 64-byte swizzle the
-// epilogue writes its staging chunks in.
-bool make_c_map(EncodeTiledFn fn, CUtensorMap* map, float* C, uint64_t M, uint64_t N) {
+// Tensor map of the output [M x N] (FP32 or BF16): box = 64 bytes of columns x 32 rows in the
+// 64-byte swizzle the epilogue writes its staging chunks in.
+bool make_c_map(EncodeTiledFn fn, CUtensorMap* map, void* C, uint64_t M, uint64_t N, bool bf16) {
   const cuuint64_t dims[2] = {N, M};
-  const cuuint64_t strides[1] = {N * 4};
-  const cuuint32_t box[2] = {kEpiChunkCols, 32};
+  const cuuint64_t strides[1] = {N * (bf16 ? 2u : 4u)};
+  const cuuint32_t box[2] = {bf16 ? 32u : kEpiChunkCols, 32};
   const cuuint32_t estr[2] = {1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+  return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims,
+            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
@@ -788,7 +818,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
                       uint32_t idesc_base) {
   CUtensorMap mc, msa, msb;
   EncodeTiledFn fn = encode_fn_cached();
-  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) ||
+  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N, a.c_bf16 != 0) ||
       !make_scale_map(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1) ||
       !make_scale_map(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, Cfg<BN>::kSfbChunks))
     return cudaErrorInvalidValue;
@@ -812,7 +842,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
                             cfg::kSfBytes;
   mx_gemm_kernel<BN><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
-      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes);
+      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, (uint32_t)a.c_bf16);
   return cudaGetLastError();
 }
 
@@ -845,7 +875,7 @@ template <bool F4>
 cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   using cfg = Cfg2<F4>;
   CUtensorMap ma, mb, msa, msb, mc;
-  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N) &&
+  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N, a.c_bf16 != 0) &&
             make_scale_map_k(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1, cfg::kKChunks) &&
             make_scale_map_k(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, 2, cfg::kKChunks);
   if (F4)
@@ -876,7 +906,8 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t idesc = (fa << 7) | (fb << 10) | (1u << 23) | ((uint32_t)(256 >> 3) << 17) |
                          ((uint32_t)(256 >> 4) << 24);
   mx_gemm_pair_kernel<F4><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
-      ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair);
+      ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
+      (uint32_t)a.c_bf16);
   return cudaGetLastError();
 }
 

@@ -46,7 +46,8 @@ struct GemmArgs {
   const uint8_t* sA;
   const void* B;
   const uint8_t* sB;
-  float* C;
+  void* C;      // FP32 [M x N], or BF16 when c_bf16 is nonzero
+  int c_bf16;
   int64_t M, N, K;
   int fmtA, fmtB;
   int sm_count;

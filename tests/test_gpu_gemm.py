@@ -284,6 +284,45 @@ def test_kernel_variants_whole_matrix(shape, fa, fb):
     _check_bound(C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].cpu().numpy(), c64, s, shape)
 
 
+@pytest.mark.parametrize("shape,fa,fb", [
+    ((384, 512, 1024), 0, 1),     # one-CTA 128 x 128 tiles
+    ((4736, 8320, 384), 3, 4),    # one-CTA 128 x 256 tiles, ragged last tile
+    ((2048, 9600, 384), 0, 2),    # two-CTA tiles, ragged N
+    ((2048, 9600, 512), 4, 4),    # kind::mxf4
+])
+def test_bf16_output(shape, fa, fb):
+    """mx_gemm_bf16 against the oracle: |C - exact| <= 1e-5 * S + 2^-8 |FP32 value| (half a
+    BF16 ulp: one rounding of the FP32 accumulator, itself within 1e-5 * S of exact), on the whole matrix through an FP64 library
+    product of the oracle-dequantized operands and on samples through the oracle's GEMM; the
+    canary bytes around the output stay intact (a BF16 row is half as long as an FP32 one)."""
+    M, N, K = shape
+    g = torch.Generator(device="cuda").manual_seed(M * 3 + N + K)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.02
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    g_out = Guarded(M * N * 2)
+    C = g_out.view.view(torch.bfloat16).view(M, N)
+    mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy() for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    ref = da @ db.T
+    bound = 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * 2.0 ** -8
+    bad = int(((C.double() - ref).abs() > bound).sum())
+    assert bad == 0, f"{shape}: {bad} outputs beyond the bound"
+    rng = np.random.default_rng(N)
+    ms, ns = rng.integers(0, M, 1000), rng.integers(0, N, 1000)
+    c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * 2.0 ** -8).all()
+    # the BF16 result is the FP32 result of the same kernel rounded once to nearest even
+    C32 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
+    assert torch.equal(C32.to(torch.bfloat16).view(torch.int16), C.view(torch.int16))
+
+
 def test_config3_full_size():
     d = inputs.config3("cuda")
     X, W = d["X"], d["W"]
