@@ -222,6 +222,21 @@ int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t*
                  int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
                  const mx_opts_t* opts);
 
+/*
+ * `batch` independent products in one launch: the matmuls of attention (scores, context)
+ * are dot products like any other (Section 4.1 counts every dot-product operation).
+ * A is the packed [batch x M x K] tensor, B [batch x N x K], C [batch x M x N] (c_dtype:
+ * MX_F32 or MX_BF16), all contiguous; sA / sB are the swizzled scale tensors of the
+ * [batch*M x K] and [batch*N x K] matrices, i.e. what mx_quantize writes for the
+ * 3-D tensors along their last axis.  C[b] = A[b] . B[b]^T as in mx_gemm.
+ * Requirements and errors as mx_gemm (M and N multiples of 128 keep every matrix on
+ * whole scale chunks); additionally MX_ERR_FMT for a bad c_dtype and MX_ERR_SHAPE when
+ * batch < 0 or batch*M or batch*N reaches 2^31.  batch == 0 is a no-op.
+ */
+int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                    mx_dtype_t c_dtype, int64_t batch, int64_t M, int64_t N, int64_t K,
+                    mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts);
+
 /* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */
 /* ------------------------------------------------------------------------- */

@@ -31,7 +31,7 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
-    "mx_gemm_bf16",
+    "mx_gemm_bf16", "mx_gemm_batched",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -76,6 +76,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_dequantize.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op]
     lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_gemm_bf16.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
+    lib.mx_gemm_batched.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
     lib.mx_quantize_host.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op, vp, sz]
@@ -218,6 +219,22 @@ def mx_gemm_bf16(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.T
     o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
     _check(_lib.mx_gemm_bf16(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
                              out.data_ptr(), M, N, K, fmtA, fmtB, ctypes.byref(o)), "mx_gemm_bf16")
+    return out
+
+
+def mx_gemm_batched(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
+                    batch: int, M: int, N: int, K: int, fmtA: int, fmtB: int,
+                    out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.float32,
+                    check_status: bool = False) -> torch.Tensor:
+    """C[b] = A[b] . B[b]^T for b < batch; operands are the MX tensors of [batch, M, K] and
+    [batch, N, K] quantized along K (swizzled scales)."""
+    assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
+    if out is None:
+        out = torch.empty((batch, M, N), dtype=out_dtype, device=A.device)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    _check(_lib.mx_gemm_batched(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
+                                out.data_ptr(), _dtype_code(out.dtype), batch, M, N, K, fmtA, fmtB,
+                                ctypes.byref(o)), "mx_gemm_batched")
     return out
 
 

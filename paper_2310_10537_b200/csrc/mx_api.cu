@@ -367,8 +367,8 @@ static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const 
 }
 
 static int gemm_device(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
-                       int c_bf16, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
-                       const mx_opts_t* opts) {
+                       int c_bf16, int64_t batch, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA,
+                       mx_fmt_t fmtB, const mx_opts_t* opts) {
   Opts o;
   int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB);
   if (rc != MX_OK) return rc;
@@ -377,10 +377,13 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
   if ((uintptr_t)A % 32 || (uintptr_t)B % 32 || (uintptr_t)sA % 16 || (uintptr_t)sB % 16 ||
       (uintptr_t)C % 16)
     return MX_ERR_ALIGN;
-  if (M == 0 || N == 0) return MX_OK;
+  if (batch < 0 || batch * M >= ((int64_t)1 << 31) || batch * N >= ((int64_t)1 << 31) ||
+      (M > 0 && N > 0 && batch * (M / 128) * (N / 128) >= ((int64_t)1 << 31)))
+    return MX_ERR_SHAPE;
+  if (M == 0 || N == 0 || batch == 0) return MX_OK;
   cudaError_t e;
   mx::GemmArgs a;
-  a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16;
+  a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16; a.batch = batch;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
   a.sm_count = sm_count(&e);
@@ -403,13 +406,20 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
 
 int mx_gemm(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, float* C,
             int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
-  return gemm_device(A, sA, B, sB, C, 0, M, N, K, fmtA, fmtB, opts);
+  return gemm_device(A, sA, B, sB, C, 0, 1, M, N, K, fmtA, fmtB, opts);
 }
 
 int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
                  int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
                  const mx_opts_t* opts) {
-  return gemm_device(A, sA, B, sB, C, 1, M, N, K, fmtA, fmtB, opts);
+  return gemm_device(A, sA, B, sB, C, 1, 1, M, N, K, fmtA, fmtB, opts);
+}
+
+int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                    mx_dtype_t c_dtype, int64_t batch, int64_t M, int64_t N, int64_t K,
+                    mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
+  if ((int)c_dtype != MX_F32 && (int)c_dtype != MX_BF16) return MX_ERR_FMT;
+  return gemm_device(A, sA, B, sB, C, (int)c_dtype == MX_BF16, batch, M, N, K, fmtA, fmtB, opts);
 }
 
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {

@@ -262,17 +262,20 @@ __device__ __forceinline__ void store_rows(const uint32_t (&r)[kLoads][32], uint
 }
 
 struct TileCoord {
-  uint32_t tm, tn;
+  uint32_t tm, tn, b;
 };
-// Output tiles are walked in bands of group_m tile rows so that the A band and
-// the B tiles of a wave of CTAs stay in L2.
+// Output tiles are walked batch by batch and, inside a matrix, in bands of group_m tile rows so
+// that the A band and the B tiles of a wave of CTAs stay in L2.
 __device__ __forceinline__ TileCoord tile_coord(uint32_t t, uint32_t tiles_m, uint32_t tiles_n,
                                                 uint32_t group_m) {
+  TileCoord c;
+  const uint32_t per_batch = tiles_m * tiles_n;
+  c.b = t / per_batch;
+  t -= c.b * per_batch;
   const uint32_t per_group = group_m * tiles_n;
   const uint32_t g = t / per_group, r = t - g * per_group;
   const uint32_t first_m = g * group_m;
   const uint32_t gm = min(group_m, tiles_m - first_m);
-  TileCoord c;
   c.tn = r / gm;
   c.tm = first_m + (r - c.tn * gm);
   return c;
@@ -289,7 +292,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                const __grid_constant__ CUtensorMap tmap_c,
                uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t tx_bytes, uint32_t c_bf16) {
+               uint32_t group_m, uint32_t tx_bytes, uint32_t c_bf16, uint32_t batch) {
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -304,7 +307,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
+  const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
   const uint32_t k_chunks = K / BK;
 
   if (threadIdx.x == 0) {
@@ -345,10 +348,12 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        // operands: (k, row, 0); scales: (0, k chunk, 128-row group).  Rows or groups past the end
-        // of B on a ragged last tile are zero-filled by the copy.
-        const int cy_fixed = lane == 0 ? (int)(tc.tm * BM) : (int)(tc.tn * BN);
-        const int cz = lane == 2 ? (int)tc.tm : lane == 3 ? (int)(tc.tn * BN / 128) : 0;
+        // operands: (k, row, 0); scales: (0, k chunk, 128-row group), rows counted through the
+        // whole batch.  Rows or groups past the end of a B matrix on a ragged last tile belong to
+        // the next matrix of the batch or are zero-filled by the copy; their columns are not stored.
+        const int cy_fixed = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * BM) : (int)(tc.b * N + tc.tn * BN);
+        const int cz = lane == 2 ? (int)(tc.b * tiles_m + tc.tm)
+                                 : lane == 3 ? (int)((tc.b * N + tc.tn * BN) / 128) : 0;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
@@ -440,7 +445,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // the MMA issuer may overwrite the accumulator
       store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)(tc.tm * BM + quarter * 32), valid_cols, lane, c_bf16);
+                         (int)col0, (int)((tc.b * tiles_m + tc.tm) * BM + quarter * 32), valid_cols, lane, c_bf16);
       if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) bulk_wait_all();  // this warp's stores have completed
@@ -553,7 +558,8 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
-                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, uint32_t c_bf16) {
+                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, uint32_t c_bf16,
+                    uint32_t batch) {
   using cfg = Cfg2<F4>;
   constexpr int BN = cfg::BN;
   constexpr int BKe = cfg::kBKe;
@@ -573,7 +579,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = tiles_m * tiles_n;
+  const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
   const uint32_t k_chunks = K / BKe;
 
   if (threadIdx.x == 0) {
@@ -616,8 +622,10 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
         // this CTA's 128 rows of A and of B (B rows may lie past N on a ragged tile: zero fill);
         // its own A scales and the B scales of all 256 columns
-        const int cy_fixed = lane == 0 ? (int)(tc.tm * 256 + rank * 128) : (int)(tc.tn * BN + rank * 128);
-        const int cz = lane == 2 ? (int)(tc.tm * 2 + rank) : lane == 3 ? (int)(tc.tn * 2) : 0;
+        const int cy_fixed = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
+                                       : (int)(tc.b * N + tc.tn * BN + rank * 128);
+        const int cz = lane == 2 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
+                                 : lane == 3 ? (int)(tc.b * (N / 128) + tc.tn * 2) : 0;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
@@ -715,7 +723,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
       store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)(tc.tm * 256 + rank * 128 + quarter * 32), valid_cols, lane, c_bf16);
+                         (int)col0, (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128 + quarter * 32), valid_cols, lane,
+                         c_bf16);
       acc_phase ^= 1u;
     }
     if (lane == 0) bulk_wait_all();
@@ -818,9 +827,9 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
                       uint32_t idesc_base) {
   CUtensorMap mc, msa, msb;
   EncodeTiledFn fn = encode_fn_cached();
-  if (!make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N, a.c_bf16 != 0) ||
-      !make_scale_map(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1) ||
-      !make_scale_map(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, Cfg<BN>::kSfbChunks))
+  if (!make_c_map(fn, &mc, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0) ||
+      !make_scale_map(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1) ||
+      !make_scale_map(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, Cfg<BN>::kSfbChunks))
     return cudaErrorInvalidValue;
   using cfg = Cfg<BN>;
   static bool attr_set[64] = {false};
@@ -833,7 +842,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)(a.M / BM) * (uint32_t)((a.N + BN - 1) / BN);
+  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / BM) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
   const uint32_t group_m = 16;
   // Bytes the producer's copies report to a stage's mbarrier: the tensor-map copies count the
@@ -842,7 +851,8 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
                             cfg::kSfBytes;
   mx_gemm_kernel<BN><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
-      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, (uint32_t)a.c_bf16);
+      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, (uint32_t)a.c_bf16,
+      (uint32_t)a.batch);
   return cudaGetLastError();
 }
 
@@ -875,15 +885,15 @@ template <bool F4>
 cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   using cfg = Cfg2<F4>;
   CUtensorMap ma, mb, msa, msb, mc;
-  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)a.M, (uint64_t)a.N, a.c_bf16 != 0) &&
-            make_scale_map_k(fn, &msa, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1, cfg::kKChunks) &&
-            make_scale_map_k(fn, &msb, a.sB, (uint64_t)a.N, (uint64_t)a.K, 2, cfg::kKChunks);
+  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0) &&
+            make_scale_map_k(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1, cfg::kKChunks) &&
+            make_scale_map_k(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 2, cfg::kKChunks);
   if (F4)
-    ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)a.M, (uint64_t)a.K) &&
-         make_f4_map(fn, &mb, a.B, (uint64_t)a.N, (uint64_t)a.K);
+    ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K) &&
+         make_f4_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K);
   else
-    ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, 128) &&
-         make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, 128);
+    ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
+         make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
   if (!ok) return cudaErrorInvalidValue;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -895,7 +905,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
+  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
   const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
   const uint32_t op_bytes = F4 ? 2u * 128u * 128u
@@ -907,7 +917,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
                          ((uint32_t)(256 >> 4) << 24);
   mx_gemm_pair_kernel<F4><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
-      (uint32_t)a.c_bf16);
+      (uint32_t)a.c_bf16, (uint32_t)a.batch);
   return cudaGetLastError();
 }
 
@@ -919,18 +929,18 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   if (!fn) return MX_ERR_CUDA;
   // 256-wide tiles move the fewest operand bytes through shared memory per flop; problems with
   // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
-  const int64_t tiles256 = (a.M / BM) * ((a.N + 255) / 256);
+  const int64_t tiles256 = a.batch * (a.M / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
   // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
-  if (a.M % 256 == 0 && (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
+  if (a.M % 256 == 0 && a.batch * (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
     const bool f4 = a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
     *cuda_err = f4 ? launch_pair<true>(a, fn) : launch_pair<false>(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
   CUtensorMap ma, mb;
-  if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, BM) ||
-      !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, (uint32_t)bn)) {
+  if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, BM) ||
+      !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, (uint32_t)bn)) {
     *cuda_err = cudaErrorInvalidValue;
     return MX_ERR_CUDA;
   }

@@ -48,6 +48,7 @@ struct GemmArgs {
   const uint8_t* sB;
   void* C;      // FP32 [M x N], or BF16 when c_bf16 is nonzero
   int c_bf16;
+  int64_t batch;  // independent products; operands and C are the matrices stacked along rows
   int64_t M, N, K;
   int fmtA, fmtB;
   int sm_count;

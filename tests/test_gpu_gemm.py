@@ -323,6 +323,58 @@ def test_bf16_output(shape, fa, fb):
     assert torch.equal(C32.to(torch.bfloat16).view(torch.int16), C.view(torch.int16))
 
 
+@pytest.mark.parametrize("batch,M,N,K,fa,fb,dt", [
+    (24, 512, 512, 128, 0, 0, torch.float32),    # attention scores S x S over d = 128: two-CTA tiles
+    (5, 384, 640, 256, 1, 3, torch.float32),     # one-CTA 128 x 128 tiles
+    (40, 384, 640, 256, 0, 4, torch.float32),    # one-CTA 128 x 256 tiles, ragged tile reaching into the next matrix
+    (30, 256, 384, 256, 4, 4, torch.bfloat16),   # kind::mxf4 pairs, ragged N, BF16 out
+    (1, 256, 256, 128, 2, 2, torch.float32),
+])
+def test_batched(batch, M, N, K, fa, fb, dt):
+    """mx_gemm_batched: every matrix of the batch against the oracle (the first and the last in
+    full through the oracle's GEMM, all of them through an FP64 library product of the
+    oracle-dequantized operands)."""
+    g = torch.Generator(device="cuda").manual_seed(batch + M + N + K)
+    A = torch.randn((batch, M, K), generator=g, device="cuda") * torch.exp(torch.randn((batch, M, 1), generator=g, device="cuda"))
+    B = torch.randn((batch, N, K), generator=g, device="cuda") * torch.exp(torch.randn((batch, 1, 1), generator=g, device="cuda"))
+    ea, sa = mx.mx_quantize(A, 2, fa)
+    eb, sb = mx.mx_quantize(B, 2, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(batch * M * N * esz)
+    C = g_out.view.view(dt).view(batch, M, N)
+    mx.mx_gemm_batched(ea, sa, eb, sb, batch, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, batch * M, K, fa, O.F64)).cuda().view(batch, M, K)
+    db = torch.from_numpy(O.dequantize(heb, hsb, batch * N, K, fb, O.F64)).cuda().view(batch, N, K)
+    ref = da @ db.transpose(1, 2)
+    S = da.abs() @ db.abs().transpose(1, 2)
+    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
+    bad = int(((C.double() - ref).abs() > 1.004 * TOL * S + ref.abs() * rel).sum())
+    assert bad == 0, f"{bad} outputs beyond the bound"
+    abytes, bbytes = M * K * O.fmt_bits(fa) // 8, N * K * O.fmt_bits(fb) // 8
+    for b in {0, batch - 1}:
+        c64, s = O.gemm(hea[b * abytes:(b + 1) * abytes], hsa[b * M * K // 32:(b + 1) * M * K // 32],
+                        heb[b * bbytes:(b + 1) * bbytes], hsb[b * N * K // 32:(b + 1) * N * K // 32],
+                        M, N, K, fa, fb)
+        got = C[b].double().cpu().numpy()
+        assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all(), f"matrix {b}"
+
+
+def test_batched_errors():
+    z = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    out = torch.full((4,), 7.0, device="cuda")
+    with pytest.raises(mx.MxError) as e:
+        mx.mx_gemm_batched(z, z, z, z, -1, 128, 128, 128, 0, 0, out=out)
+    assert e.value.status == mx.MX_ERR_SHAPE
+    with pytest.raises(mx.MxError) as e:
+        mx.mx_gemm_batched(z, z, z, z, 1 << 24, 128, 128, 128, 0, 0, out=out)
+    assert e.value.status == mx.MX_ERR_SHAPE
+    mx.mx_gemm_batched(z, z, z, z, 0, 128, 128, 128, 0, 0, out=out)   # batch 0: nothing written
+    assert (out == 7.0).all()
+
+
 def test_config3_full_size():
     d = inputs.config3("cuda")
     X, W = d["X"], d["W"]
