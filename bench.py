@@ -265,6 +265,31 @@ def run_extras(torch, mx, inputs):
     out["mxfp4_x_mxfp4_same_shape_kind_mxf4"] = {"gemm_TFLOPs": 2.0 * M * N * K / t4 / 1e12, "gemm_ms": t4 * 1e3}
     del d, W, X, C, ea, sa, eb, sb, ea4, sa4
     torch.cuda.empty_cache()
+    # two chained products (configs[2] shape): the first one's result requantized to MXFP8 for the next
+    d = inputs.config3("cuda")
+    X, W = d["X"], d["W"]
+    M, K = X.shape
+    N = W.shape[1]
+    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(W, 0, mx.MX_E4M3)
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    qe, qs = mx.mx_quantize(C, 1, mx.MX_E4M3)
+
+    def gemm_then_quantize():
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=C)
+        mx.mx_quantize(C, 1, mx.MX_E4M3, out=(qe, qs))
+
+    t2 = timed(gemm_then_quantize, 10)
+    t1 = timed(lambda: mx.mx_gemm_quantize(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, mx.MX_E4M3,
+                                           mx.MX_RNE, elems=qe, scales=qs), 10)
+    Cb = torch.empty((M, N), dtype=torch.bfloat16, device="cuda")
+    tb = timed(lambda: mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=Cb), 10)
+    out["config3_gemm_output_variants"] = {
+        "ms_gemm_fp32_then_quantize_e4m3": t2 * 1e3, "ms_gemm_with_quantizing_epilogue": t1 * 1e3,
+        "quantizing_epilogue_TFLOPs": 2.0 * M * N * K / t1 / 1e12,
+        "ms_gemm_bf16_out": tb * 1e3, "bf16_out_TFLOPs": 2.0 * M * N * K / tb / 1e12}
+    del d, W, X, C, Cb, ea, sa, eb, sb, qe, qs
+    torch.cuda.empty_cache()
     d = inputs.config4("cuda")
     Xc, Wc, dY = d["X"], d["W"], d["dY"]
     n = Xc.shape[0]

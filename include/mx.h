@@ -237,6 +237,24 @@ int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8
                     mx_dtype_t c_dtype, int64_t batch, int64_t M, int64_t N, int64_t K,
                     mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts);
 
+/*
+ * mx_gemm whose epilogue quantizes the result instead of storing it: in the paper's compute
+ * flow (Section 4.1) the output of one dot-product operation is requantized to MX before it
+ * enters the next one, and when nothing runs in between that pass over C need not touch
+ * memory.  Each FP32 accumulator row is cut into blocks of 32 consecutive columns and
+ * converted by Algorithm 1 (Section 3) while it is still in registers.
+ *   elems_out / scales_out   exactly what mx_quantize(C, shape {M, N}, axis 1, fmtC, rounding)
+ *                            writes for the FP32 C that mx_gemm produces from the same
+ *                            operands: packed codes [M x N] (N innermost) and the SWIZZLED
+ *                            scale tensor of M rows x N/32 blocks -- the A operand of a
+ *                            following mx_gemm whose K is this N.  Any format, MX_INT8 included.
+ * elems_out and scales_out 16-byte aligned.  Other requirements and errors as mx_gemm.
+ */
+int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
+                     void* elems_out, uint8_t* scales_out, int64_t M, int64_t N, int64_t K,
+                     mx_fmt_t fmtA, mx_fmt_t fmtB, mx_fmt_t fmtC, mx_round_t rounding,
+                     const mx_opts_t* opts);
+
 /* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */
 /* ------------------------------------------------------------------------- */

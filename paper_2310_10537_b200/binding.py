@@ -31,7 +31,7 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
-    "mx_gemm_bf16", "mx_gemm_batched",
+    "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -76,6 +76,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_dequantize.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op]
     lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_gemm_bf16.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
+    lib.mx_gemm_quantize.argtypes = [vp, u8p, vp, u8p, vp, u8p, i64, i64, i64, ci, ci, ci, ci, op]
     lib.mx_gemm_batched.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
@@ -236,6 +237,25 @@ def mx_gemm_batched(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torc
                                 out.data_ptr(), _dtype_code(out.dtype), batch, M, N, K, fmtA, fmtB,
                                 ctypes.byref(o)), "mx_gemm_batched")
     return out
+
+
+def mx_gemm_quantize(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
+                     M: int, N: int, K: int, fmtA: int, fmtB: int, fmtC: int, rounding: int = MX_RNE,
+                     elems: Optional[torch.Tensor] = None, scales: Optional[torch.Tensor] = None,
+                     check_status: bool = False) -> Tuple[torch.Tensor, torch.Tensor]:
+    """A . B^T quantized along N in the GEMM epilogue: the MX tensor (codes, swizzled scales)
+    mx_quantize would produce from the FP32 result."""
+    assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
+    if elems is None:
+        elems = torch.empty(M * N * mx_fmt_bits(fmtC) // 8, dtype=torch.uint8, device=A.device)
+    if scales is None:
+        scales = torch.empty(mx_scales_bytes((M, N), 1, MX_SCALES_SWIZZLED), dtype=torch.uint8,
+                             device=A.device)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    _check(_lib.mx_gemm_quantize(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
+                                 elems.data_ptr(), scales.data_ptr(), M, N, K, fmtA, fmtB, fmtC,
+                                 rounding, ctypes.byref(o)), "mx_gemm_quantize")
+    return elems, scales
 
 
 # ---- host-buffer variants: tensors live in (pinned) host memory ----------------

@@ -366,10 +366,16 @@ static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const 
   return MX_OK;
 }
 
+// C != NULL: scalar-float output; otherwise q_elems / q_scales receive C as an MX tensor.
 static int gemm_device(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
                        int c_bf16, int64_t batch, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA,
-                       mx_fmt_t fmtB, const mx_opts_t* opts) {
+                       mx_fmt_t fmtB, const mx_opts_t* opts, void* q_elems = nullptr,
+                       uint8_t* q_scales = nullptr, int q_fmt = 0, int q_round = 0) {
   Opts o;
+  if (!C) {
+    if (!q_elems || !q_scales) return MX_ERR_NULL;
+    C = q_elems;  // stands in for the output pointer in the checks below
+  }
   int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB);
   if (rc != MX_OK) return rc;
   if (!read_opts(opts, &o)) return MX_ERR_FMT;
@@ -384,6 +390,7 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
   cudaError_t e;
   mx::GemmArgs a;
   a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16; a.batch = batch;
+  a.q_elems = q_elems; a.q_scales = q_scales; a.q_fmt = q_fmt; a.q_round = q_round;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
   a.sm_count = sm_count(&e);
@@ -420,6 +427,17 @@ int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8
                     mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts) {
   if ((int)c_dtype != MX_F32 && (int)c_dtype != MX_BF16) return MX_ERR_FMT;
   return gemm_device(A, sA, B, sB, C, (int)c_dtype == MX_BF16, batch, M, N, K, fmtA, fmtB, opts);
+}
+
+int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
+                     void* elems_out, uint8_t* scales_out, int64_t M, int64_t N, int64_t K,
+                     mx_fmt_t fmtA, mx_fmt_t fmtB, mx_fmt_t fmtC, mx_round_t rounding,
+                     const mx_opts_t* opts) {
+  if (!elems_out || !scales_out) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmtC) || ((int)rounding != MX_RNE && (int)rounding != MX_RHAZ)) return MX_ERR_FMT;
+  if ((uintptr_t)scales_out % 16) return MX_ERR_ALIGN;
+  return gemm_device(A, sA, B, sB, nullptr, 0, 1, M, N, K, fmtA, fmtB, opts, elems_out, scales_out,
+                     (int)fmtC, (int)rounding);
 }
 
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {

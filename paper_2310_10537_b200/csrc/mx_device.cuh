@@ -153,19 +153,11 @@ __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
   return p;
 }
 
-// Convert 8 consecutive elements of one block.  Output bit stream (little
-// endian): 8-bit formats lo = codes 0..3, hi = codes 4..7; 6-bit formats lo =
+// Packs the four code pairs of 8 consecutive elements (cast_pair results) into the block's
+// little-endian bit stream: 8-bit formats lo = codes 0..3, hi = codes 4..7; 6-bit formats lo =
 // bits 0..31, hi = bits 32..47; 4-bit format lo = all 32 bits.
-template <int FMT, int ROUND>
-__device__ __forceinline__ void cast8(const float (&v)[8], const BlockScale& s, uint32_t& lo,
-                                      uint32_t& hi) {
-  uint32_t p[4];
-#pragma unroll
-  for (int i = 0; i < 4; ++i) {
-    float a = mul_ftz(v[2 * i], s.m1), b = mul_ftz(v[2 * i + 1], s.m1);
-    if (FMT == MX_INT8) { a *= s.m2; b *= s.m2; }
-    p[i] = cast_pair<FMT, ROUND>(a, b);
-  }
+template <int FMT>
+__device__ __forceinline__ void pack8(const uint32_t (&p)[4], uint32_t& lo, uint32_t& hi) {
   constexpr int bits = FmtTraits<FMT>::bits;
   if (bits == 8) {
     lo = __byte_perm(p[0], p[1], 0x5410);
@@ -180,6 +172,20 @@ __device__ __forceinline__ void cast8(const float (&v)[8], const BlockScale& s, 
     lo = q[0] | (q[1] << 12) | (q[2] << 24);
     hi = (q[2] >> 8) | (q[3] << 4);
   }
+}
+
+// Convert 8 consecutive elements of one block (output as pack8).
+template <int FMT, int ROUND>
+__device__ __forceinline__ void cast8(const float (&v)[8], const BlockScale& s, uint32_t& lo,
+                                      uint32_t& hi) {
+  uint32_t p[4];
+#pragma unroll
+  for (int i = 0; i < 4; ++i) {
+    float a = mul_ftz(v[2 * i], s.m1), b = mul_ftz(v[2 * i + 1], s.m1);
+    if (FMT == MX_INT8) { a *= s.m2; b *= s.m2; }
+    p[i] = cast_pair<FMT, ROUND>(a, b);
+  }
+  pack8<FMT>(p, lo, hi);
   if (!s.finite) { lo = 0; hi = 0; }
 }
 

@@ -25,6 +25,7 @@
 #include <cstring>
 
 #include "mx.h"
+#include "mx_device.cuh"
 #include "mx_launch.h"
 
 namespace mx {
@@ -261,6 +262,92 @@ __device__ __forceinline__ void store_rows(const uint32_t (&r)[kLoads][32], uint
   }
 }
 
+// What the epilogue does with a tile.
+struct EpiArgs {
+  uint32_t mode;     // 0: FP32 C through tmap_c, 1: BF16 C through tmap_c, 2: C as an MX tensor
+  uint32_t fmt;      // mode 2: element format of the output
+  uint32_t sticky;   // mode 2: 1 = ties away from zero (see cast_pair), 0 = ties to even
+  uint8_t* elems;    // mode 2: packed codes [rows x N], blocks along N
+  uint8_t* scales;   // mode 2: swizzled scale tensor, rows x N / 32
+};
+
+// Quantizes this thread's kLoads blocks of 32 consecutive columns of row `row` (Algorithm 1 on the
+// FP32 accumulators, the same helpers as the quantize kernels) and writes their codes and scale
+// bytes; col0 is a multiple of 32 * kLoads.
+template <int FMT, uint32_t kLoads>
+__device__ __forceinline__ void store_mx_fmt(const uint32_t (&r)[kLoads][32], const EpiArgs& epi,
+                                             uint32_t row, uint32_t col0, uint32_t N) {
+  constexpr uint32_t W = FmtTraits<FMT>::bits;  // 32-bit words of codes per block
+  uint32_t w[kLoads * W];
+  uint32_t sword = 0;
+#pragma unroll
+  for (uint32_t j = 0; j < kLoads; ++j) {
+    float m[16];
+#pragma unroll
+    for (int i = 0; i < 16; ++i) m[i] = absmax_nan(__uint_as_float(r[j][2 * i]), __uint_as_float(r[j][2 * i + 1]));
+#pragma unroll
+    for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+      for (int i = 0; i < n; ++i) m[i] = absmax_nan(m[i], m[i + n]);
+    const BlockScale bs = block_scale<FMT>(m[0]);
+    sword |= bs.byte << (8 * j);
+    uint32_t lo[4], hi[4];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      uint32_t p[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        float a = mul_ftz(__uint_as_float(r[j][8 * g + 2 * i]), bs.m1);
+        float b = mul_ftz(__uint_as_float(r[j][8 * g + 2 * i + 1]), bs.m1);
+        if (FMT == MX_INT8) { a *= bs.m2; b *= bs.m2; }
+        a = __uint_as_float(__float_as_uint(a) | epi.sticky);
+        b = __uint_as_float(__float_as_uint(b) | epi.sticky);
+        p[i] = cast_pair<FMT, MX_RNE>(a, b);
+      }
+      pack8<FMT>(p, lo[g], hi[g]);
+      if (!bs.finite) { lo[g] = 0; hi[g] = 0; }
+    }
+    if (W == 8) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) { w[8 * j + 2 * g] = lo[g]; w[8 * j + 2 * g + 1] = hi[g]; }
+    } else if (W == 4) {
+#pragma unroll
+      for (int g = 0; g < 4; ++g) w[4 * j + g] = lo[g];
+    } else {  // 8 codes = 48 bits: two groups fill three words
+      w[6 * j + 0] = lo[0];
+      w[6 * j + 1] = __byte_perm(hi[0], lo[1], 0x5410);
+      w[6 * j + 2] = __byte_perm(lo[1], hi[1], 0x5432);
+      w[6 * j + 3] = lo[2];
+      w[6 * j + 4] = __byte_perm(hi[2], lo[3], 0x5410);
+      w[6 * j + 5] = __byte_perm(lo[3], hi[3], 0x5432);
+    }
+  }
+  uint8_t* dst = epi.elems + ((size_t)row * N + col0) / 8 * W;
+#pragma unroll
+  for (uint32_t i = 0; i < kLoads * W / 4; ++i)
+    *reinterpret_cast<uint4*>(dst + 16 * i) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  // swizzled scale layout: the kLoads scale bytes of this row are adjacent inside one 512-byte chunk
+  const uint32_t kb = col0 / 32;
+  uint8_t* sp = epi.scales + ((size_t)(row / 128) * (N / 128) + kb / 4) * 512 + (row % 32) * 16 +
+                ((row % 128) / 32) * 4 + kb % 4;
+  if (kLoads == 4) *reinterpret_cast<uint32_t*>(sp) = sword;
+  else *reinterpret_cast<uint16_t*>(sp) = (uint16_t)sword;
+}
+
+template <uint32_t kLoads>
+__device__ __forceinline__ void store_mx_rows(const uint32_t (&r)[kLoads][32], const EpiArgs& epi,
+                                              uint32_t row, uint32_t col0, uint32_t N) {
+  static_assert(kLoads == 2 || kLoads == 4, "two or four blocks per thread");
+  switch (epi.fmt) {
+    case MX_E4M3: store_mx_fmt<MX_E4M3, kLoads>(r, epi, row, col0, N); break;
+    case MX_E5M2: store_mx_fmt<MX_E5M2, kLoads>(r, epi, row, col0, N); break;
+    case MX_E3M2: store_mx_fmt<MX_E3M2, kLoads>(r, epi, row, col0, N); break;
+    case MX_E2M3: store_mx_fmt<MX_E2M3, kLoads>(r, epi, row, col0, N); break;
+    case MX_E2M1: store_mx_fmt<MX_E2M1, kLoads>(r, epi, row, col0, N); break;
+    default: store_mx_fmt<MX_INT8, kLoads>(r, epi, row, col0, N); break;
+  }
+}
+
 struct TileCoord {
   uint32_t tm, tn, b;
 };
@@ -292,7 +379,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                const __grid_constant__ CUtensorMap tmap_c,
                uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t tx_bytes, uint32_t c_bf16, uint32_t batch) {
+               uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch) {
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -444,8 +531,13 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // the MMA issuer may overwrite the accumulator
-      store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)((tc.b * tiles_m + tc.tm) * BM + quarter * 32), valid_cols, lane, c_bf16);
+      const uint32_t row0 = (tc.b * tiles_m + tc.tm) * BM + quarter * 32;
+      if (epi.mode == 2) {
+        if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
+      } else {
+        store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                           (int)col0, (int)row0, valid_cols, lane, epi.mode);
+      }
       if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
     if (lane == 0) bulk_wait_all();  // this warp's stores have completed
@@ -558,7 +650,7 @@ __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
-                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, uint32_t c_bf16,
+                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
                     uint32_t batch) {
   using cfg = Cfg2<F4>;
   constexpr int BN = cfg::BN;
@@ -722,9 +814,13 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
-      store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                         (int)col0, (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128 + quarter * 32), valid_cols, lane,
-                         c_bf16);
+      const uint32_t row0 = (tc.b * tiles_m + tc.tm) * 256 + rank * 128 + quarter * 32;
+      if (epi.mode == 2) {
+        if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
+      } else {
+        store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                           (int)col0, (int)row0, valid_cols, lane, epi.mode);
+      }
       acc_phase ^= 1u;
     }
     if (lane == 0) bulk_wait_all();
@@ -822,12 +918,29 @@ bool make_c_map(EncodeTiledFn fn, CUtensorMap* map, void* C, uint64_t M, uint64_
             CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// The output map the kernels take.  A quantizing epilogue writes with plain stores and never uses
+// it; it still gets a valid map (over the code tensor) because the kernel prefetches the descriptor.
+bool make_out_map(EncodeTiledFn fn, CUtensorMap* map, const GemmArgs& a) {
+  if (a.q_elems) return make_c_map(fn, map, a.q_elems, (uint64_t)(a.batch * a.M), (uint64_t)a.N / 4, true);
+  return make_c_map(fn, map, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0);
+}
+
+EpiArgs epi_args(const GemmArgs& a) {
+  EpiArgs e;
+  e.mode = a.q_elems ? 2u : (a.c_bf16 ? 1u : 0u);
+  e.fmt = (uint32_t)a.q_fmt;
+  e.sticky = a.q_round == MX_RHAZ ? 1u : 0u;
+  e.elems = (uint8_t*)a.q_elems;
+  e.scales = a.q_scales;
+  return e;
+}
+
 template <int BN>
 cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb,
                       uint32_t idesc_base) {
   CUtensorMap mc, msa, msb;
   EncodeTiledFn fn = encode_fn_cached();
-  if (!make_c_map(fn, &mc, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0) ||
+  if (!make_out_map(fn, &mc, a) ||
       !make_scale_map(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1) ||
       !make_scale_map(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, Cfg<BN>::kSfbChunks))
     return cudaErrorInvalidValue;
@@ -851,7 +964,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
                             cfg::kSfBytes;
   mx_gemm_kernel<BN><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
-      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, (uint32_t)a.c_bf16,
+      idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, epi_args(a),
       (uint32_t)a.batch);
   return cudaGetLastError();
 }
@@ -885,7 +998,7 @@ template <bool F4>
 cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   using cfg = Cfg2<F4>;
   CUtensorMap ma, mb, msa, msb, mc;
-  bool ok = make_c_map(fn, &mc, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0) &&
+  bool ok = make_out_map(fn, &mc, a) &&
             make_scale_map_k(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1, cfg::kKChunks) &&
             make_scale_map_k(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 2, cfg::kKChunks);
   if (F4)
@@ -917,7 +1030,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
                          ((uint32_t)(256 >> 4) << 24);
   mx_gemm_pair_kernel<F4><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
-      (uint32_t)a.c_bf16, (uint32_t)a.batch);
+      epi_args(a), (uint32_t)a.batch);
   return cudaGetLastError();
 }
 

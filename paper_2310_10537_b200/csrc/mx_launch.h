@@ -48,6 +48,11 @@ struct GemmArgs {
   const uint8_t* sB;
   void* C;      // FP32 [M x N], or BF16 when c_bf16 is nonzero
   int c_bf16;
+  // When q_elems is set the epilogue quantizes C along N instead of storing it: packed codes
+  // [batch*M x N] and swizzled scales (rows batch*M, N / 32 blocks); C is then unused.
+  void* q_elems;
+  uint8_t* q_scales;
+  int q_fmt, q_round;
   int64_t batch;  // independent products; operands and C are the matrices stacked along rows
   int64_t M, N, K;
   int fmtA, fmtB;

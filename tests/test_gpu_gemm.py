@@ -375,6 +375,77 @@ def test_batched_errors():
     assert (out == 7.0).all()
 
 
+@pytest.mark.parametrize("shape,fa,fb", [
+    ((256, 512, 512), 0, 0),       # below the two-CTA threshold: one-CTA 128 x 128 tiles, two blocks per thread
+    ((4736, 1024, 128), 1, 3),     # one-CTA 128 x 256 tiles
+    ((2048, 2560, 256), 0, 2),     # two-CTA 256 x 256 tiles
+    ((2048, 2560, 256), 4, 4),     # kind::mxf4
+])
+@pytest.mark.parametrize("fc,rounding", [(0, 0), (1, 1), (2, 0), (3, 1), (4, 0), (4, 1), (5, 0), (5, 1)])
+def test_gemm_quantize_exact_operands(shape, fa, fb, fc, rounding):
+    """mx_gemm_quantize against the oracle chain quantize -> gemm -> quantize, bit for bit, on
+    operands whose dot products are exact in FP32 (so both sides quantize the same numbers; the
+    results are integers of up to 15 bits, full of rounding ties for every element format)."""
+    M, N, K = shape
+    rng = np.random.default_rng(M + N + K + fa)
+    rowexp = np.exp2(rng.integers(-1, 2, (M, 1))).astype(np.float32)
+    A = rng.integers(-3, 4, (M, K)).astype(np.float32)
+    B = rng.integers(-3, 4, (N, K)).astype(np.float32)
+    A[:, ::32] = 3.0   # every block holds a 3: one shared exponent per row, every value kept exactly
+    B[:, ::32] = -3.0
+    A *= rowexp
+    oa, osa = O.quantize(A, 1, fa)
+    ob, osb = O.quantize(B, 1, fb)
+    assert np.array_equal(O.dequantize(oa, osa, M, K, fa, O.F64), A.astype(np.float64))
+    assert np.array_equal(O.dequantize(ob, osb, N, K, fb, O.F64), B.astype(np.float64))
+    c64, _ = O.gemm(oa, osa, ob, osb, M, N, K, fa, fb)
+    c32 = c64.astype(np.float32)
+    assert np.array_equal(c32.astype(np.float64), c64)
+    want_e, want_s = O.quantize(c32, 1, fc, rounding)
+
+    ea, sa = mx.mx_quantize(torch.from_numpy(A).cuda(), 1, fa)
+    eb, sb = mx.mx_quantize(torch.from_numpy(B).cuda(), 1, fb)
+    assert np.array_equal(ea.cpu().numpy().reshape(-1), oa) and np.array_equal(sa.cpu().numpy().reshape(-1), osa)
+    assert np.array_equal(eb.cpu().numpy().reshape(-1), ob) and np.array_equal(sb.cpu().numpy().reshape(-1), osb)
+    ge = Guarded(want_e.size)
+    gs = Guarded(want_s.size)
+    mx.mx_gemm_quantize(ea, sa, eb, sb, M, N, K, fa, fb, fc, rounding, elems=ge.view, scales=gs.view,
+                        check_status=True)
+    torch.cuda.synchronize()
+    ge.check()
+    gs.check()
+    assert np.array_equal(gs.view.cpu().numpy(), want_s), "scale bytes"
+    got = ge.view.cpu().numpy()
+    if not np.array_equal(got, want_e):
+        i = int(np.flatnonzero(got != want_e)[0])
+        raise AssertionError(f"{int((got != want_e).sum())} code bytes differ, first at byte {i}: "
+                             f"got {got[i]:#x} want {want_e[i]:#x}")
+
+
+@pytest.mark.parametrize("fc,rounding", [(0, 0), (2, 1), (4, 0), (5, 1)])
+def test_gemm_quantize_equals_gemm_then_quantize(fc, rounding):
+    """On general operands the fused call writes, bit for bit, what mx_quantize makes of mx_gemm's
+    FP32 result (each of those two is checked against the oracle on its own); special values
+    included: a NaN scale in A poisons a row of C, whose blocks must come out as scale 0xFF."""
+    M, N, K = 2048, 2304, 512
+    g = torch.Generator(device="cuda").manual_seed(7 + fc)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(2 * torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * torch.exp(torch.randn((N, 1), generator=g, device="cuda"))
+    A[5, 40] = float("nan")
+    A[300:302] = 0.0            # zero rows of C: zero blocks
+    ea, sa = mx.mx_quantize(A, 1, 0)
+    eb, sb = mx.mx_quantize(B, 1, 1)
+    C = mx.mx_gemm(ea, sa, eb, sb, M, N, K, 0, 1, check_status=True)
+    assert bool(torch.isnan(C[5]).all())
+    we, ws = mx.mx_quantize(C, 1, fc, rounding)
+    fe, fs = mx.mx_gemm_quantize(ea, sa, eb, sb, M, N, K, 0, 1, fc, rounding, check_status=True)
+    assert torch.equal(fs.view(-1), ws.view(-1))
+    assert torch.equal(fe.view(-1), we.view(-1))
+    # and the oracle's quantization of that same FP32 matrix
+    oe, osc = O.quantize(C.cpu().numpy(), 1, fc, rounding)
+    assert np.array_equal(fe.cpu().numpy().reshape(-1), oe) and np.array_equal(fs.cpu().numpy().reshape(-1), osc)
+
+
 def test_config3_full_size():
     d = inputs.config3("cuda")
     X, W = d["X"], d["W"]
