@@ -288,7 +288,15 @@ def run_extras(torch, mx, inputs):
         "ms_gemm_fp32_then_quantize_e4m3": t2 * 1e3, "ms_gemm_with_quantizing_epilogue": t1 * 1e3,
         "quantizing_epilogue_TFLOPs": 2.0 * M * N * K / t1 / 1e12,
         "ms_gemm_bf16_out": tb * 1e3, "bf16_out_TFLOPs": 2.0 * M * N * K / tb / 1e12}
-    del d, W, X, C, Cb, ea, sa, eb, sb, qe, qs
+    # MXINT8 x MXINT8 on the same shape: dequantize to BF16 + dense BF16 tensor-core GEMM
+    ea8, sa8 = mx.mx_quantize(X, 1, mx.MX_INT8)
+    eb8, sb8 = mx.mx_quantize(W, 0, mx.MX_INT8)
+    ws = torch.empty(mx.mx_gemm_dense_workspace_bytes(M, N, K), dtype=torch.uint8, device="cuda")
+    t8 = timed(lambda: mx.mx_gemm_dense(ea8, sa8, eb8, sb8, M, N, K, mx.MX_INT8, mx.MX_INT8,
+                                        workspace=ws, out=C), 10)
+    out["config3_mxint8_x_mxint8_bf16_route"] = {
+        "ms_two_dequantizes_and_dense_gemm": t8 * 1e3, "TFLOPs": 2.0 * M * N * K / t8 / 1e12}
+    del d, W, X, C, Cb, ea, sa, eb, sb, qe, qs, ea8, sa8, eb8, sb8, ws
     torch.cuda.empty_cache()
     d = inputs.config4("cuda")
     Xc, Wc, dY = d["X"], d["W"], d["dY"]

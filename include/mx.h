@@ -203,7 +203,8 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out,
  *     accumulated in FP32 on the tensor cores.
  * Requirements: M, N multiples of 128, K a nonzero multiple of 128; A, B 32-byte
  * aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
- * (the block-scaled tensor-core instruction has no integer element type).
+ * (the block-scaled tensor-core instruction has no integer element type; use
+ * mx_gemm_dense).
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN,
  * MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT (only with
  * opts->check_status).
@@ -254,6 +255,26 @@ int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint
                      void* elems_out, uint8_t* scales_out, int64_t M, int64_t N, int64_t K,
                      mx_fmt_t fmtA, mx_fmt_t fmtB, mx_fmt_t fmtC, mx_round_t rounding,
                      const mx_opts_t* opts);
+
+/*
+ * Dot products of MX operands by way of BF16: both operands are dequantized (Section 2) into
+ * a caller-supplied DEVICE workspace and multiplied by a dense BF16 tensor-core GEMM with
+ * FP32 accumulation.  This is the route for MXINT8 (Table 1), for which the block-scaled
+ * tensor-core instruction has no element type, and it accepts every format pair.  The
+ * dequantized values are exact in BF16 (an element has at most 7 significant bits, INT8
+ * included, and the scale is a power of two) unless X * P falls below BF16's normal range
+ * (scale bytes under ~10), so the result obeys the same bound as mx_gemm; it runs at the
+ * BF16 rate, half the FP8 one, plus the two dequantize passes.
+ *   C          FP32 or BF16 (c_dtype) row-major [M x N].
+ *   workspace  at least mx_gemm_dense_workspace_bytes(M, N, K) = 2 (M + N) K bytes (rounded
+ *              up to 256 each), 256-byte aligned; contents undefined afterwards.
+ * Requirements as mx_gemm except that A and B need 16-byte alignment only and MX_INT8 is
+ * allowed.  Additional errors: MX_ERR_WORKSPACE; MX_ERR_FMT for a bad c_dtype.
+ */
+size_t mx_gemm_dense_workspace_bytes(int64_t M, int64_t N, int64_t K);
+int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                  mx_dtype_t c_dtype, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                  const mx_opts_t* opts, void* workspace, size_t workspace_bytes);
 
 /* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */

@@ -31,7 +31,8 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
-    "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize",
+    "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
+    "mx_gemm_dense",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -77,6 +78,9 @@ def _load() -> ctypes.CDLL:
     lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_gemm_bf16.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_gemm_quantize.argtypes = [vp, u8p, vp, u8p, vp, u8p, i64, i64, i64, ci, ci, ci, ci, op]
+    lib.mx_gemm_dense_workspace_bytes.argtypes = [i64, i64, i64]
+    lib.mx_gemm_dense_workspace_bytes.restype = sz
+    lib.mx_gemm_dense.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, ci, ci, op, vp, sz]
     lib.mx_gemm_batched.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
@@ -256,6 +260,28 @@ def mx_gemm_quantize(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: tor
                                  elems.data_ptr(), scales.data_ptr(), M, N, K, fmtA, fmtB, fmtC,
                                  rounding, ctypes.byref(o)), "mx_gemm_quantize")
     return elems, scales
+
+
+def mx_gemm_dense_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(_lib.mx_gemm_dense_workspace_bytes(M, N, K))
+
+
+def mx_gemm_dense(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
+                  M: int, N: int, K: int, fmtA: int, fmtB: int,
+                  workspace: Optional[torch.Tensor] = None, out: Optional[torch.Tensor] = None,
+                  out_dtype: torch.dtype = torch.float32, check_status: bool = False) -> torch.Tensor:
+    """A . B^T through BF16: dequantize both operands into ``workspace`` and run the dense BF16
+    tensor-core GEMM (any format pair, MXINT8 included)."""
+    assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
+    if workspace is None:
+        workspace = torch.empty(mx_gemm_dense_workspace_bytes(M, N, K), dtype=torch.uint8, device=A.device)
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    _check(_lib.mx_gemm_dense(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(), out.data_ptr(),
+                              _dtype_code(out.dtype), M, N, K, fmtA, fmtB, ctypes.byref(o),
+                              workspace.data_ptr(), workspace.numel()), "mx_gemm_dense")
+    return out
 
 
 # ---- host-buffer variants: tensors live in (pinned) host memory ----------------

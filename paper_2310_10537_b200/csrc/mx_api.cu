@@ -390,6 +390,7 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
   cudaError_t e;
   mx::GemmArgs a;
   a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16; a.batch = batch;
+  a.dense = 0;
   a.q_elems = q_elems; a.q_scales = q_scales; a.q_fmt = q_fmt; a.q_round = q_round;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
@@ -438,6 +439,62 @@ int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint
   if ((uintptr_t)scales_out % 16) return MX_ERR_ALIGN;
   return gemm_device(A, sA, B, sB, nullptr, 0, 1, M, N, K, fmtA, fmtB, opts, elems_out, scales_out,
                      (int)fmtC, (int)rounding);
+}
+
+size_t mx_gemm_dense_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M < 0 || N < 0 || K < 0) return 0;
+  return align_up((size_t)M * (size_t)K * 2, 256) + align_up((size_t)N * (size_t)K * 2, 256);
+}
+
+int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+                  mx_dtype_t c_dtype, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+                  const mx_opts_t* opts, void* workspace, size_t workspace_bytes) {
+  Opts o;
+  if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if ((int)c_dtype != MX_F32 && (int)c_dtype != MX_BF16) return MX_ERR_FMT;
+  if (M < 0 || N < 0 || K < 128 || M % 128 || N % 128 || K % 128) return MX_ERR_SHAPE;
+  if (M >= ((int64_t)1 << 31) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return MX_ERR_SHAPE;
+  if (o.layout != MX_SCALES_SWIZZLED) return MX_ERR_UNSUPPORTED;
+  if ((uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)sA % 16 || (uintptr_t)sB % 16 ||
+      (uintptr_t)C % 16)
+    return MX_ERR_ALIGN;
+  if (M == 0 || N == 0) return MX_OK;
+  if (!workspace) return MX_ERR_NULL;
+  if ((uintptr_t)workspace % 256) return MX_ERR_ALIGN;
+  if (workspace_bytes < mx_gemm_dense_workspace_bytes(M, N, K)) return MX_ERR_WORKSPACE;
+  if (M * K / 8 >= (int64_t)1 << 31 || N * K / 8 >= (int64_t)1 << 31) return MX_ERR_UNSUPPORTED;
+  char* dA = (char*)workspace;
+  char* dB = dA + align_up((size_t)M * (size_t)K * 2, 256);
+  cudaError_t e;
+  const int sms = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  mx::DequantizeArgs d;
+  d.dtype = MX_BF16; d.layout = MX_SCALES_SWIZZLED; d.stream = o.stream; d.sm_count = sms;
+  d.elems = (const uint8_t*)A; d.scales = sA; d.out = dA; d.rows = M; d.L = K; d.fmt = (int)fmtA;
+  if ((e = mx::launch_dequantize(d)) != cudaSuccess) return fail_cuda(e);
+  d.elems = (const uint8_t*)B; d.scales = sB; d.out = dB; d.rows = N; d.L = K; d.fmt = (int)fmtB;
+  if ((e = mx::launch_dequantize(d)) != cudaSuccess) return fail_cuda(e);
+  mx::GemmArgs a;
+  a.A = dA; a.sA = nullptr; a.B = dB; a.sB = nullptr; a.C = C; a.c_bf16 = (int)c_dtype == MX_BF16;
+  a.dense = 1; a.batch = 1;
+  a.q_elems = nullptr; a.q_scales = nullptr; a.q_fmt = 0; a.q_round = 0;
+  a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
+  a.stream = o.stream; a.sm_count = sms;
+  int rc = mx::launch_gemm(a, &e);
+  if (rc != MX_OK) return rc == MX_ERR_CUDA ? fail_cuda(e) : rc;
+  if (o.check) {
+    unsigned int st = 0;
+    rc = mx::gemm_status(o.stream, &st, &e);
+    if (rc != MX_OK) return fail_cuda(e);
+    if (st != 0) {
+      std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u gave up "
+                    "(1 producer/stage empty, 2 MMA/stage full, 3 MMA/accumulator free, "
+                    "4 epilogue/accumulator full)", st);
+      return MX_ERR_TIMEOUT;
+    }
+  }
+  return MX_OK;
 }
 
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {

@@ -148,6 +148,16 @@ __device__ __forceinline__ void tc_mma(uint32_t d_tmem, uint64_t adesc, uint64_t
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
         "r"(accumulate) : "memory");
 }
+// Dense BF16 x BF16 -> FP32 (kind::f16, K = 16 per instruction): no scale operands.
+__device__ __forceinline__ void tc_mma_dense(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                             uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tc_ld32(uint32_t taddr, uint32_t (&r)[32]) {
   asm volatile(
       "tcgen05.ld.sync.aligned.32x32b.x32.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, "
@@ -373,7 +383,9 @@ __device__ __forceinline__ void raise_abort(volatile uint32_t* abort_flag, unsig
   *abort_flag = 1u;
 }
 
-template <int BN>
+// DENSE: the operands are BF16 matrices (MX tensors dequantized beforehand, which is exact) and the
+// MMA is the plain kind::f16 one: a stage holds 64 K-elements (the same 128-byte rows), no scales.
+template <int BN, bool DENSE>
 __global__ void __launch_bounds__(kThreads, 1)
 mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
@@ -395,7 +407,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
-  const uint32_t k_chunks = K / BK;
+  constexpr uint32_t BKe = DENSE ? 64 : BK;     // K elements per stage
+  constexpr uint32_t kProd = DENSE ? 2 : 4;      // copies per stage, one producer lane each
+  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
+  const uint32_t k_chunks = K / BKe;
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
@@ -426,7 +441,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
     // lanes 0..3 issue the four copies of a stage together (see tma_load_3d)
-    if (lane < 4) {
+    if (lane < kProd) {
       const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
       const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
                                                                                          : cfg::kOffSf + 512u;
@@ -446,11 +461,11 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             ok = false;
           }
-          if (!__all_sync(0xFu, ok)) { ok = false; break; }
+          if (!__all_sync(kProdMask, ok)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           if (lane == 0) mbar_arrive_expect_tx(fb, tx_bytes);
-          __syncwarp(0xFu);
-          const int cx = lane < 2 ? (int)(kc * BK) : 0;
+          __syncwarp(kProdMask);
+          const int cx = lane < 2 ? (int)(kc * BKe) : 0;
           const int cy = lane < 2 ? cy_fixed : (int)kc;
           tma_load_3d(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
@@ -484,7 +499,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           tc_fence_after();
           const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          {
+          if (!DENSE) {
             tc_cp_scales(sf_tmem, scale_desc(sf_smem));
 #pragma unroll
             for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
@@ -495,9 +510,13 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 #pragma unroll
           for (uint32_t k = 0; k < BK / kMmaK; ++k) {
             // byte k of each 32-bit scale column belongs to MX block k of this stage
-            const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
-            tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + sfb_col,
-                   (kc | k) != 0 ? 1u : 0u);
+            if (DENSE) {
+              tc_mma_dense(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc_base, (kc | k) != 0 ? 1u : 0u);
+            } else {
+              const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
+              tc_mma(d_tmem, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + sfb_col,
+                     (kc | k) != 0 ? 1u : 0u);
+            }
           }
           tc_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
@@ -575,12 +594,15 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // F4 = both operands FP4 E2M1: kind::mxf4 takes them densely packed (two codes per byte, K = 64 per
 // MMA, two MX blocks and therefore two scales per row and instruction: scale_vec::2X), which doubles
 // the MACs per operand byte and per tensor-core cycle.  A stage then holds 256 K-elements.
-template <bool F4>
+// KIND 2 = dense BF16 operands (kind::f16, see mx_gemm_kernel): 64 K-elements per stage, no scales.
+template <int KIND>
 struct Cfg2 {
+  static constexpr bool F4 = KIND == 1;
+  static constexpr bool DENSE = KIND == 2;
   static constexpr int BN = 256;
   static constexpr int kStages = F4 ? 5 : 6;
-  static constexpr int kBKe = F4 ? 256 : 128;           // K elements per stage (128-byte operand rows)
-  static constexpr int kKChunks = kBKe / 128;           // 512-byte scale chunks (4 MX blocks) along K per stage
+  static constexpr int kBKe = F4 ? 256 : DENSE ? 64 : 128;  // K elements per stage (128-byte operand rows)
+  static constexpr int kKChunks = F4 ? 2 : 1;           // 512-byte scale chunks (4 MX blocks) along K per stage
   static constexpr int kSfColsA = 4 * kKChunks;         // TMEM columns: this CTA's 128 rows of A
   static constexpr int kSfCols = kSfColsA + 8 * kKChunks;  // ... plus all 256 rows of B
   static constexpr int kSfCol0 = BN;                    // single accumulator stage
@@ -637,6 +659,15 @@ __device__ __forceinline__ void tc_mma_pair_f4(uint32_t d_tmem, uint64_t adesc, 
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(sfa_tmem), "r"(sfb_tmem),
         "r"(accumulate) : "memory");
 }
+__device__ __forceinline__ void tc_mma_pair_dense(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc,
+                                                  uint32_t idesc, uint32_t accumulate) {
+  asm volatile(
+      "{\n\t.reg .pred p;\n\t"
+      "setp.ne.b32 p, %4, 0;\n\t"
+      "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t"
+      "}"
+      ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
   asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
 }
@@ -645,14 +676,17 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <bool F4>
+template <int KIND>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
                     uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
                     uint32_t batch) {
-  using cfg = Cfg2<F4>;
+  using cfg = Cfg2<KIND>;
+  constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
+  constexpr uint32_t kProd = DENSE ? 2 : 4;
+  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
   constexpr int BN = cfg::BN;
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
@@ -703,7 +737,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   if (warp == 0) {
     // ------------------------- TMA producer (both CTAs) -------------------------
-    if (lane < 4) {
+    if (lane < kProd) {
       const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
       const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
                                                                                          : cfg::kOffSf + cfg::kSfABytes;
@@ -723,10 +757,10 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             ok = false;
           }
-          if (!__all_sync(0xFu, ok)) { ok = false; break; }
+          if (!__all_sync(kProdMask, ok)) { ok = false; break; }
           const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
-          __syncwarp(0xFu);
+          __syncwarp(kProdMask);
           const int cx = lane < 2 ? (int)(kc * BKe) : 0;
           const int cy = lane < 2 ? cy_fixed : (int)(kc * cfg::kKChunks);
           tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
@@ -760,19 +794,23 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
           // scale chunks -> TMEM.  A: K chunk c at columns 4c.  B: the box is [row group][K chunk],
           // and the MMA wants the columns of one K chunk together: group g, chunk c -> 8c + 4g.
+          if constexpr (!DENSE) {
 #pragma unroll
-          for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
-            tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
+            for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
+              tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
 #pragma unroll
-            for (uint32_t g = 0; g < 2; ++g)
-              tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
-                                scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+              for (uint32_t g = 0; g < 2; ++g)
+                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
+                                  scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+            }
           }
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
 #pragma unroll
           for (uint32_t k = 0; k < 4; ++k) {  // every MMA advances 32 bytes along the 128-byte rows
-            if (F4) {
+            if (DENSE) {
+              tc_mma_pair_dense(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base, (kc | k) != 0 ? 1u : 0u);
+            } else if (F4) {
               // K = 64: blocks 2k and 2k+1 of the stage = bytes (2k % 4, +1) of K chunk k / 2
               const uint32_t sf_id = 2 * (k & 1);
               const uint32_t idesc = idesc_base | (sf_id << 4) | (sf_id << 29);
@@ -892,6 +930,18 @@ bool make_operand_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int f
             CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Tensor map of a dense BF16 K-major operand [rows x K]: box = 64 elements (128 bytes) x box_rows.
+bool make_dense_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
+                    uint32_t box_rows) {
+  const cuuint64_t dims[3] = {K, rows, 1};
+  const cuuint64_t strides[2] = {K * 2, K * 2 * rows};
+  const cuuint32_t box[3] = {64, box_rows, 1};
+  const cuuint32_t estr[3] = {1, 1, 1};
+  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
+            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 // Tensor map over a swizzled scale tensor seen as [row groups of 128][K chunks][128 words]:
 // one 512-byte chunk per (row group, K chunk); the box takes `groups` consecutive row groups.
 bool make_scale_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
@@ -935,22 +985,26 @@ EpiArgs epi_args(const GemmArgs& a) {
   return e;
 }
 
-template <int BN>
+template <int BN, bool DENSE>
 cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMap& mb,
                       uint32_t idesc_base) {
   CUtensorMap mc, msa, msb;
   EncodeTiledFn fn = encode_fn_cached();
-  if (!make_out_map(fn, &mc, a) ||
-      !make_scale_map(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1) ||
-      !make_scale_map(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, Cfg<BN>::kSfbChunks))
+  if (!make_out_map(fn, &mc, a)) return cudaErrorInvalidValue;
+  if (DENSE) {
+    msa = ma;  // the dense kernel takes no scales; the parameters still hold valid descriptors
+    msb = mb;
+  } else if (!make_scale_map(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1) ||
+             !make_scale_map(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, Cfg<BN>::kSfbChunks)) {
     return cudaErrorInvalidValue;
+  }
   using cfg = Cfg<BN>;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(mx_gemm_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(mx_gemm_kernel<BN, DENSE>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -960,9 +1014,10 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   const uint32_t group_m = 16;
   // Bytes the producer's copies report to a stage's mbarrier: the tensor-map copies count the
   // packed source bytes (bits/8 per element), not the expanded shared-memory footprint.
-  const uint32_t tx_bytes = (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8) +
-                            cfg::kSfBytes;
-  mx_gemm_kernel<BN><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
+  const uint32_t tx_bytes =
+      DENSE ? (uint32_t)(BM + BN) * 128u
+            : (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8) + cfg::kSfBytes;
+  mx_gemm_kernel<BN, DENSE><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
       idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, epi_args(a),
       (uint32_t)a.batch);
@@ -994,26 +1049,34 @@ bool make_scale_map_k(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint6
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <bool F4>
+template <int KIND>
 cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
-  using cfg = Cfg2<F4>;
+  using cfg = Cfg2<KIND>;
+  constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
   CUtensorMap ma, mb, msa, msb, mc;
-  bool ok = make_out_map(fn, &mc, a) &&
-            make_scale_map_k(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1, cfg::kKChunks) &&
-            make_scale_map_k(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 2, cfg::kKChunks);
-  if (F4)
-    ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K) &&
-         make_f4_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K);
-  else
-    ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
-         make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
+  bool ok = make_out_map(fn, &mc, a);
+  if (DENSE) {
+    ok = ok && make_dense_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
+         make_dense_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
+    msa = ma;  // no scales: valid descriptors the kernel never uses
+    msb = mb;
+  } else {
+    ok = ok && make_scale_map_k(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1, cfg::kKChunks) &&
+         make_scale_map_k(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 2, cfg::kKChunks);
+    if (F4)
+      ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K) &&
+           make_f4_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K);
+    else
+      ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
+           make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
+  }
   if (!ok) return cudaErrorInvalidValue;
   static bool attr_set[64] = {false};
   int dev = 0;
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(mx_gemm_pair_kernel<F4>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(mx_gemm_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
@@ -1021,14 +1084,15 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
   const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
-  const uint32_t op_bytes = F4 ? 2u * 128u * 128u
+  const uint32_t op_bytes = (F4 || DENSE) ? 2u * 128u * 128u
                                : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 128 * BK * fmt_bits(a.fmtB) / 8);
-  const uint32_t tx_pair = 2u * (op_bytes + cfg::kSfBytes);
-  // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code()
-  const uint32_t fa = F4 ? 1u : mma_fmt_code(a.fmtA), fb = F4 ? 1u : mma_fmt_code(a.fmtB);
-  const uint32_t idesc = (fa << 7) | (fb << 10) | (1u << 23) | ((uint32_t)(256 >> 3) << 17) |
-                         ((uint32_t)(256 >> 4) << 24);
-  mx_gemm_pair_kernel<F4><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
+  const uint32_t tx_pair = 2u * (op_bytes + (DENSE ? 0u : cfg::kSfBytes));
+  // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code();
+  // kind::f16: BF16 = 1 for both operands, FP32 accumulator = 1 in bits [4,6), no scale-format bit
+  const uint32_t fa = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtA), fb = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtB);
+  const uint32_t idesc = (fa << 7) | (fb << 10) | (DENSE ? (1u << 4) : (1u << 23)) |
+                         ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+  mx_gemm_pair_kernel<KIND><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
       epi_args(a), (uint32_t)a.batch);
   return cudaGetLastError();
@@ -1047,20 +1111,30 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
   if (a.M % 256 == 0 && a.batch * (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
-    const bool f4 = a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
-    *cuda_err = f4 ? launch_pair<true>(a, fn) : launch_pair<false>(a, fn);
+    const bool f4 = !a.dense && a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
+    *cuda_err = a.dense ? launch_pair<2>(a, fn) : f4 ? launch_pair<1>(a, fn) : launch_pair<0>(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
   CUtensorMap ma, mb;
-  if (!make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, BM) ||
-      !make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, (uint32_t)bn)) {
+  const bool ok =
+      a.dense ? make_dense_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K, BM) &&
+                    make_dense_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K, (uint32_t)bn)
+              : make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, BM) &&
+                    make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, (uint32_t)bn);
+  if (!ok) {
     *cuda_err = cudaErrorInvalidValue;
     return MX_ERR_CUDA;
   }
-  // a_format [7,10), b_format [10,13), K-major A and B, scale format E8M0 (bit 23), M = 128
-  const uint32_t idesc = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23) |
-                         ((uint32_t)(BM >> 4) << 24);
-  *cuda_err = bn == 256 ? launch_bn<256>(a, ma, mb, idesc) : launch_bn<128>(a, ma, mb, idesc);
+  if (a.dense) {
+    // kind::f16: FP32 accumulator (bits [4,6) = 1), BF16 operands (1), K-major A and B, M = 128
+    const uint32_t idesc = (1u << 4) | (1u << 7) | (1u << 10) | ((uint32_t)(BM >> 4) << 24);
+    *cuda_err = bn == 256 ? launch_bn<256, true>(a, ma, mb, idesc) : launch_bn<128, true>(a, ma, mb, idesc);
+  } else {
+    // a_format [7,10), b_format [10,13), K-major A and B, scale format E8M0 (bit 23), M = 128
+    const uint32_t idesc = (mma_fmt_code(a.fmtA) << 7) | (mma_fmt_code(a.fmtB) << 10) | (1u << 23) |
+                           ((uint32_t)(BM >> 4) << 24);
+    *cuda_err = bn == 256 ? launch_bn<256, false>(a, ma, mb, idesc) : launch_bn<128, false>(a, ma, mb, idesc);
+  }
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
 }
 

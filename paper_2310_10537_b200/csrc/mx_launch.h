@@ -53,6 +53,8 @@ struct GemmArgs {
   void* q_elems;
   uint8_t* q_scales;
   int q_fmt, q_round;
+  // dense != 0: A and B are BF16 K-major matrices (dequantized MX tensors), sA / sB unused.
+  int dense;
   int64_t batch;  // independent products; operands and C are the matrices stacked along rows
   int64_t M, N, K;
   int fmtA, fmtB;

@@ -446,6 +446,57 @@ def test_gemm_quantize_equals_gemm_then_quantize(fc, rounding):
     assert np.array_equal(fe.cpu().numpy().reshape(-1), oe) and np.array_equal(fs.cpu().numpy().reshape(-1), osc)
 
 
+@pytest.mark.parametrize("shape,fa,fb,dt", [
+    ((384, 512, 1024), 5, 5, torch.float32),     # MXINT8 x MXINT8, one-CTA 128 x 128 tiles
+    ((128, 128, 128), 5, 0, torch.float32),
+    ((4736, 8320, 256), 5, 0, torch.float32),    # one-CTA 128 x 256 tiles, ragged last tile
+    ((2048, 9600, 384), 0, 5, torch.float32),    # two-CTA tiles, ragged N
+    ((2048, 9600, 384), 5, 5, torch.bfloat16),
+    ((512, 640, 256), 2, 4, torch.float32),      # the BF16 route also takes the formats mx_gemm takes
+])
+def test_gemm_dense(shape, fa, fb, dt):
+    """mx_gemm_dense (dequantize to BF16 + dense BF16 tensor-core GEMM; the MXINT8 route): whole
+    matrix against an FP64 library product of the oracle-dequantized operands, samples against the
+    oracle's GEMM, same bound as mx_gemm."""
+    M, N, K = shape
+    g = torch.Generator(device="cuda").manual_seed(M + 2 * N + K + fa)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.02
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(M * N * esz)
+    g_ws = Guarded(mx.mx_gemm_dense_workspace_bytes(M, N, K))
+    C = g_out.view.view(dt).view(M, N)
+    mx.mx_gemm_dense(ea, sa, eb, sb, M, N, K, fa, fb, workspace=g_ws.view, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    g_ws.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    ref = da @ db.T
+    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
+    bad = int(((C.double() - ref).abs() > 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+    assert bad == 0, f"{shape}: {bad} outputs beyond the bound"
+    rng = np.random.default_rng(M + fa)
+    ms, ns = rng.integers(0, M, 1000), rng.integers(0, N, 1000)
+    c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+
+
+def test_gemm_dense_errors():
+    z = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    out = torch.zeros((128, 128), device="cuda")
+    with pytest.raises(mx.MxError) as e:
+        mx.mx_gemm_dense(z, z, z, z, 128, 128, 128, 5, 5, workspace=z[:1024], out=out)
+    assert e.value.status == mx.MX_ERR_WORKSPACE
+    with pytest.raises(mx.MxError) as e:
+        mx.mx_gemm(z, z, z, z, 128, 128, 128, 5, 0, out=out)
+    assert e.value.status == mx.MX_ERR_UNSUPPORTED
+
+
 def test_config3_full_size():
     d = inputs.config3("cuda")
     X, W = d["X"], d["W"]
