@@ -201,8 +201,11 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out,
  *       C[m,n] = sum over K-blocks b of X_A[m,b] * X_B[n,b] *
  *                sum_{i<32} P_A[m,32b+i] * P_B[n,32b+i]
  *     accumulated in FP32 on the tensor cores.
- * Requirements: M, N multiples of 128, K a nonzero multiple of 128; A, B 32-byte
- * aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
+ * Shapes: any M >= 0; K a nonzero multiple of 32 (the block size), of 128 when an
+ * operand has 6- or 4-bit codes; N such that a row of C is a whole number of 16-byte
+ * units (N % 4 for FP32).  Partial tiles are zero-filled on the way in and clipped on
+ * the way out; the scale tensors are the padded SWIZZLED tensors mx_quantize writes
+ * (padding bytes 0).  A, B 32-byte aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
  * (the block-scaled tensor-core instruction has no integer element type; use
  * mx_gemm_dense).
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN,
@@ -230,8 +233,8 @@ int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t*
  * MX_F32 or MX_BF16), all contiguous; sA / sB are the swizzled scale tensors of the
  * [batch*M x K] and [batch*N x K] matrices, i.e. what mx_quantize writes for the
  * 3-D tensors along their last axis.  C[b] = A[b] . B[b]^T as in mx_gemm.
- * Requirements and errors as mx_gemm (M and N multiples of 128 keep every matrix on
- * whole scale chunks); additionally MX_ERR_FMT for a bad c_dtype and MX_ERR_SHAPE when
+ * Requirements and errors as mx_gemm, except that M and N must be multiples of 128 (which
+ * keeps every matrix of the stack on whole scale chunks and tiles); additionally MX_ERR_FMT for a bad c_dtype and MX_ERR_SHAPE when
  * batch < 0 or batch*M or batch*N reaches 2^31.  batch == 0 is a no-op.
  */
 int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
@@ -249,7 +252,8 @@ int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8
  *                            operands: packed codes [M x N] (N innermost) and the SWIZZLED
  *                            scale tensor of M rows x N/32 blocks -- the A operand of a
  *                            following mx_gemm whose K is this N.  Any format, MX_INT8 included.
- * elems_out and scales_out 16-byte aligned.  Other requirements and errors as mx_gemm.
+ * M and N multiples of 128; elems_out and scales_out 16-byte aligned.  Other requirements
+ * and errors as mx_gemm.
  */
 int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
                      void* elems_out, uint8_t* scales_out, int64_t M, int64_t N, int64_t K,
@@ -268,8 +272,8 @@ int mx_gemm_quantize(const void* A, const uint8_t* sA, const void* B, const uint
  *   C          FP32 or BF16 (c_dtype) row-major [M x N].
  *   workspace  at least mx_gemm_dense_workspace_bytes(M, N, K) = 2 (M + N) K bytes (rounded
  *              up to 256 each), 256-byte aligned; contents undefined afterwards.
- * Requirements as mx_gemm except that A and B need 16-byte alignment only and MX_INT8 is
- * allowed.  Additional errors: MX_ERR_WORKSPACE; MX_ERR_FMT for a bad c_dtype.
+ * Requirements as mx_gemm except that A and B need 16-byte alignment only, K may be any
+ * nonzero multiple of 32 for every format and MX_INT8 is allowed.  Additional errors: MX_ERR_WORKSPACE; MX_ERR_FMT for a bad c_dtype.
  */
 size_t mx_gemm_dense_workspace_bytes(int64_t M, int64_t N, int64_t K);
 int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,

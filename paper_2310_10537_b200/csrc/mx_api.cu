@@ -356,12 +356,18 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
 // GEMM
 // ---------------------------------------------------------------------------
 
+// strict: every matrix must consist of whole 128-row / 128-column tiles (batched products, whose
+// matrices are stacked along rows, and the quantizing epilogue, which writes whole blocks).
 static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
-                         const void* C, int64_t M, int64_t N, int64_t K, int fmtA, int fmtB) {
+                         const void* C, int64_t M, int64_t N, int64_t K, int fmtA, int fmtB,
+                         bool strict, int c_elem_bytes) {
   if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
   if (!fmt_ok(fmtA) || !fmt_ok(fmtB)) return MX_ERR_FMT;
   if (fmtA == MX_INT8 || fmtB == MX_INT8) return MX_ERR_UNSUPPORTED;
-  if (M < 0 || N < 0 || K < 128 || M % 128 || N % 128 || K % 128) return MX_ERR_SHAPE;
+  if (M < 0 || N < 0 || K < 32 || K % 32) return MX_ERR_SHAPE;
+  // the tensor-map types of packed 6- and 4-bit codes take rows of whole 128-element groups only
+  if ((fmt_bits(fmtA) < 8 || fmt_bits(fmtB) < 8) && K % 128) return MX_ERR_SHAPE;
+  if (strict ? (M % 128 || N % 128) : (N * c_elem_bytes) % 16 != 0) return MX_ERR_SHAPE;
   if (M >= ((int64_t)1 << 31) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return MX_ERR_SHAPE;
   return MX_OK;
 }
@@ -376,7 +382,8 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
     if (!q_elems || !q_scales) return MX_ERR_NULL;
     C = q_elems;  // stands in for the output pointer in the checks below
   }
-  int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB);
+  int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB, batch != 1 || q_elems != nullptr,
+                         c_bf16 ? 2 : 4);
   if (rc != MX_OK) return rc;
   if (!read_opts(opts, &o)) return MX_ERR_FMT;
   if (o.layout != MX_SCALES_SWIZZLED) return MX_ERR_UNSUPPORTED;
@@ -384,7 +391,7 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
       (uintptr_t)C % 16)
     return MX_ERR_ALIGN;
   if (batch < 0 || batch * M >= ((int64_t)1 << 31) || batch * N >= ((int64_t)1 << 31) ||
-      (M > 0 && N > 0 && batch * (M / 128) * (N / 128) >= ((int64_t)1 << 31)))
+      (M > 0 && N > 0 && batch * ((M + 127) / 128) * ((N + 127) / 128) >= ((int64_t)1 << 31)))
     return MX_ERR_SHAPE;
   if (M == 0 || N == 0 || batch == 0) return MX_OK;
   cudaError_t e;
@@ -453,7 +460,7 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
   if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
   if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || !read_opts(opts, &o)) return MX_ERR_FMT;
   if ((int)c_dtype != MX_F32 && (int)c_dtype != MX_BF16) return MX_ERR_FMT;
-  if (M < 0 || N < 0 || K < 128 || M % 128 || N % 128 || K % 128) return MX_ERR_SHAPE;
+  if (M < 0 || N < 0 || K < 32 || K % 32 || (N * ((int)c_dtype == MX_BF16 ? 2 : 4)) % 16) return MX_ERR_SHAPE;
   if (M >= ((int64_t)1 << 31) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return MX_ERR_SHAPE;
   if (o.layout != MX_SCALES_SWIZZLED) return MX_ERR_UNSUPPORTED;
   if ((uintptr_t)A % 16 || (uintptr_t)B % 16 || (uintptr_t)sA % 16 || (uintptr_t)sB % 16 ||
@@ -511,7 +518,7 @@ int mx_gemm_host(const void* A_host, const uint8_t* sA_host, const void* B_host,
                  mx_fmt_t fmtA, mx_fmt_t fmtB, const mx_opts_t* opts, void* workspace_dev,
                  size_t workspace_bytes) {
   Opts o;
-  int rc = gemm_validate(A_host, sA_host, B_host, sB_host, C_host, M, N, K, (int)fmtA, (int)fmtB);
+  int rc = gemm_validate(A_host, sA_host, B_host, sB_host, C_host, M, N, K, (int)fmtA, (int)fmtB, false, 4);
   if (rc != MX_OK) return rc;
   if (!read_opts(opts, &o)) return MX_ERR_FMT;
   if (!workspace_dev) return MX_ERR_NULL;

@@ -406,11 +406,12 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   volatile uint32_t* abort_flag = tmem_slot + 1;
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const uint32_t tiles_m = M / BM, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
+  const uint32_t tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
+  const uint32_t num_tiles = batch * tiles_m * tiles_n;
   constexpr uint32_t BKe = DENSE ? 64 : BK;     // K elements per stage
   constexpr uint32_t kProd = DENSE ? 2 : 4;      // copies per stage, one producer lane each
   constexpr uint32_t kProdMask = (1u << kProd) - 1u;
-  const uint32_t k_chunks = K / BKe;
+  const uint32_t k_chunks = (K + BKe - 1) / BKe;  // a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
@@ -542,7 +543,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tc_fence_after();
       const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * BN + half * kHalf;
       const uint32_t col0 = tc.tn * BN + half * kHalf;
-      const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;  // multiple of 32
+      const uint32_t row0 = (tc.b * tiles_m + tc.tm) * BM + quarter * 32;
+      // columns of this half that exist; nothing is stored for rows past the end of a last,
+      // partial row tile (only a single matrix can have one: its rows end at M)
+      const uint32_t valid_cols = (col0 < N && row0 < batch * M) ? min(kHalf, N - col0) : 0u;
       uint32_t r[kLoads][32];
 #pragma unroll
       for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
@@ -550,7 +554,6 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       tc_fence_before();
       __syncwarp();
       if (lane == 0) mbar_arrive(acc_empty_bar(acc));  // the MMA issuer may overwrite the accumulator
-      const uint32_t row0 = (tc.b * tiles_m + tc.tm) * BM + quarter * 32;
       if (epi.mode == 2) {
         if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
       } else {
@@ -706,7 +709,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
   const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
-  const uint32_t k_chunks = K / BKe;
+  const uint32_t k_chunks = (K + BKe - 1) / BKe;  // a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
@@ -946,8 +949,8 @@ bool make_dense_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_
 // one 512-byte chunk per (row group, K chunk); the box takes `groups` consecutive row groups.
 bool make_scale_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
                     uint32_t groups) {
-  const uint64_t k_chunks = K / BK;
-  const cuuint64_t dims[3] = {128, k_chunks, rows / 128};
+  const uint64_t k_chunks = (K + BK - 1) / BK;  // the swizzled layout pads K to whole chunks, rows to 128
+  const cuuint64_t dims[3] = {128, k_chunks, (rows + 127) / 128};
   const cuuint64_t strides[2] = {512, 512 * k_chunks};
   const cuuint32_t box[3] = {128, 1, groups};
   const cuuint32_t estr[3] = {1, 1, 1};
@@ -1009,7 +1012,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / BM) * (uint32_t)((a.N + BN - 1) / BN);
+  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)((a.M + BM - 1) / BM) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
   const uint32_t group_m = 16;
   // Bytes the producer's copies report to a stage's mbarrier: the tensor-map copies count the
@@ -1039,8 +1042,8 @@ bool make_f4_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t r
 // Scale map whose box also spans `kchunks` K chunks: [row groups][K chunks][128 words].
 bool make_scale_map_k(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
                       uint32_t groups, uint32_t kchunks) {
-  const uint64_t k_chunks = K / BK;
-  const cuuint64_t dims[3] = {128, k_chunks, rows / 128};
+  const uint64_t k_chunks = (K + BK - 1) / BK;  // the swizzled layout pads K to whole chunks, rows to 128
+  const cuuint64_t dims[3] = {128, k_chunks, (rows + 127) / 128};
   const cuuint64_t strides[2] = {512, 512 * k_chunks};
   const cuuint32_t box[3] = {128, kchunks, groups};
   const cuuint32_t estr[3] = {1, 1, 1};
@@ -1106,7 +1109,7 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   if (!fn) return MX_ERR_CUDA;
   // 256-wide tiles move the fewest operand bytes through shared memory per flop; problems with
   // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
-  const int64_t tiles256 = a.batch * (a.M / BM) * ((a.N + 255) / 256);
+  const int64_t tiles256 = a.batch * ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
   // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
   if (a.M % 256 == 0 && a.batch * (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {

@@ -70,8 +70,10 @@ def test_argument_validation_without_gpu():
     assert d(p, p, p, shape3, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_UNSUPPORTED
     assert d(p, None, p, shape, 2, 1, 0, ctypes.byref(o)) == mx.MX_ERR_NULL
     g = lib.mx_gemm
-    assert g(p, p, p, p, p, 100, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
-    assert g(p, p, p, p, p, 128, 128, 64, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert g(p, p, p, p, p, -1, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert g(p, p, p, p, p, 128, 130, 128, 0, 0, None) == mx.MX_ERR_SHAPE   # C rows not whole 16-byte units
+    assert g(p, p, p, p, p, 128, 128, 48, 0, 0, None) == mx.MX_ERR_SHAPE    # K not a multiple of 32
+    assert g(p, p, p, p, p, 128, 128, 96, 2, 0, None) == mx.MX_ERR_SHAPE    # 6- and 4-bit codes need K % 128
     assert g(p, p, p, p, p, 128, 128, 128, 5, 0, None) == mx.MX_ERR_UNSUPPORTED
     assert g(p, p, p, p, p, 128, 128, 128, 0, 9, None) == mx.MX_ERR_FMT
     assert g(None, p, p, p, p, 128, 128, 128, 0, 0, None) == mx.MX_ERR_NULL

@@ -203,7 +203,7 @@ def test_nan_scale_poisons_row_and_gemm_errors():
     assert not np.isnan(C[fin]).any()
     _check_bound(np.where(fin, C, 0), np.where(fin, C64, 0), np.where(fin, S, 0), "finite part")
     with pytest.raises(mx.MxError) as ei:
-        mx.mx_gemm(ea, sa, eb, sb, 100, N, K, 0, 0)
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K - 16, 0, 0)
     assert ei.value.status == mx.MX_ERR_SHAPE
     with pytest.raises(mx.MxError) as ei:
         mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_INT8, 0)
@@ -495,6 +495,63 @@ def test_gemm_dense_errors():
     with pytest.raises(mx.MxError) as e:
         mx.mx_gemm(z, z, z, z, 128, 128, 128, 5, 0, out=out)
     assert e.value.status == mx.MX_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("M,N,K,fa,fb,dt", [
+    (1, 128, 128, 0, 0, torch.float32),          # a single token
+    (7, 4100, 96, 0, 1, torch.float32),          # K tail, N a multiple of 4 only
+    (100, 200, 256, 4, 0, torch.bfloat16),       # M and N tails (6- and 4-bit codes: K % 128)
+    (300, 37 * 256 + 32, 352, 0, 1, torch.float32),  # 128 x 256 tiles with tails in M, N and K
+    (2048, 9608, 416, 1, 1, torch.float32),      # two-CTA tiles, N and K tails
+    (2048, 9608, 384, 2, 3, torch.float32),      # 6-bit operands (K % 128)
+    (130, 264, 640, 4, 4, torch.bfloat16),
+])
+def test_tails(M, N, K, fa, fb, dt):
+    """Shapes that are not whole tiles: any M, K a multiple of the block size, C rows whole 16-byte
+    units.  The copies zero-fill past the edges and the stores are clipped; the guard bands catch a
+    store that is not."""
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.05
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(M * N * esz)
+    C = g_out.view.view(dt).view(M, N)
+    if dt == torch.bfloat16:
+        mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    else:
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
+    if M * N * K <= 1 << 28:
+        c64, s = O.gemm(hea, hsa, heb, hsb, M, N, K, fa, fb)
+        got = C.double().cpu().numpy()
+    else:
+        da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+        db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+        ref = da @ db.T
+        bad = int(((C.double() - ref).abs() > 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+        assert bad == 0, f"{bad} outputs beyond the bound"
+        rng = np.random.default_rng(K)
+        ms = np.concatenate([rng.integers(0, M, 1500), np.full(300, M - 1)])
+        ns = np.concatenate([rng.integers(0, N, 1500), rng.integers(N - 40, N, 300)])
+        c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+        got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+    # the BF16 route takes the same shapes
+    g_out = Guarded(M * N * esz)
+    C2 = g_out.view.view(dt).view(M, N)
+    mx.mx_gemm_dense(ea, sa, eb, sb, M, N, K, fa, fb, out=C2, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    if M * N * K <= 1 << 28:
+        assert (np.abs(C2.double().cpu().numpy() - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+    else:
+        got2 = C2[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+        assert (np.abs(got2 - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
 
 
 def test_config3_full_size():
