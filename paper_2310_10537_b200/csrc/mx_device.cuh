@@ -237,4 +237,25 @@ __device__ __forceinline__ void st_32(void* p, const uint32_t (&v)[8]) {
                : "memory");
 }
 
+// N words (a multiple of 4) to consecutive addresses: 256-bit stores where `wide` (dst 32-byte
+// aligned) allows, so that every request carries a whole 32-byte sector; else 128-bit stores.
+template <int N>
+__device__ __forceinline__ void store_run(uint8_t* dst, const uint32_t (&w)[N], bool wide) {
+  static_assert(N % 4 == 0, "whole 16-byte units");
+  if (wide) {
+#pragma unroll
+    for (int i = 0; i < N / 8; ++i) {
+      const uint32_t v[8] = {w[8 * i], w[8 * i + 1], w[8 * i + 2], w[8 * i + 3],
+                             w[8 * i + 4], w[8 * i + 5], w[8 * i + 6], w[8 * i + 7]};
+      st_32(dst + 32 * i, v);
+    }
+    if (N % 8)
+      *reinterpret_cast<uint4*>(dst + 32 * (N / 8)) = make_uint4(w[N - 4], w[N - 3], w[N - 2], w[N - 1]);
+  } else {
+#pragma unroll
+    for (int i = 0; i < N / 4; ++i)
+      *reinterpret_cast<uint4*>(dst + 16 * i) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  }
+}
+
 }  // namespace mx

@@ -333,9 +333,7 @@ __device__ __forceinline__ void store_mx_fmt(const uint32_t (&r)[kLoads][32], co
     }
   }
   uint8_t* dst = epi.elems + ((size_t)row * N + col0) / 8 * W;
-#pragma unroll
-  for (uint32_t i = 0; i < kLoads * W / 4; ++i)
-    *reinterpret_cast<uint4*>(dst + 16 * i) = make_uint4(w[4 * i], w[4 * i + 1], w[4 * i + 2], w[4 * i + 3]);
+  store_run<(int)(kLoads * W)>(dst, w, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
   // swizzled scale layout: the kLoads scale bytes of this row are adjacent inside one 512-byte chunk
   const uint32_t kb = col0 / 32;
   uint8_t* sp = epi.scales + ((size_t)(row / 128) * (N / 128) + kb / 4) * 512 + (row % 32) * 16 +

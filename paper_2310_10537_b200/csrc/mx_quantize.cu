@@ -205,6 +205,7 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
   const size_t esz = DTYPE == MX_BF16 ? 2 : 4;
   const size_t row_pitch = (size_t)inner * esz;
   const size_t out_row_bytes = (size_t)L * bits / 8;
+  const bool al32 = (reinterpret_cast<uintptr_t>(elems) & 31u) == 0;  // 8-bit rows are whole 32-byte units
 
   for (uint32_t o = blockIdx.z; o < outer; o += gridDim.z)
   for (uint32_t kb = kb_begin; kb < kb_end; ++kb) {
@@ -268,8 +269,12 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
         cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
       }
       if (bits == 8) {
-        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        if (al32) {  // one 256-bit store: a whole sector in a single request
+          st_32(dst, w);
+        } else {
+          reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
+          reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        }
       } else if (bits == 4) {
         reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[2], w[4], w[6]);
       } else {
@@ -321,6 +326,7 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
   const size_t row_pitch = (size_t)inner * esz;
   const size_t out_row_bytes = (size_t)L * bits / 8;
   const uint32_t rows_here = min(kRows, (inner - warp_col0));      // valid output rows of this warp
+  const bool al32 = (reinterpret_cast<uintptr_t>(elems) & 31u) == 0 && out_row_bytes % 32 == 0;
 
   for (uint32_t o = blockIdx.z; o < outer; o += gridDim.z) {
     const uint32_t kb0 = blockIdx.y * 4;
@@ -411,7 +417,24 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
       }
     }
     __syncwarp();
-    // write-out: 16-byte chunks, consecutive lanes on consecutive chunks of one output row
+    // write-out, consecutive lanes on consecutive chunks of one output row: 32-byte chunks (one
+    // whole sector per request: the L2 request rate bounds this kernel) when the tensor allows
+    if (al32) {
+      constexpr uint32_t kChunks32 = kSeg / 32;
+      for (uint32_t i = lane; i < kRows * kChunks32; i += 32) {
+        const uint32_t r = i / kChunks32, ch = i - r * kChunks32;
+        const uint32_t c = r >> 5, owner = r & 31;
+        const uint32_t col = owner * COLS + c;
+        if (col < rows_here) {
+          const uint2* src = reinterpret_cast<const uint2*>(area + r * kPitch + ch * 32);
+          const uint2 q0 = src[0], q1 = src[1], q2 = src[2], q3 = src[3];
+          const uint32_t v[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
+          st_32(elems + (size_t)(o * inner + warp_col0 + col) * out_row_bytes + (size_t)kb0 * kBpb + ch * 32, v);
+        }
+      }
+      __syncwarp();
+      continue;
+    }
     constexpr uint32_t kChunks = kSeg / 16;
     for (uint32_t i = lane; i < kRows * kChunks; i += 32) {
       const uint32_t r = i / kChunks, ch = i - r * kChunks;      // staging row, chunk in the row

@@ -35,8 +35,10 @@ template <int FMT, int DTYPE> struct DualCfg {
   static constexpr uint32_t kSmem = (kDualThreads / 32) * kWarpBytes;
 };
 
+// Resident CTAs per SM: BF16 tiles carry twice the elements per register and measured fastest with
+// the tile-ahead loads at four CTAs (255 registers); FP32 at six.
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
-__global__ void __launch_bounds__(kDualThreads, 4)
+__global__ void __launch_bounds__(kDualThreads, DTYPE == MX_BF16 ? 4 : 6)
 quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_row,
                      uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
                      uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C) {
@@ -65,16 +67,22 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
 #pragma unroll
   for (int c = 0; c < COLS; ++c) col_scale_word[c] = 0;
 
-#pragma unroll 1
-  for (uint32_t j = 0; j < 4; ++j) {
-    const uint32_t tile = tile0 + j;
-    uint32_t raw[kBlock][kWords];
+  // The 32 rows of a tile are loaded one tile ahead: the loads of tile j + 1 are issued as soon as
+  // the column arithmetic has consumed the registers of tile j and fly during its row arithmetic.
+  uint32_t raw[kBlock][kWords];
+  auto load_tile = [&](uint32_t tile) {
     const char* p = reinterpret_cast<const char*>(in) + (size_t)tile * kBlock * in_pitch + (size_t)col0 * esz;
 #pragma unroll
     for (int k = 0; k < kBlock; ++k) {
       const uint2 w = __ldg(reinterpret_cast<const uint2*>(p + (size_t)k * in_pitch));
       raw[k][0] = w.x; raw[k][1] = w.y;
     }
+  };
+  load_tile(tile0);
+
+#pragma unroll 1
+  for (uint32_t j = 0; j < 4; ++j) {
+    const uint32_t tile = tile0 + j;
     // transpose area first, so the shared-memory latency hides behind the column arithmetic
 #pragma unroll
     for (int k = 0; k < kBlock; ++k)
@@ -91,8 +99,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
       column_cast<FMT, ROUND, DTYPE, COLS>(raw, c, s, w);
       if (bits == 8) {
         uint8_t* dst = elems_col + (size_t)(col0 + c) * col_out_bytes + (size_t)tile * kBpb;
-        reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[1], w[2], w[3]);
-        reinterpret_cast<uint4*>(dst)[1] = make_uint4(w[4], w[5], w[6], w[7]);
+        store_run<8>(dst, w, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
       } else {
         uint8_t* dst = sarea + (c * 32 + lane) * cfg::kPitch + j * kBpb;
         if (bits == 4) {
@@ -108,6 +115,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
       }
     }
     __syncwarp();
+    if (j < 3) load_tile(tile + 1);
 
     // ---- row blocks: lane r owns row (tile * 32 + r) of the strip: kRowBlocks blocks of 32 columns
     {
@@ -141,24 +149,32 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
       }
       // contiguous run of kRowBlocks blocks in the [R x C] output
       uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)strip * kRowBlocks * kBpb;
+      const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
       if (bits == 8) {
-#pragma unroll
-        for (int q = 0; q < kRowBlocks; ++q) {
-          reinterpret_cast<uint4*>(dst)[2 * q] = make_uint4(codes[q][0], codes[q][1], codes[q][2], codes[q][3]);
-          reinterpret_cast<uint4*>(dst)[2 * q + 1] = make_uint4(codes[q][4], codes[q][5], codes[q][6], codes[q][7]);
-        }
-      } else if (bits == 4) {
+        uint32_t run[kRowBlocks * 8];
 #pragma unroll
         for (int q = 0; q < kRowBlocks; ++q)
-          reinterpret_cast<uint4*>(dst)[q] = make_uint4(codes[q][0], codes[q][2], codes[q][4], codes[q][6]);
+#pragma unroll
+          for (int i = 0; i < 8; ++i) run[8 * q + i] = codes[q][i];
+        store_run<kRowBlocks * 8>(dst, run, wide);
+      } else if (bits == 4) {
+        uint32_t run[kRowBlocks * 4];
+#pragma unroll
+        for (int q = 0; q < kRowBlocks; ++q)
+#pragma unroll
+          for (int i = 0; i < 4; ++i) run[4 * q + i] = codes[q][2 * i];
+        store_run<kRowBlocks * 4>(dst, run, wide);
       } else {
-        uint64_t qq[kRowBlocks * 3];
+        uint32_t run[kRowBlocks * 6];
 #pragma unroll
-        for (int q = 0; q < kRowBlocks; ++q) pack6(codes[q], qq[3 * q], qq[3 * q + 1], qq[3 * q + 2]);
-#pragma unroll
-        for (int i = 0; i < kRowBlocks * 3 / 2; ++i)  // 24 * kRowBlocks bytes as 16-byte stores
-          reinterpret_cast<uint4*>(dst)[i] = make_uint4((uint32_t)qq[2 * i], (uint32_t)(qq[2 * i] >> 32),
-                                                        (uint32_t)qq[2 * i + 1], (uint32_t)(qq[2 * i + 1] >> 32));
+        for (int q = 0; q < kRowBlocks; ++q) {
+          uint64_t a, b, c;
+          pack6(codes[q], a, b, c);
+          run[6 * q] = (uint32_t)a; run[6 * q + 1] = (uint32_t)(a >> 32);
+          run[6 * q + 2] = (uint32_t)b; run[6 * q + 3] = (uint32_t)(b >> 32);
+          run[6 * q + 4] = (uint32_t)c; run[6 * q + 5] = (uint32_t)(c >> 32);
+        }
+        store_run<kRowBlocks * 6>(dst, run, wide);
       }
       uint8_t* sdst = scales_row + scale_offset<LAYOUT>(row, strip * kRowBlocks, kb_row);
       if (kRowBlocks == 4) *reinterpret_cast<uint32_t*>(sdst) = row_scale_word;
@@ -173,6 +189,19 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
     *reinterpret_cast<uint32_t*>(scales_col + scale_offset<LAYOUT>(col0 + c, tile0, kb_col)) = col_scale_word[c];
   if (bits != 8) {
     __syncwarp();
+    if (((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0) {
+      // 32-byte chunks: whole sectors per request
+      constexpr uint32_t kChunks32 = cfg::kSeg / 32;
+      for (uint32_t i = lane; i < 32 * COLS * kChunks32; i += 32) {
+        const uint32_t r = i / kChunks32, ch = i - r * kChunks32;
+        const uint32_t c = r >> 5, owner = r & 31;
+        const uint2* src = reinterpret_cast<const uint2*>(sarea + r * cfg::kPitch + ch * 32);
+        const uint2 q0 = src[0], q1 = src[1], q2 = src[2], q3 = src[3];
+        const uint32_t v[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
+        st_32(elems_col + (size_t)(warp_col0 + owner * COLS + c) * col_out_bytes + (size_t)tile0 * kBpb + ch * 32, v);
+      }
+      return;
+    }
     constexpr uint32_t kChunks = cfg::kSeg / 16;
     for (uint32_t i = lane; i < 32 * COLS * kChunks; i += 32) {
       const uint32_t r = i / kChunks, ch = i - r * kChunks;
