@@ -300,10 +300,10 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
 // coalesced 16-byte stores.  Without this each lane writes its own row and the L2 sees two (8-bit),
 // three (6-bit) or one (4-bit) partial-sector request per block and row, which is what bounded the
 // direct version.  Each warp has a private staging area, so only __syncwarp is needed.
-constexpr int kStagedThreads = 64;
+constexpr int kStagedThreads = 64;  // resident CTAs per SM below: the measured optimum per variant
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
-__global__ void __launch_bounds__(kStagedThreads, 6)
+__global__ void __launch_bounds__(kStagedThreads, (DTYPE == MX_BF16 && FmtTraits<FMT>::bits == 6) ? 6 : 8)
 quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems,
                                uint8_t* __restrict__ scales, uint32_t outer, uint32_t L,
                                uint32_t inner) {
