@@ -16,6 +16,11 @@
 //             MMAs per stage, tcgen05.commit releases the stage / the accumulator
 //   warps 2-9 epilogue: tensor memory -> registers (the accumulator is released as soon as
 //             it is in registers) -> FP32 C, overlapping the next tile's MMAs
+//   warp 10   scale copier: a stage's scale chunks shared -> tensor memory (tcgen05.cp), then
+//             tcgen05.commit tells the MMA issuer.  Every tcgen05 instruction costs its issuing
+//             thread 60-70 clocks; with the three copies of a stage in the MMA thread's stream
+//             (eight instructions, ~620 clocks per stage) that thread, not the tensor pipe
+//             (520 clocks per stage), set the pace.
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status
 // word, raises a CTA-wide abort flag and every role falls through to the common
 // exit, where tensor memory is released.
@@ -34,7 +39,7 @@ namespace {
 constexpr int BM = 128;         // rows of C per tile (= MMA M, one TMEM lane per row)
 constexpr int BK = 128;         // K elements per pipeline stage: 4 MX blocks, 4 MMAs
 constexpr int kMmaK = 32;       // K of one kind::mxf8f6f4 MMA = the MX block size
-constexpr int kThreads = 320;   // 10 warps: producer, MMA issuer, 8 epilogue warps
+constexpr int kThreads = 352;   // 11 warps: producer, MMA issuer, 8 epilogue warps, scale copier
 constexpr int kTmemCols = 512;  // whole tensor memory of the SM (one CTA per SM)
 constexpr long long kSpinLimit = 2000000000LL;  // cycles (~1 s) before a wait gives up
 
@@ -44,6 +49,7 @@ enum : unsigned int {
   ST_MMA_WAIT_FULL = 2,    // MMA issuer: stage never became full
   ST_MMA_WAIT_ACC = 3,     // MMA issuer: accumulator never drained
   ST_EPILOGUE_WAIT = 4,    // epilogue: accumulator never became full
+  ST_SCALE_WAIT = 5,       // scale copier: stage never became full
 };
 
 // First failure of any GEMM launch on this device since the last check (0 = none).
@@ -71,8 +77,8 @@ struct Cfg {
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;   // 1024-byte aligned
   static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
-  // barriers: full[S], empty[S], acc_full[A], acc_empty[A]; then tmem slot + abort flag
-  static constexpr uint32_t kNumBars = 2 * kStages + 2 * kAccStages;
+  // barriers: full[S], empty[S], acc_full[A], acc_empty[A], scales_ready[S]; then tmem slot + abort flag
+  static constexpr uint32_t kNumBars = 3 * kStages + 2 * kAccStages;
   static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;  // + alignment slack
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
   static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -399,6 +405,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (cfg::kStages + s); };
   auto acc_full_bar = [&](uint32_t a) { return bar0 + 8 * (2 * cfg::kStages + a); };
   auto acc_empty_bar = [&](uint32_t a) { return bar0 + 8 * (2 * cfg::kStages + cfg::kAccStages + a); };
+  auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * cfg::kStages + 2 * cfg::kAccStages + s); };
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -415,6 +422,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
+      mbar_init(sf_ready_bar(s), 1);  // the copier's tcgen05.commit
     }
     for (uint32_t a = 0; a < cfg::kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
@@ -490,20 +498,15 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         // scales of row n of the tile sit in column (n0 % 128 + n) / 32 of the copied chunks
         const uint32_t sfb_col = 4 + ((tile_coord(t, tiles_m, tiles_n, group_m).tn * BN) % 128) / 32;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+          // scales in tensor memory (which implies that the stage has landed), then the operands
+          if ((!DENSE && !mbar_wait(sf_ready_bar(stage), phase, abort_flag)) ||
+              !mbar_wait(full_bar(stage), phase, abort_flag)) {
             raise_abort(abort_flag, ST_MMA_WAIT_FULL);
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          if (!DENSE) {
-            tc_cp_scales(sf_tmem, scale_desc(sf_smem));
-#pragma unroll
-            for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
-              tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
-          }
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
 #pragma unroll
@@ -522,6 +525,30 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
         if (ok) tc_commit(acc_full_bar(acc));
         if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp == 10) {
+    // ------------------------------ scale copier ------------------------------
+    if (!DENSE && lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+            raise_abort(abort_flag, ST_SCALE_WAIT);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+          const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
+          tc_cp_scales(sf_tmem, scale_desc(sf_smem));
+#pragma unroll
+          for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
+            tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
+          tc_commit(sf_ready_bar(stage));  // arrives when the copies above have completed
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
       }
     }
   } else {
@@ -616,7 +643,7 @@ struct Cfg2 {
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;
   static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
-  static constexpr uint32_t kNumBars = 2 * kStages + 2;
+  static constexpr uint32_t kNumBars = 3 * kStages + 2;
   static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
   static_assert(kSmemBytes <= 232448, "shared memory budget");
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
@@ -634,6 +661,12 @@ __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   asm volatile(
       "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
       ::"r"(bar), "h"((uint16_t)3) : "memory");
+}
+// The same, delivered to the leader CTA only.
+__device__ __forceinline__ void tc_commit_leader(uint32_t bar) {
+  asm volatile(
+      "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+      ::"r"(bar), "h"((uint16_t)1) : "memory");
 }
 __device__ __forceinline__ void tc_cp_scales_pair(uint32_t taddr, uint64_t sdesc) {
   asm volatile("tcgen05.cp.cta_group::2.32x128b.warpx4 [%0], %1;" ::"r"(taddr), "l"(sdesc) : "memory");
@@ -698,6 +731,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (cfg::kStages + s); };
   const uint32_t acc_full_bar = bar0 + 8 * (2 * cfg::kStages);
   const uint32_t acc_empty_bar = bar0 + 8 * (2 * cfg::kStages + 1);
+  auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * cfg::kStages + 2 + s); };
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -713,6 +747,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
       mbar_init(full_bar(s), 1);   // used in the leader only: its producer's arrive + all bytes
       mbar_init(empty_bar(s), 1);  // one tcgen05.commit per use, delivered to both CTAs
+      mbar_init(sf_ready_bar(s), 1);  // used in the leader only: the copier's tcgen05.commit
     }
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 16);  // eight epilogue warps in each CTA (the leader's barrier is used)
@@ -785,26 +820,15 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         tc_fence_after();
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+          // scales in tensor memory (which implies that the stage has landed), then the operands
+          if ((!DENSE && !mbar_wait(sf_ready_bar(stage), phase, abort_flag)) ||
+              !mbar_wait(full_bar(stage), phase, abort_flag)) {
             raise_abort(abort_flag, ST_MMA_WAIT_FULL);
             ok = false;
             break;
           }
           tc_fence_after();
-          const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          // scale chunks -> TMEM.  A: K chunk c at columns 4c.  B: the box is [row group][K chunk],
-          // and the MMA wants the columns of one K chunk together: group g, chunk c -> 8c + 4g.
-          if constexpr (!DENSE) {
-#pragma unroll
-            for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
-              tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
-#pragma unroll
-              for (uint32_t g = 0; g < 2; ++g)
-                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
-                                  scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
-            }
-          }
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
 #pragma unroll
@@ -828,6 +852,39 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         }
         if (ok) tc_commit_pair(acc_full_bar);
         acc_phase ^= 1u;
+      }
+    }
+  } else if (warp == 10) {
+    // --------------------------- scale copier (leader) ---------------------------
+    if constexpr (!DENSE) {
+      if (lane == 0 && rank == 0) {
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+          for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+            if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+              raise_abort(abort_flag, ST_SCALE_WAIT);
+              ok = false;
+              break;
+            }
+            tc_fence_after();
+            const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+            const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
+            // Each CTA copies from its own shared memory to its own tensor memory.  A: K chunk c at
+            // columns 4c.  B: the box is [row group][K chunk], and the MMA wants the columns of one
+            // K chunk together: group g, chunk c -> 8c + 4g.
+#pragma unroll
+            for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
+              tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
+#pragma unroll
+              for (uint32_t g = 0; g < 2; ++g)
+                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
+                                  scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+            }
+            tc_commit_leader(sf_ready_bar(stage));  // arrives when the copies have completed in both CTAs
+            if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
       }
     }
   } else {
