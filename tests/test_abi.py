@@ -78,3 +78,37 @@ def test_argument_validation_without_gpu():
     assert g(p, p, p, p, p, 128, 128, 128, 0, 9, None) == mx.MX_ERR_FMT
     assert g(None, p, p, p, p, 128, 128, 128, 0, 0, None) == mx.MX_ERR_NULL
     assert lib.mx_strerror(mx.MX_ERR_ALIGN) and lib.mx_strerror(-99)
+
+
+def test_gemm_variants_argument_validation_without_gpu():
+    """The GEMM entry points added beside mx_gemm reject bad arguments before any CUDA call."""
+    lib = mx.lib()
+    buf = np.zeros(4096, np.uint8)
+    p = buf.ctypes.data + (-buf.ctypes.data) % 256
+    F32, BF16 = mx.MX_F32, mx.MX_BF16
+    gb = lib.mx_gemm_bf16
+    assert gb(p, p, p, p, None, 128, 128, 128, 0, 0, None) == mx.MX_ERR_NULL
+    assert gb(p, p, p, p, p, 128, 132, 128, 0, 0, None) == mx.MX_ERR_SHAPE   # BF16 rows of C: N % 8
+    assert gb(p, p, p, p, p, 128, 128, 128, 5, 0, None) == mx.MX_ERR_UNSUPPORTED
+    bt = lib.mx_gemm_batched
+    assert bt(p, p, p, p, p, 7, 2, 128, 128, 128, 0, 0, None) == mx.MX_ERR_FMT       # output dtype
+    assert bt(p, p, p, p, p, F32, 2, 100, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE   # whole tiles only
+    assert bt(p, p, p, p, p, F32, -1, 128, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert bt(p, p, p, p, p, F32, 1 << 30, 128, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
+    assert bt(p, p, p, p, p, BF16, 0, 128, 128, 128, 0, 0, None) == mx.MX_OK         # empty batch
+    gq = lib.mx_gemm_quantize
+    assert gq(p, p, p, p, None, p, 128, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_NULL
+    assert gq(p, p, p, p, p, None, 128, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_NULL
+    assert gq(p, p, p, p, p, p, 128, 128, 128, 0, 0, 6, 0, None) == mx.MX_ERR_FMT
+    assert gq(p, p, p, p, p, p, 128, 128, 128, 0, 0, 0, 2, None) == mx.MX_ERR_FMT
+    assert gq(p, p, p, p, p, p, 100, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_SHAPE   # whole tiles only
+    assert gq(p, p, p, p, p, p + 4, 128, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_ALIGN
+    gd = lib.mx_gemm_dense
+    assert lib.mx_gemm_dense_workspace_bytes(128, 256, 512) == 2 * (128 + 256) * 512
+    assert lib.mx_gemm_dense_workspace_bytes(-1, 256, 512) == 0
+    assert gd(p, p, p, p, p, F32, 128, 128, 128, 5, 5, None, None, 0) == mx.MX_ERR_NULL        # no workspace
+    assert gd(p, p, p, p, p, F32, 128, 128, 128, 5, 5, None, p, 1024) == mx.MX_ERR_WORKSPACE
+    assert gd(p, p, p, p, p, F32, 128, 128, 48, 5, 5, None, p, 1 << 20) == mx.MX_ERR_SHAPE
+    assert gd(p, p, p, p, p, 3, 128, 128, 128, 5, 5, None, p, 1 << 20) == mx.MX_ERR_FMT
+    assert gd(p, p, p, p, p, F32, 128, 128, 128, 6, 5, None, p, 1 << 20) == mx.MX_ERR_FMT
+    assert gd(p, p, p, p, p, F32, 0, 128, 128, 5, 5, None, None, 0) == mx.MX_OK                # nothing to do
