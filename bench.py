@@ -469,7 +469,7 @@ def main_ours(args, rank, world, local_rank):
 # gemm = captured on the 4096^3 case (37.8 + 22.8 MB) and scaled by bytes moved
 # (A + B + scales + C: 640.7 MB for 8192 x 16384 x 4096 against 100.1 MB) -- DRAM traffic of the
 # GEMM grows with the operand and output sizes, each read or written once.
-NCU_TRAFFIC = {"quantize": 174.2e6, "gemm": 62.2e6 * 640.7 / 100.1}
+NCU_TRAFFIC = {"quantize": 176.8e6, "gemm": 60.6e6 * 640.7 / 100.1}
 
 
 def main_reference(args, rank, world):
