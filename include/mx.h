@@ -281,6 +281,46 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
                   const mx_opts_t* opts, void* workspace, size_t workspace_bytes);
 
 /* ------------------------------------------------------------------------- */
+/* Convolution as a dot product (Section 4.1)                                */
+/* ------------------------------------------------------------------------- */
+/*
+ * The paper counts convolution among the dot-product operations that take MX operands.
+ * Here the reduction axis of a 2-D convolution is (kh, kw, C) with the channel innermost,
+ * and an MX block is 32 consecutive channels of one filter tap (C % 32 == 0, so no block
+ * straddles two taps).  The activation x[N, H, W, C] (channels last) is then quantized ONCE
+ * with mx_quantize along C, and mx_im2col lays its codes and scales out as the K-major
+ * operand A[M x K] of mx_gemm, M = N*Ho*Wo, K = kh*kw*C; taps that fall into the zero padding
+ * become zero blocks (codes 0, scale byte 0).  No value is requantized.  With the filter
+ * w[Cout, kh, kw, C] quantized along its last axis (rows = Cout, K = kh*kw*C),
+ *     y[N, Ho, Wo, Cout] = mx_gemm(A, w)        (row-major [M x Cout] is channels-last y).
+ * Ho = (H + 2 pad_h - dil_h (kh - 1) - 1) / stride_h + 1, Wo likewise.  mx_gemm's own shape rules
+ * apply to K = kh*kw*C (a multiple of 128 for 6- and 4-bit codes).
+ */
+typedef struct {
+  int64_t N, H, W, C;          /* activation, channels last                         */
+  int32_t kh, kw;              /* filter taps                                       */
+  int32_t stride_h, stride_w;  /* >= 1                                              */
+  int32_t pad_h, pad_w;        /* zero padding on both sides, >= 0                  */
+  int32_t dil_h, dil_w;        /* >= 1                                              */
+} mx_conv_t;
+
+/* Output extent of the convolution; 0 on bad arguments. */
+int64_t mx_conv_out_h(const mx_conv_t* conv);
+int64_t mx_conv_out_w(const mx_conv_t* conv);
+
+/*
+ * elems_in, scales_in   MX tensor of x viewed as [N*H*W rows x C] (what mx_quantize writes for
+ *                       shape {N, H, W, C}, axis 3); scales in opts->scale_layout.
+ * elems_out             packed [M x kh*kw*C] codes, mx_elems_bytes of that shape.
+ * scales_out            SWIZZLED scale tensor of M rows x kh*kw*C/32 blocks (padding written 0).
+ * Requirements: C % 32 == 0 and C * bits / 8 a multiple of 16 (6-bit codes: C % 64 == 0);
+ * all four pointers 16-byte aligned; the output codes below 64 GiB (2^32 16-byte chunks).
+ * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN, MX_ERR_CUDA.
+ */
+int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, uint8_t* scales_out,
+              const mx_conv_t* conv, mx_fmt_t fmt, const mx_opts_t* opts);
+
+/* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */
 /* ------------------------------------------------------------------------- */
 /*

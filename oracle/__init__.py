@@ -2,9 +2,10 @@
 
 TEST INFRASTRUCTURE.  Only ``tests/``, ``__graft_entry__.smoke()`` and the CPU
 baseline legs of ``bench.py`` may import this package; the product package never
-does.  It holds no arithmetic of its own: every function marshals numpy arrays
-into the C routines, which restate Section 2 (values of an MX block), Section 3
-/ Algorithm 1 (conversion) and Section 4.1 (dot product) of arXiv 2310.10537.
+does.  Every function but the last two marshals numpy arrays into the C routines,
+which restate Section 2 (values of an MX block), Section 3 / Algorithm 1
+(conversion) and Section 4.1 (dot product) of arXiv 2310.10537; the convolution
+helpers at the end are the textbook definition written out in numpy (FP64).
 """
 from __future__ import annotations
 
@@ -202,3 +203,55 @@ def gemm_samples(A, sA, B, sB, M: int, N: int, K: int, fmtA: int, fmtB: int, ms,
     if rc != 0:
         raise ValueError(f"oracle_gemm_samples failed: {rc}")
     return c, s
+
+
+def conv_out_hw(H: int, W: int, kh: int, kw: int, stride, pad, dilation):
+    """Output extent of a 2-D convolution with zero padding on both sides."""
+    Ho = (H + 2 * pad[0] - dilation[0] * (kh - 1) - 1) // stride[0] + 1
+    Wo = (W + 2 * pad[1] - dilation[1] * (kw - 1) - 1) // stride[1] + 1
+    return Ho, Wo
+
+
+def conv2d_nhwc(x: np.ndarray, w: np.ndarray, stride=(1, 1), pad=(0, 0), dilation=(1, 1)):
+    """Convolution as the dot product it is (Section 4.1 lists it among the dot-product operations):
+    y[n, ho, wo, co] = sum_{i, j, c} x[n, ho*s_h - p_h + i*d_h, wo*s_w - p_w + j*d_w, c] * w[co, i, j, c],
+    with x = 0 outside the image.  x[N, H, W, C] and w[Cout, kh, kw, C] are the VALUES of the
+    operands (for MX operands: their dequantized values in FP64).  Returns (y, s) in FP64, s being the
+    same sum over absolute values (the scale of the accumulation-error bound)."""
+    x = np.asarray(x, dtype=np.float64)
+    w = np.asarray(w, dtype=np.float64)
+    N, H, W, C = x.shape
+    Cout, kh, kw, Cw = w.shape
+    assert C == Cw
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad, dilation)
+    xp = np.zeros((N, H + 2 * pad[0], W + 2 * pad[1], C), dtype=np.float64)
+    xp[:, pad[0]:pad[0] + H, pad[1]:pad[1] + W, :] = x
+    y = np.zeros((N, Ho, Wo, Cout), dtype=np.float64)
+    s = np.zeros_like(y)
+    for i in range(kh):
+        for j in range(kw):
+            h0, w0 = i * dilation[0], j * dilation[1]
+            patch = xp[:, h0:h0 + (Ho - 1) * stride[0] + 1:stride[0],
+                       w0:w0 + (Wo - 1) * stride[1] + 1:stride[1], :]          # [N, Ho, Wo, C]
+            y += patch @ w[:, i, j, :].T
+            s += np.abs(patch) @ np.abs(w[:, i, j, :]).T
+    return y, s
+
+
+def im2col_source_pixels(N: int, H: int, W: int, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
+                         dilation=(1, 1)) -> np.ndarray:
+    """For every output pixel m = (n, ho, wo) and filter tap t = (i, j): the index n*H*W + hi*W + wi
+    of the input pixel that the tap reads, or -1 where it falls into the padding.  Shape [M, kh*kw]."""
+    Ho, Wo = conv_out_hw(H, W, kh, kw, stride, pad, dilation)
+    src = np.full((N * Ho * Wo, kh * kw), -1, dtype=np.int64)
+    for n in range(N):
+        for ho in range(Ho):
+            for wo in range(Wo):
+                m = (n * Ho + ho) * Wo + wo
+                for i in range(kh):
+                    for j in range(kw):
+                        hi = ho * stride[0] - pad[0] + i * dilation[0]
+                        wi = wo * stride[1] - pad[1] + j * dilation[1]
+                        if 0 <= hi < H and 0 <= wi < W:
+                            src[m, i * kw + j] = (n * H + hi) * W + wi
+    return src

@@ -32,7 +32,7 @@ EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
     "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
-    "mx_gemm_dense",
+    "mx_gemm_dense", "mx_conv_out_h", "mx_conv_out_w", "mx_im2col",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -42,6 +42,14 @@ EXPORTS = [
 class mx_opts_t(ctypes.Structure):
     _fields_ = [("dtype", ctypes.c_int32), ("scale_layout", ctypes.c_int32),
                 ("stream", ctypes.c_void_p), ("check_status", ctypes.c_int32)]
+
+
+class mx_conv_t(ctypes.Structure):
+    _fields_ = [("N", ctypes.c_int64), ("H", ctypes.c_int64), ("W", ctypes.c_int64), ("C", ctypes.c_int64),
+                ("kh", ctypes.c_int32), ("kw", ctypes.c_int32),
+                ("stride_h", ctypes.c_int32), ("stride_w", ctypes.c_int32),
+                ("pad_h", ctypes.c_int32), ("pad_w", ctypes.c_int32),
+                ("dil_h", ctypes.c_int32), ("dil_w", ctypes.c_int32)]
 
 
 class MxError(RuntimeError):
@@ -81,6 +89,12 @@ def _load() -> ctypes.CDLL:
     lib.mx_gemm_dense_workspace_bytes.argtypes = [i64, i64, i64]
     lib.mx_gemm_dense_workspace_bytes.restype = sz
     lib.mx_gemm_dense.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, ci, ci, op, vp, sz]
+    cp = ctypes.POINTER(mx_conv_t)
+    lib.mx_conv_out_h.argtypes = [cp]
+    lib.mx_conv_out_h.restype = i64
+    lib.mx_conv_out_w.argtypes = [cp]
+    lib.mx_conv_out_w.restype = i64
+    lib.mx_im2col.argtypes = [vp, u8p, vp, u8p, cp, ci, op]
     lib.mx_gemm_batched.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
@@ -282,6 +296,30 @@ def mx_gemm_dense(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.
                               _dtype_code(out.dtype), M, N, K, fmtA, fmtB, ctypes.byref(o),
                               workspace.data_ptr(), workspace.numel()), "mx_gemm_dense")
     return out
+
+
+def mx_conv_geometry(N: int, H: int, W: int, C: int, kh: int, kw: int, stride=(1, 1), pad=(0, 0),
+                     dilation=(1, 1)) -> mx_conv_t:
+    return mx_conv_t(N, H, W, C, kh, kw, stride[0], stride[1], pad[0], pad[1], dilation[0], dilation[1])
+
+
+def mx_conv_out_hw(conv: mx_conv_t) -> Tuple[int, int]:
+    return int(_lib.mx_conv_out_h(ctypes.byref(conv))), int(_lib.mx_conv_out_w(ctypes.byref(conv)))
+
+
+def mx_im2col(elems: torch.Tensor, scales: torch.Tensor, conv: mx_conv_t, fmt: int,
+              layout: int = MX_SCALES_SWIZZLED) -> Tuple[torch.Tensor, torch.Tensor]:
+    """The MX tensor of x[N, H, W, C] (quantized along C) laid out as the K-major operand
+    [N*Ho*Wo x kh*kw*C] of mx_gemm: (codes, swizzled scales)."""
+    assert elems.is_cuda and scales.is_cuda
+    Ho, Wo = mx_conv_out_hw(conv)
+    M, K = conv.N * Ho * Wo, conv.kh * conv.kw * conv.C
+    out_e = torch.empty(M * K * mx_fmt_bits(fmt) // 8, dtype=torch.uint8, device=elems.device)
+    out_s = torch.empty(mx_scales_bytes((M, K), 1, MX_SCALES_SWIZZLED), dtype=torch.uint8, device=elems.device)
+    o = _opts(MX_F32, layout)
+    _check(_lib.mx_im2col(elems.data_ptr(), scales.data_ptr(), out_e.data_ptr(), out_s.data_ptr(),
+                          ctypes.byref(conv), fmt, ctypes.byref(o)), "mx_im2col")
+    return out_e, out_s
 
 
 # ---- host-buffer variants: tensors live in (pinned) host memory ----------------

@@ -504,6 +504,59 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
   return MX_OK;
 }
 
+static bool conv_ok(const mx_conv_t* c) {
+  return c && c->N >= 0 && c->H > 0 && c->W > 0 && c->C > 0 && c->kh > 0 && c->kw > 0 && c->stride_h > 0 &&
+         c->stride_w > 0 && c->pad_h >= 0 && c->pad_w >= 0 && c->dil_h > 0 && c->dil_w > 0 &&
+         c->H < ((int64_t)1 << 30) && c->W < ((int64_t)1 << 30);
+}
+
+int64_t mx_conv_out_h(const mx_conv_t* c) {
+  if (!conv_ok(c)) return 0;
+  const int64_t span = c->H + 2 * (int64_t)c->pad_h - (int64_t)c->dil_h * (c->kh - 1) - 1;
+  return span < 0 ? 0 : span / c->stride_h + 1;
+}
+
+int64_t mx_conv_out_w(const mx_conv_t* c) {
+  if (!conv_ok(c)) return 0;
+  const int64_t span = c->W + 2 * (int64_t)c->pad_w - (int64_t)c->dil_w * (c->kw - 1) - 1;
+  return span < 0 ? 0 : span / c->stride_w + 1;
+}
+
+int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, uint8_t* scales_out,
+              const mx_conv_t* conv, mx_fmt_t fmt, const mx_opts_t* opts) {
+  Opts o;
+  if (!conv) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (!conv_ok(conv)) return MX_ERR_SHAPE;
+  const int bits = fmt_bits((int)fmt);
+  if (conv->C % 32 || (conv->C * bits / 8) % 16) return MX_ERR_SHAPE;
+  const int64_t Ho = mx_conv_out_h(conv), Wo = mx_conv_out_w(conv);
+  if (Ho <= 0 || Wo <= 0) return MX_ERR_SHAPE;
+  const int64_t taps = (int64_t)conv->kh * conv->kw;
+  const int64_t M = conv->N * Ho * Wo;
+  // 32-bit chunk indices in the gather: the output holds fewer than 2^32 16-byte chunks
+  if (conv->N * conv->H * conv->W >= ((int64_t)1 << 31) || M * taps * (conv->C * bits / 8 / 16) >= ((int64_t)1 << 32) ||
+      M * taps >= ((int64_t)1 << 31) || taps * conv->C >= ((int64_t)1 << 31))
+    return MX_ERR_SHAPE;
+  if (M == 0) return MX_OK;
+  if (!elems_in || !scales_in || !elems_out || !scales_out) return MX_ERR_NULL;
+  if ((uintptr_t)elems_in % 16 || (uintptr_t)scales_in % 16 || (uintptr_t)elems_out % 16 ||
+      (uintptr_t)scales_out % 16)
+    return MX_ERR_ALIGN;
+  cudaError_t e;
+  mx::Im2colArgs a;
+  a.elems_in = (const uint8_t*)elems_in; a.scales_in = scales_in;
+  a.elems_out = (uint8_t*)elems_out; a.scales_out = scales_out;
+  a.N = conv->N; a.H = conv->H; a.W = conv->W; a.C = conv->C; a.Ho = Ho; a.Wo = Wo;
+  a.kh = conv->kh; a.kw = conv->kw; a.stride_h = conv->stride_h; a.stride_w = conv->stride_w;
+  a.pad_h = conv->pad_h; a.pad_w = conv->pad_w; a.dil_h = conv->dil_h; a.dil_w = conv->dil_w;
+  a.bits = bits; a.layout_in = o.layout; a.stream = o.stream;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  e = mx::launch_im2col(a);
+  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {
   if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || M < 0 || N < 0 || K < 0 || K % 32) return 0;
   return align_up((size_t)(M * K / 8 * fmt_bits((int)fmtA)), 256) +

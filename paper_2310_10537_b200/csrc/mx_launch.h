@@ -41,6 +41,20 @@ struct DequantizeArgs {
 };
 cudaError_t launch_dequantize(const DequantizeArgs& a);
 
+// Activation x[N, H, W, C] quantized along C -> K-major operand [N Ho Wo x kh kw C] (see mx_im2col()).
+struct Im2colArgs {
+  const uint8_t* elems_in;
+  const uint8_t* scales_in;
+  uint8_t* elems_out;
+  uint8_t* scales_out;  // swizzled
+  int64_t N, H, W, C, Ho, Wo;
+  int kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+  int bits, layout_in;
+  int sm_count;
+  cudaStream_t stream;
+};
+cudaError_t launch_im2col(const Im2colArgs& a);
+
 struct GemmArgs {
   const void* A;
   const uint8_t* sA;

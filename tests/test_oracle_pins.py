@@ -424,3 +424,45 @@ def test_gemm_closed_forms():
     sa3[O.scale_offset(2, 0, 8, 3, O.SWIZZLED)] = 0xFF
     C3, _ = O.gemm(ea, sa3, eb, sb, 8, 12, 96, O.E4M3, O.E2M1)
     assert np.isnan(C3[2]).all() and not np.isnan(np.delete(C3, 2, axis=0)).any()
+
+
+# ---- convolution helpers (the definition written out; pinned to brute force and to a library) ----
+
+def test_conv_oracle_against_brute_force_and_library():
+    import torch
+    rng = np.random.default_rng(5)
+    for (N, H, W, C, Cout, kh, kw, st, pd, dl) in [(1, 5, 6, 3, 2, 3, 3, (1, 1), (1, 1), (1, 1)),
+                                                   (2, 7, 5, 4, 3, 3, 2, (2, 1), (0, 2), (1, 2)),
+                                                   (1, 4, 4, 2, 2, 1, 1, (1, 1), (0, 0), (1, 1)),
+                                                   (1, 9, 8, 2, 1, 2, 3, (3, 2), (2, 1), (2, 1))]:
+        x = rng.standard_normal((N, H, W, C))
+        w = rng.standard_normal((Cout, kh, kw, C))
+        y, s = O.conv2d_nhwc(x, w, st, pd, dl)
+        Ho, Wo = O.conv_out_hw(H, W, kh, kw, st, pd, dl)
+        assert y.shape == (N, Ho, Wo, Cout)
+        # brute force, one output at a time, straight from the formula
+        for n in range(N):
+            for ho in range(Ho):
+                for wo in range(Wo):
+                    for co in range(Cout):
+                        acc = 0.0
+                        acc_abs = 0.0
+                        for i in range(kh):
+                            for j in range(kw):
+                                hi, wi = ho * st[0] - pd[0] + i * dl[0], wo * st[1] - pd[1] + j * dl[1]
+                                if 0 <= hi < H and 0 <= wi < W:
+                                    acc += float(np.dot(x[n, hi, wi], w[co, i, j]))
+                                    acc_abs += float(np.dot(np.abs(x[n, hi, wi]), np.abs(w[co, i, j])))
+                        assert abs(acc - y[n, ho, wo, co]) < 1e-12
+                        assert abs(acc_abs - s[n, ho, wo, co]) < 1e-12
+        # the library routine (channels first)
+        ref = torch.nn.functional.conv2d(torch.from_numpy(x).permute(0, 3, 1, 2),
+                                         torch.from_numpy(w).permute(0, 3, 1, 2), stride=st, padding=pd,
+                                         dilation=dl).permute(0, 2, 3, 1).numpy()
+        assert np.allclose(ref, y, atol=1e-12)
+        # the gather table agrees with the same index arithmetic done by the library on an index image
+        src = O.im2col_source_pixels(N, H, W, kh, kw, st, pd, dl)
+        idx_img = torch.arange(1, N * H * W + 1, dtype=torch.float64).view(N, 1, H, W)   # 0 = padding
+        cols = torch.nn.functional.unfold(idx_img, (kh, kw), dilation=dl, padding=pd, stride=st)  # [N, kh*kw, Ho*Wo]
+        want = cols.permute(0, 2, 1).reshape(N * Ho * Wo, kh * kw).numpy().astype(np.int64) - 1
+        assert np.array_equal(src, want)
