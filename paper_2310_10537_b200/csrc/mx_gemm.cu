@@ -623,21 +623,28 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 // MMA, two MX blocks and therefore two scales per row and instruction: scale_vec::2X), which doubles
 // the MACs per operand byte and per tensor-core cycle.  A stage then holds 256 K-elements.
 // KIND 2 = dense BF16 operands (kind::f16, see mx_gemm_kernel): 64 K-elements per stage, no scales.
-template <int KIND>
+// BN = 384: the pair computes a 256 x 384 tile -- per stage one MMA with N = 256 (B rows 0..255 of the
+// tile, 128 per CTA) and one with N = 128 (rows 256..383, 64 per CTA) -- which lowers the operand
+// bytes each SM pulls from L2 per MAC from 1/128 to 1/153.6.  384 accumulator columns leave room for
+// four stages of scale columns.
+template <int KIND, int BN_>
 struct Cfg2 {
+  static_assert(BN_ == 256 || BN_ == 384, "tile width");
   static constexpr bool F4 = KIND == 1;
   static constexpr bool DENSE = KIND == 2;
-  static constexpr int BN = 256;
-  static constexpr int kStages = F4 ? 5 : 6;
+  static constexpr int BN = BN_;
+  static constexpr int kStages = BN == 384 ? 4 : (F4 ? 5 : 6);
   static constexpr int kBKe = F4 ? 256 : DENSE ? 64 : 128;  // K elements per stage (128-byte operand rows)
   static constexpr int kKChunks = F4 ? 2 : 1;           // 512-byte scale chunks (4 MX blocks) along K per stage
+  static constexpr int kSfbGroups = BN / 128;           // 128-row scale chunks of B per K chunk
   static constexpr int kSfColsA = 4 * kKChunks;         // TMEM columns: this CTA's 128 rows of A
-  static constexpr int kSfCols = kSfColsA + 8 * kKChunks;  // ... plus all 256 rows of B
+  static constexpr int kSfCols = kSfColsA + 4 * kSfbGroups * kKChunks;  // ... plus all BN rows of B
   static constexpr int kSfCol0 = BN;                    // single accumulator stage
+  static constexpr uint32_t kBRows = BN / 2;            // rows of B this CTA stages
   static constexpr uint32_t kABytes = 128 * 128;        // this CTA's 128 rows of A, 128 bytes each
-  static constexpr uint32_t kBBytes = 128 * 128;        // this CTA's 128 rows of B
+  static constexpr uint32_t kBBytes = kBRows * 128;
   static constexpr uint32_t kSfABytes = 512 * kKChunks;
-  static constexpr uint32_t kSfBytes = kSfABytes + 1024 * kKChunks;
+  static constexpr uint32_t kSfBytes = kSfABytes + 512 * kSfbGroups * kKChunks;
   static constexpr uint32_t kOffA = 0;
   static constexpr uint32_t kOffB = kOffA + kStages * kABytes;
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;
@@ -710,18 +717,21 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <int KIND>
+template <int KIND, int BN_>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
 mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_b2,
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
                     uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
                     uint32_t batch) {
-  using cfg = Cfg2<KIND>;
+  using cfg = Cfg2<KIND, BN_>;
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
-  constexpr uint32_t kProd = DENSE ? 2 : 4;
-  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
   constexpr int BN = cfg::BN;
+  constexpr bool WIDE = BN == 384;
+  // copies per stage, one producer lane each: A, B, [second part of B], [A scales, B scales]
+  constexpr uint32_t kProd = (DENSE ? 2 : 4) + (WIDE ? 1 : 0);
+  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -774,20 +784,26 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   if (warp == 0) {
     // ------------------------- TMA producer (both CTAs) -------------------------
     if (lane < kProd) {
-      const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
-      const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
-                                                                                         : cfg::kOffSf + cfg::kSfABytes;
-      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : lane == 1 ? cfg::kBBytes : cfg::kSfBytes;
+      // role of this lane: 0 A, 1 B (rows 128 rank .. of the tile), 2 second part of B (wide tile:
+      // rows 256 + 64 rank ..), 3 A scales, 4 B scales
+      const uint32_t role = WIDE ? lane : (lane < 2 ? lane : lane + 1);
+      const CUtensorMap* map = role == 0 ? &tmap_a : role == 1 ? &tmap_b : role == 2 ? &tmap_b2
+                               : role == 3 ? &tmap_sa : &tmap_sb;
+      const uint32_t dst_off = role == 0 ? cfg::kOffA : role == 1 ? cfg::kOffB : role == 2 ? cfg::kOffB + 128u * 128u
+                               : role == 3 ? cfg::kOffSf : cfg::kOffSf + cfg::kSfABytes;
+      const uint32_t dst_stride = role == 0 ? cfg::kABytes : role < 3 ? cfg::kBBytes : cfg::kSfBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        // this CTA's 128 rows of A and of B (B rows may lie past N on a ragged tile: zero fill);
-        // its own A scales and the B scales of all 256 columns
-        const int cy_fixed = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
-                                       : (int)(tc.b * N + tc.tn * BN + rank * 128);
-        const int cz = lane == 2 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
-                                 : lane == 3 ? (int)(tc.b * (N / 128) + tc.tn * 2) : 0;
+        // this CTA's 128 rows of A and its rows of B (B rows may lie past N on a ragged tile: zero
+        // fill or the next matrix of a batch; their columns are not stored); its own A scales and the
+        // B scales of all BN columns
+        const int cy_fixed = role == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
+                             : role == 1 ? (int)(tc.b * N + tc.tn * BN + rank * 128)
+                                         : (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
+        const int cz = role == 3 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
+                                 : role == 4 ? (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups) : 0;
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
@@ -797,8 +813,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
           __syncwarp(kProdMask);
-          const int cx = lane < 2 ? (int)(kc * BKe) : 0;
-          const int cy = lane < 2 ? cy_fixed : (int)(kc * cfg::kKChunks);
+          const int cx = role < 3 ? (int)(kc * BKe) : 0;
+          const int cy = role < 3 ? cy_fixed : (int)(kc * cfg::kKChunks);
           tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
@@ -831,20 +847,33 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
           const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
           const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
+          // wide tile: columns 256..383 come from a second MMA with N = 128 on the B rows staged
+          // behind the first 128 (64 per CTA); its B scales are the third 128-row group
+          const uint64_t bdesc2 = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u);
+          const uint32_t idesc2_base = (idesc_base & ~(0x3Fu << 17)) | ((uint32_t)(128 >> 3) << 17);
+          constexpr uint32_t kSfbStep = 4 * cfg::kSfbGroups;  // B scale columns per K chunk
 #pragma unroll
           for (uint32_t k = 0; k < 4; ++k) {  // every MMA advances 32 bytes along the 128-byte rows
+            const uint32_t acc_flag = (kc | k) != 0 ? 1u : 0u;
             if (DENSE) {
-              tc_mma_pair_dense(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base, (kc | k) != 0 ? 1u : 0u);
+              tc_mma_pair_dense(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base, acc_flag);
+              if (WIDE) tc_mma_pair_dense(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base, acc_flag);
             } else if (F4) {
               // K = 64: blocks 2k and 2k+1 of the stage = bytes (2k % 4, +1) of K chunk k / 2
               const uint32_t sf_id = 2 * (k & 1);
-              const uint32_t idesc = idesc_base | (sf_id << 4) | (sf_id << 29);
-              tc_mma_pair_f4(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem + 4 * (k >> 1),
-                             sf_tmem + cfg::kSfColsA + 8 * (k >> 1), (kc | k) != 0 ? 1u : 0u);
+              const uint32_t sel = (sf_id << 4) | (sf_id << 29);
+              const uint32_t sfa = sf_tmem + 4 * (k >> 1), sfb = sf_tmem + cfg::kSfColsA + kSfbStep * (k >> 1);
+              tc_mma_pair_f4(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base | sel, sfa, sfb, acc_flag);
+              if (WIDE)
+                tc_mma_pair_f4(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base | sel, sfa, sfb + 8,
+                               acc_flag);
             } else {
-              const uint32_t idesc = idesc_base | (k << 4) | (k << 29);  // byte k of the scale columns
-              tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc, sf_tmem, sf_tmem + cfg::kSfColsA,
-                          (kc | k) != 0 ? 1u : 0u);
+              const uint32_t sel = (k << 4) | (k << 29);  // byte k of the scale columns
+              const uint32_t sfb = sf_tmem + cfg::kSfColsA;
+              tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base | sel, sf_tmem, sfb, acc_flag);
+              if (WIDE)
+                tc_mma_pair(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base | sel, sf_tmem, sfb + 8,
+                            acc_flag);
             }
           }
           tc_commit_pair(empty_bar(stage));
@@ -872,13 +901,13 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
             // Each CTA copies from its own shared memory to its own tensor memory.  A: K chunk c at
             // columns 4c.  B: the box is [row group][K chunk], and the MMA wants the columns of one
-            // K chunk together: group g, chunk c -> 8c + 4g.
+            // K chunk together: group g of G, chunk c -> 4 G c + 4g.
 #pragma unroll
             for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
               tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
 #pragma unroll
-              for (uint32_t g = 0; g < 2; ++g)
-                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 8 * c + 4 * g,
+              for (uint32_t g = 0; g < cfg::kSfbGroups; ++g)
+                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 4 * cfg::kSfbGroups * c + 4 * g,
                                   scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
             }
             tc_commit_leader(sf_ready_bar(stage));  // arrives when the copies have completed in both CTAs
@@ -900,22 +929,46 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         break;
       }
       tc_fence_after();
-      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + half * kHalf;
-      const uint32_t col0 = tc.tn * BN + half * kHalf;
-      const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;
-      uint32_t r[kLoads][32];
-#pragma unroll
-      for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
-      tc_wait_ld();
-      tc_fence_before();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
       const uint32_t row0 = (tc.b * tiles_m + tc.tm) * 256 + rank * 128 + quarter * 32;
-      if (epi.mode == 2) {
-        if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
+      if constexpr (WIDE) {
+        // 192 columns per warp in two passes of 96 (registers); the accumulator is handed back
+        // after the second pass's loads.  The quantizing epilogue is not offered at this width.
+        constexpr uint32_t kPass = 96, kPassLoads = 3;
+#pragma unroll 1
+        for (uint32_t pass = 0; pass < 2; ++pass) {
+          const uint32_t cofs = half * kHalf + pass * kPass;
+          const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + cofs;
+          const uint32_t col0 = tc.tn * BN + cofs;
+          const uint32_t valid_cols = col0 < N ? min(kPass, N - col0) : 0u;
+          uint32_t r[kPassLoads][32];
+#pragma unroll
+          for (uint32_t j = 0; j < kPassLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
+          tc_wait_ld();
+          if (pass == 1) {
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_leader(acc_empty_bar);
+          }
+          store_rows<kPassLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                                 (int)col0, (int)row0, valid_cols, lane, epi.mode);
+        }
       } else {
-        store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
-                           (int)col0, (int)row0, valid_cols, lane, epi.mode);
+        const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + half * kHalf;
+        const uint32_t col0 = tc.tn * BN + half * kHalf;
+        const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;
+        uint32_t r[kLoads][32];
+#pragma unroll
+        for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
+        tc_wait_ld();
+        tc_fence_before();
+        __syncwarp();
+        if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
+        if (epi.mode == 2) {
+          if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
+        } else {
+          store_rows<kLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
+                             (int)col0, (int)row0, valid_cols, lane, epi.mode);
+        }
       }
       acc_phase ^= 1u;
     }
@@ -1083,11 +1136,12 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
 }
 
 // Dense FP4 operand map for kind::mxf4: two codes per byte in shared memory as in global memory.
-bool make_f4_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K) {
+bool make_f4_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t rows, uint64_t K,
+                 uint32_t box_rows = 128) {
   const cuuint64_t pitch = K / 2;
   const cuuint64_t dims[3] = {K, rows, 1};
   const cuuint64_t strides[2] = {pitch, pitch * rows};
-  const cuuint32_t box[3] = {256, 128, 1};
+  const cuuint32_t box[3] = {256, box_rows, 1};
   const cuuint32_t estr[3] = {1, 1, 1};
   return fn(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN8B, 3, const_cast<void*>(ptr), dims, strides, box, estr,
             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
@@ -1107,26 +1161,30 @@ bool make_scale_map_k(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint6
             CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int KIND>
+template <int KIND, int BN>
 cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
-  using cfg = Cfg2<KIND>;
-  constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
-  CUtensorMap ma, mb, msa, msb, mc;
+  using cfg = Cfg2<KIND, BN>;
+  constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE, WIDE = BN == 384;
+  // rows of B a CTA takes with its second copy (wide tile): 64; the map is unused otherwise
+  constexpr uint32_t kB2Rows = WIDE ? 64 : 128;
+  const uint64_t rows_a = (uint64_t)(a.batch * a.M), rows_b = (uint64_t)(a.batch * a.N), K = (uint64_t)a.K;
+  CUtensorMap ma, mb, mb2, msa, msb, mc;
   bool ok = make_out_map(fn, &mc, a);
   if (DENSE) {
-    ok = ok && make_dense_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
-         make_dense_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
+    ok = ok && make_dense_map(fn, &ma, a.A, rows_a, K, 128) && make_dense_map(fn, &mb, a.B, rows_b, K, 128) &&
+         make_dense_map(fn, &mb2, a.B, rows_b, K, kB2Rows);
     msa = ma;  // no scales: valid descriptors the kernel never uses
     msb = mb;
   } else {
-    ok = ok && make_scale_map_k(fn, &msa, a.sA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 1, cfg::kKChunks) &&
-         make_scale_map_k(fn, &msb, a.sB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 2, cfg::kKChunks);
+    ok = ok && make_scale_map_k(fn, &msa, a.sA, rows_a, K, 1, cfg::kKChunks) &&
+         make_scale_map_k(fn, &msb, a.sB, rows_b, K, cfg::kSfbGroups, cfg::kKChunks);
     if (F4)
-      ok = ok && make_f4_map(fn, &ma, a.A, (uint64_t)(a.batch * a.M), (uint64_t)a.K) &&
-           make_f4_map(fn, &mb, a.B, (uint64_t)(a.batch * a.N), (uint64_t)a.K);
+      ok = ok && make_f4_map(fn, &ma, a.A, rows_a, K) && make_f4_map(fn, &mb, a.B, rows_b, K) &&
+           make_f4_map(fn, &mb2, a.B, rows_b, K, kB2Rows);
     else
-      ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, (uint64_t)(a.batch * a.M), (uint64_t)a.K, 128) &&
-           make_operand_map(fn, &mb, a.B, a.fmtB, (uint64_t)(a.batch * a.N), (uint64_t)a.K, 128);
+      ok = ok && make_operand_map(fn, &ma, a.A, a.fmtA, rows_a, K, 128) &&
+           make_operand_map(fn, &mb, a.B, a.fmtB, rows_b, K, 128) &&
+           make_operand_map(fn, &mb2, a.B, a.fmtB, rows_b, K, kB2Rows);
   }
   if (!ok) return cudaErrorInvalidValue;
   static bool attr_set[64] = {false};
@@ -1134,24 +1192,26 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   cudaError_t e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(mx_gemm_pair_kernel<KIND>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+    e = cudaFuncSetAttribute(mx_gemm_pair_kernel<KIND, BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              (int)cfg::kSmemBytes);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / 256) * (uint32_t)((a.N + 255) / 256);
+  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / 256) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
-  const uint32_t op_bytes = (F4 || DENSE) ? 2u * 128u * 128u
-                               : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 128 * BK * fmt_bits(a.fmtB) / 8);
+  const uint32_t rows_per_cta = 128u + cfg::kBRows;
+  const uint32_t op_bytes = (F4 || DENSE) ? rows_per_cta * 128u
+                               : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + cfg::kBRows * BK * fmt_bits(a.fmtB) / 8);
   const uint32_t tx_pair = 2u * (op_bytes + (DENSE ? 0u : cfg::kSfBytes));
   // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code();
-  // kind::f16: BF16 = 1 for both operands, FP32 accumulator = 1 in bits [4,6), no scale-format bit
+  // kind::f16: BF16 = 1 for both operands, FP32 accumulator = 1 in bits [4,6), no scale-format bit.
+  // N field = 256: the first (or only) MMA of a K step; the kernel derives the N = 128 one.
   const uint32_t fa = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtA), fb = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtB);
   const uint32_t idesc = (fa << 7) | (fb << 10) | (DENSE ? (1u << 4) : (1u << 23)) |
                          ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-  mx_gemm_pair_kernel<KIND><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
-      ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
+  mx_gemm_pair_kernel<KIND, BN><<<2 * pairs, kThreads, cfg::kSmemBytes, a.stream>>>(
+      ma, mb, mb2, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
       epi_args(a), (uint32_t)a.batch);
   return cudaGetLastError();
 }
@@ -1170,7 +1230,14 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   if (a.M % 256 == 0 && a.batch * (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
     const bool f4 = !a.dense && a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
-    *cuda_err = a.dense ? launch_pair<2>(a, fn) : f4 ? launch_pair<1>(a, fn) : launch_pair<0>(a, fn);
+    // 256 x 384 tiles pull fewer operand bytes per MAC from L2; taken only when pinned
+    // (force_bn): measured slower than 256 x 256 for FP8 (four stages in flight instead of six)
+    const int64_t tiles384 = a.batch * (a.M / 256) * ((a.N + 383) / 384);
+    const bool wide = a.q_elems == nullptr && a.force_bn == 384 && tiles384 >= a.sm_count / 2;
+    if (wide)
+      *cuda_err = a.dense ? launch_pair<2, 384>(a, fn) : f4 ? launch_pair<1, 384>(a, fn) : launch_pair<0, 384>(a, fn);
+    else
+      *cuda_err = a.dense ? launch_pair<2, 256>(a, fn) : f4 ? launch_pair<1, 256>(a, fn) : launch_pair<0, 256>(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
   CUtensorMap ma, mb;

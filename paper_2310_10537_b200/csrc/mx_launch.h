@@ -72,6 +72,7 @@ struct GemmArgs {
   int64_t batch;  // independent products; operands and C are the matrices stacked along rows
   int64_t M, N, K;
   int fmtA, fmtB;
+  int force_bn;  // 0: let launch_gemm choose the tile width; 256 / 384: pin it (tuning and tests)
   int sm_count;
   cudaStream_t stream;
 };
