@@ -329,6 +329,11 @@ int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, u
  * workspace of at least mx_*_host_workspace_bytes(); the call copies the
  * inputs to it, runs the device entry point above, copies the results back and
  * synchronises opts->stream.  Additional error: MX_ERR_WORKSPACE.
+ * mx_quantize_host and mx_dequantize_host cut a tensor of 8 MiB or more whose
+ * blocks run along its last axis into row chunks and overlap the copies of
+ * neighbouring chunks in the two directions of the host link; for that they
+ * create, once per device, two streams and a few events of their own (work queued
+ * on opts->stream before the call still comes first).
  */
 size_t mx_quantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis,
                                         mx_fmt_t fmt, const mx_opts_t* opts);

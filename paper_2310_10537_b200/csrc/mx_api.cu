@@ -235,9 +235,61 @@ size_t mx_quantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis
          align_up(scales_bytes(v.rows, v.kblocks, o.layout), 256);
 }
 
-int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
-                     const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
-                     const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+}  // extern "C"
+
+namespace {
+
+// Two internal streams and a few events per device for the host-buffer entry points: a tensor
+// whose blocks run along the last axis is cut into row chunks (multiples of 128 rows, so every
+// chunk owns whole pieces of the packed tensor and of either scale layout); chunk i + 1 travels to
+// the device while chunk i is converted and chunk i - 1 travels back, which keeps both directions
+// of the host link busy instead of one after the other.
+constexpr int kMaxChunks = 4;                // measured: 3 to 8 chunks differ by a few per cent
+constexpr size_t kMinChunkBytes = 4u << 20;  // of float data; below this the copies are latency-bound
+
+struct HostPipe {
+  cudaStream_t in = nullptr, out = nullptr;
+  cudaEvent_t start = nullptr, done[kMaxChunks] = {};
+  bool ready = false;
+};
+
+HostPipe* host_pipe(cudaError_t* err) {
+  static HostPipe pipes[64];
+  int dev = 0;
+  *err = cudaGetDevice(&dev);
+  if (*err != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  HostPipe* p = &pipes[dev];
+  if (p->ready) return p;
+  if ((*err = cudaStreamCreateWithFlags(&p->in, cudaStreamNonBlocking)) != cudaSuccess) return nullptr;
+  if ((*err = cudaStreamCreateWithFlags(&p->out, cudaStreamNonBlocking)) != cudaSuccess) return nullptr;
+  if ((*err = cudaEventCreateWithFlags(&p->start, cudaEventDisableTiming)) != cudaSuccess) return nullptr;
+  for (int i = 0; i < kMaxChunks; ++i)
+    if ((*err = cudaEventCreateWithFlags(&p->done[i], cudaEventDisableTiming)) != cudaSuccess) return nullptr;
+  p->ready = true;
+  return p;
+}
+
+// Rows per chunk (a multiple of 128) and the number of chunks; 1 chunk = do not pipeline.
+int plan_chunks(int64_t rows, size_t float_bytes, int64_t* rows_per_chunk) {
+  int n = (int)(float_bytes / kMinChunkBytes);
+  if (n > kMaxChunks) n = kMaxChunks;
+  if (n < 2 || rows < 256) { *rows_per_chunk = rows; return 1; }
+  int64_t rpc = (rows + n - 1) / n;
+  rpc = (rpc + 127) / 128 * 128;
+  *rows_per_chunk = rpc;
+  return (int)((rows + rpc - 1) / rpc);
+}
+
+// Byte offset of the scales of row r0 (a multiple of 128) in either layout.
+size_t scales_row_offset(int64_t r0, int64_t kblocks, int layout) {
+  return layout == MX_SCALES_LINEAR ? (size_t)r0 * (size_t)kblocks
+                                    : (size_t)(r0 / 128) * (size_t)((kblocks + 3) / 4) * 512;
+}
+
+int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                       const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
+                       const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes,
+                       bool may_pipeline) {
   Opts o;
   View v;
   if (!shape) return MX_ERR_NULL;
@@ -248,13 +300,53 @@ int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_
   if ((uintptr_t)workspace_dev % 256) return MX_ERR_ALIGN;
   if (workspace_bytes < mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts))
     return MX_ERR_WORKSPACE;
-  const size_t in_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
+  const size_t esz = o.dtype == MX_BF16 ? 2 : 4;
+  const size_t in_b = (size_t)v.numel * esz;
   const size_t el_b = (size_t)v.numel / 8 * fmt_bits((int)fmt);
   const size_t sc_b = scales_bytes(v.rows, v.kblocks, o.layout);
   char* d_in = (char*)workspace_dev;
   char* d_el = d_in + align_up(in_b, 256);
   char* d_sc = d_el + align_up(el_b, 256);
-  cudaError_t e = cudaMemcpyAsync(d_in, in_host, in_b, cudaMemcpyHostToDevice, o.stream);
+  cudaError_t e;
+  int64_t rpc = v.rows;
+  const int chunks = (may_pipeline && axis == ndim - 1) ? plan_chunks(v.rows, in_b, &rpc) : 1;
+  if (chunks > 1) {
+    HostPipe* hp = host_pipe(&e);
+    if (!hp) return fail_cuda(e);
+    // work queued on the caller's stream comes first
+    if ((e = cudaEventRecord(hp->start, o.stream)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
+      return fail_cuda(e);
+    mx_opts_t co = {o.dtype, o.layout, hp->in, 0};
+    const size_t row_in = (size_t)v.L * esz, row_el = (size_t)v.L / 8 * fmt_bits((int)fmt);
+    for (int c = 0; c < chunks; ++c) {
+      const int64_t r0 = c * rpc, nr = (r0 + rpc <= v.rows ? rpc : v.rows - r0);
+      const size_t so = scales_row_offset(r0, v.kblocks, o.layout);
+      const size_t sb = scales_bytes(nr, v.kblocks, o.layout);
+      if ((e = cudaMemcpyAsync(d_in + r0 * row_in, (const char*)in_host + r0 * row_in, nr * row_in,
+                               cudaMemcpyHostToDevice, hp->in)) != cudaSuccess)
+        return fail_cuda(e);
+      const int64_t cshape[2] = {nr, v.L};
+      const int rc = mx_quantize(d_in + r0 * row_in, d_el + r0 * row_el, (uint8_t*)d_sc + so, cshape, 2, 1, fmt,
+                                 rounding, &co);
+      if (rc != MX_OK) return rc;
+      if ((e = cudaEventRecord(hp->done[c], hp->in)) != cudaSuccess ||
+          (e = cudaStreamWaitEvent(hp->out, hp->done[c], 0)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)elems_out_host + r0 * row_el, d_el + r0 * row_el, nr * row_el,
+                               cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
+        return fail_cuda(e);
+      (void)sb;
+    }
+    // the scale tensor is small: one copy after the last chunk
+    if ((e = cudaMemcpyAsync(scales_out_host, d_sc, sc_b, cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
+      return fail_cuda(e);
+    if ((e = cudaStreamSynchronize(hp->out)) != cudaSuccess || (e = cudaStreamSynchronize(hp->in)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(o.stream)) != cudaSuccess)
+      return fail_cuda(e);
+    return MX_OK;
+  }
+  e = cudaMemcpyAsync(d_in, in_host, in_b, cudaMemcpyHostToDevice, o.stream);
   if (e != cudaSuccess) return fail_cuda(e);
   const int rc = mx_quantize(d_in, d_el, (uint8_t*)d_sc, shape, ndim, axis, fmt, rounding, opts);
   if (rc != MX_OK) return rc;
@@ -264,6 +356,17 @@ int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_
   if (e != cudaSuccess) return fail_cuda(e);
   e = cudaStreamSynchronize(o.stream);
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+}  // namespace
+
+extern "C" {
+
+int mx_quantize_host(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                     const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
+                     const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  return quantize_host_impl(in_host, elems_out_host, scales_out_host, shape, ndim, axis, fmt, rounding, opts,
+                            workspace_dev, workspace_bytes, true);
 }
 
 // ---------------------------------------------------------------------------
@@ -312,8 +415,8 @@ int mx_quantize_host_static(const void* in_host, void* elems_out_host, uint8_t* 
   if (!scratch) return fail_cuda(e);
   // mx_quantize_host copies the input in, zeroes the scale padding where there is any, runs
   // the kernel and copies exactly the produced bytes out: nothing stale is ever read back.
-  return mx_quantize_host(in_host, elems_out_host, scales_out_host, shape, ndim, axis, fmt, rounding,
-                          opts, scratch, MX_STATIC_SCRATCH_BYTES);
+  return quantize_host_impl(in_host, elems_out_host, scales_out_host, shape, ndim, axis, fmt, rounding, opts,
+                            scratch, MX_STATIC_SCRATCH_BYTES, false);  // one stream, nothing created
 }
 
 size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
@@ -341,7 +444,44 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
   char* d_out = (char*)workspace_dev;
   char* d_el = d_out + align_up(out_b, 256);
   char* d_sc = d_el + align_up(el_b, 256);
-  cudaError_t e = cudaMemcpyAsync(d_el, elems_host, el_b, cudaMemcpyHostToDevice, o.stream);
+  cudaError_t e;
+  int64_t rpc = v.rows;
+  const int chunks = plan_chunks(v.rows, out_b, &rpc);
+  if (chunks > 1) {  // row chunks over two streams, as in quantize_host_impl
+    HostPipe* hp = host_pipe(&e);
+    if (!hp) return fail_cuda(e);
+    if ((e = cudaEventRecord(hp->start, o.stream)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->in, hp->start, 0)) != cudaSuccess ||
+        (e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
+      return fail_cuda(e);
+    mx_opts_t co = {o.dtype, o.layout, hp->in, 0};
+    const size_t row_out = (size_t)v.L * (o.dtype == MX_BF16 ? 2 : 4), row_el = (size_t)v.L / 8 * fmt_bits((int)fmt);
+    for (int c = 0; c < chunks; ++c) {
+      const int64_t r0 = c * rpc, nr = (r0 + rpc <= v.rows ? rpc : v.rows - r0);
+      const size_t so = scales_row_offset(r0, v.kblocks, o.layout);
+      const size_t sb = scales_bytes(nr, v.kblocks, o.layout);
+      if (c == 0 && (e = cudaMemcpyAsync(d_sc, scales_host, sc_b, cudaMemcpyHostToDevice, hp->in)) != cudaSuccess)
+        return fail_cuda(e);  // the whole (small) scale tensor goes first
+      (void)sb;
+      if ((e = cudaMemcpyAsync(d_el + r0 * row_el, (const char*)elems_host + r0 * row_el, nr * row_el,
+                               cudaMemcpyHostToDevice, hp->in)) != cudaSuccess)
+        return fail_cuda(e);
+      const int64_t cshape[2] = {nr, v.L};
+      const int rc = mx_dequantize(d_el + r0 * row_el, (const uint8_t*)d_sc + so, d_out + r0 * row_out, cshape, 2, 1,
+                                   fmt, &co);
+      if (rc != MX_OK) return rc;
+      if ((e = cudaEventRecord(hp->done[c], hp->in)) != cudaSuccess ||
+          (e = cudaStreamWaitEvent(hp->out, hp->done[c], 0)) != cudaSuccess ||
+          (e = cudaMemcpyAsync((char*)out_host + r0 * row_out, d_out + r0 * row_out, nr * row_out,
+                               cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
+        return fail_cuda(e);
+    }
+    if ((e = cudaStreamSynchronize(hp->out)) != cudaSuccess || (e = cudaStreamSynchronize(hp->in)) != cudaSuccess ||
+        (e = cudaStreamSynchronize(o.stream)) != cudaSuccess)
+      return fail_cuda(e);
+    return MX_OK;
+  }
+  e = cudaMemcpyAsync(d_el, elems_host, el_b, cudaMemcpyHostToDevice, o.stream);
   if (e != cudaSuccess) return fail_cuda(e);
   e = cudaMemcpyAsync(d_sc, scales_host, sc_b, cudaMemcpyHostToDevice, o.stream);
   if (e != cudaSuccess) return fail_cuda(e);

@@ -220,6 +220,39 @@ def test_host_buffer_entry_points():
         assert ei.value.status == mx.MX_ERR_WORKSPACE
 
 
+@pytest.mark.parametrize("rows,cols,dtype,fmt,layout", [
+    (2048, 4096, torch.bfloat16, 0, 1),     # eight chunks of 256 rows
+    (1000, 4064, torch.float32, 2, 1),      # ragged: last chunk of 104 rows, 127 blocks per row (padded chunks)
+    (1000, 4064, torch.float32, 4, 0),      # the same with linear scales
+    (700, 8192, torch.bfloat16, 5, 1),
+])
+def test_host_buffer_entry_points_pipelined(rows, cols, dtype, fmt, layout):
+    """Sizes at which the host-buffer calls cut the tensor into row chunks and overlap the copies
+    of neighbouring chunks on two internal streams: every output byte against the oracle, guard
+    bytes around the pinned outputs intact."""
+    x = inputs.adversarial("cpu", rows=rows, cols=cols, dtype=dtype, seed=rows + fmt).pin_memory()
+    shape = [rows, cols]
+    G = 4096
+    eb, sb = mx.mx_elems_bytes(shape, 1, fmt), mx.mx_scales_bytes(shape, 1, layout)
+    e_raw = torch.full((eb + 2 * G,), 0xA5, dtype=torch.uint8).pin_memory()
+    s_raw = torch.full((sb + 2 * G,), 0xA5, dtype=torch.uint8).pin_memory()
+    elems, scales = e_raw[G:G + eb], s_raw[G:G + sb]
+    ws = torch.empty(mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, dtype, layout), dtype=torch.uint8, device="cuda")
+    mx.mx_quantize_host(x, elems, scales, 1, fmt, mx.MX_RHAZ, ws, layout)
+    we, ws_ = O.quantize(to_oracle_input(x), 1, fmt, O.RHAZ, layout)
+    assert (elems.numpy() == we).all() and (scales.numpy() == ws_).all()
+    for raw, n in ((e_raw, eb), (s_raw, sb)):
+        assert bool((raw[:G] == 0xA5).all()) and bool((raw[G + n:] == 0xA5).all())
+    o_raw = torch.full((rows * cols * x.element_size() + 2 * G,), 0xA5, dtype=torch.uint8).pin_memory()
+    out = o_raw[G:G + rows * cols * x.element_size()].view(dtype).view(rows, cols)
+    ws2 = torch.empty(mx.mx_dequantize_host_workspace_bytes(shape, fmt, dtype, layout), dtype=torch.uint8, device="cuda")
+    mx.mx_dequantize_host(elems, scales, out, fmt, ws2, layout)
+    want = O.dequantize(we, ws_, rows, cols, fmt, O.BF16 if dtype == torch.bfloat16 else O.F32, layout)
+    got = out.view(torch.int16).numpy().view(np.uint16) if dtype == torch.bfloat16 else out.numpy()
+    assert np.array_equal(got.view(np.uint8), want.view(np.uint8))
+    assert bool((o_raw[:G] == 0xA5).all()) and bool((o_raw[-G:] == 0xA5).all())
+
+
 @pytest.mark.parametrize("fmt", FMTS)
 def test_config2_full_size_sweep(fmt):
     """The 8192 x 8192 BF16 sweep tensor in the launch configuration the benchmark
