@@ -605,3 +605,28 @@ def test_host_buffer_gemm():
     mx.mx_gemm_host(ea.cpu().pin_memory(), sa.cpu().pin_memory(), eb.cpu().pin_memory(),
                     sb.cpu().pin_memory(), hC, M, N, K, mx.MX_E4M3, mx.MX_E2M1, ws)
     assert torch.equal(hC, ref.cpu())
+
+
+def test_output_beyond_4gib():
+    """C = 36864 x 36864 FP32 (5.4 GB): output offsets pass 2^32.  Samples from the last rows and
+    columns against the oracle; the guard bytes behind the output stay intact."""
+    M = N = 36864
+    K = 128
+    g = torch.Generator(device="cuda").manual_seed(11)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    ea, sa = mx.mx_quantize(A, 1, 0)
+    eb, sb = mx.mx_quantize(B, 1, 1)
+    g_out = Guarded(M * N * 4)
+    C = g_out.view.view(torch.float32).view(M, N)
+    mx.mx_gemm(ea, sa, eb, sb, M, N, K, 0, 1, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    rng = np.random.default_rng(3)
+    ms = np.concatenate([rng.integers(0, M, 1500), rng.integers(M - 300, M, 1500), [M - 1, M - 1, 0]])
+    ns = np.concatenate([rng.integers(0, N, 1500), rng.integers(N - 300, N, 1500), [N - 1, 0, N - 1]])
+    c64, s = O.gemm_samples(*(t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb)), M, N, K, 0, 1, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= TOL * s).all()
+    # every element was written: an untouched output would keep the fill value
+    assert not bool((C.view(torch.int32) == -1515870811).any())     # 0xA5A5A5A5

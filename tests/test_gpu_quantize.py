@@ -290,3 +290,36 @@ def test_config2_full_size_sweep(fmt):
         sb = s.cpu().numpy()
         assert 0.0005 < (sb == 0).mean() < 0.002
         assert 0.0005 < ((sb > 0) & (sb < 40)).mean() < 0.002
+
+
+def test_offsets_beyond_4gib():
+    """A 6.4 GB BF16 tensor (49152 x 65536): byte offsets of input, codes and outputs pass 2^32.
+    Sampled rows from both ends and the middle against the oracle, last axis and strided axis,
+    and the dequantized tensor."""
+    rows, cols = 49152, 65536
+    g = torch.Generator(device="cuda").manual_seed(99)
+    x = torch.empty((rows, cols), dtype=torch.bfloat16, device="cuda")
+    for r0 in range(0, rows, 8192):   # filled in slabs: no FP32 copy of the whole tensor
+        x[r0:r0 + 8192] = (torch.randn((8192, cols), generator=g, device="cuda") *
+                           torch.exp(torch.randn((8192, 1), generator=g, device="cuda"))).to(torch.bfloat16)
+    sel = np.array([0, 1, 127, 128, 20000, 32767, 32768, 32769, 40001, rows - 129, rows - 2, rows - 1])
+    sel_t = torch.from_numpy(sel).cuda()
+    xin = to_oracle_input(x[sel_t].contiguous())
+    for fmt in (mx.MX_E4M3, mx.MX_E3M2):
+        w = O.fmt_bits(fmt)
+        e, s = mx.mx_quantize(x, 1, fmt, mx.MX_RNE, mx.MX_SCALES_LINEAR)
+        we, ws = O.quantize(xin, 1, fmt, O.RNE, O.LINEAR)
+        assert np.array_equal(e.view(rows, cols * w // 8)[sel_t].cpu().numpy().reshape(-1), we)
+        assert np.array_equal(s.view(rows, cols // 32)[sel_t].cpu().numpy().reshape(-1), ws)
+        d = mx.mx_dequantize(e, s, [rows, cols], fmt, torch.bfloat16, mx.MX_SCALES_LINEAR)
+        want = O.dequantize(we, ws, len(sel), cols, fmt, O.BF16, O.LINEAR)
+        assert np.array_equal(d[sel_t].view(torch.int16).cpu().numpy().view(np.uint16), want)
+        del e, s, d
+    # blocks along axis 0: output row = input column; columns from both ends
+    csel = np.array([0, 3, 4, 31, 32768, cols - 5, cols - 1])
+    csel_t = torch.from_numpy(csel).cuda()
+    e, s = mx.mx_quantize(x, 0, mx.MX_E4M3, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
+    xt = to_oracle_input(x[:, csel_t].t().contiguous())           # [columns, rows]: blocks along the last axis
+    we, ws = O.quantize(xt, 1, mx.MX_E4M3, O.RHAZ, O.LINEAR)
+    assert np.array_equal(e.view(cols, rows)[csel_t].cpu().numpy().reshape(-1), we)
+    assert np.array_equal(s.view(cols, rows // 32)[csel_t].cpu().numpy().reshape(-1), ws)
