@@ -534,13 +534,36 @@ def main_case(args):
         C = torch.empty((n, n), dtype=torch.float32, device="cuda")
         for _ in range(reps):
             mx.mx_gemm(ea, sa, eb, sb, n, n, n, fmt, fmt, out=C, check_status=True)
+    elif args.case == "gemm_dense":   # MXINT8 x MXINT8 through BF16: two dequantize launches + the dense GEMM
+        n = 4096
+        d = inputs.config4("cuda", n)
+        ea, sa = mx.mx_quantize(d["X"], 1, mx.MX_INT8)
+        eb, sb = mx.mx_quantize(d["W"], 0, mx.MX_INT8)
+        C = torch.empty((n, n), dtype=torch.float32, device="cuda")
+        ws = torch.empty(mx.mx_gemm_dense_workspace_bytes(n, n, n), dtype=torch.uint8, device="cuda")
+        for _ in range(reps):
+            mx.mx_gemm_dense(ea, sa, eb, sb, n, n, n, mx.MX_INT8, mx.MX_INT8, workspace=ws, out=C, check_status=True)
+    elif args.case == "quantize_dual":
+        T = inputs.config2("cuda", SWEEP_ROWS, SWEEP_COLS)
+        fmt = mx.FORMATS[args.fmt]
+        out = mx.mx_quantize_dual(T, fmt)
+        for _ in range(reps):
+            mx.mx_quantize_dual(T, fmt, out=out)
+    elif args.case == "im2col":       # N 32, 56 x 56, C 256, 3 x 3, padding 1: 231 MB of E4M3 codes out
+        x = torch.randn((32, 56, 56, 256), device="cuda", dtype=torch.bfloat16)
+        fmt = mx.FORMATS[args.fmt]
+        conv = mx.mx_conv_geometry(32, 56, 56, 256, 3, 3, (1, 1), (1, 1), (1, 1))
+        ex, sx = mx.mx_quantize(x, 3, fmt)
+        for _ in range(reps):
+            mx.mx_im2col(ex, sx, conv, fmt)
     torch.cuda.synchronize()
     print(json.dumps({"case": args.case, "fmt": args.fmt, "launches": reps}))
 
 
 def main():
     ap = argparse.ArgumentParser()
-    ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm"],
+    ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm", "gemm_dense",
+                                       "quantize_dual", "im2col"],
                     default="step", help="'step' = the benchmark; the others run three launches of one "
                                          "kernel on a small case for a profiler capture")
     ap.add_argument("--fmt", choices=FMT_NAMES, default="e4m3")
