@@ -12,10 +12,11 @@
 //   warp 0    TMA producer: packed A / B tiles (the sub-byte tensor-map types
 //             expand FP6 / FP4 to one byte per element on the way in) and the
 //             512-byte swizzled scale chunks -> shared-memory ring
-//   warp 1    MMA issuer: scales shared -> tensor memory (tcgen05.cp), four
-//             MMAs per stage, tcgen05.commit releases the stage / the accumulator
+//   warp 1    MMA issuer: four MMAs per stage, tcgen05.commit releases the stage /
+//             publishes the accumulator
 //   warps 2-9 epilogue: tensor memory -> registers (the accumulator is released as soon as
-//             it is in registers) -> FP32 C, overlapping the next tile's MMAs
+//             it is in registers) -> FP32 or BF16 C through shared memory and TMA stores, or the
+//             quantizing epilogue (C as an MX tensor), overlapping the next tile's MMAs
 //   warp 10   scale copier: a stage's scale chunks shared -> tensor memory (tcgen05.cp), then
 //             tcgen05.commit tells the MMA issuer.  Every tcgen05 instruction costs its issuing
 //             thread 60-70 clocks; with the three copies of a stage in the MMA thread's stream

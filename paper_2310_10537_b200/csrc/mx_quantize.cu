@@ -1,14 +1,15 @@
 // Float -> MX conversion kernels (Algorithm 1, Section 3 of arXiv 2310.10537).
 //
-//   quantize_lastaxis_kernel  blocks run along the contiguous axis: a pure
-//                             stream, 8 elements per thread, 4 lanes per block.
-//   quantize_strided_kernel   blocks run along a strided axis (the transposed
-//                             operands of dgrad / wgrad, Section 4.1): each
-//                             thread owns whole blocks of a few columns, reads
-//                             rows coalesced across the warp and writes the
-//                             result with the block axis innermost.
+//   quantize_lastaxis_kernel        blocks run along the contiguous axis: a pure stream, 64 bytes
+//                                   of input per thread (a whole BF16 block, half an FP32 block).
+//   quantize_strided_kernel         blocks run along a strided axis (the transposed operands of
+//                                   dgrad / wgrad, Section 4.1): a thread owns whole blocks of a
+//                                   few adjacent columns, rows are read coalesced across the warp
+//                                   and the result is written with the block axis innermost.
+//   quantize_strided_staged_kernel  the same for 6- and 4-bit codes, whose output runs are gathered
+//                                   in shared memory so that they leave as whole 32-byte sectors.
 //
-// Both are bound by HBM bandwidth: in_bytes + bits/8 + 1/32 bytes per element.
+// All are bound by HBM bandwidth: in_bytes + bits/8 + 1/32 bytes per element.
 #include "mx_device.cuh"
 #include "mx_launch.h"
 #include "mx_quantize_common.cuh"
@@ -297,9 +298,9 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
 // Staged variant of the same kernel for the common case (kblocks % 4 == 0, output rows 16-byte
 // aligned): a thread still owns COLS columns, but it walks four consecutive blocks, parks their
 // codes in shared memory, and the warp then writes every output row's 128 / 96 / 64-byte run with
-// coalesced 16-byte stores.  Without this each lane writes its own row and the L2 sees two (8-bit),
-// three (6-bit) or one (4-bit) partial-sector request per block and row, which is what bounded the
-// direct version.  Each warp has a private staging area, so only __syncwarp is needed.
+// coalesced 32-byte (else 16-byte) stores.  Without this each lane writes its own row and the L2
+// sees three (6-bit) or one (4-bit) partial-sector request per block and row, which is what
+// bounded the direct version.  Each warp has a private staging area, so only __syncwarp is needed.
 constexpr int kStagedThreads = 64;  // resident CTAs per SM below: the measured optimum per variant
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int COLS>
