@@ -185,6 +185,8 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void*
   a.R = R; a.C = C; a.fmt = (int)fmt; a.rounding = (int)rounding; a.dtype = o.dtype; a.layout = o.layout;
   a.stream = o.stream;
   cudaError_t e;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
   // swizzled scale tensors have padding when kblocks % 4 != 0 (rows are multiples of 128 here)
   if (o.layout == MX_SCALES_SWIZZLED && (C / 32) % 4 != 0) {
     e = cudaMemsetAsync(scales_row, 0, scales_bytes(R, C / 32, o.layout), o.stream);

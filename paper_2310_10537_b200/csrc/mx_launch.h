@@ -26,6 +26,7 @@ struct DualArgs {
   uint8_t *elems_col, *scales_col;  // blocks along axis 0: [C x R]
   int64_t R, C;
   int fmt, rounding, dtype, layout;
+  int sm_count;
   cudaStream_t stream;
 };
 cudaError_t launch_quantize_dual(const DualArgs& a);

@@ -41,7 +41,7 @@ template <int FMT, int ROUND, int DTYPE, int LAYOUT>
 __global__ void __launch_bounds__(kDualThreads, DTYPE == MX_BF16 ? 4 : 6)
 quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_row,
                      uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
-                     uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C) {
+                     uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_per_warp) {
   using cfg = DualCfg<FMT, DTYPE>;
   constexpr int bits = cfg::bits;
   constexpr int COLS = cfg::COLS;
@@ -61,7 +61,10 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   const size_t in_pitch = (size_t)C * esz;
   const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;          // blocks per output row
   const size_t row_out_bytes = (size_t)C * bits / 8, col_out_bytes = (size_t)R * bits / 8;
-  const uint32_t tile0 = blockIdx.y * 4;                             // first 32-row tile of this CTA
+  // 32-row tiles this warp walks: four (the staged 6- and 4-bit column codes need four), or fewer
+  // for 8-bit codes when that fills the machine more evenly
+  const uint32_t T = bits == 8 ? tiles_per_warp : 4u;
+  const uint32_t tile0 = blockIdx.y * T;                             // first 32-row tile of this CTA
 
   uint32_t col_scale_word[COLS];
 #pragma unroll
@@ -81,7 +84,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   load_tile(tile0);
 
 #pragma unroll 1
-  for (uint32_t j = 0; j < 4; ++j) {
+  for (uint32_t j = 0; j < T; ++j) {
     const uint32_t tile = tile0 + j;
     // transpose area first, so the shared-memory latency hides behind the column arithmetic
 #pragma unroll
@@ -115,7 +118,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
       }
     }
     __syncwarp();
-    if (j < 3) load_tile(tile + 1);
+    if (j + 1 < T) load_tile(tile + 1);
 
     // ---- row blocks: lane r owns row (tile * 32 + r) of the strip: kRowBlocks blocks of 32 columns
     {
@@ -186,7 +189,12 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   // ---- column outputs of the four tiles
 #pragma unroll
   for (int c = 0; c < COLS; ++c)
-    *reinterpret_cast<uint32_t*>(scales_col + scale_offset<LAYOUT>(col0 + c, tile0, kb_col)) = col_scale_word[c];
+  {
+    uint8_t* sp = scales_col + scale_offset<LAYOUT>(col0 + c, tile0, kb_col);  // T adjacent bytes, T-aligned
+    if (T == 4) *reinterpret_cast<uint32_t*>(sp) = col_scale_word[c];
+    else if (T == 2) *reinterpret_cast<uint16_t*>(sp) = (uint16_t)col_scale_word[c];
+    else *sp = (uint8_t)col_scale_word[c];
+  }
   if (bits != 8) {
     __syncwarp();
     if (((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0) {
@@ -225,10 +233,24 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
   using cfg = DualCfg<FMT, DTYPE>;
   static_assert(cfg::kSmem <= 48 * 1024, "fits the default shared-memory limit");
   const uint32_t strips = (uint32_t)(a.C / (32 * cfg::COLS));
-  dim3 grid((strips + kDualThreads / 32 - 1) / (kDualThreads / 32), (uint32_t)(a.R / 128));
+  const uint32_t ctas_x = (strips + kDualThreads / 32 - 1) / (kDualThreads / 32);
+  // Tiles per warp (8-bit codes): the choice that needs the least time in units of one tile, given
+  // how many warps are resident at once -- e.g. 4096 x 4096 FP32 is 1.15 waves of four-tile warps
+  // (two rounds) but 4.6 waves of one-tile warps (five rounds of a quarter the length).
+  uint32_t T = 4;
+  if (cfg::bits == 8) {
+    const uint64_t slots = (uint64_t)a.sm_count * (DTYPE == MX_BF16 ? 4 : 6);  // resident CTAs
+    uint64_t best = ~0ull;
+    for (uint32_t t : {4u, 2u, 1u}) {
+      const uint64_t ctas = (uint64_t)ctas_x * (uint64_t)(a.R / 32 / t);
+      const uint64_t cost = (ctas + slots - 1) / slots * t;
+      if (cost < best) { best = cost; T = t; }
+    }
+  }
+  dim3 grid(ctas_x, (uint32_t)(a.R / 32 / T));
   return launch_pdl(quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT>, grid, dim3(kDualThreads), cfg::kSmem,
                     a.stream, a.in, a.elems_row, a.scales_row, a.elems_col, a.scales_col, (uint32_t)a.R,
-                    (uint32_t)a.C);
+                    (uint32_t)a.C, T);
 }
 
 template <int FMT, int ROUND>
