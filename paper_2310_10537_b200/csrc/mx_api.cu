@@ -564,7 +564,7 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
     if (st != 0) {
       std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u gave up "
                     "(1 producer/stage empty, 2 MMA/stage full, 3 MMA/accumulator free, "
-                    "4 epilogue/accumulator full, 5 scale copier/stage full)", st);
+                    "4 epilogue/accumulator full, 5 scale copier/stage full, 6 shared-memory alignment)", st);
       return MX_ERR_TIMEOUT;
     }
   }
@@ -649,7 +649,7 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
     if (st != 0) {
       std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u gave up "
                     "(1 producer/stage empty, 2 MMA/stage full, 3 MMA/accumulator free, "
-                    "4 epilogue/accumulator full, 5 scale copier/stage full)", st);
+                    "4 epilogue/accumulator full, 5 scale copier/stage full, 6 shared-memory alignment)", st);
       return MX_ERR_TIMEOUT;
     }
   }

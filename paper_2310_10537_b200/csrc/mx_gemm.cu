@@ -51,6 +51,7 @@ enum : unsigned int {
   ST_MMA_WAIT_ACC = 3,     // MMA issuer: accumulator never drained
   ST_EPILOGUE_WAIT = 4,    // epilogue: accumulator never became full
   ST_SCALE_WAIT = 5,       // scale copier: stage never became full
+  ST_SMEM_ALIGN = 6,       // shared memory window not aligned as the tight configuration needs
 };
 
 // First failure of any GEMM launch on this device since the last check (0 = none).
@@ -634,7 +635,7 @@ struct Cfg2 {
   static constexpr bool F4 = KIND == 1;
   static constexpr bool DENSE = KIND == 2;
   static constexpr int BN = BN_;
-  static constexpr int kStages = BN == 384 ? 4 : (F4 ? 5 : 6);
+  static constexpr int kStages = BN == 384 ? (F4 ? 4 : 5) : (F4 ? 5 : 6);
   static constexpr int kBKe = F4 ? 256 : DENSE ? 64 : 128;  // K elements per stage (128-byte operand rows)
   static constexpr int kKChunks = F4 ? 2 : 1;           // 512-byte scale chunks (4 MX blocks) along K per stage
   static constexpr int kSfbGroups = BN / 128;           // 128-row scale chunks of B per K chunk
@@ -652,8 +653,11 @@ struct Cfg2 {
   static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
   static constexpr uint32_t kNumBars = 3 * kStages + 2;
-  static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;
-  static_assert(kSmemBytes <= 232448, "shared memory budget");
+  // Bytes used from the 1024-byte aligned base, and the request: up to 1024 bytes of slack for the
+  // alignment, fewer where the budget is tight (the kernel checks that what it got suffices).
+  static constexpr uint32_t kUsedBytes = kOffBar + kNumBars * 8 + 16;
+  static constexpr uint32_t kSmemBytes = kUsedBytes + 1024 <= 232448 ? kUsedBytes + 1024 : 232448;
+  static_assert(kUsedBytes <= 232448, "shared memory budget");
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
 };
 
@@ -736,6 +740,12 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  if (smem_base - smem_u32(smem_raw) + cfg::kUsedBytes > cfg::kSmemBytes) {
+    // the alignment cost more than the request left room for: give up before anything is set up
+    // (uniform over the grid: every CTA sees the same offset)
+    if (threadIdx.x == 0) atomicCAS(&g_gemm_status, 0u, (unsigned int)ST_SMEM_ALIGN);
+    return;
+  }
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
   const uint32_t bar0 = smem_base + cfg::kOffBar;
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
