@@ -192,28 +192,33 @@ def run_e2e(torch, mx, inputs, steps: int, warmup: int):
     rows, cols = T.shape
     shape = [rows, cols]
     n = rows * cols
-    bufs = []
-    ws_bytes = 0
+    bufs, outs, wss = [], [], []
     for fmt in range(6):
         e = torch.empty(mx.mx_elems_bytes(shape, 1, fmt), dtype=torch.uint8).pin_memory()
         s = torch.empty(mx.mx_scales_bytes(shape, 1), dtype=torch.uint8).pin_memory()
         bufs.append((e, s))
-        ws_bytes = max(ws_bytes, mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, torch.bfloat16))
-    out = torch.empty(shape, dtype=torch.bfloat16).pin_memory()
-    ws = torch.empty(ws_bytes, dtype=torch.uint8, device="cuda")
+        outs.append(torch.empty(shape, dtype=torch.bfloat16).pin_memory())
+        wss.append(torch.empty(mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, torch.bfloat16),
+                               dtype=torch.uint8, device="cuda"))
     h2d = d2h = 0
 
     def one():
+        # the six quantizes are queued back to back (the upload of one overlaps the download of the
+        # one before), then waited for; the six dequantizes likewise
         nonlocal h2d, d2h
         h2d = d2h = 0
         for fmt in range(6):
             e, s = bufs[fmt]
-            mx.mx_quantize_host(T, e, s, 1, fmt, mx.MX_RNE, ws)
+            mx.mx_quantize_host(T, e, s, 1, fmt, mx.MX_RNE, wss[fmt], queue=True)
             h2d += T.numel() * 2
             d2h += e.numel() + s.numel()
-            mx.mx_dequantize_host(e, s, out, fmt, ws)
+        mx.mx_host_synchronize()
+        for fmt in range(6):
+            e, s = bufs[fmt]
+            mx.mx_dequantize_host(e, s, outs[fmt], fmt, wss[fmt], queue=True)
             h2d += e.numel() + s.numel()
-            d2h += out.numel() * 2
+            d2h += outs[fmt].numel() * 2
+        mx.mx_host_synchronize()
 
     for _ in range(max(1, warmup)):
         one()
@@ -226,8 +231,8 @@ def run_e2e(torch, mx, inputs, steps: int, warmup: int):
     total_bytes = 2.0 * sum(algorithmic_bytes(n, 2, b) for b in FMT_BITS)
     return {"value": total_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3,
-            "workload": f"sweep on a {rows}x{cols} BF16 slice via mx_quantize_host / mx_dequantize_host "
-                        "(pinned host buffers, copies timed)"}
+            "workload": f"sweep on a {rows}x{cols} BF16 slice via mx_quantize_host_async / "
+                        "mx_dequantize_host_async + mx_host_synchronize (pinned host buffers, copies timed)"}
 
 
 def run_extras(torch, mx, inputs):

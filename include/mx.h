@@ -379,6 +379,26 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
                        mx_fmt_t fmt, const mx_opts_t* opts,
                        void* workspace_dev, size_t workspace_bytes);
 
+/*
+ * Asynchronous forms of the two calls above, for a sequence of conversions whose copies should
+ * overlap ACROSS calls: each returns after queueing its work on the library's internal copy
+ * pipeline; calls execute in the order issued, the upload of one call overlapping the download
+ * of the one before.  Results (and the host input buffers) may be touched again only after
+ * mx_host_synchronize().  Until then every queued call needs its own workspace, and a call must
+ * not read host memory that an earlier, still queued call writes.  Blocks must run along the
+ * last axis (otherwise MX_ERR_UNSUPPORTED); other arguments and errors as the synchronous forms.
+ * mx_host_synchronize waits for everything queued on the current device.
+ */
+int mx_quantize_host_async(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                           const int64_t* shape, int ndim, int axis,
+                           mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts,
+                           void* workspace_dev, size_t workspace_bytes);
+int mx_dequantize_host_async(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                             const int64_t* shape, int ndim, int axis,
+                             mx_fmt_t fmt, const mx_opts_t* opts,
+                             void* workspace_dev, size_t workspace_bytes);
+int mx_host_synchronize(void);
+
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K,
                                     mx_fmt_t fmtA, mx_fmt_t fmtB);
 int mx_gemm_host(const void* A_host, const uint8_t* sA_host,

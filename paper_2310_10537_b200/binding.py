@@ -33,6 +33,7 @@ EXPORTS = [
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
     "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
     "mx_gemm_dense", "mx_conv_out_h", "mx_conv_out_w", "mx_im2col",
+    "mx_quantize_host_async", "mx_dequantize_host_async", "mx_host_synchronize",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
     "mx_gemm_host_workspace_bytes", "mx_gemm_host",
@@ -99,10 +100,13 @@ def _load() -> ctypes.CDLL:
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
     lib.mx_quantize_host.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op, vp, sz]
+    lib.mx_quantize_host_async.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op, vp, sz]
+    lib.mx_host_synchronize.argtypes = []
     lib.mx_quantize_host_static.argtypes = [vp, vp, u8p, i64p, ci, ci, ci, ci, op]
     lib.mx_dequantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_dequantize_host_workspace_bytes.restype = sz
     lib.mx_dequantize_host.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op, vp, sz]
+    lib.mx_dequantize_host_async.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op, vp, sz]
     lib.mx_gemm_host_workspace_bytes.argtypes = [i64, i64, i64, ci, ci]
     lib.mx_gemm_host_workspace_bytes.restype = sz
     lib.mx_gemm_host.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op, vp, sz]
@@ -332,11 +336,14 @@ def mx_quantize_host_workspace_bytes(shape, axis, fmt, dtype, layout=MX_SCALES_S
 
 def mx_quantize_host(x: torch.Tensor, elems: torch.Tensor, scales: torch.Tensor, axis: int,
                      fmt: int, rounding: int, workspace: torch.Tensor,
-                     layout: int = MX_SCALES_SWIZZLED) -> None:
+                     layout: int = MX_SCALES_SWIZZLED, queue: bool = False) -> None:
+    """Host tensors in and out.  ``queue=True`` uses the asynchronous entry point: the call only
+    queues its work (own workspace per queued call) and ``mx_host_synchronize()`` waits for it."""
     assert not x.is_cuda and not elems.is_cuda and not scales.is_cuda and workspace.is_cuda
     shape = list(x.shape)
     o = _opts(_dtype_code(x.dtype), layout)
-    _check(_lib.mx_quantize_host(x.data_ptr(), elems.data_ptr(), scales.data_ptr(),
+    fn = _lib.mx_quantize_host_async if queue else _lib.mx_quantize_host
+    _check(fn(x.data_ptr(), elems.data_ptr(), scales.data_ptr(),
                                  _shape_arr(shape), len(shape), axis % len(shape), fmt, rounding,
                                  ctypes.byref(o), workspace.data_ptr(), workspace.numel()),
            "mx_quantize_host")
@@ -364,12 +371,18 @@ def mx_dequantize_host_workspace_bytes(shape, fmt, dtype, layout=MX_SCALES_SWIZZ
                                                        len(shape) - 1, fmt, ctypes.byref(o)))
 
 
+def mx_host_synchronize() -> None:
+    """Waits for every queued host-buffer call on the current device."""
+    _check(_lib.mx_host_synchronize(), "mx_host_synchronize")
+
+
 def mx_dequantize_host(elems: torch.Tensor, scales: torch.Tensor, out: torch.Tensor, fmt: int,
-                       workspace: torch.Tensor, layout: int = MX_SCALES_SWIZZLED) -> None:
+                       workspace: torch.Tensor, layout: int = MX_SCALES_SWIZZLED, queue: bool = False) -> None:
     assert not elems.is_cuda and not scales.is_cuda and not out.is_cuda and workspace.is_cuda
     shape = list(out.shape)
     o = _opts(_dtype_code(out.dtype), layout)
-    _check(_lib.mx_dequantize_host(elems.data_ptr(), scales.data_ptr(), out.data_ptr(),
+    fn = _lib.mx_dequantize_host_async if queue else _lib.mx_dequantize_host
+    _check(fn(elems.data_ptr(), scales.data_ptr(), out.data_ptr(),
                                    _shape_arr(shape), len(shape), len(shape) - 1, fmt,
                                    ctypes.byref(o), workspace.data_ptr(), workspace.numel()),
            "mx_dequantize_host")

@@ -291,7 +291,7 @@ size_t scales_row_offset(int64_t r0, int64_t kblocks, int layout) {
 int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
                        const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
                        const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes,
-                       bool may_pipeline) {
+                       bool may_pipeline, bool async = false) {
   Opts o;
   View v;
   if (!shape) return MX_ERR_NULL;
@@ -312,7 +312,8 @@ int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scale
   cudaError_t e;
   int64_t rpc = v.rows;
   const int chunks = (may_pipeline && axis == ndim - 1) ? plan_chunks(v.rows, in_b, &rpc) : 1;
-  if (chunks > 1) {
+  if (async && axis != ndim - 1) return MX_ERR_UNSUPPORTED;
+  if (chunks > 1 || async) {
     HostPipe* hp = host_pipe(&e);
     if (!hp) return fail_cuda(e);
     // work queued on the caller's stream comes first
@@ -343,6 +344,7 @@ int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scale
     // the scale tensor is small: one copy after the last chunk
     if ((e = cudaMemcpyAsync(scales_out_host, d_sc, sc_b, cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
       return fail_cuda(e);
+    if (async) return MX_OK;  // mx_host_synchronize() waits for it
     if ((e = cudaStreamSynchronize(hp->out)) != cudaSuccess || (e = cudaStreamSynchronize(hp->in)) != cudaSuccess ||
         (e = cudaStreamSynchronize(o.stream)) != cudaSuccess)
       return fail_cuda(e);
@@ -426,9 +428,9 @@ size_t mx_dequantize_host_workspace_bytes(const int64_t* shape, int ndim, int ax
   return mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts);
 }
 
-int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void* out_host,
-                       const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
-                       const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+static int dequantize_host_impl(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                                const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, const mx_opts_t* opts,
+                                void* workspace_dev, size_t workspace_bytes, bool async) {
   Opts o;
   View v;
   if (!shape) return MX_ERR_NULL;
@@ -449,7 +451,7 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
   cudaError_t e;
   int64_t rpc = v.rows;
   const int chunks = plan_chunks(v.rows, out_b, &rpc);
-  if (chunks > 1) {  // row chunks over two streams, as in quantize_host_impl
+  if (chunks > 1 || async) {  // row chunks over two streams, as in quantize_host_impl
     HostPipe* hp = host_pipe(&e);
     if (!hp) return fail_cuda(e);
     if ((e = cudaEventRecord(hp->start, o.stream)) != cudaSuccess ||
@@ -478,6 +480,7 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
                                cudaMemcpyDeviceToHost, hp->out)) != cudaSuccess)
         return fail_cuda(e);
     }
+    if (async) return MX_OK;
     if ((e = cudaStreamSynchronize(hp->out)) != cudaSuccess || (e = cudaStreamSynchronize(hp->in)) != cudaSuccess ||
         (e = cudaStreamSynchronize(o.stream)) != cudaSuccess)
       return fail_cuda(e);
@@ -493,6 +496,36 @@ int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void*
   if (e != cudaSuccess) return fail_cuda(e);
   e = cudaStreamSynchronize(o.stream);
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
+}
+
+int mx_dequantize_host(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                       const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                       const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  return dequantize_host_impl(elems_host, scales_host, out_host, shape, ndim, axis, fmt, opts, workspace_dev,
+                              workspace_bytes, false);
+}
+
+int mx_quantize_host_async(const void* in_host, void* elems_out_host, uint8_t* scales_out_host,
+                           const int64_t* shape, int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding,
+                           const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  return quantize_host_impl(in_host, elems_out_host, scales_out_host, shape, ndim, axis, fmt, rounding, opts,
+                            workspace_dev, workspace_bytes, true, true);
+}
+
+int mx_dequantize_host_async(const void* elems_host, const uint8_t* scales_host, void* out_host,
+                             const int64_t* shape, int ndim, int axis, mx_fmt_t fmt,
+                             const mx_opts_t* opts, void* workspace_dev, size_t workspace_bytes) {
+  return dequantize_host_impl(elems_host, scales_host, out_host, shape, ndim, axis, fmt, opts, workspace_dev,
+                              workspace_bytes, true);
+}
+
+int mx_host_synchronize(void) {
+  cudaError_t e;
+  HostPipe* hp = host_pipe(&e);
+  if (!hp) return fail_cuda(e);
+  if ((e = cudaStreamSynchronize(hp->in)) != cudaSuccess || (e = cudaStreamSynchronize(hp->out)) != cudaSuccess)
+    return fail_cuda(e);
+  return MX_OK;
 }
 
 // ---------------------------------------------------------------------------

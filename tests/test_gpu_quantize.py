@@ -323,3 +323,33 @@ def test_offsets_beyond_4gib():
     we, ws = O.quantize(xt, 1, mx.MX_E4M3, O.RHAZ, O.LINEAR)
     assert np.array_equal(e.view(cols, rows)[csel_t].cpu().numpy().reshape(-1), we)
     assert np.array_equal(s.view(cols, rows // 32)[csel_t].cpu().numpy().reshape(-1), ws)
+
+
+def test_queued_host_calls():
+    """Six quantizes queued back to back (own outputs and workspaces), one synchronize, then six
+    queued dequantizes: every byte against the oracle.  Sizes on both sides of the chunking limit."""
+    for rows, cols in ((2048, 4096), (96, 512)):
+        x = inputs.adversarial("cpu", rows=rows, cols=cols, dtype=torch.bfloat16, seed=rows).pin_memory()
+        shape = [rows, cols]
+        outs, wss = [], []
+        for fmt in FMTS:
+            e = torch.full((mx.mx_elems_bytes(shape, 1, fmt),), 0xA5, dtype=torch.uint8).pin_memory()
+            s = torch.full((mx.mx_scales_bytes(shape, 1),), 0xA5, dtype=torch.uint8).pin_memory()
+            ws = torch.empty(mx.mx_quantize_host_workspace_bytes(shape, 1, fmt, torch.bfloat16), dtype=torch.uint8, device="cuda")
+            outs.append((e, s))
+            wss.append(ws)
+            mx.mx_quantize_host(x, e, s, 1, fmt, mx.MX_RNE, ws, queue=True)
+        mx.mx_host_synchronize()
+        want = []
+        for fmt, (e, s) in zip(FMTS, outs):
+            we, ws_ = O.quantize(to_oracle_input(x), 1, fmt, O.RNE, O.SWIZZLED)
+            assert (e.numpy() == we).all() and (s.numpy() == ws_).all(), fmt
+            want.append(O.dequantize(we, ws_, rows, cols, fmt, O.BF16, O.SWIZZLED))
+        backs = []
+        for fmt, (e, s), ws in zip(FMTS, outs, wss):
+            out = torch.zeros(shape, dtype=torch.bfloat16).pin_memory()
+            backs.append(out)
+            mx.mx_dequantize_host(e, s, out, fmt, ws, queue=True)
+        mx.mx_host_synchronize()
+        for fmt, out, w in zip(FMTS, backs, want):
+            assert (out.view(torch.int16).numpy().view(np.uint16) == w).all(), fmt
