@@ -112,3 +112,22 @@ def test_gemm_variants_argument_validation_without_gpu():
     assert gd(p, p, p, p, p, 3, 128, 128, 128, 5, 5, None, p, 1 << 20) == mx.MX_ERR_FMT
     assert gd(p, p, p, p, p, F32, 128, 128, 128, 6, 5, None, p, 1 << 20) == mx.MX_ERR_FMT
     assert gd(p, p, p, p, p, F32, 0, 128, 128, 5, 5, None, None, 0) == mx.MX_OK                # nothing to do
+
+
+def test_header_is_plain_c(tmp_path):
+    """include/mx.h compiles as C99 on its own (the boundary is a C ABI: no C++ in the signatures)
+    and a C program can link against the library and call a host-only helper."""
+    import shutil
+    import subprocess
+    if shutil.which("gcc") is None:
+        import pytest
+        pytest.skip("no C compiler")
+    src = tmp_path / "t.c"
+    src.write_text('#include "mx.h"\n'
+                   'int main(void) { mx_conv_t c; mx_opts_t o; (void)c; (void)o;\n'
+                   '  return mx_fmt_bits(MX_E2M3) == 6 && mx_scale_offset(33, 5, 128, 8, MX_SCALES_SWIZZLED) == 512 + 16 + 4 + 1 ? 0 : 1; }\n')
+    exe = tmp_path / "t"
+    libdir = os.path.dirname(mx.LIB_PATH)
+    subprocess.check_call(["gcc", "-std=c99", "-Wall", "-Wextra", "-pedantic", "-Werror", "-I", os.path.join(ROOT, "include"),
+                           str(src), "-o", str(exe), "-L", libdir, "-lmx_b200", "-Wl,-rpath," + libdir])
+    assert subprocess.call([str(exe)]) == 0
