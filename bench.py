@@ -336,6 +336,158 @@ def run_extras(torch, mx, inputs):
     return out
 
 
+def run_report(torch, mx, inputs):
+    """The per-kernel measurement protocol, as markdown on stdout (kept in BENCH.md): every kernel of
+    every benchmark configuration, 10 warm-up launches, then 50 launches each timed with its own pair
+    of CUDA events (median and best) and the same 50 launches timed as one back-to-back run, rotating
+    over buffer sets larger than twice the L2; the GEMMs also as a two-second sustained loop; the
+    oracle's GEMM on a slab of configuration 3 on the host cores."""
+    import numpy as np
+
+    import oracle as O
+    peaks = measured_peaks()
+    hbm, hbm_nom = peaks["hbm_gbs"], 8000.0
+    fp8_burst, fp8_sust, fp8_nom = 2 * peaks["bf16_tflops"], 2 * peaks["bf16_tflops_sustained"], 4500.0
+    lines = []
+
+    def protocol(fn_of_i, n_sets, reps=50, warm=10):
+        for i in range(warm):
+            fn_of_i(i % n_sets)
+        torch.cuda.synchronize()
+        ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(reps)]
+        for i, (a, b) in enumerate(ev):
+            a.record()
+            fn_of_i(i % n_sets)
+            b.record()
+        torch.cuda.synchronize()
+        each = sorted(a.elapsed_time(b) * 1e-3 for a, b in ev)
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        for i in range(reps):
+            fn_of_i(i % n_sets)
+        b.record()
+        torch.cuda.synchronize()
+        return each[len(each) // 2], each[0], a.elapsed_time(b) * 1e-3 / reps
+
+    def stream_row(name, byts, times):
+        med, best, b2b = times
+        lines.append(f"| {name} | {byts / 1e6:.1f} | {med * 1e6:.1f} | {best * 1e6:.1f} | {b2b * 1e6:.1f} | "
+                     f"{byts / b2b / 1e9:.0f} | {100 * byts / b2b / 1e9 / hbm:.1f} | {100 * byts / b2b / 1e9 / hbm_nom:.1f} |")
+
+    lines += ["## Quantize / dequantize (HBM-bound)", "",
+              f"Peaks: measured copy {hbm:.1f} GB/s, nominal {hbm_nom:.0f} GB/s (80 % of nominal = 6400 GB/s = "
+              f"{100 * 6400 / hbm:.1f} % of the measured copy peak).  Times in µs: median and best of 50 launches "
+              "timed one by one, and the mean of the same 50 launches back to back (what a stream of "
+              "conversions sees; the launches overlap their neighbours' tails).", "",
+              "| kernel, config | MB | median | best | back-to-back | GB/s | % measured | % nominal |",
+              "|---|---|---|---|---|---|---|---|"]
+
+    def quantize_rows(label, X, axis, fmts, rounding=0):
+        shape = list(X.shape)
+        n, esz = X.numel(), X.element_size()
+        Xs = [X, X.clone(), X.clone()]
+        for fmt in fmts:
+            outs = [mx.mx_quantize(Xs[0], axis, fmt, rounding) for _ in range(3)]
+            t = protocol(lambda i: mx.mx_quantize(Xs[i], axis, fmt, rounding, out=outs[i]), 3)
+            stream_row(f"quantize {label} -> {FMT_NAMES[fmt]} (axis {axis})", algorithmic_bytes(n, esz, FMT_BITS[fmt]), t)
+            if axis == len(shape) - 1:
+                ds = [torch.empty_like(X) for _ in range(3)]
+                t = protocol(lambda i: mx.mx_dequantize(outs[i][0], outs[i][1], shape, fmt, X.dtype, out=ds[i]), 3)
+                stream_row(f"dequantize {FMT_NAMES[fmt]} -> {label}", algorithmic_bytes(n, esz, FMT_BITS[fmt]), t)
+                del ds
+            del outs
+        del Xs
+        torch.cuda.empty_cache()
+
+    quantize_rows("C2 BF16 8192x8192", inputs.config2("cuda"), 1, range(6))
+    d3 = inputs.config3("cuda")
+    quantize_rows("C3 X BF16 8192x4096", d3["X"], 1, [0])
+    quantize_rows("C3 W BF16 4096x16384", d3["W"], 0, [0])
+    d4 = inputs.config4("cuda")
+    quantize_rows("C4 X FP32 4096x4096 (half-away)", d4["X"], 1, [2], 1)
+    quantize_rows("C4 X FP32 4096x4096 (half-away)", d4["X"], 0, [2], 1)
+    quantize_rows("C4 W FP32 4096x4096 (half-away)", d4["W"], 0, [3], 1)
+    d5 = inputs.config5("cuda")
+    quantize_rows("C5 X BF16 16384x8192", d5["X"], 1, [0])
+    quantize_rows("C5 W BF16 8192x28672", d5["W"], 0, [4])
+
+    lines += ["", "## GEMM (tensor-bound)", "",
+              f"Peaks: 2 x measured BF16 burst = {fp8_burst:.0f} TFLOP/s, 2 x measured BF16 sustained = "
+              f"{fp8_sust:.0f}, nominal dense FP8 {fp8_nom:.0f}.  Columns as above; `sustained` = a loop of at "
+              "least two seconds of back-to-back launches (the clocks sag under the power cap).", "",
+              "| config | GFLOP | median µs | best µs | back-to-back µs | TFLOP/s | % 2xBF16 burst | % nominal | sustained TFLOP/s | % 2xBF16 sustained |",
+              "|---|---|---|---|---|---|---|---|---|---|"]
+
+    pending = []   # sustained loops run after every burst measurement: two seconds under the power
+                   # cap leave the clocks low for a while and would colour the next row
+
+    def gemm_row(label, A, B, axisA, axisB, fa, fb, M, N, K, rounding=0):
+        ea, sa = mx.mx_quantize(A, axisA, fa, rounding)
+        eb, sb = mx.mx_quantize(B, axisB, fb, rounding)
+        Cs = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(2)]
+        # warm-up by time (30 ms): the SM clock needs tens of milliseconds of load to
+        # come up, which ten launches of a 70 us kernel do not give it
+        fn = lambda i: mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=Cs[i])
+        fn(0)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
+        k = 0
+        while time.perf_counter() - t0 < 0.03:
+            fn(k & 1)
+            k += 1
+            if k % 64 == 0:
+                torch.cuda.synchronize()
+        med, best, b2b = protocol(fn, 2, reps=50)
+        del Cs
+        torch.cuda.empty_cache()
+        pending.append((label, (ea, sa, eb, sb), (fa, fb, M, N, K), (med, best, b2b)))
+        return ea, sa, eb, sb
+
+    def sustained_rows():
+        for label, (ea, sa, eb, sb), (fa, fb, M, N, K), (med, best, b2b) in pending:
+            Cs = [torch.empty((M, N), dtype=torch.float32, device="cuda") for _ in range(2)]
+            flops = 2.0 * M * N * K
+            n_loop = min(20000, max(10, int(2.2 / b2b)))
+            torch.cuda.synchronize()
+            time.sleep(1.0)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(n_loop):
+                mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=Cs[i & 1])
+            b.record()
+            torch.cuda.synchronize()
+            sust = flops * n_loop / (a.elapsed_time(b) * 1e-3) / 1e12
+            tf = flops / b2b / 1e12
+            lines.append(f"| {label} | {flops / 1e9:.4g} | {med * 1e6:.1f} | {best * 1e6:.1f} | {b2b * 1e6:.1f} | {tf:.0f} | "
+                         f"{100 * tf / fp8_burst:.1f} | {100 * tf / fp8_nom:.1f} | {sust:.0f} | {100 * sust / fp8_sust:.1f} |")
+            del Cs
+            torch.cuda.empty_cache()
+
+    d1 = inputs.config1("cuda")
+    gemm_row("C1 256x256x1024 E4M3 (latency-bound, no roofline claim)", d1["A"], d1["B"], 1, 0, 0, 0, 256, 256, 1024)
+    ops3 = gemm_row("C3 8192x16384x4096 E4M3 x E4M3", d3["X"], d3["W"], 1, 0, 0, 0, 8192, 16384, 4096)
+    n = 4096
+    gemm_row("C4 forward 4096^3 E3M2 x E2M3", d4["X"], d4["W"], 1, 0, 2, 3, n, n, n, 1)
+    gemm_row("C4 dgrad 4096^3 E3M2 x E2M3", d4["dY"], d4["W"], 1, 1, 2, 3, n, n, n, 1)
+    gemm_row("C4 wgrad 4096^3 E3M2 x E3M2", d4["X"], d4["dY"], 0, 0, 2, 2, n, n, n, 1)
+    gemm_row("C5 16384x28672x8192 E4M3 x E2M1", d5["X"], d5["W"], 1, 0, 0, 4, 16384, 28672, 8192)
+    sustained_rows()
+
+    # the oracle's dot products on a slab of C3, all host cores
+    ea, sa, eb, sb = (t.cpu().numpy().reshape(-1) for t in ops3)
+    Ms, Ns, K = 128, 1024, 4096
+    t0 = time.perf_counter()
+    O.gemm(ea[:Ms * K], sa[:Ms * K // 32], eb[:Ns * K], sb[:Ns * K // 32], Ms, Ns, K, 0, 0)
+    dt = time.perf_counter() - t0
+    gf = 2.0 * Ms * Ns * K / dt / 1e9
+    lines += ["", "## Oracle on the host cores (reported baseline, not a target)", "",
+              f"FP64 dot products of configuration 3 on a {Ms} x {Ns} x {K} slab: {dt:.2f} s on {O.threads()} threads = "
+              f"{gf:.1f} GFLOP/s; the full 8192 x 16384 x 4096 product would take {2.0 * 8192 * 16384 * 4096 / gf / 1e9:.0f} s "
+              "(extrapolated).  The quantize / dequantize sweep of the oracle is timed by the default run "
+              "(`cpu_baseline` in the JSON line).", ""]
+    return "\n".join(lines)
+
+
 def run_cpu_baseline(rows: int = 2048, seconds_target: float = 15.0):
     """The oracle, as it stands, on the host cores: the same sweep on `rows` rows of the tensor."""
     import numpy as np
@@ -576,11 +728,21 @@ def main():
     ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--impl", choices=["ours", "reference"], default="ours")
+    ap.add_argument("--report", action="store_true", help="per-kernel protocol on every configuration, as markdown "
+                                                          "on stdout (one GPU, a few minutes)")
     args = ap.parse_args()
     rank = int(os.environ.get("RANK", "0"))
     world = int(os.environ.get("WORLD_SIZE", "1"))
     local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    if args.case != "step":
+    if args.report:
+        import torch
+
+        import paper_2310_10537_b200 as mx
+        from paper_2310_10537_b200 import inputs
+        torch.cuda.set_device(0)
+        print("# Per-kernel measurements on one B200 (`python bench.py --report`)\n")
+        print(run_report(torch, mx, inputs))
+    elif args.case != "step":
         main_case(args)
     elif args.impl == "reference":
         main_reference(args, rank, world)
