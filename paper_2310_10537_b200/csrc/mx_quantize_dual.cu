@@ -61,9 +61,9 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   const size_t in_pitch = (size_t)C * esz;
   const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;          // blocks per output row
   const size_t row_out_bytes = (size_t)C * bits / 8, col_out_bytes = (size_t)R * bits / 8;
-  // 32-row tiles this warp walks: four (the staged 6- and 4-bit column codes need four), or fewer
-  // for 8-bit codes when that fills the machine more evenly
-  const uint32_t T = bits == 8 ? tiles_per_warp : 4u;
+  // 32-row tiles this warp walks: four, or fewer when that fills the machine more evenly (the staged
+  // 6- and 4-bit column codes: at least two, so that a row's run is 48 / 32 bytes)
+  const uint32_t T = bits == 8 ? tiles_per_warp : max(tiles_per_warp, 2u);
   const uint32_t tile0 = blockIdx.y * T;                             // first 32-row tile of this CTA
 
   uint32_t col_scale_word[COLS];
@@ -197,33 +197,24 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   }
   if (bits != 8) {
     __syncwarp();
-    if (((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0) {
-      // 32-byte chunks: whole sectors per request
-      constexpr uint32_t kChunks32 = cfg::kSeg / 32;
-      for (uint32_t i = lane; i < 32 * COLS * kChunks32; i += 32) {
-        const uint32_t r = i / kChunks32, ch = i - r * kChunks32;
-        const uint32_t c = r >> 5, owner = r & 31;
-        const uint2* src = reinterpret_cast<const uint2*>(sarea + r * cfg::kPitch + ch * 32);
-        const uint2 q0 = src[0], q1 = src[1], q2 = src[2], q3 = src[3];
-        const uint32_t v[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
-        st_32(elems_col + (size_t)(warp_col0 + owner * COLS + c) * col_out_bytes + (size_t)tile0 * kBpb + ch * 32, v);
-      }
-      return;
-    }
-    constexpr uint32_t kChunks = cfg::kSeg / 16;
-    for (uint32_t i = lane; i < 32 * COLS * kChunks; i += 32) {
-      const uint32_t r = i / kChunks, ch = i - r * kChunks;
+    // every output row's run of T blocks, consecutive lanes on consecutive chunks: 32-byte chunks
+    // (whole sectors per request) where the run and the tensor allow, else 16-byte ones
+    const uint32_t seg = T * kBpb;
+    const bool wide = ((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0 && seg % 32 == 0;
+    const uint32_t cb = wide ? 32u : 16u, nch = seg / cb;
+    for (uint32_t i = lane; i < 32 * COLS * nch; i += 32) {
+      const uint32_t r = i / nch, ch = i - r * nch;
       const uint32_t c = r >> 5, owner = r & 31;
-      const uint8_t* src = sarea + r * cfg::kPitch + ch * 16;
-      uint4 v;
-      if (bits == 6) {
-        const uint2 a = reinterpret_cast<const uint2*>(src)[0], b = reinterpret_cast<const uint2*>(src)[1];
-        v = make_uint4(a.x, a.y, b.x, b.y);
+      const uint2* src = reinterpret_cast<const uint2*>(sarea + r * cfg::kPitch + ch * cb);
+      uint8_t* g = elems_col + (size_t)(warp_col0 + owner * COLS + c) * col_out_bytes + (size_t)tile0 * kBpb + ch * cb;
+      const uint2 q0 = src[0], q1 = src[1];
+      if (wide) {
+        const uint2 q2 = src[2], q3 = src[3];
+        const uint32_t v[8] = {q0.x, q0.y, q1.x, q1.y, q2.x, q2.y, q3.x, q3.y};
+        st_32(g, v);
       } else {
-        v = *reinterpret_cast<const uint4*>(src);
+        *reinterpret_cast<uint4*>(g) = make_uint4(q0.x, q0.y, q1.x, q1.y);
       }
-      uint8_t* g = elems_col + (size_t)(warp_col0 + owner * COLS + c) * col_out_bytes + (size_t)tile0 * kBpb + ch * 16;
-      *reinterpret_cast<uint4*>(g) = v;
     }
   }
 }
@@ -234,16 +225,19 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
   static_assert(cfg::kSmem <= 48 * 1024, "fits the default shared-memory limit");
   const uint32_t strips = (uint32_t)(a.C / (32 * cfg::COLS));
   const uint32_t ctas_x = (strips + kDualThreads / 32 - 1) / (kDualThreads / 32);
-  // Tiles per warp (8-bit codes): the choice that needs the least time in units of one tile, given
+  // Tiles per warp: the choice that needs the least time in units of one tile, given
   // how many warps are resident at once -- e.g. 4096 x 4096 FP32 is 1.15 waves of four-tile warps
   // (two rounds) but 4.6 waves of one-tile warps (five rounds of a quarter the length).
   uint32_t T = 4;
-  if (cfg::bits == 8) {
+  {
     const uint64_t slots = (uint64_t)a.sm_count * (DTYPE == MX_BF16 ? 4 : 6);  // resident CTAs
     uint64_t best = ~0ull;
     for (uint32_t t : {4u, 2u, 1u}) {
+      if (t == 1 && cfg::bits != 8) continue;
       const uint64_t ctas = (uint64_t)ctas_x * (uint64_t)(a.R / 32 / t);
-      const uint64_t cost = (ctas + slots - 1) / slots * t;
+      // in units of a fifth of a tile; two-tile warps of 6-bit codes write 48-byte runs as half
+      // sectors, which measured about a fifth slower per tile
+      const uint64_t cost = (ctas + slots - 1) / slots * t * ((cfg::bits == 6 && t == 2) ? 6 : 5);
       if (cost < best) { best = cost; T = t; }
     }
   }
