@@ -154,8 +154,9 @@ def quantize(x: np.ndarray, axis: int, fmt: int, rounding: int = RNE, layout: in
     L = x.shape[axis]
     inner = int(np.prod(x.shape[axis + 1:], dtype=np.int64))
     rows = outer * inner
-    elems = np.zeros(rows * L * fmt_bits(fmt) // 8, dtype=np.uint8)
-    scales = np.zeros(scales_bytes(rows, L // 32, layout), dtype=np.uint8)
+    kblocks = (L + 31) // 32     # a partial last block is padded with zero codes
+    elems = np.zeros(rows * kblocks * 32 * fmt_bits(fmt) // 8, dtype=np.uint8)
+    scales = np.zeros(scales_bytes(rows, kblocks, layout), dtype=np.uint8)
     rc = lib().oracle_quantize(_ptr(x), dt, outer, L, inner, fmt, rounding, layout,
                                _ptr(elems), _ptr(scales))
     if rc != 0:

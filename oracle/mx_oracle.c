@@ -26,6 +26,10 @@
  *   - INT8: emax_elem = 0, value n/64, symmetric saturation at +-127
  *   - |X * P| above the FP32 range dequantizes to +-Inf
  *   - codes are a little-endian bit stream along the row
+ *   - an axis whose length is not a multiple of 32 ends in a partial block: the
+ *     elements that are missing are taken as +0 (they cannot change the block
+ *     maximum and encode as code 0), and the stored row is padded with those
+ *     zero codes to a whole block
  */
 #include <math.h>
 #include <stddef.h>
@@ -283,10 +287,10 @@ int oracle_quantize_block(const float* v32, int fmt, int rounding, uint8_t* code
 int oracle_quantize(const void* in, int in_dtype, int64_t outer, int64_t L, int64_t inner,
                     int fmt, int rounding, int scale_layout, uint8_t* elems, uint8_t* scales) {
   if (!fmt_ok(fmt)) return -3;
-  if (L % BLOCK != 0 || outer < 0 || inner < 0) return -2;
+  if (L < 0 || outer < 0 || inner < 0) return -2;
   const int w = FMT[fmt].bits;
-  const int64_t rows = outer * inner, kblocks = L / BLOCK;
-  const int64_t row_bytes = L * w / 8;
+  const int64_t rows = outer * inner, kblocks = (L + BLOCK - 1) / BLOCK;
+  const int64_t row_bytes = kblocks * BLOCK * w / 8; /* rows padded to whole blocks */
   memset(elems, 0, (size_t)(rows * row_bytes));
   memset(scales, 0, oracle_scales_bytes(rows, kblocks, scale_layout)); /* padding = 0x00 */
 #pragma omp parallel for schedule(static)
@@ -296,8 +300,8 @@ int oracle_quantize(const void* in, int in_dtype, int64_t outer, int64_t L, int6
     for (int64_t b = 0; b < kblocks; ++b) {
       uint32_t bits[BLOCK];
       uint8_t codes[BLOCK], sb;
-      for (int i = 0; i < BLOCK; ++i)
-        bits[i] = load_bits(in, in_dtype, (o * L + (b * BLOCK + i)) * inner + j);
+      for (int i = 0; i < BLOCK; ++i) /* positions past the end of the axis: +0 */
+        bits[i] = b * BLOCK + i < L ? load_bits(in, in_dtype, (o * L + (b * BLOCK + i)) * inner + j) : 0u;
       quantize_block_bits(bits, fmt, rounding, codes, &sb);
       for (int i = 0; i < BLOCK; ++i) put_code(out_row, b * BLOCK + i, w, codes[i]);
       scales[oracle_scale_offset(row, b, rows, kblocks, scale_layout)] = sb;
@@ -332,9 +336,9 @@ static uint16_t to_bf16(double v) {
 int oracle_dequantize(const uint8_t* elems, const uint8_t* scales, int64_t rows, int64_t L,
                       int fmt, int scale_layout, int out_dtype, void* out) {
   if (!fmt_ok(fmt)) return -3;
-  if (L % BLOCK != 0) return -2;
+  if (L < 0) return -2;
   const int w = FMT[fmt].bits;
-  const int64_t kblocks = L / BLOCK, row_bytes = L * w / 8;
+  const int64_t kblocks = (L + BLOCK - 1) / BLOCK, row_bytes = kblocks * BLOCK * w / 8;
 #pragma omp parallel for schedule(static)
   for (int64_t row = 0; row < rows; ++row) {
     const uint8_t* in_row = elems + row * row_bytes;

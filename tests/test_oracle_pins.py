@@ -466,3 +466,43 @@ def test_conv_oracle_against_brute_force_and_library():
         cols = torch.nn.functional.unfold(idx_img, (kh, kw), dilation=dl, padding=pd, stride=st)  # [N, kh*kw, Ho*Wo]
         want = cols.permute(0, 2, 1).reshape(N * Ho * Wo, kh * kw).numpy().astype(np.int64) - 1
         assert np.array_equal(src, want)
+
+
+# ---- partial last block (axis length not a multiple of 32) ----
+
+def test_partial_block_is_the_zero_padded_block():
+    """Reading: the missing elements of a last, partial block are +0 and the stored row is padded
+    with zero codes.  So quantizing a tensor with a tail must equal quantizing the tensor padded
+    with +0.0 to whole blocks (an all-explicit computation the other pins already cover), on either
+    axis, and dequantizing must return exactly the unpadded part."""
+    rng = np.random.default_rng(11)
+    for (R, L) in ((3, 1), (5, 31), (4, 33), (7, 40), (2, 100)):
+        Lp = (L + 31) // 32 * 32
+        x = (rng.standard_normal((R, L)) * np.exp(rng.standard_normal((R, 1)))).astype(np.float32)
+        x[0, -1] = -0.0
+        xp = np.zeros((R, Lp), np.float32)
+        xp[:, :L] = x
+        for fmt in range(6):
+            for layout in (O.LINEAR, O.SWIZZLED):
+                e, s = O.quantize(x, 1, fmt, O.RHAZ, layout)
+                ep, sp = O.quantize(xp, 1, fmt, O.RHAZ, layout)
+                assert e.size == R * Lp * O.fmt_bits(fmt) // 8
+                assert np.array_equal(e, ep) and np.array_equal(s, sp)
+                d = O.dequantize(e, s, R, L, fmt, O.F32, layout)
+                dp = O.dequantize(ep, sp, R, Lp, fmt, O.F32, layout)
+                assert d.shape == (R, L) and np.array_equal(d.view(np.uint32), dp[:, :L].view(np.uint32))
+            # blocks along axis 0 of the transposed tensor: the same codes, row for row
+            et, st = O.quantize(np.ascontiguousarray(x.T), 0, fmt, O.RNE, O.LINEAR)
+            e1, s1 = O.quantize(x, 1, fmt, O.RNE, O.LINEAR)
+            assert np.array_equal(et, e1) and np.array_equal(st, s1)
+
+
+def test_partial_block_worked_example():
+    """Eight elements: the scale comes from the largest of the eight, positions 8..31 hold code 0."""
+    v = np.array([[1.0, -2.0, 3.0, 0.5, 96.0, -0.25, 7.0, 12.0]], np.float32)
+    e, s = O.quantize(v, 1, O.E4M3, O.RNE, O.LINEAR)
+    assert s.tolist() == [127 + 6 - 8]                      # floor(log2 96) = 6, emax(E4M3) = 8
+    codes = O.unpack_codes(e, 32, O.E4M3)
+    assert (codes[8:] == 0).all()
+    X = 2.0 ** (6 - 8)
+    assert [O.decode_element(int(c), O.E4M3) * X for c in codes[:8]] == v[0].tolist()   # all exactly representable
