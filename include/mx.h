@@ -96,12 +96,13 @@ typedef struct {
 int mx_fmt_bits(mx_fmt_t fmt);
 
 /* Bytes of the packed element tensor produced by mx_quantize for a float tensor
- * of shape[ndim] quantized along `axis`: numel * bits / 8.  0 on bad arguments
- * (including shape[axis] % 32 != 0). */
+ * of shape[ndim] quantized along `axis`: rows * Lp * bits / 8 with rows = numel /
+ * shape[axis] and Lp = shape[axis] rounded up to a multiple of 32 (a partial last
+ * block is stored padded, see mx_quantize).  0 on bad arguments. */
 size_t mx_elems_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt);
 
 /* Bytes of the scale tensor for the same call.  rows = numel / shape[axis],
- * kblocks = shape[axis] / 32.  LINEAR: rows * kblocks.
+ * kblocks = ceil(shape[axis] / 32).  LINEAR: rows * kblocks.
  * SWIZZLED: ceil(rows/128) * ceil(kblocks/4) * 512.  0 on bad arguments. */
 size_t mx_scales_bytes(const int64_t* shape, int ndim, int axis, mx_scale_layout_t layout);
 
@@ -122,12 +123,18 @@ const char* mx_last_cuda_error(void);
 /*
  * in         contiguous row-major float tensor of shape[ndim] (opts->dtype),
  *            16-byte aligned.  View it as [outer, L, inner] with
- *            L = shape[axis]; L must be a multiple of 32.
+ *            L = shape[axis].  When L is not a multiple of 32 the axis ends in a
+ *            partial block: the paper only ever shows whole blocks, and this
+ *            library takes the missing elements as +0 (they cannot change the
+ *            block maximum) and stores every row padded with zero codes to
+ *            Lp = 32 * ceil(L / 32) elements, so that a padded row is again a
+ *            valid K-major operand (K = Lp) for mx_gemm.  Such shapes run on a
+ *            plain, slower kernel.
  * axis       the axis the scale is shared along (Section 3, last paragraph:
  *            normally the reduction dimension of the matmul that consumes the
  *            tensor).  Block (o, j, b) is in[o, 32b .. 32b+31, j].
  * elems_out  packed element codes, ALWAYS with the quantization axis innermost
- *            ("K-major"): logical [outer*inner, L], output row o*inner + j.
+ *            ("K-major"): logical [outer*inner, Lp], output row o*inner + j.
  *            For axis == ndim-1 nothing moves; for a 2-D [K x N] tensor with
  *            axis == 0 the result is the [N x K] operand that dgrad / wgrad
  *            need (Section 3: quantizing and transposing do not commute, so
@@ -148,7 +155,7 @@ const char* mx_last_cuda_error(void);
  * note).  Results that round to zero keep their sign bit in the FP formats.
  *
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE (ndim < 1 or > 8, axis out of range,
- * shape[axis] % 32 != 0, an extent < 0), MX_ERR_FMT, MX_ERR_ALIGN,
+ * an extent < 0), MX_ERR_FMT, MX_ERR_ALIGN,
  * MX_ERR_CUDA.  A tensor with zero elements is a successful no-op.
  */
 int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out,
@@ -178,7 +185,9 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row,
 /*
  * elems, scales  an MX tensor as mx_quantize writes it (K-major).
  * shape, ndim    logical float shape of that K-major tensor; axis must be
- *                ndim-1 (anything else: MX_ERR_UNSUPPORTED).
+ *                ndim-1 (anything else: MX_ERR_UNSUPPORTED).  shape[axis] need not
+ *                be a multiple of 32: the packed rows are then the padded ones
+ *                mx_quantize writes, the output rows are not padded.
  * out            contiguous float tensor of that shape (opts->dtype), 16-byte
  *                aligned.
  * v = decode(P) * 2^(byte-127); scale byte 0xFF -> NaN for the whole block;

@@ -32,6 +32,8 @@ int fmt_bits(int f) {
 
 struct View {
   int64_t outer, L, inner, numel, rows, kblocks;
+  int64_t Lp;            // L rounded up to whole blocks: the length of a packed row in elements
+  int64_t padded_numel;  // rows * Lp
 };
 
 // [outer, L, inner] view of shape[ndim] around `axis`; false on a bad shape.
@@ -44,10 +46,11 @@ bool make_view(const int64_t* shape, int ndim, int axis, View* v) {
     if (i > axis) v->inner *= shape[i];
   }
   v->L = shape[axis];
-  if (v->L % 32 != 0) return false;
   v->numel = v->outer * v->L * v->inner;
   v->rows = v->outer * v->inner;
-  v->kblocks = v->L / 32;
+  v->kblocks = (v->L + 31) / 32;  // a last, partial block is stored padded with zero codes
+  v->Lp = v->kblocks * 32;
+  v->padded_numel = v->rows * v->Lp;
   return true;
 }
 
@@ -94,7 +97,7 @@ int mx_fmt_bits(mx_fmt_t fmt) { return fmt_bits((int)fmt); }
 size_t mx_elems_bytes(const int64_t* shape, int ndim, int axis, mx_fmt_t fmt) {
   View v;
   if (!fmt_ok((int)fmt) || !make_view(shape, ndim, axis, &v)) return 0;
-  return (size_t)(v.numel / 8 * fmt_bits((int)fmt));
+  return (size_t)(v.padded_numel / 8 * fmt_bits((int)fmt));
 }
 
 size_t mx_scales_bytes(const int64_t* shape, int ndim, int axis, mx_scale_layout_t layout) {
@@ -144,7 +147,8 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
   if (!in || !elems_out || !scales_out) return MX_ERR_NULL;
   if ((uintptr_t)in % 16 || (uintptr_t)elems_out % 16 || (uintptr_t)scales_out % 16)
     return MX_ERR_ALIGN;
-  if (v.numel / 8 >= (int64_t)1 << 31 || v.rows >= (int64_t)1 << 31 || v.inner >= (int64_t)1 << 31)
+  if (v.padded_numel / 8 >= (int64_t)1 << 31 || v.rows >= (int64_t)1 << 31 || v.inner >= (int64_t)1 << 31 ||
+      v.L >= (int64_t)1 << 31)
     return MX_ERR_UNSUPPORTED;
   cudaError_t e;
   mx::QuantizeArgs a;
@@ -211,7 +215,7 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out, const int
   if (v.numel == 0) return MX_OK;
   if (!elems || !scales || !out) return MX_ERR_NULL;
   if ((uintptr_t)elems % 16 || (uintptr_t)scales % 16 || (uintptr_t)out % 16) return MX_ERR_ALIGN;
-  if (v.numel / 8 >= (int64_t)1 << 31) return MX_ERR_UNSUPPORTED;
+  if (v.padded_numel / 8 >= (int64_t)1 << 31 || v.L >= (int64_t)1 << 31) return MX_ERR_UNSUPPORTED;
   cudaError_t e;
   mx::DequantizeArgs a;
   a.elems = (const uint8_t*)elems; a.scales = scales; a.out = out;
@@ -233,7 +237,7 @@ size_t mx_quantize_host_workspace_bytes(const int64_t* shape, int ndim, int axis
   View v;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o) || !make_view(shape, ndim, axis, &v)) return 0;
   const size_t in_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
-  return align_up(in_b, 256) + align_up((size_t)v.numel / 8 * fmt_bits((int)fmt), 256) +
+  return align_up(in_b, 256) + align_up((size_t)v.padded_numel / 8 * fmt_bits((int)fmt), 256) +
          align_up(scales_bytes(v.rows, v.kblocks, o.layout), 256);
 }
 
@@ -304,7 +308,7 @@ int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scale
     return MX_ERR_WORKSPACE;
   const size_t esz = o.dtype == MX_BF16 ? 2 : 4;
   const size_t in_b = (size_t)v.numel * esz;
-  const size_t el_b = (size_t)v.numel / 8 * fmt_bits((int)fmt);
+  const size_t el_b = (size_t)v.padded_numel / 8 * fmt_bits((int)fmt);
   const size_t sc_b = scales_bytes(v.rows, v.kblocks, o.layout);
   char* d_in = (char*)workspace_dev;
   char* d_el = d_in + align_up(in_b, 256);
@@ -322,7 +326,7 @@ int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scale
         (e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
       return fail_cuda(e);
     mx_opts_t co = {o.dtype, o.layout, hp->in, 0};
-    const size_t row_in = (size_t)v.L * esz, row_el = (size_t)v.L / 8 * fmt_bits((int)fmt);
+    const size_t row_in = (size_t)v.L * esz, row_el = (size_t)v.Lp / 8 * fmt_bits((int)fmt);
     for (int c = 0; c < chunks; ++c) {
       const int64_t r0 = c * rpc, nr = (r0 + rpc <= v.rows ? rpc : v.rows - r0);
       const size_t so = scales_row_offset(r0, v.kblocks, o.layout);
@@ -443,7 +447,7 @@ static int dequantize_host_impl(const void* elems_host, const uint8_t* scales_ho
   if (workspace_bytes < mx_dequantize_host_workspace_bytes(shape, ndim, axis, fmt, opts))
     return MX_ERR_WORKSPACE;
   const size_t out_b = (size_t)v.numel * (o.dtype == MX_BF16 ? 2 : 4);
-  const size_t el_b = (size_t)v.numel / 8 * fmt_bits((int)fmt);
+  const size_t el_b = (size_t)v.padded_numel / 8 * fmt_bits((int)fmt);
   const size_t sc_b = scales_bytes(v.rows, v.kblocks, o.layout);
   char* d_out = (char*)workspace_dev;
   char* d_el = d_out + align_up(out_b, 256);
@@ -459,7 +463,7 @@ static int dequantize_host_impl(const void* elems_host, const uint8_t* scales_ho
         (e = cudaStreamWaitEvent(hp->out, hp->start, 0)) != cudaSuccess)
       return fail_cuda(e);
     mx_opts_t co = {o.dtype, o.layout, hp->in, 0};
-    const size_t row_out = (size_t)v.L * (o.dtype == MX_BF16 ? 2 : 4), row_el = (size_t)v.L / 8 * fmt_bits((int)fmt);
+    const size_t row_out = (size_t)v.L * (o.dtype == MX_BF16 ? 2 : 4), row_el = (size_t)v.Lp / 8 * fmt_bits((int)fmt);
     for (int c = 0; c < chunks; ++c) {
       const int64_t r0 = c * rpc, nr = (r0 + rpc <= v.rows ? rpc : v.rows - r0);
       const size_t so = scales_row_offset(r0, v.kblocks, o.layout);

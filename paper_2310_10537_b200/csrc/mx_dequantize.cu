@@ -205,8 +205,69 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
   }
 }
 
+// Axis lengths that are not a multiple of 32: the packed rows are padded to whole blocks, the
+// output rows are not.  One thread per block, element by element, on the exact decode path.
+template <int FMT, int DTYPE, int LAYOUT>
+__global__ void __launch_bounds__(kDqThreads)
+dequantize_tail_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__ scales,
+                       void* __restrict__ out, uint32_t rows, uint32_t L, uint32_t kblocks, uint64_t total_blocks) {
+  constexpr int bits = FmtTraits<FMT>::bits;
+  constexpr int kWords = bits;  // 32-bit words of codes per block
+  pdl_prologue();
+  for (uint64_t b = (uint64_t)blockIdx.x * kDqThreads + threadIdx.x; b < total_blocks;
+       b += (uint64_t)gridDim.x * kDqThreads) {
+    const uint32_t row = (uint32_t)(b / kblocks), kb = (uint32_t)(b - (uint64_t)row * kblocks);
+    const uint32_t* src = reinterpret_cast<const uint32_t*>(elems + (size_t)row * (kblocks * (kBlock * bits / 8)) +
+                                                            (size_t)kb * (kBlock * bits / 8));
+    uint32_t w[kWords];
+#pragma unroll
+    for (int i = 0; i < kWords; ++i) w[i] = __ldg(src + i);
+    const uint32_t sb = __ldg(scales + scale_offset<LAYOUT>(row, kb, kblocks));
+    const float X = __uint_as_float(sb == 0 ? 0x00400000u : (sb == 255 ? 0x7FC00000u : sb << 23));
+#pragma unroll
+    for (int i = 0; i < kBlock / 2; ++i) {
+      uint32_t pair;  // code(2i) | code(2i+1) << 8   (4-bit: both in the low byte)
+      if (bits == 8) {
+        pair = (w[i / 2] >> (16 * (i & 1))) & 0xFFFFu;
+      } else if (bits == 4) {
+        pair = (w[i / 4] >> (8 * (i & 3))) & 0xFFu;
+      } else {
+        const int bit = 12 * i;
+        uint32_t q = w[bit / 32] >> (bit % 32);
+        if (bit % 32 > 20) q |= w[(bit / 32 + 1) % kWords] << (32 - bit % 32);
+        q &= 0xFFFu;
+        pair = (q & 0x3Fu) | ((q & 0xFC0u) << 2);
+      }
+      float v[2];
+      decode_pair<FMT>(pair, v[0], v[1]);
+#pragma unroll
+      for (int h = 0; h < 2; ++h) {
+        const uint32_t k = kb * kBlock + 2 * i + h;
+        if (k >= L) continue;
+        const float r = v[h] * X;  // exact unless it overflows to Inf
+        const size_t idx = (size_t)row * L + k;
+        if (DTYPE == MX_F32) {
+          reinterpret_cast<uint32_t*>(out)[idx] = (r != r) ? 0x7FC00000u : __float_as_uint(r);
+        } else {
+          uint32_t pk;
+          asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(pk) : "f"(0.0f), "f"(r));  // round to nearest even
+          reinterpret_cast<uint16_t*>(out)[idx] = (r != r) ? (uint16_t)0x7FC0u : (uint16_t)(pk & 0xFFFFu);
+        }
+      }
+    }
+  }
+}
+
 template <int FMT, int DTYPE, int LAYOUT>
 static cudaError_t launch_dq(const DequantizeArgs& a) {
+  if (a.L % kBlock != 0) {
+    const uint32_t kb = (uint32_t)((a.L + kBlock - 1) / kBlock);
+    const uint64_t total = (uint64_t)a.rows * kb;
+    const uint64_t want = (total + kDqThreads - 1) / kDqThreads, cap = (uint64_t)a.sm_count * 64;
+    return launch_pdl(dequantize_tail_kernel<FMT, DTYPE, LAYOUT>, dim3((uint32_t)(want < cap ? want : cap)),
+                      dim3(kDqThreads), 0, a.stream, a.elems, a.scales, a.out, (uint32_t)a.rows, (uint32_t)a.L, kb,
+                      total);
+  }
   constexpr int kElems = DTYPE == MX_BF16 ? 32 : 16;
   const uint32_t n_units = (uint32_t)(a.rows * a.L / kElems);
   const uint32_t kblocks = (uint32_t)(a.L / kBlock);

@@ -532,8 +532,91 @@ static cudaError_t launch_strided(const QuantizeArgs& a) {
   return launch_strided_cols<FMT, ROUND, DTYPE, LAYOUT, 1>(a);
 }
 
+// ---------------------------------------------------------------------------
+// Axis lengths that are not a multiple of 32
+// ---------------------------------------------------------------------------
+
+// The axis then ends in a partial block: its missing elements count as +0 (they cannot change the
+// block maximum and encode as code 0) and the stored row is padded with zero codes to a whole
+// block.  Rare shapes, so one plain kernel serves every layout: a thread converts one block of the
+// [outer, L, inner] tensor, element by element; consecutive threads take consecutive inner
+// positions (coalesced when the axis is strided) or consecutive blocks of a row.
+template <int FMT, int ROUND, int DTYPE, int LAYOUT>
+__global__ void __launch_bounds__(256)
+quantize_tail_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems, uint8_t* __restrict__ scales,
+                     uint32_t outer, uint32_t L, uint32_t inner, uint32_t kblocks, uint64_t total_blocks) {
+  constexpr int bits = FmtTraits<FMT>::bits;
+  pdl_prologue();
+  for (uint64_t b = (uint64_t)blockIdx.x * 256 + threadIdx.x; b < total_blocks; b += (uint64_t)gridDim.x * 256) {
+    uint32_t o, kb, j;
+    if (inner > 1) {
+      j = (uint32_t)(b % inner);
+      const uint64_t t = b / inner;
+      kb = (uint32_t)(t % kblocks);
+      o = (uint32_t)(t / kblocks);
+    } else {
+      j = 0;
+      kb = (uint32_t)(b % kblocks);
+      o = (uint32_t)(b / kblocks);
+    }
+    const uint32_t row = o * inner + j;
+    float v[kBlock];
+#pragma unroll
+    for (int i = 0; i < kBlock; ++i) {
+      const uint32_t k = kb * kBlock + i;
+      float x = 0.0f;
+      if (k < L) {
+        const size_t idx = ((size_t)o * L + k) * inner + j;
+        if (DTYPE == MX_BF16)
+          x = __uint_as_float((uint32_t)__ldg(reinterpret_cast<const uint16_t*>(in) + idx) << 16);
+        else
+          x = __ldg(reinterpret_cast<const float*>(in) + idx);
+      }
+      v[i] = x;
+    }
+    float m = v[0];
+#pragma unroll
+    for (int i = 1; i < kBlock; ++i) m = absmax_nan(m, v[i]);
+    const BlockScale s = block_scale<FMT>(m);
+    uint32_t w[8];
+#pragma unroll
+    for (int g = 0; g < 4; ++g) {
+      const float x[8] = {v[8 * g], v[8 * g + 1], v[8 * g + 2], v[8 * g + 3],
+                          v[8 * g + 4], v[8 * g + 5], v[8 * g + 6], v[8 * g + 7]};
+      cast8<FMT, ROUND>(x, s, w[2 * g], w[2 * g + 1]);
+    }
+    uint32_t* dst = reinterpret_cast<uint32_t*>(elems + (size_t)row * (kblocks * (kBlock * bits / 8)) +
+                                                (size_t)kb * (kBlock * bits / 8));
+    if (bits == 8) {
+#pragma unroll
+      for (int i = 0; i < 8; ++i) dst[i] = w[i];
+    } else if (bits == 4) {
+#pragma unroll
+      for (int i = 0; i < 4; ++i) dst[i] = w[2 * i];
+    } else {
+      uint64_t q0, q1, q2;
+      pack6(w, q0, q1, q2);
+      dst[0] = (uint32_t)q0; dst[1] = (uint32_t)(q0 >> 32);
+      dst[2] = (uint32_t)q1; dst[3] = (uint32_t)(q1 >> 32);
+      dst[4] = (uint32_t)q2; dst[5] = (uint32_t)(q2 >> 32);
+    }
+    scales[scale_offset<LAYOUT>(row, kb, kblocks)] = (uint8_t)s.byte;
+  }
+}
+
+template <int FMT, int ROUND, int DTYPE, int LAYOUT>
+static cudaError_t launch_tail(const QuantizeArgs& a) {
+  const uint32_t kblocks = (uint32_t)((a.L + kBlock - 1) / kBlock);
+  const uint64_t total = (uint64_t)a.outer * a.inner * kblocks;
+  const uint64_t want = (total + 255) / 256, cap = (uint64_t)a.sm_count * 64;
+  return launch_pdl(quantize_tail_kernel<FMT, ROUND, DTYPE, LAYOUT>, dim3((uint32_t)(want < cap ? want : cap)),
+                    dim3(256), 0, a.stream, a.in, a.elems, a.scales, (uint32_t)a.outer, (uint32_t)a.L,
+                    (uint32_t)a.inner, kblocks, total);
+}
+
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
 static cudaError_t launch_any(const QuantizeArgs& a) {
+  if (a.L % kBlock != 0) return launch_tail<FMT, ROUND, DTYPE, LAYOUT>(a);
   if (a.inner == 1) return launch_lastaxis<FMT, ROUND, DTYPE, LAYOUT>(a);
   return launch_strided<FMT, ROUND, DTYPE, LAYOUT>(a);
 }

@@ -41,7 +41,8 @@ def test_helpers_match_oracle_layouts():
                 for k in range(kb):
                     assert mx.mx_scale_offset(r, k, rows, kb, layout) == O.scale_offset(r, k, rows, kb, layout)
     assert mx.mx_scale_offset(5, 0, 5, 1, 1) == ctypes.c_size_t(-1).value
-    assert mx.mx_elems_bytes([4, 33], 1, 0) == 0
+    assert mx.mx_elems_bytes([4, 33], 1, 0) == 4 * 64          # a partial block is stored padded
+    assert mx.mx_scales_bytes([4, 33], 1, 0) == 4 * 2
     assert mx.mx_scales_bytes([4, 64], 2, 0) == 0
 
 
@@ -56,7 +57,6 @@ def test_argument_validation_without_gpu():
     assert q(p, p, p, None, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_NULL
     assert q(p, p, p, shape, 2, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
     assert q(p, p, p, shape, 0, 0, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
-    assert q(p, p, p, shape, 2, 0, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE  # 4 % 32 != 0
     assert q(p, p, p, shape, 2, 1, 6, 0, ctypes.byref(o)) == mx.MX_ERR_FMT
     assert q(p, p, p, shape, 2, 1, 0, 2, ctypes.byref(o)) == mx.MX_ERR_FMT
     assert q(p + 4, p, p, shape, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_ALIGN
@@ -65,7 +65,10 @@ def test_argument_validation_without_gpu():
     empty = (ctypes.c_int64 * 2)(0, 64)
     assert q(None, None, None, empty, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_OK
     d = lib.mx_dequantize
-    assert d(p, p, p, shape, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
+    assert d(p, p, p, shape, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_UNSUPPORTED   # blocks must run along the last axis
+    neg = (ctypes.c_int64 * 2)(4, -64)
+    assert d(p, p, p, neg, 2, 1, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
+    assert q(p, p, p, neg, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE
     shape3 = (ctypes.c_int64 * 2)(64, 4)
     assert d(p, p, p, shape3, 2, 0, 0, ctypes.byref(o)) == mx.MX_ERR_UNSUPPORTED
     assert d(p, None, p, shape, 2, 1, 0, ctypes.byref(o)) == mx.MX_ERR_NULL

@@ -186,11 +186,10 @@ def test_empty_and_error_paths_on_device():
     x = torch.empty((0, 64), device="cuda")
     e, s = mx.mx_quantize(x, 1, mx.MX_E4M3)
     assert e.numel() == 0 and s.numel() == 0
-    with pytest.raises(mx.MxError) as ei:
-        mx.mx_quantize(torch.zeros((4, 48), device="cuda"), 1, mx.MX_E4M3,
-                       out=(torch.zeros(256, dtype=torch.uint8, device="cuda"),
-                            torch.zeros(512, dtype=torch.uint8, device="cuda")))
-    assert ei.value.status == mx.MX_ERR_SHAPE
+    shape_neg = (ctypes.c_int64 * 2)(4, -48)
+    z = torch.zeros(4096, dtype=torch.uint8, device="cuda")
+    assert mx.lib().mx_quantize(z.data_ptr(), z.data_ptr() + 1024, z.data_ptr() + 2048, shape_neg, 2, 1, 0, 0,
+                                None) == mx.MX_ERR_SHAPE
     buf = torch.zeros(4096, dtype=torch.uint8, device="cuda")
     shape = (ctypes.c_int64 * 2)(4, 64)
     rc = mx.lib().mx_quantize(buf.data_ptr() + 4, buf.data_ptr() + 2048, buf.data_ptr() + 3072,
@@ -225,12 +224,15 @@ def test_host_buffer_entry_points():
     (1000, 4064, torch.float32, 2, 1),      # ragged: last chunk of 104 rows, 127 blocks per row (padded chunks)
     (1000, 4064, torch.float32, 4, 0),      # the same with linear scales
     (700, 8192, torch.bfloat16, 5, 1),
+    (600, 4100, torch.float32, 3, 1),       # a partial last block in every row, chunked
+    (50, 70, torch.bfloat16, 0, 0),         # the same below the chunking limit
 ])
 def test_host_buffer_entry_points_pipelined(rows, cols, dtype, fmt, layout):
     """Sizes at which the host-buffer calls cut the tensor into row chunks and overlap the copies
     of neighbouring chunks on two internal streams: every output byte against the oracle, guard
     bytes around the pinned outputs intact."""
-    x = inputs.adversarial("cpu", rows=rows, cols=cols, dtype=dtype, seed=rows + fmt).pin_memory()
+    padded = (cols + 31) // 32 * 32      # the generator builds whole blocks; a tail is cut afterwards
+    x = inputs.adversarial("cpu", rows=rows, cols=padded, dtype=dtype, seed=rows + fmt)[:, :cols].contiguous().pin_memory()
     shape = [rows, cols]
     G = 4096
     eb, sb = mx.mx_elems_bytes(shape, 1, fmt), mx.mx_scales_bytes(shape, 1, layout)
@@ -353,3 +355,58 @@ def test_queued_host_calls():
         mx.mx_host_synchronize()
         for fmt, out, w in zip(FMTS, backs, want):
             assert (out.view(torch.int16).numpy().view(np.uint16) == w).all(), fmt
+
+
+@pytest.mark.parametrize("shape,axis", [
+    ((5, 40), 1), ((300, 1), 1), ((129, 31), 1), ((7, 100), 1), ((64, 4100), 1),      # last axis
+    ((40, 300), 0), ((33, 7), 0), ((100, 130), 0), ((1, 257), 0),                    # strided axis
+    ((3, 50, 6), 1), ((2, 3, 45), 2),
+])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_partial_blocks(shape, axis, dtype):
+    """Axis lengths that are not multiples of 32: a partial last block, rows stored padded with zero
+    codes.  Codes, scales and the dequantized tensor byte for byte against the oracle, six formats,
+    both layouts, guard bands around the outputs."""
+    g = torch.Generator(device="cuda").manual_seed(sum(shape) + axis)
+    x = (torch.randn(shape, generator=g, device="cuda") * torch.exp(2 * torch.randn(shape[:1] + (1,) * (len(shape) - 1), generator=g, device="cuda"))).to(dtype)
+    x.view(-1)[::17] = 0.0
+    x.view(-1)[3::29] = float("inf") if x.numel() > 40 else 1.0
+    L = shape[axis]
+    rows = x.numel() // L
+    for fmt in FMTS:
+        for layout in (mx.MX_SCALES_LINEAR, mx.MX_SCALES_SWIZZLED):
+            nb_e, nb_s = mx.mx_elems_bytes(list(shape), axis, fmt), mx.mx_scales_bytes(list(shape), axis, layout)
+            ge, gs = Guarded(nb_e), Guarded(nb_s)
+            mx.mx_quantize(x, axis, fmt, mx.MX_RHAZ, layout, out=(ge.view, gs.view))
+            torch.cuda.synchronize()
+            ge.check()
+            gs.check()
+            we, ws = O.quantize(to_oracle_input(x), axis, fmt, O.RHAZ, layout)
+            assert nb_e == we.size and nb_s == ws.size
+            assert np.array_equal(ge.view.cpu().numpy(), we), (fmt, layout, "codes")
+            assert np.array_equal(gs.view.cpu().numpy(), ws), (fmt, layout, "scales")
+            # back: the packed tensor is [rows, L] with blocks along its last axis
+            go = Guarded(rows * L * x.element_size())
+            out = go.view.view(dtype).view(rows, L)
+            mx.mx_dequantize(ge.view, gs.view, [rows, L], fmt, dtype, layout, out=out)
+            torch.cuda.synchronize()
+            go.check()
+            want = O.dequantize(we, ws, rows, L, fmt, O.BF16 if dtype == torch.bfloat16 else O.F32, layout)
+            got = out.view(torch.int16).cpu().numpy().view(np.uint16) if dtype == torch.bfloat16 else out.cpu().numpy()
+            assert np.array_equal(got.view(np.uint8), want.view(np.uint8)), (fmt, layout, "dequantized")
+
+
+def test_partial_block_operand_feeds_the_gemm():
+    """A K that is not a multiple of 32: the padded rows are a valid operand with K rounded up."""
+    M, N, K = 256, 384, 200
+    Kp = 224
+    g = torch.Generator(device="cuda").manual_seed(5)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    ea, sa = mx.mx_quantize(A, 1, mx.MX_E4M3)
+    eb, sb = mx.mx_quantize(B, 1, mx.MX_E5M2)
+    C = mx.mx_gemm(ea, sa, eb, sb, M, N, Kp, mx.MX_E4M3, mx.MX_E5M2, check_status=True)
+    oa, osa = O.quantize(A.cpu().numpy(), 1, O.E4M3)
+    ob, osb = O.quantize(B.cpu().numpy(), 1, O.E5M2)
+    c64, s = O.gemm(oa, osa, ob, osb, M, N, Kp, O.E4M3, O.E5M2)
+    assert (np.abs(C.double().cpu().numpy() - c64) <= 1e-5 * s).all()
