@@ -630,3 +630,46 @@ def test_output_beyond_4gib():
     assert (np.abs(got - c64) <= TOL * s).all()
     # every element was written: an untouched output would keep the fill value
     assert not bool((C.view(torch.int32) == -1515870811).any())     # 0xA5A5A5A5
+
+
+def test_cuda_graph_replay():
+    """The device entry points only queue work on the caller's stream, so a step (quantize both
+    operands, GEMM, dequantize) can be captured in a CUDA graph after one warm-up call and replayed
+    on new data: the replay must give what the eager calls give on that data."""
+    M, N, K = 256, 512, 1024
+    g = torch.Generator(device="cuda").manual_seed(21)
+    A = torch.randn((M, K), generator=g, device="cuda", dtype=torch.bfloat16)
+    B = torch.randn((K, N), generator=g, device="cuda", dtype=torch.bfloat16)
+    fa, fb = mx.MX_E4M3, mx.MX_E2M1
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 0, fb)
+    C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+    back = torch.empty_like(A)
+
+    def step():
+        mx.mx_quantize(A, 1, fa, out=(ea, sa))
+        mx.mx_quantize(B, 0, fb, out=(eb, sb))
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C)
+        mx.mx_dequantize(ea, sa, [M, K], fa, torch.bfloat16, out=back)
+
+    side = torch.cuda.Stream()
+    side.wait_stream(torch.cuda.current_stream())
+    with torch.cuda.stream(side):
+        step()                      # warm-up: one-time attribute settings happen outside the capture
+    torch.cuda.current_stream().wait_stream(side)
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(graph):
+        step()
+    # new data in the same buffers, then replay
+    A.copy_(torch.randn((M, K), generator=g, device="cuda").to(torch.bfloat16))
+    B.copy_(torch.randn((K, N), generator=g, device="cuda").to(torch.bfloat16) * 0.1)
+    graph.replay()
+    torch.cuda.synchronize()
+    got = (ea.clone(), sa.clone(), eb.clone(), sb.clone(), C.clone(), back.clone())
+    step()
+    torch.cuda.synchronize()
+    for a, b in zip(got, (ea, sa, eb, sb, C, back)):
+        assert torch.equal(a.view(torch.uint8), b.view(torch.uint8))
+    # and the eager result is the oracle's
+    c64, s = O.gemm(*(t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb)), M, N, K, fa, fb)
+    assert (np.abs(C.double().cpu().numpy() - c64) <= TOL * s).all()
