@@ -40,7 +40,7 @@ namespace {
 constexpr int BM = 128;         // rows of C per tile (= MMA M, one TMEM lane per row)
 constexpr int BK = 128;         // K elements per pipeline stage: 4 MX blocks, 4 MMAs
 constexpr int kMmaK = 32;       // K of one kind::mxf8f6f4 MMA = the MX block size
-constexpr int kThreads = 352;   // 11 warps: producer, MMA issuer, 8 epilogue warps, scale copier
+constexpr int kThreads = 384;   // 12 warps: producer, MMA issuer, 8 epilogue warps, scale copier, scale producer
 constexpr int kTmemCols = 512;  // whole tensor memory of the SM (one CTA per SM)
 constexpr long long kSpinLimit = 2000000000LL;  // cycles (~1 s) before a wait gives up
 
@@ -553,6 +553,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         }
       }
     }
+  } else if (warp == 11) {
+    // the pair kernel's scale producer; no work here
   } else {
     // -------------------------------- epilogue --------------------------------
     // Two warps per TMEM lane quarter, each taking half of the tile's columns into registers;
@@ -652,7 +654,7 @@ struct Cfg2 {
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;
   static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
-  static constexpr uint32_t kNumBars = 3 * kStages + 2;
+  static constexpr uint32_t kNumBars = 4 * kStages + 2;  // full, empty, scales ready, scales landed; accumulator x 2
   // Bytes used from the 1024-byte aligned base, and the request: up to 1024 bytes of slack for the
   // alignment, fewer where the budget is tight (the kernel checks that what it got suffices).
   static constexpr uint32_t kUsedBytes = kOffBar + kNumBars * 8 + 16;
@@ -734,9 +736,9 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
   constexpr int BN = cfg::BN;
   constexpr bool WIDE = BN == 384;
-  // copies per stage, one producer lane each: A, B, [second part of B], [A scales, B scales]
-  constexpr uint32_t kProd = (DENSE ? 2 : 4) + (WIDE ? 1 : 0);
-  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
+  // operand copies per stage, one producer lane each: A, B, [second part of B]
+  constexpr uint32_t kOperandCopies = 2 + (WIDE ? 1 : 0);
+  constexpr uint32_t kOperandMask = (1u << kOperandCopies) - 1u;
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -753,6 +755,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t acc_full_bar = bar0 + 8 * (2 * cfg::kStages);
   const uint32_t acc_empty_bar = bar0 + 8 * (2 * cfg::kStages + 1);
   auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * cfg::kStages + 2 + s); };
+  auto sf_full_bar = [&](uint32_t s) { return bar0 + 8 * (3 * cfg::kStages + 2 + s); };
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -769,6 +772,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       mbar_init(full_bar(s), 1);   // used in the leader only: its producer's arrive + all bytes
       mbar_init(empty_bar(s), 1);  // one tcgen05.commit per use, delivered to both CTAs
       mbar_init(sf_ready_bar(s), 1);  // used in the leader only: the copier's tcgen05.commit
+      mbar_init(sf_full_bar(s), 1);   // used in the leader only: the scale producer's arrive + scale bytes
     }
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 16);  // eight epilogue warps in each CTA (the leader's barrier is used)
@@ -794,39 +798,34 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   if (warp == 0) {
     // ------------------------- TMA producer (both CTAs) -------------------------
-    if (lane < kProd) {
+    // Operand tiles only: the scale chunks have a producer warp of their own (below) -- with all four
+    // copies of a stage issued from here the kernel ran a tenth slower than with two.
+    if (lane < kOperandCopies) {
       // role of this lane: 0 A, 1 B (rows 128 rank .. of the tile), 2 second part of B (wide tile:
-      // rows 256 + 64 rank ..), 3 A scales, 4 B scales
-      const uint32_t role = WIDE ? lane : (lane < 2 ? lane : lane + 1);
-      const CUtensorMap* map = role == 0 ? &tmap_a : role == 1 ? &tmap_b : role == 2 ? &tmap_b2
-                               : role == 3 ? &tmap_sa : &tmap_sb;
-      const uint32_t dst_off = role == 0 ? cfg::kOffA : role == 1 ? cfg::kOffB : role == 2 ? cfg::kOffB + 128u * 128u
-                               : role == 3 ? cfg::kOffSf : cfg::kOffSf + cfg::kSfABytes;
-      const uint32_t dst_stride = role == 0 ? cfg::kABytes : role < 3 ? cfg::kBBytes : cfg::kSfBytes;
+      // rows 256 + 64 rank ..)
+      const uint32_t role = lane;
+      const CUtensorMap* map = role == 0 ? &tmap_a : role == 1 ? &tmap_b : &tmap_b2;
+      const uint32_t dst_off = role == 0 ? cfg::kOffA : role == 1 ? cfg::kOffB : cfg::kOffB + 128u * 128u;
+      const uint32_t dst_stride = role == 0 ? cfg::kABytes : cfg::kBBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
         // this CTA's 128 rows of A and its rows of B (B rows may lie past N on a ragged tile: zero
-        // fill or the next matrix of a batch; their columns are not stored); its own A scales and the
-        // B scales of all BN columns
-        const int cy_fixed = role == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
-                             : role == 1 ? (int)(tc.b * N + tc.tn * BN + rank * 128)
-                                         : (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
-        const int cz = role == 3 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
-                                 : role == 4 ? (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups) : 0;
+        // fill or the next matrix of a batch; their columns are not stored)
+        const int cy = role == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
+                       : role == 1 ? (int)(tc.b * N + tc.tn * BN + rank * 128)
+                                   : (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             ok = false;
           }
-          if (!__all_sync(kProdMask, ok)) { ok = false; break; }
+          if (!__all_sync(kOperandMask, ok)) { ok = false; break; }
           const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
           if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
-          __syncwarp(kProdMask);
-          const int cx = role < 3 ? (int)(kc * BKe) : 0;
-          const int cy = role < 3 ? cy_fixed : (int)(kc * cfg::kKChunks);
-          tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
+          __syncwarp(kOperandMask);
+          tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, (int)(kc * BKe), cy, 0, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -902,7 +901,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         bool ok = true;
         for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
           for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-            if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+            if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
               raise_abort(abort_flag, ST_SCALE_WAIT);
               ok = false;
               break;
@@ -924,6 +923,40 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             tc_commit_leader(sf_ready_bar(stage));  // arrives when the copies have completed in both CTAs
             if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
           }
+        }
+      }
+    }
+  } else if (warp == 11) {
+    // ------------------------ scale producer (both CTAs) ------------------------
+    // lane 0: this CTA's A scales, lane 1: the B scales of all BN columns; both complete on the
+    // leader's per-stage "scales landed" barrier, which the leader's lane 0 arms.  A stage's scale
+    // buffer and scale columns are free when the stage is (the MMAs that read them have completed).
+    if constexpr (!DENSE) {
+      if (lane < 2) {
+        const CUtensorMap* map = lane == 0 ? &tmap_sa : &tmap_sb;
+        const uint32_t dst_off = lane == 0 ? cfg::kOffSf : cfg::kOffSf + cfg::kSfABytes;
+        uint32_t stage = 0, phase = 0;
+        bool ok = true;
+        for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+          const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+          const int cz = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
+                                   : (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups);
+          for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+              raise_abort(abort_flag, ST_PRODUCER_WAIT);
+              ok = false;
+            }
+            if (!__all_sync(0x3u, ok)) { ok = false; break; }
+            if (rank == 0 && lane == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * cfg::kSfBytes);
+            __syncwarp(0x3u);
+            tma_load_3d_pair(smem_base + dst_off + stage * cfg::kSfBytes, map, 0, (int)(kc * cfg::kKChunks), cz,
+                             sf_full_bar(stage) & kPeerMask);
+            if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+        if (!ok) {
+          const long long t0 = clock64();
+          while (clock64() - t0 < 2000000LL) {}
         }
       }
     }
@@ -1214,7 +1247,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t rows_per_cta = 128u + cfg::kBRows;
   const uint32_t op_bytes = (F4 || DENSE) ? rows_per_cta * 128u
                                : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + cfg::kBRows * BK * fmt_bits(a.fmtB) / 8);
-  const uint32_t tx_pair = 2u * (op_bytes + (DENSE ? 0u : cfg::kSfBytes));
+  const uint32_t tx_pair = 2u * op_bytes;  // the scale chunks complete on a barrier of their own
   // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code();
   // kind::f16: BF16 = 1 for both operands, FP32 accumulator = 1 in bits [4,6), no scale-format bit.
   // N field = 256: the first (or only) MMA of a K step; the kernel derives the N = 128 one.
