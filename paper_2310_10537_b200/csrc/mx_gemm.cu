@@ -79,8 +79,9 @@ struct Cfg {
   static constexpr uint32_t kOffEpi = kOffB + kStages * kBBytes;   // 1024-byte aligned
   static constexpr uint32_t kOffSf = kOffEpi + kEpiBytes;
   static constexpr uint32_t kOffBar = kOffSf + kStages * kSfBytes;
-  // barriers: full[S], empty[S], acc_full[A], acc_empty[A], scales_ready[S]; then tmem slot + abort flag
-  static constexpr uint32_t kNumBars = 3 * kStages + 2 * kAccStages;
+  // barriers: full[S], empty[S], acc_full[A], acc_empty[A], scales_ready[S], scales_landed[S]; then
+  // tmem slot + abort flag
+  static constexpr uint32_t kNumBars = 4 * kStages + 2 * kAccStages;
   static constexpr uint32_t kSmemBytes = kOffBar + kNumBars * 8 + 16 + 1024;  // + alignment slack
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
   static_assert(kSmemBytes <= 232448, "shared memory budget");
@@ -408,6 +409,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   auto acc_full_bar = [&](uint32_t a) { return bar0 + 8 * (2 * cfg::kStages + a); };
   auto acc_empty_bar = [&](uint32_t a) { return bar0 + 8 * (2 * cfg::kStages + cfg::kAccStages + a); };
   auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * cfg::kStages + 2 * cfg::kAccStages + s); };
+  auto sf_full_bar = [&](uint32_t s) { return bar0 + 8 * (3 * cfg::kStages + 2 * cfg::kAccStages + s); };
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -416,8 +418,6 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
   const uint32_t tiles_m = (M + BM - 1) / BM, tiles_n = (N + BN - 1) / BN;
   const uint32_t num_tiles = batch * tiles_m * tiles_n;
   constexpr uint32_t BKe = DENSE ? 64 : BK;     // K elements per stage
-  constexpr uint32_t kProd = DENSE ? 2 : 4;      // copies per stage, one producer lane each
-  constexpr uint32_t kProdMask = (1u << kProd) - 1u;
   const uint32_t k_chunks = (K + BKe - 1) / BKe;  // a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
@@ -425,6 +425,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       mbar_init(full_bar(s), 1);
       mbar_init(empty_bar(s), 1);
       mbar_init(sf_ready_bar(s), 1);  // the copier's tcgen05.commit
+      mbar_init(sf_full_bar(s), 1);   // the scale producer's arrive + scale bytes
     }
     for (uint32_t a = 0; a < cfg::kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
@@ -449,34 +450,30 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    // lanes 0..3 issue the four copies of a stage together (see tma_load_3d)
-    if (lane < kProd) {
-      const CUtensorMap* map = lane == 0 ? &tmap_a : lane == 1 ? &tmap_b : lane == 2 ? &tmap_sa : &tmap_sb;
-      const uint32_t dst_off = lane == 0 ? cfg::kOffA : lane == 1 ? cfg::kOffB : lane == 2 ? cfg::kOffSf
-                                                                                         : cfg::kOffSf + 512u;
-      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : lane == 1 ? cfg::kBBytes : cfg::kSfBytes;
+    // lanes 0 and 1 issue the two operand copies of a stage together (see tma_load_3d); the scale
+    // chunks have a producer warp of their own (warp 11)
+    if (lane < 2) {
+      const CUtensorMap* map = lane == 0 ? &tmap_a : &tmap_b;
+      const uint32_t dst_off = lane == 0 ? cfg::kOffA : cfg::kOffB;
+      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : cfg::kBBytes;
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        // operands: (k, row, 0); scales: (0, k chunk, 128-row group), rows counted through the
-        // whole batch.  Rows or groups past the end of a B matrix on a ragged last tile belong to
-        // the next matrix of the batch or are zero-filled by the copy; their columns are not stored.
-        const int cy_fixed = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * BM) : (int)(tc.b * N + tc.tn * BN);
-        const int cz = lane == 2 ? (int)(tc.b * tiles_m + tc.tm)
-                                 : lane == 3 ? (int)((tc.b * N + tc.tn * BN) / 128) : 0;
+        // (k, row, 0), rows counted through the whole batch.  Rows past the end of a B matrix on a
+        // ragged last tile belong to the next matrix of the batch or are zero-filled by the copy;
+        // their columns are not stored.
+        const int cy = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * BM) : (int)(tc.b * N + tc.tn * BN);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             ok = false;
           }
-          if (!__all_sync(kProdMask, ok)) { ok = false; break; }
+          if (!__all_sync(0x3u, ok)) { ok = false; break; }
           const uint32_t fb = full_bar(stage);
           if (lane == 0) mbar_arrive_expect_tx(fb, tx_bytes);
-          __syncwarp(kProdMask);
-          const int cx = lane < 2 ? (int)(kc * BKe) : 0;
-          const int cy = lane < 2 ? cy_fixed : (int)kc;
-          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
+          __syncwarp(0x3u);
+          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, (int)(kc * BKe), cy, 0, fb);
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -536,7 +533,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(full_bar(stage), phase, abort_flag)) {
+          if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
             raise_abort(abort_flag, ST_SCALE_WAIT);
             ok = false;
             break;
@@ -554,7 +551,36 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       }
     }
   } else if (warp == 11) {
-    // the pair kernel's scale producer; no work here
+    // ----------------------------- scale producer -----------------------------
+    // lane 0: the A scales of the tile's 128 rows, lane 1: the B scales of its BN columns -- (0, K
+    // chunk, 128-row group), groups counted through the whole batch; both complete on the per-stage
+    // "scales landed" barrier.  A stage's scale buffer and scale columns are free when the stage is.
+    if (!DENSE && lane < 2) {
+      const CUtensorMap* map = lane == 0 ? &tmap_sa : &tmap_sb;
+      const uint32_t dst_off = lane == 0 ? cfg::kOffSf : cfg::kOffSf + 512u;
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        const int cz = lane == 0 ? (int)(tc.b * tiles_m + tc.tm) : (int)((tc.b * N + tc.tn * BN) / 128);
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+            raise_abort(abort_flag, ST_PRODUCER_WAIT);
+            ok = false;
+          }
+          if (!__all_sync(0x3u, ok)) { ok = false; break; }
+          const uint32_t fb = sf_full_bar(stage);
+          if (lane == 0) mbar_arrive_expect_tx(fb, cfg::kSfBytes);
+          __syncwarp(0x3u);
+          tma_load_3d(smem_base + dst_off + stage * cfg::kSfBytes, map, 0, (int)kc, cz, fb);
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
   } else {
     // -------------------------------- epilogue --------------------------------
     // Two warps per TMEM lane quarter, each taking half of the tile's columns into registers;
@@ -1167,11 +1193,12 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   const uint32_t tiles = (uint32_t)a.batch * (uint32_t)((a.M + BM - 1) / BM) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
   const uint32_t group_m = 16;
-  // Bytes the producer's copies report to a stage's mbarrier: the tensor-map copies count the
-  // packed source bytes (bits/8 per element), not the expanded shared-memory footprint.
+  // Bytes the operand copies report to a stage's mbarrier: the tensor-map copies count the packed
+  // source bytes (bits/8 per element), not the expanded shared-memory footprint.  The scale chunks
+  // complete on a barrier of their own.
   const uint32_t tx_bytes =
       DENSE ? (uint32_t)(BM + BN) * 128u
-            : (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8) + cfg::kSfBytes;
+            : (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8);
   mx_gemm_kernel<BN, DENSE><<<grid, kThreads, cfg::kSmemBytes, a.stream>>>(
       ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
       idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, epi_args(a),
