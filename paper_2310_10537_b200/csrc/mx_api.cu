@@ -544,6 +544,15 @@ static int tile_width_override() {
   return n == 256 || n == 384 ? n : 0;
 }
 
+// Largest M that takes the swapped-operand kernel; MX_GEMM_SKINNY_M=0..128 in the environment
+// overrides it (tuning, tests).
+static int skinny_m_limit() {
+  const char* v = std::getenv("MX_GEMM_SKINNY_M");
+  if (!v) return 96;
+  const int n = std::atoi(v);
+  return n < 0 ? 0 : n > 128 ? 128 : n;
+}
+
 // strict: every matrix must consist of whole 128-row / 128-column tiles (batched products, whose
 // matrices are stacked along rows, and the quantizing epilogue, which writes whole blocks).
 static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB,
@@ -587,6 +596,7 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
   a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16; a.batch = batch;
   a.dense = 0;
   a.force_bn = tile_width_override();
+  a.skinny_m = skinny_m_limit();
   a.q_elems = q_elems; a.q_scales = q_scales; a.q_fmt = q_fmt; a.q_round = q_round;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
@@ -673,7 +683,7 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
   if ((e = mx::launch_dequantize(d)) != cudaSuccess) return fail_cuda(e);
   mx::GemmArgs a;
   a.A = dA; a.sA = nullptr; a.B = dB; a.sB = nullptr; a.C = C; a.c_bf16 = (int)c_dtype == MX_BF16;
-  a.dense = 1; a.batch = 1; a.force_bn = tile_width_override();
+  a.dense = 1; a.batch = 1; a.force_bn = tile_width_override(); a.skinny_m = 0;
   a.q_elems = nullptr; a.q_scales = nullptr; a.q_fmt = 0; a.q_round = 0;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream; a.sm_count = sms;

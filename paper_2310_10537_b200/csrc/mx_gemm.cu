@@ -632,6 +632,228 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
 
 // ============================================================================
+// Few rows of A (M <= 128; a decode step: a handful of activation rows against a weight matrix).
+// The product is bound by reading B once from HBM, and what a CTA can have in flight is bounded by
+// its shared memory, so the operands change places: the tile's 128 rows of B take the M side of
+// the MMA (one TMEM lane per row of B) and the MP = M rounded up to 16 rows of A its N side.  A
+// stage is then 16 KB of B + MP x 128 bytes of A instead of 16 KB + 16 KB, and the ring holds up
+// to twelve of them.  The accumulator is C transposed -- lane = column n of C, column = row m --
+// which the epilogue writes with plain stores: for every m the 32 lanes of a warp store 32
+// consecutive columns.
+// Warps: 0 operand producer, 1 MMA issuer, 2..5 epilogue (one per TMEM lane quarter), 10 scale
+// copier, 11 scale producer; two accumulator stages.
+// ============================================================================
+constexpr uint32_t kSkinnyMaxStages = 12;
+constexpr uint32_t kSkinnyBars = 4 * kSkinnyMaxStages + 4;
+constexpr uint32_t kSkinnySfCol0 = 256;  // accumulators at columns 0 and 128, 8 scale columns per stage behind
+
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
+  asm volatile(
+      "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, "
+      "%12, %13, %14, %15}, [%16];"
+      : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]),
+        "=r"(r[7]), "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]),
+        "=r"(r[14]), "=r"(r[15])
+      : "r"(taddr) : "memory");
+}
+
+__global__ void __launch_bounds__(kThreads, 1)
+mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                      const __grid_constant__ CUtensorMap tmap_sw, const __grid_constant__ CUtensorMap tmap_sx,
+                      void* __restrict__ C, uint32_t M, uint32_t N, uint32_t K, uint32_t MP,
+                      uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t c_bf16) {
+  extern __shared__ uint8_t smem_raw[];
+  const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+  uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
+  const uint32_t x_bytes = MP * 128u;
+  const uint32_t off_x = stages * 16384u;
+  const uint32_t off_sf = off_x + stages * x_bytes;
+  const uint32_t off_bar = off_sf + stages * 1024u;
+  const uint32_t bar0 = smem_base + off_bar;
+  auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
+  auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (kSkinnyMaxStages + s); };
+  auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * kSkinnyMaxStages + s); };
+  auto sf_full_bar = [&](uint32_t s) { return bar0 + 8 * (3 * kSkinnyMaxStages + s); };
+  auto acc_full_bar = [&](uint32_t a) { return bar0 + 8 * (4 * kSkinnyMaxStages + a); };
+  auto acc_empty_bar = [&](uint32_t a) { return bar0 + 8 * (4 * kSkinnyMaxStages + 2 + a); };
+  volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(smem_gen + off_bar + kSkinnyBars * 8);
+  volatile uint32_t* abort_flag = tmem_slot + 1;
+
+  const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t tiles_n = (N + 127u) / 128u;
+  const uint32_t k_chunks = (K + BK - 1) / BK;  // a K tail is zero-filled by the copies
+
+  if (threadIdx.x == 0) {
+    for (uint32_t s = 0; s < stages; ++s) {
+      mbar_init(full_bar(s), 1);
+      mbar_init(empty_bar(s), 1);
+      mbar_init(sf_ready_bar(s), 1);
+      mbar_init(sf_full_bar(s), 1);
+    }
+    for (uint32_t a = 0; a < 2; ++a) {
+      mbar_init(acc_full_bar(a), 1);
+      mbar_init(acc_empty_bar(a), 4);  // one arrival per epilogue warp
+    }
+    *abort_flag = 0;
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_w)) : "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_x)) : "memory");
+  }
+  if (warp == 1) {
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+  }
+  tc_fence_before();
+  __syncthreads();
+  tc_fence_after();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0 || warp == 11) {
+    // ---------------- producers: warp 0 the operand boxes, warp 11 the scale chunks ----------------
+    // lane 0: the tile's 128 rows of B (and their scales), lane 1: all MP rows of A (and theirs).
+    // Rows past N or M are zero-filled by the copy: zero codes, value +0.
+    if (lane < 2) {
+      const bool scales = warp == 11;
+      const CUtensorMap* map = scales ? (lane == 0 ? &tmap_sw : &tmap_sx) : (lane == 0 ? &tmap_w : &tmap_x);
+      const uint32_t dst_off = scales ? off_sf + lane * 512u : (lane == 0 ? 0u : off_x);
+      const uint32_t dst_stride = scales ? 1024u : (lane == 0 ? 16384u : x_bytes);
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+            raise_abort(abort_flag, ST_PRODUCER_WAIT);
+            ok = false;
+          }
+          if (!__all_sync(0x3u, ok)) { ok = false; break; }
+          const uint32_t fb = scales ? sf_full_bar(stage) : full_bar(stage);
+          if (lane == 0) mbar_arrive_expect_tx(fb, scales ? 1024u : tx_bytes);
+          __syncwarp(0x3u);
+          // operands: (k, row, 0); scales: (0, K chunk, 128-row group)
+          const int cx = scales ? 0 : (int)(kc * BK);
+          const int cy = scales ? (int)kc : (lane == 0 ? (int)(t * 128u) : 0);
+          const int cz = scales && lane == 0 ? (int)t : 0;
+          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      if (!ok) {  // let copies that are still in flight land before the CTA goes away
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp == 10) {
+    // ------------------------------ scale copier ------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
+            raise_abort(abort_flag, ST_SCALE_WAIT);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sf_smem = smem_base + off_sf + stage * 1024u;
+          const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+          tc_cp_scales(sf_tmem, scale_desc(sf_smem));            // rows of B: the MMA's A-side scales
+          tc_cp_scales(sf_tmem + 4, scale_desc(sf_smem + 512));  // rows of A: its B-side scales
+          tc_commit(sf_ready_bar(stage));
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------- MMA issuer -------------------------------
+    if (lane == 0) {
+      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+      bool ok = true;
+      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+        if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) {
+          raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t d_tmem = tmem_base + acc * 128u;
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          if (!mbar_wait(sf_ready_bar(stage), phase, abort_flag) ||
+              !mbar_wait(full_bar(stage), phase, abort_flag)) {
+            raise_abort(abort_flag, ST_MMA_WAIT_FULL);
+            ok = false;
+            break;
+          }
+          tc_fence_after();
+          const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+          const uint64_t wdesc = operand_desc(smem_base + stage * 16384u);
+          const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_bytes);
+#pragma unroll
+          for (uint32_t k = 0; k < BK / kMmaK; ++k) {
+            // byte k of each 32-bit scale column belongs to MX block k of this stage
+            const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
+            tc_mma(d_tmem, wdesc + 2 * k, xdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4, (kc | k) != 0 ? 1u : 0u);
+          }
+          tc_commit(empty_bar(stage));
+          if (++stage == stages) { stage = 0; phase ^= 1u; }
+        }
+        if (ok) tc_commit(acc_full_bar(acc));
+        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+      }
+    }
+  } else if (warp >= 2 && warp < 6) {
+    // -------------------------------- epilogue --------------------------------
+    const uint32_t quarter = warp & 3u;  // TMEM lanes this warp may read: 32 * quarter .. + 31
+    uint32_t acc = 0, acc_phase = 0;
+    for (uint32_t t = blockIdx.x; t < tiles_n; t += gridDim.x) {
+      if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) {
+        if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t n = t * 128u + quarter * 32u + lane;  // this thread's column of C
+      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * 128u;
+      for (uint32_t c = 0; c < MP; c += 16) {
+        uint32_t r[16];
+        tc_ld16(taddr + c, r);
+        tc_wait_ld();
+        if (c + 16 >= MP) {  // the accumulator is in registers: hand it back before the stores
+          tc_fence_before();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(acc_empty_bar(acc));
+        }
+        if (n < N) {
+#pragma unroll
+          for (uint32_t j = 0; j < 16; ++j) {
+            const uint32_t m = c + j;
+            if (m < M) {
+              const size_t idx = (size_t)m * N + n;
+              if (c_bf16) {
+                uint16_t h;
+                asm("cvt.rn.bf16.f32 %0, %1;" : "=h"(h) : "f"(__uint_as_float(r[j])));
+                reinterpret_cast<uint16_t*>(C)[idx] = h;
+              } else
+                reinterpret_cast<float*>(C)[idx] = __uint_as_float(r[j]);
+            }
+          }
+        }
+      }
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+    }
+  }
+
+  // common exit: every role falls through to here, also after a wait that gave up
+  tc_fence_before();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after();
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
+                 "r"((uint32_t)kTmemCols) : "memory");
+  }
+}
+
+// ============================================================================
 // Two-CTA variant: a cluster of two CTAs (two SMs) computes one 256 x 256 tile
 // with tcgen05.mma.cta_group::2.  CTA r of the pair stages rows 128r.. of the A
 // tile and rows 128r.. of the B tile, so each SM moves half of B through its
@@ -1287,6 +1509,42 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   return cudaGetLastError();
 }
 
+// M <= 128: operands swapped (see mx_gemm_skinny_kernel).
+cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
+  const uint32_t MP = ((uint32_t)a.M + 15u) / 16u * 16u;
+  CUtensorMap mw, mx_, msw, msx;
+  if (!make_operand_map(fn, &mw, a.B, a.fmtB, (uint64_t)a.N, (uint64_t)a.K, 128) ||
+      !make_operand_map(fn, &mx_, a.A, a.fmtA, (uint64_t)a.M, (uint64_t)a.K, MP) ||
+      !make_scale_map(fn, &msw, a.sB, (uint64_t)a.N, (uint64_t)a.K, 1) ||
+      !make_scale_map(fn, &msx, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1))
+    return cudaErrorInvalidValue;
+  const uint32_t stage_bytes = 16384u + MP * 128u + 1024u;
+  const uint32_t fixed = kSkinnyBars * 8u + 16u + 1024u;  // barriers, TMEM slot + abort flag, alignment slack
+  uint32_t stages = (232448u - fixed) / stage_bytes;
+  if (stages > kSkinnyMaxStages) stages = kSkinnyMaxStages;
+  const uint32_t smem = stages * stage_bytes + fixed;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(mx_gemm_skinny_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, 232448);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint32_t tiles = (uint32_t)((a.N + 127) / 128);
+  const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
+  // bytes the two operand copies report (packed source bytes, rows past the end included)
+  const uint32_t tx_bytes = (uint32_t)(128 * BK * fmt_bits(a.fmtB) / 8) + MP * (uint32_t)(BK * fmt_bits(a.fmtA) / 8);
+  // the MMA's A side is B (format field [7,10)), its B side is A ([10,13)); N field = MP, M = 128
+  const uint32_t idesc = (mma_fmt_code(a.fmtB) << 7) | (mma_fmt_code(a.fmtA) << 10) | (1u << 23) |
+                         ((MP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
+  mx_gemm_skinny_kernel<<<grid, kThreads, smem, a.stream>>>(mw, mx_, msw, msx, a.C, (uint32_t)a.M, (uint32_t)a.N,
+                                                            (uint32_t)a.K, MP, idesc, tx_bytes, stages,
+                                                            a.c_bf16 ? 1u : 0u);
+  return cudaGetLastError();
+}
+
 }  // namespace
 
 int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
@@ -1309,6 +1567,11 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
       *cuda_err = a.dense ? launch_pair<2, 384>(a, fn) : f4 ? launch_pair<1, 384>(a, fn) : launch_pair<0, 384>(a, fn);
     else
       *cuda_err = a.dense ? launch_pair<2, 256>(a, fn) : f4 ? launch_pair<1, 256>(a, fn) : launch_pair<0, 256>(a, fn);
+    return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
+  }
+  // few rows of A: operands swapped, deep ring (see mx_gemm_skinny_kernel)
+  if (!a.dense && a.batch == 1 && a.q_elems == nullptr && a.M <= a.skinny_m) {
+    *cuda_err = launch_skinny(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
   CUtensorMap ma, mb;

@@ -74,6 +74,7 @@ struct GemmArgs {
   int64_t M, N, K;
   int fmtA, fmtB;
   int force_bn;  // 0: let launch_gemm choose the tile width; 256 / 384: pin it (tuning and tests)
+  int skinny_m;  // products with M <= skinny_m (at most 128) take the swapped-operand kernel
   int sm_count;
   cudaStream_t stream;
 };

@@ -82,6 +82,52 @@ def test_scale_identification_exact(fa, fb, N):
     assert (C.cpu().numpy().astype(np.float64) == C64).all()
 
 
+@pytest.mark.parametrize("fa,fb", [(0, 0), (1, 4), (2, 3), (4, 4), (3, 0)])
+@pytest.mark.parametrize("M,N", [(16, 256), (40, 384), (96, 19200)])
+def test_scale_identification_few_rows(fa, fb, M, N):
+    """The same probe for M <= 96, where the kernel swaps the operands' places in the MMA (rows of
+    B on the M side): every (row, K-block) scale of either operand must still meet its own codes.
+    N = 19200 gives 150 tiles, so some CTAs walk a second tile (ring wrap, second accumulator)."""
+    K = 256
+    kb = K // 32
+    rng = np.random.default_rng(fa * 7 + fb + N + M)
+    a_codes = np.full((M, K), ONE[fa], np.uint8)
+    b_codes = np.full((N, K), ONE[fb], np.uint8)
+    sa = (127 + rng.integers(-3, 4, (M, kb))).astype(np.uint8)
+    sb = (127 + rng.integers(-3, 4, (N, kb))).astype(np.uint8)
+    sa_sw, sb_sw = _swizzle_scales(sa), _swizzle_scales(sb)
+    ea, eb = O.pack_codes(a_codes.reshape(-1), fa), O.pack_codes(b_codes.reshape(-1), fb)
+    C = _gemm_guarded(torch.from_numpy(ea).cuda(), torch.from_numpy(sa_sw).cuda(),
+                      torch.from_numpy(eb).cuda(), torch.from_numpy(sb_sw).cuda(), M, N, K, fa, fb)
+    want = 32.0 * (2.0 ** (sa.astype(np.float64) - 127)) @ (2.0 ** (sb.astype(np.float64) - 127)).T
+    assert (C.cpu().numpy().astype(np.float64) == want).all()
+
+
+@pytest.mark.parametrize("fa,fb", [(0, 0), (1, 0), (2, 3), (3, 3), (4, 4), (0, 4), (4, 1)])
+@pytest.mark.parametrize("M,N,K,dt", [(1, 512, 128, torch.float32), (5, 1000, 384, torch.bfloat16),
+                                      (33, 640, 1024, torch.float32), (96, 264, 640, torch.bfloat16)])
+def test_few_rows_against_oracle(M, N, K, fa, fb, dt):
+    """M <= 96 (the swapped-operand kernel), every format pair, both output types, tails in M and N."""
+    g = torch.Generator(device="cuda").manual_seed(M + N + K + 10 * fa + fb)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.05
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(M * N * esz)
+    C = g_out.view.view(dt).view(M, N)
+    if dt == torch.bfloat16:
+        mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    else:
+        mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    c64, s = O.gemm(hea, hsa, heb, hsb, M, N, K, fa, fb)
+    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
+    assert (np.abs(C.double().cpu().numpy() - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+
+
 @pytest.mark.parametrize("fa,fb,K", [(0, 0, 1024), (4, 4, 1024), (4, 4, 768), (2, 4, 512)])
 def test_scale_identification_two_cta_kernels(fa, fb, K):
     """The same exact probe at a shape that selects the two-CTA kernels: E4M3 x E4M3 and FP6 x FP4 on
