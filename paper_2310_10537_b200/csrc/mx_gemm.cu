@@ -132,6 +132,16 @@ __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map
       "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
 }
+// One lane of a converged warp (the pattern the compiler knows for single-thread instructions).
+__device__ __forceinline__ bool elect_one() {
+  uint32_t p;
+  asm volatile(
+      "{\n\t.reg .pred P;\n\t"
+      "elect.sync _|P, 0xffffffff;\n\t"
+      "selp.u32 %0, 1, 0, P;\n\t}"
+      : "=r"(p));
+  return p != 0;
+}
 __device__ __forceinline__ void tc_fence_before() {
   asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory");
 }
@@ -984,9 +994,6 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
   constexpr int BN = cfg::BN;
   constexpr bool WIDE = BN == 384;
-  // operand copies per stage, one producer lane each: A, B, [second part of B]
-  constexpr uint32_t kOperandCopies = 2 + (WIDE ? 1 : 0);
-  constexpr uint32_t kOperandMask = (1u << kOperandCopies) - 1u;
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -1046,59 +1053,59 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
 
   if (warp == 0) {
     // ------------------------- TMA producer (both CTAs) -------------------------
-    // Operand tiles only: the scale chunks have a producer warp of their own (below) -- with all four
-    // copies of a stage issued from here the kernel ran a tenth slower than with two.
-    if (lane < kOperandCopies) {
-      // role of this lane: 0 A, 1 B (rows 128 rank .. of the tile), 2 second part of B (wide tile:
-      // rows 256 + 64 rank ..)
-      const uint32_t role = lane;
-      const CUtensorMap* map = role == 0 ? &tmap_a : role == 1 ? &tmap_b : &tmap_b2;
-      const uint32_t dst_off = role == 0 ? cfg::kOffA : role == 1 ? cfg::kOffB : cfg::kOffB + 128u * 128u;
-      const uint32_t dst_stride = role == 0 ? cfg::kABytes : cfg::kBBytes;
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        // this CTA's 128 rows of A and its rows of B (B rows may lie past N on a ragged tile: zero
-        // fill or the next matrix of a batch; their columns are not stored)
-        const int cy = role == 0 ? (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128)
-                       : role == 1 ? (int)(tc.b * N + tc.tn * BN + rank * 128)
-                                   : (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
-            raise_abort(abort_flag, ST_PRODUCER_WAIT);
-            ok = false;
-          }
-          if (!__all_sync(kOperandMask, ok)) { ok = false; break; }
-          const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
-          if (rank == 0 && lane == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
-          __syncwarp(kOperandMask);
-          tma_load_3d_pair(smem_base + dst_off + stage * dst_stride, map, (int)(kc * BKe), cy, 0, fb);
-          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+    // Operand tiles only: the scale chunks have a producer warp of their own (below).  The whole
+    // warp runs the loop converged and one elected lane issues the copies (see elect_one).
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+      const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+      // this CTA's 128 rows of A and its rows of B: rows 128 rank .. of the tile and, for the wide
+      // tile, rows 256 + 64 rank .. (B rows may lie past N on a ragged tile: zero fill or the next
+      // matrix of a batch; their columns are not stored)
+      const int cy_a = (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128);
+      const int cy_b = (int)(tc.b * N + tc.tn * BN + rank * 128);
+      const int cy_b2 = (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_PRODUCER_WAIT);
+          break;
         }
+        if (elect_one()) {
+          const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
+          const int cx = (int)(kc * BKe);
+          tma_load_3d_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, cx, cy_a, 0, fb);
+          tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, cx, cy_b, 0, fb);
+          if (WIDE)
+            tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u, &tmap_b2, cx, cy_b2, 0, fb);
+        }
+        __syncwarp();
+        if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
       }
-      if (!ok) {
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) {}
-      }
+    }
+    if (!ok) {  // let copies that are still in flight land before the CTA goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000LL) {}
     }
   } else if (warp == 1) {
     // --------------------------- MMA issuer (leader) ---------------------------
-    if (lane == 0 && rank == 0) {
+    // the warp runs converged; one elected lane issues a stage's MMAs and the commit
+    if (rank == 0) {
       uint32_t stage = 0, phase = 0, acc_phase = 0;
       bool ok = true;
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-        if (!mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag)) {
+        if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag))) {
           raise_abort(abort_flag, ST_MMA_WAIT_ACC);
           break;
         }
         tc_fence_after();
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          // scales in tensor memory (which implies that the stage has landed), then the operands
-          if ((!DENSE && !mbar_wait(sf_ready_bar(stage), phase, abort_flag)) ||
-              !mbar_wait(full_bar(stage), phase, abort_flag)) {
+          // scales in tensor memory, then the operands
+          ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag)) &&
+                                           mbar_wait(full_bar(stage), phase, abort_flag));
+          if (!ok) {
             raise_abort(abort_flag, ST_MMA_WAIT_FULL);
-            ok = false;
             break;
           }
           tc_fence_after();
@@ -1110,6 +1117,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint64_t bdesc2 = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u);
           const uint32_t idesc2_base = (idesc_base & ~(0x3Fu << 17)) | ((uint32_t)(128 >> 3) << 17);
           constexpr uint32_t kSfbStep = 4 * cfg::kSfbGroups;  // B scale columns per K chunk
+          if (elect_one()) {
 #pragma unroll
           for (uint32_t k = 0; k < 4; ++k) {  // every MMA advances 32 bytes along the 128-byte rows
             const uint32_t acc_flag = (kc | k) != 0 ? 1u : 0u;
@@ -1135,23 +1143,26 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             }
           }
           tc_commit_pair(empty_bar(stage));
+          }
+          __syncwarp();
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit_pair(acc_full_bar);
+        if (ok && elect_one()) tc_commit_pair(acc_full_bar);
+        __syncwarp();
         acc_phase ^= 1u;
       }
     }
   } else if (warp == 10) {
     // --------------------------- scale copier (leader) ---------------------------
     if constexpr (!DENSE) {
-      if (lane == 0 && rank == 0) {
+      if (rank == 0) {
         uint32_t stage = 0, phase = 0;
         bool ok = true;
         for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
           for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-            if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
+            ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+            if (!ok) {
               raise_abort(abort_flag, ST_SCALE_WAIT);
-              ok = false;
               break;
             }
             tc_fence_after();
@@ -1160,15 +1171,18 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             // Each CTA copies from its own shared memory to its own tensor memory.  A: K chunk c at
             // columns 4c.  B: the box is [row group][K chunk], and the MMA wants the columns of one
             // K chunk together: group g of G, chunk c -> 4 G c + 4g.
+            if (elect_one()) {
 #pragma unroll
-            for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
-              tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
+              for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
+                tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
 #pragma unroll
-              for (uint32_t g = 0; g < cfg::kSfbGroups; ++g)
-                tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 4 * cfg::kSfbGroups * c + 4 * g,
-                                  scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+                for (uint32_t g = 0; g < cfg::kSfbGroups; ++g)
+                  tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 4 * cfg::kSfbGroups * c + 4 * g,
+                                    scale_desc(sf_smem + cfg::kSfABytes + 512 * (g * cfg::kKChunks + c)));
+              }
+              tc_commit_leader(sf_ready_bar(stage));  // arrives when the copies have completed in both CTAs
             }
-            tc_commit_leader(sf_ready_bar(stage));  // arrives when the copies have completed in both CTAs
+            __syncwarp();
             if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
           }
         }
@@ -1176,36 +1190,36 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     }
   } else if (warp == 11) {
     // ------------------------ scale producer (both CTAs) ------------------------
-    // lane 0: this CTA's A scales, lane 1: the B scales of all BN columns; both complete on the
-    // leader's per-stage "scales landed" barrier, which the leader's lane 0 arms.  A stage's scale
-    // buffer and scale columns are free when the stage is (the MMAs that read them have completed).
+    // This CTA's A scales and the B scales of all BN columns; both copies complete on the leader's
+    // per-stage "scales landed" barrier, which the leader arms.  A stage's scale buffer and scale
+    // columns are free when the stage is (the MMAs that read them have completed).
     if constexpr (!DENSE) {
-      if (lane < 2) {
-        const CUtensorMap* map = lane == 0 ? &tmap_sa : &tmap_sb;
-        const uint32_t dst_off = lane == 0 ? cfg::kOffSf : cfg::kOffSf + cfg::kSfABytes;
-        uint32_t stage = 0, phase = 0;
-        bool ok = true;
-        for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-          const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-          const int cz = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * 2 + rank)
-                                   : (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups);
-          for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-            if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
-              raise_abort(abort_flag, ST_PRODUCER_WAIT);
-              ok = false;
-            }
-            if (!__all_sync(0x3u, ok)) { ok = false; break; }
-            if (rank == 0 && lane == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * cfg::kSfBytes);
-            __syncwarp(0x3u);
-            tma_load_3d_pair(smem_base + dst_off + stage * cfg::kSfBytes, map, 0, (int)(kc * cfg::kKChunks), cz,
-                             sf_full_bar(stage) & kPeerMask);
-            if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+      uint32_t stage = 0, phase = 0;
+      bool ok = true;
+      for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        const int cz_a = (int)((tc.b * tiles_m + tc.tm) * 2 + rank);
+        const int cz_b = (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups);
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+          if (!ok) {
+            raise_abort(abort_flag, ST_PRODUCER_WAIT);
+            break;
           }
+          if (elect_one()) {
+            const uint32_t fb = sf_full_bar(stage) & kPeerMask;
+            if (rank == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * cfg::kSfBytes);
+            const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+            tma_load_3d_pair(dst, &tmap_sa, 0, (int)(kc * cfg::kKChunks), cz_a, fb);
+            tma_load_3d_pair(dst + cfg::kSfABytes, &tmap_sb, 0, (int)(kc * cfg::kKChunks), cz_b, fb);
+          }
+          __syncwarp();
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (!ok) {
-          const long long t0 = clock64();
-          while (clock64() - t0 < 2000000LL) {}
-        }
+      }
+      if (!ok) {
+        const long long t0 = clock64();
+        while (clock64() - t0 < 2000000LL) {}
       }
     }
   } else {
