@@ -122,10 +122,11 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
     }
   }
 }
-// Every copy of a stage (A tile, B tile, A scales, B scales) goes through a rank-3 tensor map, so
-// that lanes 0..3 of the producer warp can issue all four with ONE warp instruction, each lane
-// with its own map, coordinates and destination: issuing them one after the other from a single
-// thread costs more than the 512 clocks a stage's MMAs take.
+// Every copy of a stage (A tile, B tile, A scales, B scales) goes through a rank-3 tensor map.
+// The warps that issue copies, tcgen05.cp, tcgen05.mma and tcgen05.commit run their loops converged
+// and issue from the lane elect_one() picks: issued from inside a `lane == 0` branch each of
+// these instructions cost its thread 58-69 clocks (their operands are uniform registers, which
+// divergent code has to fill per instruction), and the MMA thread could not keep the tensor pipe fed.
 __device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, int x, int y, int z,
                                             uint32_t bar) {
   asm volatile(
@@ -460,64 +461,63 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------
-    // lanes 0 and 1 issue the two operand copies of a stage together (see tma_load_3d); the scale
-    // chunks have a producer warp of their own (warp 11)
-    if (lane < 2) {
-      const CUtensorMap* map = lane == 0 ? &tmap_a : &tmap_b;
-      const uint32_t dst_off = lane == 0 ? cfg::kOffA : cfg::kOffB;
-      const uint32_t dst_stride = lane == 0 ? cfg::kABytes : cfg::kBBytes;
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        // (k, row, 0), rows counted through the whole batch.  Rows past the end of a B matrix on a
-        // ragged last tile belong to the next matrix of the batch or are zero-filled by the copy;
-        // their columns are not stored.
-        const int cy = lane == 0 ? (int)((tc.b * tiles_m + tc.tm) * BM) : (int)(tc.b * N + tc.tn * BN);
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
-            raise_abort(abort_flag, ST_PRODUCER_WAIT);
-            ok = false;
-          }
-          if (!__all_sync(0x3u, ok)) { ok = false; break; }
-          const uint32_t fb = full_bar(stage);
-          if (lane == 0) mbar_arrive_expect_tx(fb, tx_bytes);
-          __syncwarp(0x3u);
-          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, (int)(kc * BKe), cy, 0, fb);
-          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+    // The two operand copies of a stage; the scale chunks have a producer warp of their own (warp
+    // 11).  The whole warp runs the loop converged and one elected lane issues (see elect_one).
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+      // (k, row, 0), rows counted through the whole batch.  Rows past the end of a B matrix on a
+      // ragged last tile belong to the next matrix of the batch or are zero-filled by the copy;
+      // their columns are not stored.
+      const int cy_a = (int)((tc.b * tiles_m + tc.tm) * BM), cy_b = (int)(tc.b * N + tc.tn * BN);
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_PRODUCER_WAIT);
+          break;
         }
+        if (elect_one()) {
+          const uint32_t fb = full_bar(stage);
+          mbar_arrive_expect_tx(fb, tx_bytes);
+          tma_load_3d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BKe), cy_a, 0, fb);
+          tma_load_3d(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, (int)(kc * BKe), cy_b, 0, fb);
+        }
+        __syncwarp();
+        if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
       }
-      if (!ok) {  // let copies that are still in flight land before the CTA goes away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) {}
-      }
+    }
+    if (!ok) {  // let copies that are still in flight land before the CTA goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000LL) {}
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
-      bool ok = true;
-      for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-        if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) {
-          raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+    // the warp runs converged; one elected lane issues a stage's MMAs and the commit
+    uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag))) {
+        raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + acc * BN;
+      // scales of row n of the tile sit in column (n0 % 128 + n) / 32 of the copied chunks
+      const uint32_t sfb_col = 4 + ((tile_coord(t, tiles_m, tiles_n, group_m).tn * BN) % 128) / 32;
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        // scales in tensor memory, then the operands
+        ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag)) &&
+                                         mbar_wait(full_bar(stage), phase, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_MMA_WAIT_FULL);
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * BN;
-        // scales of row n of the tile sit in column (n0 % 128 + n) / 32 of the copied chunks
-        const uint32_t sfb_col = 4 + ((tile_coord(t, tiles_m, tiles_n, group_m).tn * BN) % 128) / 32;
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          // scales in tensor memory (which implies that the stage has landed), then the operands
-          if ((!DENSE && !mbar_wait(sf_ready_bar(stage), phase, abort_flag)) ||
-              !mbar_wait(full_bar(stage), phase, abort_flag)) {
-            raise_abort(abort_flag, ST_MMA_WAIT_FULL);
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
-          const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
+        const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
+        const uint64_t adesc = operand_desc(smem_base + cfg::kOffA + stage * cfg::kABytes);
+        const uint64_t bdesc = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes);
+        if (elect_one()) {
 #pragma unroll
           for (uint32_t k = 0; k < BK / kMmaK; ++k) {
             // byte k of each 32-bit scale column belongs to MX block k of this stage
@@ -530,59 +530,66 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
             }
           }
           tc_commit(empty_bar(stage));  // the stage is free once these MMAs have read it
-          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit(acc_full_bar(acc));
-        if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
+        __syncwarp();
+        if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
       }
+      if (ok && elect_one()) tc_commit(acc_full_bar(acc));
+      __syncwarp();
+      if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
   } else if (warp == 10) {
     // ------------------------------ scale copier ------------------------------
-    if (!DENSE && lane == 0) {
+    if constexpr (!DENSE) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
+          ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+          if (!ok) {
             raise_abort(abort_flag, ST_SCALE_WAIT);
-            ok = false;
             break;
           }
           tc_fence_after();
           const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
-          tc_cp_scales(sf_tmem, scale_desc(sf_smem));
+          if (elect_one()) {
+            tc_cp_scales(sf_tmem, scale_desc(sf_smem));
 #pragma unroll
-          for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
-            tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
-          tc_commit(sf_ready_bar(stage));  // arrives when the copies above have completed
+            for (uint32_t j = 0; j < cfg::kSfbChunks; ++j)
+              tc_cp_scales(sf_tmem + 4 + 4 * j, scale_desc(sf_smem + 512 + 512 * j));
+            tc_commit(sf_ready_bar(stage));  // arrives when the copies above have completed
+          }
+          __syncwarp();
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
     }
   } else if (warp == 11) {
     // ----------------------------- scale producer -----------------------------
-    // lane 0: the A scales of the tile's 128 rows, lane 1: the B scales of its BN columns -- (0, K
-    // chunk, 128-row group), groups counted through the whole batch; both complete on the per-stage
-    // "scales landed" barrier.  A stage's scale buffer and scale columns are free when the stage is.
-    if (!DENSE && lane < 2) {
-      const CUtensorMap* map = lane == 0 ? &tmap_sa : &tmap_sb;
-      const uint32_t dst_off = lane == 0 ? cfg::kOffSf : cfg::kOffSf + 512u;
+    // The A scales of the tile's 128 rows and the B scales of its BN columns -- (0, K chunk, 128-row
+    // group), groups counted through the whole batch; both complete on the per-stage "scales
+    // landed" barrier.  A stage's scale buffer and scale columns are free when the stage is.
+    if constexpr (!DENSE) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-        const int cz = lane == 0 ? (int)(tc.b * tiles_m + tc.tm) : (int)((tc.b * N + tc.tn * BN) / 128);
+        const int cz_a = (int)(tc.b * tiles_m + tc.tm), cz_b = (int)((tc.b * N + tc.tn * BN) / 128);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+          if (!ok) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
-            ok = false;
+            break;
           }
-          if (!__all_sync(0x3u, ok)) { ok = false; break; }
-          const uint32_t fb = sf_full_bar(stage);
-          if (lane == 0) mbar_arrive_expect_tx(fb, cfg::kSfBytes);
-          __syncwarp(0x3u);
-          tma_load_3d(smem_base + dst_off + stage * cfg::kSfBytes, map, 0, (int)kc, cz, fb);
+          if (elect_one()) {
+            const uint32_t fb = sf_full_bar(stage);
+            mbar_arrive_expect_tx(fb, cfg::kSfBytes);
+            const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+            tma_load_3d(dst, &tmap_sa, 0, (int)kc, cz_a, fb);
+            tma_load_3d(dst + 512u, &tmap_sb, 0, (int)kc, cz_b, fb);
+          }
+          __syncwarp();
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
@@ -722,83 +729,85 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
 
   if (warp == 0 || warp == 11) {
     // ---------------- producers: warp 0 the operand boxes, warp 11 the scale chunks ----------------
-    // lane 0: the tile's 128 rows of B (and their scales), lane 1: all MP rows of A (and theirs).
-    // Rows past N or M are zero-filled by the copy: zero codes, value +0.
-    if (lane < 2) {
-      const bool scales = warp == 11;
-      const CUtensorMap* map = scales ? (lane == 0 ? &tmap_sw : &tmap_sx) : (lane == 0 ? &tmap_w : &tmap_x);
-      const uint32_t dst_off = scales ? off_sf + lane * 512u : (lane == 0 ? 0u : off_x);
-      const uint32_t dst_stride = scales ? 1024u : (lane == 0 ? 16384u : x_bytes);
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag)) {
-            raise_abort(abort_flag, ST_PRODUCER_WAIT);
-            ok = false;
-          }
-          if (!__all_sync(0x3u, ok)) { ok = false; break; }
-          const uint32_t fb = scales ? sf_full_bar(stage) : full_bar(stage);
-          if (lane == 0) mbar_arrive_expect_tx(fb, scales ? 1024u : tx_bytes);
-          __syncwarp(0x3u);
-          // operands: (k, row, 0); scales: (0, K chunk, 128-row group)
-          const int cx = scales ? 0 : (int)(kc * BK);
-          const int cy = scales ? (int)kc : (lane == 0 ? (int)(t * 128u) : 0);
-          const int cz = scales && lane == 0 ? (int)t : 0;
-          tma_load_3d(smem_base + dst_off + stage * dst_stride, map, cx, cy, cz, fb);
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
+    // The tile's 128 rows of B and all MP rows of A (or their scale chunks).  Rows past N or M are
+    // zero-filled by the copy: zero codes, value +0.  The warp runs converged, one elected lane issues.
+    const bool scales = warp == 11;
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_PRODUCER_WAIT);
+          break;
         }
+        if (elect_one()) {
+          if (scales) {  // (0, K chunk, 128-row group)
+            const uint32_t fb = sf_full_bar(stage);
+            mbar_arrive_expect_tx(fb, 1024u);
+            tma_load_3d(smem_base + off_sf + stage * 1024u, &tmap_sw, 0, (int)kc, (int)t, fb);
+            tma_load_3d(smem_base + off_sf + stage * 1024u + 512u, &tmap_sx, 0, (int)kc, 0, fb);
+          } else {  // (k, row, 0)
+            const uint32_t fb = full_bar(stage);
+            mbar_arrive_expect_tx(fb, tx_bytes);
+            tma_load_3d(smem_base + stage * 16384u, &tmap_w, (int)(kc * BK), (int)(t * 128u), 0, fb);
+            tma_load_3d(smem_base + off_x + stage * x_bytes, &tmap_x, (int)(kc * BK), 0, 0, fb);
+          }
+        }
+        __syncwarp();
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
-      if (!ok) {  // let copies that are still in flight land before the CTA goes away
-        const long long t0 = clock64();
-        while (clock64() - t0 < 2000000LL) {}
-      }
+    }
+    if (!ok) {  // let copies that are still in flight land before the CTA goes away
+      const long long t0 = clock64();
+      while (clock64() - t0 < 2000000LL) {}
     }
   } else if (warp == 10) {
     // ------------------------------ scale copier ------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0;
-      bool ok = true;
-      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(sf_full_bar(stage), phase, abort_flag)) {
-            raise_abort(abort_flag, ST_SCALE_WAIT);
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t sf_smem = smem_base + off_sf + stage * 1024u;
-          const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+    uint32_t stage = 0, phase = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_SCALE_WAIT);
+          break;
+        }
+        tc_fence_after();
+        const uint32_t sf_smem = smem_base + off_sf + stage * 1024u;
+        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+        if (elect_one()) {
           tc_cp_scales(sf_tmem, scale_desc(sf_smem));            // rows of B: the MMA's A-side scales
           tc_cp_scales(sf_tmem + 4, scale_desc(sf_smem + 512));  // rows of A: its B-side scales
           tc_commit(sf_ready_bar(stage));
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
+        __syncwarp();
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
     }
   } else if (warp == 1) {
     // ------------------------------- MMA issuer -------------------------------
-    if (lane == 0) {
-      uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
-      bool ok = true;
-      for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
-        if (!mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag)) {
-          raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+    uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+    bool ok = true;
+    for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag))) {
+        raise_abort(abort_flag, ST_MMA_WAIT_ACC);
+        break;
+      }
+      tc_fence_after();
+      const uint32_t d_tmem = tmem_base + acc * 128u;
+      for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        ok = __all_sync(0xffffffffu, mbar_wait(sf_ready_bar(stage), phase, abort_flag) &&
+                                         mbar_wait(full_bar(stage), phase, abort_flag));
+        if (!ok) {
+          raise_abort(abort_flag, ST_MMA_WAIT_FULL);
           break;
         }
         tc_fence_after();
-        const uint32_t d_tmem = tmem_base + acc * 128u;
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          if (!mbar_wait(sf_ready_bar(stage), phase, abort_flag) ||
-              !mbar_wait(full_bar(stage), phase, abort_flag)) {
-            raise_abort(abort_flag, ST_MMA_WAIT_FULL);
-            ok = false;
-            break;
-          }
-          tc_fence_after();
-          const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
-          const uint64_t wdesc = operand_desc(smem_base + stage * 16384u);
-          const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_bytes);
+        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+        const uint64_t wdesc = operand_desc(smem_base + stage * 16384u);
+        const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_bytes);
+        if (elect_one()) {
 #pragma unroll
           for (uint32_t k = 0; k < BK / kMmaK; ++k) {
             // byte k of each 32-bit scale column belongs to MX block k of this stage
@@ -806,11 +815,13 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
             tc_mma(d_tmem, wdesc + 2 * k, xdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4, (kc | k) != 0 ? 1u : 0u);
           }
           tc_commit(empty_bar(stage));
-          if (++stage == stages) { stage = 0; phase ^= 1u; }
         }
-        if (ok) tc_commit(acc_full_bar(acc));
-        if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
+        __syncwarp();
+        if (++stage == stages) { stage = 0; phase ^= 1u; }
       }
+      if (ok && elect_one()) tc_commit(acc_full_bar(acc));
+      __syncwarp();
+      if (++acc == 2) { acc = 0; acc_phase ^= 1u; }
     }
   } else if (warp >= 2 && warp < 6) {
     // -------------------------------- epilogue --------------------------------
