@@ -74,52 +74,73 @@ def job_throughput(units_per_rank: float, world: int, slowest_seconds: float) ->
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    """Samples SM clock, power and throttle reasons of one GPU with nvidia-smi (a process of its
+    own, started well before the timed region so that it is already polling) while the timed region
+    runs.  Every sample carries nvidia-smi's timestamp; the caller marks the timed region with
+    begin() / end(), both right after a device synchronize, and the samples inside that window are
+    the ones reported.  If the window caught none (a very short run), the samples taken under load
+    -- power above half of the maximum seen -- stand in, and the result says so."""
 
-    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+    FIELDS = ("timestamp,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
 
     def __init__(self, gpu_index: int):
         self.proc = None
+        self.t0 = self.t1 = None
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", "-i", str(gpu_index), f"--query-gpu={self.FIELDS}",
-                 "--format=csv,noheader,nounits", "-lms", "20"],
+                 "--format=csv,noheader,nounits", "-lms", "10"],
                 stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
 
+    def begin(self):
+        self.t0 = time.time()
+
+    def end(self):
+        self.t1 = time.time()
+
+    @staticmethod
+    def _epoch(stamp: str):
+        import datetime
+        try:
+            return datetime.datetime.strptime(stamp, "%Y/%m/%d %H:%M:%S.%f").timestamp()
+        except ValueError:
+            return None
+
     def stop(self):
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        time.sleep(0.25)
+        time.sleep(0.05)
         self.proc.terminate()
         try:
             out, _ = self.proc.communicate(timeout=5)
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx_, power, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        samples = []  # (epoch or None, sm, max sm, power, reasons)
         for line in out.strip().splitlines():
             parts = [p.strip() for p in line.split(",")]
-            if len(parts) < 7:
+            if len(parts) < 8:
                 continue
             try:
-                sm.append(float(parts[0]))
-                mx_.append(float(parts[1]))
-                power.append(float(parts[2]))
+                sm, mx_, power = float(parts[1]), float(parts[2]), float(parts[3])
             except ValueError:
                 continue
-            for n, v in zip(names, parts[3:7]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        if not sm:
+            samples.append((self._epoch(parts[0]), sm, mx_, power,
+                            {n for n, v in zip(names, parts[4:8]) if v.lower().startswith("active")}))
+        if not samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        busy = [s for s, p in zip(sm, power) if p > 0.5 * max(power)] or sm
-        return {"sm_mhz": statistics.median(busy), "sm_max_mhz": max(mx_), "samples": len(sm),
-                "power_w_max": max(power), "reasons": sorted(reasons)}
+        inside = [x for x in samples
+                  if x[0] is not None and self.t0 is not None and self.t0 <= x[0] <= self.t1]
+        pmax = max(x[3] for x in samples)
+        use = inside or [x for x in samples if x[3] > 0.5 * pmax] or samples
+        return {"sm_mhz": statistics.median(x[1] for x in use), "sm_max_mhz": max(x[2] for x in samples),
+                "samples": len(use), "in_timed_region": bool(inside),
+                "power_w_max": max(x[3] for x in use), "reasons": sorted(set().union(*[x[4] for x in use]))}
 
 
 # --------------------------------------------------------------------------------------
@@ -526,6 +547,7 @@ def main_ours(args, rank, world, local_rank):
         import torch.distributed as dist
         dist.init_process_group("nccl", device_id=dev)
     peaks = measured_peaks()
+    sampler = ClockSampler(local_rank) if rank == 0 else None  # polling by the time the timed region starts
     w = Workload(torch, mx, inputs, dev, seed_offset=rank)
 
     def barrier():
@@ -537,16 +559,19 @@ def main_ours(args, rank, world, local_rank):
     for _ in range(max(args.warmup, 3)):
         w.step()
     barrier()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
     evs = [[torch.cuda.Event(enable_timing=True) for _ in range(8)] for _ in range(args.steps)]
     t_begin = torch.cuda.Event(enable_timing=True)
     t_end = torch.cuda.Event(enable_timing=True)
     barrier()
+    if sampler:
+        sampler.begin()
     t_begin.record()
     for i in range(args.steps):
         w.step(evs[i])
     t_end.record()
     barrier()
+    if sampler:
+        sampler.end()
     clocks = sampler.stop() if sampler else None
 
     def phase(a, b):
