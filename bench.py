@@ -314,6 +314,28 @@ def run_extras(torch, mx, inputs):
         "ms_gemm_fp32_then_quantize_e4m3": t2 * 1e3, "ms_gemm_with_quantizing_epilogue": t1 * 1e3,
         "quantizing_epilogue_TFLOPs": 2.0 * M * N * K / t1 / 1e12,
         "ms_gemm_bf16_out": tb * 1e3, "bf16_out_TFLOPs": 2.0 * M * N * K / tb / 1e12}
+    # Reference point, not part of the path: the vendor library's MXFP8 GEMM (torch._scaled_mm) on the
+    # very same packed operands and swizzled scales, timed in alternation with mx_gemm_bf16.
+    try:
+        a8 = ea.view(torch.float8_e4m3fn).view(M, K)
+        b8 = eb.view(torch.float8_e4m3fn).view(N, K)
+        s_a, s_b = sa.view(torch.float8_e8m0fnu), sb.view(torch.float8_e8m0fnu)
+        ref = torch._scaled_mm(a8, b8.t(), scale_a=s_a, scale_b=s_b, out_dtype=torch.bfloat16)
+        mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=Cb)
+        same = bool(torch.equal(ref, Cb))
+        del ref
+        t_ours, t_lib = [], []
+        for _ in range(4):
+            t_ours.append(timed(lambda: mx.mx_gemm_bf16(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=Cb), 4))
+            t_lib.append(timed(lambda: torch._scaled_mm(a8, b8.t(), scale_a=s_a, scale_b=s_b,
+                                                        out_dtype=torch.bfloat16), 4))
+        out["config3_vendor_library_reference_bf16_out"] = {
+            "mx_gemm_bf16_TFLOPs": 2.0 * M * N * K / statistics.median(t_ours) / 1e12,
+            "torch_scaled_mm_TFLOPs": 2.0 * M * N * K / statistics.median(t_lib) / 1e12,
+            "outputs_bit_identical": same}
+        del a8, b8, s_a, s_b
+    except Exception as e:  # a torch build without block-scaled _scaled_mm: no reference point
+        out["config3_vendor_library_reference_bf16_out"] = {"unavailable": str(e)[:120]}
     # MXINT8 x MXINT8 on the same shape: dequantize to BF16 + dense BF16 tensor-core GEMM
     ea8, sa8 = mx.mx_quantize(X, 1, mx.MX_INT8)
     eb8, sb8 = mx.mx_quantize(W, 0, mx.MX_INT8)
