@@ -216,8 +216,8 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out,
  * the way out; the scale tensors are the padded SWIZZLED tensors mx_quantize writes
  * (padding bytes 0).  A, B 32-byte aligned, sA, sB, C 16-byte aligned.  MX_INT8 operands: MX_ERR_UNSUPPORTED
  * (the block-scaled tensor-core instruction has no integer element type; use
- * mx_gemm_dense).  The result does not depend on which kernel a shape takes (256- or
- * 128-row tiles, or, for M <= 96, the kernel that puts B on the M side of the MMA).
+ * mx_gemm_dense).  Products with M <= 96 take a kernel that puts B on the M side of the
+ * MMA; its results are bit-identical to the tiled kernels'.
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE, MX_ERR_FMT, MX_ERR_ALIGN,
  * MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT (only with
  * opts->check_status).

@@ -128,6 +128,23 @@ def test_few_rows_against_oracle(M, N, K, fa, fb, dt):
     assert (np.abs(C.double().cpu().numpy() - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
 
 
+@pytest.mark.parametrize("M,N,K,fa,fb", [(64, 1024, 512, 0, 0), (17, 19200, 256, 4, 1), (96, 640, 1024, 2, 3)])
+def test_few_rows_kernel_equals_tiled_kernel(M, N, K, fa, fb, monkeypatch):
+    """The same product through the swapped-operand kernel and (threshold pinned to 0 through the
+    environment) through the 128-row tiles: bit-identical outputs."""
+    g = torch.Generator(device="cuda").manual_seed(M * N + K)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda")
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    C1 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
+    monkeypatch.setenv("MX_GEMM_SKINNY_M", "0")
+    C2 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
+    torch.cuda.synchronize()
+    assert torch.equal(C1, C2)
+    assert C1.abs().max().item() > 0
+
+
 @pytest.mark.parametrize("fa,fb,K", [(0, 0, 1024), (4, 4, 1024), (4, 4, 768), (2, 4, 512)])
 def test_scale_identification_two_cta_kernels(fa, fb, K):
     """The same exact probe at a shape that selects the two-CTA kernels: E4M3 x E4M3 and FP6 x FP4 on
