@@ -8,20 +8,21 @@
 // per row of B -- exactly one MX block (k = 32) deep -- accumulating in FP32 in
 // tensor memory.
 //
-// Kernel structure (one CTA per SM, persistent over output tiles):
-//   warp 0    TMA producer: packed A / B tiles (the sub-byte tensor-map types
-//             expand FP6 / FP4 to one byte per element on the way in) and the
-//             512-byte swizzled scale chunks -> shared-memory ring
-//   warp 1    MMA issuer: four MMAs per stage, tcgen05.commit releases the stage /
-//             publishes the accumulator
-//   warps 2-9 epilogue: tensor memory -> registers (the accumulator is released as soon as
-//             it is in registers) -> FP32 or BF16 C through shared memory and TMA stores, or the
-//             quantizing epilogue (C as an MX tensor), overlapping the next tile's MMAs
+// Kernel structure (one CTA per SM, persistent over output tiles; three kernels: 128-row tiles,
+// 256-row tiles on CTA pairs, and swapped operands for few rows of A):
+//   warp 0    operand producer: packed A / B tiles by TMA (the sub-byte tensor-map types expand
+//             FP6 / FP4 to one byte per element on the way in) -> shared-memory ring
+//   warp 11   scale producer: the stage's 512-byte swizzled scale chunks -> shared memory, on a
+//             barrier of their own
 //   warp 10   scale copier: a stage's scale chunks shared -> tensor memory (tcgen05.cp), then
-//             tcgen05.commit tells the MMA issuer.  Every tcgen05 instruction costs its issuing
-//             thread 60-70 clocks; with the three copies of a stage in the MMA thread's stream
-//             (eight instructions, ~620 clocks per stage) that thread, not the tensor pipe
-//             (520 clocks per stage), set the pace.
+//             tcgen05.commit tells the MMA issuer
+//   warp 1    MMA issuer: four MMAs per stage, tcgen05.commit releases the stage / publishes the
+//             accumulator
+//   warps 2-9 epilogue: tensor memory -> registers (the accumulator is released as soon as it is
+//             in registers) -> FP32 or BF16 C through shared memory and TMA stores, or the
+//             quantizing epilogue (C as an MX tensor), overlapping the next tile's MMAs
+// The four issuing warps run their loops converged -- all lanes wait on the barriers -- and issue
+// from the lane elect.sync picks (see elect_one).
 // Every wait on an mbarrier is bounded; on expiry the kernel records a status
 // word, raises a CTA-wide abort flag and every role falls through to the common
 // exit, where tensor memory is released.
