@@ -1597,8 +1597,11 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
   const int64_t tiles256 = a.batch * ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
-  // two-CTA kernel: needs whole 256-row tiles and enough of them to occupy the SM pairs
-  if (a.M % 256 == 0 && a.batch * (a.M / 256) * ((a.N + 255) / 256) >= a.sm_count / 2) {
+  // two-CTA kernel: needs whole 256-row tiles, and pays as soon as the same problem cut into
+  // 128 x 128 tiles would need more than one wave of the SMs (a 128 x 128 tile, bound by operand
+  // delivery, takes 0.8 of the time of a pair's 256 x 256 tile: 512 x 4096 x 4096, 32 pair tiles or
+  // 128 single ones, 0.73 against 0.88 PFLOP/s; 768 x 4096 x 4096, 48 or 192, 1.09 against 0.87)
+  if (a.M % 256 == 0 && 4 * a.batch * (a.M / 256) * ((a.N + 255) / 256) > a.sm_count) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
     const bool f4 = !a.dense && a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
     // 256 x 384 tiles pull fewer operand bytes per MAC from L2; taken only when pinned
