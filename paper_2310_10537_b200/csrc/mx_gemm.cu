@@ -1043,7 +1043,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const uint32_t tiles_m = M / 256, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
+  const uint32_t tiles_m = (M + 255) / 256, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
   const uint32_t k_chunks = (K + BKe - 1) / BKe;  // a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
@@ -1270,7 +1270,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t cofs = half * kHalf + pass * kPass;
           const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + cofs;
           const uint32_t col0 = tc.tn * BN + cofs;
-          const uint32_t valid_cols = col0 < N ? min(kPass, N - col0) : 0u;
+          // nothing to store for a warp whose rows or columns lie past the matrix
+          const uint32_t valid_cols = (col0 < N && row0 < batch * M) ? min(kPass, N - col0) : 0u;
           uint32_t r[kPassLoads][32];
 #pragma unroll
           for (uint32_t j = 0; j < kPassLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
@@ -1286,7 +1287,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       } else {
         const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + half * kHalf;
         const uint32_t col0 = tc.tn * BN + half * kHalf;
-        const uint32_t valid_cols = col0 < N ? min(kHalf, N - col0) : 0u;
+        // nothing to store for a warp whose rows or columns lie past the matrix
+        const uint32_t valid_cols = (col0 < N && row0 < batch * M) ? min(kHalf, N - col0) : 0u;
         uint32_t r[kLoads][32];
 #pragma unroll
         for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
@@ -1535,7 +1537,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)(a.M / 256) * (uint32_t)((a.N + BN - 1) / BN);
+  const uint32_t tiles = (uint32_t)a.batch * (uint32_t)((a.M + 255) / 256) * (uint32_t)((a.N + BN - 1) / BN);
   const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
   const uint32_t rows_per_cta = 128u + cfg::kBRows;
@@ -1593,30 +1595,39 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   *cuda_err = cudaSuccess;
   EncodeTiledFn fn = encode_fn(cuda_err);
   if (!fn) return MX_ERR_CUDA;
-  // 256-wide tiles move the fewest operand bytes through shared memory per flop; problems with
-  // fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
+  // few rows of A: operands swapped, deep ring (see mx_gemm_skinny_kernel)
+  if (!a.dense && a.batch == 1 && a.q_elems == nullptr && a.M <= a.skinny_m) {
+    *cuda_err = launch_skinny(a, fn);
+    return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
+  }
+  // One-CTA kernel: 256-wide tiles move the fewest operand bytes through shared memory per flop;
+  // problems with fewer such tiles than SMs use 128-wide tiles to occupy more SMs.
   const int64_t tiles256 = a.batch * ((a.M + BM - 1) / BM) * ((a.N + 255) / 256);
   const int bn = tiles256 >= a.sm_count ? 256 : 128;
-  // two-CTA kernel: needs whole 256-row tiles, and pays as soon as the same problem cut into
-  // 128 x 128 tiles would need more than one wave of the SMs (a 128 x 128 tile, bound by operand
-  // delivery, takes 0.8 of the time of a pair's 256 x 256 tile: 512 x 4096 x 4096, 32 pair tiles or
-  // 128 single ones, 0.73 against 0.88 PFLOP/s; 768 x 4096 x 4096, 48 or 192, 1.09 against 0.87)
-  if (a.M % 256 == 0 && 4 * a.batch * (a.M / 256) * ((a.N + 255) / 256) > a.sm_count) {
+  // Two-CTA kernel or one-CTA kernel: by waves x time per tile.  Measured on tiles with K = 4096, in
+  // units of a pair's 256 x 256 tile: a 128 x 256 tile of the one-CTA kernel takes 1.05 (8320 x 8192:
+  // 14.6 us a wave against 13.9), a 128 x 128 tile 0.82 (512 x 4096 x 4096, 32 pair tiles or 128 single
+  // ones: 0.73 against 0.88 PFLOP/s; 768 x 4096, 48 or 192: 1.09 against 0.87) -- both are bound by
+  // operand delivery, of which the pair needs half per flop.  The pair kernel's tiles may be ragged in
+  // M as in N (rows past M are zero-filled on the way in and clipped on the way out), except for
+  // stacked matrices and the quantizing epilogue, which need whole tiles.
+  const int64_t tiles_pair = a.batch * ((a.M + 255) / 256) * ((a.N + 255) / 256);
+  const int64_t tiles_one = a.batch * ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
+  const int64_t pairs = a.sm_count / 2;
+  const double cost_pair = (double)((tiles_pair + pairs - 1) / pairs);
+  const double cost_one = (double)((tiles_one + a.sm_count - 1) / a.sm_count) * (bn == 256 ? 1.05 : 0.82);
+  const bool pair_ok = a.M % 256 == 0 || (a.batch == 1 && a.q_elems == nullptr);
+  if (pair_ok && a.M >= 256 && cost_pair < cost_one) {
     // FP4 x FP4 with whole 256-element K stages runs on kind::mxf4 (twice the MMA rate)
     const bool f4 = !a.dense && a.fmtA == MX_E2M1 && a.fmtB == MX_E2M1 && a.K % 256 == 0;
-    // 256 x 384 tiles pull fewer operand bytes per MAC from L2; taken only when pinned
-    // (force_bn): measured slower than 256 x 256 for FP8 (four stages in flight instead of six)
-    const int64_t tiles384 = a.batch * (a.M / 256) * ((a.N + 383) / 384);
+    // 256 x 384 tiles pull fewer operand bytes per MAC from L2; taken only when pinned (force_bn):
+    // a tie with 256 x 256 on the large configurations
+    const int64_t tiles384 = a.batch * ((a.M + 255) / 256) * ((a.N + 383) / 384);
     const bool wide = a.q_elems == nullptr && a.force_bn == 384 && tiles384 >= a.sm_count / 2;
     if (wide)
       *cuda_err = a.dense ? launch_pair<2, 384>(a, fn) : f4 ? launch_pair<1, 384>(a, fn) : launch_pair<0, 384>(a, fn);
     else
       *cuda_err = a.dense ? launch_pair<2, 256>(a, fn) : f4 ? launch_pair<1, 256>(a, fn) : launch_pair<0, 256>(a, fn);
-    return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
-  }
-  // few rows of A: operands swapped, deep ring (see mx_gemm_skinny_kernel)
-  if (!a.dense && a.batch == 1 && a.q_elems == nullptr && a.M <= a.skinny_m) {
-    *cuda_err = launch_skinny(a, fn);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
   CUtensorMap ma, mb;

@@ -568,6 +568,8 @@ def test_gemm_dense_errors():
     (2048, 9608, 416, 1, 1, torch.float32),      # two-CTA tiles, N and K tails
     (2048, 9608, 384, 2, 3, torch.float32),      # 6-bit operands (K % 128)
     (130, 264, 640, 4, 4, torch.bfloat16),
+    (640, 4104, 384, 0, 0, torch.float32),       # two-CTA tiles with a half-empty last tile row, N tail
+    (900, 8200, 256, 2, 3, torch.bfloat16),      # the same with 6-bit operands and BF16 out
 ])
 def test_tails(M, N, K, fa, fb, dt):
     """Shapes that are not whole tiles: any M, K a multiple of the block size, C rows whole 16-byte
