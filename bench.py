@@ -120,9 +120,14 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
+        return self.summarize(out, self.t0, self.t1)
+
+    @classmethod
+    def summarize(cls, text: str, t0, t1):
+        """The clocks record from nvidia-smi's CSV lines and the timed region's host times."""
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         samples = []  # (epoch or None, sm, max sm, power, reasons)
-        for line in out.strip().splitlines():
+        for line in text.strip().splitlines():
             parts = [p.strip() for p in line.split(",")]
             if len(parts) < 8:
                 continue
@@ -130,12 +135,11 @@ class ClockSampler:
                 sm, mx_, power = float(parts[1]), float(parts[2]), float(parts[3])
             except ValueError:
                 continue
-            samples.append((self._epoch(parts[0]), sm, mx_, power,
+            samples.append((cls._epoch(parts[0]), sm, mx_, power,
                             {n for n, v in zip(names, parts[4:8]) if v.lower().startswith("active")}))
         if not samples:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no samples"]}
-        inside = [x for x in samples
-                  if x[0] is not None and self.t0 is not None and self.t0 <= x[0] <= self.t1]
+        inside = [x for x in samples if x[0] is not None and t0 is not None and t0 <= x[0] <= t1]
         pmax = max(x[3] for x in samples)
         use = inside or [x for x in samples if x[3] > 0.5 * pmax] or samples
         return {"sm_mhz": statistics.median(x[1] for x in use), "sm_max_mhz": max(x[2] for x in samples),

@@ -41,3 +41,30 @@ def test_two_rank_aggregation_with_gloo(tmp_path):
     import bench
     assert bench.max_over_ranks([3.0, 4.0], "cpu", 1) == [3.0, 4.0]
     assert bench.job_throughput(10.0, 1, 2.0) == 5.0
+
+
+def test_clock_record_keeps_the_samples_inside_the_timed_region():
+    """bench.py's clock record: nvidia-smi lines carry timestamps, and only those between the two
+    host times that bracket the timed region count; throttle reasons are collected from them."""
+    import datetime
+    sys.path.insert(0, os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    import bench
+
+    base = datetime.datetime(2026, 1, 2, 3, 4, 5)
+
+    def line(ms, sm, power, cap="Not Active", hw="Not Active"):
+        t = (base + datetime.timedelta(milliseconds=ms)).strftime("%Y/%m/%d %H:%M:%S.%f")[:-3]
+        return f"{t}, {sm}, 1965, {power}, {hw}, Not Active, Not Active, {cap}"
+
+    text = "\n".join([line(0, 345, 150.0), line(10, 1965, 300.0), line(20, 1905, 420.0, cap="Active"),
+                      line(30, 1965, 310.0), line(500, 345, 140.0, hw="Active"), "garbage line"])
+    t0 = (base + datetime.timedelta(milliseconds=5)).timestamp()
+    t1 = (base + datetime.timedelta(milliseconds=35)).timestamp()
+    rec = bench.ClockSampler.summarize(text, t0, t1)
+    assert rec["in_timed_region"] and rec["samples"] == 3
+    assert rec["sm_mhz"] == 1965 and rec["sm_max_mhz"] == 1965 and rec["power_w_max"] == 420.0
+    assert rec["reasons"] == ["sw_power_cap"]  # the hw_slowdown sample lies outside the region
+    # a region that caught no sample: the samples taken under load stand in, and the record says so
+    rec = bench.ClockSampler.summarize(text, t1 + 100, t1 + 101)
+    assert not rec["in_timed_region"] and rec["samples"] == 3
+    assert bench.ClockSampler.summarize("", t0, t1)["reasons"] == ["no samples"]
