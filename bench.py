@@ -742,6 +742,15 @@ def main_case(args):
         C = torch.empty((n, n), dtype=torch.float32, device="cuda")
         for _ in range(reps):
             mx.mx_gemm(ea, sa, eb, sb, n, n, n, fmt, fmt, out=C, check_status=True)
+    elif args.case == "gemm_few_rows":  # a decode step: 16 activation rows against 16384 x 4096 weights (67 MB)
+        M, N, K = 16, 16384, 4096
+        g = torch.Generator(device="cuda").manual_seed(7)
+        fmt = mx.FORMATS[args.fmt]
+        ea, sa = mx.mx_quantize(torch.randn((M, K), generator=g, device="cuda", dtype=torch.bfloat16), 1, mx.MX_E4M3)
+        eb, sb = mx.mx_quantize(torch.randn((N, K), generator=g, device="cuda", dtype=torch.bfloat16) * 0.05, 1, fmt)
+        C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        for _ in range(reps):
+            mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, fmt, out=C, check_status=True)
     elif args.case == "gemm_dense":   # MXINT8 x MXINT8 through BF16: two dequantize launches + the dense GEMM
         n = 4096
         d = inputs.config4("cuda", n)
@@ -771,7 +780,7 @@ def main_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm", "gemm_dense",
-                                       "quantize_dual", "im2col"],
+                                       "gemm_few_rows", "quantize_dual", "im2col"],
                     default="step", help="'step' = the benchmark; the others run three launches of one "
                                          "kernel on a small case for a profiler capture")
     ap.add_argument("--fmt", choices=FMT_NAMES, default="e4m3")
