@@ -541,7 +541,7 @@ def run_cpu_baseline(rows: int = 2048, seconds_target: float = 15.0):
     import torch
 
     import oracle as O
-    from paper_2310_10537_b200 import inputs
+    import workloads as inputs
     T = inputs.config2("cpu", rows, SWEEP_COLS, seed=2002)
     x = T.view(torch.int16).numpy().view(np.uint16)
     n = rows * SWEEP_COLS
@@ -563,7 +563,7 @@ def main_ours(args, rank, world, local_rank):
     import torch
 
     import paper_2310_10537_b200 as mx
-    from paper_2310_10537_b200 import inputs
+    import workloads as inputs
 
     if not torch.cuda.is_available():
         raise SystemExit("bench.py needs a CUDA device (there is no CPU fallback)")
@@ -715,7 +715,7 @@ def main_case(args):
     import torch
 
     import paper_2310_10537_b200 as mx
-    from paper_2310_10537_b200 import inputs
+    import workloads as inputs
     torch.cuda.set_device(0)
     reps = 3
     if args.case in ("quantize", "dequantize"):
@@ -798,7 +798,7 @@ def main():
         import torch
 
         import paper_2310_10537_b200 as mx
-        from paper_2310_10537_b200 import inputs
+        import workloads as inputs
         torch.cuda.set_device(0)
         print("# Per-kernel measurements on one B200 (`python bench.py --report`)\n")
         print(run_report(torch, mx, inputs))

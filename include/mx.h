@@ -49,7 +49,7 @@ typedef enum {
   MX_INT8 = 5  /* 1 sign + 1 integer + 6 fraction bits, max 127/64       */
 } mx_fmt_t;
 
-/* Rounding of V_i / X onto the element grid (Algorithm 1, line 4).
+/* Rounding of V_i / X onto the element grid (the element cast of Algorithm 1).
  * Section 4.3 uses round-half-to-even for inference, Section 4.5
  * round-half-away-from-zero for training. */
 typedef enum { MX_RNE = 0, MX_RHAZ = 1 } mx_round_t;
@@ -151,7 +151,7 @@ const char* mx_last_cuda_error(void);
  * emax_elem, clamped to [-127, 127]; an all-zero block gets scale byte 0x00; a
  * block holding Inf or NaN gets scale byte 0xFF (X = NaN) and zero codes;
  * P_i = V_i / X rounded (rounding) to the element grid, subnormals included,
- * and saturated to +-max normal with the sign kept (Algorithm 1 line 4 and its
+ * and saturated to +-max normal with the sign kept (the element cast of Algorithm 1 and its
  * note).  Results that round to zero keep their sign bit in the FP formats.
  *
  * Errors: MX_ERR_NULL, MX_ERR_SHAPE (ndim < 1 or > 8, axis out of range,

@@ -108,8 +108,9 @@ static double round_mode(double t, int rounding) {
 }
 
 /*
- * Algorithm 1, line 4: quantize the exact quotient r = V_i / X to the element
- * format, clamping normal numbers.  sign is the sign bit of V_i.
+ * The element cast of Section 3, Algorithm 1: the exact quotient r = V_i / X is
+ * rounded onto the element format's grid and saturated at its largest normal
+ * value.  sign is the sign bit of V_i.
  */
 static uint8_t encode_element(double r, int sign, int fmt, int rounding) {
   const fmt_info* f = &FMT[fmt];
@@ -229,7 +230,10 @@ void oracle_unpack_codes(const uint8_t* packed, int64_t n, int fmt, uint8_t* cod
 /* Algorithm 1 on one block                                                */
 /* ---------------------------------------------------------------------- */
 
-/* bits[32]: FP32 bit patterns of V_1..V_32.  Writes 32 codes and the scale byte. */
+/* Section 3, Algorithm 1.  bits[32]: FP32 bit patterns of V_1..V_32.  The shared exponent is
+ * the exponent of the block maximum less the element format's largest exponent; the scale is
+ * that power of two; every element is divided by it and cast with saturation.  Writes 32 codes
+ * and the scale byte. */
 static void quantize_block_bits(const uint32_t* bits, int fmt, int rounding,
                                 uint8_t* codes, uint8_t* scale_byte) {
   uint32_t v[BLOCK];
@@ -254,12 +258,12 @@ static void quantize_block_bits(const uint32_t* bits, int fmt, int rounding,
     shared_exp = -127; /* log2(0): smallest scale */
   } else {
     int E = (int)((amax_bits >> 23) & 0xFF) - 127; /* floor(log2(amax)), amax is normal */
-    shared_exp = E - FMT[fmt].emax;                /* line 1 */
+    shared_exp = E - FMT[fmt].emax;                /* shared exponent */
     if (shared_exp < -127) shared_exp = -127;
     if (shared_exp > 127) shared_exp = 127;
   }
-  *scale_byte = (uint8_t)(shared_exp + 127); /* line 2: X = 2^shared_exp */
-  for (int i = 0; i < BLOCK; ++i) {           /* lines 3-5 */
+  *scale_byte = (uint8_t)(shared_exp + 127); /* X = 2^shared_exp as an E8M0 byte */
+  for (int i = 0; i < BLOCK; ++i) {           /* the elements, each scaled by 1/X and cast */
     double V = (double)bits_f32(v[i]);
     double r = ldexp(V, -shared_exp); /* V / X, exact in double */
     codes[i] = encode_element(r, (int)(v[i] >> 31), fmt, rounding);

@@ -36,21 +36,31 @@ struct View {
   int64_t padded_numel;  // rows * Lp
 };
 
-// [outer, L, inner] view of shape[ndim] around `axis`; false on a bad shape.
+// [outer, L, inner] view of shape[ndim] around `axis`; false on a bad shape.  Every product is
+// formed with an overflow check and the padded element count is held below 2^44, so that no byte
+// count derived from the view (at most 4 bytes per element plus alignment) can wrap a size_t or
+// come out smaller than the tensor it describes.
+constexpr int64_t kMaxElements = (int64_t)1 << 44;
+
 bool make_view(const int64_t* shape, int ndim, int axis, View* v) {
   if (!shape || ndim < 1 || ndim > 8 || axis < 0 || axis >= ndim) return false;
   v->outer = v->inner = 1;
   for (int i = 0; i < ndim; ++i) {
     if (shape[i] < 0) return false;
-    if (i < axis) v->outer *= shape[i];
-    if (i > axis) v->inner *= shape[i];
+    if (i < axis && __builtin_mul_overflow(v->outer, shape[i], &v->outer)) return false;
+    if (i > axis && __builtin_mul_overflow(v->inner, shape[i], &v->inner)) return false;
   }
   v->L = shape[axis];
-  v->numel = v->outer * v->L * v->inner;
-  v->rows = v->outer * v->inner;
+  if (v->L > kMaxElements) return false;
   v->kblocks = (v->L + 31) / 32;  // a last, partial block is stored padded with zero codes
   v->Lp = v->kblocks * 32;
-  v->padded_numel = v->rows * v->Lp;
+  if (__builtin_mul_overflow(v->outer, v->inner, &v->rows)) return false;
+  if (__builtin_mul_overflow(v->rows, v->L, &v->numel)) return false;
+  if (__builtin_mul_overflow(v->rows, v->Lp, &v->padded_numel)) return false;
+  if (v->padded_numel > kMaxElements) return false;
+  // the swizzled scale tensor pads rows to 128 and blocks to 4: bounded by 16 x (rows + 128) x (kblocks + 4)
+  int64_t sc;
+  if (__builtin_mul_overflow(v->rows + 128, v->kblocks + 4, &sc) || sc > kMaxElements) return false;
   return true;
 }
 

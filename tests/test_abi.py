@@ -83,6 +83,34 @@ def test_argument_validation_without_gpu():
     assert lib.mx_strerror(mx.MX_ERR_ALIGN) and lib.mx_strerror(-99)
 
 
+def test_extents_whose_products_wrap_are_rejected():
+    """Shapes whose element count wraps a 64-bit integer (2^32 x 2^32 has numel 0 mod 2^64) or is
+    simply absurd must come back as MX_ERR_SHAPE / size 0 from every entry point that derives a
+    byte count from the shape -- above all from the entry point whose staging area is a fixed
+    array, where a wrapped count would pass the size check."""
+    lib = mx.lib()
+    buf = np.zeros(4096, np.uint8)
+    p = buf.ctypes.data + (-buf.ctypes.data) % 256
+    o = mx.binding.mx_opts_t(mx.MX_F32, mx.MX_SCALES_SWIZZLED, None, 0)
+    for dims in ((1 << 32, 1 << 32), (1 << 62, 4), (3, 1 << 62), (1 << 31, 1 << 31, 1 << 31), (1 << 45, 32)):
+        shape = (ctypes.c_int64 * len(dims))(*dims)
+        nd = len(dims)
+        for axis in range(nd):
+            assert mx.mx_elems_bytes(list(dims), axis, 0) == 0, dims
+            assert mx.mx_scales_bytes(list(dims), axis, 1) == 0, dims
+            assert lib.mx_quantize_host_workspace_bytes(shape, nd, axis, 0, ctypes.byref(o)) == 0
+            assert lib.mx_quantize(p, p, p, shape, nd, axis, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE, dims
+            assert lib.mx_quantize_host_static(p, p, p, shape, nd, axis, 0, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE, dims
+            assert lib.mx_quantize_host(p, p, p, shape, nd, axis, 0, 0, ctypes.byref(o), p, 1 << 20) == mx.MX_ERR_SHAPE
+            assert lib.mx_dequantize_host(p, p, p, shape, nd, axis, 0, ctypes.byref(o), p, 1 << 20) == mx.MX_ERR_SHAPE
+        assert lib.mx_dequantize(p, p, p, shape, nd, nd - 1, 0, ctypes.byref(o)) == mx.MX_ERR_SHAPE, dims
+    # large but legitimate extents still get their sizes
+    assert mx.mx_elems_bytes([1 << 20, 1 << 20], 1, 4) == 1 << 39
+    # a request just over the fixed staging array is a workspace error, not a shape error
+    shape = (ctypes.c_int64 * 2)(4096, 4096)
+    assert lib.mx_quantize_host_static(p, p, p, shape, 2, 1, 0, 0, ctypes.byref(o)) == mx.MX_ERR_WORKSPACE
+
+
 def test_gemm_variants_argument_validation_without_gpu():
     """The GEMM entry points added beside mx_gemm reject bad arguments before any CUDA call."""
     lib = mx.lib()

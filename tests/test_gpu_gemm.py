@@ -10,11 +10,21 @@ import torch
 
 import oracle as O
 import paper_2310_10537_b200 as mx
-from paper_2310_10537_b200 import inputs
-from gpu_util import Guarded, to_oracle_input
+import workloads as inputs
+from gpu_util import Guarded, assert_operand_rows_match_oracle, to_oracle_input
 
 pytestmark = pytest.mark.gpu
 TOL = 1e-5
+# BF16 output: the FP32 accumulator c32 obeys |c32 - c64| <= TOL * S and is rounded once to nearest
+# even, |c_bf16 - c32| <= 2^-8 |c32| (half an ulp of an 8-bit significand), hence
+#   |c_bf16 - c64| <= (1 + 2^-8) * TOL * S + 2^-8 * |c64|.
+# FP32 output is held to TOL * S as stated, with no factor.
+BF16_REL = 2.0 ** -8
+
+
+def _bound_terms(dt):
+    """(factor on TOL * S, relative term on |c64|) for an output of type dt."""
+    return (1.0 + BF16_REL, BF16_REL) if dt == torch.bfloat16 else (1.0, 0.0)
 FP = [mx.MX_E4M3, mx.MX_E5M2, mx.MX_E3M2, mx.MX_E2M3, mx.MX_E2M1]
 
 
@@ -124,8 +134,8 @@ def test_few_rows_against_oracle(M, N, K, fa, fb, dt):
     g_out.check()
     hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
     c64, s = O.gemm(hea, hsa, heb, hsb, M, N, K, fa, fb)
-    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
-    assert (np.abs(C.double().cpu().numpy() - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+    fac, rel = _bound_terms(dt)
+    assert (np.abs(C.double().cpu().numpy() - c64) <= fac * TOL * s + np.abs(c64) * rel).all()
 
 
 @pytest.mark.parametrize("M,N,K,fa,fb", [(64, 1024, 512, 0, 0), (17, 19200, 256, 4, 1), (96, 640, 1024, 2, 3)])
@@ -373,14 +383,14 @@ def test_bf16_output(shape, fa, fb):
     da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
     db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
     ref = da @ db.T
-    bound = 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * 2.0 ** -8
+    bound = (1.0 + BF16_REL) * TOL * (da.abs() @ db.abs().T) + ref.abs() * BF16_REL
     bad = int(((C.double() - ref).abs() > bound).sum())
     assert bad == 0, f"{shape}: {bad} outputs beyond the bound"
     rng = np.random.default_rng(N)
     ms, ns = rng.integers(0, M, 1000), rng.integers(0, N, 1000)
     c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
     got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
-    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * 2.0 ** -8).all()
+    assert (np.abs(got - c64) <= (1.0 + BF16_REL) * TOL * s + np.abs(c64) * BF16_REL).all()
     # the BF16 result is the FP32 result of the same kernel rounded once to nearest even
     C32 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
     assert torch.equal(C32.to(torch.bfloat16).view(torch.int16), C.view(torch.int16))
@@ -413,8 +423,8 @@ def test_batched(batch, M, N, K, fa, fb, dt):
     db = torch.from_numpy(O.dequantize(heb, hsb, batch * N, K, fb, O.F64)).cuda().view(batch, N, K)
     ref = da @ db.transpose(1, 2)
     S = da.abs() @ db.abs().transpose(1, 2)
-    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
-    bad = int(((C.double() - ref).abs() > 1.004 * TOL * S + ref.abs() * rel).sum())
+    fac, rel = _bound_terms(dt)
+    bad = int(((C.double() - ref).abs() > fac * TOL * S + ref.abs() * rel).sum())
     assert bad == 0, f"{bad} outputs beyond the bound"
     abytes, bbytes = M * K * O.fmt_bits(fa) // 8, N * K * O.fmt_bits(fb) // 8
     for b in {0, batch - 1}:
@@ -422,7 +432,7 @@ def test_batched(batch, M, N, K, fa, fb, dt):
                         heb[b * bbytes:(b + 1) * bbytes], hsb[b * N * K // 32:(b + 1) * N * K // 32],
                         M, N, K, fa, fb)
         got = C[b].double().cpu().numpy()
-        assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all(), f"matrix {b}"
+        assert (np.abs(got - c64) <= fac * TOL * s + np.abs(c64) * rel).all(), f"matrix {b}"
 
 
 def test_batched_errors():
@@ -539,14 +549,14 @@ def test_gemm_dense(shape, fa, fb, dt):
     da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
     db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
     ref = da @ db.T
-    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
-    bad = int(((C.double() - ref).abs() > 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+    fac, rel = _bound_terms(dt)
+    bad = int(((C.double() - ref).abs() > fac * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
     assert bad == 0, f"{shape}: {bad} outputs beyond the bound"
     rng = np.random.default_rng(M + fa)
     ms, ns = rng.integers(0, M, 1000), rng.integers(0, N, 1000)
     c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
     got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
-    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+    assert (np.abs(got - c64) <= fac * TOL * s + np.abs(c64) * rel).all()
 
 
 def test_gemm_dense_errors():
@@ -590,7 +600,7 @@ def test_tails(M, N, K, fa, fb, dt):
     torch.cuda.synchronize()
     g_out.check()
     hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
-    rel = 2.0 ** -8 if dt == torch.bfloat16 else 0.0
+    fac, rel = _bound_terms(dt)
     if M * N * K <= 1 << 28:
         c64, s = O.gemm(hea, hsa, heb, hsb, M, N, K, fa, fb)
         got = C.double().cpu().numpy()
@@ -598,14 +608,14 @@ def test_tails(M, N, K, fa, fb, dt):
         da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
         db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
         ref = da @ db.T
-        bad = int(((C.double() - ref).abs() > 1.004 * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+        bad = int(((C.double() - ref).abs() > fac * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
         assert bad == 0, f"{bad} outputs beyond the bound"
         rng = np.random.default_rng(K)
         ms = np.concatenate([rng.integers(0, M, 1500), np.full(300, M - 1)])
         ns = np.concatenate([rng.integers(0, N, 1500), rng.integers(N - 40, N, 300)])
         c64, s = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
         got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
-    assert (np.abs(got - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+    assert (np.abs(got - c64) <= fac * TOL * s + np.abs(c64) * rel).all()
     # the BF16 route takes the same shapes
     g_out = Guarded(M * N * esz)
     C2 = g_out.view.view(dt).view(M, N)
@@ -613,10 +623,26 @@ def test_tails(M, N, K, fa, fb, dt):
     torch.cuda.synchronize()
     g_out.check()
     if M * N * K <= 1 << 28:
-        assert (np.abs(C2.double().cpu().numpy() - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+        assert (np.abs(C2.double().cpu().numpy() - c64) <= fac * TOL * s + np.abs(c64) * rel).all()
     else:
         got2 = C2[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
-        assert (np.abs(got2 - c64) <= 1.004 * TOL * s + np.abs(c64) * rel).all()
+        assert (np.abs(got2 - c64) <= fac * TOL * s + np.abs(c64) * rel).all()
+
+
+def _quantized_operand(x, axis, fmt, rounding, what, seed):
+    """Quantizes one GEMM operand on the GPU and proves the bytes before they are used: sampled
+    output rows byte for byte against the oracle on the same input, and -- for the transposing
+    axis-0 pass, whose kernels are not the last-axis one -- the WHOLE tensor against the last-axis
+    kernel run on the transposed input (quantizing along axis 0 is by definition quantizing the
+    transpose along its last axis, and that kernel is compared with the oracle on whole tensors)."""
+    e, s = mx.mx_quantize(x, axis, fmt, rounding)
+    assert_operand_rows_match_oracle(O, x, axis, fmt, rounding, e, s, what, count=256, seed=seed)
+    if axis == 0:
+        xt = x.t().contiguous()
+        e2, s2 = mx.mx_quantize(xt, 1, fmt, rounding)
+        assert torch.equal(e, e2) and torch.equal(s, s2), what + ": axis-0 pass differs from the transposed last-axis pass"
+        del xt, e2, s2
+    return e, s
 
 
 def test_config3_full_size():
@@ -624,25 +650,45 @@ def test_config3_full_size():
     X, W = d["X"], d["W"]
     M, K = X.shape
     N = W.shape[1]
-    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
-    eb, sb = mx.mx_quantize(W, 0, mx.MX_E4M3)
+    ea, sa = _quantized_operand(X, 1, mx.MX_E4M3, mx.MX_RNE, "config 3 X", 31)
+    eb, sb = _quantized_operand(W, 0, mx.MX_E4M3, mx.MX_RNE, "config 3 W (axis 0)", 32)
     _full_size_check("config 3", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, 3)
 
 
 def test_config4_training_step():
+    """The MXFP6 training step at its own size: FP32 tensors, half-away rounding, every operand
+    quantized along its own reduction axis (Section 4.1) and every one of the six compared with
+    the oracle before its product is."""
     d = inputs.config4("cuda")
     X, W, dY = d["X"], d["W"], d["dY"]
     n = X.shape[0]
     act, wt, rnd = mx.MX_E3M2, mx.MX_E2M3, mx.MX_RHAZ
     # forward Y = X W: A = Q(X, axis 1), B = Q(W, axis 0) -> [N x K]
-    _full_size_check("config 4 fwd", *mx.mx_quantize(X, 1, act, rnd), *mx.mx_quantize(W, 0, wt, rnd),
-                     n, n, n, act, wt, 41)
+    _full_size_check("config 4 fwd", *_quantized_operand(X, 1, act, rnd, "config 4 X rows", 411),
+                     *_quantized_operand(W, 0, wt, rnd, "config 4 W columns", 412), n, n, n, act, wt, 41)
     # dgrad dX = dY W^T: A = Q(dY, axis 1), B = Q(W, axis 1)
-    _full_size_check("config 4 dgrad", *mx.mx_quantize(dY, 1, act, rnd), *mx.mx_quantize(W, 1, wt, rnd),
-                     n, n, n, act, wt, 42)
+    _full_size_check("config 4 dgrad", *_quantized_operand(dY, 1, act, rnd, "config 4 dY rows", 421),
+                     *_quantized_operand(W, 1, wt, rnd, "config 4 W rows", 422), n, n, n, act, wt, 42)
     # wgrad dW = X^T dY: A = Q(X, axis 0), B = Q(dY, axis 0)
-    _full_size_check("config 4 wgrad", *mx.mx_quantize(X, 0, act, rnd), *mx.mx_quantize(dY, 0, act, rnd),
-                     n, n, n, act, act, 43)
+    _full_size_check("config 4 wgrad", *_quantized_operand(X, 0, act, rnd, "config 4 X columns", 431),
+                     *_quantized_operand(dY, 0, act, rnd, "config 4 dY columns", 432), n, n, n, act, act, 43)
+
+
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16], ids=["f32", "bf16"])
+def test_config4_dual_axis_operands(dtype):
+    """The same six operands out of three mx_quantize_dual calls (each tensor read once): sampled
+    rows of both outputs against the oracle, and both outputs whole against the single-axis calls."""
+    d = inputs.config4("cuda", dtype=dtype)
+    rnd = mx.MX_RHAZ
+    for name, fmt in (("X", mx.MX_E3M2), ("W", mx.MX_E2M3), ("dY", mx.MX_E3M2)):
+        x = d[name]
+        (er, sr), (ec, sc) = mx.mx_quantize_dual(x, fmt, rnd)
+        assert_operand_rows_match_oracle(O, x, 1, fmt, rnd, er, sr, f"dual {name} rows", seed=51)
+        assert_operand_rows_match_oracle(O, x, 0, fmt, rnd, ec, sc, f"dual {name} columns", seed=52)
+        e1, s1 = mx.mx_quantize(x, 1, fmt, rnd)
+        e0, s0 = mx.mx_quantize(x, 0, fmt, rnd)
+        assert torch.equal(er, e1) and torch.equal(sr, s1), name
+        assert torch.equal(ec, e0) and torch.equal(sc, s0), name
 
 
 def test_config5_full_size():
@@ -650,9 +696,10 @@ def test_config5_full_size():
     W, X = d["W"], d["X"]
     M, K = X.shape
     N = W.shape[1]
-    ea, sa = mx.mx_quantize(X, 1, mx.MX_E4M3)
-    eb, sb = mx.mx_quantize(W, 0, mx.MX_E2M1)
+    ea, sa = _quantized_operand(X, 1, mx.MX_E4M3, mx.MX_RNE, "config 5 X", 51)
+    eb, sb = _quantized_operand(W, 0, mx.MX_E2M1, mx.MX_RNE, "config 5 W (axis 0, FP4)", 52)
     del d, W, X
+    torch.cuda.empty_cache()
     _full_size_check("config 5", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, 5)
 
 

@@ -8,7 +8,7 @@ import torch
 
 import oracle as O
 import paper_2310_10537_b200 as mx
-from paper_2310_10537_b200 import inputs
+import workloads as inputs
 from gpu_util import Guarded, to_oracle_input
 
 pytestmark = pytest.mark.gpu

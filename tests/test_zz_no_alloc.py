@@ -3,16 +3,21 @@ memory (a plug-in whose host application owns every free byte of the GPU, a loop
 enter the CUDA allocator).  Its staging area is a fixed array inside the library, so the test
 checks the two things that could go wrong with a shared, never-cleared scratch area: the result
 must equal that of the existing mx_quantize_host (which stages in a caller-supplied workspace)
-byte for byte, and a second call right after the first -- with a different shape, format and
-scale layout, so that stale bytes of the first call sit where the second one works -- must be
-just as exact.  Collected last on purpose: a failure here cannot hide another test's result."""
+and that of the CPU oracle byte for byte, and a second call right after the first -- with a
+different shape, format and scale layout, so that stale bytes of the first call sit where the
+second one works -- must be just as exact.  The promise itself is checked too: the free device
+memory the driver reports is the same before and after a call, on the first call of the process
+and on a later one.  Collected last on purpose: a failure here cannot hide another test's result."""
 import ctypes
 
+import numpy as np
 import pytest
 import torch
 
+import oracle as O
 import paper_2310_10537_b200 as mx
-from paper_2310_10537_b200 import inputs
+import workloads as inputs
+from gpu_util import to_oracle_input
 
 pytestmark = pytest.mark.gpu
 
@@ -37,6 +42,39 @@ def _both_ways(x, axis, fmt, rounding, layout):
     mx.mx_quantize_host_static(x, got_e, got_s, axis, fmt, rounding, layout)
     assert torch.equal(got_e, ref_e), "element codes differ from mx_quantize_host"
     assert torch.equal(got_s, ref_s), "scale bytes differ from mx_quantize_host"
+    # and against the definition itself: the oracle on the same input bytes
+    want_e, want_s = O.quantize(to_oracle_input(x), axis, fmt, rounding, layout)
+    assert np.array_equal(got_e.numpy(), want_e), "element codes differ from the oracle"
+    assert np.array_equal(got_s.numpy(), want_s), "scale bytes differ from the oracle"
+
+
+def _free_bytes():
+    torch.cuda.synchronize()
+    return torch.cuda.mem_get_info()[0]
+
+
+def test_static_scratch_call_allocates_no_device_memory():
+    """Free device memory as the driver reports it must not move across a call.  The first call of
+    a process is let through unmeasured: that is when the driver loads the library's device code
+    and, with it, claims the built-in array (the header says so) -- module loading, not an
+    allocation by the call.  Every later call is held to a difference of exactly zero, also one
+    with another shape that leaves stale bytes behind.  Host outputs are pinned beforehand, so
+    nothing else in the measured window can allocate."""
+    x = inputs.adversarial("cpu", rows=256, cols=512, dtype=torch.bfloat16, seed=33).pin_memory()
+    y = inputs.adversarial("cpu", rows=128, cols=300, dtype=torch.bfloat16, seed=35)[:, :300].contiguous().pin_memory()
+    ex, sx = _host_outputs(list(x.shape), 1, mx.MX_E4M3, mx.MX_SCALES_SWIZZLED)
+    ey, sy = _host_outputs(list(y.shape), 1, mx.MX_E4M3, mx.MX_SCALES_SWIZZLED)
+    torch.zeros(1, device="cuda")            # the CUDA context and torch's pool exist before measuring
+    # first calls: set-up (address look-up, device code of both kernels used below loaded)
+    mx.mx_quantize_host_static(x, ex, sx, 1, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+    mx.mx_quantize_host_static(y, ey, sy, 1, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+    for call, (t, e, s) in enumerate(((x, ex, sx), (y, ey, sy), (x, ex, sx))):
+        before = _free_bytes()
+        mx.mx_quantize_host_static(t, e, s, 1, mx.MX_E4M3, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+        after = _free_bytes()
+        assert after == before, f"later call {call}: free device memory moved by {before - after} bytes"
+        want_e, want_s = O.quantize(to_oracle_input(t), 1, mx.MX_E4M3, O.RNE, O.SWIZZLED)
+        assert np.array_equal(e.numpy(), want_e) and np.array_equal(s.numpy(), want_s)
 
 
 def test_static_scratch_matches_workspace_variant_twice_in_a_row():
@@ -48,6 +86,11 @@ def test_static_scratch_matches_workspace_variant_twice_in_a_row():
     _both_ways(x2, 0, mx.MX_E3M2, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
     # and the first request again: its padding must be clean although call 2 wrote there
     _both_ways(x1, 1, mx.MX_E2M1, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+    # a row length that is not a whole number of blocks, after larger calls: the zero codes that pad
+    # the partial last block and the padding of the scale tensor sit on stale bytes of the calls above
+    x3 = inputs.adversarial("cpu", rows=100, cols=320, dtype=torch.bfloat16, seed=34)[:, :300].contiguous().pin_memory()
+    _both_ways(x3, 1, mx.MX_E3M2, mx.MX_RNE, mx.MX_SCALES_SWIZZLED)
+    _both_ways(x3, 0, mx.MX_E4M3, mx.MX_RHAZ, mx.MX_SCALES_LINEAR)
 
 
 def test_static_scratch_rejects_oversized_request():
