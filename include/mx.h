@@ -237,6 +237,38 @@ int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t*
                  const mx_opts_t* opts);
 
 /*
+ * mx_gemm / mx_gemm_bf16 with the kernel selection and the device-side wait budget in the caller's
+ * hands (Section 4.1 defines the product; this call adds nothing to it).  It exists for tuning, for
+ * tests that must reach a particular kernel variant, and for the failure drill below; a NULL plan,
+ * or a field left at its "library's choice" value, gives exactly mx_gemm.
+ *   c_dtype         MX_F32 (C is float*) or MX_BF16.
+ *   tile_n          0 = library's choice; 256 or 384 pins the tile width of the two-CTA kernel.
+ *   few_rows_limit  -1 = library's choice (96); 0..128 = largest M that takes the kernel that puts
+ *                   B on the M side of the MMA (0 sends every product through the tiled kernels).
+ *   wait_cycles     0 = library's choice (about one second); otherwise the budget, in SM clock
+ *                   cycles, after which a device-side wait for one pipeline stage gives up (waits
+ *                   for a whole tile get four times as much).  When a wait gives up the kernel
+ *                   records which one, every warp leaves through the common exit, tensor memory is
+ *                   released and the context stays usable; the call (with opts->check_status) or
+ *                   the next checked call returns MX_ERR_TIMEOUT and the output is undefined.
+ *   drop_fill       -1 = off.  Failure drill: the operand producer leaves out the pipeline fill
+ *                   with this running number (0 = the first K chunk of the CTA's first tile): no
+ *                   copy is issued for it, so nothing is in flight when the kernel gives up, and
+ *                   the MMA issuer's wait for that stage runs out.  Use with a small wait_cycles.
+ * Errors as mx_gemm; MX_ERR_FMT for a bad c_dtype, MX_ERR_SHAPE for a field out of range.
+ */
+typedef struct {
+  int32_t c_dtype;
+  int32_t tile_n;
+  int32_t few_rows_limit;
+  int32_t drop_fill;
+  int64_t wait_cycles;
+} mx_gemm_plan_t;
+int mx_gemm_ex(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+               int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+               const mx_opts_t* opts, const mx_gemm_plan_t* plan);
+
+/*
  * `batch` independent products in one launch: the matmuls of attention (scores, context)
  * are dot products like any other (Section 4.1 counts every dot-product operation).
  * A is the packed [batch x M x K] tensor, B [batch x N x K], C [batch x M x N] (c_dtype:

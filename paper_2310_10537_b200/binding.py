@@ -31,7 +31,7 @@ MX_ERR_UNSUPPORTED, MX_ERR_CUDA, MX_ERR_TIMEOUT, MX_ERR_WORKSPACE = -5, -6, -7, 
 EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
-    "mx_gemm_bf16", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
+    "mx_gemm_bf16", "mx_gemm_ex", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
     "mx_gemm_dense", "mx_conv_out_h", "mx_conv_out_w", "mx_im2col",
     "mx_quantize_host_async", "mx_dequantize_host_async", "mx_host_synchronize",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
@@ -43,6 +43,12 @@ EXPORTS = [
 class mx_opts_t(ctypes.Structure):
     _fields_ = [("dtype", ctypes.c_int32), ("scale_layout", ctypes.c_int32),
                 ("stream", ctypes.c_void_p), ("check_status", ctypes.c_int32)]
+
+
+class mx_gemm_plan_t(ctypes.Structure):
+    _fields_ = [("c_dtype", ctypes.c_int32), ("tile_n", ctypes.c_int32),
+                ("few_rows_limit", ctypes.c_int32), ("drop_fill", ctypes.c_int32),
+                ("wait_cycles", ctypes.c_int64)]
 
 
 class mx_conv_t(ctypes.Structure):
@@ -86,6 +92,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_dequantize.argtypes = [vp, u8p, vp, i64p, ci, ci, ci, op]
     lib.mx_gemm.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
     lib.mx_gemm_bf16.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op]
+    lib.mx_gemm_ex.argtypes = [vp, u8p, vp, u8p, vp, i64, i64, i64, ci, ci, op, ctypes.POINTER(mx_gemm_plan_t)]
     lib.mx_gemm_quantize.argtypes = [vp, u8p, vp, u8p, vp, u8p, i64, i64, i64, ci, ci, ci, ci, op]
     lib.mx_gemm_dense_workspace_bytes.argtypes = [i64, i64, i64]
     lib.mx_gemm_dense_workspace_bytes.restype = sz
@@ -242,6 +249,22 @@ def mx_gemm_bf16(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.T
     o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
     _check(_lib.mx_gemm_bf16(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
                              out.data_ptr(), M, N, K, fmtA, fmtB, ctypes.byref(o)), "mx_gemm_bf16")
+    return out
+
+
+def mx_gemm_ex(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
+               M: int, N: int, K: int, fmtA: int, fmtB: int, out: Optional[torch.Tensor] = None,
+               out_dtype: torch.dtype = torch.float32, tile_n: int = 0, few_rows_limit: int = -1,
+               wait_cycles: int = 0, drop_fill: int = -1, check_status: bool = False) -> torch.Tensor:
+    """mx_gemm / mx_gemm_bf16 with the kernel selection (tile_n, few_rows_limit) and the device-side
+    wait budget (wait_cycles; drop_fill is the failure drill) in the caller's hands."""
+    assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
+    if out is None:
+        out = torch.empty((M, N), dtype=out_dtype, device=A.device)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    plan = mx_gemm_plan_t(_dtype_code(out.dtype), tile_n, few_rows_limit, drop_fill, wait_cycles)
+    _check(_lib.mx_gemm_ex(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(), out.data_ptr(),
+                           M, N, K, fmtA, fmtB, ctypes.byref(o), ctypes.byref(plan)), "mx_gemm_ex")
     return out
 
 

@@ -546,22 +546,7 @@ int mx_host_synchronize(void) {
 // GEMM
 // ---------------------------------------------------------------------------
 
-// MX_GEMM_TILE_N=256|384 in the environment pins the two-CTA kernel's tile width (tuning, tests).
-static int tile_width_override() {
-  const char* v = std::getenv("MX_GEMM_TILE_N");
-  if (!v) return 0;
-  const int n = std::atoi(v);
-  return n == 256 || n == 384 ? n : 0;
-}
-
-// Largest M that takes the swapped-operand kernel; MX_GEMM_SKINNY_M=0..128 in the environment
-// overrides it (tuning, tests).
-static int skinny_m_limit() {
-  const char* v = std::getenv("MX_GEMM_SKINNY_M");
-  if (!v) return 96;
-  const int n = std::atoi(v);
-  return n < 0 ? 0 : n > 128 ? 128 : n;
-}
+constexpr int kFewRowsDefault = 96;  // largest M that takes the swapped-operand kernel
 
 // strict: every matrix must consist of whole 128-row / 128-column tiles (batched products, whose
 // matrices are stacked along rows, and the quantizing epilogue, which writes whole blocks).
@@ -583,7 +568,8 @@ static int gemm_validate(const void* A, const uint8_t* sA, const void* B, const 
 static int gemm_device(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
                        int c_bf16, int64_t batch, int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA,
                        mx_fmt_t fmtB, const mx_opts_t* opts, void* q_elems = nullptr,
-                       uint8_t* q_scales = nullptr, int q_fmt = 0, int q_round = 0) {
+                       uint8_t* q_scales = nullptr, int q_fmt = 0, int q_round = 0,
+                       const mx_gemm_plan_t* plan = nullptr) {
   Opts o;
   if (!C) {
     if (!q_elems || !q_scales) return MX_ERR_NULL;
@@ -605,8 +591,10 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
   mx::GemmArgs a;
   a.A = A; a.sA = sA; a.B = B; a.sB = sB; a.C = C; a.c_bf16 = c_bf16; a.batch = batch;
   a.dense = 0;
-  a.force_bn = tile_width_override();
-  a.skinny_m = skinny_m_limit();
+  a.force_bn = plan ? plan->tile_n : 0;
+  a.skinny_m = plan && plan->few_rows_limit >= 0 ? plan->few_rows_limit : kFewRowsDefault;
+  a.wait_cycles = plan ? plan->wait_cycles : 0;
+  a.drop_fill = plan ? plan->drop_fill : -1;
   a.q_elems = q_elems; a.q_scales = q_scales; a.q_fmt = q_fmt; a.q_round = q_round;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream;
@@ -637,6 +625,18 @@ int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t*
                  int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
                  const mx_opts_t* opts) {
   return gemm_device(A, sA, B, sB, C, 1, 1, M, N, K, fmtA, fmtB, opts);
+}
+
+int mx_gemm_ex(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
+               int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB,
+               const mx_opts_t* opts, const mx_gemm_plan_t* plan) {
+  if (!plan) return gemm_device(A, sA, B, sB, C, 0, 1, M, N, K, fmtA, fmtB, opts);
+  if (plan->c_dtype != MX_F32 && plan->c_dtype != MX_BF16) return MX_ERR_FMT;
+  if ((plan->tile_n != 0 && plan->tile_n != 256 && plan->tile_n != 384) || plan->few_rows_limit < -1 ||
+      plan->few_rows_limit > 128 || plan->drop_fill < -1 || plan->wait_cycles < 0)
+    return MX_ERR_SHAPE;
+  return gemm_device(A, sA, B, sB, C, plan->c_dtype == MX_BF16, 1, M, N, K, fmtA, fmtB, opts, nullptr, nullptr,
+                     0, 0, plan);
 }
 
 int mx_gemm_batched(const void* A, const uint8_t* sA, const void* B, const uint8_t* sB, void* C,
@@ -693,7 +693,7 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
   if ((e = mx::launch_dequantize(d)) != cudaSuccess) return fail_cuda(e);
   mx::GemmArgs a;
   a.A = dA; a.sA = nullptr; a.B = dB; a.sB = nullptr; a.C = C; a.c_bf16 = (int)c_dtype == MX_BF16;
-  a.dense = 1; a.batch = 1; a.force_bn = tile_width_override(); a.skinny_m = 0;
+  a.dense = 1; a.batch = 1; a.force_bn = 0; a.skinny_m = 0; a.wait_cycles = 0; a.drop_fill = -1;
   a.q_elems = nullptr; a.q_scales = nullptr; a.q_fmt = 0; a.q_round = 0;
   a.M = M; a.N = N; a.K = K; a.fmtA = (int)fmtA; a.fmtB = (int)fmtB;
   a.stream = o.stream; a.sm_count = sms;

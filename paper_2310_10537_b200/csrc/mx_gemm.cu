@@ -43,7 +43,8 @@ constexpr int BK = 128;         // K elements per pipeline stage: 4 MX blocks, 4
 constexpr int kMmaK = 32;       // K of one kind::mxf8f6f4 MMA = the MX block size
 constexpr int kThreads = 384;   // 12 warps: producer, MMA issuer, 8 epilogue warps, scale copier, scale producer
 constexpr int kTmemCols = 512;  // whole tensor memory of the SM (one CTA per SM)
-constexpr long long kSpinLimit = 2000000000LL;  // cycles (~1 s) before a wait gives up
+constexpr long long kSpinLimit = 2000000000LL;  // default budget of a wait in cycles (~1 s)
+constexpr uint32_t kNoDrop = 0xFFFFFFFFu;       // "failure drill off" value of the drop_fill argument
 
 enum : unsigned int {
   ST_OK = 0,
@@ -110,16 +111,18 @@ __device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
       : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
   return ok != 0;
 }
-// Bounded wait: false if the abort flag was raised or the cycle budget ran out.
+// Bounded wait: false if the abort flag was raised or the cycle budget `limit` ran out.  Waits for
+// one pipeline stage get the kernel's budget; waits for a whole tile (the accumulator hand-overs)
+// get four times as much, so that when a stage never arrives it is the stage wait that reports it.
 __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity,
-                                          const volatile uint32_t* abort_flag) {
+                                          const volatile uint32_t* abort_flag, long long limit) {
   if (mbar_try_wait(bar, parity)) return true;
   const long long t0 = clock64();
   for (uint32_t it = 1;; ++it) {
     if (mbar_try_wait(bar, parity)) return true;
     if ((it & 31u) == 0) {
       if (*abort_flag != 0) return false;
-      if (clock64() - t0 > kSpinLimit) return false;
+      if (clock64() - t0 > limit) return false;
     }
   }
 }
@@ -410,7 +413,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
                const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                const __grid_constant__ CUtensorMap tmap_c,
                uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch) {
+               uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch,
+               long long spin_limit, uint32_t drop_fill) {
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -470,7 +474,9 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     // ------------------------------ TMA producer ------------------------------
     // The two operand copies of a stage; the scale chunks have a producer warp of their own (warp
     // 11).  The whole warp runs the loop converged and one elected lane issues (see elect_one).
-    uint32_t stage = 0, phase = 0;
+    // Failure drill (drop_fill != kNoDrop): the fill with that running number is left out -- no copy
+    // is issued and its barrier is not armed -- so that the MMA issuer's wait for it runs out.
+    uint32_t stage = 0, phase = 0, fill = 0;
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
       const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
@@ -479,12 +485,12 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // their columns are not stored.
       const int cy_a = (int)((tc.b * tiles_m + tc.tm) * BM), cy_b = (int)(tc.b * N + tc.tn * BN);
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_PRODUCER_WAIT);
           break;
         }
-        if (elect_one()) {
+        if (fill++ != drop_fill && elect_one()) {
           const uint32_t fb = full_bar(stage);
           mbar_arrive_expect_tx(fb, tx_bytes);
           tma_load_3d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BKe), cy_a, 0, fb);
@@ -504,7 +510,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
-      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, 4 * spin_limit))) {
         raise_abort(abort_flag, ST_MMA_WAIT_ACC);
         break;
       }
@@ -514,8 +520,8 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       const uint32_t sfb_col = 4 + ((tile_coord(t, tiles_m, tiles_n, group_m).tn * BN) % 128) / 32;
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
         // scales in tensor memory, then the operands
-        ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag)) &&
-                                         mbar_wait(full_bar(stage), phase, abort_flag));
+        ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag, spin_limit)) &&
+                                         mbar_wait(full_bar(stage), phase, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_MMA_WAIT_FULL);
           break;
@@ -552,7 +558,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       bool ok = true;
       for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag, spin_limit));
           if (!ok) {
             raise_abort(abort_flag, ST_SCALE_WAIT);
             break;
@@ -584,7 +590,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
         const int cz_a = (int)(tc.b * tiles_m + tc.tm), cz_b = (int)((tc.b * N + tc.tn * BN) / 128);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
           if (!ok) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             break;
@@ -615,7 +621,7 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     uint32_t acc = 0, acc_phase = 0;
     for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x) {
       const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-      if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) {
+      if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, 4 * spin_limit)) {
         if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
         break;
       }
@@ -685,7 +691,8 @@ __global__ void __launch_bounds__(kThreads, 1)
 mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                       const __grid_constant__ CUtensorMap tmap_sw, const __grid_constant__ CUtensorMap tmap_sx,
                       void* __restrict__ C, uint32_t M, uint32_t N, uint32_t K, uint32_t MP,
-                      uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t c_bf16) {
+                      uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t c_bf16,
+                      long long spin_limit, uint32_t drop_fill) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -745,16 +752,16 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
     // The tile's 128 rows of B and all MP rows of A (or their scale chunks).  Rows past N or M are
     // zero-filled by the copy: zero codes, value +0.  The warp runs converged, one elected lane issues.
     const bool scales = warp == 11;
-    uint32_t stage = 0, phase = 0;
+    uint32_t stage = 0, phase = 0, fill = 0;  // drop_fill: see the operand producer of mx_gemm_kernel
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_PRODUCER_WAIT);
           break;
         }
-        if (elect_one()) {
+        if ((scales || fill++ != drop_fill) && elect_one()) {
           if (scales) {  // (0, K chunk, 128-row group)
             const uint32_t fb = sf_full_bar(stage);
             mbar_arrive_expect_tx(fb, 1024u);
@@ -781,7 +788,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_SCALE_WAIT);
           break;
@@ -803,15 +810,15 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
     uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
     bool ok = true;
     for (uint32_t t = blockIdx.x; t < tiles_n && ok; t += gridDim.x) {
-      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag))) {
+      if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar(acc), acc_phase ^ 1u, abort_flag, 4 * spin_limit))) {
         raise_abort(abort_flag, ST_MMA_WAIT_ACC);
         break;
       }
       tc_fence_after();
       const uint32_t d_tmem = tmem_base + acc * 128u;
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(sf_ready_bar(stage), phase, abort_flag) &&
-                                         mbar_wait(full_bar(stage), phase, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(sf_ready_bar(stage), phase, abort_flag, spin_limit) &&
+                                         mbar_wait(full_bar(stage), phase, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_MMA_WAIT_FULL);
           break;
@@ -841,7 +848,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
     const uint32_t quarter = warp & 3u;  // TMEM lanes this warp may read: 32 * quarter .. + 31
     uint32_t acc = 0, acc_phase = 0;
     for (uint32_t t = blockIdx.x; t < tiles_n; t += gridDim.x) {
-      if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag)) {
+      if (!mbar_wait(acc_full_bar(acc), acc_phase, abort_flag, 4 * spin_limit)) {
         if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
         break;
       }
@@ -945,7 +952,12 @@ struct Cfg2 {
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
 };
 
-constexpr uint32_t kPeerMask = 0xFEFFFFFFu;  // clears the CTA-rank bit of a shared::cluster address
+// shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster.
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t saddr, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(saddr), "r"(rank));
+  return r;
+}
 
 __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap* map, int x, int y,
                                                  int z, uint32_t bar) {
@@ -998,8 +1010,9 @@ __device__ __forceinline__ void tc_mma_pair_dense(uint32_t d_tmem, uint64_t ades
       "}"
       ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate) : "memory");
 }
-__device__ __forceinline__ void mbar_arrive_leader(uint32_t bar) {
-  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar & kPeerMask) : "memory");
+// bar: shared::cluster address of a barrier (here: the leader CTA's, see leader_bar in the kernel)
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t bar) {
+  asm volatile("mbarrier.arrive.shared::cluster.b64 _, [%0];" ::"r"(bar) : "memory");
 }
 __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
@@ -1013,7 +1026,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
                     uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
-                    uint32_t batch) {
+                    uint32_t batch, long long spin_limit, uint32_t drop_fill) {
   using cfg = Cfg2<KIND, BN_>;
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
   constexpr int BN = cfg::BN;
@@ -1038,6 +1051,10 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
+  // the leader CTA's copy of one of the barriers above, as a shared::cluster address (both CTAs
+  // use the same shared-memory layout, so it is the mapped base plus the barrier's offset)
+  const uint32_t bar0_leader = map_to_cta(bar0, 0);
+  auto leader_bar = [&](uint32_t local_bar) { return bar0_leader + (local_bar - bar0); };
 
   uint32_t rank;
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
@@ -1080,7 +1097,8 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     // ------------------------- TMA producer (both CTAs) -------------------------
     // Operand tiles only: the scale chunks have a producer warp of their own (below).  The whole
     // warp runs the loop converged and one elected lane issues the copies (see elect_one).
-    uint32_t stage = 0, phase = 0;
+    // drop_fill: see the operand producer of mx_gemm_kernel (both CTAs leave out the same fill).
+    uint32_t stage = 0, phase = 0, fill = 0;
     bool ok = true;
     for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
       const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
@@ -1091,13 +1109,13 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const int cy_b = (int)(tc.b * N + tc.tn * BN + rank * 128);
       const int cy_b2 = (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+        ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
         if (!ok) {
           raise_abort(abort_flag, ST_PRODUCER_WAIT);
           break;
         }
-        if (elect_one()) {
-          const uint32_t fb = full_bar(stage) & kPeerMask;  // the leader's barrier
+        if (fill++ != drop_fill && elect_one()) {
+          const uint32_t fb = leader_bar(full_bar(stage));
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
           const int cx = (int)(kc * BKe);
           tma_load_3d_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, cx, cy_a, 0, fb);
@@ -1120,15 +1138,15 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       uint32_t stage = 0, phase = 0, acc_phase = 0;
       bool ok = true;
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-        if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag))) {
+        if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag, 4 * spin_limit))) {
           raise_abort(abort_flag, ST_MMA_WAIT_ACC);
           break;
         }
         tc_fence_after();
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
           // scales in tensor memory, then the operands
-          ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag)) &&
-                                           mbar_wait(full_bar(stage), phase, abort_flag));
+          ok = __all_sync(0xffffffffu, (DENSE || mbar_wait(sf_ready_bar(stage), phase, abort_flag, spin_limit)) &&
+                                           mbar_wait(full_bar(stage), phase, abort_flag, spin_limit));
           if (!ok) {
             raise_abort(abort_flag, ST_MMA_WAIT_FULL);
             break;
@@ -1185,7 +1203,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         bool ok = true;
         for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
           for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-            ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag));
+            ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag, spin_limit));
             if (!ok) {
               raise_abort(abort_flag, ST_SCALE_WAIT);
               break;
@@ -1226,13 +1244,13 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         const int cz_a = (int)((tc.b * tiles_m + tc.tm) * 2 + rank);
         const int cz_b = (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag));
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
           if (!ok) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
             break;
           }
           if (elect_one()) {
-            const uint32_t fb = sf_full_bar(stage) & kPeerMask;
+            const uint32_t fb = leader_bar(sf_full_bar(stage));
             if (rank == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * cfg::kSfBytes);
             const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
             tma_load_3d_pair(dst, &tmap_sa, 0, (int)(kc * cfg::kKChunks), cz_a, fb);
@@ -1255,7 +1273,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     uint32_t acc_phase = 0;
     for (uint32_t t = pair; t < num_tiles; t += num_pairs) {
       const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
-      if (!mbar_wait(acc_full_bar, acc_phase, abort_flag)) {
+      if (!mbar_wait(acc_full_bar, acc_phase, abort_flag, 4 * spin_limit)) {
         if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
         break;
       }
@@ -1279,7 +1297,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           if (pass == 1) {
             tc_fence_before();
             __syncwarp();
-            if (lane == 0) mbar_arrive_leader(acc_empty_bar);
+            if (lane == 0) mbar_arrive_cluster(leader_bar(acc_empty_bar));
           }
           store_rows<kPassLoads>(r, smem_base + cfg::kOffEpi + (warp - 2u) * kEpiBufs * kEpiChunkBytes, &tmap_c,
                                  (int)col0, (int)row0, valid_cols, lane, epi.mode);
@@ -1295,7 +1313,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
         tc_wait_ld();
         tc_fence_before();
         __syncwarp();
-        if (lane == 0) mbar_arrive_leader(acc_empty_bar);  // accumulator rows of this CTA are in registers
+        if (lane == 0) mbar_arrive_cluster(leader_bar(acc_empty_bar));  // accumulator rows of this CTA are in registers
         if (epi.mode == 2) {
           if (valid_cols) store_mx_rows<kLoads>(r, epi, row0 + lane, col0, N);
         } else {
@@ -1343,6 +1361,51 @@ EncodeTiledFn encode_fn_cached() {
   return encode_fn(&e);
 }
 
+// Encoding a tensor map is a driver call of about a microsecond, and a GEMM needs five or six; a
+// layer that is called again with the same buffers (every step of a training or decoding loop)
+// asks for the very same maps.  The encoder's result depends on its arguments only (address,
+// extents, strides, box, type, swizzle), so the last results are kept per thread, keyed on all of
+// them, in a small direct-mapped table; a repeated GEMM then makes no driver call at all.
+struct MapKey {
+  uint64_t ptr, dims[3], strides[2];
+  uint32_t box[3], dtype, rank, swizzle, promo, pad;
+  bool operator==(const MapKey& o) const { return std::memcmp(this, &o, sizeof(MapKey)) == 0; }
+};
+struct MapSlot {
+  MapKey key;
+  CUtensorMap map;
+  bool used;
+};
+constexpr int kMapSlots = 64;
+
+bool encode_cached(EncodeTiledFn fn, CUtensorMap* map, CUtensorMapDataType dt, uint32_t rank, const void* ptr,
+                   const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                   CUtensorMapSwizzle swz, CUtensorMapL2promotion promo) {
+  static thread_local MapSlot slots[kMapSlots];
+  MapKey k;
+  std::memset(&k, 0, sizeof(k));
+  k.ptr = (uint64_t)(uintptr_t)ptr;
+  for (uint32_t i = 0; i < rank; ++i) { k.dims[i] = dims[i]; k.box[i] = box[i]; }
+  for (uint32_t i = 0; i + 1 < rank; ++i) k.strides[i] = strides[i];
+  k.dtype = (uint32_t)dt; k.rank = rank; k.swizzle = (uint32_t)swz; k.promo = (uint32_t)promo;
+  uint64_t h = 1469598103934665603ull;  // FNV-1a over the key
+  const unsigned char* b = reinterpret_cast<const unsigned char*>(&k);
+  for (size_t i = 0; i < sizeof(k); ++i) h = (h ^ b[i]) * 1099511628211ull;
+  MapSlot& slot = slots[h % kMapSlots];
+  if (slot.used && slot.key == k) {
+    *map = slot.map;
+    return true;
+  }
+  const cuuint32_t estr[3] = {1, 1, 1};
+  if (fn(map, dt, rank, const_cast<void*>(ptr), dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, swz,
+         promo, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return false;
+  slot.key = k;
+  slot.map = *map;
+  slot.used = true;
+  return true;
+}
+
 int fmt_bits(int f) { return f == MX_E2M1 ? 4 : ((f == MX_E3M2 || f == MX_E2M3) ? 6 : 8); }
 
 // Format field of the instruction descriptor.
@@ -1368,10 +1431,8 @@ bool make_operand_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, int f
   const cuuint64_t dims[3] = {K, rows, 1};
   const cuuint64_t strides[2] = {pitch, pitch * rows};
   const cuuint32_t box[3] = {(cuuint32_t)BK, box_rows, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, dt, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, dt, 3, ptr, dims, strides, box, CU_TENSOR_MAP_SWIZZLE_128B,
+                       CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Tensor map of a dense BF16 K-major operand [rows x K]: box = 64 elements (128 bytes) x box_rows.
@@ -1380,10 +1441,8 @@ bool make_dense_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_
   const cuuint64_t dims[3] = {K, rows, 1};
   const cuuint64_t strides[2] = {K * 2, K * 2 * rows};
   const cuuint32_t box[3] = {64, box_rows, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, ptr, dims, strides, box,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Tensor map over a swizzled scale tensor seen as [row groups of 128][K chunks][128 words]:
@@ -1394,10 +1453,8 @@ bool make_scale_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_
   const cuuint64_t dims[3] = {128, k_chunks, (rows + 127) / 128};
   const cuuint64_t strides[2] = {512, 512 * k_chunks};
   const cuuint32_t box[3] = {128, 1, groups};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, ptr, dims, strides, box,
+                       CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 // Tensor map of the output [M x N] (FP32 or BF16): box = 64 bytes of columns x 32 rows in the
@@ -1406,10 +1463,8 @@ bool make_c_map(EncodeTiledFn fn, CUtensorMap* map, void* C, uint64_t M, uint64_
   const cuuint64_t dims[2] = {N, M};
   const cuuint64_t strides[1] = {N * (bf16 ? 2u : 4u)};
   const cuuint32_t box[2] = {bf16 ? 32u : kEpiChunkCols, 32};
-  const cuuint32_t estr[2] = {1, 1};
-  return fn(map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C, dims,
-            strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
-            CU_TENSOR_MAP_L2_PROMOTION_NONE, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, bf16 ? CU_TENSOR_MAP_DATA_TYPE_BFLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, C,
+                       dims, strides, box, CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE);
 }
 
 // The output map the kernels take.  A quantizing epilogue writes with plain stores and never uses
@@ -1425,6 +1480,9 @@ bool make_out_map(EncodeTiledFn fn, CUtensorMap* map, const GemmArgs& a) {
 bool small_product(const GemmArgs& a) {
   return (double)a.batch * (double)a.M * (double)a.N * (double)a.K < 4.0e9;
 }
+
+long long wait_budget(const GemmArgs& a) { return a.wait_cycles > 0 ? (long long)a.wait_cycles : kSpinLimit; }
+uint32_t drop_fill(const GemmArgs& a) { return a.drop_fill >= 0 ? (uint32_t)a.drop_fill : kNoDrop; }
 
 EpiArgs epi_args(const GemmArgs& a) {
   EpiArgs e;
@@ -1472,7 +1530,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   return launch_pdl_if(small_product(a), mx_gemm_kernel<BN, DENSE>, dim3(grid), dim3(kThreads), cfg::kSmemBytes, a.stream,
                     ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
                     idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, epi_args(a),
-                    (uint32_t)a.batch);
+                    (uint32_t)a.batch, wait_budget(a), drop_fill(a));
 }
 
 // Dense FP4 operand map for kind::mxf4: two codes per byte in shared memory as in global memory.
@@ -1482,10 +1540,8 @@ bool make_f4_map(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint64_t r
   const cuuint64_t dims[3] = {K, rows, 1};
   const cuuint64_t strides[2] = {pitch, pitch * rows};
   const cuuint32_t box[3] = {256, box_rows, 1};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN8B, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_256B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, CU_TENSOR_MAP_DATA_TYPE_16U4_ALIGN8B, 3, ptr, dims, strides, box,
+                       CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B);
 }
 
 // Scale map whose box also spans `kchunks` K chunks: [row groups][K chunks][128 words].
@@ -1495,10 +1551,8 @@ bool make_scale_map_k(EncodeTiledFn fn, CUtensorMap* map, const void* ptr, uint6
   const cuuint64_t dims[3] = {128, k_chunks, (rows + 127) / 128};
   const cuuint64_t strides[2] = {512, 512 * k_chunks};
   const cuuint32_t box[3] = {128, kchunks, groups};
-  const cuuint32_t estr[3] = {1, 1, 1};
-  return fn(map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, const_cast<void*>(ptr), dims, strides, box, estr,
-            CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE,
-            CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+  return encode_cached(fn, map, CU_TENSOR_MAP_DATA_TYPE_UINT32, 3, ptr, dims, strides, box,
+                       CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_128B);
 }
 
 template <int KIND, int BN>
@@ -1552,7 +1606,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
                          ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
   return launch_pdl_if(small_product(a), mx_gemm_pair_kernel<KIND, BN>, dim3(2 * pairs), dim3(kThreads), cfg::kSmemBytes, a.stream,
                     ma, mb, mb2, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
-                    epi_args(a), (uint32_t)a.batch);
+                    epi_args(a), (uint32_t)a.batch, wait_budget(a), drop_fill(a));
 }
 
 // M <= 128: operands swapped (see mx_gemm_skinny_kernel).
@@ -1586,7 +1640,8 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t idesc = (mma_fmt_code(a.fmtB) << 7) | (mma_fmt_code(a.fmtA) << 10) | (1u << 23) |
                          ((MP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   return launch_pdl_if(small_product(a), mx_gemm_skinny_kernel, dim3(grid), dim3(kThreads), smem, a.stream, mw, mx_, msw, msx, a.C,
-                    (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, a.c_bf16 ? 1u : 0u);
+                    (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, a.c_bf16 ? 1u : 0u,
+                    wait_budget(a), drop_fill(a));
 }
 
 }  // namespace

@@ -75,6 +75,8 @@ struct GemmArgs {
   int fmtA, fmtB;
   int force_bn;  // 0: let launch_gemm choose the tile width; 256 / 384: pin it (tuning and tests)
   int skinny_m;  // products with M <= skinny_m (at most 128) take the swapped-operand kernel
+  int64_t wait_cycles;  // budget of a device-side wait in SM clock cycles; <= 0: the default (~1 s)
+  int drop_fill;        // failure drill: the operand producer leaves out this pipeline fill; < 0: off
   int sm_count;
   cudaStream_t stream;
 };

@@ -127,6 +127,15 @@ def test_gemm_variants_argument_validation_without_gpu():
     assert bt(p, p, p, p, p, F32, -1, 128, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
     assert bt(p, p, p, p, p, F32, 1 << 30, 128, 128, 128, 0, 0, None) == mx.MX_ERR_SHAPE
     assert bt(p, p, p, p, p, BF16, 0, 128, 128, 128, 0, 0, None) == mx.MX_OK         # empty batch
+    ge = lib.mx_gemm_ex
+    P = mx.binding.mx_gemm_plan_t
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, None) == ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(0, 0, -1, -1, 0)))
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(2, 0, -1, -1, 0))) == mx.MX_ERR_FMT
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(0, 320, -1, -1, 0))) == mx.MX_ERR_SHAPE
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(0, 0, 129, -1, 0))) == mx.MX_ERR_SHAPE
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(0, 0, -1, -2, 0))) == mx.MX_ERR_SHAPE
+    assert ge(p, p, p, p, p, 128, 128, 128, 0, 0, None, ctypes.byref(P(0, 0, -1, -1, -5))) == mx.MX_ERR_SHAPE
+    assert ge(p, p, p, p, p, 128, 132, 128, 0, 0, None, ctypes.byref(P(1, 0, -1, -1, 0))) == mx.MX_ERR_SHAPE  # BF16 rows: N % 8
     gq = lib.mx_gemm_quantize
     assert gq(p, p, p, p, None, p, 128, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_NULL
     assert gq(p, p, p, p, p, None, 128, 128, 128, 0, 0, 0, 0, None) == mx.MX_ERR_NULL

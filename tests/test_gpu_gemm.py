@@ -139,17 +139,16 @@ def test_few_rows_against_oracle(M, N, K, fa, fb, dt):
 
 
 @pytest.mark.parametrize("M,N,K,fa,fb", [(64, 1024, 512, 0, 0), (17, 19200, 256, 4, 1), (96, 640, 1024, 2, 3)])
-def test_few_rows_kernel_equals_tiled_kernel(M, N, K, fa, fb, monkeypatch):
-    """The same product through the swapped-operand kernel and (threshold pinned to 0 through the
-    environment) through the 128-row tiles: bit-identical outputs."""
+def test_few_rows_kernel_equals_tiled_kernel(M, N, K, fa, fb):
+    """The same product through the swapped-operand kernel and (mx_gemm_ex with the threshold
+    pinned to 0) through the 128-row tiles: bit-identical outputs."""
     g = torch.Generator(device="cuda").manual_seed(M * N + K)
     A = torch.randn((M, K), generator=g, device="cuda")
     B = torch.randn((N, K), generator=g, device="cuda")
     ea, sa = mx.mx_quantize(A, 1, fa)
     eb, sb = mx.mx_quantize(B, 1, fb)
     C1 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
-    monkeypatch.setenv("MX_GEMM_SKINNY_M", "0")
-    C2 = mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, check_status=True)
+    C2 = mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, few_rows_limit=0, check_status=True)
     torch.cuda.synchronize()
     assert torch.equal(C1, C2)
     assert C1.abs().max().item() > 0
@@ -701,6 +700,75 @@ def test_config5_full_size():
     del d, W, X
     torch.cuda.empty_cache()
     _full_size_check("config 5", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, 5)
+
+
+@pytest.mark.parametrize("fa,fb,K,dt", [(0, 0, 640, torch.float32), (4, 4, 512, torch.float32), (2, 0, 384, torch.bfloat16)])
+def test_wide_tile_variant_whole_matrix(fa, fb, K, dt):
+    """The 256 x 384 tile of the two-CTA kernel (mx_gemm_ex, tile_n = 384) on a shape with a ragged
+    last tile: whole matrix against the FP64 product of the oracle-dequantized operands, samples
+    against the oracle, and bit-identical to the default 256 x 256 tiles."""
+    M, N = 2048, 9608
+    g = torch.Generator(device="cuda").manual_seed(K + fa)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.02
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(M * N * esz)
+    C = g_out.view.view(dt).view(M, N)
+    mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, out=C, tile_n=384, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    ref = da @ db.T
+    fac, rel = _bound_terms(dt)
+    bad = int(((C.double() - ref).abs() > fac * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+    assert bad == 0, f"{bad} outputs beyond the bound"
+    rng = np.random.default_rng(K)
+    ms = np.concatenate([rng.integers(0, M, 1000), np.full(200, M - 1)])
+    ns = np.concatenate([rng.integers(0, N, 1000), rng.integers(N - 40, N, 200)])
+    c64, s_ = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= fac * TOL * s_ + np.abs(c64) * rel).all()
+    C0 = mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, out_dtype=dt, check_status=True)   # 256 x 256 tiles
+    assert torch.equal(C0, C)
+
+
+@pytest.mark.parametrize("M,N,K,fa,fb,drop", [
+    (256, 256, 1024, 0, 0, 2),     # one-CTA kernel, 128 x 128 tiles
+    (1024, 4096, 512, 0, 4, 1),    # two-CTA kernel
+    (16, 1024, 1024, 0, 0, 3),     # few rows of A: operands swapped
+])
+def test_device_wait_runs_out_and_context_survives(M, N, K, fa, fb, drop):
+    """Failure detection without a GPU fault: the operand producer is told to leave out one pipeline
+    fill (nothing is copied for it, so nothing is in flight later) and every device-side wait gets
+    a budget of about a millisecond.  The MMA issuer's wait for that stage must run out, the kernel
+    must leave through its common exit (tensor memory released), the checked call must return
+    MX_ERR_TIMEOUT naming that wait, and the very next ordinary product on the same context must
+    be right against the oracle."""
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    A = torch.randn((M, K), generator=g, device="cuda")
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.1
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    torch.cuda.synchronize()
+    with pytest.raises(mx.MxError) as ei:
+        mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, wait_cycles=2_000_000, drop_fill=drop, check_status=True)
+    assert ei.value.status == mx.MX_ERR_TIMEOUT
+    assert "wait 2 gave up" in str(ei.value), str(ei.value)       # 2 = MMA issuer / stage full
+    # the status word was cleared by the failed check; the context and the tensor memory are usable
+    g_out = Guarded(M * N * 4)
+    C = g_out.view.view(torch.float32).view(M, N)
+    mx.mx_gemm(ea, sa, eb, sb, M, N, K, fa, fb, out=C, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    c64, s_ = O.gemm(*(t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb)), M, N, K, fa, fb)
+    assert (np.abs(C.double().cpu().numpy() - c64) <= TOL * s_).all()
+    # a budget without a drill changes nothing
+    C2 = mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, wait_cycles=2_000_000_000, check_status=True)
+    assert torch.equal(C, C2)
 
 
 def test_host_buffer_gemm():

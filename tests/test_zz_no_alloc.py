@@ -61,7 +61,7 @@ def test_static_scratch_call_allocates_no_device_memory():
     with another shape that leaves stale bytes behind.  Host outputs are pinned beforehand, so
     nothing else in the measured window can allocate."""
     x = inputs.adversarial("cpu", rows=256, cols=512, dtype=torch.bfloat16, seed=33).pin_memory()
-    y = inputs.adversarial("cpu", rows=128, cols=300, dtype=torch.bfloat16, seed=35)[:, :300].contiguous().pin_memory()
+    y = inputs.adversarial("cpu", rows=128, cols=320, dtype=torch.bfloat16, seed=35)[:, :300].contiguous().pin_memory()
     ex, sx = _host_outputs(list(x.shape), 1, mx.MX_E4M3, mx.MX_SCALES_SWIZZLED)
     ey, sy = _host_outputs(list(y.shape), 1, mx.MX_E4M3, mx.MX_SCALES_SWIZZLED)
     torch.zeros(1, device="cuda")            # the CUDA context and torch's pool exist before measuring
