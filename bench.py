@@ -224,7 +224,7 @@ class Workload:
 def run_e2e(torch, mx, inputs, steps: int, warmup: int):
     """The sweep through the host-buffer entry points: pinned host tensors in, pinned host
     results out, every copy inside the timed region."""
-    T = inputs.config2("cpu", 2048, SWEEP_COLS, seed=2002).pin_memory()  # a quarter of the sweep tensor
+    T = inputs.config2("cpu", SWEEP_ROWS, SWEEP_COLS, seed=2002).pin_memory()  # the whole sweep tensor
     rows, cols = T.shape
     shape = [rows, cols]
     n = rows * cols
@@ -267,14 +267,48 @@ def run_e2e(torch, mx, inputs, steps: int, warmup: int):
     total_bytes = 2.0 * sum(algorithmic_bytes(n, 2, b) for b in FMT_BITS)
     return {"value": total_bytes / dt / 1e9, "unit": "GB/s", "h2d_bytes_per_step": h2d,
             "d2h_bytes_per_step": d2h, "ms_per_step": dt * 1e3,
-            "workload": f"sweep on a {rows}x{cols} BF16 slice via mx_quantize_host_async / "
+            "workload": f"configs[1] sweep on the whole {rows}x{cols} BF16 tensor via mx_quantize_host_async / "
                         "mx_dequantize_host_async + mx_host_synchronize (pinned host buffers, copies timed)"}
 
 
-def run_extras(torch, mx, inputs):
+def run_extras(torch, mx, inputs, peaks, gpu_index):
     """The other benchmark configurations, outside the timed step: the FP4-weight x FP8-activation
     GEMM (16384 x 28672 x 8192), the same shape with both operands FP4 (kind::mxf4), and the
-    MXFP6 training step of one 4096^3 linear layer (six quantizes, three GEMMs)."""
+    MXFP6 training step of one 4096^3 linear layer (six quantizes, three GEMMs).  Returns
+    (other_configs, gemm_rooflines): the second holds, per configuration, the burst figure against
+    2 x the measured BF16 burst peak and -- for configurations 3 and 5 -- a loop of at least two
+    seconds of back-to-back launches against 2 x the measured sustained BF16 peak, with the SM
+    clock and board power sampled inside that loop."""
+    fp8_burst, fp8_sust = 2.0 * peaks["bf16_tflops"], 2.0 * peaks["bf16_tflops_sustained"]
+    rooflines = {}
+
+    def burst_entry(flops, seconds):
+        tf = flops / seconds / 1e12
+        return {"TFLOPs": tf, "ms": seconds * 1e3, "frac_of_2x_bf16_burst": tf / fp8_burst,
+                "frac_of_nominal_4500": tf / 4500.0}
+
+    def sustained(fn, flops, t_one, seconds=2.2):
+        """fn() queued back to back for >= `seconds`; clocks and power from the samples inside."""
+        n = max(4, int(seconds / t_one) + 1)
+        sampler = ClockSampler(gpu_index)
+        time.sleep(0.3)                      # the sampler is polling before the loop starts
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        sampler.begin()
+        e0.record()
+        for _ in range(n):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        sampler.end()
+        clk = sampler.stop()
+        sec = e0.elapsed_time(e1) * 1e-3
+        tf = flops * n / sec / 1e12
+        return {"TFLOPs": tf, "seconds": sec, "launches": n, "frac_of_2x_bf16_sustained": tf / fp8_sust,
+                "frac_of_nominal_4500": tf / 4500.0, "sm_mhz_median": clk.get("sm_mhz"),
+                "power_w_median": clk.get("power_w_median"), "power_w_max": clk.get("power_w_max"),
+                "clock_samples": clk.get("samples"), "reasons": clk.get("reasons")}
+
     def timed(fn, reps):
         fn()
         torch.cuda.synchronize()
@@ -297,6 +331,9 @@ def run_extras(torch, mx, inputs):
     t_qx = timed(lambda: mx.mx_quantize(X, 1, mx.MX_E4M3, out=(ea, sa)), 5)
     C = torch.empty((M, N), dtype=torch.float32, device="cuda")
     t = timed(lambda: mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, out=C), 5)
+    rooflines["config5"] = {"workload": "configs[4] E4M3 x E2M1 16384x28672x8192, FP32 out",
+                            "burst": burst_entry(2.0 * M * N * K, t)}
+    c5 = (ea, sa, eb, sb, C, M, N, K, t)
     out["config5_mxfp4_weights_x_mxfp8_activations"] = {
         "gemm_TFLOPs": 2.0 * M * N * K / t / 1e12, "gemm_ms": t * 1e3,
         "quantize_w_strided_GBps": algorithmic_bytes(K * N, 2, 4) / t_qw / 1e9,
@@ -304,7 +341,7 @@ def run_extras(torch, mx, inputs):
     ea4, sa4 = mx.mx_quantize(X, 1, mx.MX_E2M1)
     t4 = timed(lambda: mx.mx_gemm(ea4, sa4, eb, sb, M, N, K, mx.MX_E2M1, mx.MX_E2M1, out=C), 5)
     out["mxfp4_x_mxfp4_same_shape_kind_mxf4"] = {"gemm_TFLOPs": 2.0 * M * N * K / t4 / 1e12, "gemm_ms": t4 * 1e3}
-    del d, W, X, C, ea, sa, eb, sb, ea4, sa4
+    del d, W, X, ea4, sa4
     torch.cuda.empty_cache()
     # two chained products (configs[2] shape): the first one's result requantized to MXFP8 for the next
     d = inputs.config3("cuda")
@@ -315,6 +352,10 @@ def run_extras(torch, mx, inputs):
     eb, sb = mx.mx_quantize(W, 0, mx.MX_E4M3)
     C = torch.empty((M, N), dtype=torch.float32, device="cuda")
     qe, qs = mx.mx_quantize(C, 1, mx.MX_E4M3)
+    t3 = timed(lambda: mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=C), 10)
+    rooflines["config3"] = {"workload": "configs[2] E4M3 x E4M3 8192x16384x4096, FP32 out",
+                            "burst": burst_entry(2.0 * M * N * K, t3)}
+    c3 = (ea, sa, eb, sb, C, M, N, K, t3)
 
     def gemm_then_quantize():
         mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E4M3, out=C)
@@ -359,7 +400,7 @@ def run_extras(torch, mx, inputs):
                                         workspace=ws, out=C), 10)
     out["config3_mxint8_x_mxint8_bf16_route"] = {
         "ms_two_dequantizes_and_dense_gemm": t8 * 1e3, "TFLOPs": 2.0 * M * N * K / t8 / 1e12}
-    del d, W, X, C, Cb, ea, sa, eb, sb, qe, qs, ea8, sa8, eb8, sb8, ws
+    del d, W, X, Cb, qe, qs, ea8, sa8, eb8, sb8, ws
     torch.cuda.empty_cache()
     d = inputs.config4("cuda")
     Xc, Wc, dY = d["X"], d["W"], d["dY"]
@@ -391,7 +432,23 @@ def run_extras(torch, mx, inputs):
     out["config4_mxfp6_training_step"] = {
         "ms_six_quantizes_three_gemms": ts * 1e3, "ms_three_dual_quantizes_three_gemms": tf * 1e3,
         "gemm_flops_per_step": 3 * 2.0 * n ** 3}
-    return out
+    # the three products of the step, each on its own (operands quantized beforehand)
+    (xa, xt), (wb2, wb), (ga, gt) = (mx.mx_quantize_dual(Xc, act, rnd), mx.mx_quantize_dual(Wc, wt, rnd),
+                                     mx.mx_quantize_dual(dY, act, rnd))
+    c4 = {}
+    for name, a_, b_, fb_ in (("forward", xa, wb, wt), ("dgrad", ga, wb2, wt), ("wgrad", xt, gt, act)):
+        tt = timed(lambda: mx.mx_gemm(*a_, *b_, n, n, n, act, fb_, out=Y), 20)
+        c4[name] = burst_entry(2.0 * n ** 3, tt)
+    rooflines["config4"] = {"workload": "configs[3] MXFP6 4096^3: forward E3M2 x E2M3, dgrad E3M2 x E2M3, "
+                                        "wgrad E3M2 x E3M2, FP32 out", "burst": c4}
+    del d, Xc, Wc, dY, Y, xa, xt, wb2, wb, ga, gt
+    torch.cuda.empty_cache()
+    # last: the two-second loops
+    for key, (ea, sa, eb, sb, C, M, N, K, t_one), fb_ in (("config3", c3, mx.MX_E4M3), ("config5", c5, mx.MX_E2M1)):
+        time.sleep(1.0)
+        rooflines[key]["sustained"] = sustained(
+            lambda: mx.mx_gemm(ea, sa, eb, sb, M, N, K, mx.MX_E4M3, fb_, out=C), 2.0 * M * N * K, t_one)
+    return out, rooflines
 
 
 def run_report(torch, mx, inputs):
@@ -677,7 +734,9 @@ def main_ours(args, rank, world, local_rank):
         line["cpu_baseline"] = cpu
         del w
         torch.cuda.empty_cache()
-        line["other_configs"] = run_extras(torch, mx, inputs)
+        line["other_configs"], per_config = run_extras(torch, mx, inputs, peaks, local_rank)
+        line["roofline_gemm"]["per_config"] = per_config
+        line["roofline_gemm"]["sustained"] = {k: v["sustained"] for k, v in per_config.items() if "sustained" in v}
     else:
         line["e2e"] = None
     print(json.dumps(line))
