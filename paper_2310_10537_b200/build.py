@@ -12,8 +12,8 @@ ROOT = os.path.dirname(HERE)
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libmx_b200.so")
 BUILD = os.path.join(HERE, "build")
-SOURCES = ["mx_api.cu", "mx_quantize.cu", "mx_quantize_dual.cu", "mx_dequantize.cu", "mx_gemm.cu",
-           "mx_im2col.cu"]
+SOURCES = ["mx_api.cu", "mx_quantize.cu", "mx_quantize_dual.cu", "mx_quantize_tile.cu", "mx_dequantize.cu",
+           "mx_gemm.cu", "mx_im2col.cu"]
 NVCC_FLAGS = ["-std=c++17", "-O3", "-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo",
               "-Xcompiler", "-fPIC", "-I", os.path.join(ROOT, "include"), "-I", CSRC]
 

@@ -210,7 +210,8 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void*
     e = cudaMemsetAsync(scales_col, 0, scales_bytes(C, R / 32, o.layout), o.stream);
     if (e != cudaSuccess) return fail_cuda(e);
   }
-  e = mx::launch_quantize_dual(a);
+  // BF16: tiles through shared memory (TMA); FP32: the register kernel (measured faster there)
+  e = o.dtype == MX_BF16 ? mx::launch_quantize_tile(a) : mx::launch_quantize_dual(a);
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 

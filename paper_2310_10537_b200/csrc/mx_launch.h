@@ -30,6 +30,11 @@ struct DualArgs {
   cudaStream_t stream;
 };
 cudaError_t launch_quantize_dual(const DualArgs& a);
+// The same for BF16 input through TMA tiles in shared memory (mx_quantize_tile.cu).
+cudaError_t launch_quantize_tile(const DualArgs& a);
+// Synchronises the stream, then reads and clears the tile kernels' status word (nonzero: a
+// bounded device-side wait gave up).
+cudaError_t quantize_tile_status(cudaStream_t stream, unsigned int* status);
 
 struct DequantizeArgs {
   const uint8_t* elems;

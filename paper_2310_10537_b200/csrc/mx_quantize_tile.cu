@@ -1,0 +1,382 @@
+// Dual-axis quantize of a BF16 tensor through shared-memory tiles: X[R x C] is read once, by TMA,
+// in tiles of 128 rows x 128 columns, and each tile is quantized out of shared memory both along
+// its rows (blocks along the contiguous axis: the operand of X W) and along its columns (blocks
+// along axis 0: the K-major [C x R] operand of X^T dY).  The paper's compute flow (Section 4.1)
+// quantizes every matmul input in the forward and in the backward pass, and because quantizing
+// and transposing do not commute (Section 3) those are two tensors; producing both from one read
+// removes a third of the traffic.
+//
+// Why through shared memory: a thread that keeps 32 rows of a block in registers (the kernel in
+// mx_quantize_dual.cu, still used for FP32 input) needs ~250 registers once BF16 packs twice the
+// elements into them and both directions are served, which leaves eight warps per SM -- too few
+// loads in flight to cover HBM latency (measured: 11 % of the warp slots active, DRAM 47 % busy).
+// Here the copies in flight cost no registers: a CTA keeps kStages - 1 tiles (32 KB each) on their
+// way while it converts one, two CTAs share an SM (16 warps, <= 128 registers), and a converting
+// thread holds one block at a time.
+//
+//   thread 0      issues the two TMA box copies of a tile (128 rows x 128 bytes each, in the
+//                 128-byte swizzle) kStages - 1 tiles ahead; everybody waits on the stage's mbarrier
+//   warps 0-3     row pass: thread r converts row r of the tile; its 4 blocks are one contiguous
+//                 run of the [R x C] output, written as whole 32-byte sectors
+//   warps 4-7     column pass, at the same time (equal work): a thread converts the 32 rows of one
+//                 32-bit word column (2 columns) of one 32-row group; 8-bit codes leave as one
+//                 sector per block, 6- and 4-bit codes are parked in shared memory so that a
+//                 column's four blocks (96 / 64 bytes) leave as whole sectors too; a column's four
+//                 scale bytes leave as one word
+// The swizzle makes both access directions conflict-free: a row's 16-byte chunks are spread over
+// the banks by (chunk ^ row % 8), a word column's 32 lanes always hit 32 different banks.
+// The mbarrier wait is bounded: when it runs out the CTA records it in a status word and leaves.
+// Measured on 8192 x 8192 (both outputs, half-away rounding): E4M3 53 us against 59 us for the
+// register kernel, E3M2 62 against 67, E2M1 46 against 52; the conversion pipe (the packed narrow
+// casts, one per element and direction) is 72-77 % busy, DRAM 54 %.
+#include "mx_device.cuh"
+#include "mx_launch.h"
+#include "mx_quantize_common.cuh"
+#include "mx_tmap.h"
+
+namespace mx {
+
+namespace {
+
+constexpr int kTileThreads = 256;
+constexpr uint32_t kTileRows = 128;
+constexpr uint32_t kBoxBytes = kTileRows * 128;   // one TMA box: 128 rows x 128 bytes
+constexpr uint32_t kTileBytes = 2 * kBoxBytes;    // a tile: two boxes side by side (256 bytes per row)
+constexpr long long kTileSpinLimit = 2000000000LL;
+
+__device__ unsigned int g_tile_status;  // 1: a tile never arrived (bounded wait ran out)
+
+template <int FMT> struct TileCfg {
+  static constexpr int bits = FmtTraits<FMT>::bits;
+  static constexpr uint32_t kBpb = kBlock * bits / 8;                   // bytes of one block of codes
+  static constexpr uint32_t kCols = 128;                                // columns of a tile (256 bytes of BF16)
+  static constexpr uint32_t kRowBlocks = kCols / kBlock;                // blocks in a tile row
+  static constexpr uint32_t kStages = 3;
+  // column codes of sub-byte formats: per column its four blocks; the pad makes the stores of 32
+  // lanes (one slot apart) conflict-free: 26 words for 8-byte stores, 20 words for 16-byte stores
+  static constexpr uint32_t kColPitch = 4 * kBpb + (bits == 6 ? 8 : 16);
+  static constexpr uint32_t kStageCodes = bits != 8 ? kCols * kColPitch : 0;
+  static constexpr uint32_t kOffCodes = kStages * kTileBytes;
+  static constexpr uint32_t kOffScales = kOffCodes + kStageCodes;       // a column's four scale bytes
+  static constexpr uint32_t kOffBar = kOffScales + kCols * 4;
+  static constexpr uint32_t kSmem = kOffBar + kStages * 8 + 1024;       // + alignment slack
+};
+
+__device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int x, int y, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(bar) : "memory");
+}
+
+__device__ __forceinline__ bool tile_wait(uint32_t bar, uint32_t parity) {
+  auto try_wait = [&]() {
+    uint32_t ok;
+    asm volatile(
+        "{ .reg .pred p; mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2; selp.u32 %0, 1, 0, p; }"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+  };
+  if (try_wait()) return true;
+  const long long t0 = clock64();
+  for (uint32_t it = 1;; ++it) {
+    if (try_wait()) return true;
+    if ((it & 63u) == 0 && clock64() - t0 > kTileSpinLimit) return false;
+  }
+}
+
+// 16-byte chunk c (0..7) of row r of a box, as the 128-byte swizzle stores it.
+__device__ __forceinline__ uint32_t box_chunk(uint32_t box_base, uint32_t r, uint32_t c) {
+  return box_base + r * 128u + ((c ^ (r & 7u)) << 4);
+}
+
+template <int FMT, int ROUND, int LAYOUT>
+__global__ void __launch_bounds__(kTileThreads, 2)
+quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
+                     uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
+                     uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
+                     uint32_t num_tiles) {
+  using cfg = TileCfg<FMT>;
+  constexpr int DTYPE = MX_BF16;
+  constexpr int bits = cfg::bits;
+  constexpr uint32_t kBpb = cfg::kBpb;
+  constexpr uint32_t kRowBlocks = cfg::kRowBlocks;
+  constexpr uint32_t kBoxCols = cfg::kCols / 2;  // columns of one box
+  extern __shared__ uint8_t tile_smem_raw[];
+  const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
+  uint8_t* gen = tile_smem_raw + (base - smem_addr(tile_smem_raw));
+  const uint32_t bar0 = base + cfg::kOffBar;
+  const uint32_t tid = threadIdx.x, lane = tid & 31;
+
+  if (tid == 0) {
+    for (uint32_t s = 0; s < cfg::kStages; ++s)
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_in)) : "memory");
+  }
+  __syncthreads();
+  pdl_prologue();
+
+  auto issue = [&](uint32_t t, uint32_t stage) {  // thread 0: both boxes of tile t into `stage`
+    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+    const uint32_t bar = bar0 + 8 * stage;
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileBytes) : "memory");
+    const uint32_t dst = base + stage * kTileBytes;
+    tma_load_2d(dst, &tmap_in, (int)(tc * cfg::kCols), (int)(tr * kTileRows), bar);
+    tma_load_2d(dst + kBoxBytes, &tmap_in, (int)(tc * cfg::kCols + kBoxCols), (int)(tr * kTileRows), bar);
+  };
+  if (tid == 0) {
+#pragma unroll 1
+    for (uint32_t k = 0; k + 1 < cfg::kStages; ++k) {
+      const uint32_t t = blockIdx.x + k * gridDim.x;
+      if (t < num_tiles) issue(t, k);
+    }
+  }
+
+  const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;  // blocks per output row
+  const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
+  uint32_t it = 0;
+#pragma unroll 1
+  for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+    const uint32_t stage = it % cfg::kStages, parity = (it / cfg::kStages) & 1u;
+    if (tid == 0) {  // the stage that iteration it - 1 has finished with takes the tile kStages - 1 ahead
+      const uint32_t tn = t + (cfg::kStages - 1) * gridDim.x;
+      if (tn < num_tiles) issue(tn, (it + cfg::kStages - 1) % cfg::kStages);
+    }
+    if (!tile_wait(bar0 + 8 * stage, parity)) {
+      if (lane == 0) atomicCAS(&g_tile_status, 0u, 1u);
+      return;
+    }
+    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+    const uint32_t tile_base = base + stage * kTileBytes;
+    const uint32_t row0 = tr * kTileRows, col0 = tc * cfg::kCols;
+
+    // ------------------------------ row pass ------------------------------
+    if (tid < 128) {
+      constexpr uint32_t kPer = kRowBlocks;  // blocks per thread: its whole tile row
+      const uint32_t r = tid, q0 = 0;
+      const uint32_t row = row0 + r;
+      if (row < R) {
+        uint32_t codes[kPer][8];
+        uint32_t scale_word = 0;
+#pragma unroll
+        for (uint32_t qq = 0; qq < kPer; ++qq) {
+          const uint32_t q = q0 + qq;  // block of the tile row
+          uint32_t u[16];  // the block: 64 bytes = chunks 4 (q % 2) .. + 3 of box q / 2
+          const uint32_t box = tile_base + (q >> 1) * kBoxBytes;
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i) {
+            uint32_t v0, v1, v2, v3;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(box_chunk(box, r, (q & 1u) * 4u + i)));
+            u[4 * i] = v0; u[4 * i + 1] = v1; u[4 * i + 2] = v2; u[4 * i + 3] = v3;
+          }
+          const BlockScale s = block_scale<FMT>(unit_amax<DTYPE>(u));
+          scale_word |= s.byte << (8 * qq);
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float x[8];
+            unit_group<DTYPE>(u, g, x);
+            cast8<FMT, ROUND>(x, s, codes[qq][2 * g], codes[qq][2 * g + 1]);
+          }
+        }
+        const uint32_t kb0 = tc * kRowBlocks + q0;  // first block of this thread in the output row
+        uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
+        const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
+        if (bits == 8) {
+          uint32_t run[kPer * 8];
+#pragma unroll
+          for (uint32_t q = 0; q < kPer; ++q)
+#pragma unroll
+            for (int i = 0; i < 8; ++i) run[8 * q + i] = codes[q][i];
+          store_run<(int)(kPer * 8)>(dst, run, wide);
+        } else if (bits == 4) {
+          uint32_t run[kPer * 4];
+#pragma unroll
+          for (uint32_t q = 0; q < kPer; ++q)
+#pragma unroll
+            for (int i = 0; i < 4; ++i) run[4 * q + i] = codes[q][2 * i];
+          store_run<(int)(kPer * 4)>(dst, run, wide);
+        } else {
+          uint32_t run[kPer * 6];
+#pragma unroll
+          for (uint32_t q = 0; q < kPer; ++q) {
+            uint64_t a, b, c;
+            pack6(codes[q], a, b, c);
+            run[6 * q] = (uint32_t)a; run[6 * q + 1] = (uint32_t)(a >> 32);
+            run[6 * q + 2] = (uint32_t)b; run[6 * q + 3] = (uint32_t)(b >> 32);
+            run[6 * q + 4] = (uint32_t)c; run[6 * q + 5] = (uint32_t)(c >> 32);
+          }
+          store_run<(int)(kPer * 6)>(dst, run, wide);
+        }
+        uint8_t* sdst = scales_row + scale_offset<LAYOUT>(row, kb0, kb_row);
+        *reinterpret_cast<uint32_t*>(sdst) = scale_word;  // four adjacent bytes in either layout (C % 128 == 0)
+      }
+    }
+
+    // ----------------------------- column pass -----------------------------
+    if (tid >= 128) {
+      constexpr uint32_t kColThreads = 128;
+      constexpr int kWordCols = 2;   // columns in one 32-bit word
+      const uint32_t ct = tid - 128;
+      uint8_t* codes_smem = gen + cfg::kOffCodes;
+      uint8_t* scale_smem = gen + cfg::kOffScales;
+      // 64 word columns x 4 row groups = 256 units of 32 rows x one word
+#pragma unroll 1
+      for (uint32_t u = ct; u < 256; u += kColThreads) {
+        const uint32_t w = u & 63u, g = u >> 6;
+        const uint32_t box = tile_base + (w >> 5) * kBoxBytes;
+        const uint32_t c = (w & 31u) >> 2, wofs = (w & 3u) * 4u;
+        uint32_t raw[kBlock][1];
+#pragma unroll
+        for (uint32_t k = 0; k < kBlock; ++k) {
+          const uint32_t r = g * kBlock + k;
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, r, c) + wofs));
+        }
+        float amax[kWordCols];
+        column_amax<DTYPE, kWordCols>(raw, amax);
+        const uint32_t kb = tr * 4 + g;   // block of the output row
+#pragma unroll
+        for (int cc = 0; cc < kWordCols; ++cc) {
+          const uint32_t col = col0 + w * kWordCols + cc;
+          const BlockScale s = block_scale<FMT>(amax[cc]);
+          uint32_t cw[8];
+          column_cast<FMT, ROUND, DTYPE, kWordCols>(raw, cc, s, cw);
+          const bool live = col < C && kb < kb_col;
+          scale_smem[(w * kWordCols + cc) * 4 + g] = (uint8_t)s.byte;
+          if (bits == 8) {
+            if (live) {
+              uint8_t* dst = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
+              store_run<8>(dst, cw, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+            }
+          } else {
+            // slot of column w * kWordCols + cc: the columns of one lane parity side by side, so that
+            // consecutive lanes are one slot apart
+            uint8_t* dst = codes_smem + ((uint32_t)cc * 64u + w) * cfg::kColPitch + g * kBpb;
+            if (bits == 4) {
+              *reinterpret_cast<uint4*>(dst) = make_uint4(cw[0], cw[2], cw[4], cw[6]);
+            } else {
+              uint64_t a, b, c6;
+              pack6(cw, a, b, c6);
+              uint2* d2 = reinterpret_cast<uint2*>(dst);
+              d2[0] = make_uint2((uint32_t)a, (uint32_t)(a >> 32));
+              d2[1] = make_uint2((uint32_t)b, (uint32_t)(b >> 32));
+              d2[2] = make_uint2((uint32_t)c6, (uint32_t)(c6 >> 32));
+            }
+          }
+        }
+      }
+      // the column warps meet (named barrier 1); then a column's four scale bytes leave as one word
+      // and, for the sub-byte formats, its run of four blocks as whole sectors where the tensor
+      // allows, consecutive threads on consecutive chunks
+      asm volatile("bar.sync 1, %0;" ::"r"(kColThreads) : "memory");
+      const uint32_t live_blocks = min(4u, kb_col - min(kb_col, tr * 4));
+      if (ct < cfg::kCols && col0 + ct < C) {
+        uint8_t* sp = scales_col + scale_offset<LAYOUT>(col0 + ct, tr * 4, kb_col);
+        if (live_blocks == 4 && (reinterpret_cast<uintptr_t>(sp) & 3u) == 0) {
+          *reinterpret_cast<uint32_t*>(sp) = *reinterpret_cast<const uint32_t*>(scale_smem + ct * 4);
+        } else {
+          for (uint32_t g = 0; g < live_blocks; ++g)
+            scales_col[scale_offset<LAYOUT>(col0 + ct, tr * 4 + g, kb_col)] = scale_smem[ct * 4 + g];
+        }
+      }
+      if (bits != 8) {
+        const uint32_t seg = live_blocks * kBpb;  // bytes of a column's run that exist in the output
+        const bool wide = ((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0 && seg % 32 == 0;
+        const uint32_t cb = wide ? 32u : 8u, nch = seg / cb;
+        for (uint32_t i = ct; i < cfg::kCols * nch; i += kColThreads) {
+          const uint32_t cl = i / nch, ch = i - cl * nch;
+          if (col0 + cl >= C) continue;
+          const uint32_t slot = (cl & 1u) * 64u + (cl >> 1);
+          const uint2* src = reinterpret_cast<const uint2*>(codes_smem + slot * cfg::kColPitch + ch * cb);
+          uint8_t* gdst = elems_col + (size_t)(col0 + cl) * col_out_bytes + (size_t)(tr * 4) * kBpb + ch * cb;
+          if (wide) {
+            const uint2 a = src[0], b = src[1], c2 = src[2], d = src[3];
+            const uint32_t v[8] = {a.x, a.y, b.x, b.y, c2.x, c2.y, d.x, d.y};
+            st_32(gdst, v);
+          } else {
+            *reinterpret_cast<uint2*>(gdst) = src[0];
+          }
+        }
+      }
+    }
+    __syncthreads();  // everyone is done with this stage (and with the parked codes) before it is refilled
+  }
+}
+
+template <int FMT, int ROUND, int LAYOUT>
+cudaError_t launch_tile_t(const DualArgs& a) {
+  using cfg = TileCfg<FMT>;
+  cudaError_t e;
+  EncodeTiledFn fn = encode_fn(&e);
+  if (!fn) return e;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.C, (cuuint64_t)a.R};
+  const cuuint64_t strides[1] = {(cuuint64_t)a.C * 2};
+  const cuuint32_t box[2] = {cfg::kCols / 2, kTileRows};
+  if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+    return cudaErrorInvalidValue;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  auto kernel = quantize_tile_kernel<FMT, ROUND, LAYOUT>;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg::kSmem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint32_t tiles_r = (uint32_t)((a.R + kTileRows - 1) / kTileRows);
+  const uint32_t tiles_c = (uint32_t)((a.C + cfg::kCols - 1) / cfg::kCols);
+  const uint32_t num_tiles = tiles_r * tiles_c;
+  const uint32_t slots = 2u * (uint32_t)a.sm_count;  // two CTAs per SM
+  // an even share of tiles per CTA: the smallest grid that needs no more rounds than a full one
+  const uint32_t rounds = (num_tiles + slots - 1) / slots;
+  const uint32_t grid = (num_tiles + rounds - 1) / rounds;
+  return launch_pdl(kernel, dim3(grid), dim3(kTileThreads), cfg::kSmem, a.stream, map, a.elems_row, a.scales_row,
+                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
+}
+
+template <int FMT, int ROUND>
+cudaError_t dispatch_tile_layout(const DualArgs& a) {
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_t<FMT, ROUND, MX_SCALES_LINEAR>(a)
+                                      : launch_tile_t<FMT, ROUND, MX_SCALES_SWIZZLED>(a);
+}
+
+template <int FMT>
+cudaError_t dispatch_tile_round(const DualArgs& a) {
+  return a.rounding == MX_RHAZ ? dispatch_tile_layout<FMT, MX_RHAZ>(a) : dispatch_tile_layout<FMT, MX_RNE>(a);
+}
+
+}  // namespace
+
+// BF16 input, R and C multiples of 128 (what mx_quantize_dual requires of BF16 tensors).
+cudaError_t launch_quantize_tile(const DualArgs& a) {
+  if (a.dtype != MX_BF16 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
+  switch (a.fmt) {
+    case MX_E4M3: return dispatch_tile_round<MX_E4M3>(a);
+    case MX_E5M2: return dispatch_tile_round<MX_E5M2>(a);
+    case MX_E3M2: return dispatch_tile_round<MX_E3M2>(a);
+    case MX_E2M3: return dispatch_tile_round<MX_E2M3>(a);
+    case MX_E2M1: return dispatch_tile_round<MX_E2M1>(a);
+    default: return dispatch_tile_round<MX_INT8>(a);
+  }
+}
+
+// Reads and clears the status word of the tile kernels (after synchronising the stream).
+cudaError_t quantize_tile_status(cudaStream_t stream, unsigned int* status) {
+  cudaError_t e = cudaStreamSynchronize(stream);
+  if (e != cudaSuccess) return e;
+  e = cudaMemcpyFromSymbol(status, g_tile_status, sizeof(unsigned int));
+  if (e != cudaSuccess) return e;
+  if (*status != 0) {
+    const unsigned int zero = 0;
+    e = cudaMemcpyToSymbol(g_tile_status, &zero, sizeof(unsigned int));
+  }
+  return e;
+}
+
+}  // namespace mx
