@@ -362,6 +362,29 @@ int64_t mx_conv_out_w(const mx_conv_t* conv);
 int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, uint8_t* scales_out,
               const mx_conv_t* conv, mx_fmt_t fmt, const mx_opts_t* opts);
 
+/*
+ * mx_conv2d -- the same convolution without the materialized operand (Section 4.1).
+ *
+ * Block (m, kb) of the operand mx_im2col would write is a copy of a block of the quantized
+ * activation (or zero), so the GEMM kernel can fetch it from there itself: four warps gather each
+ * pipeline stage's 128 rows x 128 codes and their scale bytes while the tensor core works on the
+ * stages before, and the [M x kh kw C] operand (kh kw times the activation) is never written or
+ * read.  The arithmetic is that of mx_im2col + mx_gemm; results obey the same bound.
+ *   x_elems, x_scales   MX tensor of x[N, H, W, C] quantized along C (rows N*H*W); scales in
+ *                       opts->scale_layout.  MX_E4M3 or MX_E5M2 (one byte per code: the gather copies
+ *                       bytes into the tensor core's operand layout; 6- and 4-bit activations:
+ *                       MX_ERR_UNSUPPORTED, use mx_im2col + mx_gemm).
+ *   w_elems, w_scales   the filter w[Cout, kh, kw, C] quantized along (kh, kw, C) as one axis: packed
+ *                       [Cout x kh kw C], SWIZZLED scales.  Any format but MX_INT8; kh*kw*C a
+ *                       multiple of 128 for 6- and 4-bit filters.
+ *   y                   FP32 or BF16 (y_dtype) [N, Ho, Wo, Cout], channels last.
+ * C % 32 == 0; Cout * sizeof(y element) a multiple of 16; x_elems, x_scales, y 16-byte aligned,
+ * w_elems 32-byte, w_scales 16-byte aligned.  Errors as mx_gemm and mx_im2col.
+ */
+int mx_conv2d(const void* x_elems, const uint8_t* x_scales, const void* w_elems, const uint8_t* w_scales,
+              void* y, mx_dtype_t y_dtype, const mx_conv_t* conv, int64_t Cout, mx_fmt_t fmt_x,
+              mx_fmt_t fmt_w, const mx_opts_t* opts);
+
 /* ------------------------------------------------------------------------- */
 /* Host-buffer variants                                                      */
 /* ------------------------------------------------------------------------- */

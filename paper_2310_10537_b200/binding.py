@@ -32,7 +32,7 @@ EXPORTS = [
     "mx_fmt_bits", "mx_elems_bytes", "mx_scales_bytes", "mx_scale_offset", "mx_strerror",
     "mx_last_cuda_error", "mx_quantize", "mx_quantize_dual", "mx_dequantize", "mx_gemm",
     "mx_gemm_bf16", "mx_gemm_ex", "mx_gemm_batched", "mx_gemm_quantize", "mx_gemm_dense_workspace_bytes",
-    "mx_gemm_dense", "mx_conv_out_h", "mx_conv_out_w", "mx_im2col",
+    "mx_gemm_dense", "mx_conv_out_h", "mx_conv_out_w", "mx_im2col", "mx_conv2d",
     "mx_quantize_host_async", "mx_dequantize_host_async", "mx_host_synchronize",
     "mx_quantize_host_workspace_bytes", "mx_quantize_host", "mx_quantize_host_static",
     "mx_dequantize_host_workspace_bytes", "mx_dequantize_host",
@@ -103,6 +103,7 @@ def _load() -> ctypes.CDLL:
     lib.mx_conv_out_w.argtypes = [cp]
     lib.mx_conv_out_w.restype = i64
     lib.mx_im2col.argtypes = [vp, u8p, vp, u8p, cp, ci, op]
+    lib.mx_conv2d.argtypes = [vp, u8p, vp, u8p, vp, ci, cp, i64, ci, ci, op]
     lib.mx_gemm_batched.argtypes = [vp, u8p, vp, u8p, vp, ci, i64, i64, i64, i64, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.argtypes = [i64p, ci, ci, ci, op]
     lib.mx_quantize_host_workspace_bytes.restype = sz
@@ -347,6 +348,24 @@ def mx_im2col(elems: torch.Tensor, scales: torch.Tensor, conv: mx_conv_t, fmt: i
     _check(_lib.mx_im2col(elems.data_ptr(), scales.data_ptr(), out_e.data_ptr(), out_s.data_ptr(),
                           ctypes.byref(conv), fmt, ctypes.byref(o)), "mx_im2col")
     return out_e, out_s
+
+
+def mx_conv2d(x_elems: torch.Tensor, x_scales: torch.Tensor, w_elems: torch.Tensor, w_scales: torch.Tensor,
+              conv: mx_conv_t, Cout: int, fmt_x: int, fmt_w: int, layout: int = MX_SCALES_SWIZZLED,
+              out: Optional[torch.Tensor] = None, out_dtype: torch.dtype = torch.float32,
+              check_status: bool = False) -> torch.Tensor:
+    """y[N*Ho*Wo, Cout] = the convolution of the MX activation (quantized along C, 8-bit codes, scales
+    in `layout`) with the MX filter [Cout x kh*kw*C], the im2col operand gathered inside the GEMM."""
+    assert x_elems.is_cuda and x_scales.is_cuda and w_elems.is_cuda and w_scales.is_cuda
+    Ho, Wo = mx_conv_out_hw(conv)
+    M = conv.N * Ho * Wo
+    if out is None:
+        out = torch.empty((M, Cout), dtype=out_dtype, device=x_elems.device)
+    o = _opts(MX_F32, layout, check=check_status)
+    _check(_lib.mx_conv2d(x_elems.data_ptr(), x_scales.data_ptr(), w_elems.data_ptr(), w_scales.data_ptr(),
+                          out.data_ptr(), _dtype_code(out.dtype), ctypes.byref(conv), Cout, fmt_x, fmt_w,
+                          ctypes.byref(o)), "mx_conv2d")
+    return out
 
 
 # ---- host-buffer variants: tensors live in (pinned) host memory ----------------

@@ -767,6 +767,56 @@ int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, u
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 
+int mx_conv2d(const void* x_elems, const uint8_t* x_scales, const void* w_elems, const uint8_t* w_scales,
+              void* y, mx_dtype_t y_dtype, const mx_conv_t* conv, int64_t Cout, mx_fmt_t fmt_x,
+              mx_fmt_t fmt_w, const mx_opts_t* opts) {
+  Opts o;
+  if (!conv) return MX_ERR_NULL;
+  if (!fmt_ok((int)fmt_x) || !fmt_ok((int)fmt_w) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if ((int)y_dtype != MX_F32 && (int)y_dtype != MX_BF16) return MX_ERR_FMT;
+  if (!conv_ok(conv)) return MX_ERR_SHAPE;
+  if (fmt_x == MX_INT8 || fmt_w == MX_INT8 || fmt_bits((int)fmt_x) != 8) return MX_ERR_UNSUPPORTED;
+  const int64_t Ho = mx_conv_out_h(conv), Wo = mx_conv_out_w(conv);
+  const int64_t K = (int64_t)conv->kh * conv->kw * conv->C;
+  const int esz = (int)y_dtype == MX_BF16 ? 2 : 4;
+  if (Ho <= 0 || Wo <= 0 || conv->C % 32 || Cout < 0 || (Cout * esz) % 16) return MX_ERR_SHAPE;
+  if (fmt_bits((int)fmt_w) < 8 && K % 128) return MX_ERR_SHAPE;
+  const int64_t M = conv->N * Ho * Wo;
+  if (M >= ((int64_t)1 << 31) || Cout >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31) ||
+      conv->N * conv->H * conv->W >= ((int64_t)1 << 31) ||
+      (M > 0 && Cout > 0 && ((M + 127) / 128) * ((Cout + 127) / 128) >= ((int64_t)1 << 31)))
+    return MX_ERR_SHAPE;
+  if (M == 0 || Cout == 0) return MX_OK;
+  if (!x_elems || !x_scales || !w_elems || !w_scales || !y) return MX_ERR_NULL;
+  if ((uintptr_t)x_elems % 16 || (uintptr_t)x_scales % 16 || (uintptr_t)w_elems % 32 || (uintptr_t)w_scales % 16 ||
+      (uintptr_t)y % 16)
+    return MX_ERR_ALIGN;
+  cudaError_t e;
+  mx::ConvArgs a;
+  a.x_elems = (const uint8_t*)x_elems; a.x_scales = x_scales; a.w_elems = w_elems; a.w_scales = w_scales;
+  a.y = y; a.y_bf16 = (int)y_dtype == MX_BF16;
+  a.N = conv->N; a.H = conv->H; a.W = conv->W; a.C = conv->C; a.Ho = Ho; a.Wo = Wo; a.Cout = Cout;
+  a.kh = conv->kh; a.kw = conv->kw; a.stride_h = conv->stride_h; a.stride_w = conv->stride_w;
+  a.pad_h = conv->pad_h; a.pad_w = conv->pad_w; a.dil_h = conv->dil_h; a.dil_w = conv->dil_w;
+  a.fmt_x = (int)fmt_x; a.fmt_w = (int)fmt_w; a.x_layout = o.layout; a.stream = o.stream;
+  a.sm_count = sm_count(&e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  int rc = mx::launch_conv(a, &e);
+  if (rc != MX_OK) return rc == MX_ERR_CUDA ? fail_cuda(e) : rc;
+  if (o.check) {
+    unsigned int st = 0;
+    rc = mx::gemm_status(o.stream, &st, &e);
+    if (rc != MX_OK) return fail_cuda(e);
+    if (st != 0) {
+      std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u gave up "
+                    "(1 producer/stage empty, 2 MMA/stage full, 3 MMA/accumulator free, "
+                    "4 epilogue/accumulator full, 5 scale copier/stage full, 6 shared-memory alignment)", st);
+      return MX_ERR_TIMEOUT;
+    }
+  }
+  return MX_OK;
+}
+
 size_t mx_gemm_host_workspace_bytes(int64_t M, int64_t N, int64_t K, mx_fmt_t fmtA, mx_fmt_t fmtB) {
   if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || M < 0 || N < 0 || K < 0 || K % 32) return 0;
   return align_up((size_t)(M * K / 8 * fmt_bits((int)fmtA)), 256) +

@@ -406,16 +406,49 @@ __device__ __forceinline__ void raise_abort(volatile uint32_t* abort_flag, unsig
   *abort_flag = 1u;
 }
 
+// Implicit-GEMM convolution (CONV): the A operand [N Ho Wo x kh kw C] is never materialized.  The
+// activation x[N, H, W, C] was quantized once along C (8-bit codes), so block (m, kb) of A is block
+// kb % (C / 32) of the input pixel that filter tap kb / (C / 32) of output pixel m reads -- or a zero
+// block where the tap falls into the padding.  When C is a multiple of 128 a stage's 128 K elements
+// lie in one filter tap and ONE copy through an im2col-mode tensor map brings the stage's 128 rows
+// x 128 bytes (128 consecutive output pixels, their input pixels found by the copy engine, padding
+// filled with zeros); otherwise four extra warps gather them with 16-byte cp.async copies straight
+// into the 128-byte-swizzled operand layout.  In both cases those warps compose each row's four
+// scale bytes into the stage's scale chunk.
+struct ConvGeom {
+  const uint8_t* x_codes;   // [N H W][C] codes, one byte each
+  const uint8_t* x_scales;  // [N H W rows][C / 32]
+  uint32_t H, W, Ho, Wo, kw, C, cb, kblocks, M, x_rows, x_layout;
+  uint32_t tma;  // 1: the codes come through an im2col tensor map (C % 128 == 0), the gather warps only place scales
+  int32_t stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+  FastDiv d_wo, d_howo, d_kw, d_cb;
+};
+constexpr int kConvThreads = kThreads + 128;  // + four gather warps
+constexpr int kConvLag = 2;                   // stages a gather thread keeps in flight before it signals one
+
+// 128 pixels x 128 channels of x[N, H, W, C] for one filter tap: (c, w, h, n) is the first channel
+// and the input position that tap (0, 0) of the first output pixel reads, (ow, oh) the tap's offset.
+__device__ __forceinline__ void tma_load_im2col(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                uint32_t ow, uint32_t oh, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar),
+        "h"((uint16_t)ow), "h"((uint16_t)oh) : "memory");
+}
+
+__device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+
 // DENSE: the operands are BF16 matrices (MX tensors dequantized beforehand, which is exact) and the
 // MMA is the plain kind::f16 one: a stage holds 64 K-elements (the same 128-byte rows), no scales.
-template <int BN, bool DENSE>
-__global__ void __launch_bounds__(kThreads, 1)
-mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-               const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
-               const __grid_constant__ CUtensorMap tmap_c,
-               uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
-               uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch,
-               long long spin_limit, uint32_t drop_fill) {
+template <int BN, bool DENSE, bool CONV>
+__device__ __forceinline__ void
+gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_sa,
+                 const CUtensorMap& tmap_sb, const CUtensorMap& tmap_c, uint32_t M, uint32_t N, uint32_t K,
+                 uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch,
+                 long long spin_limit, uint32_t drop_fill, const ConvGeom& cg) {
+  static_assert(!CONV || (!DENSE && BN == 128), "the gather warps fit the register budget of the 128-wide tile");
   using cfg = Cfg<BN>;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -439,10 +472,10 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < cfg::kStages; ++s) {
-      mbar_init(full_bar(s), 1);
+      mbar_init(full_bar(s), (CONV && !cg.tma) ? 5 : 1);  // the producer's arrive + bytes (gathered codes: + one arrival per gather warp)
       mbar_init(empty_bar(s), 1);
       mbar_init(sf_ready_bar(s), 1);  // the copier's tcgen05.commit
-      mbar_init(sf_full_bar(s), 1);   // the scale producer's arrive + scale bytes
+      mbar_init(sf_full_bar(s), CONV ? 5 : 1);    // the scale producer's arrive + scale bytes (CONV: + the gather warps)
     }
     for (uint32_t a = 0; a < cfg::kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
@@ -485,6 +518,15 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       // ragged last tile belong to the next matrix of the batch or are zero-filled by the copy;
       // their columns are not stored.
       const int cy_a = (int)((tc.b * tiles_m + tc.tm) * BM), cy_b = (int)(tc.b * N + tc.tn * BN);
+      // CONV through the im2col map: where tap (0, 0) of the tile's first output pixel reads
+      int cv_w = 0, cv_h = 0, cv_n = 0;
+      if (CONV) {
+        const uint32_t m0 = tc.tm * BM, n0 = fastdiv(m0, cg.d_howo), rem = m0 - n0 * (cg.Ho * cg.Wo);
+        const uint32_t ho = fastdiv(rem, cg.d_wo), wo = rem - ho * cg.Wo;
+        cv_n = (int)n0;
+        cv_h = (int)ho * cg.stride_h - cg.pad_h;
+        cv_w = (int)wo * cg.stride_w - cg.pad_w;
+      }
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
         ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
         if (!ok) {
@@ -494,7 +536,14 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
         if (fill++ != drop_fill && elect_one()) {
           const uint32_t fb = full_bar(stage);
           mbar_arrive_expect_tx(fb, tx_bytes);
-          tma_load_3d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BKe), cy_a, 0, fb);
+          if (!CONV) {
+            tma_load_3d(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(kc * BKe), cy_a, 0, fb);
+          } else if (cg.tma) {  // the stage's K chunk = 128 channels of one filter tap
+            const uint32_t tap = fastdiv(kc * 4, cg.d_cb), cblk = kc * 4 - tap * cg.cb;
+            const uint32_t ti = fastdiv(tap, cg.d_kw), tj = tap - ti * cg.kw;
+            tma_load_im2col(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(cblk * 32u), cv_w, cv_h, cv_n,
+                            tj * (uint32_t)cg.dil_w, ti * (uint32_t)cg.dil_h, fb);
+          }
           tma_load_3d(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, (int)(kc * BKe), cy_b, 0, fb);
         }
         __syncwarp();
@@ -598,9 +647,9 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
           }
           if (elect_one()) {
             const uint32_t fb = sf_full_bar(stage);
-            mbar_arrive_expect_tx(fb, cfg::kSfBytes);
+            mbar_arrive_expect_tx(fb, CONV ? cfg::kSfBytes - 512u : cfg::kSfBytes);
             const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
-            tma_load_3d(dst, &tmap_sa, 0, (int)kc, cz_a, fb);
+            if (!CONV) tma_load_3d(dst, &tmap_sa, 0, (int)kc, cz_a, fb);
             tma_load_3d(dst + 512u, &tmap_sb, 0, (int)kc, cz_b, fb);
           }
           __syncwarp();
@@ -610,6 +659,137 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
       if (!ok) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) {}
+      }
+    }
+  } else if (warp >= 12) {
+    // ------------------- gather warps (CONV): thread r serves row r of the tile -------------------
+    if constexpr (CONV) {
+      // Codes: thread (p, q) copies 16-byte chunk p of rows q, q + 16, ..., q + 112, so that one
+      // warp instruction moves four whole 128-byte rows (four input pixels' channel runs: full
+      // lines from L2, conflict-free rows in shared memory).  Scales: thread r composes the word
+      // of row r.
+      const uint32_t gt = threadIdx.x - (uint32_t)kThreads;
+      const uint32_t p = gt & 7u, q = gt >> 3;
+      uint32_t stage = 0, phase = 0, issued = 0, signalled = 0;
+      bool ok = true;
+      // a stage's codes are signalled kConvLag stages after they were requested: the copies of the
+      // stages in between are then in flight, and the thread itself makes them visible to the
+      // tensor core's proxy before its warp arrives (one arrival per warp: 128 arrivals on one
+      // barrier word would serialise)
+      auto signal_oldest = [&]() {
+        const uint32_t st = signalled % cfg::kStages;
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+        __syncwarp();
+        if (lane == 0) mbar_arrive(full_bar(st));
+        ++signalled;
+      };
+      // C a multiple of 128: the four blocks of a stage belong to one filter tap, their scale
+      // bytes are one aligned word
+      const bool one_tap = (cg.cb & 3u) == 0;
+      struct RowGeom {
+        int32_t h0, w0;   // input coordinates of tap (0, 0)
+        uint32_t pix0;    // first pixel of the row's image; 0xFFFFFFFF: row past M
+      };
+      auto row_geom = [&](uint32_t m) -> RowGeom {
+        RowGeom g;
+        const uint32_t n = fastdiv(m, cg.d_howo), rem = m - n * (cg.Ho * cg.Wo);
+        const uint32_t ho = fastdiv(rem, cg.d_wo), wo = rem - ho * cg.Wo;
+        g.h0 = (int32_t)ho * cg.stride_h - cg.pad_h;
+        g.w0 = (int32_t)wo * cg.stride_w - cg.pad_w;
+        g.pix0 = m < cg.M ? n * cg.H * cg.W : 0xFFFFFFFFu;
+        return g;
+      };
+      // MX block kb of the reduction axis (kh, kw, C): filter tap offsets and channel block
+      struct Tap {
+        int32_t dh, dw;
+        uint32_t cblk;
+        bool ok;
+      };
+      auto tap_of = [&](uint32_t kb) -> Tap {
+        Tap tp;
+        const uint32_t tap = fastdiv(kb, cg.d_cb);
+        tp.cblk = kb - tap * cg.cb;
+        const uint32_t ti = fastdiv(tap, cg.d_kw), tj = tap - ti * cg.kw;
+        tp.dh = (int32_t)ti * cg.dil_h;
+        tp.dw = (int32_t)tj * cg.dil_w;
+        tp.ok = kb < cg.kblocks;
+        return tp;
+      };
+      // input pixel a row reads through a tap; false where the tap falls into the padding
+      auto source = [&](const RowGeom& g, const Tap& tp, uint32_t& px) -> bool {
+        const int32_t hi = g.h0 + tp.dh, wi = g.w0 + tp.dw;
+        const bool live = tp.ok && g.pix0 != 0xFFFFFFFFu && hi >= 0 && hi < (int32_t)cg.H && wi >= 0 && wi < (int32_t)cg.W;
+        px = live ? g.pix0 + (uint32_t)hi * cg.W + (uint32_t)wi : 0u;
+        return live;
+      };
+      auto scale_at = [&](uint32_t px, uint32_t cblk) -> const uint8_t* {
+        return cg.x_scales + (cg.x_layout == MX_SCALES_LINEAR ? (size_t)px * cg.cb + cblk
+                                                              : scale_offset<MX_SCALES_SWIZZLED>(px, cblk, cg.cb));
+      };
+      for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        RowGeom rows[8];
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) rows[i] = row_geom(tc.tm * BM + q + 16 * i);
+        const RowGeom mine = row_geom(tc.tm * BM + gt);  // the row whose scale word this thread writes
+        // the four scale bytes of K chunk kc of that row (requested one chunk ahead of their use)
+        auto scale_word = [&](uint32_t kc) -> uint32_t {
+          uint32_t px, word = 0;
+          if (one_tap) {
+            const Tap tp = tap_of(kc * 4);
+            if (source(mine, tp, px)) word = __ldg(reinterpret_cast<const uint32_t*>(scale_at(px, tp.cblk)));
+          } else {
+#pragma unroll
+            for (uint32_t b = 0; b < 4; ++b) {
+              const Tap tp = tap_of(kc * 4 + b);
+              if (source(mine, tp, px)) word |= (uint32_t)__ldg(scale_at(px, tp.cblk)) << (8 * b);
+            }
+          }
+          return word;
+        };
+        uint32_t sword_next = scale_word(0);
+        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+          ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
+          if (!ok) {
+            raise_abort(abort_flag, ST_PRODUCER_WAIT);
+            break;
+          }
+          if (!cg.tma) {
+            const uint32_t a_base = smem_base + cfg::kOffA + stage * cfg::kABytes;
+            const Tap tp = tap_of(kc * 4 + (p >> 1));  // the block chunk p lies in
+            const uint32_t in_block = tp.cblk * 32u + (p & 1u) * 16u;
+            // zero blocks (padding taps, rows past M, K tail) are written by copies of zero source bytes
+#pragma unroll
+            for (uint32_t i = 0; i < 8; ++i) {
+              const uint32_t row = q + 16 * i;
+              uint32_t px;
+              const bool live = source(rows[i], tp, px);
+              cp_async_16(a_base + row * 128u + ((p ^ (row & 7u)) << 4),
+                          live ? cg.x_codes + (size_t)px * cg.C + in_block : cg.x_codes, live ? 16u : 0u);
+            }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+          }
+          const uint32_t sword = sword_next;
+          if (kc + 1 < k_chunks) sword_next = scale_word(kc + 1);
+          // row gt's four scale bytes, where the swizzled chunk keeps them
+          asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_base + cfg::kOffSf + stage * cfg::kSfBytes +
+                                                      (gt & 31u) * 16u + (gt >> 5) * 4u), "r"(sword) : "memory");
+          asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+          __syncwarp();
+          if (lane == 0) mbar_arrive(sf_full_bar(stage));
+          if (!cg.tma) {
+            ++issued;
+            if (issued - signalled > (uint32_t)kConvLag) {
+              asm volatile("cp.async.wait_group %0;" ::"n"(kConvLag) : "memory");
+              signal_oldest();
+            }
+          }
+          if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+        }
+      }
+      asm volatile("cp.async.wait_group 0;" ::: "memory");
+      if (ok) {
+        while (signalled < issued) signal_oldest();
       }
     }
   } else {
@@ -659,6 +839,31 @@ mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"((uint32_t)kTmemCols) : "memory");
   }
+}
+
+template <int BN, bool DENSE>
+__global__ void __launch_bounds__(kThreads, 1)
+mx_gemm_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+               const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
+               const __grid_constant__ CUtensorMap tmap_c,
+               uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base,
+               uint32_t group_m, uint32_t tx_bytes, EpiArgs epi, uint32_t batch,
+               long long spin_limit, uint32_t drop_fill) {
+  const ConvGeom none = {};
+  gemm_kernel_body<BN, DENSE, false>(tmap_a, tmap_b, tmap_sa, tmap_sb, tmap_c, M, N, K, idesc_base, group_m, tx_bytes,
+                                     epi, batch, spin_limit, drop_fill, none);
+}
+
+// Implicit-GEMM convolution: the same kernel with four gather warps in place of the A copies
+// (tmap_b / tmap_sb: the filter [Cout x kh kw C] and its scales; M = N Ho Wo, N = Cout, K = kh kw C).
+__global__ void __launch_bounds__(kConvThreads, 1)
+mx_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
+               const __grid_constant__ CUtensorMap tmap_sb, const __grid_constant__ CUtensorMap tmap_c, uint32_t M,
+               uint32_t N, uint32_t K, uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes, EpiArgs epi,
+               long long spin_limit, const __grid_constant__ ConvGeom cg) {
+  // tmap_x: the im2col-mode map over x's codes (cg.tma), else any valid map (unused)
+  gemm_kernel_body<128, false, true>(tmap_x, tmap_b, tmap_sb, tmap_sb, tmap_c, M, N, K, idesc_base, group_m, tx_bytes,
+                                     epi, 1u, spin_limit, kNoDrop, cg);
 }
 
 
@@ -1639,6 +1844,77 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
                            ((uint32_t)(BM >> 4) << 24);
     *cuda_err = bn == 256 ? launch_bn<256, false>(a, ma, mb, idesc) : launch_bn<128, false>(a, ma, mb, idesc);
   }
+  return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
+}
+
+// Implicit-GEMM convolution on the one-CTA kernel with 128 x 128 tiles (see mx_conv_kernel).
+int launch_conv(const ConvArgs& a, cudaError_t* cuda_err) {
+  *cuda_err = cudaSuccess;
+  EncodeTiledFn fn = encode_fn(cuda_err);
+  if (!fn) return MX_ERR_CUDA;
+  constexpr int BN = 128;
+  using cfg = Cfg<BN>;
+  const int64_t M = a.N * a.Ho * a.Wo, K = (int64_t)a.kh * a.kw * a.C;
+  GemmArgs ga = {};
+  ga.C = a.y; ga.c_bf16 = a.y_bf16; ga.batch = 1; ga.M = M; ga.N = a.Cout; ga.K = K;
+  CUtensorMap mb, msb, mc;
+  if (!make_out_map(fn, &mc, ga) || !make_operand_map(fn, &mb, a.w_elems, a.fmt_w, (uint64_t)a.Cout, (uint64_t)K, BN) ||
+      !make_scale_map(fn, &msb, a.w_scales, (uint64_t)a.Cout, (uint64_t)K, cfg::kSfbChunks)) {
+    *cuda_err = cudaErrorInvalidValue;
+    return MX_ERR_CUDA;
+  }
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  cudaError_t e = cudaGetDevice(&dev);
+  if (e == cudaSuccess && (dev < 0 || dev >= 64 || !attr_set[dev])) {
+    e = cudaFuncSetAttribute(mx_conv_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg::kSmemBytes);
+    if (e == cudaSuccess && dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  if (e != cudaSuccess) {
+    *cuda_err = e;
+    return MX_ERR_CUDA;
+  }
+  // im2col-mode map over x[N, H, W, C] (dims C, W, H, N): 128 channels x 128 pixels per copy, the
+  // pixels walked along W, H, N with the convolution's strides inside the box of base positions
+  // [-pad, extent + pad - (k - 1) dilation); usable when a 128-element K chunk lies in one tap
+  CUtensorMap mx_ = mb;
+  const bool tma = a.C % 128 == 0 && (a.kw - 1) * a.dil_w < 256 && (a.kh - 1) * a.dil_h < 256 && a.pad_w <= 127 &&
+                   a.pad_h <= 127 && a.stride_w <= 8 && a.stride_h <= 8;
+  if (tma) {
+    Im2colFn im2col = im2col_fn(cuda_err);
+    if (!im2col) return MX_ERR_CUDA;
+    const cuuint64_t dims[4] = {(cuuint64_t)a.C, (cuuint64_t)a.W, (cuuint64_t)a.H, (cuuint64_t)a.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)a.C, (cuuint64_t)a.C * a.W, (cuuint64_t)a.C * a.W * a.H};
+    const int lower[2] = {-a.pad_w, -a.pad_h};
+    const int upper[2] = {a.pad_w - (a.kw - 1) * a.dil_w, a.pad_h - (a.kh - 1) * a.dil_h};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)a.stride_w, (cuuint32_t)a.stride_h, 1};
+    if (im2col(&mx_, CU_TENSOR_MAP_DATA_TYPE_UINT8, 4, const_cast<uint8_t*>(a.x_elems), dims, strides, lower, upper, 128,
+               128, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS) {
+      *cuda_err = cudaErrorInvalidValue;
+      return MX_ERR_CUDA;
+    }
+  }
+  ConvGeom g;
+  g.tma = tma ? 1u : 0u;
+  g.x_codes = a.x_elems; g.x_scales = a.x_scales;
+  g.H = (uint32_t)a.H; g.W = (uint32_t)a.W; g.Ho = (uint32_t)a.Ho; g.Wo = (uint32_t)a.Wo; g.kw = (uint32_t)a.kw;
+  g.C = (uint32_t)a.C; g.cb = (uint32_t)(a.C / 32); g.kblocks = (uint32_t)(K / 32); g.M = (uint32_t)M;
+  g.x_rows = (uint32_t)(a.N * a.H * a.W); g.x_layout = (uint32_t)a.x_layout;
+  g.stride_h = a.stride_h; g.stride_w = a.stride_w; g.pad_h = a.pad_h; g.pad_w = a.pad_w;
+  g.dil_h = a.dil_h; g.dil_w = a.dil_w;
+  g.d_wo = make_fastdiv(g.Wo); g.d_howo = make_fastdiv(g.Ho * g.Wo); g.d_kw = make_fastdiv(g.kw);
+  g.d_cb = make_fastdiv(g.cb);
+  const uint32_t tiles = (uint32_t)((M + BM - 1) / BM) * (uint32_t)((a.Cout + BN - 1) / BN);
+  const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
+  // the filter tile, plus the 128 x 128 codes of x when they come through the im2col map
+  const uint32_t tx_bytes = (uint32_t)(BN * BK * fmt_bits(a.fmt_w) / 8) + (tma ? (uint32_t)(BM * BK) : 0u);
+  const uint32_t idesc = (mma_fmt_code(a.fmt_x) << 7) | (mma_fmt_code(a.fmt_w) << 10) | (1u << 23) |
+                         ((uint32_t)(BM >> 4) << 24) | ((uint32_t)(BN >> 3) << 17);
+  EpiArgs epi;
+  epi.mode = a.y_bf16 ? 1u : 0u; epi.fmt = 0; epi.sticky = 0; epi.elems = nullptr; epi.scales = nullptr;
+  *cuda_err = launch_pdl_if(false, mx_conv_kernel, dim3(grid), dim3(kConvThreads), cfg::kSmemBytes, a.stream, mx_, mb, msb,
+                            mc, (uint32_t)M, (uint32_t)a.Cout, (uint32_t)K, idesc, 16u, tx_bytes, epi, kSpinLimit, g);
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
 }
 

@@ -61,6 +61,24 @@ struct Im2colArgs {
 };
 cudaError_t launch_im2col(const Im2colArgs& a);
 
+// Convolution without a materialized operand (see mx_conv2d()): x quantized along C (8-bit codes),
+// filter w[Cout][kh kw C] quantized along its last axis (any block-scaled format, swizzled scales).
+struct ConvArgs {
+  const uint8_t* x_elems;
+  const uint8_t* x_scales;
+  const void* w_elems;
+  const uint8_t* w_scales;
+  void* y;  // FP32 or BF16 [N Ho Wo x Cout]
+  int y_bf16;
+  int64_t N, H, W, C, Ho, Wo, Cout;
+  int kh, kw, stride_h, stride_w, pad_h, pad_w, dil_h, dil_w;
+  int fmt_x, fmt_w, x_layout;
+  int sm_count;
+  cudaStream_t stream;
+};
+// Returns MX_OK or a negative mx_status_t; fills *cuda_err on MX_ERR_CUDA.
+int launch_conv(const ConvArgs& a, cudaError_t* cuda_err);
+
 struct GemmArgs {
   const void* A;
   const uint8_t* sA;

@@ -27,6 +27,24 @@ inline EncodeTiledFn encode_fn(cudaError_t* err) {
   return fn;
 }
 
+typedef CUresult (*Im2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                             const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                             CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                             CUtensorMapFloatOOBfill);
+
+// The driver's im2col-mode encoder (convolution: the copy engine walks the input pixels itself).
+inline Im2colFn im2col_fn(cudaError_t* err) {
+  static Im2colFn fn = nullptr;
+  if (fn) { *err = cudaSuccess; return fn; }
+  void* p = nullptr;
+  cudaDriverEntryPointQueryResult q;
+  *err = cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &p, cudaEnableDefault, &q);
+  if (*err != cudaSuccess) return nullptr;
+  if (q != cudaDriverEntryPointSuccess || !p) { *err = cudaErrorNotSupported; return nullptr; }
+  fn = (Im2colFn)p;
+  return fn;
+}
+
 inline EncodeTiledFn encode_fn_cached() {
   cudaError_t e;
   return encode_fn(&e);

@@ -20,6 +20,12 @@ CASES = [
     (1, 12, 12, 128, 128, 5, 3, (1, 2), (2, 0), (2, 1), 2, 3, 1),     # 6-bit codes (K % 128), dilation, asymmetric
     (2, 8, 8, 128, 128, 3, 3, (1, 1), (1, 1), (1, 1), 4, 4, 0),       # FP4 both (K = 1152)
     (1, 30, 30, 96, 384, 3, 3, (1, 1), (0, 0), (1, 1), 0, 0, 1),      # M = 784: ragged row tiles
+    (2, 20, 20, 32, 128, 3, 3, (1, 1), (1, 1), (1, 1), 0, 1, 1),      # C = 32: a K chunk spans four taps, K tail (288)
+    (4, 28, 28, 256, 256, 3, 3, (1, 1), (1, 1), (1, 1), 0, 0, 1),     # 25 row tiles x 2 column tiles, 18 K chunks
+    (2, 16, 16, 64, 136, 2, 2, (2, 2), (0, 0), (1, 1), 1, 4, 0),      # FP4 filter, Cout not a multiple of 128
+    (1, 12, 12, 128, 128, 5, 3, (1, 2), (2, 0), (2, 1), 0, 0, 1),     # C % 128 == 0: codes through the im2col map; asymmetric filter, stride, padding, dilation
+    (2, 15, 17, 128, 256, 3, 3, (2, 2), (1, 1), (1, 1), 1, 0, 0),     # im2col map, stride 2, odd extents, last tile crosses the batch end
+    (3, 7, 9, 384, 128, 2, 4, (1, 1), (0, 2), (1, 1), 0, 2, 1),       # im2col map, three channel chunks per tap, 6-bit filter
 ]
 
 
@@ -84,6 +90,23 @@ def test_conv_matches_oracle(case):
     y64, s64 = O.conv2d_nhwc(xq, wq, st, pd, dl)
     err = np.abs(y.cpu().numpy().astype(np.float64).reshape(N, Ho, Wo, Cout) - y64)
     assert (err <= TOL * s64).all(), f"{int((err > TOL * s64).sum())} outputs beyond 1e-5 * S"
+
+    # (c) the same convolution with the operand gathered inside the GEMM (8-bit activations)
+    if O.fmt_bits(fx) == 8:
+        g2 = Guarded(M * Cout * 4)
+        y2 = g2.view.view(torch.float32).view(M, Cout)
+        mx.mx_conv2d(ex, sx, ew, sw, conv, Cout, fx, fw, layout=layout, out=y2, check_status=True)
+        torch.cuda.synchronize()
+        g2.check()
+        err2 = np.abs(y2.cpu().numpy().astype(np.float64).reshape(N, Ho, Wo, Cout) - y64)
+        assert (err2 <= TOL * s64).all(), f"implicit: {int((err2 > TOL * s64).sum())} outputs beyond 1e-5 * S"
+        assert torch.equal(y2, y), "the gathered operand must give the materialized operand's result bit for bit"
+        yb = mx.mx_conv2d(ex, sx, ew, sw, conv, Cout, fx, fw, layout=layout, out_dtype=torch.bfloat16, check_status=True)
+        assert torch.equal(yb, y2.to(torch.bfloat16))
+    else:
+        with pytest.raises(mx.MxError) as ei:
+            mx.mx_conv2d(ex, sx, ew, sw, conv, Cout, fx, fw, layout=layout)
+        assert ei.value.status == mx.MX_ERR_UNSUPPORTED
 
 
 def test_im2col_errors():
