@@ -440,6 +440,18 @@ __device__ __forceinline__ void cp_async_16(uint32_t dst, const void* src, uint3
   asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
 }
 
+// One scale word global -> shared without passing through a register (src_bytes 0: a zero word), and
+// an arrival on a barrier of this CTA that happens when the thread's copies so far have landed
+// (counted in the barrier's expected arrivals).  A thread that fetched the words through registers
+// would have to order them with a release before signalling, and a release waits for every load the
+// thread has in flight -- the ones it requested ahead included.
+__device__ __forceinline__ void cp_async_4(uint32_t dst, const void* src, uint32_t src_bytes) {
+  asm volatile("cp.async.ca.shared.global [%0], [%1], 4, %2;" ::"r"(dst), "l"(src), "r"(src_bytes) : "memory");
+}
+__device__ __forceinline__ void cp_async_arrive(uint32_t bar) {
+  asm volatile("cp.async.mbarrier.arrive.noinc.shared::cta.b64 [%0];" ::"r"(bar) : "memory");
+}
+
 // DENSE: the operands are BF16 matrices (MX tensors dequantized beforehand, which is exact) and the
 // MMA is the plain kind::f16 one: a stage holds 64 K-elements (the same 128-byte rows), no scales.
 template <int BN, bool DENSE, bool CONV>
@@ -475,7 +487,7 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
       mbar_init(full_bar(s), (CONV && !cg.tma) ? 5 : 1);  // the producer's arrive + bytes (gathered codes: + one arrival per gather warp)
       mbar_init(empty_bar(s), 1);
       mbar_init(sf_ready_bar(s), 1);  // the copier's tcgen05.commit
-      mbar_init(sf_full_bar(s), CONV ? 5 : 1);    // the scale producer's arrive + scale bytes (CONV: + the gather warps)
+      mbar_init(sf_full_bar(s), CONV ? (cg.tma ? 33 : 5) : 1);  // the scale producer's arrive + scale bytes (CONV: + the lanes of the warp that copies the A scale words, or the four gather warps)
     }
     for (uint32_t a = 0; a < cfg::kAccStages; ++a) {
       mbar_init(acc_full_bar(a), 1);
@@ -613,6 +625,7 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
             raise_abort(abort_flag, ST_SCALE_WAIT);
             break;
           }
+          if (CONV) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");  // the A scale words were written by ordinary copies
           tc_fence_after();
           const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
           const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
@@ -664,6 +677,51 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
   } else if (warp >= 12) {
     // ------------------- gather warps (CONV): thread r serves row r of the tile -------------------
     if constexpr (CONV) {
+      if (cg.tma) {
+        // The codes come through the im2col map; warp 12 alone copies the A scale words (lane l: rows
+        // l, l + 32, l + 64, l + 96), asynchronously, each lane's arrival following its copies.
+        if (warp == 12) {
+          uint32_t stage = 0, phase = 0;
+          bool ok = true;
+          for (uint32_t t = blockIdx.x; t < num_tiles && ok; t += gridDim.x) {
+            const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+            int32_t cvh[4], cvw[4];
+            uint32_t cvp[4];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint32_t m = tc.tm * BM + lane + 32 * j;
+              const uint32_t n0 = fastdiv(m, cg.d_howo), rem = m - n0 * (cg.Ho * cg.Wo);
+              const uint32_t ho = fastdiv(rem, cg.d_wo), wo = rem - ho * cg.Wo;
+              cvh[j] = (int32_t)ho * cg.stride_h - cg.pad_h;
+              cvw[j] = (int32_t)wo * cg.stride_w - cg.pad_w;
+              cvp[j] = m < cg.M ? n0 * cg.H * cg.W : 0xFFFFFFFFu;
+            }
+            for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+              ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
+              if (!ok) {
+                raise_abort(abort_flag, ST_PRODUCER_WAIT);
+                break;
+              }
+              const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
+              const uint32_t tap = fastdiv(kc * 4, cg.d_cb), cblk = kc * 4 - tap * cg.cb;
+              const uint32_t ti = fastdiv(tap, cg.d_kw), tj = tap - ti * cg.kw;
+              const int32_t dh = (int32_t)ti * cg.dil_h, dw = (int32_t)tj * cg.dil_w;
+#pragma unroll
+              for (int j = 0; j < 4; ++j) {
+                const int32_t hi = cvh[j] + dh, wi = cvw[j] + dw;
+                const bool live = cvp[j] != 0xFFFFFFFFu && hi >= 0 && hi < (int32_t)cg.H && wi >= 0 && wi < (int32_t)cg.W;
+                const uint32_t px = live ? cvp[j] + (uint32_t)hi * cg.W + (uint32_t)wi : 0u;
+                const size_t so = cg.x_layout == MX_SCALES_LINEAR ? (size_t)px * cg.cb + cblk
+                                                                  : scale_offset<MX_SCALES_SWIZZLED>(px, cblk, cg.cb);
+                cp_async_4(dst + lane * 16u + (uint32_t)j * 4u, cg.x_scales + (live ? so : 0), live ? 4u : 0u);
+              }
+              cp_async_arrive(sf_full_bar(stage));
+              if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+            }
+          }
+          asm volatile("cp.async.wait_all;" ::: "memory");
+        }
+      } else {
       // Codes: thread (p, q) copies 16-byte chunk p of rows q, q + 16, ..., q + 112, so that one
       // warp instruction moves four whole 128-byte rows (four input pixels' channel runs: full
       // lines from L2, conflict-free rows in shared memory).  Scales: thread r composes the word
@@ -747,8 +805,18 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
           }
           return word;
         };
-        uint32_t sword_next = scale_word(0);
-        for (uint32_t kc = 0; kc < k_chunks; ++kc) {
+        // requested kScaleAhead K chunks before their use: a load takes longer than a stage
+        constexpr uint32_t kScaleAhead = 4;
+        uint32_t sword_queue[kScaleAhead] = {};
+#pragma unroll
+        for (uint32_t d = 0; d < kScaleAhead; ++d)
+          if (d < k_chunks) sword_queue[d] = scale_word(d);
+        // (unrolled by the queue depth: every queue slot is a fixed register, see the pair kernel)
+        for (uint32_t kc0 = 0; kc0 < k_chunks && ok; kc0 += kScaleAhead) {
+#pragma unroll
+        for (uint32_t d = 0; d < kScaleAhead; ++d) {
+          const uint32_t kc = kc0 + d;
+          if (kc >= k_chunks || !ok) break;
           ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
           if (!ok) {
             raise_abort(abort_flag, ST_PRODUCER_WAIT);
@@ -769,8 +837,8 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
             }
             asm volatile("cp.async.commit_group;" ::: "memory");
           }
-          const uint32_t sword = sword_next;
-          if (kc + 1 < k_chunks) sword_next = scale_word(kc + 1);
+          const uint32_t sword = sword_queue[d];
+          if (kc + kScaleAhead < k_chunks) sword_queue[d] = scale_word(kc + kScaleAhead);
           // row gt's four scale bytes, where the swizzled chunk keeps them
           asm volatile("st.shared.b32 [%0], %1;" ::"r"(smem_base + cfg::kOffSf + stage * cfg::kSfBytes +
                                                       (gt & 31u) * 16u + (gt >> 5) * 4u), "r"(sword) : "memory");
@@ -786,10 +854,12 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
           }
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
+        }
       }
       asm volatile("cp.async.wait_group 0;" ::: "memory");
       if (ok) {
         while (signalled < issued) signal_oldest();
+      }
       }
     }
   } else {
@@ -1156,6 +1226,14 @@ struct Cfg2 {
   static constexpr uint32_t kSmemBytes = kUsedBytes + 1024 <= 232448 ? kUsedBytes + 1024 : 232448;
   static_assert(kUsedBytes <= 232448, "shared memory budget");
   static_assert(kSfCol0 + kStages * kSfCols <= kTmemCols, "tensor memory budget");
+  // Convolution (mx_conv_pair_kernel): the A scale words of a K chunk are composed one trip round the
+  // operand ring ahead of their use, into a ring of their own with twice as many slots, each with a
+  // barrier in the leader (its own words + the peer's "mine have landed") and one in the peer.
+  static constexpr uint32_t kConvSlots = 2 * kStages;
+  static constexpr uint32_t kOffConvA = (kUsedBytes + 15u) & ~15u;
+  static constexpr uint32_t kOffConvBar = kOffConvA + kConvSlots * 512;
+  static constexpr uint32_t kConvUsedBytes = kOffConvBar + 2 * kConvSlots * 8;
+  static constexpr uint32_t kConvSmemBytes = kConvUsedBytes + 1024;  // (checked where the kernel is defined)
 };
 
 // shared::cluster address of the same shared-memory offset in CTA `rank` of the cluster.
@@ -1170,6 +1248,13 @@ __device__ __forceinline__ void tma_load_3d_pair(uint32_t dst, const CUtensorMap
   asm volatile(
       "cp.async.bulk.tensor.3d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4}], [%5];"
       ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(x), "r"(y), "r"(z), "r"(bar) : "memory");
+}
+__device__ __forceinline__ void tma_load_im2col_pair(uint32_t dst, const CUtensorMap* map, int c, int w, int h, int n,
+                                                     uint32_t ow, uint32_t oh, uint32_t bar) {
+  asm volatile(
+      "cp.async.bulk.tensor.4d.cta_group::2.shared::cluster.global.im2col.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3, %4, %5}], [%6], {%7, %8};"
+      ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c), "r"(w), "r"(h), "r"(n), "r"(bar),
+        "h"((uint16_t)ow), "h"((uint16_t)oh) : "memory");
 }
 __device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
   asm volatile(
@@ -1225,14 +1310,17 @@ __device__ __forceinline__ void cluster_sync() {
   asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
 
-template <int KIND, int BN_>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
-mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
-                    const __grid_constant__ CUtensorMap tmap_b2,
-                    const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
-                    const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
-                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
-                    uint32_t batch, long long spin_limit, uint32_t drop_fill) {
+// CONV: the implicit-GEMM convolution of mx_conv_kernel on the 256 x 256 pair tile (C % 128 == 0, so
+// the codes of each CTA's 128 output pixels come through the im2col-mode map `tmap_a`); each CTA's
+// scale-producer warp also composes the scale words of its 128 rows (four rows per lane).
+template <int KIND, int BN_, bool CONV>
+__device__ __forceinline__ void
+pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_b2,
+                 const CUtensorMap& tmap_sa, const CUtensorMap& tmap_sb, const CUtensorMap& tmap_c,
+                 uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base, uint32_t group_m,
+                 uint32_t tx_bytes_pair, EpiArgs epi, uint32_t batch, long long spin_limit,
+                 uint32_t drop_fill, const ConvGeom& cg) {
+  static_assert(!CONV || (KIND == 0 && BN_ == 256), "convolution runs on the block-scaled 256 x 256 tile");
   using cfg = Cfg2<KIND, BN_>;
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
   constexpr int BN = cfg::BN;
@@ -1240,7 +1328,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   constexpr int BKe = cfg::kBKe;
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
-  if (smem_base - smem_u32(smem_raw) + cfg::kUsedBytes > cfg::kSmemBytes) {
+  if (smem_base - smem_u32(smem_raw) + (CONV ? cfg::kConvUsedBytes : cfg::kUsedBytes) > (CONV ? cfg::kConvSmemBytes : cfg::kSmemBytes)) {
     // the alignment cost more than the request left room for: give up before anything is set up
     // (uniform over the grid: every CTA sees the same offset)
     if (threadIdx.x == 0) atomicCAS(&g_gemm_status, 0u, (unsigned int)ST_SMEM_ALIGN);
@@ -1254,6 +1342,9 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
   const uint32_t acc_empty_bar = bar0 + 8 * (2 * cfg::kStages + 1);
   auto sf_ready_bar = [&](uint32_t s) { return bar0 + 8 * (2 * cfg::kStages + 2 + s); };
   auto sf_full_bar = [&](uint32_t s) { return bar0 + 8 * (3 * cfg::kStages + 2 + s); };
+  auto conv_a_slot = [&](uint32_t j) { return smem_base + cfg::kOffConvA + 512u * j; };
+  auto a_ok_bar = [&](uint32_t j) { return smem_base + cfg::kOffConvBar + 8u * j; };                  // used in the leader
+  auto asf_bar = [&](uint32_t j) { return smem_base + cfg::kOffConvBar + 8u * (cfg::kConvSlots + j); };  // used in the peer
   volatile uint32_t* tmem_slot =
       reinterpret_cast<volatile uint32_t*>(smem_gen + cfg::kOffBar + cfg::kNumBars * 8);
   volatile uint32_t* abort_flag = tmem_slot + 1;
@@ -1274,10 +1365,17 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       mbar_init(full_bar(s), 1);   // used in the leader only: its producer's arrive + all bytes
       mbar_init(empty_bar(s), 1);  // one tcgen05.commit per use, delivered to both CTAs
       mbar_init(sf_ready_bar(s), 1);  // used in the leader only: the copier's tcgen05.commit
-      mbar_init(sf_full_bar(s), 1);   // used in the leader only: the scale producer's arrive + scale bytes
+      // used in the leader only: the scale producer's arrive + scale bytes
+      mbar_init(sf_full_bar(s), 1);
     }
     mbar_init(acc_full_bar, 1);
     mbar_init(acc_empty_bar, 16);  // eight epilogue warps in each CTA (the leader's barrier is used)
+    if (CONV) {
+      for (uint32_t j = 0; j < cfg::kConvSlots; ++j) {
+        mbar_init(a_ok_bar(j), 33);  // the 32 lanes of the leader's scale-producer warp + the peer's relay
+        mbar_init(asf_bar(j), 32);   // the 32 lanes of the peer's scale-producer warp
+      }
+    }
     *abort_flag = 0;
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -1314,6 +1412,15 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
       const int cy_a = (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128);
       const int cy_b = (int)(tc.b * N + tc.tn * BN + rank * 128);
       const int cy_b2 = (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
+      // CONV: where tap (0, 0) of the first of this CTA's 128 output pixels reads
+      int cv_w = 0, cv_h = 0, cv_n = 0;
+      if (CONV) {
+        const uint32_t m0 = tc.tm * 256 + rank * 128, n0 = fastdiv(m0, cg.d_howo), rem = m0 - n0 * (cg.Ho * cg.Wo);
+        const uint32_t ho = fastdiv(rem, cg.d_wo), wo = rem - ho * cg.Wo;
+        cv_n = (int)n0;
+        cv_h = (int)ho * cg.stride_h - cg.pad_h;
+        cv_w = (int)wo * cg.stride_w - cg.pad_w;
+      }
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
         ok = __all_sync(0xffffffffu, mbar_wait(empty_bar(stage), phase ^ 1u, abort_flag, spin_limit));
         if (!ok) {
@@ -1324,7 +1431,14 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           const uint32_t fb = leader_bar(full_bar(stage));
           if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
           const int cx = (int)(kc * BKe);
-          tma_load_3d_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, cx, cy_a, 0, fb);
+          if (CONV) {  // the stage's K chunk = 128 channels of one filter tap
+            const uint32_t tap = fastdiv(kc * 4, cg.d_cb), cblk = kc * 4 - tap * cg.cb;
+            const uint32_t ti = fastdiv(tap, cg.d_kw), tj = tap - ti * cg.kw;
+            tma_load_im2col_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, (int)(cblk * 32u), cv_w, cv_h,
+                                 cv_n, tj * (uint32_t)cg.dil_w, ti * (uint32_t)cg.dil_h, fb);
+          } else {
+            tma_load_3d_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, cx, cy_a, 0, fb);
+          }
           tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, cx, cy_b, 0, fb);
           if (WIDE)
             tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u, &tmap_b2, cx, cy_b2, 0, fb);
@@ -1405,15 +1519,20 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     // --------------------------- scale copier (leader) ---------------------------
     if constexpr (!DENSE) {
       if (rank == 0) {
-        uint32_t stage = 0, phase = 0;
+        uint32_t stage = 0, phase = 0, conv_chunk = 0;
         bool ok = true;
         for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
           for (uint32_t kc = 0; kc < k_chunks; ++kc) {
-            ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag, spin_limit));
+            const uint32_t aslot = conv_chunk % cfg::kConvSlots, aparity = (conv_chunk / cfg::kConvSlots) & 1u;
+            ok = __all_sync(0xffffffffu, mbar_wait(sf_full_bar(stage), phase, abort_flag, spin_limit) &&
+                                             (!CONV || mbar_wait(a_ok_bar(aslot), aparity, abort_flag, spin_limit)));
             if (!ok) {
               raise_abort(abort_flag, ST_SCALE_WAIT);
               break;
             }
+            // CONV: the A scale words were written by ordinary copies (the peer fenced its own before it arrived)
+            if (CONV) asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            ++conv_chunk;
             tc_fence_after();
             const uint32_t sf_smem = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
             const uint32_t sf_tmem = tmem_base + cfg::kSfCol0 + stage * cfg::kSfCols;
@@ -1423,7 +1542,7 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             if (elect_one()) {
 #pragma unroll
               for (uint32_t c = 0; c < cfg::kKChunks; ++c) {
-                tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(sf_smem + 512 * c));
+                tc_cp_scales_pair(sf_tmem + 4 * c, scale_desc(CONV ? conv_a_slot(aslot) : sf_smem + 512 * c));
 #pragma unroll
                 for (uint32_t g = 0; g < cfg::kSfbGroups; ++g)
                   tc_cp_scales_pair(sf_tmem + cfg::kSfColsA + 4 * cfg::kSfbGroups * c + 4 * g,
@@ -1433,6 +1552,29 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
             }
             __syncwarp();
             if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
+          }
+        }
+      } else if (CONV) {
+        // the peer CTA: pass "my A scale words of chunk g are in my shared memory (and visible to
+        // the tensor core's proxy)" on to the leader's barrier of that slot; this warp has no copies
+        // of its own in flight, so its fence and its arrival wait for nothing
+        uint32_t g = 0;
+        bool ok = true;
+        for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+          for (uint32_t kc = 0; kc < k_chunks; ++kc, ++g) {
+            const uint32_t j = g % cfg::kConvSlots;
+            ok = __all_sync(0xffffffffu, mbar_wait(asf_bar(j), (g / cfg::kConvSlots) & 1u, abort_flag, spin_limit));
+            if (!ok) {
+              raise_abort(abort_flag, ST_SCALE_WAIT);
+              break;
+            }
+            asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+            __syncwarp();
+            // An arrival with the default semantics: the words stay in this CTA's shared memory and
+            // the fence above has made them visible to this SM's tensor-core proxy, which is the only
+            // reader; nothing is published to the other CTA's threads.  (A release at cluster scope
+            // here took ~0.8 us per arrival and set the pace of the whole kernel: 92 against 61 us.)
+            if (lane == 0) mbar_arrive_cluster(map_to_cta(a_ok_bar(j), 0));
           }
         }
       }
@@ -1445,6 +1587,54 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     if constexpr (!DENSE) {
       uint32_t stage = 0, phase = 0;
       bool ok = true;
+      // CONV: the A scale words.  Lane l copies the words of rows l, l + 32, l + 64, l + 96 of this
+      // CTA's 128 output pixels from the activation's scale tensor, asynchronously, into the slot of
+      // the chunk's running number; a cursor walks the CTA's chunks one ring round ahead of the loop
+      // below (so a word has a whole round to arrive, and the hop through the peer's relay is hidden).
+      uint32_t g_tile = pair, g_kc = 0, g_num = 0;   // the cursor: tile, K chunk, running chunk number
+      int32_t cvh[4] = {0, 0, 0, 0}, cvw[4] = {0, 0, 0, 0};
+      uint32_t cvp[4] = {0, 0, 0, 0};  // first pixel of the row's image; 0xFFFFFFFF: row past M
+      auto conv_rows = [&]() {  // geometry of the cursor's tile
+        const TileCoord gc = tile_coord(g_tile, tiles_m, tiles_n, group_m);
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const uint32_t m = gc.tm * 256 + rank * 128 + lane + 32 * j;
+          const uint32_t n0 = fastdiv(m, cg.d_howo), rem = m - n0 * (cg.Ho * cg.Wo);
+          const uint32_t ho = fastdiv(rem, cg.d_wo), wo = rem - ho * cg.Wo;
+          cvh[j] = (int32_t)ho * cg.stride_h - cg.pad_h;
+          cvw[j] = (int32_t)wo * cg.stride_w - cg.pad_w;
+          cvp[j] = m < cg.M ? n0 * cg.H * cg.W : 0xFFFFFFFFu;
+        }
+      };
+      auto conv_gather = [&]() {  // the cursor's chunk, then move the cursor on
+        if (g_tile >= num_tiles) return;
+        const uint32_t slot = g_num % cfg::kConvSlots;
+        // the K chunk is 128 channels of one filter tap: one aligned word of scales per row
+        const uint32_t tap = fastdiv(g_kc * 4, cg.d_cb), cblk = g_kc * 4 - tap * cg.cb;
+        const uint32_t ti = fastdiv(tap, cg.d_kw), tj = tap - ti * cg.kw;
+        const int32_t dh = (int32_t)ti * cg.dil_h, dw = (int32_t)tj * cg.dil_w;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+          const int32_t hi = cvh[j] + dh, wi = cvw[j] + dw;
+          const bool live = cvp[j] != 0xFFFFFFFFu && hi >= 0 && hi < (int32_t)cg.H && wi >= 0 && wi < (int32_t)cg.W;
+          const uint32_t px = live ? cvp[j] + (uint32_t)hi * cg.W + (uint32_t)wi : 0u;
+          const size_t so = cg.x_layout == MX_SCALES_LINEAR ? (size_t)px * cg.cb + cblk
+                                                            : scale_offset<MX_SCALES_SWIZZLED>(px, cblk, cg.cb);
+          // row r = lane + 32 j of the chunk lives at byte (r % 32) * 16 + (r / 32) * 4
+          cp_async_4(conv_a_slot(slot) + lane * 16u + (uint32_t)j * 4u, cg.x_scales + (live ? so : 0), live ? 4u : 0u);
+        }
+        cp_async_arrive(rank == 0 ? a_ok_bar(slot) : asf_bar(slot));
+        ++g_num;
+        if (++g_kc == k_chunks) {
+          g_kc = 0;
+          g_tile += num_pairs;
+          if (g_tile < num_tiles) conv_rows();
+        }
+      };
+      if (CONV && g_tile < num_tiles) {
+        conv_rows();
+        for (uint32_t i = 0; i < (uint32_t)cfg::kStages; ++i) conv_gather();  // the first round's chunks at once
+      }
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
         const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
         const int cz_a = (int)((tc.b * tiles_m + tc.tm) * 2 + rank);
@@ -1457,15 +1647,19 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
           }
           if (elect_one()) {
             const uint32_t fb = leader_bar(sf_full_bar(stage));
-            if (rank == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * cfg::kSfBytes);
+            if (rank == 0) mbar_arrive_expect_tx(sf_full_bar(stage), 2u * (CONV ? cfg::kSfBytes - cfg::kSfABytes : cfg::kSfBytes));
             const uint32_t dst = smem_base + cfg::kOffSf + stage * cfg::kSfBytes;
-            tma_load_3d_pair(dst, &tmap_sa, 0, (int)(kc * cfg::kKChunks), cz_a, fb);
+            if (!CONV) tma_load_3d_pair(dst, &tmap_sa, 0, (int)(kc * cfg::kKChunks), cz_a, fb);
             tma_load_3d_pair(dst + cfg::kSfABytes, &tmap_sb, 0, (int)(kc * cfg::kKChunks), cz_b, fb);
           }
           __syncwarp();
+          // the stage just freed belonged to the chunk one ring round back, and so did the A-scale
+          // slot that the chunk one round AHEAD will use: compose that chunk's words now
+          if (CONV) conv_gather();
           if (++stage == cfg::kStages) { stage = 0; phase ^= 1u; }
         }
       }
+      if (CONV) asm volatile("cp.async.wait_all;" ::: "memory");
       if (!ok) {
         const long long t0 = clock64();
         while (clock64() - t0 < 2000000LL) {}
@@ -1541,6 +1735,30 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
     asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
                  "r"((uint32_t)kTmemCols) : "memory");
   }
+}
+
+template <int KIND, int BN_>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_b2,
+                    const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
+                    const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
+                    uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
+                    uint32_t batch, long long spin_limit, uint32_t drop_fill) {
+  const ConvGeom none = {};
+  pair_kernel_body<KIND, BN_, false>(tmap_a, tmap_b, tmap_b2, tmap_sa, tmap_sb, tmap_c, M, N, K, idesc_base, group_m,
+                                     tx_bytes_pair, epi, batch, spin_limit, drop_fill, none);
+}
+
+static_assert(Cfg2<0, 256>::kConvSmemBytes <= 232448, "shared memory budget of the convolution kernel");
+// Implicit-GEMM convolution on the pair tile (tmap_x: the im2col-mode map over the activation's codes).
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(kThreads, 1)
+mx_conv_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_b,
+                    const __grid_constant__ CUtensorMap tmap_sb, const __grid_constant__ CUtensorMap tmap_c,
+                    uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base, uint32_t group_m,
+                    uint32_t tx_bytes_pair, EpiArgs epi, long long spin_limit, const __grid_constant__ ConvGeom cg) {
+  pair_kernel_body<0, 256, true>(tmap_x, tmap_b, tmap_b, tmap_sb, tmap_sb, tmap_c, M, N, K, idesc_base, group_m,
+                                 tx_bytes_pair, epi, 1u, spin_limit, kNoDrop, cg);
 }
 
 // ---- host side ---------------------------------------------------------------
@@ -1905,14 +2123,44 @@ int launch_conv(const ConvArgs& a, cudaError_t* cuda_err) {
   g.dil_h = a.dil_h; g.dil_w = a.dil_w;
   g.d_wo = make_fastdiv(g.Wo); g.d_howo = make_fastdiv(g.Ho * g.Wo); g.d_kw = make_fastdiv(g.kw);
   g.d_cb = make_fastdiv(g.cb);
+  EpiArgs epi;
+  epi.mode = a.y_bf16 ? 1u : 0u; epi.fmt = 0; epi.sticky = 0; epi.elems = nullptr; epi.scales = nullptr;
   const uint32_t tiles = (uint32_t)((M + BM - 1) / BM) * (uint32_t)((a.Cout + BN - 1) / BN);
+  // 256 x 256 tiles on CTA pairs where the codes come through the im2col map and that costs fewer
+  // waves (same weighting as launch_gemm: a 128 x 128 tile takes 0.82 of a pair tile's time)
+  const int64_t tiles_pair = ((M + 255) / 256) * ((a.Cout + 255) / 256), pairs = a.sm_count / 2;
+  const double cost_pair = (double)((tiles_pair + pairs - 1) / pairs);
+  const double cost_one = (double)((tiles + a.sm_count - 1) / a.sm_count) * 0.82;
+  if (tma && M >= 256 && cost_pair < cost_one) {
+    using cfg2 = Cfg2<0, 256>;
+    CUtensorMap msb2;
+    if (!make_scale_map_k(fn, &msb2, a.w_scales, (uint64_t)a.Cout, (uint64_t)K, cfg2::kSfbGroups, cfg2::kKChunks)) {
+      *cuda_err = cudaErrorInvalidValue;
+      return MX_ERR_CUDA;
+    }
+    static bool attr2_set[64] = {false};
+    if (dev < 0 || dev >= 64 || !attr2_set[dev]) {
+      e = cudaFuncSetAttribute(mx_conv_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg2::kConvSmemBytes);
+      if (e != cudaSuccess) {
+        *cuda_err = e;
+        return MX_ERR_CUDA;
+      }
+      if (dev >= 0 && dev < 64) attr2_set[dev] = true;
+    }
+    const uint32_t np = tiles_pair < pairs ? (uint32_t)tiles_pair : (uint32_t)pairs;
+    // bytes both CTAs report to the leader's stage barrier: 128 x 128 codes of x and 128 rows of the filter each
+    const uint32_t tx_pair = 2u * (uint32_t)(128 * BK + 128 * BK * fmt_bits(a.fmt_w) / 8);
+    const uint32_t idesc2 = (mma_fmt_code(a.fmt_x) << 7) | (mma_fmt_code(a.fmt_w) << 10) | (1u << 23) |
+                            ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
+    *cuda_err = launch_pdl_if(false, mx_conv_pair_kernel, dim3(2 * np), dim3(kThreads), cfg2::kConvSmemBytes, a.stream, mx_, mb,
+                              msb2, mc, (uint32_t)M, (uint32_t)a.Cout, (uint32_t)K, idesc2, 8u, tx_pair, epi, kSpinLimit, g);
+    return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
+  }
   const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
   // the filter tile, plus the 128 x 128 codes of x when they come through the im2col map
   const uint32_t tx_bytes = (uint32_t)(BN * BK * fmt_bits(a.fmt_w) / 8) + (tma ? (uint32_t)(BM * BK) : 0u);
   const uint32_t idesc = (mma_fmt_code(a.fmt_x) << 7) | (mma_fmt_code(a.fmt_w) << 10) | (1u << 23) |
                          ((uint32_t)(BM >> 4) << 24) | ((uint32_t)(BN >> 3) << 17);
-  EpiArgs epi;
-  epi.mode = a.y_bf16 ? 1u : 0u; epi.fmt = 0; epi.sticky = 0; epi.elems = nullptr; epi.scales = nullptr;
   *cuda_err = launch_pdl_if(false, mx_conv_kernel, dim3(grid), dim3(kConvThreads), cfg::kSmemBytes, a.stream, mx_, mb, msb,
                             mc, (uint32_t)M, (uint32_t)a.Cout, (uint32_t)K, idesc, 16u, tx_bytes, epi, kSpinLimit, g);
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;

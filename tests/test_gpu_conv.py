@@ -26,6 +26,9 @@ CASES = [
     (1, 12, 12, 128, 128, 5, 3, (1, 2), (2, 0), (2, 1), 0, 0, 1),     # C % 128 == 0: codes through the im2col map; asymmetric filter, stride, padding, dilation
     (2, 15, 17, 128, 256, 3, 3, (2, 2), (1, 1), (1, 1), 1, 0, 0),     # im2col map, stride 2, odd extents, last tile crosses the batch end
     (3, 7, 9, 384, 128, 2, 4, (1, 1), (0, 2), (1, 1), 0, 2, 1),       # im2col map, three channel chunks per tap, 6-bit filter
+    (8, 56, 56, 128, 256, 3, 3, (1, 1), (1, 1), (1, 1), 0, 0, 1),     # large enough for the 256 x 256 CTA-pair tiles (two waves)
+    (5, 40, 40, 128, 320, 3, 3, (1, 1), (1, 1), (1, 1), 1, 0, 0),     # pair tiles ragged in M (8000 rows) and in Cout, linear scales in
+    (6, 33, 31, 256, 256, 3, 3, (2, 2), (1, 1), (1, 1), 0, 4, 1),     # pair tiles, stride 2, FP4 filter
 ]
 
 
