@@ -432,6 +432,24 @@ def run_extras(torch, mx, inputs, peaks, gpu_index):
     out["config4_mxfp6_training_step"] = {
         "ms_six_quantizes_three_gemms": ts * 1e3, "ms_three_dual_quantizes_three_gemms": tf * 1e3,
         "gemm_flops_per_step": 3 * 2.0 * n ** 3}
+    # convolution (Section 4.1 counts it among the dot-product operations): N 32, 56 x 56, C 256 -> 256, 3 x 3
+    xc = torch.randn((32, 56, 56, 256), device="cuda", dtype=torch.bfloat16)
+    wc = torch.randn((256, 3 * 3 * 256), device="cuda", dtype=torch.bfloat16) * 0.05
+    geom = mx.mx_conv_geometry(32, 56, 56, 256, 3, 3, (1, 1), (1, 1), (1, 1))
+    Mc, Kc = 32 * 56 * 56, 3 * 3 * 256
+    exc, sxc = mx.mx_quantize(xc, 3, mx.MX_E4M3)
+    ewc, swc = mx.mx_quantize(wc, 1, mx.MX_E4M3)
+    eac, sac = mx.mx_im2col(exc, sxc, geom, mx.MX_E4M3)
+    yc = torch.empty((Mc, 256), dtype=torch.float32, device="cuda")
+    t_q = timed(lambda: mx.mx_quantize(xc, 3, mx.MX_E4M3, out=(exc, sxc)), 20)
+    t_i = timed(lambda: mx.mx_im2col(exc, sxc, geom, mx.MX_E4M3), 20)
+    t_g = timed(lambda: mx.mx_gemm(eac, sac, ewc, swc, Mc, 256, Kc, mx.MX_E4M3, mx.MX_E4M3, out=yc), 20)
+    t_c = timed(lambda: mx.mx_conv2d(exc, sxc, ewc, swc, geom, 256, mx.MX_E4M3, mx.MX_E4M3, out=yc), 20)
+    out["conv_n32_56x56_c256_to_256_3x3_e4m3"] = {
+        "us_quantize_x": t_q * 1e6, "us_materialized_im2col": t_i * 1e6, "us_gemm_on_materialized_operand": t_g * 1e6,
+        "us_conv2d_operand_fetched_in_gemm": t_c * 1e6, "conv2d_TFLOPs": 2.0 * Mc * 256 * Kc / t_c / 1e12}
+    del xc, wc, exc, sxc, ewc, swc, eac, sac, yc
+    torch.cuda.empty_cache()
     # the three products of the step, each on its own (operands quantized beforehand)
     (xa, xt), (wb2, wb), (ga, gt) = (mx.mx_quantize_dual(Xc, act, rnd), mx.mx_quantize_dual(Wc, wt, rnd),
                                      mx.mx_quantize_dual(dY, act, rnd))
@@ -837,6 +855,16 @@ def main_case(args):
         out = mx.mx_quantize_dual(T, fmt)
         for _ in range(reps):
             mx.mx_quantize_dual(T, fmt, out=out)
+    elif args.case == "conv":         # N 32, 56 x 56, C 256 -> 256, 3 x 3, padding 1: the operand fetched inside the GEMM
+        x = torch.randn((32, 56, 56, 256), device="cuda", dtype=torch.bfloat16)
+        wt = torch.randn((256, 3 * 3 * 256), device="cuda", dtype=torch.bfloat16) * 0.05
+        fmt = mx.FORMATS[args.fmt]
+        conv = mx.mx_conv_geometry(32, 56, 56, 256, 3, 3, (1, 1), (1, 1), (1, 1))
+        ex, sx = mx.mx_quantize(x, 3, fmt)
+        ew, sw = mx.mx_quantize(wt, 1, fmt)
+        y = torch.empty((32 * 56 * 56, 256), dtype=torch.float32, device="cuda")
+        for _ in range(reps):
+            mx.mx_conv2d(ex, sx, ew, sw, conv, 256, fmt, fmt, out=y, check_status=True)
     elif args.case == "im2col":       # N 32, 56 x 56, C 256, 3 x 3, padding 1: 231 MB of E4M3 codes out
         x = torch.randn((32, 56, 56, 256), device="cuda", dtype=torch.bfloat16)
         fmt = mx.FORMATS[args.fmt]
@@ -851,7 +879,7 @@ def main_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm", "gemm_dense",
-                                       "gemm_few_rows", "quantize_dual", "im2col"],
+                                       "gemm_few_rows", "quantize_dual", "im2col", "conv"],
                     default="step", help="'step' = the benchmark; the others run three launches of one "
                                          "kernel on a small case for a profiler capture")
     ap.add_argument("--fmt", choices=FMT_NAMES, default="e4m3")
