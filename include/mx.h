@@ -78,7 +78,7 @@ typedef enum {
 } mx_status_t;
 
 /* Optional arguments.  A NULL pointer means
- * { MX_F32, MX_SCALES_SWIZZLED, NULL stream, check_status = 0 }. */
+ * { MX_F32, MX_SCALES_SWIZZLED, NULL stream, check_status = 0, pad_k128 = 0 }. */
 typedef struct {
   int32_t dtype;        /* mx_dtype_t of the float tensor (input of quantize,
                            output of dequantize); ignored by mx_gemm          */
@@ -86,6 +86,16 @@ typedef struct {
   void* stream;         /* cudaStream_t                                        */
   int32_t check_status; /* mx_gemm: nonzero = synchronise the stream and return
                            MX_ERR_TIMEOUT if a device-side wait expired        */
+  int32_t pad_k128;     /* 0 or 1.  1: MX tensors are stored as those of the float
+                           tensor zero-extended along the block axis to a multiple
+                           of 128 elements (zero codes under scale byte 0, which
+                           add nothing to a dot product).  mx_quantize writes such
+                           tensors -- sizes: mx_elems_bytes / mx_scales_bytes of the
+                           shape with shape[axis] rounded up to 128 -- and mx_gemm,
+                           mx_gemm_bf16, mx_gemm_ex read them, which lifts the
+                           K % 128 rule of 6- and 4-bit operands to K % 32 == 0.
+                           Every other entry point returns MX_ERR_UNSUPPORTED for 1;
+                           other values: MX_ERR_FMT.                            */
 } mx_opts_t;
 
 /* ------------------------------------------------------------------------- */

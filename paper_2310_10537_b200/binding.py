@@ -42,7 +42,8 @@ EXPORTS = [
 
 class mx_opts_t(ctypes.Structure):
     _fields_ = [("dtype", ctypes.c_int32), ("scale_layout", ctypes.c_int32),
-                ("stream", ctypes.c_void_p), ("check_status", ctypes.c_int32)]
+                ("stream", ctypes.c_void_p), ("check_status", ctypes.c_int32),
+                ("pad_k128", ctypes.c_int32)]
 
 
 class mx_gemm_plan_t(ctypes.Structure):
@@ -141,10 +142,11 @@ def _dtype_code(dt: torch.dtype) -> int:
     raise TypeError(f"unsupported float dtype {dt}")
 
 
-def _opts(dtype: int, layout: int, check: bool = False, stream: Optional[int] = None) -> mx_opts_t:
+def _opts(dtype: int, layout: int, check: bool = False, stream: Optional[int] = None,
+          pad_k128: bool = False) -> mx_opts_t:
     if stream is None:
         stream = torch.cuda.current_stream().cuda_stream
-    return mx_opts_t(dtype, layout, ctypes.c_void_p(stream), 1 if check else 0)
+    return mx_opts_t(dtype, layout, ctypes.c_void_p(stream), 1 if check else 0, 1 if pad_k128 else 0)
 
 
 def _check(status: int, where: str) -> None:
@@ -171,21 +173,25 @@ def mx_scale_offset(row: int, kblock: int, rows: int, kblocks: int,
 
 def mx_quantize(x: torch.Tensor, axis: int, fmt: int, rounding: int = MX_RNE,
                 layout: int = MX_SCALES_SWIZZLED,
-                out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None
-                ) -> Tuple[torch.Tensor, torch.Tensor]:
+                out: Optional[Tuple[torch.Tensor, torch.Tensor]] = None,
+                pad_k128: bool = False) -> Tuple[torch.Tensor, torch.Tensor]:
     """Quantize a contiguous CUDA tensor along ``axis`` (Algorithm 1).
 
     Returns (elems, scales) as flat uint8 tensors; the packed tensor has the
-    quantization axis innermost.  ``out`` lets the caller reuse buffers."""
+    quantization axis innermost.  ``out`` lets the caller reuse buffers.  ``pad_k128``: the
+    result is the MX tensor of x zero-extended along ``axis`` to a multiple of 128."""
     assert x.is_cuda and x.is_contiguous()
     axis %= x.dim()
     shape = list(x.shape)
     if out is None:
-        elems = torch.empty(mx_elems_bytes(shape, axis, fmt), dtype=torch.uint8, device=x.device)
-        scales = torch.empty(mx_scales_bytes(shape, axis, layout), dtype=torch.uint8, device=x.device)
+        stored = list(shape)
+        if pad_k128:
+            stored[axis] = (stored[axis] + 127) // 128 * 128
+        elems = torch.empty(mx_elems_bytes(stored, axis, fmt), dtype=torch.uint8, device=x.device)
+        scales = torch.empty(mx_scales_bytes(stored, axis, layout), dtype=torch.uint8, device=x.device)
     else:
         elems, scales = out
-    o = _opts(_dtype_code(x.dtype), layout)
+    o = _opts(_dtype_code(x.dtype), layout, pad_k128=pad_k128)
     _check(_lib.mx_quantize(x.data_ptr(), elems.data_ptr(), scales.data_ptr(), _shape_arr(shape),
                             len(shape), axis, fmt, rounding, ctypes.byref(o)), "mx_quantize")
     return elems, scales
@@ -228,12 +234,14 @@ def mx_dequantize(elems: torch.Tensor, scales: torch.Tensor, shape: Sequence[int
 
 def mx_gemm(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
             M: int, N: int, K: int, fmtA: int, fmtB: int,
-            out: Optional[torch.Tensor] = None, check_status: bool = False) -> torch.Tensor:
-    """C[M,N] = A[M,K] . B[N,K]^T on MX operands (swizzled scales), FP32 output."""
+            out: Optional[torch.Tensor] = None, check_status: bool = False,
+            pad_k128: bool = False) -> torch.Tensor:
+    """C[M,N] = A[M,K] . B[N,K]^T on MX operands (swizzled scales), FP32 output.  ``pad_k128``:
+    both operands were written by mx_quantize with the same option (K % 32 == 0 then suffices)."""
     assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
     if out is None:
         out = torch.empty((M, N), dtype=torch.float32, device=A.device)
-    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status, pad_k128=pad_k128)
     _check(_lib.mx_gemm(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(), out.data_ptr(),
                         M, N, K, fmtA, fmtB, ctypes.byref(o)), "mx_gemm")
     return out
@@ -241,13 +249,14 @@ def mx_gemm(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor
 
 def mx_gemm_bf16(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
                  M: int, N: int, K: int, fmtA: int, fmtB: int,
-                 out: Optional[torch.Tensor] = None, check_status: bool = False) -> torch.Tensor:
+                 out: Optional[torch.Tensor] = None, check_status: bool = False,
+                 pad_k128: bool = False) -> torch.Tensor:
     """mx_gemm with the FP32 accumulator rounded to nearest even into a BF16 output."""
     assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
     if out is None:
         out = torch.empty((M, N), dtype=torch.bfloat16, device=A.device)
     assert out.dtype == torch.bfloat16
-    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status, pad_k128=pad_k128)
     _check(_lib.mx_gemm_bf16(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(),
                              out.data_ptr(), M, N, K, fmtA, fmtB, ctypes.byref(o)), "mx_gemm_bf16")
     return out
@@ -256,13 +265,14 @@ def mx_gemm_bf16(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.T
 def mx_gemm_ex(A: torch.Tensor, sA: torch.Tensor, B: torch.Tensor, sB: torch.Tensor,
                M: int, N: int, K: int, fmtA: int, fmtB: int, out: Optional[torch.Tensor] = None,
                out_dtype: torch.dtype = torch.float32, tile_n: int = 0, few_rows_limit: int = -1,
-               wait_cycles: int = 0, drop_fill: int = -1, check_status: bool = False) -> torch.Tensor:
+               wait_cycles: int = 0, drop_fill: int = -1, check_status: bool = False,
+               pad_k128: bool = False) -> torch.Tensor:
     """mx_gemm / mx_gemm_bf16 with the kernel selection (tile_n, few_rows_limit) and the device-side
     wait budget (wait_cycles; drop_fill is the failure drill) in the caller's hands."""
     assert A.is_cuda and B.is_cuda and sA.is_cuda and sB.is_cuda
     if out is None:
         out = torch.empty((M, N), dtype=out_dtype, device=A.device)
-    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status)
+    o = _opts(MX_F32, MX_SCALES_SWIZZLED, check=check_status, pad_k128=pad_k128)
     plan = mx_gemm_plan_t(_dtype_code(out.dtype), tile_n, few_rows_limit, drop_fill, wait_cycles)
     _check(_lib.mx_gemm_ex(A.data_ptr(), sA.data_ptr(), B.data_ptr(), sB.data_ptr(), out.data_ptr(),
                            M, N, K, fmtA, fmtB, ctypes.byref(o), ctypes.byref(plan)), "mx_gemm_ex")

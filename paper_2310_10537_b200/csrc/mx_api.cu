@@ -42,7 +42,9 @@ struct View {
 // come out smaller than the tensor it describes.
 constexpr int64_t kMaxElements = (int64_t)1 << 44;
 
-bool make_view(const int64_t* shape, int ndim, int axis, View* v) {
+// pad128: the packed rows (and the scale tensor) are those of the tensor zero-extended along the
+// axis to a multiple of 128 elements (mx_opts_t::pad_k128).
+bool make_view(const int64_t* shape, int ndim, int axis, View* v, bool pad128 = false) {
   if (!shape || ndim < 1 || ndim > 8 || axis < 0 || axis >= ndim) return false;
   v->outer = v->inner = 1;
   for (int i = 0; i < ndim; ++i) {
@@ -53,6 +55,7 @@ bool make_view(const int64_t* shape, int ndim, int axis, View* v) {
   v->L = shape[axis];
   if (v->L > kMaxElements) return false;
   v->kblocks = (v->L + 31) / 32;  // a last, partial block is stored padded with zero codes
+  if (pad128) v->kblocks = (v->kblocks + 3) / 4 * 4;
   v->Lp = v->kblocks * 32;
   if (__builtin_mul_overflow(v->outer, v->inner, &v->rows)) return false;
   if (__builtin_mul_overflow(v->rows, v->L, &v->numel)) return false;
@@ -70,7 +73,7 @@ size_t scales_bytes(int64_t rows, int64_t kblocks, int layout) {
 }
 
 struct Opts {
-  int dtype, layout, check;
+  int dtype, layout, check, pad128;
   cudaStream_t stream;
 };
 bool read_opts(const mx_opts_t* o, Opts* out) {
@@ -78,7 +81,8 @@ bool read_opts(const mx_opts_t* o, Opts* out) {
   out->layout = o ? o->scale_layout : MX_SCALES_SWIZZLED;
   out->stream = o ? (cudaStream_t)o->stream : nullptr;
   out->check = o ? o->check_status : 0;
-  return (out->dtype == MX_F32 || out->dtype == MX_BF16) &&
+  out->pad128 = o ? o->pad_k128 : 0;
+  return (out->pad128 == 0 || out->pad128 == 1) && (out->dtype == MX_F32 || out->dtype == MX_BF16) &&
          (out->layout == MX_SCALES_LINEAR || out->layout == MX_SCALES_SWIZZLED);
 }
 
@@ -152,7 +156,7 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
   if (!shape) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || (rounding != MX_RNE && rounding != MX_RHAZ) || !read_opts(opts, &o))
     return MX_ERR_FMT;
-  if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
+  if (!make_view(shape, ndim, axis, &v, o.pad128 != 0)) return MX_ERR_SHAPE;
   if (v.numel == 0) return MX_OK;
   if (!in || !elems_out || !scales_out) return MX_ERR_NULL;
   if ((uintptr_t)in % 16 || (uintptr_t)elems_out % 16 || (uintptr_t)scales_out % 16)
@@ -163,7 +167,7 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
   cudaError_t e;
   mx::QuantizeArgs a;
   a.in = in; a.elems = (uint8_t*)elems_out; a.scales = scales_out;
-  a.outer = v.outer; a.L = v.L; a.inner = v.inner; a.numel = v.numel;
+  a.outer = v.outer; a.L = v.L; a.L_store = v.Lp; a.inner = v.inner; a.numel = v.numel;
   a.fmt = (int)fmt; a.rounding = (int)rounding; a.dtype = o.dtype; a.layout = o.layout;
   a.stream = o.stream;
   a.sm_count = sm_count(&e);
@@ -184,6 +188,7 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void*
   Opts o;
   if (!fmt_ok((int)fmt) || (rounding != MX_RNE && rounding != MX_RHAZ) || !read_opts(opts, &o))
     return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (R < 0 || C < 0 || R % 32 || C % 32) return MX_ERR_SHAPE;
   if (R == 0 || C == 0) return MX_OK;
   if (!in || !elems_row || !scales_row || !elems_col || !scales_col) return MX_ERR_NULL;
@@ -221,6 +226,7 @@ int mx_dequantize(const void* elems, const uint8_t* scales, void* out, const int
   View v;
   if (!shape) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
   if (axis != ndim - 1) return MX_ERR_UNSUPPORTED;
   if (v.numel == 0) return MX_OK;
@@ -311,6 +317,7 @@ int quantize_host_impl(const void* in_host, void* elems_out_host, uint8_t* scale
   View v;
   if (!shape) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
   if (v.numel == 0) return MX_OK;
   if (!in_host || !elems_out_host || !scales_out_host || !workspace_dev) return MX_ERR_NULL;
@@ -426,6 +433,7 @@ int mx_quantize_host_static(const void* in_host, void* elems_out_host, uint8_t* 
   View v;
   if (!shape) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
   if (mx_quantize_host_workspace_bytes(shape, ndim, axis, fmt, opts) > MX_STATIC_SCRATCH_BYTES)
     return MX_ERR_WORKSPACE;
@@ -450,6 +458,7 @@ static int dequantize_host_impl(const void* elems_host, const uint8_t* scales_ho
   View v;
   if (!shape) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!make_view(shape, ndim, axis, &v)) return MX_ERR_SHAPE;
   if (axis != ndim - 1) return MX_ERR_UNSUPPORTED;
   if (v.numel == 0) return MX_OK;
@@ -576,10 +585,17 @@ static int gemm_device(const void* A, const uint8_t* sA, const void* B, const ui
     if (!q_elems || !q_scales) return MX_ERR_NULL;
     C = q_elems;  // stands in for the output pointer in the checks below
   }
+  if (!read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) {
+    // Operands stored as the tensors zero-extended along K to a multiple of 128 (mx_quantize with
+    // the same option): the product over the extended K is the product over K, term for term.
+    if (batch != 1 || q_elems != nullptr) return MX_ERR_UNSUPPORTED;
+    if (K < 32 || K % 32 || K >= ((int64_t)1 << 31) - 128) return MX_ERR_SHAPE;
+    K = (K + 127) / 128 * 128;
+  }
   int rc = gemm_validate(A, sA, B, sB, C, M, N, K, (int)fmtA, (int)fmtB, batch != 1 || q_elems != nullptr,
                          c_bf16 ? 2 : 4);
   if (rc != MX_OK) return rc;
-  if (!read_opts(opts, &o)) return MX_ERR_FMT;
   if (o.layout != MX_SCALES_SWIZZLED) return MX_ERR_UNSUPPORTED;
   if ((uintptr_t)A % 32 || (uintptr_t)B % 32 || (uintptr_t)sA % 16 || (uintptr_t)sB % 16 ||
       (uintptr_t)C % 16)
@@ -669,6 +685,7 @@ int mx_gemm_dense(const void* A, const uint8_t* sA, const void* B, const uint8_t
   Opts o;
   if (!A || !sA || !B || !sB || !C) return MX_ERR_NULL;
   if (!fmt_ok((int)fmtA) || !fmt_ok((int)fmtB) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if ((int)c_dtype != MX_F32 && (int)c_dtype != MX_BF16) return MX_ERR_FMT;
   if (M < 0 || N < 0 || K < 32 || K % 32 || (N * ((int)c_dtype == MX_BF16 ? 2 : 4)) % 16) return MX_ERR_SHAPE;
   if (M >= ((int64_t)1 << 31) || N >= ((int64_t)1 << 31) || K >= ((int64_t)1 << 31)) return MX_ERR_SHAPE;
@@ -737,6 +754,7 @@ int mx_im2col(const void* elems_in, const uint8_t* scales_in, void* elems_out, u
   Opts o;
   if (!conv) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!conv_ok(conv)) return MX_ERR_SHAPE;
   const int bits = fmt_bits((int)fmt);
   if (conv->C % 32 || (conv->C * bits / 8) % 16) return MX_ERR_SHAPE;
@@ -773,6 +791,7 @@ int mx_conv2d(const void* x_elems, const uint8_t* x_scales, const void* w_elems,
   Opts o;
   if (!conv) return MX_ERR_NULL;
   if (!fmt_ok((int)fmt_x) || !fmt_ok((int)fmt_w) || !read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if ((int)y_dtype != MX_F32 && (int)y_dtype != MX_BF16) return MX_ERR_FMT;
   if (!conv_ok(conv)) return MX_ERR_SHAPE;
   if (fmt_x == MX_INT8 || fmt_w == MX_INT8 || fmt_bits((int)fmt_x) != 8) return MX_ERR_UNSUPPORTED;
@@ -834,6 +853,7 @@ int mx_gemm_host(const void* A_host, const uint8_t* sA_host, const void* B_host,
   int rc = gemm_validate(A_host, sA_host, B_host, sB_host, C_host, M, N, K, (int)fmtA, (int)fmtB, false, 4);
   if (rc != MX_OK) return rc;
   if (!read_opts(opts, &o)) return MX_ERR_FMT;
+  if (o.pad128) return MX_ERR_UNSUPPORTED;  // zero-extended rows: mx_quantize and mx_gemm* only
   if (!workspace_dev) return MX_ERR_NULL;
   if ((uintptr_t)workspace_dev % 256) return MX_ERR_ALIGN;
   if (workspace_bytes < mx_gemm_host_workspace_bytes(M, N, K, fmtA, fmtB)) return MX_ERR_WORKSPACE;

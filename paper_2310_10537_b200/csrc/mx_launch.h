@@ -13,6 +13,7 @@ struct QuantizeArgs {
   uint8_t* elems;
   uint8_t* scales;
   int64_t outer, L, inner;  // input viewed as [outer, L, inner], blocks along L
+  int64_t L_store;          // elements per stored row: L rounded up to whole blocks, or to 128 (zero codes)
   int64_t numel;
   int fmt, rounding, dtype, layout;
   int sm_count;

@@ -538,7 +538,9 @@ static cudaError_t launch_strided(const QuantizeArgs& a) {
 
 // The axis then ends in a partial block: its missing elements count as +0 (they cannot change the
 // block maximum and encode as code 0) and the stored row is padded with zero codes to a whole
-// block.  Rare shapes, so one plain kernel serves every layout: a thread converts one block of the
+// block.  The same kernel writes rows zero-extended to a multiple of 128 elements when the caller asks
+// for them (kblocks then counts the stored blocks; those past the axis end come out as zero codes
+// under scale byte 0).  Rare shapes, so one plain kernel serves every layout: a thread converts one block of the
 // [outer, L, inner] tensor, element by element; consecutive threads take consecutive inner
 // positions (coalesced when the axis is strided) or consecutive blocks of a row.
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
@@ -606,7 +608,7 @@ quantize_tail_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems, u
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
 static cudaError_t launch_tail(const QuantizeArgs& a) {
-  const uint32_t kblocks = (uint32_t)((a.L + kBlock - 1) / kBlock);
+  const uint32_t kblocks = (uint32_t)(a.L_store / kBlock);  // blocks past the axis end are all zero
   const uint64_t total = (uint64_t)a.outer * a.inner * kblocks;
   const uint64_t want = (total + 255) / 256, cap = (uint64_t)a.sm_count * 64;
   return launch_pdl(quantize_tail_kernel<FMT, ROUND, DTYPE, LAYOUT>, dim3((uint32_t)(want < cap ? want : cap)),
@@ -616,7 +618,7 @@ static cudaError_t launch_tail(const QuantizeArgs& a) {
 
 template <int FMT, int ROUND, int DTYPE, int LAYOUT>
 static cudaError_t launch_any(const QuantizeArgs& a) {
-  if (a.L % kBlock != 0) return launch_tail<FMT, ROUND, DTYPE, LAYOUT>(a);
+  if (a.L % kBlock != 0 || a.L_store != a.L) return launch_tail<FMT, ROUND, DTYPE, LAYOUT>(a);
   if (a.inner == 1) return launch_lastaxis<FMT, ROUND, DTYPE, LAYOUT>(a);
   return launch_strided<FMT, ROUND, DTYPE, LAYOUT>(a);
 }

@@ -83,6 +83,28 @@ def test_argument_validation_without_gpu():
     assert lib.mx_strerror(mx.MX_ERR_ALIGN) and lib.mx_strerror(-99)
 
 
+def test_pad_k128_option_is_validated_without_gpu():
+    """pad_k128 takes 0 or 1; only mx_quantize and the plain GEMM entry points accept 1, and with
+    it the K % 128 rule of 6- and 4-bit operands becomes K % 32."""
+    lib = mx.lib()
+    shape = (ctypes.c_int64 * 2)(128, 96)
+    buf = np.zeros(1 << 16, np.uint8)
+    p = buf.ctypes.data + (-buf.ctypes.data) % 256
+    pad = mx.binding.mx_opts_t(mx.MX_F32, mx.MX_SCALES_SWIZZLED, None, 0, 1)
+    bad = mx.binding.mx_opts_t(mx.MX_F32, mx.MX_SCALES_SWIZZLED, None, 0, 2)
+    assert lib.mx_quantize(p, p, p, shape, 2, 1, 4, 0, ctypes.byref(bad)) == mx.MX_ERR_FMT
+    assert lib.mx_gemm(p, p, p, p, p, 128, 128, 96, 4, 4, ctypes.byref(bad)) == mx.MX_ERR_FMT
+    assert lib.mx_quantize(p + 4, p, p, shape, 2, 1, 4, 0, ctypes.byref(pad)) == mx.MX_ERR_ALIGN  # accepted up to here
+    assert lib.mx_gemm(p, p, p, p, p, 128, 128, 48, 4, 4, ctypes.byref(pad)) == mx.MX_ERR_SHAPE   # K % 32 stays
+    assert lib.mx_gemm(p, p, p, p, p + 4, 128, 128, 96, 4, 4, ctypes.byref(pad)) == mx.MX_ERR_ALIGN  # K = 96 passes the shape rules
+    assert lib.mx_gemm(p, p, p, p, p + 4, 128, 128, 96, 4, 4, None) == mx.MX_ERR_SHAPE
+    assert lib.mx_dequantize(p, p, p, shape, 2, 1, 4, ctypes.byref(pad)) == mx.MX_ERR_UNSUPPORTED
+    assert lib.mx_quantize_dual(p, p, p, p, p, 128, 128, 4, 0, ctypes.byref(pad)) == mx.MX_ERR_UNSUPPORTED
+    assert lib.mx_gemm_batched(p, p, p, p, p, 0, 2, 128, 128, 96, 4, 4, ctypes.byref(pad)) == mx.MX_ERR_UNSUPPORTED
+    assert lib.mx_gemm_dense(p, p, p, p, p, 0, 128, 128, 96, 4, 4, ctypes.byref(pad), p, 1 << 20) == mx.MX_ERR_UNSUPPORTED
+    assert lib.mx_quantize_host_static(p, p, p, shape, 2, 1, 4, 0, ctypes.byref(pad)) == mx.MX_ERR_UNSUPPORTED
+
+
 def test_extents_whose_products_wrap_are_rejected():
     """Shapes whose element count wraps a 64-bit integer (2^32 x 2^32 has numel 0 mod 2^64) or is
     simply absurd must come back as MX_ERR_SHAPE / size 0 from every entry point that derives a
