@@ -232,9 +232,6 @@ template <int N>
 __device__ __forceinline__ void bulk_wait_read() {
   asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(N) : "memory");
 }
-__device__ __forceinline__ void bulk_wait_all() {
-  asm volatile("cp.async.bulk.wait_group 0;" ::: "memory");
-}
 
 // r[j][i] = column 32 j + i of this thread's row (row0 + lane) starting at column col0 of C.
 // A staging chunk is 32 rows x 64 bytes: 16 FP32 columns, or 32 BF16 columns (each FP32
@@ -898,7 +895,7 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
       }
       if (++acc == cfg::kAccStages) { acc = 0; acc_phase ^= 1u; }
     }
-    if (lane == 0) bulk_wait_all();  // this warp's stores have completed
+    if (lane == 0) bulk_wait_read<0>();  // the stores have left shared memory; the kernel's end orders the writes
   }
 
   // common exit: every role arrives here, also after an abort
@@ -1723,7 +1720,7 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
       }
       acc_phase ^= 1u;
     }
-    if (lane == 0) bulk_wait_all();
+    if (lane == 0) bulk_wait_read<0>();  // the stores have left shared memory; the kernel's end orders the writes
   }
 
   // common exit: both CTAs of the pair leave together, then the pair's tensor memory is freed
