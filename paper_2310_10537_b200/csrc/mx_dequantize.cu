@@ -42,7 +42,8 @@ __device__ __forceinline__ void decode_pair(uint32_t pair, float& a, float& b) {
 template <int BITS, int KWORDS>
 __device__ __forceinline__ uint32_t code_at_top(const uint32_t (&w)[KWORDS], int e) {
   const int pos = BITS * e, wi = pos / 32, off = pos % 32;
-  if (off + BITS <= 32) return off + BITS == 32 ? w[wi] : w[wi] << (32 - BITS - off);
+  // (the shift runs on the multiply-add unit: the logic / shift pipe is this kernel's busiest)
+  if (off + BITS <= 32) return off + BITS == 32 ? w[wi] : imad(w[wi], 1u << (32 - BITS - off), 0u);
   return __funnelshift_r(w[wi], w[(wi + 1) % KWORDS], off) << (32 - BITS);  // 6-bit code across two words
 }
 
@@ -62,7 +63,9 @@ __device__ __forceinline__ float raw_value(uint32_t t) {
   constexpr int MSHIFT = (FMT == MX_E4M3 || FMT == MX_E2M3) ? 20 : (FMT == MX_E2M1 ? 22 : 21);
   constexpr uint32_t MASK = ((1u << (W - 1)) - 1u) << MSHIFT;
   constexpr int SH = (32 - W) - MSHIFT;
-  return __uint_as_float((t & 0x80000000u) | ((t >> SH) & MASK));
+  // the arithmetic shift drags copies of the sign along down to the magnitude field's top: one
+  // mask keeps bit 31 and the magnitude
+  return __uint_as_float((uint32_t)((int32_t)t >> SH) & (0x80000000u | MASK));
 }
 template <int FMT>
 __device__ __forceinline__ float bias_fix() {  // 2^(127 - bias); INT8: 2^-6

@@ -148,9 +148,17 @@ __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
     // complement for negative x: no float-to-int conversion needed.
     const float a = clamp_abs(lo, 127.0f) + 12582912.0f;
     const float b = clamp_abs(hi, 127.0f) + 12582912.0f;
-    p = (uint16_t)((__float_as_uint(a) & 0xFFu) | ((__float_as_uint(b) & 0xFFu) << 8));
+    p = (uint16_t)__byte_perm(__float_as_uint(a), __float_as_uint(b), 0x0040);  // low bytes of a and b
   }
   return p;
+}
+
+// a * b + c on the integer multiply-add unit (written as PTX so that it is not turned back into
+// shifts and logic operations).
+__device__ __forceinline__ uint32_t imad(uint32_t a, uint32_t b, uint32_t c) {
+  uint32_t d;
+  asm("mad.lo.u32 %0, %1, %2, %3;" : "=r"(d) : "r"(a), "r"(b), "r"(c));
+  return d;
 }
 
 // Packs the four code pairs of 8 consecutive elements (cast_pair results) into the block's
@@ -163,14 +171,17 @@ __device__ __forceinline__ void pack8(const uint32_t (&p)[4], uint32_t& lo, uint
     lo = __byte_perm(p[0], p[1], 0x5410);
     hi = __byte_perm(p[2], p[3], 0x5410);
   } else if (bits == 4) {
-    lo = p[0] | (p[1] << 8) | (p[2] << 16) | (p[3] << 24);
+    lo = imad(p[3], 1u << 24, imad(p[2], 1u << 16, imad(p[1], 1u << 8, p[0])));  // disjoint bytes: sums are ors
     hi = 0;
   } else {
+    // Fields that do not overlap are joined by multiply-add instead of shift + or: the integer
+    // multiply-add issues on the FMA pipe, which this kernel leaves idle, while the logic / shift
+    // pipe is its busiest unit.  p = c0 + 256 c1 (codes below 64)  ->  q = c0 + 64 c1 = p - 192 (p >> 8).
     uint32_t q[4];
 #pragma unroll
-    for (int i = 0; i < 4; ++i) q[i] = (p[i] & 0x3Fu) | ((p[i] >> 2) & 0xFC0u);  // 2 codes -> 12 bits
-    lo = q[0] | (q[1] << 12) | (q[2] << 24);
-    hi = (q[2] >> 8) | (q[3] << 4);
+    for (int i = 0; i < 4; ++i) q[i] = imad(p[i] >> 8, 0xFFFFFF40u, p[i]);  // 2 codes -> 12 bits
+    lo = imad(q[2], 1u << 24, imad(q[1], 1u << 12, q[0]));
+    hi = imad(q[3], 16u, q[2] >> 8);
   }
 }
 

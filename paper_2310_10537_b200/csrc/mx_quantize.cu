@@ -119,22 +119,20 @@ quantize_lastaxis_kernel(const void* __restrict__ in, uint8_t* __restrict__ elem
         }
       } else {
         // 6-bit: each group of 8 codes is 48 bits (lo 32 + hi 16)
-        const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
-        const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
         if (kElems == 32) {
-          const uint64_t g2 = (uint64_t)w[4 % (kElems / 4)] | ((uint64_t)w[5 % (kElems / 4)] << 32);
-          const uint64_t g3 = (uint64_t)w[6 % (kElems / 4)] | ((uint64_t)w[7 % (kElems / 4)] << 32);
-          const uint64_t q0 = g0 | (g1 << 48), q1 = (g1 >> 16) | (g2 << 32), q2 = (g2 >> 32) | (g3 << 16);
+          const uint32_t cw[8] = {w[0], w[1], w[2], w[3], w[4 % (kElems / 4)], w[5 % (kElems / 4)],
+                                  w[6 % (kElems / 4)], w[7 % (kElems / 4)]};
+          uint32_t o[6];
+          pack6_words(cw, o);
           if (ok[u]) {
             uint2* d2 = reinterpret_cast<uint2*>(dst);  // 24-byte blocks are 8-byte aligned
-            d2[0] = make_uint2((uint32_t)q0, (uint32_t)(q0 >> 32));
-            d2[1] = make_uint2((uint32_t)q1, (uint32_t)(q1 >> 32));
-            d2[2] = make_uint2((uint32_t)q2, (uint32_t)(q2 >> 32));
+            d2[0] = make_uint2(o[0], o[1]);
+            d2[1] = make_uint2(o[2], o[3]);
+            d2[2] = make_uint2(o[4], o[5]);
           }
         } else {
           // 12 bytes per lane, 24 per block: the even lane stores bytes 0..15, the odd lane 16..23
-          const uint32_t t0 = (uint32_t)g0, t1 = (uint32_t)(g0 >> 32) | ((uint32_t)g1 << 16),
-                         t2 = (uint32_t)(g1 >> 16);
+          const uint32_t t0 = w[0], t1 = imad(w[2], 1u << 16, w[1]), t2 = __byte_perm(w[2], w[3], 0x5432);
           const uint32_t n0 = __shfl_down_sync(0xFFFFFFFFu, t0, 1);
           if (ok[u]) {
             uint8_t* blk = elems + (size_t)(unit >> 1) * 24;
@@ -279,12 +277,8 @@ quantize_strided_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems
       } else if (bits == 4) {
         reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[2], w[4], w[6]);
       } else {
-        // four 48-bit groups -> 24 bytes
-        const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
-        const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
-        const uint64_t g2 = (uint64_t)w[4] | ((uint64_t)w[5] << 32);
-        const uint64_t g3 = (uint64_t)w[6] | ((uint64_t)w[7] << 32);
-        const uint64_t q0 = g0 | (g1 << 48), q1 = (g1 >> 16) | (g2 << 32), q2 = (g2 >> 32) | (g3 << 16);
+        uint64_t q0, q1, q2;
+        pack6(w, q0, q1, q2);
         uint2* d2 = reinterpret_cast<uint2*>(dst);
         d2[0] = make_uint2((uint32_t)q0, (uint32_t)(q0 >> 32));
         d2[1] = make_uint2((uint32_t)q1, (uint32_t)(q1 >> 32));
@@ -398,11 +392,8 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
         } else if (bits == 4) {
           reinterpret_cast<uint4*>(dst)[0] = make_uint4(w[0], w[2], w[4], w[6]);
         } else {
-          const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
-          const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
-          const uint64_t g2 = (uint64_t)w[4] | ((uint64_t)w[5] << 32);
-          const uint64_t g3 = (uint64_t)w[6] | ((uint64_t)w[7] << 32);
-          const uint64_t q0 = g0 | (g1 << 48), q1 = (g1 >> 16) | (g2 << 32), q2 = (g2 >> 32) | (g3 << 16);
+          uint64_t q0, q1, q2;
+          pack6(w, q0, q1, q2);
           uint2* d2 = reinterpret_cast<uint2*>(dst);  // 8-byte aligned: pitch and 24 j are multiples of 8
           d2[0] = make_uint2((uint32_t)q0, (uint32_t)(q0 >> 32));
           d2[1] = make_uint2((uint32_t)q1, (uint32_t)(q1 >> 32));

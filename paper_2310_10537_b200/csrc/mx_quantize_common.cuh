@@ -34,7 +34,7 @@ __device__ __forceinline__ void unit_group(const uint32_t (&w)[16], int g, float
   if (DTYPE == MX_BF16) {
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
-      x[2 * i] = __uint_as_float(w[4 * g + i] << 16);  // BF16 widens exactly
+      x[2 * i] = __uint_as_float(imad(w[4 * g + i], 1u << 16, 0u));  // BF16 widens exactly (shift on the multiply-add unit)
       x[2 * i + 1] = __uint_as_float(w[4 * g + i] & 0xFFFF0000u);
     }
   } else {
@@ -54,7 +54,7 @@ __device__ __forceinline__ float strided_elem(const uint32_t (&raw)[kBlock][Stri
                                               int k, int c) {
   if (DTYPE == MX_BF16) {
     const uint32_t w = raw[k][(c / 2) % StridedRow<DTYPE, COLS>::kWords];
-    return __uint_as_float((c & 1) ? (w & 0xFFFF0000u) : (w << 16));
+    return __uint_as_float((c & 1) ? (w & 0xFFFF0000u) : imad(w, 1u << 16, 0u));
   }
   return __uint_as_float(raw[k][c % StridedRow<DTYPE, COLS>::kWords]);
 }
@@ -108,15 +108,22 @@ __device__ __forceinline__ void column_cast(const uint32_t (&raw)[kBlock][Stride
   }
 }
 
-// The 24 bytes of a 6-bit block from cast8's four (32 + 16)-bit groups.
+// The 24 bytes of a 6-bit block from cast8's four (32 + 16)-bit groups, as six words: joins of
+// disjoint fields go through the multiply-add unit or one byte permute (see pack8).
+__device__ __forceinline__ void pack6_words(const uint32_t (&w)[8], uint32_t (&o)[6]) {
+  o[0] = w[0];
+  o[1] = imad(w[2], 1u << 16, w[1]);          // w[1] holds 16 bits
+  o[2] = __byte_perm(w[2], w[3], 0x5432);     // (w[2] >> 16) | (w[3] << 16)
+  o[3] = w[4];
+  o[4] = imad(w[6], 1u << 16, w[5]);
+  o[5] = __byte_perm(w[6], w[7], 0x5432);
+}
 __device__ __forceinline__ void pack6(const uint32_t (&w)[8], uint64_t& q0, uint64_t& q1, uint64_t& q2) {
-  const uint64_t g0 = (uint64_t)w[0] | ((uint64_t)w[1] << 32);
-  const uint64_t g1 = (uint64_t)w[2] | ((uint64_t)w[3] << 32);
-  const uint64_t g2 = (uint64_t)w[4] | ((uint64_t)w[5] << 32);
-  const uint64_t g3 = (uint64_t)w[6] | ((uint64_t)w[7] << 32);
-  q0 = g0 | (g1 << 48);
-  q1 = (g1 >> 16) | (g2 << 32);
-  q2 = (g2 >> 32) | (g3 << 16);
+  uint32_t o[6];
+  pack6_words(w, o);
+  q0 = (uint64_t)o[0] | ((uint64_t)o[1] << 32);
+  q1 = (uint64_t)o[2] | ((uint64_t)o[3] << 32);
+  q2 = (uint64_t)o[4] | ((uint64_t)o[5] << 32);
 }
 
 }  // namespace mx
