@@ -91,7 +91,7 @@ __device__ __forceinline__ uint32_t box_chunk(uint32_t box_base, uint32_t r, uin
   return box_base + r * 128u + ((c ^ (r & 7u)) << 4);
 }
 
-template <int FMT, int ROUND, int LAYOUT>
+template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY>
 __global__ void __launch_bounds__(kTileThreads, 2)
 quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
                      uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
@@ -154,7 +154,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
     const uint32_t row0 = tr * kTileRows, col0 = tc * cfg::kCols;
 
     // ------------------------------ row pass ------------------------------
-    if (tid < 128) {
+    if (!COLS_ONLY && tid < 128) {
       constexpr uint32_t kPer = kRowBlocks;  // blocks per thread: its whole tile row
       const uint32_t r = tid, q0 = 0;
       const uint32_t row = row0 + r;
@@ -217,10 +217,11 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
     }
 
     // ----------------------------- column pass -----------------------------
-    if (tid >= 128) {
-      constexpr uint32_t kColThreads = 128;
+    // (COLS_ONLY: the kernel serves mx_quantize along axis 0 and all eight warps take this pass)
+    if (COLS_ONLY || tid >= 128) {
+      constexpr uint32_t kColThreads = COLS_ONLY ? 256 : 128;
       constexpr int kWordCols = 2;   // columns in one 32-bit word
-      const uint32_t ct = tid - 128;
+      const uint32_t ct = COLS_ONLY ? tid : tid - 128;
       uint8_t* codes_smem = gen + cfg::kOffCodes;
       uint8_t* scale_smem = gen + cfg::kOffScales;
       // 64 word columns x 4 row groups = 256 units of 32 rows x one word
@@ -306,7 +307,7 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
   }
 }
 
-template <int FMT, int ROUND, int LAYOUT>
+template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY>
 cudaError_t launch_tile_t(const DualArgs& a) {
   using cfg = TileCfg<FMT>;
   cudaError_t e;
@@ -323,7 +324,7 @@ cudaError_t launch_tile_t(const DualArgs& a) {
   int dev = 0;
   e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  auto kernel = quantize_tile_kernel<FMT, ROUND, LAYOUT>;
+  auto kernel = quantize_tile_kernel<FMT, ROUND, LAYOUT, COLS_ONLY>;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg::kSmem);
     if (e != cudaSuccess) return e;
@@ -340,15 +341,16 @@ cudaError_t launch_tile_t(const DualArgs& a) {
                     a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
 }
 
-template <int FMT, int ROUND>
+template <int FMT, int ROUND, bool COLS_ONLY>
 cudaError_t dispatch_tile_layout(const DualArgs& a) {
-  return a.layout == MX_SCALES_LINEAR ? launch_tile_t<FMT, ROUND, MX_SCALES_LINEAR>(a)
-                                      : launch_tile_t<FMT, ROUND, MX_SCALES_SWIZZLED>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_t<FMT, ROUND, MX_SCALES_LINEAR, COLS_ONLY>(a)
+                                      : launch_tile_t<FMT, ROUND, MX_SCALES_SWIZZLED, COLS_ONLY>(a);
 }
 
-template <int FMT>
+template <int FMT, bool COLS_ONLY>
 cudaError_t dispatch_tile_round(const DualArgs& a) {
-  return a.rounding == MX_RHAZ ? dispatch_tile_layout<FMT, MX_RHAZ>(a) : dispatch_tile_layout<FMT, MX_RNE>(a);
+  return a.rounding == MX_RHAZ ? dispatch_tile_layout<FMT, MX_RHAZ, COLS_ONLY>(a)
+                               : dispatch_tile_layout<FMT, MX_RNE, COLS_ONLY>(a);
 }
 
 }  // namespace
@@ -357,12 +359,24 @@ cudaError_t dispatch_tile_round(const DualArgs& a) {
 cudaError_t launch_quantize_tile(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
   switch (a.fmt) {
-    case MX_E4M3: return dispatch_tile_round<MX_E4M3>(a);
-    case MX_E5M2: return dispatch_tile_round<MX_E5M2>(a);
-    case MX_E3M2: return dispatch_tile_round<MX_E3M2>(a);
-    case MX_E2M3: return dispatch_tile_round<MX_E2M3>(a);
-    case MX_E2M1: return dispatch_tile_round<MX_E2M1>(a);
-    default: return dispatch_tile_round<MX_INT8>(a);
+    case MX_E4M3: return dispatch_tile_round<MX_E4M3, false>(a);
+    case MX_E5M2: return dispatch_tile_round<MX_E5M2, false>(a);
+    case MX_E3M2: return dispatch_tile_round<MX_E3M2, false>(a);
+    case MX_E2M3: return dispatch_tile_round<MX_E2M3, false>(a);
+    case MX_E2M1: return dispatch_tile_round<MX_E2M1, false>(a);
+    default: return dispatch_tile_round<MX_INT8, false>(a);
+  }
+}
+
+// The column-block tensor alone ([C x R], blocks along axis 0 of X[R x C]) for the 6-bit formats:
+// mx_quantize along axis 0 of a 2-D BF16 tensor of whole tiles, where it beats the register kernels
+// (measured on 4096 x 16384: 32.4 against 35.1 us; 8- and 4-bit codes are faster there).
+cudaError_t launch_quantize_tile_cols(const DualArgs& a) {
+  if (a.dtype != MX_BF16 || !a.elems_col || !a.scales_col) return cudaErrorInvalidValue;
+  switch (a.fmt) {
+    case MX_E3M2: return dispatch_tile_round<MX_E3M2, true>(a);
+    case MX_E2M3: return dispatch_tile_round<MX_E2M3, true>(a);
+    default: return cudaErrorInvalidValue;
   }
 }
 

@@ -71,6 +71,23 @@ def test_strided_axis_adversarial_bit_exact(fmt, dtype, inner):
         _assert_same_bytes(s, ws, ("scales", fmt, dtype, inner, layout))
 
 
+@pytest.mark.parametrize("fmt", FMTS)
+@pytest.mark.parametrize("rows,cols", [(128, 128), (384, 640), (1152, 256)])
+def test_strided_axis_whole_tiles_bit_exact(fmt, rows, cols):
+    """Axis 0 of 2-D BF16 tensors made of whole 128 x 128 tiles: the shapes from which the 6-bit
+    formats take the shared-memory tile kernel's column pass (the others keep the register
+    kernels); adversarial blocks, both roundings, both scale layouts, against the oracle."""
+    x = inputs.adversarial("cuda", rows=cols, cols=rows, dtype=torch.bfloat16, seed=21 + fmt).t().contiguous()
+    assert list(x.shape) == [rows, cols]
+    xin = to_oracle_input(x)
+    for rounding in (mx.MX_RNE, mx.MX_RHAZ):
+        for layout in (mx.MX_SCALES_LINEAR, mx.MX_SCALES_SWIZZLED):
+            e, s = _quantize_guarded(x, 0, fmt, rounding, layout)
+            we, ws = O.quantize(xin, 0, fmt, rounding, layout)
+            _assert_same_bytes(e, we, ("elems", fmt, rows, cols, rounding, layout))
+            _assert_same_bytes(s, ws, ("scales", fmt, rows, cols, rounding, layout))
+
+
 @pytest.mark.parametrize("fmt", [mx.MX_E4M3, mx.MX_E3M2, mx.MX_E2M1, mx.MX_INT8])
 def test_middle_axis_of_3d_tensor(fmt):
     x = inputs.adversarial("cuda", rows=3 * 40, cols=64, dtype=torch.float32, seed=3)
