@@ -1199,7 +1199,7 @@ struct Cfg2 {
   static constexpr bool F4 = KIND == 1;
   static constexpr bool DENSE = KIND == 2;
   static constexpr int BN = BN_;
-  static constexpr int kStages = BN == 384 ? (F4 ? 4 : 5) : (F4 ? 5 : 6);
+  static constexpr int kStages = BN == 384 ? (F4 ? 4 : 5) : 6;
   static constexpr int kBKe = F4 ? 256 : DENSE ? 64 : 128;  // K elements per stage (128-byte operand rows)
   static constexpr int kKChunks = F4 ? 2 : 1;           // 512-byte scale chunks (4 MX blocks) along K per stage
   static constexpr int kSfbGroups = BN / 128;           // 128-row scale chunks of B per K chunk
