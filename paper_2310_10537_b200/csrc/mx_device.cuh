@@ -125,7 +125,9 @@ __device__ __forceinline__ BlockScale block_scale(float amax) {
 // has that bit clear, so a tie moves just past the half-way point and nothing
 // else crosses one.
 // Result: code(lo) | code(hi) << 8   (FP4: code(lo) | code(hi) << 4).
-template <int FMT, int ROUND>
+// CLAMP (INT8 only): false when the caller knows that no element of the block reaches 127.5 in
+// magnitude after scaling (the saturation then has nothing to do).
+template <int FMT, int ROUND, bool CLAMP = true>
 __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
   if (ROUND == MX_RHAZ) {
     lo = __uint_as_float(__float_as_uint(lo) | 1u);
@@ -146,8 +148,8 @@ __device__ __forceinline__ uint32_t cast_pair(float lo, float hi) {
   } else {  // INT8: value n/64, inputs already multiplied by 64; saturate at +-127
     // x + 1.5 * 2^23 rounds x to an integer (nearest even) in the low mantissa bits, as two's
     // complement for negative x: no float-to-int conversion needed.
-    const float a = clamp_abs(lo, 127.0f) + 12582912.0f;
-    const float b = clamp_abs(hi, 127.0f) + 12582912.0f;
+    const float a = (CLAMP ? clamp_abs(lo, 127.0f) : lo) + 12582912.0f;
+    const float b = (CLAMP ? clamp_abs(hi, 127.0f) : hi) + 12582912.0f;
     p = (uint16_t)__byte_perm(__float_as_uint(a), __float_as_uint(b), 0x0040);  // low bytes of a and b
   }
   return p;
@@ -186,7 +188,7 @@ __device__ __forceinline__ void pack8(const uint32_t (&p)[4], uint32_t& lo, uint
 }
 
 // Convert 8 consecutive elements of one block (output as pack8).
-template <int FMT, int ROUND>
+template <int FMT, int ROUND, bool CLAMP = true>
 __device__ __forceinline__ void cast8(const float (&v)[8], const BlockScale& s, uint32_t& lo,
                                       uint32_t& hi) {
   uint32_t p[4];
@@ -194,7 +196,7 @@ __device__ __forceinline__ void cast8(const float (&v)[8], const BlockScale& s, 
   for (int i = 0; i < 4; ++i) {
     float a = mul_ftz(v[2 * i], s.m1), b = mul_ftz(v[2 * i + 1], s.m1);
     if (FMT == MX_INT8) { a *= s.m2; b *= s.m2; }
-    p[i] = cast_pair<FMT, ROUND>(a, b);
+    p[i] = cast_pair<FMT, ROUND, CLAMP>(a, b);
   }
   pack8<FMT>(p, lo, hi);
   if (!s.finite) { lo = 0; hi = 0; }

@@ -71,6 +71,35 @@ def test_strided_axis_adversarial_bit_exact(fmt, dtype, inner):
         _assert_same_bytes(s, ws, ("scales", fmt, dtype, inner, layout))
 
 
+@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("rounding", [mx.MX_RNE, mx.MX_RHAZ])
+def test_int8_saturation_boundary(dtype, rounding):
+    """MXINT8 saturates at +-127: block maxima that scale to just below, exactly and just above
+    127.5 (the smallest value that rounds to 128), of either sign, scattered so that some warps of
+    the kernel hold a saturating block and others none (the kernel skips the clamp for those)."""
+    rows, cols = 96, 2048
+    g = torch.Generator().manual_seed(17)
+    x = (torch.rand((rows, cols), generator=g) - 0.5) * 0.5           # |x| < 0.25: never the block maximum
+    tops = [127.5 / 64, 127.0 / 64, 1.984375, 1.99609375, 1.0, 127.5 / 64 * 4, -127.5 / 64, -1.99609375 / 8]
+    if dtype == torch.float32:
+        t = np.float32(127.5 / 64)
+        tops += [float(np.nextafter(t, np.float32(0))), float(np.nextafter(t, np.float32(4))),
+                 -float(np.nextafter(t, np.float32(0)))]
+    k = 0
+    for r in range(0, rows, 3):                 # every third row gets maxima, the rows between get none
+        for b in range(0, cols // 32, 5):
+            x[r, b * 32 + (k * 7) % 32] = tops[k % len(tops)]
+            k += 1
+    x = x.to(dtype).cuda()
+    xin = to_oracle_input(x)
+    for layout in (mx.MX_SCALES_LINEAR, mx.MX_SCALES_SWIZZLED):
+        e, s = _quantize_guarded(x, 1, mx.MX_INT8, rounding, layout)
+        we, ws = O.quantize(xin, 1, mx.MX_INT8, rounding, layout)
+        _assert_same_bytes(e, we, ("elems", dtype, rounding, layout))
+        _assert_same_bytes(s, ws, ("scales", dtype, rounding, layout))
+    assert (we == 0x7F).any() and (we == 0x81).any()   # the clamp did have something to do
+
+
 @pytest.mark.parametrize("fmt", FMTS)
 @pytest.mark.parametrize("rows,cols", [(128, 128), (384, 640), (1152, 256)])
 def test_strided_axis_whole_tiles_bit_exact(fmt, rows, cols):
