@@ -939,8 +939,8 @@ mx_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 // The product is bound by reading B once from HBM, and what a CTA can have in flight is bounded by
 // its shared memory, so the operands change places: the tile's 128 rows of B take the M side of
 // the MMA (one TMEM lane per row of B) and the MP = M rounded up to 16 rows of A its N side.  A
-// stage is then 16 KB of B + MP x 128 bytes of A instead of 16 KB + 16 KB, and the ring holds up
-// to twelve of them.  The accumulator is C transposed -- lane = column n of C, column = row m --
+// K chunk is then 16 KB of B + MP x 128 bytes of A instead of 16 KB + 16 KB; a stage holds two
+// chunks and the ring up to six stages.  The accumulator is C transposed -- lane = column n of C, column = row m --
 // which the epilogue writes with plain stores: for every m the 32 lanes of a warp store 32
 // consecutive columns.
 // Warps: 0 operand producer, 1 MMA issuer, 2..5 epilogue (one per TMEM lane quarter), 10 scale
@@ -964,15 +964,18 @@ __global__ void __launch_bounds__(kThreads, 1)
 mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                       const __grid_constant__ CUtensorMap tmap_sw, const __grid_constant__ CUtensorMap tmap_sx,
                       void* __restrict__ C, uint32_t M, uint32_t N, uint32_t K, uint32_t MP,
-                      uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t c_bf16,
+                      uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t kch, uint32_t c_bf16,
                       long long spin_limit, uint32_t drop_fill) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
-  const uint32_t x_bytes = MP * 128u;
-  const uint32_t off_x = stages * 16384u;
-  const uint32_t off_sf = off_x + stages * x_bytes;
-  const uint32_t off_bar = off_sf + stages * 1024u;
+  // a stage holds kch K chunks of 128 elements (two where the weights are sub-byte codes: their
+  // chunk is half the HBM bytes for the same per-stage hand-shakes)
+  const uint32_t x_bytes = MP * 128u;                 // per K chunk
+  const uint32_t w_stage = kch * 16384u, x_stage = kch * x_bytes, sf_stage = kch * 1024u;
+  const uint32_t off_x = stages * w_stage;
+  const uint32_t off_sf = off_x + stages * x_stage;
+  const uint32_t off_bar = off_sf + stages * sf_stage;
   const uint32_t bar0 = smem_base + off_bar;
   auto full_bar = [&](uint32_t s) { return bar0 + 8 * s; };
   auto empty_bar = [&](uint32_t s) { return bar0 + 8 * (kSkinnyMaxStages + s); };
@@ -985,7 +988,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
 
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t tiles_n = (N + 127u) / 128u;
-  const uint32_t k_chunks = (K + BK - 1) / BK;  // a K tail is zero-filled by the copies
+  const uint32_t k_chunks = ((K + BK - 1) / BK + kch - 1) / kch;  // stages per tile; a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
     for (uint32_t s = 0; s < stages; ++s) {
@@ -1035,16 +1038,22 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
           break;
         }
         if ((scales || fill++ != drop_fill) && elect_one()) {
-          if (scales) {  // (0, K chunk, 128-row group)
+          if (scales) {  // (0, K chunk, 128-row group); a chunk past K is zero-filled like a tail
             const uint32_t fb = sf_full_bar(stage);
-            mbar_arrive_expect_tx(fb, 1024u);
-            tma_load_3d(smem_base + off_sf + stage * 1024u, &tmap_sw, 0, (int)kc, (int)t, fb);
-            tma_load_3d(smem_base + off_sf + stage * 1024u + 512u, &tmap_sx, 0, (int)kc, 0, fb);
+            mbar_arrive_expect_tx(fb, sf_stage);
+            for (uint32_t c = 0; c < kch; ++c) {
+              const uint32_t dst = smem_base + off_sf + stage * sf_stage + c * 1024u;
+              tma_load_3d(dst, &tmap_sw, 0, (int)(kc * kch + c), (int)t, fb);
+              tma_load_3d(dst + 512u, &tmap_sx, 0, (int)(kc * kch + c), 0, fb);
+            }
           } else {  // (k, row, 0)
             const uint32_t fb = full_bar(stage);
-            mbar_arrive_expect_tx(fb, tx_bytes);
-            tma_load_3d(smem_base + stage * 16384u, &tmap_w, (int)(kc * BK), (int)(t * 128u), 0, fb);
-            tma_load_3d(smem_base + off_x + stage * x_bytes, &tmap_x, (int)(kc * BK), 0, 0, fb);
+            mbar_arrive_expect_tx(fb, kch * tx_bytes);
+            for (uint32_t c = 0; c < kch; ++c) {
+              const int kx = (int)((kc * kch + c) * BK);
+              tma_load_3d(smem_base + stage * w_stage + c * 16384u, &tmap_w, kx, (int)(t * 128u), 0, fb);
+              tma_load_3d(smem_base + off_x + stage * x_stage + c * x_bytes, &tmap_x, kx, 0, 0, fb);
+            }
           }
         }
         __syncwarp();
@@ -1067,11 +1076,13 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
           break;
         }
         tc_fence_after();
-        const uint32_t sf_smem = smem_base + off_sf + stage * 1024u;
-        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
+        const uint32_t sf_smem = smem_base + off_sf + stage * sf_stage;
+        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u * kch;
         if (elect_one()) {
-          tc_cp_scales(sf_tmem, scale_desc(sf_smem));            // rows of B: the MMA's A-side scales
-          tc_cp_scales(sf_tmem + 4, scale_desc(sf_smem + 512));  // rows of A: its B-side scales
+          for (uint32_t c = 0; c < kch; ++c) {
+            tc_cp_scales(sf_tmem + 8 * c, scale_desc(sf_smem + 1024 * c));            // rows of B: the MMA's A-side scales
+            tc_cp_scales(sf_tmem + 8 * c + 4, scale_desc(sf_smem + 1024 * c + 512));  // rows of A: its B-side scales
+          }
           tc_commit(sf_ready_bar(stage));
         }
         __syncwarp();
@@ -1097,15 +1108,17 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
           break;
         }
         tc_fence_after();
-        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u;
-        const uint64_t wdesc = operand_desc(smem_base + stage * 16384u);
-        const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_bytes);
         if (elect_one()) {
+          for (uint32_t c = 0; c < kch; ++c) {
+            const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u * kch + 8 * c;
+            const uint64_t wdesc = operand_desc(smem_base + stage * w_stage + c * 16384u);
+            const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_stage + c * x_bytes);
 #pragma unroll
-          for (uint32_t k = 0; k < BK / kMmaK; ++k) {
-            // byte k of each 32-bit scale column belongs to MX block k of this stage
-            const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
-            tc_mma(d_tmem, wdesc + 2 * k, xdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4, (kc | k) != 0 ? 1u : 0u);
+            for (uint32_t k = 0; k < BK / kMmaK; ++k) {
+              // byte k of each 32-bit scale column belongs to MX block k of this chunk
+              const uint32_t idesc = idesc_base | (k << 4) | (k << 29);
+              tc_mma(d_tmem, wdesc + 2 * k, xdesc + 2 * k, idesc, sf_tmem, sf_tmem + 4, (kc | c | k) != 0 ? 1u : 0u);
+            }
           }
           tc_commit(empty_bar(stage));
         }
@@ -1972,10 +1985,14 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
       !make_scale_map(fn, &msw, a.sB, (uint64_t)a.N, (uint64_t)a.K, 1) ||
       !make_scale_map(fn, &msx, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1))
     return cudaErrorInvalidValue;
-  const uint32_t stage_bytes = 16384u + MP * 128u + 1024u;
+  // K chunks per stage: with one, the per-stage hand-shakes (about 550 cycles for four small MMAs)
+  // set the pace -- 16 x 28672 x 8192: 48.6 us with E4M3 weights, 41.5 us with E2M1 weights, whose
+  // chunk is half the HBM bytes; with two 42.3 and 29.8 us; three or four (fewer stages) are slower
+  constexpr uint32_t kch = 2;
+  const uint32_t stage_bytes = kch * (16384u + MP * 128u + 1024u);
   const uint32_t fixed = kSkinnyBars * 8u + 16u + 1024u;  // barriers, TMEM slot + abort flag, alignment slack
   uint32_t stages = (232448u - fixed) / stage_bytes;
-  if (stages > kSkinnyMaxStages) stages = kSkinnyMaxStages;
+  if (stages > kSkinnyMaxStages / kch) stages = kSkinnyMaxStages / kch;
   const uint32_t smem = stages * stage_bytes + fixed;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -1994,7 +2011,7 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t idesc = (mma_fmt_code(a.fmtB) << 7) | (mma_fmt_code(a.fmtA) << 10) | (1u << 23) |
                          ((MP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   return launch_pdl_if(small_product(a), mx_gemm_skinny_kernel, dim3(grid), dim3(kThreads), smem, a.stream, mw, mx_, msw, msx, a.C,
-                    (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, a.c_bf16 ? 1u : 0u,
+                    (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, kch, a.c_bf16 ? 1u : 0u,
                     wait_budget(a), drop_fill(a));
 }
 
