@@ -544,6 +544,28 @@ def run_report(torch, mx, inputs):
     quantize_rows("C5 X BF16 16384x8192", d5["X"], 1, [0])
     quantize_rows("C5 W BF16 8192x28672", d5["W"], 0, [4])
 
+    # decode-shaped products: a few rows of activations against a weight matrix (the weights are read once);
+    # measured before the tensor-bound loops, which leave the SM clock low for a while
+    lines += ["", "## GEMM with few rows of A (HBM-bound on the weights)", "",
+              "Bytes = weight codes + weight scales (what has to come from HBM once); columns as in the first table.", "",
+              "| shape, formats | MB | median | best | back-to-back | GB/s | % measured | % nominal |",
+              "|---|---|---|---|---|---|---|---|"]
+    g = torch.Generator(device="cuda").manual_seed(2024)
+    for (M, N, K, fb) in ((16, 16384, 4096, 0), (16, 28672, 8192, 0), (64, 28672, 8192, 0), (16, 28672, 8192, 2),
+                          (16, 28672, 8192, 4)):
+        A = torch.randn((M, K), generator=g, device="cuda", dtype=torch.bfloat16)
+        ea, sa = mx.mx_quantize(A, 1, 0)
+        Ws = []
+        for _ in range(3):
+            W = torch.randn((N, K), generator=g, device="cuda", dtype=torch.bfloat16) * 0.02
+            Ws.append(mx.mx_quantize(W, 1, fb))
+            del W
+        C = torch.empty((M, N), dtype=torch.float32, device="cuda")
+        t = protocol(lambda i: mx.mx_gemm(ea, sa, Ws[i][0], Ws[i][1], M, N, K, 0, fb, out=C), 3)
+        stream_row(f"{M} x {N} x {K}, E4M3 activations x {FMT_NAMES[fb]} weights", Ws[0][0].numel() + Ws[0][1].numel(), t)
+        del Ws, C
+        torch.cuda.empty_cache()
+
     lines += ["", "## GEMM (tensor-bound)", "",
               f"Peaks: 2 x measured BF16 burst = {fp8_burst:.0f} TFLOP/s, 2 x measured BF16 sustained = "
               f"{fp8_sust:.0f}, nominal dense FP8 {fp8_nom:.0f}.  Columns as above; `sustained` = a loop of at "
