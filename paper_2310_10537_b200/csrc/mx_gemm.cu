@@ -948,7 +948,13 @@ mx_conv_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant
 // ============================================================================
 constexpr uint32_t kSkinnyMaxStages = 12;
 constexpr uint32_t kSkinnyBars = 4 * kSkinnyMaxStages + 4;
-constexpr uint32_t kSkinnySfCol0 = 256;  // accumulators at columns 0 and 128, 8 scale columns per stage behind
+// Tensor memory of the few-rows kernel: two accumulators of MP columns, `acc_stride` columns apart,
+// and 8 scale columns per K chunk of every stage behind them.  One CTA per SM takes all 512 columns
+// (accumulators at 0 and 128, scales from 256); where two CTAs share an SM (MP <= 96) each takes 256
+// (accumulators at 0 and 96, scales from 192).
+struct SkinnyTmem {
+  uint32_t cols, acc_stride, sf_col0;
+};
 
 __device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t (&r)[16]) {
   asm volatile(
@@ -965,7 +971,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
                       const __grid_constant__ CUtensorMap tmap_sw, const __grid_constant__ CUtensorMap tmap_sx,
                       void* __restrict__ C, uint32_t M, uint32_t N, uint32_t K, uint32_t MP,
                       uint32_t idesc_base, uint32_t tx_bytes, uint32_t stages, uint32_t kch, uint32_t c_bf16,
-                      long long spin_limit, uint32_t drop_fill) {
+                      long long spin_limit, uint32_t drop_fill, SkinnyTmem tm) {
   extern __shared__ uint8_t smem_raw[];
   const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
   uint8_t* smem_gen = smem_raw + (smem_base - smem_u32(smem_raw));
@@ -1009,7 +1015,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
   }
   if (warp == 1) {
     asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
-                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"((uint32_t)kTmemCols) : "memory");
+                 ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))), "r"(tm.cols) : "memory");
     asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
   }
   tc_fence_before();
@@ -1077,7 +1083,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
         }
         tc_fence_after();
         const uint32_t sf_smem = smem_base + off_sf + stage * sf_stage;
-        const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u * kch;
+        const uint32_t sf_tmem = tmem_base + tm.sf_col0 + stage * 8u * kch;
         if (elect_one()) {
           for (uint32_t c = 0; c < kch; ++c) {
             tc_cp_scales(sf_tmem + 8 * c, scale_desc(sf_smem + 1024 * c));            // rows of B: the MMA's A-side scales
@@ -1099,7 +1105,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
         break;
       }
       tc_fence_after();
-      const uint32_t d_tmem = tmem_base + acc * 128u;
+      const uint32_t d_tmem = tmem_base + acc * tm.acc_stride;
       for (uint32_t kc = 0; kc < k_chunks; ++kc) {
         ok = __all_sync(0xffffffffu, mbar_wait(sf_ready_bar(stage), phase, abort_flag, spin_limit) &&
                                          mbar_wait(full_bar(stage), phase, abort_flag, spin_limit));
@@ -1110,7 +1116,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
         tc_fence_after();
         if (elect_one()) {
           for (uint32_t c = 0; c < kch; ++c) {
-            const uint32_t sf_tmem = tmem_base + kSkinnySfCol0 + stage * 8u * kch + 8 * c;
+            const uint32_t sf_tmem = tmem_base + tm.sf_col0 + stage * 8u * kch + 8 * c;
             const uint64_t wdesc = operand_desc(smem_base + stage * w_stage + c * 16384u);
             const uint64_t xdesc = operand_desc(smem_base + off_x + stage * x_stage + c * x_bytes);
 #pragma unroll
@@ -1140,7 +1146,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
       }
       tc_fence_after();
       const uint32_t n = t * 128u + quarter * 32u + lane;  // this thread's column of C
-      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * 128u;
+      const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + acc * tm.acc_stride;
       for (uint32_t c = 0; c < MP; c += 16) {
         uint32_t r[16];
         tc_ld16(taddr + c, r);
@@ -1176,7 +1182,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
   if (warp == 1) {
     tc_fence_after();
     asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base),
-                 "r"((uint32_t)kTmemCols) : "memory");
+                 "r"(tm.cols) : "memory");
   }
 }
 
@@ -1985,14 +1991,23 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
       !make_scale_map(fn, &msw, a.sB, (uint64_t)a.N, (uint64_t)a.K, 1) ||
       !make_scale_map(fn, &msx, a.sA, (uint64_t)a.M, (uint64_t)a.K, 1))
     return cudaErrorInvalidValue;
-  // K chunks per stage: with one, the per-stage hand-shakes (about 550 cycles for four small MMAs)
-  // set the pace -- 16 x 28672 x 8192: 48.6 us with E4M3 weights, 41.5 us with E2M1 weights, whose
-  // chunk is half the HBM bytes; with two 42.3 and 29.8 us; three or four (fewer stages) are slower
-  constexpr uint32_t kch = 2;
+  // One CTA per SM: two K chunks per stage (with one, the per-stage hand-shakes -- about 550 cycles
+  // for four small MMAs -- set the pace: 16 x 28672 x 8192 took 48.6 us with E4M3 weights and 41.5 us
+  // with E2M1 weights, whose chunk is half the HBM bytes; with two 42.3 and 29.8 us; three or four,
+  // i.e. fewer stages, are slower).  Where the tiles would need a second, partly empty round -- more
+  // tiles than SMs, at most twice as many -- two CTAs share an SM instead (MP <= 96: half the shared
+  // and tensor memory each, one chunk per stage): every tile is resident at once and an SM has two
+  // MMA issuers (E2M1 weights 29.8 -> 27.2 us, 96 rows of E4M3 52.9 -> 50.9; slower outside that range).
+  const uint32_t tiles = (uint32_t)((a.N + 127) / 128);
+  const bool two = MP <= 96 && tiles > (uint32_t)a.sm_count && tiles <= 2u * (uint32_t)a.sm_count;
+  const uint32_t kch = two ? 1u : 2u;
+  const uint32_t budget = kch == 1 ? 232448u / 2 : 232448u;
   const uint32_t stage_bytes = kch * (16384u + MP * 128u + 1024u);
   const uint32_t fixed = kSkinnyBars * 8u + 16u + 1024u;  // barriers, TMEM slot + abort flag, alignment slack
-  uint32_t stages = (232448u - fixed) / stage_bytes;
+  uint32_t stages = (budget - fixed) / stage_bytes;
   if (stages > kSkinnyMaxStages / kch) stages = kSkinnyMaxStages / kch;
+  if (kch == 1 && stages > 8) stages = 8;  // 8 scale columns per stage behind column 192 of 256
+  const SkinnyTmem tm = kch == 1 ? SkinnyTmem{256u, 96u, 192u} : SkinnyTmem{(uint32_t)kTmemCols, 128u, 256u};
   const uint32_t smem = stages * stage_bytes + fixed;
   static bool attr_set[64] = {false};
   int dev = 0;
@@ -2003,8 +2018,8 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles = (uint32_t)((a.N + 127) / 128);
-  const uint32_t grid = tiles < (uint32_t)a.sm_count ? tiles : (uint32_t)a.sm_count;
+  const uint32_t slots = (kch == 1 ? 2u : 1u) * (uint32_t)a.sm_count;
+  const uint32_t grid = tiles < slots ? tiles : slots;
   // bytes the two operand copies report (packed source bytes, rows past the end included)
   const uint32_t tx_bytes = (uint32_t)(128 * BK * fmt_bits(a.fmtB) / 8) + MP * (uint32_t)(BK * fmt_bits(a.fmtA) / 8);
   // the MMA's A side is B (format field [7,10)), its B side is A ([10,13)); N field = MP, M = 128
@@ -2012,7 +2027,7 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
                          ((MP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
   return launch_pdl_if(small_product(a), mx_gemm_skinny_kernel, dim3(grid), dim3(kThreads), smem, a.stream, mw, mx_, msw, msx, a.C,
                     (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, kch, a.c_bf16 ? 1u : 0u,
-                    wait_budget(a), drop_fill(a));
+                    wait_budget(a), drop_fill(a), tm);
 }
 
 }  // namespace
