@@ -117,6 +117,21 @@ def test_strided_axis_whole_tiles_bit_exact(fmt, rows, cols):
             _assert_same_bytes(s, ws, ("scales", fmt, rows, cols, rounding, layout))
 
 
+@pytest.mark.parametrize("fmt,rounding", [(mx.MX_E3M2, mx.MX_RNE), (mx.MX_E2M3, mx.MX_RHAZ)])
+def test_strided_axis_6bit_at_weight_size(fmt, rounding):
+    """The FFN weight of configuration 3 (4096 x 16384 BF16) quantized along axis 0 to the 6-bit
+    formats -- the size at which this path is timed, and the one that takes the tile kernel's column
+    pass: 256 sampled output rows (both ends, tile seams, middle) byte for byte against the oracle,
+    and the whole tensor against the last-axis kernel on the transposed input."""
+    from gpu_util import assert_operand_rows_match_oracle
+    w = inputs.config3("cuda")["W"]
+    assert list(w.shape) == [4096, 16384] and w.dtype == torch.bfloat16
+    e, s = mx.mx_quantize(w, 0, fmt, rounding)
+    assert_operand_rows_match_oracle(O, w, 0, fmt, rounding, e, s, f"W axis 0 fmt {fmt}", count=256, seed=fmt)
+    et, st = mx.mx_quantize(w.t().contiguous(), 1, fmt, rounding)
+    assert torch.equal(e, et) and torch.equal(s, st)
+
+
 @pytest.mark.parametrize("fmt", [mx.MX_E4M3, mx.MX_E3M2, mx.MX_E2M1, mx.MX_INT8])
 def test_middle_axis_of_3d_tensor(fmt):
     x = inputs.adversarial("cuda", rows=3 * 40, cols=64, dtype=torch.float32, seed=3)
