@@ -506,7 +506,7 @@ gemm_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // A small product is launched with programmatic stream serialization: everything above then
+  // The kernel is launched with programmatic stream serialization: everything above then
   // overlapped the tail of the kernel before, and nothing below touches global memory before that
   // kernel has completed.  The kernel does not announce its own dependents early: CTAs of a
   // following kernel that wait on SMs this grid has already left slowed the rest of it down (a
@@ -1022,7 +1022,7 @@ mx_gemm_skinny_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_c
   __syncthreads();
   tc_fence_after();
   const uint32_t tmem_base = *tmem_slot;
-  // A small product is launched with programmatic stream serialization: everything above then
+  // The kernel is launched with programmatic stream serialization: everything above then
   // overlapped the tail of the kernel before, and nothing below touches global memory before that
   // kernel has completed.  The kernel does not announce its own dependents early: CTAs of a
   // following kernel that wait on SMs this grid has already left slowed the rest of it down (a
@@ -1847,12 +1847,11 @@ bool make_out_map(EncodeTiledFn fn, CUtensorMap* map, const GemmArgs& a) {
   return make_c_map(fn, map, a.C, (uint64_t)(a.batch * a.M), (uint64_t)a.N, a.c_bf16 != 0);
 }
 
-// Products of a few microseconds are launched with programmatic stream serialization like the
-// streaming kernels (their set-up overlaps the tail of the kernel before them: 14.0 -> 12.5 us per
-// launch back to back); chains of large products measured 3 % slower with it, so those are not.
-bool small_product(const GemmArgs& a) {
-  return (double)a.batch * (double)a.M * (double)a.N * (double)a.K < 4.0e9;
-}
+// The GEMM kernels are launched with programmatic stream serialization like the streaming kernels:
+// their set-up (barriers, tensor-memory allocation, descriptor fetch) overlaps the tail of the kernel
+// before them -- 14.0 -> 12.5 us per launch for back-to-back 256 x 256 x 1024 products, 57.8 -> 56.1
+// us for 4096^3, nothing lost on the largest ones (when the kernels still announced their own
+// dependents early, chains of large products were 3 % slower with it; they no longer do).
 
 long long wait_budget(const GemmArgs& a) { return a.wait_cycles > 0 ? (long long)a.wait_cycles : kSpinLimit; }
 uint32_t drop_fill(const GemmArgs& a) { return a.drop_fill >= 0 ? (uint32_t)a.drop_fill : kNoDrop; }
@@ -1900,7 +1899,7 @@ cudaError_t launch_bn(const GemmArgs& a, const CUtensorMap& ma, const CUtensorMa
   const uint32_t tx_bytes =
       DENSE ? (uint32_t)(BM + BN) * 128u
             : (uint32_t)(BM * BK * fmt_bits(a.fmtA) / 8 + BN * BK * fmt_bits(a.fmtB) / 8);
-  return launch_pdl_if(small_product(a), mx_gemm_kernel<BN, DENSE>, dim3(grid), dim3(kThreads), cfg::kSmemBytes, a.stream,
+  return launch_pdl(mx_gemm_kernel<BN, DENSE>, dim3(grid), dim3(kThreads), cfg::kSmemBytes, a.stream,
                     ma, mb, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K,
                     idesc_base | ((uint32_t)(BN >> 3) << 17), group_m, tx_bytes, epi_args(a),
                     (uint32_t)a.batch, wait_budget(a), drop_fill(a));
@@ -1977,7 +1976,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   const uint32_t fa = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtA), fb = (F4 || DENSE) ? 1u : mma_fmt_code(a.fmtB);
   const uint32_t idesc = (fa << 7) | (fb << 10) | (DENSE ? (1u << 4) : (1u << 23)) |
                          ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-  return launch_pdl_if(small_product(a), mx_gemm_pair_kernel<KIND, BN>, dim3(2 * pairs), dim3(kThreads), cfg::kSmemBytes, a.stream,
+  return launch_pdl(mx_gemm_pair_kernel<KIND, BN>, dim3(2 * pairs), dim3(kThreads), cfg::kSmemBytes, a.stream,
                     ma, mb, mb2, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
                     epi_args(a), (uint32_t)a.batch, wait_budget(a), drop_fill(a));
 }
@@ -2025,7 +2024,7 @@ cudaError_t launch_skinny(const GemmArgs& a, EncodeTiledFn fn) {
   // the MMA's A side is B (format field [7,10)), its B side is A ([10,13)); N field = MP, M = 128
   const uint32_t idesc = (mma_fmt_code(a.fmtB) << 7) | (mma_fmt_code(a.fmtA) << 10) | (1u << 23) |
                          ((MP >> 3) << 17) | ((uint32_t)(128 >> 4) << 24);
-  return launch_pdl_if(small_product(a), mx_gemm_skinny_kernel, dim3(grid), dim3(kThreads), smem, a.stream, mw, mx_, msw, msx, a.C,
+  return launch_pdl(mx_gemm_skinny_kernel, dim3(grid), dim3(kThreads), smem, a.stream, mw, mx_, msw, msx, a.C,
                     (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, MP, idesc, tx_bytes, stages, kch, a.c_bf16 ? 1u : 0u,
                     wait_budget(a), drop_fill(a), tm);
 }
