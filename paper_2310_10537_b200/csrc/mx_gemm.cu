@@ -2180,7 +2180,7 @@ int launch_conv(const ConvArgs& a, cudaError_t* cuda_err) {
     const uint32_t tx_pair = 2u * (uint32_t)(128 * BK + 128 * BK * fmt_bits(a.fmt_w) / 8);
     const uint32_t idesc2 = (mma_fmt_code(a.fmt_x) << 7) | (mma_fmt_code(a.fmt_w) << 10) | (1u << 23) |
                             ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
-    *cuda_err = launch_pdl_if(false, mx_conv_pair_kernel, dim3(2 * np), dim3(kThreads), cfg2::kConvSmemBytes, a.stream, mx_, mb,
+    *cuda_err = launch_pdl(mx_conv_pair_kernel, dim3(2 * np), dim3(kThreads), cfg2::kConvSmemBytes, a.stream, mx_, mb,
                               msb2, mc, (uint32_t)M, (uint32_t)a.Cout, (uint32_t)K, idesc2, 8u, tx_pair, epi, kSpinLimit, g);
     return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
   }
@@ -2189,7 +2189,7 @@ int launch_conv(const ConvArgs& a, cudaError_t* cuda_err) {
   const uint32_t tx_bytes = (uint32_t)(BN * BK * fmt_bits(a.fmt_w) / 8) + (tma ? (uint32_t)(BM * BK) : 0u);
   const uint32_t idesc = (mma_fmt_code(a.fmt_x) << 7) | (mma_fmt_code(a.fmt_w) << 10) | (1u << 23) |
                          ((uint32_t)(BM >> 4) << 24) | ((uint32_t)(BN >> 3) << 17);
-  *cuda_err = launch_pdl_if(false, mx_conv_kernel, dim3(grid), dim3(kConvThreads), cfg::kSmemBytes, a.stream, mx_, mb, msb,
+  *cuda_err = launch_pdl(mx_conv_kernel, dim3(grid), dim3(kConvThreads), cfg::kSmemBytes, a.stream, mx_, mb, msb,
                             mc, (uint32_t)M, (uint32_t)a.Cout, (uint32_t)K, idesc, 16u, tx_bytes, epi, kSpinLimit, g);
   return *cuda_err == cudaSuccess ? MX_OK : MX_ERR_CUDA;
 }
