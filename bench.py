@@ -408,27 +408,36 @@ def run_extras(torch, mx, inputs, peaks, gpu_index):
     act, wt, rnd = mx.MX_E3M2, mx.MX_E2M3, mx.MX_RHAZ
     Y = torch.empty((n, n), dtype=torch.float32, device="cuda")
 
+    # every output buffer exists before the timed loops (no allocator calls inside them)
+    q = {k: mx.mx_quantize(t, ax, f, rnd) for k, (t, ax, f) in
+         {"xa": (Xc, 1, act), "wb": (Wc, 0, wt), "ga": (dY, 1, act), "wb2": (Wc, 1, wt), "xt": (Xc, 0, act),
+          "gt": (dY, 0, act)}.items()}
+
     def train_step():
-        xa = mx.mx_quantize(Xc, 1, act, rnd)
-        wb = mx.mx_quantize(Wc, 0, wt, rnd)
-        mx.mx_gemm(*xa, *wb, n, n, n, act, wt, out=Y)            # Y = X W
-        ga = mx.mx_quantize(dY, 1, act, rnd)
-        wb2 = mx.mx_quantize(Wc, 1, wt, rnd)
-        mx.mx_gemm(*ga, *wb2, n, n, n, act, wt, out=Y)           # dX = dY W^T
-        xt = mx.mx_quantize(Xc, 0, act, rnd)
-        gt = mx.mx_quantize(dY, 0, act, rnd)
-        mx.mx_gemm(*xt, *gt, n, n, n, act, act, out=Y)           # dW = X^T dY
+        mx.mx_quantize(Xc, 1, act, rnd, out=q["xa"])
+        mx.mx_quantize(Wc, 0, wt, rnd, out=q["wb"])
+        mx.mx_gemm(*q["xa"], *q["wb"], n, n, n, act, wt, out=Y)            # Y = X W
+        mx.mx_quantize(dY, 1, act, rnd, out=q["ga"])
+        mx.mx_quantize(Wc, 1, wt, rnd, out=q["wb2"])
+        mx.mx_gemm(*q["ga"], *q["wb2"], n, n, n, act, wt, out=Y)           # dX = dY W^T
+        mx.mx_quantize(Xc, 0, act, rnd, out=q["xt"])
+        mx.mx_quantize(dY, 0, act, rnd, out=q["gt"])
+        mx.mx_gemm(*q["xt"], *q["gt"], n, n, n, act, act, out=Y)           # dW = X^T dY
 
     def train_step_fused():  # each tensor is read once: both of its MX tensors come from one pass
-        (xa, xt) = mx.mx_quantize_dual(Xc, act, rnd)
-        (wb2, wb) = mx.mx_quantize_dual(Wc, wt, rnd)
-        (ga, gt) = mx.mx_quantize_dual(dY, act, rnd)
-        mx.mx_gemm(*xa, *wb, n, n, n, act, wt, out=Y)
-        mx.mx_gemm(*ga, *wb2, n, n, n, act, wt, out=Y)
-        mx.mx_gemm(*xt, *gt, n, n, n, act, act, out=Y)
+        mx.mx_quantize_dual(Xc, act, rnd, out=(q["xa"], q["xt"]))
+        mx.mx_quantize_dual(Wc, wt, rnd, out=(q["wb2"], q["wb"]))
+        mx.mx_quantize_dual(dY, act, rnd, out=(q["ga"], q["gt"]))
+        mx.mx_gemm(*q["xa"], *q["wb"], n, n, n, act, wt, out=Y)
+        mx.mx_gemm(*q["ga"], *q["wb2"], n, n, n, act, wt, out=Y)
+        mx.mx_gemm(*q["xt"], *q["gt"], n, n, n, act, act, out=Y)
 
-    ts = timed(train_step, 10)
-    tf = timed(train_step_fused, 10)
+    # the two variants in alternation (what ran before colours a GEMM-heavy timing), medians
+    ts_all, tf_all = [], []
+    for _ in range(5):
+        ts_all.append(timed(train_step, 6))
+        tf_all.append(timed(train_step_fused, 6))
+    ts, tf = sorted(ts_all)[2], sorted(tf_all)[2]
     out["config4_mxfp6_training_step"] = {
         "ms_six_quantizes_three_gemms": ts * 1e3, "ms_three_dual_quantizes_three_gemms": tf * 1e3,
         "gemm_flops_per_step": 3 * 2.0 * n ** 3}
