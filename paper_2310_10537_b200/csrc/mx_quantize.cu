@@ -324,7 +324,11 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
   constexpr int bits = FmtTraits<FMT>::bits;
   constexpr int kWords = StridedRow<DTYPE, COLS>::kWords;
   constexpr uint32_t kBpb = kBlock * bits / 8;                     // bytes of one block's codes
-  constexpr uint32_t kSeg = 4 * kBpb;                              // four blocks: 128 / 96 / 64
+  // blocks a CTA walks: four, but two for 4-bit codes -- their two-block run is already a whole
+  // sector, and a CTA that lives half as long halves the ragged end of the grid (a fifth of the
+  // launch at these sizes)
+  constexpr uint32_t NB = bits == 4 ? 2 : 4;
+  constexpr uint32_t kSeg = NB * kBpb;                             // the run of a row: 128 / 96 / 64 (32) bytes
   constexpr uint32_t kPitch = kSeg + (bits == 6 ? 8 : 16);         // conflict-free lane stride
   constexpr uint32_t kRows = 32 * COLS;                            // output rows per warp
   extern __shared__ __align__(16) uint8_t staging[];
@@ -343,12 +347,12 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
   const bool al32 = (reinterpret_cast<uintptr_t>(elems) & 31u) == 0 && out_row_bytes % 32 == 0;
 
   for (uint32_t o = blockIdx.z; o < outer; o += gridDim.z) {
-    const uint32_t kb0 = blockIdx.y * 4;
+    const uint32_t kb0 = blockIdx.y * NB;
     uint32_t scale_word[COLS];
 #pragma unroll
     for (int c = 0; c < COLS; ++c) scale_word[c] = 0;
 #pragma unroll 1
-    for (uint32_t j = 0; j < 4; ++j) {
+    for (uint32_t j = 0; j < NB; ++j) {
       const uint32_t kb = kb0 + j;
       uint32_t raw[kBlock][kWords];
       if (lane_ok) {
@@ -424,7 +428,9 @@ quantize_strided_staged_kernel(const void* __restrict__ in, uint8_t* __restrict_
 #pragma unroll
       for (int c = 0; c < COLS; ++c) {  // four scale bytes of a row are one aligned word in both layouts
         const uint32_t row = o * inner + col0 + c;
-        *reinterpret_cast<uint32_t*>(scales + scale_offset<LAYOUT>(row, kb0, kblocks)) = scale_word[c];
+        uint8_t* sp = scales + scale_offset<LAYOUT>(row, kb0, kblocks);
+        if (NB == 4) *reinterpret_cast<uint32_t*>(sp) = scale_word[c];
+        else *reinterpret_cast<uint16_t*>(sp) = (uint16_t)scale_word[c];  // kb0 even: two adjacent, aligned bytes
       }
     }
     __syncwarp();
@@ -528,11 +534,12 @@ static cudaError_t launch_strided(const QuantizeArgs& a) {
   const bool staged = bits != 8 && wide && kblocks % 4 == 0 && (a.L * bits / 8) % 16 == 0 && (uintptr_t)a.elems % 16 == 0 &&
                       (uintptr_t)a.scales % 4 == 0;
   if (staged) {
-    constexpr uint32_t kPitch = 4 * kBlock * bits / 8 + (bits == 6 ? 8 : 16);
+    constexpr uint32_t NB = bits == 4 ? 2 : 4;  // blocks per CTA, as in the kernel
+    constexpr uint32_t kPitch = NB * kBlock * bits / 8 + (bits == 6 ? 8 : 16);
     constexpr uint32_t smem = (kStagedThreads / 32) * 32 * kWide * kPitch;
     static_assert(smem <= 48 * 1024, "staging fits the default shared-memory limit");
     const uint32_t threads_x = (uint32_t)(a.inner / kWide);
-    dim3 grid((threads_x + kStagedThreads - 1) / kStagedThreads, kblocks / 4,
+    dim3 grid((threads_x + kStagedThreads - 1) / kStagedThreads, kblocks / NB,
               (uint32_t)(a.outer < 65535 ? a.outer : 65535));
     return launch_pdl(quantize_strided_staged_kernel<FMT, ROUND, DTYPE, LAYOUT, kWide>, grid,
                       dim3(kStagedThreads), smem, a.stream, a.in, a.elems, a.scales, (uint32_t)a.outer,
