@@ -26,9 +26,11 @@
 // The swizzle makes both access directions conflict-free: a row's 16-byte chunks are spread over
 // the banks by (chunk ^ row % 8), a word column's 32 lanes always hit 32 different banks.
 // The mbarrier wait is bounded: when it runs out the CTA records it in a status word and leaves.
-// Measured on 8192 x 8192 (both outputs, half-away rounding): E4M3 53 us against 59 us for the
-// register kernel, E3M2 62 against 67, E2M1 46 against 52; the conversion pipe (the packed narrow
-// casts, one per element and direction) is 72-77 % busy, DRAM 54 %.
+// Measured on 8192 x 8192 (both outputs): E4M3 53 us against 59 us for the register kernel, E3M2 47
+// against 67, E2M1 41 against 52.  Timing-only builds say what the time is made of: copies alone 22
+// us, both passes without their stores 33 us, one pass with its stores 35 us -- the two conversions
+// are ~5 instructions per element each and do not overlap the 42 us the bytes need well enough.
+// 8-bit codes have a kernel of their own below (no meeting of warps): 51 us.
 #include "mx_device.cuh"
 #include "mx_launch.h"
 #include "mx_quantize_common.cuh"
@@ -307,6 +309,193 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
   }
 }
 
+
+// ---------------------------------------------------------------------------------------------
+// 8-bit codes, both passes, no meeting of warps.  A block of 8-bit codes is a whole 32-byte sector
+// and its scale a byte of its own, so nothing has to be gathered across warps before it is
+// written: every warp converts its share of a tile straight out of the (read-only) stage and the
+// only synchronisation left is the stage's two barriers -- "tile landed" (the copy engine) and
+// "tile read" (one arrival per warp), which a producer warp waits on before it refills the stage.
+//   warps 0-7   row pass: lane (r, h) = (lane % 16, lane / 16) converts the two blocks of row
+//               16 w + r that lie in box h (one 128-byte box row: eight conflict-free 16-byte loads);
+//               column pass: warp w = (box b, row group g) = (w % 2, w / 2), lane = one 32-bit word
+//               column of box b (two columns), 32 rows down (32 conflict-free 4-byte loads)
+//   warp 8      producer: one lane issues the two box copies of a tile into a stage once its eight
+//               readers have released it
+// ---------------------------------------------------------------------------------------------
+// Tile of the 8-bit kernel: 128 rows x NBOX boxes of 64 columns side by side (NBOX x 128 contiguous
+// bytes of every row), 4 NBOX reader warps + the producer warp.
+constexpr uint32_t kT8Boxes = 4;  // (two boxes and two CTAs per SM measured 52.8 us against 51.3 on 8192 x 8192)
+constexpr uint32_t kT8Warps = 4 * kT8Boxes;
+constexpr int kTile8Threads = 32 * (kT8Warps + 1);
+constexpr uint32_t kT8TileBytes = kT8Boxes * kBoxBytes;
+constexpr uint32_t kT8Cols = 64 * kT8Boxes;
+constexpr int kT8CtasPerSm = kT8Boxes == 2 ? 2 : 1;
+
+template <int FMT, int ROUND, int LAYOUT>
+__global__ void __launch_bounds__(kTile8Threads, kT8CtasPerSm)
+quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
+                      uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
+                      uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
+                      uint32_t num_tiles) {
+  static_assert(FmtTraits<FMT>::bits == 8, "8-bit codes only");
+  constexpr int DTYPE = MX_BF16;
+  constexpr uint32_t kStages = 3;
+  constexpr uint32_t kBpb = 32;
+  extern __shared__ uint8_t tile_smem_raw[];
+  const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = base + kStages * kT8TileBytes;      // full[s] at 8 s, empty[s] at 8 (kStages + s)
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (uint32_t s = 0; s < kStages; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kT8Warps) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_in)) : "memory");
+  }
+  __syncthreads();
+  pdl_prologue();
+  const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;
+  const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
+
+  if (warp == kT8Warps) {
+    // ------------------------------- producer -------------------------------
+    uint32_t it = 0;
+    for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+      const uint32_t stage = it % kStages, use = it / kStages;
+      if (use > 0 && !tile_wait(bar0 + 8 * (kStages + stage), (use - 1) & 1u)) {  // its readers of the round before
+        if (lane == 0) atomicCAS(&g_tile_status, 0u, 2u);
+        return;
+      }
+      if (lane == 0) {
+        const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+        const uint32_t bar = bar0 + 8 * stage;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kT8TileBytes) : "memory");
+        const uint32_t dst = base + stage * kT8TileBytes;
+        for (uint32_t b = 0; b < kT8Boxes; ++b)
+          tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kT8Cols + 64u * b), (int)(tr * kTileRows), bar);
+      }
+      __syncwarp();
+    }
+    return;
+  }
+
+  // -------------------------------- readers --------------------------------
+  uint32_t it = 0;
+#pragma unroll 1
+  for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+    const uint32_t stage = it % kStages, parity = (it / kStages) & 1u;
+    if (!tile_wait(bar0 + 8 * stage, parity)) {
+      if (lane == 0) atomicCAS(&g_tile_status, 0u, 1u);
+      return;
+    }
+    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+    const uint32_t tile_base = base + stage * kT8TileBytes;
+    const uint32_t row0 = tr * kTileRows, col0 = tc * kT8Cols;
+    {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
+      constexpr uint32_t kRowsPerWarp = 32 / kT8Boxes;   // 16 or 8
+      const uint32_t r = warp * kRowsPerWarp + (lane % kRowsPerWarp), h = lane / kRowsPerWarp;
+      const uint32_t box = tile_base + h * kBoxBytes;
+      uint32_t codes[2][8];
+      uint32_t scale_pair = 0;
+#pragma unroll
+      for (uint32_t q = 0; q < 2; ++q) {
+        uint32_t u[16];
+#pragma unroll
+        for (uint32_t i = 0; i < 4; ++i) {
+          uint32_t v0, v1, v2, v3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(box_chunk(box, r, q * 4u + i)));
+          u[4 * i] = v0; u[4 * i + 1] = v1; u[4 * i + 2] = v2; u[4 * i + 3] = v3;
+        }
+        const BlockScale s = block_scale<FMT>(unit_amax<DTYPE>(u));
+        scale_pair |= s.byte << (8 * q);
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float x[8];
+          unit_group<DTYPE>(u, g, x);
+          cast8<FMT, ROUND>(x, s, codes[q][2 * g], codes[q][2 * g + 1]);
+        }
+      }
+      const uint32_t row = row0 + r, kb0 = tc * (kT8Cols / kBlock) + 2u * h;
+      uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
+      const uint32_t run[16] = {codes[0][0], codes[0][1], codes[0][2], codes[0][3], codes[0][4], codes[0][5],
+                                codes[0][6], codes[0][7], codes[1][0], codes[1][1], codes[1][2], codes[1][3],
+                                codes[1][4], codes[1][5], codes[1][6], codes[1][7]};
+      store_run<16>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      // two adjacent bytes in either layout (kb0 even, C % 128 == 0)
+      *reinterpret_cast<uint16_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = (uint16_t)scale_pair;
+    }
+    {  // column pass: one word column (two columns) of one box, one 32-row group
+      const uint32_t b = warp % kT8Boxes, g = warp / kT8Boxes;
+      const uint32_t box = tile_base + b * kBoxBytes;
+      const uint32_t c = lane >> 2, wofs = (lane & 3u) * 4u;
+      uint32_t raw[kBlock][1];
+#pragma unroll
+      for (uint32_t k = 0; k < kBlock; ++k)
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, g * kBlock + k, c) + wofs));
+      float amax[2];
+      column_amax<DTYPE, 2>(raw, amax);
+      const uint32_t kb = tr * 4u + g;
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const uint32_t col = col0 + b * 64u + lane * 2u + cc;
+        const BlockScale s = block_scale<FMT>(amax[cc]);
+        uint32_t cw[8];
+        column_cast<FMT, ROUND, DTYPE, 2>(raw, cc, s, cw);
+        uint8_t* dst = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
+        store_run<8>(dst, cw, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+        scales_col[scale_offset<LAYOUT>(col, kb, kb_col)] = (uint8_t)s.byte;
+      }
+    }
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8 * (kStages + stage)) : "memory");
+  }
+}
+
+template <int FMT, int ROUND, int LAYOUT>
+cudaError_t launch_tile8_t(const DualArgs& a) {
+  cudaError_t e;
+  EncodeTiledFn fn = encode_fn(&e);
+  if (!fn) return e;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.C, (cuuint64_t)a.R};
+  const cuuint64_t strides[1] = {(cuuint64_t)a.C * 2};
+  const cuuint32_t box[2] = {64, kTileRows};
+  if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+    return cudaErrorInvalidValue;
+  constexpr uint32_t smem = 3 * kT8TileBytes + 6 * 8 + 1024;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  auto kernel = quantize_tile8_kernel<FMT, ROUND, LAYOUT>;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint32_t tiles_r = (uint32_t)(a.R / kTileRows), tiles_c = (uint32_t)(a.C / kT8Cols);
+  const uint32_t num_tiles = tiles_r * tiles_c;
+  const uint32_t slots = (uint32_t)kT8CtasPerSm * (uint32_t)a.sm_count;
+  const uint32_t rounds = (num_tiles + slots - 1) / slots;
+  const uint32_t grid = (num_tiles + rounds - 1) / rounds;
+  return launch_pdl(kernel, dim3(grid), dim3(kTile8Threads), smem, a.stream, map, a.elems_row, a.scales_row,
+                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
+}
+
+template <int FMT>
+cudaError_t dispatch_tile8(const DualArgs& a) {
+  if (a.rounding == MX_RHAZ)
+    return a.layout == MX_SCALES_LINEAR ? launch_tile8_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
+                                        : launch_tile8_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile8_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
+                                      : launch_tile8_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
+}
+
 template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY>
 cudaError_t launch_tile_t(const DualArgs& a) {
   using cfg = TileCfg<FMT>;
@@ -358,13 +547,14 @@ cudaError_t dispatch_tile_round(const DualArgs& a) {
 // BF16 input, R and C multiples of 128 (what mx_quantize_dual requires of BF16 tensors).
 cudaError_t launch_quantize_tile(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
+  const bool wide8 = a.C % kT8Cols == 0;  // the 8-bit kernel's tiles; other widths take the general tile kernel
   switch (a.fmt) {
-    case MX_E4M3: return dispatch_tile_round<MX_E4M3, false>(a);
-    case MX_E5M2: return dispatch_tile_round<MX_E5M2, false>(a);
+    case MX_E4M3: return wide8 ? dispatch_tile8<MX_E4M3>(a) : dispatch_tile_round<MX_E4M3, false>(a);
+    case MX_E5M2: return wide8 ? dispatch_tile8<MX_E5M2>(a) : dispatch_tile_round<MX_E5M2, false>(a);
     case MX_E3M2: return dispatch_tile_round<MX_E3M2, false>(a);
     case MX_E2M3: return dispatch_tile_round<MX_E2M3, false>(a);
     case MX_E2M1: return dispatch_tile_round<MX_E2M1, false>(a);
-    default: return dispatch_tile_round<MX_INT8, false>(a);
+    default: return wide8 ? dispatch_tile8<MX_INT8>(a) : dispatch_tile_round<MX_INT8, false>(a);
   }
 }
 

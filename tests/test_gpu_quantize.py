@@ -149,13 +149,16 @@ def test_middle_axis_of_3d_tensor(fmt):
     _assert_same_bytes(s, ws, "scales")
 
 
-@pytest.mark.parametrize("dtype", DTYPES, ids=["f32", "bf16"])
+@pytest.mark.parametrize("dtype,R,C", [(torch.float32, 384, 320), (torch.bfloat16, 256, 384),
+                                       (torch.bfloat16, 384, 512), (torch.bfloat16, 128, 256),
+                                       (torch.bfloat16, 640, 1280)],
+                         ids=["f32", "bf16", "bf16-wide-tiles", "bf16-one-wide-tile", "bf16-many-wide-tiles"])
 @pytest.mark.parametrize("fmt", FMTS)
-def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype):
+def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype, R, C):
     """mx_quantize_dual reads the tensor once and must write exactly the two tensors that
     quantizing along axis 1 and along axis 0 give (checked against the oracle, not against
-    mx_quantize)."""
-    R, C = (384, 320) if dtype == torch.float32 else (256, 384)
+    mx_quantize).  BF16 tensors whose width is a multiple of 256 take the 8-bit formats through the
+    kernel with 128 x 256 tiles, the other widths and formats through the general tile kernel."""
     x = inputs.adversarial("cuda", rows=R, cols=C, dtype=dtype, seed=41 + fmt)
     xin = to_oracle_input(x)
     for rounding, layout in ((mx.MX_RNE, mx.MX_SCALES_SWIZZLED), (mx.MX_RHAZ, mx.MX_SCALES_LINEAR)):
@@ -174,6 +177,22 @@ def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype):
     with pytest.raises(mx.MxError) as ei:
         mx.mx_quantize_dual(torch.zeros((96, 128), dtype=dtype, device="cuda"), fmt)
     assert ei.value.status == mx.MX_ERR_UNSUPPORTED
+
+
+@pytest.mark.parametrize("fmt,rounding", [(mx.MX_E4M3, mx.MX_RHAZ), (mx.MX_INT8, mx.MX_RNE)])
+def test_dual_axis_8bit_at_sweep_size(fmt, rounding):
+    """The 8192 x 8192 BF16 sweep tensor through mx_quantize_dual with 8-bit codes (the size it is
+    timed at): 256 sampled rows of each of the two outputs byte for byte against the oracle, and both
+    whole tensors against the single-axis kernels."""
+    from gpu_util import assert_operand_rows_match_oracle
+    x = inputs.config2("cuda")
+    assert list(x.shape) == [8192, 8192] and x.dtype == torch.bfloat16
+    (er, sr), (ec, sc) = mx.mx_quantize_dual(x, fmt, rounding)
+    assert_operand_rows_match_oracle(O, x, 1, fmt, rounding, er, sr, "dual, row blocks", count=256, seed=1)
+    assert_operand_rows_match_oracle(O, x, 0, fmt, rounding, ec, sc, "dual, column blocks", count=256, seed=2)
+    e1, s1 = mx.mx_quantize(x, 1, fmt, rounding)
+    e0, s0 = mx.mx_quantize(x, 0, fmt, rounding)
+    assert torch.equal(er, e1) and torch.equal(sr, s1) and torch.equal(ec, e0) and torch.equal(sc, s0)
 
 
 def test_worked_blocks_on_device():
