@@ -35,10 +35,12 @@ template <int FMT, int DTYPE> struct DualCfg {
   static constexpr uint32_t kSmem = (kDualThreads / 32) * kWarpBytes;
 };
 
-// Resident CTAs per SM: BF16 tiles carry twice the elements per register and measured fastest with
-// the tile-ahead loads at four CTAs (255 registers); FP32 at six.
-template <int FMT, int ROUND, int DTYPE, int LAYOUT>
-__global__ void __launch_bounds__(kDualThreads, DTYPE == MX_BF16 ? 4 : 6)
+// Resident CTAs per SM (CTAS): BF16 tiles carry twice the elements per register and measured
+// fastest with the tile-ahead loads at four CTAs (255 registers); FP32 at six (about 150 registers),
+// except 8-bit codes on tensors of several waves, which gain 5 % at eight (128 registers; the staged
+// 6- and 4-bit variants lose a quarter there, and so does everything on a one-wave tensor).
+template <int FMT, int ROUND, int DTYPE, int LAYOUT, int CTAS>
+__global__ void __launch_bounds__(kDualThreads, CTAS)
 quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_row,
                      uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
                      uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_per_warp) {
@@ -219,8 +221,8 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
   }
 }
 
-template <int FMT, int ROUND, int DTYPE, int LAYOUT>
-static cudaError_t launch_dual_t(const DualArgs& a) {
+template <int FMT, int ROUND, int DTYPE, int LAYOUT, int CTAS>
+static cudaError_t launch_dual_ctas(const DualArgs& a) {
   using cfg = DualCfg<FMT, DTYPE>;
   static_assert(cfg::kSmem <= 48 * 1024, "fits the default shared-memory limit");
   const uint32_t strips = (uint32_t)(a.C / (32 * cfg::COLS));
@@ -230,7 +232,7 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
   // (two rounds) but 4.6 waves of one-tile warps (five rounds of a quarter the length).
   uint32_t T = 4;
   {
-    const uint64_t slots = (uint64_t)a.sm_count * (DTYPE == MX_BF16 ? 4 : 6);  // resident CTAs
+    const uint64_t slots = (uint64_t)a.sm_count * CTAS;  // resident CTAs
     uint64_t best = ~0ull;
     for (uint32_t t : {4u, 2u, 1u}) {
       if (t == 1 && cfg::bits != 8) continue;
@@ -242,9 +244,23 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
     }
   }
   dim3 grid(ctas_x, (uint32_t)(a.R / 32 / T));
-  return launch_pdl(quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT>, grid, dim3(kDualThreads), cfg::kSmem,
+  return launch_pdl(quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT, CTAS>, grid, dim3(kDualThreads), cfg::kSmem,
                     a.stream, a.in, a.elems_row, a.scales_row, a.elems_col, a.scales_col, (uint32_t)a.R,
                     (uint32_t)a.C, T);
+}
+
+template <int FMT, int ROUND, int DTYPE, int LAYOUT>
+static cudaError_t launch_dual_t(const DualArgs& a) {
+  if constexpr (DTYPE == MX_BF16) {
+    return launch_dual_ctas<FMT, ROUND, DTYPE, LAYOUT, 4>(a);
+  } else {
+    if constexpr (FmtTraits<FMT>::bits == 8) {
+      // four-tile warps of the whole tensor against the warps resident at eight CTAs per SM
+      const uint64_t warps = (uint64_t)(a.C / 64) * (uint64_t)(a.R / 128);
+      if (warps >= 3ull * 16ull * (uint64_t)a.sm_count) return launch_dual_ctas<FMT, ROUND, DTYPE, LAYOUT, 8>(a);
+    }
+    return launch_dual_ctas<FMT, ROUND, DTYPE, LAYOUT, 6>(a);
+  }
 }
 
 template <int FMT, int ROUND>

@@ -179,6 +179,40 @@ def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype, R, C):
     assert ei.value.status == mx.MX_ERR_UNSUPPORTED
 
 
+@pytest.mark.parametrize("fmt", FMTS)
+def test_dual_axis_bf16_subnormal_inputs_in_blocks_of_small_maxima(fmt):
+    """Algorithm 1 treats FP32-subnormal inputs as zero.  In a block whose maximum is itself tiny the
+    scaled value of a subnormal input would reach the element grid if it were not flushed, so the
+    kernels may scale BF16 pairs with a packed multiply (which keeps subnormals) only in blocks
+    where that cannot happen.  32 x 32 regions with maxima 2^-126 .. 2^-87 (every scale byte from 0
+    up past each format's limit), filled with subnormals of both signs, the smallest normals and
+    zeros: both outputs byte for byte against the oracle, both roundings."""
+    R, C = 256, 256
+    g = torch.Generator().manual_seed(7 + fmt)
+    bits = torch.randint(0, 0x80, (R, C), generator=g, dtype=torch.int32)          # BF16 subnormals and +0
+    bits[torch.rand((R, C), generator=g) < 0.2] = 0x0080                           # smallest normal
+    bits |= (torch.randint(0, 2, (R, C), generator=g, dtype=torch.int32) << 15)    # signs
+    for i in range(R // 32):
+        for j in range(C // 32):
+            e = 1 + (i * (C // 32) + j) % 40                                       # biased exponent of the maximum
+            r0, c0 = 32 * i, 32 * j
+            for d in range(32):                                                    # one per row and per column
+                bits[r0 + d, c0 + (5 * d + 3) % 32] = (e << 7) | int(torch.randint(0, 0x80, (1,), generator=g))
+    x = bits.to(torch.int16).view(torch.bfloat16).cuda()
+    xin = to_oracle_input(x)
+    for rounding in (mx.MX_RNE, mx.MX_RHAZ):
+        (er, sr), (ec, sc) = mx.mx_quantize_dual(x, fmt, rounding, mx.MX_SCALES_LINEAR)
+        wer, wsr = O.quantize(xin, 1, fmt, rounding, O.LINEAR)
+        wec, wsc = O.quantize(xin, 0, fmt, rounding, O.LINEAR)
+        _assert_same_bytes(er, wer, ("row elems", fmt, rounding))
+        _assert_same_bytes(sr, wsr, ("row scales", fmt, rounding))
+        _assert_same_bytes(ec, wec, ("col elems", fmt, rounding))
+        _assert_same_bytes(sc, wsc, ("col scales", fmt, rounding))
+        for axis, (ge, gs) in ((1, (er, sr)), (0, (ec, sc))):                      # and the single-axis kernels
+            e1, s1 = mx.mx_quantize(x, axis, fmt, rounding, mx.MX_SCALES_LINEAR)
+            assert torch.equal(e1, ge) and torch.equal(s1, gs)
+
+
 @pytest.mark.parametrize("fmt,rounding", [(mx.MX_E4M3, mx.MX_RHAZ), (mx.MX_INT8, mx.MX_RNE)])
 def test_dual_axis_8bit_at_sweep_size(fmt, rounding):
     """The 8192 x 8192 BF16 sweep tensor through mx_quantize_dual with 8-bit codes (the size it is
