@@ -553,6 +553,23 @@ def run_report(torch, mx, inputs):
     quantize_rows("C5 X BF16 16384x8192", d5["X"], 1, [0])
     quantize_rows("C5 W BF16 8192x28672", d5["W"], 0, [4])
 
+    def dual_rows(label, X, fmts, rounding=0):
+        # both MX tensors of X from one read: in + 2 x (codes + scales) bytes
+        n, esz = X.numel(), X.element_size()
+        Xs = [X, X.clone(), X.clone()]
+        for fmt in fmts:
+            outs = [mx.mx_quantize_dual(Xs[0], fmt, rounding) for _ in range(3)]
+            t = protocol(lambda i: mx.mx_quantize_dual(Xs[i], fmt, rounding, out=outs[i]), 3)
+            stream_row(f"quantize both axes {label} -> {FMT_NAMES[fmt]}",
+                       2 * algorithmic_bytes(n, esz, FMT_BITS[fmt]) - n * esz, t)
+            del outs
+        del Xs
+        torch.cuda.empty_cache()
+
+    dual_rows("C2 BF16 8192x8192", inputs.config2("cuda"), [0, 2, 4])
+    dual_rows("C4 X FP32 4096x4096 (half-away)", d4["X"], [2], 1)
+    dual_rows("C4 W FP32 4096x4096 (half-away)", d4["W"], [3], 1)
+
     # decode-shaped products: a few rows of activations against a weight matrix (the weights are read once);
     # measured before the tensor-bound loops, which leave the SM clock low for a while
     lines += ["", "## GEMM with few rows of A (HBM-bound on the weights)", "",

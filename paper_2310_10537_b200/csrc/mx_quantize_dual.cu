@@ -35,10 +35,13 @@ template <int FMT, int DTYPE> struct DualCfg {
   static constexpr uint32_t kSmem = (kDualThreads / 32) * kWarpBytes;
 };
 
-// Resident CTAs per SM (CTAS): BF16 tiles carry twice the elements per register and measured
-// fastest with the tile-ahead loads at four CTAs (255 registers); FP32 at six (about 150 registers),
-// except 8-bit codes on tensors of several waves, which gain 5 % at eight (128 registers; the staged
-// 6- and 4-bit variants lose a quarter there, and so does everything on a one-wave tensor).
+// Resident CTAs per SM (CTAS): six for FP32 input (about 150 registers), except 8-bit codes on
+// tensors of three waves or more, which gain 5 % at eight (128 registers).  The staged 6- and 4-bit
+// variants cannot follow: seven or eight of their CTAs need more than 196 KB of shared memory, which
+// leaves 28 KB of L1, and the loads in flight live there (69 -> 89 us on 8192 x 8192; the same
+// happens to every variant when the largest shared-memory carve-out is forced).  One-wave tensors
+// lose at eight too (4096 x 4096: 20.1 -> 21.6 us).  (The BF16 instances, four CTAs of 255
+// registers, are no longer built: the tile kernels replaced them.)
 template <int FMT, int ROUND, int DTYPE, int LAYOUT, int CTAS>
 __global__ void __launch_bounds__(kDualThreads, CTAS)
 quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_row,
@@ -79,7 +82,7 @@ quantize_dual_kernel(const void* __restrict__ in, uint8_t* __restrict__ elems_ro
     const char* p = reinterpret_cast<const char*>(in) + (size_t)tile * kBlock * in_pitch + (size_t)col0 * esz;
 #pragma unroll
     for (int k = 0; k < kBlock; ++k) {
-      const uint2 w = __ldg(reinterpret_cast<const uint2*>(p + (size_t)k * in_pitch));
+      const uint2 w = ld_cg8(p + (size_t)k * in_pitch);
       raw[k][0] = w.x; raw[k][1] = w.y;
     }
   };
@@ -244,7 +247,8 @@ static cudaError_t launch_dual_ctas(const DualArgs& a) {
     }
   }
   dim3 grid(ctas_x, (uint32_t)(a.R / 32 / T));
-  return launch_pdl(quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT, CTAS>, grid, dim3(kDualThreads), cfg::kSmem,
+  auto kernel = quantize_dual_kernel<FMT, ROUND, DTYPE, LAYOUT, CTAS>;
+  return launch_pdl(kernel, grid, dim3(kDualThreads), cfg::kSmem,
                     a.stream, a.in, a.elems_row, a.scales_row, a.elems_col, a.scales_col, (uint32_t)a.R,
                     (uint32_t)a.C, T);
 }
@@ -263,12 +267,11 @@ static cudaError_t launch_dual_t(const DualArgs& a) {
   }
 }
 
+// FP32 input only: BF16 tensors go through the tile kernels (mx_quantize_tile.cu), which replaced
+// this kernel's BF16 instances (255 registers, 8 warps per SM).
 template <int FMT, int ROUND>
 static cudaError_t dispatch_dual(const DualArgs& a) {
-  if (a.dtype == MX_BF16) {
-    return a.layout == MX_SCALES_LINEAR ? launch_dual_t<FMT, ROUND, MX_BF16, MX_SCALES_LINEAR>(a)
-                                        : launch_dual_t<FMT, ROUND, MX_BF16, MX_SCALES_SWIZZLED>(a);
-  }
+  if (a.dtype != MX_F32) return cudaErrorInvalidValue;
   return a.layout == MX_SCALES_LINEAR ? launch_dual_t<FMT, ROUND, MX_F32, MX_SCALES_LINEAR>(a)
                                       : launch_dual_t<FMT, ROUND, MX_F32, MX_SCALES_SWIZZLED>(a);
 }

@@ -316,15 +316,18 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
 // written: every warp converts its share of a tile straight out of the (read-only) stage and the
 // only synchronisation left is the stage's two barriers -- "tile landed" (the copy engine) and
 // "tile read" (one arrival per warp), which a producer warp waits on before it refills the stage.
-//   warps 0-7   row pass: lane (r, h) = (lane % 16, lane / 16) converts the two blocks of row
-//               16 w + r that lie in box h (one 128-byte box row: eight conflict-free 16-byte loads);
-//               column pass: warp w = (box b, row group g) = (w % 2, w / 2), lane = one 32-bit word
-//               column of box b (two columns), 32 rows down (32 conflict-free 4-byte loads)
-//   warp 8      producer: one lane issues the two box copies of a tile into a stage once its eight
-//               readers have released it
+//   warps 0-15  row pass: lane (r, h) = (lane % 8, lane / 8) converts the two blocks of row
+//               8 w + r that lie in box h (one 128-byte box row: eight 16-byte loads; a quarter-warp
+//               reads eight rows of one box, conflict-free under the 128-byte swizzle) and writes
+//               them as one 64-byte run plus two adjacent scale bytes;
+//               column pass: warp w = (box b, row group g) = (w % 4, w / 4), lane = one 32-bit word
+//               column of box b (two columns), 32 rows down (32 conflict-free 4-byte loads): two
+//               whole-sector stores and two scale bytes
+//   warp 16     producer: one lane issues the four box copies of a tile into a stage once its
+//               sixteen readers have released it
 // ---------------------------------------------------------------------------------------------
-// Tile of the 8-bit kernel: 128 rows x NBOX boxes of 64 columns side by side (NBOX x 128 contiguous
-// bytes of every row), 4 NBOX reader warps + the producer warp.
+// Tile of the 8-bit kernel: 128 rows x four boxes of 64 columns side by side (512 contiguous bytes
+// of every row), 16 reader warps + the producer warp, three stages of 64 KB.
 constexpr uint32_t kT8Boxes = 4;  // (two boxes and two CTAs per SM measured 52.8 us against 51.3 on 8192 x 8192)
 constexpr uint32_t kT8Warps = 4 * kT8Boxes;
 constexpr int kTile8Threads = 32 * (kT8Warps + 1);
