@@ -213,14 +213,20 @@ def test_dual_axis_bf16_subnormal_inputs_in_blocks_of_small_maxima(fmt):
             assert torch.equal(e1, ge) and torch.equal(s1, gs)
 
 
-@pytest.mark.parametrize("fmt,rounding", [(mx.MX_E4M3, mx.MX_RHAZ), (mx.MX_INT8, mx.MX_RNE)])
-def test_dual_axis_8bit_at_sweep_size(fmt, rounding):
-    """The 8192 x 8192 BF16 sweep tensor through mx_quantize_dual with 8-bit codes (the size it is
-    timed at): 256 sampled rows of each of the two outputs byte for byte against the oracle, and both
-    whole tensors against the single-axis kernels."""
+@pytest.mark.parametrize("fmt,rounding,dtype", [(mx.MX_E4M3, mx.MX_RHAZ, torch.bfloat16),
+                                                (mx.MX_INT8, mx.MX_RNE, torch.bfloat16),
+                                                (mx.MX_E5M2, mx.MX_RNE, torch.float32),
+                                                (mx.MX_E3M2, mx.MX_RHAZ, torch.float32)])
+def test_dual_axis_at_sweep_size(fmt, rounding, dtype):
+    """The 8192 x 8192 sweep tensor through mx_quantize_dual (the size it is timed at; BF16 with 8-bit
+    codes takes the kernel with 128 x 256 tiles, FP32 with 8-bit codes the register kernel in its
+    many-waves configuration, FP32 with 6-bit codes its staged form): 256 sampled rows of each of the
+    two outputs byte for byte against the oracle, and both whole tensors against the single-axis
+    kernels."""
     from gpu_util import assert_operand_rows_match_oracle
     x = inputs.config2("cuda")
     assert list(x.shape) == [8192, 8192] and x.dtype == torch.bfloat16
+    x = x.to(dtype)
     (er, sr), (ec, sc) = mx.mx_quantize_dual(x, fmt, rounding)
     assert_operand_rows_match_oracle(O, x, 1, fmt, rounding, er, sr, "dual, row blocks", count=256, seed=1)
     assert_operand_rows_match_oracle(O, x, 0, fmt, rounding, ec, sc, "dual, column blocks", count=256, seed=2)
