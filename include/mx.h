@@ -252,7 +252,9 @@ int mx_gemm_bf16(const void* A, const uint8_t* sA, const void* B, const uint8_t*
  * tests that must reach a particular kernel variant, and for the failure drill below; a NULL plan,
  * or a field left at its "library's choice" value, gives exactly mx_gemm.
  *   c_dtype         MX_F32 (C is float*) or MX_BF16.
- *   tile_n          0 = library's choice; 256 or 384 pins the tile width of the two-CTA kernel.
+ *   tile_n          0 = library's choice; 256 or 384 pins the tile width of the two-CTA kernel
+ *                   (with 0 a last, less than half full round of 256-wide tiles is computed in
+ *                   halves of 128 columns; results do not depend on it).
  *   few_rows_limit  -1 = library's choice (96); 0..128 = largest M that takes the kernel that puts
  *                   B on the M side of the MMA (0 sends every product through the tiled kernels).
  *   wait_cycles     0 = library's choice (about one second); otherwise the budget, in SM clock

@@ -1329,13 +1329,29 @@ __device__ __forceinline__ void cluster_sync() {
 // CONV: the implicit-GEMM convolution of mx_conv_kernel on the 256 x 256 pair tile (C % 128 == 0, so
 // the codes of each CTA's 128 output pixels come through the im2col-mode map `tmap_a`); each CTA's
 // scale-producer warp also composes the scale words of its 128 rows (four rows per lane).
+// Work items of the pair kernel.  Tiles [0, split_from) are computed whole, pair p taking items p,
+// p + P, ...; every tile from split_from on -- the last, less than half full round of the grid -- is
+// dealt out as two items of 128 columns each (h = 1: columns 0..127 of the tile, h = 2: columns
+// 128..255), so that twice as many pairs share that round and it takes about half a tile's time.
+// A half item loads 64 rows of B per CTA (the second B map), issues MMAs with N = 128 into
+// accumulator columns 0..127 and reads the B scales of its own 128-row group; the element order of
+// every dot product is unchanged, so results do not depend on the split.
+struct PairItem {
+  uint32_t tile, h;
+};
+__device__ __forceinline__ PairItem pair_item(uint32_t i, uint32_t split_from) {
+  if (i < split_from) return {i, 0u};
+  const uint32_t j = i - split_from;
+  return {split_from + (j >> 1), 1u + (j & 1u)};
+}
+
 template <int KIND, int BN_, bool CONV>
 __device__ __forceinline__ void
 pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUtensorMap& tmap_b2,
                  const CUtensorMap& tmap_sa, const CUtensorMap& tmap_sb, const CUtensorMap& tmap_c,
                  uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base, uint32_t group_m,
                  uint32_t tx_bytes_pair, EpiArgs epi, uint32_t batch, long long spin_limit,
-                 uint32_t drop_fill, const ConvGeom& cg) {
+                 uint32_t drop_fill, const ConvGeom& cg, uint32_t split_from, uint32_t tx_bytes_half) {
   static_assert(!CONV || (KIND == 0 && BN_ == 256), "convolution runs on the block-scaled 256 x 256 tile");
   using cfg = Cfg2<KIND, BN_>;
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE;
@@ -1373,7 +1389,9 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
   asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(rank));
   const uint32_t warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const uint32_t pair = blockIdx.x >> 1, num_pairs = gridDim.x >> 1;
-  const uint32_t tiles_m = (M + 255) / 256, tiles_n = (N + BN - 1) / BN, num_tiles = batch * tiles_m * tiles_n;
+  const uint32_t tiles_m = (M + 255) / 256, tiles_n = (N + BN - 1) / BN;
+  // items, not tiles, are what the roles below walk (see pair_item); without a split the two are the same
+  const uint32_t num_tiles = split_from + 2u * (batch * tiles_m * tiles_n - split_from);
   const uint32_t k_chunks = (K + BKe - 1) / BKe;  // a K tail is zero-filled by the copies
 
   if (threadIdx.x == 0) {
@@ -1421,13 +1439,15 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
     uint32_t stage = 0, phase = 0, fill = 0;
     bool ok = true;
     for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-      const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+      const PairItem it = pair_item(t, split_from);
+      const TileCoord tc = tile_coord(it.tile, tiles_m, tiles_n, group_m);
       // this CTA's 128 rows of A and its rows of B: rows 128 rank .. of the tile and, for the wide
       // tile, rows 256 + 64 rank .. (B rows may lie past N on a ragged tile: zero fill or the next
-      // matrix of a batch; their columns are not stored)
+      // matrix of a batch; their columns are not stored); a half item: rows 128 (h - 1) + 64 rank ..
       const int cy_a = (int)((tc.b * tiles_m + tc.tm) * 256 + rank * 128);
       const int cy_b = (int)(tc.b * N + tc.tn * BN + rank * 128);
-      const int cy_b2 = (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
+      const int cy_b2 = it.h ? (int)(tc.b * N + tc.tn * BN + (it.h - 1u) * 128u + rank * 64)
+                             : (int)(tc.b * N + tc.tn * BN + 256 + rank * 64);
       // CONV: where tap (0, 0) of the first of this CTA's 128 output pixels reads
       int cv_w = 0, cv_h = 0, cv_n = 0;
       if (CONV) {
@@ -1445,7 +1465,7 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
         }
         if (fill++ != drop_fill && elect_one()) {
           const uint32_t fb = leader_bar(full_bar(stage));
-          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), tx_bytes_pair);
+          if (rank == 0) mbar_arrive_expect_tx(full_bar(stage), it.h ? tx_bytes_half : tx_bytes_pair);
           const int cx = (int)(kc * BKe);
           if (CONV) {  // the stage's K chunk = 128 channels of one filter tap
             const uint32_t tap = fastdiv(kc * 4, cg.d_cb), cblk = kc * 4 - tap * cg.cb;
@@ -1455,7 +1475,10 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
           } else {
             tma_load_3d_pair(smem_base + cfg::kOffA + stage * cfg::kABytes, &tmap_a, cx, cy_a, 0, fb);
           }
-          tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, cx, cy_b, 0, fb);
+          if (it.h)  // 64 rows of B at the start of the stage's B area
+            tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b2, cx, cy_b2, 0, fb);
+          else
+            tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes, &tmap_b, cx, cy_b, 0, fb);
           if (WIDE)
             tma_load_3d_pair(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u, &tmap_b2, cx, cy_b2, 0, fb);
         }
@@ -1474,6 +1497,7 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
       uint32_t stage = 0, phase = 0, acc_phase = 0;
       bool ok = true;
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
+        const uint32_t hsel = pair_item(t, split_from).h;
         if (!__all_sync(0xffffffffu, mbar_wait(acc_empty_bar, acc_phase ^ 1u, abort_flag, 4 * spin_limit))) {
           raise_abort(abort_flag, ST_MMA_WAIT_ACC);
           break;
@@ -1496,26 +1520,29 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
           const uint64_t bdesc2 = operand_desc(smem_base + cfg::kOffB + stage * cfg::kBBytes + 128u * 128u);
           const uint32_t idesc2_base = (idesc_base & ~(0x3Fu << 17)) | ((uint32_t)(128 >> 3) << 17);
           constexpr uint32_t kSfbStep = 4 * cfg::kSfbGroups;  // B scale columns per K chunk
+          // a half item: N = 128, the B scales of its own 128-row group (4 columns further for h = 2)
+          const uint32_t idesc1 = hsel ? idesc2_base : idesc_base;
+          const uint32_t sfb_h = hsel ? 4u * (hsel - 1u) : 0u;
           if (elect_one()) {
 #pragma unroll
           for (uint32_t k = 0; k < 4; ++k) {  // every MMA advances 32 bytes along the 128-byte rows
             const uint32_t acc_flag = (kc | k) != 0 ? 1u : 0u;
             if (DENSE) {
-              tc_mma_pair_dense(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base, acc_flag);
+              tc_mma_pair_dense(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc1, acc_flag);
               if (WIDE) tc_mma_pair_dense(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base, acc_flag);
             } else if (F4) {
               // K = 64: blocks 2k and 2k+1 of the stage = bytes (2k % 4, +1) of K chunk k / 2
               const uint32_t sf_id = 2 * (k & 1);
               const uint32_t sel = (sf_id << 4) | (sf_id << 29);
-              const uint32_t sfa = sf_tmem + 4 * (k >> 1), sfb = sf_tmem + cfg::kSfColsA + kSfbStep * (k >> 1);
-              tc_mma_pair_f4(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base | sel, sfa, sfb, acc_flag);
+              const uint32_t sfa = sf_tmem + 4 * (k >> 1), sfb = sf_tmem + cfg::kSfColsA + kSfbStep * (k >> 1) + sfb_h;
+              tc_mma_pair_f4(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc1 | sel, sfa, sfb, acc_flag);
               if (WIDE)
                 tc_mma_pair_f4(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base | sel, sfa, sfb + 8,
                                acc_flag);
             } else {
               const uint32_t sel = (k << 4) | (k << 29);  // byte k of the scale columns
-              const uint32_t sfb = sf_tmem + cfg::kSfColsA;
-              tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc_base | sel, sf_tmem, sfb, acc_flag);
+              const uint32_t sfb = sf_tmem + cfg::kSfColsA + sfb_h;
+              tc_mma_pair(tmem_base, adesc + 2 * k, bdesc + 2 * k, idesc1 | sel, sf_tmem, sfb, acc_flag);
               if (WIDE)
                 tc_mma_pair(tmem_base + 256, adesc + 2 * k, bdesc2 + 2 * k, idesc2_base | sel, sf_tmem, sfb + 8,
                             acc_flag);
@@ -1652,7 +1679,8 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
         for (uint32_t i = 0; i < (uint32_t)cfg::kStages; ++i) conv_gather();  // the first round's chunks at once
       }
       for (uint32_t t = pair; t < num_tiles && ok; t += num_pairs) {
-        const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+        // (a half item fetches the B scales of both 128-row groups of its tile; its MMAs read one)
+        const TileCoord tc = tile_coord(pair_item(t, split_from).tile, tiles_m, tiles_n, group_m);
         const int cz_a = (int)((tc.b * tiles_m + tc.tm) * 2 + rank);
         const int cz_b = (int)(tc.b * (N / 128) + tc.tn * cfg::kSfbGroups);
         for (uint32_t kc = 0; kc < k_chunks; ++kc) {
@@ -1688,7 +1716,8 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
     constexpr uint32_t kHalf = BN / 2, kLoads = kHalf / 32;
     uint32_t acc_phase = 0;
     for (uint32_t t = pair; t < num_tiles; t += num_pairs) {
-      const TileCoord tc = tile_coord(t, tiles_m, tiles_n, group_m);
+      const PairItem it = pair_item(t, split_from);
+      const TileCoord tc = tile_coord(it.tile, tiles_m, tiles_n, group_m);
       if (!mbar_wait(acc_full_bar, acc_phase, abort_flag, 4 * spin_limit)) {
         if (lane == 0) raise_abort(abort_flag, ST_EPILOGUE_WAIT);
         break;
@@ -1720,9 +1749,11 @@ pair_kernel_body(const CUtensorMap& tmap_a, const CUtensorMap& tmap_b, const CUt
         }
       } else {
         const uint32_t taddr = tmem_base + ((quarter * 32u) << 16) + half * kHalf;
-        const uint32_t col0 = tc.tn * BN + half * kHalf;
+        // a half item: its 128 columns are accumulator columns 0..127, read out by the first four
+        // warps; the other four only hand the accumulator back
+        const uint32_t col0 = it.h ? tc.tn * BN + (it.h - 1u) * 128u : tc.tn * BN + half * kHalf;
         // nothing to store for a warp whose rows or columns lie past the matrix
-        const uint32_t valid_cols = (col0 < N && row0 < batch * M) ? min(kHalf, N - col0) : 0u;
+        const uint32_t valid_cols = (col0 < N && row0 < batch * M && !(it.h && half)) ? min(kHalf, N - col0) : 0u;
         uint32_t r[kLoads][32];
 #pragma unroll
         for (uint32_t j = 0; j < kLoads; ++j) tc_ld32(taddr + 32 * j, r[j]);
@@ -1760,10 +1791,11 @@ mx_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_a, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_sa, const __grid_constant__ CUtensorMap tmap_sb,
                     const __grid_constant__ CUtensorMap tmap_c, uint32_t M, uint32_t N, uint32_t K,
                     uint32_t idesc_base, uint32_t group_m, uint32_t tx_bytes_pair, EpiArgs epi,
-                    uint32_t batch, long long spin_limit, uint32_t drop_fill) {
+                    uint32_t batch, long long spin_limit, uint32_t drop_fill, uint32_t split_from,
+                    uint32_t tx_bytes_half) {
   const ConvGeom none = {};
   pair_kernel_body<KIND, BN_, false>(tmap_a, tmap_b, tmap_b2, tmap_sa, tmap_sb, tmap_c, M, N, K, idesc_base, group_m,
-                                     tx_bytes_pair, epi, batch, spin_limit, drop_fill, none);
+                                     tx_bytes_pair, epi, batch, spin_limit, drop_fill, none, split_from, tx_bytes_half);
 }
 
 static_assert(Cfg2<0, 256>::kConvSmemBytes <= 232448, "shared memory budget of the convolution kernel");
@@ -1773,8 +1805,9 @@ mx_conv_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const __grid_constant__ CUtensorMap tmap_sb, const __grid_constant__ CUtensorMap tmap_c,
                     uint32_t M, uint32_t N, uint32_t K, uint32_t idesc_base, uint32_t group_m,
                     uint32_t tx_bytes_pair, EpiArgs epi, long long spin_limit, const __grid_constant__ ConvGeom cg) {
+  // (no split of the last round: every tile whole)
   pair_kernel_body<0, 256, true>(tmap_x, tmap_b, tmap_b, tmap_sb, tmap_sb, tmap_c, M, N, K, idesc_base, group_m,
-                                 tx_bytes_pair, epi, 1u, spin_limit, kNoDrop, cg);
+                                 tx_bytes_pair, epi, 1u, spin_limit, kNoDrop, cg, ((M + 255) / 256) * ((N + 255) / 256), 0u);
 }
 
 // ---- host side ---------------------------------------------------------------
@@ -1932,7 +1965,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
   using cfg = Cfg2<KIND, BN>;
   constexpr bool F4 = cfg::F4, DENSE = cfg::DENSE, WIDE = BN == 384;
   // rows of B a CTA takes with its second copy (wide tile): 64; the map is unused otherwise
-  constexpr uint32_t kB2Rows = WIDE ? 64 : 128;
+  constexpr uint32_t kB2Rows = 64;  // (also what a CTA loads for a half item, see pair_item)
   const uint64_t rows_a = (uint64_t)(a.batch * a.M), rows_b = (uint64_t)(a.batch * a.N), K = (uint64_t)a.K;
   CUtensorMap ma, mb, mb2, msa, msb, mc;
   bool ok = make_out_map(fn, &mc, a);
@@ -1964,12 +1997,25 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
   const uint32_t tiles = (uint32_t)a.batch * (uint32_t)((a.M + 255) / 256) * (uint32_t)((a.N + BN - 1) / BN);
-  const uint32_t pairs = tiles < (uint32_t)a.sm_count / 2 ? tiles : (uint32_t)a.sm_count / 2;
+  // A last round that would occupy at most half of the pairs is dealt out in halves of 128 columns
+  // (4096^3: 256 tiles on 74 pairs = three rounds + 34 tiles -> 68 half items: 57.3 -> 55.0 us; a half
+  // item takes about 0.75 of a tile's time, not 0.5: 24 KB of operands per 256 cycles of MMAs is
+  // what an SM can pull).  Not with less than one whole round: 4 to 32 tiles measured 3-4 % slower
+  // in halves.
+  const uint32_t max_pairs = (uint32_t)a.sm_count / 2;
+  const uint32_t rest = tiles % max_pairs;
+  const bool split = !WIDE && a.force_bn == 0 && tiles > max_pairs && rest != 0 && 2 * rest <= max_pairs;  // a pinned width: whole tiles
+  const uint32_t split_from = split ? tiles - rest : tiles;
+  const uint32_t items = split_from + 2 * (tiles - split_from);
+  const uint32_t pairs = items < max_pairs ? items : max_pairs;
   // bytes both CTAs report to the leader's stage barrier (operand copies count packed bytes)
   const uint32_t rows_per_cta = 128u + cfg::kBRows;
   const uint32_t op_bytes = (F4 || DENSE) ? rows_per_cta * 128u
                                : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + cfg::kBRows * BK * fmt_bits(a.fmtB) / 8);
   const uint32_t tx_pair = 2u * op_bytes;  // the scale chunks complete on a barrier of their own
+  const uint32_t op_bytes_half = (F4 || DENSE) ? (128u + 64u) * 128u
+                                    : (uint32_t)(128 * BK * fmt_bits(a.fmtA) / 8 + 64 * BK * fmt_bits(a.fmtB) / 8);
+  const uint32_t tx_half = 2u * op_bytes_half;
   // formats: kind::mxf4 encodes E2M1 as 1; kind::mxf8f6f4 uses the codes of mma_fmt_code();
   // kind::f16: BF16 = 1 for both operands, FP32 accumulator = 1 in bits [4,6), no scale-format bit.
   // N field = 256: the first (or only) MMA of a K step; the kernel derives the N = 128 one.
@@ -1978,7 +2024,7 @@ cudaError_t launch_pair(const GemmArgs& a, EncodeTiledFn fn) {
                          ((uint32_t)(256 >> 3) << 17) | ((uint32_t)(256 >> 4) << 24);
   return launch_pdl(mx_gemm_pair_kernel<KIND, BN>, dim3(2 * pairs), dim3(kThreads), cfg::kSmemBytes, a.stream,
                     ma, mb, mb2, msa, msb, mc, (uint32_t)a.M, (uint32_t)a.N, (uint32_t)a.K, idesc, 8u, tx_pair,
-                    epi_args(a), (uint32_t)a.batch, wait_budget(a), drop_fill(a));
+                    epi_args(a), (uint32_t)a.batch, wait_budget(a), drop_fill(a), split_from, tx_half);
 }
 
 // M <= 128: operands swapped (see mx_gemm_skinny_kernel).
@@ -2054,7 +2100,11 @@ int launch_gemm(const GemmArgs& a, cudaError_t* cuda_err) {
   const int64_t tiles_pair = a.batch * ((a.M + 255) / 256) * ((a.N + 255) / 256);
   const int64_t tiles_one = a.batch * ((a.M + BM - 1) / BM) * ((a.N + bn - 1) / bn);
   const int64_t pairs = a.sm_count / 2;
-  const double cost_pair = (double)((tiles_pair + pairs - 1) / pairs);
+  // (a last round of at most half the pairs runs as half-width items, see launch_pair: about 0.75)
+  const int64_t rest_pair = tiles_pair % pairs;
+  const double cost_pair = (a.force_bn == 0 && tiles_pair > pairs && rest_pair != 0 && 2 * rest_pair <= pairs)
+                               ? (double)(tiles_pair / pairs) + 0.75
+                               : (double)((tiles_pair + pairs - 1) / pairs);
   const double cost_one = (double)((tiles_one + a.sm_count - 1) / a.sm_count) * (bn == 256 ? 1.05 : 0.82);
   const bool pair_ok = a.M % 256 == 0 || (a.batch == 1 && a.q_elems == nullptr);
   if (pair_ok && a.M >= 256 && cost_pair < cost_one) {

@@ -702,6 +702,46 @@ def test_config5_full_size():
     _full_size_check("config 5", ea, sa, eb, sb, M, N, K, mx.MX_E4M3, mx.MX_E2M1, 5)
 
 
+@pytest.mark.parametrize("M,N,K,fa,fb,dt", [
+    (4096, 4096, 256, 0, 0, torch.float32),     # 256 tiles on 74 pairs: three whole rounds + 34 tiles in halves
+    (2560, 2048, 384, 2, 3, torch.float32),     # 80 tiles: one round + 6 in halves
+    (2560, 1984, 512, 4, 4, torch.bfloat16),    # kind::mxf4; the last right halves hold 64 columns
+    (2400, 1900, 256, 0, 4, torch.float32),     # ragged in M and N; the last right halves lie past N
+    (2304, 4096, 128, 1, 0, torch.bfloat16),    # 144 tiles: one whole round + 70 (more than half the pairs: no halving)
+])
+def test_last_round_in_halves_equals_whole_tiles(M, N, K, fa, fb, dt):
+    """A last round of the two-CTA kernel that would occupy at most half of the CTA pairs is computed
+    as items of 128 columns (the library's choice, tile_n = 0).  Whole matrix against the FP64
+    product of the oracle-dequantized operands and samples against the oracle, and bit-identical to
+    the product computed in whole 256-wide tiles (tile_n = 256)."""
+    g = torch.Generator(device="cuda").manual_seed(M + N + K)
+    A = torch.randn((M, K), generator=g, device="cuda") * torch.exp(torch.randn((M, 1), generator=g, device="cuda"))
+    B = torch.randn((N, K), generator=g, device="cuda") * 0.02
+    ea, sa = mx.mx_quantize(A, 1, fa)
+    eb, sb = mx.mx_quantize(B, 1, fb)
+    esz = 2 if dt == torch.bfloat16 else 4
+    g_out = Guarded(M * N * esz)
+    C = g_out.view.view(dt).view(M, N)
+    mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, out=C, few_rows_limit=0, check_status=True)
+    torch.cuda.synchronize()
+    g_out.check()
+    hea, hsa, heb, hsb = (t.cpu().numpy().reshape(-1) for t in (ea, sa, eb, sb))
+    da = torch.from_numpy(O.dequantize(hea, hsa, M, K, fa, O.F64)).cuda()
+    db = torch.from_numpy(O.dequantize(heb, hsb, N, K, fb, O.F64)).cuda()
+    ref = da @ db.T
+    fac, rel = _bound_terms(dt)
+    bad = int(((C.double() - ref).abs() > fac * TOL * (da.abs() @ db.abs().T) + ref.abs() * rel).sum())
+    assert bad == 0, f"{bad} outputs beyond the bound"
+    rng = np.random.default_rng(K)
+    ms = np.concatenate([rng.integers(0, M, 600), np.full(100, M - 1)])
+    ns = np.concatenate([rng.integers(0, N, 600), rng.integers(max(0, N - 40), N, 100)])
+    c64, s_ = O.gemm_samples(hea, hsa, heb, hsb, M, N, K, fa, fb, ms, ns)
+    got = C[torch.from_numpy(ms).cuda(), torch.from_numpy(ns).cuda()].double().cpu().numpy()
+    assert (np.abs(got - c64) <= fac * TOL * s_ + np.abs(c64) * rel).all()
+    C1 = mx.mx_gemm_ex(ea, sa, eb, sb, M, N, K, fa, fb, out_dtype=dt, tile_n=256, few_rows_limit=0, check_status=True)
+    assert torch.equal(C1, C)
+
+
 @pytest.mark.parametrize("fa,fb,K,dt", [(0, 0, 640, torch.float32), (4, 4, 512, torch.float32), (2, 0, 384, torch.bfloat16)])
 def test_wide_tile_variant_whole_matrix(fa, fb, K, dt):
     """The 256 x 384 tile of the two-CTA kernel (mx_gemm_ex, tile_n = 384) on a shape with a ragged
