@@ -503,13 +503,16 @@ def run_report(torch, mx, inputs):
             b.record()
         torch.cuda.synchronize()
         each = sorted(a.elapsed_time(b) * 1e-3 for a, b in ev)
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        for i in range(reps):
-            fn_of_i(i % n_sets)
-        b.record()
-        torch.cuda.synchronize()
-        return each[len(each) // 2], each[0], a.elapsed_time(b) * 1e-3 / reps
+        runs = []
+        for _ in range(2):  # the faster of two back-to-back runs (the first one after a change of kernel can catch the clocks mid-ramp)
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record()
+            for i in range(reps):
+                fn_of_i(i % n_sets)
+            b.record()
+            torch.cuda.synchronize()
+            runs.append(a.elapsed_time(b) * 1e-3 / reps)
+        return each[len(each) // 2], each[0], min(runs)
 
     def stream_row(name, byts, times):
         med, best, b2b = times
@@ -519,8 +522,8 @@ def run_report(torch, mx, inputs):
     lines += ["## Quantize / dequantize (HBM-bound)", "",
               f"Peaks: measured copy {hbm:.1f} GB/s, nominal {hbm_nom:.0f} GB/s (80 % of nominal = 6400 GB/s = "
               f"{100 * 6400 / hbm:.1f} % of the measured copy peak).  Times in µs: median and best of 50 launches "
-              "timed one by one, and the mean of the same 50 launches back to back (what a stream of "
-              "conversions sees; the launches overlap their neighbours' tails).", "",
+              "timed one by one, and the mean of the same 50 launches back to back, the faster of two such runs "
+              "(what a stream of conversions sees; the launches overlap their neighbours' tails).", "",
               "| kernel, config | MB | median | best | back-to-back | GB/s | % measured | % nominal |",
               "|---|---|---|---|---|---|---|---|"]
 
