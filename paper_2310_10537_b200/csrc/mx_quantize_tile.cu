@@ -31,6 +31,8 @@
 // us, both passes without their stores 33 us, one pass with its stores 35 us -- the two conversions
 // are ~5 instructions per element each and do not overlap the 42 us the bytes need well enough.
 // 8-bit codes have a kernel of their own below (no meeting of warps): 51 us.
+#include <atomic>
+
 #include "mx_device.cuh"
 #include "mx_launch.h"
 #include "mx_quantize_common.cuh"
@@ -47,6 +49,18 @@ constexpr uint32_t kTileBytes = 2 * kBoxBytes;    // a tile: two boxes side by s
 constexpr long long kTileSpinLimit = 2000000000LL;
 
 __device__ unsigned int g_tile_status;  // 1: a tile never arrived (bounded wait ran out)
+
+// Tile counters of the kernels that deal their tiles out at run time: a launch takes one slot of
+// two words -- [0] tiles handed out beyond every CTA's first, [1] CTAs that have finished -- and
+// leaves both at zero: the CTA that finishes last resets the slot (no CTA asks for a tile after it
+// has been told that there are none left, and it is counted as finished only after that).  The host
+// cycles through the slots, so that launches in flight on different streams do not share one.
+constexpr uint32_t kSchedSlots = 256;
+__device__ unsigned int g_tile_sched[2 * kSchedSlots];
+inline uint32_t next_sched_slot() {
+  static std::atomic<uint32_t> next{0};
+  return next.fetch_add(1, std::memory_order_relaxed) % kSchedSlots;
+}
 
 template <int FMT> struct TileCfg {
   static constexpr int bits = FmtTraits<FMT>::bits;
@@ -340,7 +354,7 @@ __global__ void __launch_bounds__(kTile8Threads, kT8CtasPerSm)
 quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
                       uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
                       uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
-                      uint32_t num_tiles) {
+                      uint32_t num_tiles, uint32_t sched_slot) {
   static_assert(FmtTraits<FMT>::bits == 8, "8-bit codes only");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
@@ -348,6 +362,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
   extern __shared__ uint8_t tile_smem_raw[];
   const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
   const uint32_t bar0 = base + kStages * kT8TileBytes;      // full[s] at 8 s, empty[s] at 8 (kStages + s)
+  const uint32_t tile_id0 = bar0 + 16 * kStages;            // the tile a stage holds (written by the producer)
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (uint32_t s = 0; s < kStages; ++s) {
@@ -365,35 +380,58 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
 
   if (warp == kT8Warps) {
     // ------------------------------- producer -------------------------------
-    uint32_t it = 0;
-    for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+    // Tiles are dealt out at run time: an SM's share of the memory system's bandwidth varies (the
+    // slowest of 147 CTAs with 14 tiles each took 95 k cycles, the median 79 k), so a CTA's first
+    // tile is its own index and every further one comes from a counter.  The tile a stage holds is
+    // written beside the barriers before the stage is armed; a number past the last tile tells the
+    // readers to stop.
+    unsigned int* sched = g_tile_sched + 2 * sched_slot;
+    for (uint32_t it = 0;; ++it) {
       const uint32_t stage = it % kStages, use = it / kStages;
       if (use > 0 && !tile_wait(bar0 + 8 * (kStages + stage), (use - 1) & 1u)) {  // its readers of the round before
         if (lane == 0) atomicCAS(&g_tile_status, 0u, 2u);
-        return;
+        break;
+      }
+      uint32_t t = blockIdx.x;
+      if (it > 0) {
+        if (lane == 0) t = gridDim.x + atomicAdd(&sched[0], 1u);
+        t = __shfl_sync(0xFFFFFFFFu, t, 0);
       }
       if (lane == 0) {
-        const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
         const uint32_t bar = bar0 + 8 * stage;
-        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kT8TileBytes) : "memory");
-        const uint32_t dst = base + stage * kT8TileBytes;
-        for (uint32_t b = 0; b < kT8Boxes; ++b)
-          tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kT8Cols + 64u * b), (int)(tr * kTileRows), bar);
+        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tile_id0 + 4 * stage), "r"(t) : "memory");
+        if (t < num_tiles) {
+          const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kT8TileBytes) : "memory");
+          const uint32_t dst = base + stage * kT8TileBytes;
+          for (uint32_t b = 0; b < kT8Boxes; ++b)
+            tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kT8Cols + 64u * b), (int)(tr * kTileRows), bar);
+        } else {
+          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");  // nothing will land: complete the phase
+        }
       }
       __syncwarp();
+      if (t >= num_tiles) break;
+    }
+    // this CTA asks for no more tiles: count it; the last one leaves the slot as it found it
+    if (lane == 0) {
+      __threadfence();
+      if (atomicInc(&sched[1], gridDim.x - 1u) == gridDim.x - 1u) atomicExch(&sched[0], 0u);
     }
     return;
   }
 
   // -------------------------------- readers --------------------------------
-  uint32_t it = 0;
 #pragma unroll 1
-  for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
+  for (uint32_t it = 0;; ++it) {
     const uint32_t stage = it % kStages, parity = (it / kStages) & 1u;
     if (!tile_wait(bar0 + 8 * stage, parity)) {
       if (lane == 0) atomicCAS(&g_tile_status, 0u, 1u);
       return;
     }
+    uint32_t t;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t) : "r"(tile_id0 + 4 * stage) : "memory");
+    if (t >= num_tiles) return;  // no tile left
     const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
     const uint32_t tile_base = base + stage * kT8TileBytes;
     const uint32_t row0 = tr * kTileRows, col0 = tc * kT8Cols;
@@ -470,7 +508,7 @@ cudaError_t launch_tile8_t(const DualArgs& a) {
   if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
     return cudaErrorInvalidValue;
-  constexpr uint32_t smem = 3 * kT8TileBytes + 6 * 8 + 1024;
+  constexpr uint32_t smem = 3 * kT8TileBytes + 6 * 8 + 3 * 4 + 4 + 1024;  // stages, barriers, tile numbers, alignment slack
   static bool attr_set[64] = {false};
   int dev = 0;
   e = cudaGetDevice(&dev);
@@ -484,10 +522,10 @@ cudaError_t launch_tile8_t(const DualArgs& a) {
   const uint32_t tiles_r = (uint32_t)(a.R / kTileRows), tiles_c = (uint32_t)(a.C / kT8Cols);
   const uint32_t num_tiles = tiles_r * tiles_c;
   const uint32_t slots = (uint32_t)kT8CtasPerSm * (uint32_t)a.sm_count;
-  const uint32_t rounds = (num_tiles + slots - 1) / slots;
-  const uint32_t grid = (num_tiles + rounds - 1) / rounds;
+  const uint32_t grid = num_tiles < slots ? num_tiles : slots;
+  const uint32_t sched_slot = next_sched_slot();
   return launch_pdl(kernel, dim3(grid), dim3(kTile8Threads), smem, a.stream, map, a.elems_row, a.scales_row,
-                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
+                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles, sched_slot);
 }
 
 template <int FMT>
