@@ -330,19 +330,23 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
 // written: every warp converts its share of a tile straight out of the (read-only) stage and the
 // only synchronisation left is the stage's two barriers -- "tile landed" (the copy engine) and
 // "tile read" (one arrival per warp), which a producer warp waits on before it refills the stage.
-//   warps 0-15  row pass: lane (r, h) = (lane % 8, lane / 8) converts the two blocks of row
-//               8 w + r that lie in box h (one 128-byte box row: eight 16-byte loads; a quarter-warp
-//               reads eight rows of one box, conflict-free under the 128-byte swizzle) and writes
-//               them as one 64-byte run plus two adjacent scale bytes;
-//               column pass: warp w = (box b, row group g) = (w % 4, w / 4), lane = one 32-bit word
-//               column of box b (two columns), 32 rows down (32 conflict-free 4-byte loads): two
-//               whole-sector stores and two scale bytes
-//   warp 16     producer: one lane issues the four box copies of a tile into a stage once its
-//               sixteen readers have released it
+// With NBOX boxes of 64 columns side by side in a tile (NBOX x 128 contiguous bytes of every row):
+//   warps 0 .. 4 NBOX - 1
+//               row pass: lane (r, h) = (lane % (32 / NBOX), lane / (32 / NBOX)) converts the two
+//               blocks that row (32 / NBOX) w + r has in box h (one 128-byte box row: eight 16-byte
+//               loads; a quarter-warp reads eight rows of one box, conflict-free under the
+//               128-byte swizzle) and writes them as one 64-byte run plus two adjacent scale bytes;
+//               column pass: warp w = (box b, row group g) = (w % NBOX, w / NBOX), lane = one 32-bit
+//               word column of box b (two columns), 32 rows down (32 conflict-free 4-byte loads):
+//               two whole-sector stores and two scale bytes
+//   warp 4 NBOX producer: one lane issues the box copies of a tile into a stage once its readers
+//               have released it
 // ---------------------------------------------------------------------------------------------
-// Tile of the 8-bit kernel: 128 rows x four boxes of 64 columns side by side (512 contiguous bytes
-// of every row), 16 reader warps + the producer warp, three stages of 64 KB.
-constexpr uint32_t kT8Boxes = 4;  // (two boxes and two CTAs per SM measured 52.8 us against 51.3 on 8192 x 8192)
+// Two boxes: tiles of 128 x 128, eight reader warps + the producer, three stages of 32 KB, two
+// CTAs per SM.  Measured with the tiles dealt out at run time (see the producer): 46.9 us on 8192 x
+// 8192 and 15.7 on 4096 x 4096, against 47.2 and 16.4 with four boxes (128 x 256 tiles, 16 reader
+// warps, one CTA per SM); with a static split of the tiles it was the other way round (52.8 / 51.3).
+constexpr uint32_t kT8Boxes = 2;
 constexpr uint32_t kT8Warps = 4 * kT8Boxes;
 constexpr int kTile8Threads = 32 * (kT8Warps + 1);
 constexpr uint32_t kT8TileBytes = kT8Boxes * kBoxBytes;
@@ -380,8 +384,9 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
 
   if (warp == kT8Warps) {
     // ------------------------------- producer -------------------------------
-    // Tiles are dealt out at run time: an SM's share of the memory system's bandwidth varies (the
-    // slowest of 147 CTAs with 14 tiles each took 95 k cycles, the median 79 k), so a CTA's first
+    // Tiles are dealt out at run time: an SM's share of the memory system's bandwidth varies (with
+    // 128 x 256 tiles split evenly, 14 per CTA, the slowest of 147 CTAs took 95 k cycles and the
+    // median 79 k: 8192 x 8192 in 51.3 us; dealt out, 47.0 us), so a CTA's first
     // tile is its own index and every further one comes from a counter.  The tile a stage holds is
     // written beside the barriers before the stage is armed; a number past the last tile tells the
     // readers to stop.
@@ -588,14 +593,13 @@ cudaError_t dispatch_tile_round(const DualArgs& a) {
 // BF16 input, R and C multiples of 128 (what mx_quantize_dual requires of BF16 tensors).
 cudaError_t launch_quantize_tile(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
-  const bool wide8 = a.C % kT8Cols == 0;  // the 8-bit kernel's tiles; other widths take the general tile kernel
   switch (a.fmt) {
-    case MX_E4M3: return wide8 ? dispatch_tile8<MX_E4M3>(a) : dispatch_tile_round<MX_E4M3, false>(a);
-    case MX_E5M2: return wide8 ? dispatch_tile8<MX_E5M2>(a) : dispatch_tile_round<MX_E5M2, false>(a);
+    case MX_E4M3: return dispatch_tile8<MX_E4M3>(a);
+    case MX_E5M2: return dispatch_tile8<MX_E5M2>(a);
     case MX_E3M2: return dispatch_tile_round<MX_E3M2, false>(a);
     case MX_E2M3: return dispatch_tile_round<MX_E2M3, false>(a);
     case MX_E2M1: return dispatch_tile_round<MX_E2M1, false>(a);
-    default: return wide8 ? dispatch_tile8<MX_INT8>(a) : dispatch_tile_round<MX_INT8, false>(a);
+    default: return dispatch_tile8<MX_INT8>(a);
   }
 }
 
