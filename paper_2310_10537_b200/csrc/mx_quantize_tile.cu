@@ -359,10 +359,11 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
                       uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
                       uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
                       uint32_t num_tiles, uint32_t sched_slot) {
-  static_assert(FmtTraits<FMT>::bits == 8, "8-bit codes only");
+  constexpr int bits = FmtTraits<FMT>::bits;
+  static_assert(bits == 8 || (bits == 4 && kT8Boxes == 2), "8-bit codes, or 4-bit codes on 128 x 128 tiles");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
-  constexpr uint32_t kBpb = 32;
+  constexpr uint32_t kBpb = kBlock * bits / 8;  // 32 or 16 bytes of codes per block
   extern __shared__ uint8_t tile_smem_raw[];
   const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
   const uint32_t bar0 = base + kStages * kT8TileBytes;      // full[s] at 8 s, empty[s] at 8 (kStages + s)
@@ -467,14 +468,20 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
       }
       const uint32_t row = row0 + r, kb0 = tc * (kT8Cols / kBlock) + 2u * h;
       uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
-      const uint32_t run[16] = {codes[0][0], codes[0][1], codes[0][2], codes[0][3], codes[0][4], codes[0][5],
-                                codes[0][6], codes[0][7], codes[1][0], codes[1][1], codes[1][2], codes[1][3],
-                                codes[1][4], codes[1][5], codes[1][6], codes[1][7]};
-      store_run<16>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      if (bits == 8) {
+        const uint32_t run[16] = {codes[0][0], codes[0][1], codes[0][2], codes[0][3], codes[0][4], codes[0][5],
+                                  codes[0][6], codes[0][7], codes[1][0], codes[1][1], codes[1][2], codes[1][3],
+                                  codes[1][4], codes[1][5], codes[1][6], codes[1][7]};
+        store_run<16>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      } else {  // 4-bit: a block is four words (cast8 leaves them in the even positions), two blocks one sector
+        const uint32_t run[8] = {codes[0][0], codes[0][2], codes[0][4], codes[0][6],
+                                 codes[1][0], codes[1][2], codes[1][4], codes[1][6]};
+        store_run<8>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      }
       // two adjacent bytes in either layout (kb0 even, C % 128 == 0)
       *reinterpret_cast<uint16_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = (uint16_t)scale_pair;
     }
-    {  // column pass: one word column (two columns) of one box, one 32-row group
+    if constexpr (bits == 8) {  // column pass: one word column (two columns) of one box, one 32-row group
       const uint32_t b = warp % kT8Boxes, g = warp / kT8Boxes;
       const uint32_t box = tile_base + b * kBoxBytes;
       const uint32_t c = lane >> 2, wofs = (lane & 3u) * 4u;
@@ -495,6 +502,54 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
         store_run<8>(dst, cw, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
         scales_col[scale_offset<LAYOUT>(col, kb, kb_col)] = (uint8_t)s.byte;
       }
+    }
+    if constexpr (bits == 4) {
+      // column pass, 4-bit codes: a block is 16 bytes, so two lanes -- the same word column, row groups
+      // 2 gp and 2 gp + 1 -- make up the 32-byte sector of each of their two columns: each keeps one
+      // column and hands the other column's block (and scale byte) to its partner.  Warp w = (quarter
+      // wq of the tile's 64 word columns, pair of row groups gp) = (w % 4, w / 4); lane = (word
+      // column lane % 16, row group 2 gp + lane / 16).  (16 lanes read half a 128-byte row: a load
+      // instruction touches two rows, two wavefronts.)
+      const uint32_t wq = warp % 4u, gp = warp / 4u, hi = lane >> 4, g = 2u * gp + hi;
+      const uint32_t w = 16u * (wq & 1u) + (lane & 15u);          // word column inside the box
+      const uint32_t box = tile_base + (wq >> 1) * kBoxBytes;
+      const uint32_t c = w >> 2, wofs = (w & 3u) * 4u;
+      uint32_t raw[kBlock][1];
+#pragma unroll
+      for (uint32_t k = 0; k < kBlock; ++k)
+        asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, g * kBlock + k, c) + wofs));
+      float amax[2];
+      column_amax<DTYPE, 2>(raw, amax);
+      uint32_t blk[2][4], sbyte[2];
+#pragma unroll
+      for (int cc = 0; cc < 2; ++cc) {
+        const BlockScale s = block_scale<FMT>(amax[cc]);
+        uint32_t cw[8];
+        column_cast<FMT, ROUND, DTYPE, 2>(raw, cc, s, cw);
+        sbyte[cc] = s.byte;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) blk[cc][i] = cw[2 * i];
+      }
+      // keep column `hi`, give away column 1 - hi
+      uint32_t mine[4], theirs[4];
+#pragma unroll
+      for (int i = 0; i < 4; ++i) {
+        mine[i] = hi ? blk[1][i] : blk[0][i];
+        theirs[i] = __shfl_xor_sync(0xFFFFFFFFu, hi ? blk[0][i] : blk[1][i], 16);
+      }
+      const uint32_t their_scale = __shfl_xor_sync(0xFFFFFFFFu, hi ? sbyte[0] : sbyte[1], 16);
+      const uint32_t my_scale = hi ? sbyte[1] : sbyte[0];
+      // blocks in order of their row groups: the even group's first
+      const uint32_t run[8] = {hi ? theirs[0] : mine[0], hi ? theirs[1] : mine[1], hi ? theirs[2] : mine[2],
+                               hi ? theirs[3] : mine[3], hi ? mine[0] : theirs[0], hi ? mine[1] : theirs[1],
+                               hi ? mine[2] : theirs[2], hi ? mine[3] : theirs[3]};
+      const uint32_t col = col0 + (wq >> 1) * 64u + w * 2u + hi;
+      const uint32_t kb = tr * 4u + 2u * gp;
+      uint8_t* dst = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
+      store_run<8>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      const uint32_t pair = hi ? (their_scale | (my_scale << 8)) : (my_scale | (their_scale << 8));
+      // two adjacent bytes in either layout (kb even)
+      *reinterpret_cast<uint16_t*>(scales_col + scale_offset<LAYOUT>(col, kb, kb_col)) = (uint16_t)pair;
     }
     __syncwarp();
     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8 * (kStages + stage)) : "memory");
@@ -598,7 +653,7 @@ cudaError_t launch_quantize_tile(const DualArgs& a) {
     case MX_E5M2: return dispatch_tile8<MX_E5M2>(a);
     case MX_E3M2: return dispatch_tile_round<MX_E3M2, false>(a);
     case MX_E2M3: return dispatch_tile_round<MX_E2M3, false>(a);
-    case MX_E2M1: return dispatch_tile_round<MX_E2M1, false>(a);
+    case MX_E2M1: return dispatch_tile8<MX_E2M1>(a);
     default: return dispatch_tile8<MX_INT8>(a);
   }
 }
