@@ -360,7 +360,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
                       uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
                       uint32_t num_tiles, uint32_t sched_slot) {
   constexpr int bits = FmtTraits<FMT>::bits;
-  static_assert(bits == 8 || (bits == 4 && kT8Boxes == 2), "8-bit codes, or 4-bit codes on 128 x 128 tiles");
+  static_assert(bits == 8 || kT8Boxes == 2, "sub-byte codes: 128 x 128 tiles (their lane maps assume two boxes)");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
   constexpr uint32_t kBpb = kBlock * bits / 8;  // 32 or 16 bytes of codes per block
@@ -441,7 +441,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
     const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
     const uint32_t tile_base = base + stage * kT8TileBytes;
     const uint32_t row0 = tr * kTileRows, col0 = tc * kT8Cols;
-    {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
+    if constexpr (bits != 6) {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
       constexpr uint32_t kRowsPerWarp = 32 / kT8Boxes;   // 16 or 8
       const uint32_t r = warp * kRowsPerWarp + (lane % kRowsPerWarp), h = lane / kRowsPerWarp;
       const uint32_t box = tile_base + h * kBoxBytes;
@@ -473,7 +473,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
                                   codes[0][6], codes[0][7], codes[1][0], codes[1][1], codes[1][2], codes[1][3],
                                   codes[1][4], codes[1][5], codes[1][6], codes[1][7]};
         store_run<16>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
-      } else {  // 4-bit: a block is four words (cast8 leaves them in the even positions), two blocks one sector
+      } else if (bits == 4) {  // a block is four words (cast8 leaves them in the even positions), two blocks one sector
         const uint32_t run[8] = {codes[0][0], codes[0][2], codes[0][4], codes[0][6],
                                  codes[1][0], codes[1][2], codes[1][4], codes[1][6]};
         store_run<8>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
@@ -550,6 +550,103 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
       const uint32_t pair = hi ? (their_scale | (my_scale << 8)) : (my_scale | (their_scale << 8));
       // two adjacent bytes in either layout (kb even)
       *reinterpret_cast<uint16_t*>(scales_col + scale_offset<LAYOUT>(col, kb, kb_col)) = (uint16_t)pair;
+    }
+    if constexpr (bits == 6) {
+      // 6-bit codes: a block is 24 bytes, four blocks three sectors, so whole sectors need all four
+      // blocks of a tile row or of a tile column in one place.  The warps split the roles: warps 4-7
+      // convert rows (lane = one tile row: its four blocks, one 96-byte run), warps 0-3 columns --
+      // warp w the w-th quarter of the tile's 64 word columns, in two steps of two row groups each
+      // (lane = (word column lane % 16, row group 2 step + lane / 16): a load instruction touches two
+      // rows, two wavefronts); the two lanes of a word column then hold row groups {0, 2} and {1, 3}
+      // of both columns and pass eight words to each other so that one writes sectors 0 and 1 of
+      // each column and the other sector 2.  Both roles convert 128 elements per lane and tile.
+      if (warp >= 4u) {
+        const uint32_t r = (warp - 4u) * 32u + lane;
+        uint32_t run[24];
+        uint32_t scale_word = 0;
+#pragma unroll
+        for (uint32_t q = 0; q < 4; ++q) {
+          const uint32_t box = tile_base + (q >> 1) * kBoxBytes;
+          uint32_t u[16];
+#pragma unroll
+          for (uint32_t i = 0; i < 4; ++i) {
+            uint32_t v0, v1, v2, v3;
+            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                         : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(box_chunk(box, r, (q & 1u) * 4u + i)));
+            u[4 * i] = v0; u[4 * i + 1] = v1; u[4 * i + 2] = v2; u[4 * i + 3] = v3;
+          }
+          const BlockScale s = block_scale<FMT>(unit_amax<DTYPE>(u));
+          scale_word |= s.byte << (8 * q);
+          uint32_t cw[8], o[6];
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {
+            float x[8];
+            unit_group<DTYPE>(u, g, x);
+            cast8<FMT, ROUND>(x, s, cw[2 * g], cw[2 * g + 1]);
+          }
+          pack6_words(cw, o);
+#pragma unroll
+          for (int i = 0; i < 6; ++i) run[6 * q + i] = o[i];
+        }
+        const uint32_t row = row0 + r, kb0 = tc * 4u;
+        uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
+        store_run<24>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+        // four adjacent bytes in either layout (kb0 % 4 == 0)
+        *reinterpret_cast<uint32_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = scale_word;
+      } else {
+        const uint32_t hi = lane >> 4;
+        const uint32_t w = 16u * (warp & 1u) + (lane & 15u);        // word column inside the box
+        const uint32_t box = tile_base + (warp >> 1) * kBoxBytes;
+        const uint32_t c = w >> 2, wofs = (w & 3u) * 4u;
+        uint32_t o[2][2][6];   // [step][column][word]: row group 2 step + hi
+        uint32_t sb[2] = {0u, 0u};  // per column: this lane's two scale bytes at their positions in the word
+#pragma unroll
+        for (uint32_t step = 0; step < 2; ++step) {
+          const uint32_t g = 2u * step + hi;
+          uint32_t raw[kBlock][1];
+#pragma unroll
+          for (uint32_t k = 0; k < kBlock; ++k)
+            asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, g * kBlock + k, c) + wofs));
+          float amax[2];
+          column_amax<DTYPE, 2>(raw, amax);
+#pragma unroll
+          for (int cc = 0; cc < 2; ++cc) {
+            const BlockScale s = block_scale<FMT>(amax[cc]);
+            uint32_t cw[8];
+            column_cast<FMT, ROUND, DTYPE, 2>(raw, cc, s, cw);
+            pack6_words(cw, o[step][cc]);
+            sb[cc] |= s.byte << (8 * g);
+          }
+        }
+        const uint32_t kb = tr * 4u;
+#pragma unroll
+        for (int cc = 0; cc < 2; ++cc) {
+          // the run's 24 words: groups 0 and 2 in lane hi = 0 (o[0], o[1]), groups 1 and 3 in lane hi = 1.
+          // sector 0 = g0[0..5] g1[0..1], sector 1 = g1[2..5] g2[0..3] (both written by hi = 0),
+          // sector 2 = g2[4..5] g3[0..5] (written by hi = 1)
+          uint32_t p1[6], p2[2];
+#pragma unroll
+          for (int i = 0; i < 6; ++i) p1[i] = __shfl_xor_sync(0xFFFFFFFFu, o[0][cc][i], 16);       // hi = 0 receives g1
+#pragma unroll
+          for (int i = 0; i < 2; ++i) p2[i] = __shfl_xor_sync(0xFFFFFFFFu, o[1][cc][4 + i], 16);   // hi = 1 receives g2[4..5]
+          const uint32_t col = col0 + (warp >> 1) * 64u + w * 2u + cc;
+          uint8_t* run0 = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
+          const bool wide = (reinterpret_cast<uintptr_t>(run0) & 31u) == 0;
+          if (hi == 0) {
+            const uint32_t run[16] = {o[0][cc][0], o[0][cc][1], o[0][cc][2], o[0][cc][3], o[0][cc][4], o[0][cc][5],
+                                      p1[0], p1[1], p1[2], p1[3], p1[4], p1[5],
+                                      o[1][cc][0], o[1][cc][1], o[1][cc][2], o[1][cc][3]};
+            store_run<16>(run0, run, wide);
+          } else {
+            const uint32_t run[8] = {p2[0], p2[1], o[1][cc][0], o[1][cc][1], o[1][cc][2], o[1][cc][3],
+                                     o[1][cc][4], o[1][cc][5]};
+            store_run<8>(run0 + 64, run, wide);
+          }
+          // the column's four scale bytes as one word (adjacent in either layout: kb % 4 == 0)
+          const uint32_t word = sb[cc] | __shfl_xor_sync(0xFFFFFFFFu, sb[cc], 16);
+          if (hi == 1) *reinterpret_cast<uint32_t*>(scales_col + scale_offset<LAYOUT>(col, kb, kb_col)) = word;
+        }
+      }
     }
     __syncwarp();
     if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8 * (kStages + stage)) : "memory");
@@ -651,8 +748,8 @@ cudaError_t launch_quantize_tile(const DualArgs& a) {
   switch (a.fmt) {
     case MX_E4M3: return dispatch_tile8<MX_E4M3>(a);
     case MX_E5M2: return dispatch_tile8<MX_E5M2>(a);
-    case MX_E3M2: return dispatch_tile_round<MX_E3M2, false>(a);
-    case MX_E2M3: return dispatch_tile_round<MX_E2M3, false>(a);
+    case MX_E3M2: return dispatch_tile8<MX_E3M2>(a);
+    case MX_E2M3: return dispatch_tile8<MX_E2M3>(a);
     case MX_E2M1: return dispatch_tile8<MX_E2M1>(a);
     default: return dispatch_tile8<MX_INT8>(a);
   }
