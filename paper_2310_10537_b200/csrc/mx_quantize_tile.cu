@@ -1,36 +1,36 @@
-// Dual-axis quantize of a BF16 tensor through shared-memory tiles: X[R x C] is read once, by TMA,
-// in tiles of 128 rows x 128 columns, and each tile is quantized out of shared memory both along
-// its rows (blocks along the contiguous axis: the operand of X W) and along its columns (blocks
-// along axis 0: the K-major [C x R] operand of X^T dY).  The paper's compute flow (Section 4.1)
-// quantizes every matmul input in the forward and in the backward pass, and because quantizing
-// and transposing do not commute (Section 3) those are two tensors; producing both from one read
-// removes a third of the traffic.
+// Quantize of a BF16 tensor through shared-memory tiles: X[R x C] is read once, by TMA, in tiles of
+// 128 rows x 128 columns, and each tile is quantized out of shared memory along its rows (blocks
+// along the contiguous axis: the operand of X W) and along its columns (blocks along axis 0: the
+// K-major [C x R] operand of X^T dY).  The paper's compute flow (Section 4.1) quantizes every matmul
+// input in the forward and in the backward pass, and because quantizing and transposing do not
+// commute (Section 3) those are two tensors; producing both from one read removes a third of the
+// traffic.
 //
 // Why through shared memory: a thread that keeps 32 rows of a block in registers (the kernel in
-// mx_quantize_dual.cu, still used for FP32 input) needs ~250 registers once BF16 packs twice the
+// mx_quantize_dual.cu, used for FP32 input) needs ~250 registers once BF16 packs twice the
 // elements into them and both directions are served, which leaves eight warps per SM -- too few
 // loads in flight to cover HBM latency (measured: 11 % of the warp slots active, DRAM 47 % busy).
-// Here the copies in flight cost no registers: a CTA keeps kStages - 1 tiles (32 KB each) on their
-// way while it converts one, two CTAs share an SM (16 warps, <= 128 registers), and a converting
-// thread holds one block at a time.
+// Here the copies in flight cost no registers: a CTA keeps tiles (32 KB each, two TMA boxes of 128
+// rows x 128 bytes in the 128-byte swizzle) on their way while it converts one, two CTAs share an
+// SM, and a converting thread holds one block at a time.  The swizzle makes both access directions
+// conflict-free: a row's 16-byte chunks are spread over the banks by (chunk ^ row % 8), a word
+// column's 32 lanes always hit 32 different banks.  Every mbarrier wait is bounded: when one runs
+// out the CTA records it in a status word and leaves.
 //
-//   thread 0      issues the two TMA box copies of a tile (128 rows x 128 bytes each, in the
-//                 128-byte swizzle) kStages - 1 tiles ahead; everybody waits on the stage's mbarrier
-//   warps 0-3     row pass: thread r converts row r of the tile; its 4 blocks are one contiguous
-//                 run of the [R x C] output, written as whole 32-byte sectors
-//   warps 4-7     column pass, at the same time (equal work): a thread converts the 32 rows of one
-//                 32-bit word column (2 columns) of one 32-row group; 8-bit codes leave as one
-//                 sector per block, 6- and 4-bit codes are parked in shared memory so that a
-//                 column's four blocks (96 / 64 bytes) leave as whole sectors too; a column's four
-//                 scale bytes leave as one word
-// The swizzle makes both access directions conflict-free: a row's 16-byte chunks are spread over
-// the banks by (chunk ^ row % 8), a word column's 32 lanes always hit 32 different banks.
-// The mbarrier wait is bounded: when it runs out the CTA records it in a status word and leaves.
-// Measured on 8192 x 8192 (both outputs): E4M3 53 us against 59 us for the register kernel, E3M2 47
-// against 67, E2M1 41 against 52.  Timing-only builds say what the time is made of: copies alone 22
-// us, both passes without their stores 33 us, one pass with its stores 35 us -- the two conversions
-// are ~5 instructions per element each and do not overlap the 42 us the bytes need well enough.
-// 8-bit codes have a kernel of their own below (no meeting of warps): 51 us.
+// Two kernels:
+//   quantize_tile_dual_kernel      both outputs (mx_quantize_dual), every format.  No meeting of warps:
+//                              every warp writes whole 32-byte sectors by itself (sub-byte codes:
+//                              lanes exchange part sectors by shuffle), a producer warp refills a
+//                              stage when its readers have released it, tiles are dealt out at run
+//                              time.  8192 x 8192: E4M3 46.8 us, E3M2 44.0, E2M1 34.5 (0.89 / 0.83 /
+//                              0.91 of the copy bandwidth on in + 2 x out bytes).
+//   quantize_tile_cols_kernel  the column-block tensor alone, 6-bit codes (mx_quantize along axis 0
+//                              of whole-tile tensors, where it beats the register kernels): all
+//                              eight warps convert word columns, the codes are parked in shared
+//                              memory and leave as whole sectors after a meeting of the warps.
+// (The second kernel used to do both passes -- warps 0-3 rows, warps 4-7 columns, a CTA barrier per
+// tile -- and measured 53 / 47 / 41 us on 8192 x 8192 for E4M3 / E3M2 / E2M1; timing-only builds of
+// it: copies alone 22 us, both passes without their stores 33, one pass with its stores 35.)
 #include <atomic>
 
 #include "mx_device.cuh"
@@ -66,7 +66,6 @@ template <int FMT> struct TileCfg {
   static constexpr int bits = FmtTraits<FMT>::bits;
   static constexpr uint32_t kBpb = kBlock * bits / 8;                   // bytes of one block of codes
   static constexpr uint32_t kCols = 128;                                // columns of a tile (256 bytes of BF16)
-  static constexpr uint32_t kRowBlocks = kCols / kBlock;                // blocks in a tile row
   static constexpr uint32_t kStages = 3;
   // column codes of sub-byte formats: per column its four blocks; the pad makes the stores of 32
   // lanes (one slot apart) conflict-free: 26 words for 8-byte stores, 20 words for 16-byte stores
@@ -107,17 +106,15 @@ __device__ __forceinline__ uint32_t box_chunk(uint32_t box_base, uint32_t r, uin
   return box_base + r * 128u + ((c ^ (r & 7u)) << 4);
 }
 
-template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY>
+template <int FMT, int ROUND, int LAYOUT>
 __global__ void __launch_bounds__(kTileThreads, 2)
-quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
-                     uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
-                     uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
-                     uint32_t num_tiles) {
+quantize_tile_cols_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_col,
+                          uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
+                          uint32_t num_tiles) {
   using cfg = TileCfg<FMT>;
   constexpr int DTYPE = MX_BF16;
   constexpr int bits = cfg::bits;
   constexpr uint32_t kBpb = cfg::kBpb;
-  constexpr uint32_t kRowBlocks = cfg::kRowBlocks;
   constexpr uint32_t kBoxCols = cfg::kCols / 2;  // columns of one box
   extern __shared__ uint8_t tile_smem_raw[];
   const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
@@ -151,8 +148,8 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
     }
   }
 
-  const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;  // blocks per output row
-  const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
+  const uint32_t kb_col = R / kBlock;  // blocks per output row
+  const size_t col_out_bytes = (size_t)kb_col * kBpb;
   uint32_t it = 0;
 #pragma unroll 1
   for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
@@ -167,77 +164,13 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
     }
     const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
     const uint32_t tile_base = base + stage * kTileBytes;
-    const uint32_t row0 = tr * kTileRows, col0 = tc * cfg::kCols;
-
-    // ------------------------------ row pass ------------------------------
-    if (!COLS_ONLY && tid < 128) {
-      constexpr uint32_t kPer = kRowBlocks;  // blocks per thread: its whole tile row
-      const uint32_t r = tid, q0 = 0;
-      const uint32_t row = row0 + r;
-      if (row < R) {
-        uint32_t codes[kPer][8];
-        uint32_t scale_word = 0;
-#pragma unroll
-        for (uint32_t qq = 0; qq < kPer; ++qq) {
-          const uint32_t q = q0 + qq;  // block of the tile row
-          uint32_t u[16];  // the block: 64 bytes = chunks 4 (q % 2) .. + 3 of box q / 2
-          const uint32_t box = tile_base + (q >> 1) * kBoxBytes;
-#pragma unroll
-          for (uint32_t i = 0; i < 4; ++i) {
-            uint32_t v0, v1, v2, v3;
-            asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
-                         : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(box_chunk(box, r, (q & 1u) * 4u + i)));
-            u[4 * i] = v0; u[4 * i + 1] = v1; u[4 * i + 2] = v2; u[4 * i + 3] = v3;
-          }
-          const BlockScale s = block_scale<FMT>(unit_amax<DTYPE>(u));
-          scale_word |= s.byte << (8 * qq);
-#pragma unroll
-          for (int g = 0; g < 4; ++g) {
-            float x[8];
-            unit_group<DTYPE>(u, g, x);
-            cast8<FMT, ROUND>(x, s, codes[qq][2 * g], codes[qq][2 * g + 1]);
-          }
-        }
-        const uint32_t kb0 = tc * kRowBlocks + q0;  // first block of this thread in the output row
-        uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
-        const bool wide = (reinterpret_cast<uintptr_t>(dst) & 31u) == 0;
-        if (bits == 8) {
-          uint32_t run[kPer * 8];
-#pragma unroll
-          for (uint32_t q = 0; q < kPer; ++q)
-#pragma unroll
-            for (int i = 0; i < 8; ++i) run[8 * q + i] = codes[q][i];
-          store_run<(int)(kPer * 8)>(dst, run, wide);
-        } else if (bits == 4) {
-          uint32_t run[kPer * 4];
-#pragma unroll
-          for (uint32_t q = 0; q < kPer; ++q)
-#pragma unroll
-            for (int i = 0; i < 4; ++i) run[4 * q + i] = codes[q][2 * i];
-          store_run<(int)(kPer * 4)>(dst, run, wide);
-        } else {
-          uint32_t run[kPer * 6];
-#pragma unroll
-          for (uint32_t q = 0; q < kPer; ++q) {
-            uint64_t a, b, c;
-            pack6(codes[q], a, b, c);
-            run[6 * q] = (uint32_t)a; run[6 * q + 1] = (uint32_t)(a >> 32);
-            run[6 * q + 2] = (uint32_t)b; run[6 * q + 3] = (uint32_t)(b >> 32);
-            run[6 * q + 4] = (uint32_t)c; run[6 * q + 5] = (uint32_t)(c >> 32);
-          }
-          store_run<(int)(kPer * 6)>(dst, run, wide);
-        }
-        uint8_t* sdst = scales_row + scale_offset<LAYOUT>(row, kb0, kb_row);
-        *reinterpret_cast<uint32_t*>(sdst) = scale_word;  // four adjacent bytes in either layout (C % 128 == 0)
-      }
-    }
+    const uint32_t col0 = tc * cfg::kCols;
 
     // ----------------------------- column pass -----------------------------
-    // (COLS_ONLY: the kernel serves mx_quantize along axis 0 and all eight warps take this pass)
-    if (COLS_ONLY || tid >= 128) {
-      constexpr uint32_t kColThreads = COLS_ONLY ? 256 : 128;
+    {
+      constexpr uint32_t kColThreads = kTileThreads;  // all eight warps
       constexpr int kWordCols = 2;   // columns in one 32-bit word
-      const uint32_t ct = COLS_ONLY ? tid : tid - 128;
+      const uint32_t ct = tid;
       uint8_t* codes_smem = gen + cfg::kOffCodes;
       uint8_t* scale_smem = gen + cfg::kOffScales;
       // 64 word columns x 4 row groups = 256 units of 32 rows x one word
@@ -325,11 +258,13 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
 
 
 // ---------------------------------------------------------------------------------------------
-// 8-bit codes, both passes, no meeting of warps.  A block of 8-bit codes is a whole 32-byte sector
-// and its scale a byte of its own, so nothing has to be gathered across warps before it is
-// written: every warp converts its share of a tile straight out of the (read-only) stage and the
-// only synchronisation left is the stage's two barriers -- "tile landed" (the copy engine) and
-// "tile read" (one arrival per warp), which a producer warp waits on before it refills the stage.
+// Both passes, no meeting of warps.  Nothing is gathered across warps before it is written: every
+// warp converts its share of a tile straight out of the (read-only) stage and writes whole 32-byte
+// sectors by itself, and the only synchronisation left is the stage's two barriers -- "tile landed"
+// (the copy engine) and "tile read" (one arrival per warp), which a producer warp waits on before
+// it refills the stage.  A block of 8-bit codes is a sector; two blocks of 4-bit codes are, and
+// four blocks of 6-bit codes are three, so for those two or four lanes pass words to each other
+// (see the 4- and 6-bit branches).  The lane maps of 8- and 4-bit codes:
 // With NBOX boxes of 64 columns side by side in a tile (NBOX x 128 contiguous bytes of every row):
 //   warps 0 .. 4 NBOX - 1
 //               row pass: lane (r, h) = (lane % (32 / NBOX), lane / (32 / NBOX)) converts the two
@@ -346,33 +281,33 @@ quantize_tile_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __res
 // CTAs per SM.  Measured with the tiles dealt out at run time (see the producer): 46.9 us on 8192 x
 // 8192 and 15.7 on 4096 x 4096, against 47.2 and 16.4 with four boxes (128 x 256 tiles, 16 reader
 // warps, one CTA per SM); with a static split of the tiles it was the other way round (52.8 / 51.3).
-constexpr uint32_t kT8Boxes = 2;
-constexpr uint32_t kT8Warps = 4 * kT8Boxes;
-constexpr int kTile8Threads = 32 * (kT8Warps + 1);
-constexpr uint32_t kT8TileBytes = kT8Boxes * kBoxBytes;
-constexpr uint32_t kT8Cols = 64 * kT8Boxes;
-constexpr int kT8CtasPerSm = kT8Boxes == 2 ? 2 : 1;
+constexpr uint32_t kTdBoxes = 2;
+constexpr uint32_t kTdWarps = 4 * kTdBoxes;
+constexpr int kTileDualThreads = 32 * (kTdWarps + 1);
+constexpr uint32_t kTdTileBytes = kTdBoxes * kBoxBytes;
+constexpr uint32_t kTdCols = 64 * kTdBoxes;
+constexpr int kTdCtasPerSm = kTdBoxes == 2 ? 2 : 1;
 
 template <int FMT, int ROUND, int LAYOUT>
-__global__ void __launch_bounds__(kTile8Threads, kT8CtasPerSm)
-quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
+__global__ void __launch_bounds__(kTileDualThreads, kTdCtasPerSm)
+quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
                       uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
                       uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
                       uint32_t num_tiles, uint32_t sched_slot) {
   constexpr int bits = FmtTraits<FMT>::bits;
-  static_assert(bits == 8 || kT8Boxes == 2, "sub-byte codes: 128 x 128 tiles (their lane maps assume two boxes)");
+  static_assert(bits == 8 || kTdBoxes == 2, "sub-byte codes: 128 x 128 tiles (their lane maps assume two boxes)");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
   constexpr uint32_t kBpb = kBlock * bits / 8;  // 32 or 16 bytes of codes per block
   extern __shared__ uint8_t tile_smem_raw[];
   const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
-  const uint32_t bar0 = base + kStages * kT8TileBytes;      // full[s] at 8 s, empty[s] at 8 (kStages + s)
+  const uint32_t bar0 = base + kStages * kTdTileBytes;      // full[s] at 8 s, empty[s] at 8 (kStages + s)
   const uint32_t tile_id0 = bar0 + 16 * kStages;            // the tile a stage holds (written by the producer)
   const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
   if (tid == 0) {
     for (uint32_t s = 0; s < kStages; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kT8Warps) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kTdWarps) : "memory");
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -383,7 +318,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
   const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;
   const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
 
-  if (warp == kT8Warps) {
+  if (warp == kTdWarps) {
     // ------------------------------- producer -------------------------------
     // Tiles are dealt out at run time: an SM's share of the memory system's bandwidth varies (with
     // 128 x 256 tiles split evenly, 14 per CTA, the slowest of 147 CTAs took 95 k cycles and the
@@ -408,10 +343,10 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
         asm volatile("st.shared.u32 [%0], %1;" ::"r"(tile_id0 + 4 * stage), "r"(t) : "memory");
         if (t < num_tiles) {
           const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kT8TileBytes) : "memory");
-          const uint32_t dst = base + stage * kT8TileBytes;
-          for (uint32_t b = 0; b < kT8Boxes; ++b)
-            tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kT8Cols + 64u * b), (int)(tr * kTileRows), bar);
+          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTdTileBytes) : "memory");
+          const uint32_t dst = base + stage * kTdTileBytes;
+          for (uint32_t b = 0; b < kTdBoxes; ++b)
+            tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kTdCols + 64u * b), (int)(tr * kTileRows), bar);
         } else {
           asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");  // nothing will land: complete the phase
         }
@@ -439,10 +374,10 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
     asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t) : "r"(tile_id0 + 4 * stage) : "memory");
     if (t >= num_tiles) return;  // no tile left
     const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
-    const uint32_t tile_base = base + stage * kT8TileBytes;
-    const uint32_t row0 = tr * kTileRows, col0 = tc * kT8Cols;
+    const uint32_t tile_base = base + stage * kTdTileBytes;
+    const uint32_t row0 = tr * kTileRows, col0 = tc * kTdCols;
     if constexpr (bits != 6) {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
-      constexpr uint32_t kRowsPerWarp = 32 / kT8Boxes;   // 16 or 8
+      constexpr uint32_t kRowsPerWarp = 32 / kTdBoxes;   // 16 or 8
       const uint32_t r = warp * kRowsPerWarp + (lane % kRowsPerWarp), h = lane / kRowsPerWarp;
       const uint32_t box = tile_base + h * kBoxBytes;
       uint32_t codes[2][8];
@@ -466,7 +401,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
           cast8<FMT, ROUND>(x, s, codes[q][2 * g], codes[q][2 * g + 1]);
         }
       }
-      const uint32_t row = row0 + r, kb0 = tc * (kT8Cols / kBlock) + 2u * h;
+      const uint32_t row = row0 + r, kb0 = tc * (kTdCols / kBlock) + 2u * h;
       uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
       if (bits == 8) {
         const uint32_t run[16] = {codes[0][0], codes[0][1], codes[0][2], codes[0][3], codes[0][4], codes[0][5],
@@ -482,7 +417,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
       *reinterpret_cast<uint16_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = (uint16_t)scale_pair;
     }
     if constexpr (bits == 8) {  // column pass: one word column (two columns) of one box, one 32-row group
-      const uint32_t b = warp % kT8Boxes, g = warp / kT8Boxes;
+      const uint32_t b = warp % kTdBoxes, g = warp / kTdBoxes;
       const uint32_t box = tile_base + b * kBoxBytes;
       const uint32_t c = lane >> 2, wofs = (lane & 3u) * 4u;
       uint32_t raw[kBlock][1];
@@ -654,7 +589,7 @@ quantize_tile8_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __re
 }
 
 template <int FMT, int ROUND, int LAYOUT>
-cudaError_t launch_tile8_t(const DualArgs& a) {
+cudaError_t launch_tile_dual_t(const DualArgs& a) {
   cudaError_t e;
   EncodeTiledFn fn = encode_fn(&e);
   if (!fn) return e;
@@ -665,37 +600,37 @@ cudaError_t launch_tile8_t(const DualArgs& a) {
   if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
     return cudaErrorInvalidValue;
-  constexpr uint32_t smem = 3 * kT8TileBytes + 6 * 8 + 3 * 4 + 4 + 1024;  // stages, barriers, tile numbers, alignment slack
+  constexpr uint32_t smem = 3 * kTdTileBytes + 6 * 8 + 3 * 4 + 4 + 1024;  // stages, barriers, tile numbers, alignment slack
   static bool attr_set[64] = {false};
   int dev = 0;
   e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  auto kernel = quantize_tile8_kernel<FMT, ROUND, LAYOUT>;
+  auto kernel = quantize_tile_dual_kernel<FMT, ROUND, LAYOUT>;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
     if (dev >= 0 && dev < 64) attr_set[dev] = true;
   }
-  const uint32_t tiles_r = (uint32_t)(a.R / kTileRows), tiles_c = (uint32_t)(a.C / kT8Cols);
+  const uint32_t tiles_r = (uint32_t)(a.R / kTileRows), tiles_c = (uint32_t)(a.C / kTdCols);
   const uint32_t num_tiles = tiles_r * tiles_c;
-  const uint32_t slots = (uint32_t)kT8CtasPerSm * (uint32_t)a.sm_count;
+  const uint32_t slots = (uint32_t)kTdCtasPerSm * (uint32_t)a.sm_count;
   const uint32_t grid = num_tiles < slots ? num_tiles : slots;
   const uint32_t sched_slot = next_sched_slot();
-  return launch_pdl(kernel, dim3(grid), dim3(kTile8Threads), smem, a.stream, map, a.elems_row, a.scales_row,
+  return launch_pdl(kernel, dim3(grid), dim3(kTileDualThreads), smem, a.stream, map, a.elems_row, a.scales_row,
                     a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles, sched_slot);
 }
 
 template <int FMT>
-cudaError_t dispatch_tile8(const DualArgs& a) {
+cudaError_t dispatch_tile_dual(const DualArgs& a) {
   if (a.rounding == MX_RHAZ)
-    return a.layout == MX_SCALES_LINEAR ? launch_tile8_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
-                                        : launch_tile8_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
-  return a.layout == MX_SCALES_LINEAR ? launch_tile8_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
-                                      : launch_tile8_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
+    return a.layout == MX_SCALES_LINEAR ? launch_tile_dual_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
+                                        : launch_tile_dual_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
+                                      : launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
 }
 
-template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY>
-cudaError_t launch_tile_t(const DualArgs& a) {
+template <int FMT, int ROUND, int LAYOUT>
+cudaError_t launch_tile_cols_t(const DualArgs& a) {
   using cfg = TileCfg<FMT>;
   cudaError_t e;
   EncodeTiledFn fn = encode_fn(&e);
@@ -711,7 +646,7 @@ cudaError_t launch_tile_t(const DualArgs& a) {
   int dev = 0;
   e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  auto kernel = quantize_tile_kernel<FMT, ROUND, LAYOUT, COLS_ONLY>;
+  auto kernel = quantize_tile_cols_kernel<FMT, ROUND, LAYOUT>;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg::kSmem);
     if (e != cudaSuccess) return e;
@@ -724,20 +659,17 @@ cudaError_t launch_tile_t(const DualArgs& a) {
   // an even share of tiles per CTA: the smallest grid that needs no more rounds than a full one
   const uint32_t rounds = (num_tiles + slots - 1) / slots;
   const uint32_t grid = (num_tiles + rounds - 1) / rounds;
-  return launch_pdl(kernel, dim3(grid), dim3(kTileThreads), cfg::kSmem, a.stream, map, a.elems_row, a.scales_row,
-                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
+  return launch_pdl(kernel, dim3(grid), dim3(kTileThreads), cfg::kSmem, a.stream, map, a.elems_col, a.scales_col,
+                    (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
 }
 
-template <int FMT, int ROUND, bool COLS_ONLY>
-cudaError_t dispatch_tile_layout(const DualArgs& a) {
-  return a.layout == MX_SCALES_LINEAR ? launch_tile_t<FMT, ROUND, MX_SCALES_LINEAR, COLS_ONLY>(a)
-                                      : launch_tile_t<FMT, ROUND, MX_SCALES_SWIZZLED, COLS_ONLY>(a);
-}
-
-template <int FMT, bool COLS_ONLY>
-cudaError_t dispatch_tile_round(const DualArgs& a) {
-  return a.rounding == MX_RHAZ ? dispatch_tile_layout<FMT, MX_RHAZ, COLS_ONLY>(a)
-                               : dispatch_tile_layout<FMT, MX_RNE, COLS_ONLY>(a);
+template <int FMT>
+cudaError_t dispatch_tile_cols(const DualArgs& a) {
+  if (a.rounding == MX_RHAZ)
+    return a.layout == MX_SCALES_LINEAR ? launch_tile_cols_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
+                                        : launch_tile_cols_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_cols_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
+                                      : launch_tile_cols_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
 }
 
 }  // namespace
@@ -746,12 +678,12 @@ cudaError_t dispatch_tile_round(const DualArgs& a) {
 cudaError_t launch_quantize_tile(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
   switch (a.fmt) {
-    case MX_E4M3: return dispatch_tile8<MX_E4M3>(a);
-    case MX_E5M2: return dispatch_tile8<MX_E5M2>(a);
-    case MX_E3M2: return dispatch_tile8<MX_E3M2>(a);
-    case MX_E2M3: return dispatch_tile8<MX_E2M3>(a);
-    case MX_E2M1: return dispatch_tile8<MX_E2M1>(a);
-    default: return dispatch_tile8<MX_INT8>(a);
+    case MX_E4M3: return dispatch_tile_dual<MX_E4M3>(a);
+    case MX_E5M2: return dispatch_tile_dual<MX_E5M2>(a);
+    case MX_E3M2: return dispatch_tile_dual<MX_E3M2>(a);
+    case MX_E2M3: return dispatch_tile_dual<MX_E2M3>(a);
+    case MX_E2M1: return dispatch_tile_dual<MX_E2M1>(a);
+    default: return dispatch_tile_dual<MX_INT8>(a);
   }
 }
 
@@ -761,8 +693,8 @@ cudaError_t launch_quantize_tile(const DualArgs& a) {
 cudaError_t launch_quantize_tile_cols(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_col || !a.scales_col) return cudaErrorInvalidValue;
   switch (a.fmt) {
-    case MX_E3M2: return dispatch_tile_round<MX_E3M2, true>(a);
-    case MX_E2M3: return dispatch_tile_round<MX_E2M3, true>(a);
+    case MX_E3M2: return dispatch_tile_cols<MX_E3M2>(a);
+    case MX_E2M3: return dispatch_tile_cols<MX_E2M3>(a);
     default: return cudaErrorInvalidValue;
   }
 }
