@@ -228,8 +228,11 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void*
     e = cudaMemsetAsync(scales_col, 0, scales_bytes(C, R / 32, o.layout), o.stream);
     if (e != cudaSuccess) return fail_cuda(e);
   }
-  // BF16: tiles through shared memory (TMA); FP32: the register kernel (measured faster there)
-  e = o.dtype == MX_BF16 ? mx::launch_quantize_tile(a) : mx::launch_quantize_dual(a);
+  // BF16: tiles through shared memory (TMA); FP32: the register kernel, except 6-bit codes of whole
+  // 128 x 128 tiles, which take a tile kernel too (the register kernel's staged variants are the slow ones)
+  const bool f32_tiles = o.dtype == MX_F32 && (fmt == MX_E3M2 || fmt == MX_E2M3) && C % 128 == 0;
+  e = o.dtype == MX_BF16 ? mx::launch_quantize_tile(a) : f32_tiles ? mx::launch_quantize_tile_f32(a)
+                                                                   : mx::launch_quantize_dual(a);
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
 }
 

@@ -257,6 +257,54 @@ quantize_tile_cols_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
 }
 
 
+// The producer warp of the kernels below.  Tiles are dealt out at run time: an SM's share of the
+// memory system's bandwidth varies (with 128 x 256 tiles split evenly, 14 per CTA, the slowest of
+// 147 CTAs took 95 k cycles and the median 79 k: 8192 x 8192 BF16 -> E4M3 in 51.3 us; dealt out, 47.0),
+// so a CTA's first tile is its own index and every further one comes from the launch's counter.  The
+// tile a stage holds is written beside the barriers before the stage is armed; a number past the
+// last tile tells the readers to stop.  Barriers: "stage s has landed" at bar0 + 8 s, "stage s has
+// been read" at bar0 + 8 (STAGES + s); tile numbers at tile_id0 + 4 s.  A tile is BOXES boxes of 128
+// rows x 128 bytes (box_cols elements) side by side.
+template <uint32_t STAGES, uint32_t BOXES>
+__device__ __forceinline__ void tile_producer(const CUtensorMap* tmap, uint32_t base, uint32_t bar0, uint32_t tile_id0,
+                                              uint32_t box_cols, uint32_t tiles_c, uint32_t num_tiles,
+                                              uint32_t sched_slot, uint32_t lane) {
+  constexpr uint32_t kBytes = BOXES * kBoxBytes;
+  unsigned int* sched = g_tile_sched + 2 * sched_slot;
+  for (uint32_t it = 0;; ++it) {
+    const uint32_t stage = it % STAGES, use = it / STAGES;
+    if (use > 0 && !tile_wait(bar0 + 8 * (STAGES + stage), (use - 1) & 1u)) {  // its readers of the round before
+      if (lane == 0) atomicCAS(&g_tile_status, 0u, 2u);
+      break;
+    }
+    uint32_t t = blockIdx.x;
+    if (it > 0) {
+      if (lane == 0) t = gridDim.x + atomicAdd(&sched[0], 1u);
+      t = __shfl_sync(0xFFFFFFFFu, t, 0);
+    }
+    if (lane == 0) {
+      const uint32_t bar = bar0 + 8 * stage;
+      asm volatile("st.shared.u32 [%0], %1;" ::"r"(tile_id0 + 4 * stage), "r"(t) : "memory");
+      if (t < num_tiles) {
+        const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+        asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kBytes) : "memory");
+        const uint32_t dst = base + stage * kBytes;
+        for (uint32_t b = 0; b < BOXES; ++b)
+          tma_load_2d(dst + b * kBoxBytes, tmap, (int)((tc * BOXES + b) * box_cols), (int)(tr * kTileRows), bar);
+      } else {
+        asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");  // nothing will land: complete the phase
+      }
+    }
+    __syncwarp();
+    if (t >= num_tiles) break;
+  }
+  // this CTA asks for no more tiles: count it; the last one leaves the slot as it found it
+  if (lane == 0) {
+    __threadfence();
+    if (atomicInc(&sched[1], gridDim.x - 1u) == gridDim.x - 1u) atomicExch(&sched[0], 0u);
+  }
+}
+
 // ---------------------------------------------------------------------------------------------
 // Both passes, no meeting of warps.  Nothing is gathered across warps before it is written: every
 // warp converts its share of a tile straight out of the (read-only) stage and writes whole 32-byte
@@ -319,46 +367,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
   const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
 
   if (warp == kTdWarps) {
-    // ------------------------------- producer -------------------------------
-    // Tiles are dealt out at run time: an SM's share of the memory system's bandwidth varies (with
-    // 128 x 256 tiles split evenly, 14 per CTA, the slowest of 147 CTAs took 95 k cycles and the
-    // median 79 k: 8192 x 8192 in 51.3 us; dealt out, 47.0 us), so a CTA's first
-    // tile is its own index and every further one comes from a counter.  The tile a stage holds is
-    // written beside the barriers before the stage is armed; a number past the last tile tells the
-    // readers to stop.
-    unsigned int* sched = g_tile_sched + 2 * sched_slot;
-    for (uint32_t it = 0;; ++it) {
-      const uint32_t stage = it % kStages, use = it / kStages;
-      if (use > 0 && !tile_wait(bar0 + 8 * (kStages + stage), (use - 1) & 1u)) {  // its readers of the round before
-        if (lane == 0) atomicCAS(&g_tile_status, 0u, 2u);
-        break;
-      }
-      uint32_t t = blockIdx.x;
-      if (it > 0) {
-        if (lane == 0) t = gridDim.x + atomicAdd(&sched[0], 1u);
-        t = __shfl_sync(0xFFFFFFFFu, t, 0);
-      }
-      if (lane == 0) {
-        const uint32_t bar = bar0 + 8 * stage;
-        asm volatile("st.shared.u32 [%0], %1;" ::"r"(tile_id0 + 4 * stage), "r"(t) : "memory");
-        if (t < num_tiles) {
-          const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
-          asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTdTileBytes) : "memory");
-          const uint32_t dst = base + stage * kTdTileBytes;
-          for (uint32_t b = 0; b < kTdBoxes; ++b)
-            tma_load_2d(dst + b * kBoxBytes, &tmap_in, (int)(tc * kTdCols + 64u * b), (int)(tr * kTileRows), bar);
-        } else {
-          asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");  // nothing will land: complete the phase
-        }
-      }
-      __syncwarp();
-      if (t >= num_tiles) break;
-    }
-    // this CTA asks for no more tiles: count it; the last one leaves the slot as it found it
-    if (lane == 0) {
-      __threadfence();
-      if (atomicInc(&sched[1], gridDim.x - 1u) == gridDim.x - 1u) atomicExch(&sched[0], 0u);
-    }
+    tile_producer<kStages, kTdBoxes>(&tmap_in, base, bar0, tile_id0, 64u, tiles_c, num_tiles, sched_slot, lane);
     return;
   }
 
@@ -588,6 +597,199 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
   }
 }
 
+// ---------------------------------------------------------------------------------------------
+// The same for FP32 input and 6-bit codes (configuration 4's tensors, whose register kernel needs
+// six tile-times on a one-wave tensor where 4.6 would do).  An FP32 box row of 128 bytes is exactly
+// one MX block, so a tile is four boxes side by side -- 128 x 128 elements, 64 KB, a row's four
+// blocks = one 96-byte run --, three stages, one CTA per SM:
+//   warps 0-3   rows: lane = one tile row, four blocks (eight 16-byte loads each)
+//   warps 4-11  columns: warp w the w-th sixteenth... of the tile's 128 columns: lane = (column
+//               lane % 16 of the warp's 16, row group 2 step + lane / 16), two steps; the two lanes of
+//               a column then hold row groups {0, 2} and {1, 3} and pass eight words to each other
+//               so that one writes sectors 0 and 1 of the column's 96-byte run and the other sector 2
+//   warp 12     producer
+// Rows convert 128 elements per lane and tile, columns 64: the twelve warps carry equal shares.
+// ---------------------------------------------------------------------------------------------
+constexpr uint32_t kTfBoxes = 4;
+constexpr uint32_t kTfWarps = 12;
+constexpr int kTileF32Threads = 32 * (kTfWarps + 1);
+constexpr uint32_t kTfTileBytes = kTfBoxes * kBoxBytes;
+constexpr uint32_t kTfCols = 32 * kTfBoxes;
+constexpr uint32_t kTfStages = 3;
+constexpr uint32_t kTfSmem = kTfStages * kTfTileBytes + 2 * kTfStages * 8 + kTfStages * 4 + 4 + 1024;
+
+template <int FMT, int ROUND, int LAYOUT>
+__global__ void __launch_bounds__(kTileF32Threads, 1)
+quantize_tile_dual_f32_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
+                              uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
+                              uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
+                              uint32_t num_tiles, uint32_t sched_slot) {
+  static_assert(FmtTraits<FMT>::bits == 6, "6-bit codes");
+  constexpr uint32_t kStages = kTfStages;
+  constexpr uint32_t kBpb = 24;
+  extern __shared__ uint8_t tile_smem_raw[];
+  const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
+  const uint32_t bar0 = base + kStages * kTfTileBytes;      // landed[s] at 8 s, read[s] at 8 (kStages + s)
+  const uint32_t tile_id0 = bar0 + 16 * kStages;
+  const uint32_t tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+  if (tid == 0) {
+    for (uint32_t s = 0; s < kStages; ++s) {
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kTfWarps) : "memory");
+    }
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_in)) : "memory");
+  }
+  __syncthreads();
+  pdl_prologue();
+  const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;
+  const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
+  if (warp == kTfWarps) {
+    tile_producer<kStages, kTfBoxes>(&tmap_in, base, bar0, tile_id0, 32u, tiles_c, num_tiles, sched_slot, lane);
+    return;
+  }
+#pragma unroll 1
+  for (uint32_t it = 0;; ++it) {
+    const uint32_t stage = it % kStages, parity = (it / kStages) & 1u;
+    if (!tile_wait(bar0 + 8 * stage, parity)) {
+      if (lane == 0) atomicCAS(&g_tile_status, 0u, 1u);
+      return;
+    }
+    uint32_t t;
+    asm volatile("ld.shared.u32 %0, [%1];" : "=r"(t) : "r"(tile_id0 + 4 * stage) : "memory");
+    if (t >= num_tiles) return;  // no tile left
+    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
+    const uint32_t tile_base = base + stage * kTfTileBytes;
+    const uint32_t row0 = tr * kTileRows, col0 = tc * kTfCols;
+    if (warp < 4u) {
+      const uint32_t r = warp * 32u + lane;
+      uint32_t run[24];
+      uint32_t scale_word = 0;
+#pragma unroll
+      for (uint32_t q = 0; q < 4; ++q) {  // block q of the row = row r of box q
+        const uint32_t box = tile_base + q * kBoxBytes;
+        uint32_t u[32];
+#pragma unroll
+        for (uint32_t i = 0; i < 8; ++i) {
+          uint32_t v0, v1, v2, v3;
+          asm volatile("ld.shared.v4.b32 {%0, %1, %2, %3}, [%4];"
+                       : "=r"(v0), "=r"(v1), "=r"(v2), "=r"(v3) : "r"(box_chunk(box, r, i)));
+          u[4 * i] = v0; u[4 * i + 1] = v1; u[4 * i + 2] = v2; u[4 * i + 3] = v3;
+        }
+        float m[16];
+#pragma unroll
+        for (int i = 0; i < 16; ++i) m[i] = absmax_nan(__uint_as_float(u[2 * i]), __uint_as_float(u[2 * i + 1]));
+#pragma unroll
+        for (int n = 8; n >= 1; n >>= 1)
+#pragma unroll
+          for (int i = 0; i < n; ++i) m[i] = absmax_nan(m[2 * i], m[2 * i + 1]);
+        const BlockScale s = block_scale<FMT>(m[0]);
+        scale_word |= s.byte << (8 * q);
+        uint32_t cw[8], o[6];
+#pragma unroll
+        for (int g = 0; g < 4; ++g) {
+          float x[8];
+#pragma unroll
+          for (int i = 0; i < 8; ++i) x[i] = __uint_as_float(u[8 * g + i]);
+          cast8<FMT, ROUND>(x, s, cw[2 * g], cw[2 * g + 1]);
+        }
+        pack6_words(cw, o);
+#pragma unroll
+        for (int i = 0; i < 6; ++i) run[6 * q + i] = o[i];
+      }
+      const uint32_t row = row0 + r, kb0 = tc * 4u;
+      uint8_t* dst = elems_row + (size_t)row * row_out_bytes + (size_t)kb0 * kBpb;
+      store_run<24>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
+      // four adjacent bytes in either layout (kb0 % 4 == 0)
+      *reinterpret_cast<uint32_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = scale_word;
+    } else {
+      const uint32_t cwarp = warp - 4u, hi = lane >> 4;
+      const uint32_t w = 16u * (cwarp & 1u) + (lane & 15u);        // column (= word) inside the box
+      const uint32_t box = tile_base + (cwarp >> 1) * kBoxBytes;
+      const uint32_t c = w >> 2, wofs = (w & 3u) * 4u;
+      uint32_t o[2][6];   // [step][word]: row group 2 step + hi
+      uint32_t sb = 0;    // this lane's two scale bytes at their positions in the column's word
+#pragma unroll
+      for (uint32_t step = 0; step < 2; ++step) {
+        const uint32_t g = 2u * step + hi;
+        uint32_t raw[kBlock][1];
+#pragma unroll
+        for (uint32_t k = 0; k < kBlock; ++k)
+          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, g * kBlock + k, c) + wofs));
+        float amax[1];
+        column_amax<MX_F32, 1>(raw, amax);
+        const BlockScale s = block_scale<FMT>(amax[0]);
+        uint32_t cw[8];
+        column_cast<FMT, ROUND, MX_F32, 1>(raw, 0, s, cw);
+        pack6_words(cw, o[step]);
+        sb |= s.byte << (8 * g);
+      }
+      // the run's 24 words: groups 0 and 2 in lane hi = 0 (o[0], o[1]), groups 1 and 3 in lane hi = 1.
+      // sector 0 = g0[0..5] g1[0..1], sector 1 = g1[2..5] g2[0..3] (both written by hi = 0),
+      // sector 2 = g2[4..5] g3[0..5] (written by hi = 1)
+      uint32_t p1[6], p2[2];
+#pragma unroll
+      for (int i = 0; i < 6; ++i) p1[i] = __shfl_xor_sync(0xFFFFFFFFu, o[0][i], 16);       // hi = 0 receives g1
+#pragma unroll
+      for (int i = 0; i < 2; ++i) p2[i] = __shfl_xor_sync(0xFFFFFFFFu, o[1][4 + i], 16);   // hi = 1 receives g2[4..5]
+      const uint32_t col = col0 + (cwarp >> 1) * 32u + w, kb = tr * 4u;
+      uint8_t* run0 = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
+      const bool wide = (reinterpret_cast<uintptr_t>(run0) & 31u) == 0;
+      if (hi == 0) {
+        const uint32_t run[16] = {o[0][0], o[0][1], o[0][2], o[0][3], o[0][4], o[0][5], p1[0], p1[1],
+                                  p1[2], p1[3], p1[4], p1[5], o[1][0], o[1][1], o[1][2], o[1][3]};
+        store_run<16>(run0, run, wide);
+      } else {
+        const uint32_t run[8] = {p2[0], p2[1], o[1][0], o[1][1], o[1][2], o[1][3], o[1][4], o[1][5]};
+        store_run<8>(run0 + 64, run, wide);
+      }
+      const uint32_t word = sb | __shfl_xor_sync(0xFFFFFFFFu, sb, 16);
+      if (hi == 1) *reinterpret_cast<uint32_t*>(scales_col + scale_offset<LAYOUT>(col, kb, kb_col)) = word;
+    }
+    __syncwarp();
+    if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar0 + 8 * (kStages + stage)) : "memory");
+  }
+}
+
+template <int FMT, int ROUND, int LAYOUT>
+cudaError_t launch_tile_f32_t(const DualArgs& a) {
+  cudaError_t e;
+  EncodeTiledFn fn = encode_fn(&e);
+  if (!fn) return e;
+  CUtensorMap map;
+  const cuuint64_t dims[2] = {(cuuint64_t)a.C, (cuuint64_t)a.R};
+  const cuuint64_t strides[1] = {(cuuint64_t)a.C * 4};
+  const cuuint32_t box[2] = {32, kTileRows};
+  if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, a.in, dims, strides, box,
+                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
+    return cudaErrorInvalidValue;
+  static bool attr_set[64] = {false};
+  int dev = 0;
+  e = cudaGetDevice(&dev);
+  if (e != cudaSuccess) return e;
+  auto kernel = quantize_tile_dual_f32_kernel<FMT, ROUND, LAYOUT>;
+  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
+    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)kTfSmem);
+    if (e != cudaSuccess) return e;
+    if (dev >= 0 && dev < 64) attr_set[dev] = true;
+  }
+  const uint32_t tiles_r = (uint32_t)(a.R / kTileRows), tiles_c = (uint32_t)(a.C / kTfCols);
+  const uint32_t num_tiles = tiles_r * tiles_c;
+  const uint32_t grid = num_tiles < (uint32_t)a.sm_count ? num_tiles : (uint32_t)a.sm_count;
+  return launch_pdl(kernel, dim3(grid), dim3(kTileF32Threads), kTfSmem, a.stream, map, a.elems_row, a.scales_row,
+                    a.elems_col, a.scales_col, (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles, next_sched_slot());
+}
+
+template <int FMT>
+cudaError_t dispatch_tile_f32(const DualArgs& a) {
+  if (a.rounding == MX_RHAZ)
+    return a.layout == MX_SCALES_LINEAR ? launch_tile_f32_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
+                                        : launch_tile_f32_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_f32_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
+                                      : launch_tile_f32_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
+}
+
 template <int FMT, int ROUND, int LAYOUT>
 cudaError_t launch_tile_dual_t(const DualArgs& a) {
   cudaError_t e;
@@ -684,6 +886,16 @@ cudaError_t launch_quantize_tile(const DualArgs& a) {
     case MX_E2M3: return dispatch_tile_dual<MX_E2M3>(a);
     case MX_E2M1: return dispatch_tile_dual<MX_E2M1>(a);
     default: return dispatch_tile_dual<MX_INT8>(a);
+  }
+}
+
+// FP32 input, 6-bit codes, R and C multiples of 128.
+cudaError_t launch_quantize_tile_f32(const DualArgs& a) {
+  if (a.dtype != MX_F32 || !a.elems_row || !a.elems_col) return cudaErrorInvalidValue;
+  switch (a.fmt) {
+    case MX_E3M2: return dispatch_tile_f32<MX_E3M2>(a);
+    case MX_E2M3: return dispatch_tile_f32<MX_E2M3>(a);
+    default: return cudaErrorInvalidValue;
   }
 }
 

@@ -149,16 +149,17 @@ def test_middle_axis_of_3d_tensor(fmt):
     _assert_same_bytes(s, ws, "scales")
 
 
-@pytest.mark.parametrize("dtype,R,C", [(torch.float32, 384, 320), (torch.bfloat16, 256, 384),
-                                       (torch.bfloat16, 384, 512), (torch.bfloat16, 128, 256),
-                                       (torch.bfloat16, 640, 1280)],
-                         ids=["f32", "bf16", "bf16-wide-tiles", "bf16-one-wide-tile", "bf16-many-wide-tiles"])
+@pytest.mark.parametrize("dtype,R,C", [(torch.float32, 384, 320), (torch.float32, 256, 384), (torch.float32, 1280, 640),
+                                       (torch.bfloat16, 256, 384), (torch.bfloat16, 384, 512),
+                                       (torch.bfloat16, 128, 256), (torch.bfloat16, 640, 1280)],
+                         ids=["f32", "f32-whole-tiles", "f32-many-tiles", "bf16", "bf16-4-tiles-wide", "bf16-one-row-of-tiles",
+                              "bf16-many-tiles"])
 @pytest.mark.parametrize("fmt", FMTS)
 def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype, R, C):
     """mx_quantize_dual reads the tensor once and must write exactly the two tensors that
     quantizing along axis 1 and along axis 0 give (checked against the oracle, not against
-    mx_quantize).  BF16 tensors whose width is a multiple of 256 take the 8-bit formats through the
-    kernel with 128 x 256 tiles, the other widths and formats through the general tile kernel."""
+    mx_quantize).  BF16 tensors go through the tile kernel (128 x 128 tiles), FP32 tensors through
+    the register kernel except 6-bit codes of whole 128 x 128 tiles, which have a tile kernel too."""
     x = inputs.adversarial("cuda", rows=R, cols=C, dtype=dtype, seed=41 + fmt)
     xin = to_oracle_input(x)
     for rounding, layout in ((mx.MX_RNE, mx.MX_SCALES_SWIZZLED), (mx.MX_RHAZ, mx.MX_SCALES_LINEAR)):
