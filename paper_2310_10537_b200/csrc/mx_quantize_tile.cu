@@ -17,20 +17,22 @@
 // column's 32 lanes always hit 32 different banks.  Every mbarrier wait is bounded: when one runs
 // out the CTA records it in a status word and leaves.
 //
-// Two kernels:
-//   quantize_tile_dual_kernel      both outputs (mx_quantize_dual), every format.  No meeting of warps:
-//                              every warp writes whole 32-byte sectors by itself (sub-byte codes:
-//                              lanes exchange part sectors by shuffle), a producer warp refills a
-//                              stage when its readers have released it, tiles are dealt out at run
-//                              time.  8192 x 8192: E4M3 46.8 us, E3M2 44.0, E2M1 34.5 (0.89 / 0.83 /
-//                              0.91 of the copy bandwidth on in + 2 x out bytes).
-//   quantize_tile_cols_kernel  the column-block tensor alone, 6-bit codes (mx_quantize along axis 0
-//                              of whole-tile tensors, where it beats the register kernels): all
-//                              eight warps convert word columns, the codes are parked in shared
-//                              memory and leave as whole sectors after a meeting of the warps.
-// (The second kernel used to do both passes -- warps 0-3 rows, warps 4-7 columns, a CTA barrier per
-// tile -- and measured 53 / 47 / 41 us on 8192 x 8192 for E4M3 / E3M2 / E2M1; timing-only builds of
-// it: copies alone 22 us, both passes without their stores 33, one pass with its stores 35.)
+// The kernels (no meeting of warps in any of them: every warp writes whole 32-byte sectors by
+// itself -- sub-byte codes: lanes exchange part sectors by shuffle --, a producer warp refills a
+// stage when its readers have released it, tiles are dealt out at run time):
+//   quantize_tile_dual_kernel      BF16 input, every format, both outputs (mx_quantize_dual).
+//                                  8192 x 8192: E4M3 46.8 us, E3M2 44.0, E2M1 34.5 (0.89 / 0.83 /
+//                                  0.91 of the copy bandwidth on in + 2 x out bytes).  With its
+//                                  row warps idle it also serves mx_quantize along axis 0 for the
+//                                  6-bit formats (whole-tile tensors; 4096 x 16384: 30.2-32 us
+//                                  against 35 for the register kernel).
+//   quantize_tile_dual_f32_kernel  FP32 input, 6-bit codes, both outputs: 8192 x 8192 in 56.9 us
+//                                  (the copy bandwidth).
+// (A first tile kernel -- 256 threads, warps 0-3 rows, warps 4-7 columns with the sub-byte codes
+// parked in shared memory, a CTA barrier per tile, tiles split evenly -- measured 53 / 47 / 41 us
+// on 8192 x 8192 BF16 for E4M3 / E3M2 / E2M1 and 32.3 us in its column-only form on 4096 x 16384;
+// timing-only builds of it: copies alone 22 us, both passes without their stores 33, one pass with
+// its stores 35.)
 #include <atomic>
 
 #include "mx_device.cuh"
@@ -42,10 +44,8 @@ namespace mx {
 
 namespace {
 
-constexpr int kTileThreads = 256;
 constexpr uint32_t kTileRows = 128;
 constexpr uint32_t kBoxBytes = kTileRows * 128;   // one TMA box: 128 rows x 128 bytes
-constexpr uint32_t kTileBytes = 2 * kBoxBytes;    // a tile: two boxes side by side (256 bytes per row)
 constexpr long long kTileSpinLimit = 2000000000LL;
 
 __device__ unsigned int g_tile_status;  // 1: a tile never arrived (bounded wait ran out)
@@ -61,21 +61,6 @@ inline uint32_t next_sched_slot() {
   static std::atomic<uint32_t> next{0};
   return next.fetch_add(1, std::memory_order_relaxed) % kSchedSlots;
 }
-
-template <int FMT> struct TileCfg {
-  static constexpr int bits = FmtTraits<FMT>::bits;
-  static constexpr uint32_t kBpb = kBlock * bits / 8;                   // bytes of one block of codes
-  static constexpr uint32_t kCols = 128;                                // columns of a tile (256 bytes of BF16)
-  static constexpr uint32_t kStages = 3;
-  // column codes of sub-byte formats: per column its four blocks; the pad makes the stores of 32
-  // lanes (one slot apart) conflict-free: 26 words for 8-byte stores, 20 words for 16-byte stores
-  static constexpr uint32_t kColPitch = 4 * kBpb + (bits == 6 ? 8 : 16);
-  static constexpr uint32_t kStageCodes = bits != 8 ? kCols * kColPitch : 0;
-  static constexpr uint32_t kOffCodes = kStages * kTileBytes;
-  static constexpr uint32_t kOffScales = kOffCodes + kStageCodes;       // a column's four scale bytes
-  static constexpr uint32_t kOffBar = kOffScales + kCols * 4;
-  static constexpr uint32_t kSmem = kOffBar + kStages * 8 + 1024;       // + alignment slack
-};
 
 __device__ __forceinline__ uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -105,157 +90,6 @@ __device__ __forceinline__ bool tile_wait(uint32_t bar, uint32_t parity) {
 __device__ __forceinline__ uint32_t box_chunk(uint32_t box_base, uint32_t r, uint32_t c) {
   return box_base + r * 128u + ((c ^ (r & 7u)) << 4);
 }
-
-template <int FMT, int ROUND, int LAYOUT>
-__global__ void __launch_bounds__(kTileThreads, 2)
-quantize_tile_cols_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_col,
-                          uint8_t* __restrict__ scales_col, uint32_t R, uint32_t C, uint32_t tiles_c,
-                          uint32_t num_tiles) {
-  using cfg = TileCfg<FMT>;
-  constexpr int DTYPE = MX_BF16;
-  constexpr int bits = cfg::bits;
-  constexpr uint32_t kBpb = cfg::kBpb;
-  constexpr uint32_t kBoxCols = cfg::kCols / 2;  // columns of one box
-  extern __shared__ uint8_t tile_smem_raw[];
-  const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
-  uint8_t* gen = tile_smem_raw + (base - smem_addr(tile_smem_raw));
-  const uint32_t bar0 = base + cfg::kOffBar;
-  const uint32_t tid = threadIdx.x, lane = tid & 31;
-
-  if (tid == 0) {
-    for (uint32_t s = 0; s < cfg::kStages; ++s)
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
-    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
-    asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
-    asm volatile("prefetch.tensormap [%0];" ::"l"(reinterpret_cast<uint64_t>(&tmap_in)) : "memory");
-  }
-  __syncthreads();
-  pdl_prologue();
-
-  auto issue = [&](uint32_t t, uint32_t stage) {  // thread 0: both boxes of tile t into `stage`
-    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
-    const uint32_t bar = bar0 + 8 * stage;
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(kTileBytes) : "memory");
-    const uint32_t dst = base + stage * kTileBytes;
-    tma_load_2d(dst, &tmap_in, (int)(tc * cfg::kCols), (int)(tr * kTileRows), bar);
-    tma_load_2d(dst + kBoxBytes, &tmap_in, (int)(tc * cfg::kCols + kBoxCols), (int)(tr * kTileRows), bar);
-  };
-  if (tid == 0) {
-#pragma unroll 1
-    for (uint32_t k = 0; k + 1 < cfg::kStages; ++k) {
-      const uint32_t t = blockIdx.x + k * gridDim.x;
-      if (t < num_tiles) issue(t, k);
-    }
-  }
-
-  const uint32_t kb_col = R / kBlock;  // blocks per output row
-  const size_t col_out_bytes = (size_t)kb_col * kBpb;
-  uint32_t it = 0;
-#pragma unroll 1
-  for (uint32_t t = blockIdx.x; t < num_tiles; t += gridDim.x, ++it) {
-    const uint32_t stage = it % cfg::kStages, parity = (it / cfg::kStages) & 1u;
-    if (tid == 0) {  // the stage that iteration it - 1 has finished with takes the tile kStages - 1 ahead
-      const uint32_t tn = t + (cfg::kStages - 1) * gridDim.x;
-      if (tn < num_tiles) issue(tn, (it + cfg::kStages - 1) % cfg::kStages);
-    }
-    if (!tile_wait(bar0 + 8 * stage, parity)) {
-      if (lane == 0) atomicCAS(&g_tile_status, 0u, 1u);
-      return;
-    }
-    const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
-    const uint32_t tile_base = base + stage * kTileBytes;
-    const uint32_t col0 = tc * cfg::kCols;
-
-    // ----------------------------- column pass -----------------------------
-    {
-      constexpr uint32_t kColThreads = kTileThreads;  // all eight warps
-      constexpr int kWordCols = 2;   // columns in one 32-bit word
-      const uint32_t ct = tid;
-      uint8_t* codes_smem = gen + cfg::kOffCodes;
-      uint8_t* scale_smem = gen + cfg::kOffScales;
-      // 64 word columns x 4 row groups = 256 units of 32 rows x one word
-#pragma unroll 1
-      for (uint32_t u = ct; u < 256; u += kColThreads) {
-        const uint32_t w = u & 63u, g = u >> 6;
-        const uint32_t box = tile_base + (w >> 5) * kBoxBytes;
-        const uint32_t c = (w & 31u) >> 2, wofs = (w & 3u) * 4u;
-        uint32_t raw[kBlock][1];
-#pragma unroll
-        for (uint32_t k = 0; k < kBlock; ++k) {
-          const uint32_t r = g * kBlock + k;
-          asm volatile("ld.shared.b32 %0, [%1];" : "=r"(raw[k][0]) : "r"(box_chunk(box, r, c) + wofs));
-        }
-        float amax[kWordCols];
-        column_amax<DTYPE, kWordCols>(raw, amax);
-        const uint32_t kb = tr * 4 + g;   // block of the output row
-#pragma unroll
-        for (int cc = 0; cc < kWordCols; ++cc) {
-          const uint32_t col = col0 + w * kWordCols + cc;
-          const BlockScale s = block_scale<FMT>(amax[cc]);
-          uint32_t cw[8];
-          column_cast<FMT, ROUND, DTYPE, kWordCols>(raw, cc, s, cw);
-          const bool live = col < C && kb < kb_col;
-          scale_smem[(w * kWordCols + cc) * 4 + g] = (uint8_t)s.byte;
-          if (bits == 8) {
-            if (live) {
-              uint8_t* dst = elems_col + (size_t)col * col_out_bytes + (size_t)kb * kBpb;
-              store_run<8>(dst, cw, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
-            }
-          } else {
-            // slot of column w * kWordCols + cc: the columns of one lane parity side by side, so that
-            // consecutive lanes are one slot apart
-            uint8_t* dst = codes_smem + ((uint32_t)cc * 64u + w) * cfg::kColPitch + g * kBpb;
-            if (bits == 4) {
-              *reinterpret_cast<uint4*>(dst) = make_uint4(cw[0], cw[2], cw[4], cw[6]);
-            } else {
-              uint64_t a, b, c6;
-              pack6(cw, a, b, c6);
-              uint2* d2 = reinterpret_cast<uint2*>(dst);
-              d2[0] = make_uint2((uint32_t)a, (uint32_t)(a >> 32));
-              d2[1] = make_uint2((uint32_t)b, (uint32_t)(b >> 32));
-              d2[2] = make_uint2((uint32_t)c6, (uint32_t)(c6 >> 32));
-            }
-          }
-        }
-      }
-      // the column warps meet (named barrier 1); then a column's four scale bytes leave as one word
-      // and, for the sub-byte formats, its run of four blocks as whole sectors where the tensor
-      // allows, consecutive threads on consecutive chunks
-      asm volatile("bar.sync 1, %0;" ::"r"(kColThreads) : "memory");
-      const uint32_t live_blocks = min(4u, kb_col - min(kb_col, tr * 4));
-      if (ct < cfg::kCols && col0 + ct < C) {
-        uint8_t* sp = scales_col + scale_offset<LAYOUT>(col0 + ct, tr * 4, kb_col);
-        if (live_blocks == 4 && (reinterpret_cast<uintptr_t>(sp) & 3u) == 0) {
-          *reinterpret_cast<uint32_t*>(sp) = *reinterpret_cast<const uint32_t*>(scale_smem + ct * 4);
-        } else {
-          for (uint32_t g = 0; g < live_blocks; ++g)
-            scales_col[scale_offset<LAYOUT>(col0 + ct, tr * 4 + g, kb_col)] = scale_smem[ct * 4 + g];
-        }
-      }
-      if (bits != 8) {
-        const uint32_t seg = live_blocks * kBpb;  // bytes of a column's run that exist in the output
-        const bool wide = ((reinterpret_cast<uintptr_t>(elems_col) | col_out_bytes) & 31u) == 0 && seg % 32 == 0;
-        const uint32_t cb = wide ? 32u : 8u, nch = seg / cb;
-        for (uint32_t i = ct; i < cfg::kCols * nch; i += kColThreads) {
-          const uint32_t cl = i / nch, ch = i - cl * nch;
-          if (col0 + cl >= C) continue;
-          const uint32_t slot = (cl & 1u) * 64u + (cl >> 1);
-          const uint2* src = reinterpret_cast<const uint2*>(codes_smem + slot * cfg::kColPitch + ch * cb);
-          uint8_t* gdst = elems_col + (size_t)(col0 + cl) * col_out_bytes + (size_t)(tr * 4) * kBpb + ch * cb;
-          if (wide) {
-            const uint2 a = src[0], b = src[1], c2 = src[2], d = src[3];
-            const uint32_t v[8] = {a.x, a.y, b.x, b.y, c2.x, c2.y, d.x, d.y};
-            st_32(gdst, v);
-          } else {
-            *reinterpret_cast<uint2*>(gdst) = src[0];
-          }
-        }
-      }
-    }
-    __syncthreads();  // everyone is done with this stage (and with the parked codes) before it is refilled
-  }
-}
-
 
 // The producer warp of the kernels below.  Tiles are dealt out at run time: an SM's share of the
 // memory system's bandwidth varies (with 128 x 256 tiles split evenly, 14 per CTA, the slowest of
@@ -336,7 +170,7 @@ constexpr uint32_t kTdTileBytes = kTdBoxes * kBoxBytes;
 constexpr uint32_t kTdCols = 64 * kTdBoxes;
 constexpr int kTdCtasPerSm = kTdBoxes == 2 ? 2 : 1;
 
-template <int FMT, int ROUND, int LAYOUT>
+template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY = false>
 __global__ void __launch_bounds__(kTileDualThreads, kTdCtasPerSm)
 quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* __restrict__ elems_row,
                       uint8_t* __restrict__ scales_row, uint8_t* __restrict__ elems_col,
@@ -344,8 +178,10 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
                       uint32_t num_tiles, uint32_t sched_slot) {
   constexpr int bits = FmtTraits<FMT>::bits;
   static_assert(bits == 8 || kTdBoxes == 2, "sub-byte codes: 128 x 128 tiles (their lane maps assume two boxes)");
+  static_assert(!COLS_ONLY || bits == 6, "the column-only form serves the 6-bit formats");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
+  constexpr uint32_t kWarps = kTdWarps;  // reader warps
   constexpr uint32_t kBpb = kBlock * bits / 8;  // 32 or 16 bytes of codes per block
   extern __shared__ uint8_t tile_smem_raw[];
   const uint32_t base = (smem_addr(tile_smem_raw) + 1023u) & ~1023u;
@@ -355,7 +191,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
   if (tid == 0) {
     for (uint32_t s = 0; s < kStages; ++s) {
       asm volatile("mbarrier.init.shared::cta.b64 [%0], 1;" ::"r"(bar0 + 8 * s) : "memory");
-      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kTdWarps) : "memory");
+      asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar0 + 8 * (kStages + s)), "r"(kWarps) : "memory");
     }
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
     asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -366,7 +202,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
   const uint32_t kb_row = C / kBlock, kb_col = R / kBlock;
   const size_t row_out_bytes = (size_t)kb_row * kBpb, col_out_bytes = (size_t)kb_col * kBpb;
 
-  if (warp == kTdWarps) {
+  if (warp == kWarps) {
     tile_producer<kStages, kTdBoxes>(&tmap_in, base, bar0, tile_id0, 64u, tiles_c, num_tiles, sched_slot, lane);
     return;
   }
@@ -505,6 +341,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
       // of both columns and pass eight words to each other so that one writes sectors 0 and 1 of
       // each column and the other sector 2.  Both roles convert 128 elements per lane and tile.
       if (warp >= 4u) {
+        if constexpr (!COLS_ONLY) {
         const uint32_t r = (warp - 4u) * 32u + lane;
         uint32_t run[24];
         uint32_t scale_word = 0;
@@ -537,6 +374,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
         store_run<24>(dst, run, (reinterpret_cast<uintptr_t>(dst) & 31u) == 0);
         // four adjacent bytes in either layout (kb0 % 4 == 0)
         *reinterpret_cast<uint32_t*>(scales_row + scale_offset<LAYOUT>(row, kb0, kb_row)) = scale_word;
+        }  // (COLS_ONLY: these warps only take part in the stage's barriers)
       } else {
         const uint32_t hi = lane >> 4;
         const uint32_t w = 16u * (warp & 1u) + (lane & 15u);        // word column inside the box
@@ -790,7 +628,7 @@ cudaError_t dispatch_tile_f32(const DualArgs& a) {
                                       : launch_tile_f32_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
 }
 
-template <int FMT, int ROUND, int LAYOUT>
+template <int FMT, int ROUND, int LAYOUT, bool COLS_ONLY = false>
 cudaError_t launch_tile_dual_t(const DualArgs& a) {
   cudaError_t e;
   EncodeTiledFn fn = encode_fn(&e);
@@ -802,12 +640,13 @@ cudaError_t launch_tile_dual_t(const DualArgs& a) {
   if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
                      CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
     return cudaErrorInvalidValue;
-  constexpr uint32_t smem = 3 * kTdTileBytes + 6 * 8 + 3 * 4 + 4 + 1024;  // stages, barriers, tile numbers, alignment slack
+  constexpr uint32_t kSt = 3;
+  constexpr uint32_t smem = kSt * kTdTileBytes + 2 * kSt * 8 + kSt * 4 + 4 + 1024;  // stages, barriers, tile numbers, alignment slack
   static bool attr_set[64] = {false};
   int dev = 0;
   e = cudaGetDevice(&dev);
   if (e != cudaSuccess) return e;
-  auto kernel = quantize_tile_dual_kernel<FMT, ROUND, LAYOUT>;
+  auto kernel = quantize_tile_dual_kernel<FMT, ROUND, LAYOUT, COLS_ONLY>;
   if (dev < 0 || dev >= 64 || !attr_set[dev]) {
     e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem);
     if (e != cudaSuccess) return e;
@@ -831,47 +670,14 @@ cudaError_t dispatch_tile_dual(const DualArgs& a) {
                                       : launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
 }
 
-template <int FMT, int ROUND, int LAYOUT>
-cudaError_t launch_tile_cols_t(const DualArgs& a) {
-  using cfg = TileCfg<FMT>;
-  cudaError_t e;
-  EncodeTiledFn fn = encode_fn(&e);
-  if (!fn) return e;
-  CUtensorMap map;
-  const cuuint64_t dims[2] = {(cuuint64_t)a.C, (cuuint64_t)a.R};
-  const cuuint64_t strides[1] = {(cuuint64_t)a.C * 2};
-  const cuuint32_t box[2] = {cfg::kCols / 2, kTileRows};
-  if (!encode_cached(fn, &map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, a.in, dims, strides, box,
-                     CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B))
-    return cudaErrorInvalidValue;
-  static bool attr_set[64] = {false};
-  int dev = 0;
-  e = cudaGetDevice(&dev);
-  if (e != cudaSuccess) return e;
-  auto kernel = quantize_tile_cols_kernel<FMT, ROUND, LAYOUT>;
-  if (dev < 0 || dev >= 64 || !attr_set[dev]) {
-    e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)cfg::kSmem);
-    if (e != cudaSuccess) return e;
-    if (dev >= 0 && dev < 64) attr_set[dev] = true;
-  }
-  const uint32_t tiles_r = (uint32_t)((a.R + kTileRows - 1) / kTileRows);
-  const uint32_t tiles_c = (uint32_t)((a.C + cfg::kCols - 1) / cfg::kCols);
-  const uint32_t num_tiles = tiles_r * tiles_c;
-  const uint32_t slots = 2u * (uint32_t)a.sm_count;  // two CTAs per SM
-  // an even share of tiles per CTA: the smallest grid that needs no more rounds than a full one
-  const uint32_t rounds = (num_tiles + slots - 1) / slots;
-  const uint32_t grid = (num_tiles + rounds - 1) / rounds;
-  return launch_pdl(kernel, dim3(grid), dim3(kTileThreads), cfg::kSmem, a.stream, map, a.elems_col, a.scales_col,
-                    (uint32_t)a.R, (uint32_t)a.C, tiles_c, num_tiles);
-}
-
+// The column-block tensor alone (the 6-bit formats): the same kernel with its row warps idle.
 template <int FMT>
 cudaError_t dispatch_tile_cols(const DualArgs& a) {
   if (a.rounding == MX_RHAZ)
-    return a.layout == MX_SCALES_LINEAR ? launch_tile_cols_t<FMT, MX_RHAZ, MX_SCALES_LINEAR>(a)
-                                        : launch_tile_cols_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED>(a);
-  return a.layout == MX_SCALES_LINEAR ? launch_tile_cols_t<FMT, MX_RNE, MX_SCALES_LINEAR>(a)
-                                      : launch_tile_cols_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
+    return a.layout == MX_SCALES_LINEAR ? launch_tile_dual_t<FMT, MX_RHAZ, MX_SCALES_LINEAR, true>(a)
+                                        : launch_tile_dual_t<FMT, MX_RHAZ, MX_SCALES_SWIZZLED, true>(a);
+  return a.layout == MX_SCALES_LINEAR ? launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_LINEAR, true>(a)
+                                      : launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_SWIZZLED, true>(a);
 }
 
 }  // namespace
