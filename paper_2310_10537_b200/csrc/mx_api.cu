@@ -178,10 +178,10 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
     e = cudaMemsetAsync(scales_out, 0, scales_bytes(v.rows, v.kblocks, o.layout), o.stream);
     if (e != cudaSuccess) return fail_cuda(e);
   }
-  // Axis 0 of a 2-D BF16 tensor of whole 128 x 128 tiles, 6-bit codes: the tile kernel's column pass
-  // (its copies in flight cost no registers; the register kernels are request-bound at the occupancy
-  // the 6-bit variant has)
-  if (o.dtype == MX_BF16 && fmt_bits((int)fmt) == 6 && v.outer == 1 && v.inner > 1 && v.L % 128 == 0 &&
+  // Axis 0 of a 2-D BF16 tensor of whole 128 x 128 tiles, 6- or 4-bit codes: the tile kernel's column
+  // pass (its copies in flight cost no registers; the register kernels are request-bound at the
+  // occupancy their staged variants have)
+  if (o.dtype == MX_BF16 && fmt_bits((int)fmt) != 8 && v.outer == 1 && v.inner > 1 && v.L % 128 == 0 &&
       v.inner % 128 == 0 && v.Lp == v.L) {
     mx::DualArgs d;
     d.in = in; d.elems_row = nullptr; d.scales_row = nullptr;

@@ -23,9 +23,9 @@
 //   quantize_tile_dual_kernel      BF16 input, every format, both outputs (mx_quantize_dual).
 //                                  8192 x 8192: E4M3 46.8 us, E3M2 44.0, E2M1 34.5 (0.89 / 0.83 /
 //                                  0.91 of the copy bandwidth on in + 2 x out bytes).  With its
-//                                  row warps idle it also serves mx_quantize along axis 0 for the
-//                                  6-bit formats (whole-tile tensors; 4096 x 16384: 30.2-32 us
-//                                  against 35 for the register kernel).
+//                                  Without its row pass it also serves mx_quantize along axis 0 for
+//                                  6- and 4-bit codes (whole-tile tensors; 4096 x 16384: 30.2 us
+//                                  against 35 for the 6-bit register kernel, 28.2 against 29.2 for 4-bit).
 //   quantize_tile_dual_f32_kernel  FP32 input, 6-bit codes, both outputs: 8192 x 8192 in 56.9 us
 //                                  (the copy bandwidth).
 // (A first tile kernel -- 256 threads, warps 0-3 rows, warps 4-7 columns with the sub-byte codes
@@ -178,7 +178,6 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
                       uint32_t num_tiles, uint32_t sched_slot) {
   constexpr int bits = FmtTraits<FMT>::bits;
   static_assert(bits == 8 || kTdBoxes == 2, "sub-byte codes: 128 x 128 tiles (their lane maps assume two boxes)");
-  static_assert(!COLS_ONLY || bits == 6, "the column-only form serves the 6-bit formats");
   constexpr int DTYPE = MX_BF16;
   constexpr uint32_t kStages = 3;
   constexpr uint32_t kWarps = kTdWarps;  // reader warps
@@ -221,7 +220,7 @@ quantize_tile_dual_kernel(const __grid_constant__ CUtensorMap tmap_in, uint8_t* 
     const uint32_t tr = t / tiles_c, tc = t - tr * tiles_c;
     const uint32_t tile_base = base + stage * kTdTileBytes;
     const uint32_t row0 = tr * kTileRows, col0 = tc * kTdCols;
-    if constexpr (bits != 6) {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
+    if constexpr (bits != 6 && !COLS_ONLY) {  // row pass: the two blocks of one row that lie in one box; a quarter-warp = 8 consecutive rows of a box
       constexpr uint32_t kRowsPerWarp = 32 / kTdBoxes;   // 16 or 8
       const uint32_t r = warp * kRowsPerWarp + (lane % kRowsPerWarp), h = lane / kRowsPerWarp;
       const uint32_t box = tile_base + h * kBoxBytes;
@@ -670,7 +669,7 @@ cudaError_t dispatch_tile_dual(const DualArgs& a) {
                                       : launch_tile_dual_t<FMT, MX_RNE, MX_SCALES_SWIZZLED>(a);
 }
 
-// The column-block tensor alone (the 6-bit formats): the same kernel with its row warps idle.
+// The column-block tensor alone (6- and 4-bit codes): the same kernel without its row pass (6-bit: the row warps idle).
 template <int FMT>
 cudaError_t dispatch_tile_cols(const DualArgs& a) {
   if (a.rounding == MX_RHAZ)
@@ -705,14 +704,16 @@ cudaError_t launch_quantize_tile_f32(const DualArgs& a) {
   }
 }
 
-// The column-block tensor alone ([C x R], blocks along axis 0 of X[R x C]) for the 6-bit formats:
+// The column-block tensor alone ([C x R], blocks along axis 0 of X[R x C]) for the sub-byte formats:
 // mx_quantize along axis 0 of a 2-D BF16 tensor of whole tiles, where it beats the register kernels
-// (measured on 4096 x 16384: 32.4 against 35.1 us; 8- and 4-bit codes are faster there).
+// (measured on 4096 x 16384: 6-bit 30.2 against 35.1 us, 4-bit 28.2 against 29.2; 8192 x 8192: 4-bit
+// 28.6 against 30.3; 8-bit codes are faster in the register kernel, 33.9 against 34.5).
 cudaError_t launch_quantize_tile_cols(const DualArgs& a) {
   if (a.dtype != MX_BF16 || !a.elems_col || !a.scales_col) return cudaErrorInvalidValue;
   switch (a.fmt) {
     case MX_E3M2: return dispatch_tile_cols<MX_E3M2>(a);
     case MX_E2M3: return dispatch_tile_cols<MX_E2M3>(a);
+    case MX_E2M1: return dispatch_tile_cols<MX_E2M1>(a);
     default: return cudaErrorInvalidValue;
   }
 }
