@@ -236,6 +236,39 @@ def test_dual_axis_at_sweep_size(fmt, rounding, dtype):
     assert torch.equal(er, e1) and torch.equal(sr, s1) and torch.equal(ec, e0) and torch.equal(sc, s0)
 
 
+def test_dual_axis_many_launches_on_two_streams():
+    """The tile kernels of mx_quantize_dual deal their tiles out at run time from per-launch counter
+    slots that the host hands out round-robin (256 of them) and the kernels leave at zero.  More
+    launches than slots, interleaved on two streams with different shapes, formats and input types:
+    every result equals the single-axis kernels' (which the other tests pin to the oracle)."""
+    cases = [(torch.bfloat16, 512, 1024, mx.MX_E4M3), (torch.bfloat16, 1280, 384, mx.MX_E2M1),
+             (torch.bfloat16, 256, 2048, mx.MX_E3M2), (torch.float32, 640, 768, mx.MX_E2M3)]
+    g = torch.Generator(device="cuda").manual_seed(99)
+    xs, want = [], []
+    for dt, R, C, fmt in cases:
+        x = (torch.randn((R, C), generator=g, device="cuda") * torch.exp(torch.randn((R, 1), generator=g, device="cuda"))).to(dt)
+        xs.append(x)
+        want.append((mx.mx_quantize(x, 1, fmt), mx.mx_quantize(x, 0, fmt)))
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    outs = [[mx.mx_quantize_dual(x, fmt) for (_, _, _, fmt), x in zip(cases, xs)] for _ in streams]
+    torch.cuda.synchronize()
+    for rep in range(90):                       # 90 x 4 cases x 2 streams = 720 launches
+        for si, st in enumerate(streams):
+            with torch.cuda.stream(st):
+                for ci, ((_, _, _, fmt), x) in enumerate(zip(cases, xs)):
+                    if rep % 30 == 29:          # poison the outputs now and then, so stale results cannot pass
+                        for pair in outs[si][ci]:
+                            for t in pair:
+                                t.fill_(0xA5)
+                    mx.mx_quantize_dual(x, fmt, out=outs[si][ci])
+    torch.cuda.synchronize()
+    for si in range(2):
+        for ci in range(len(cases)):
+            (er, sr), (ec, sc) = outs[si][ci]
+            (e1, s1), (e0, s0) = want[ci]
+            assert torch.equal(er, e1) and torch.equal(sr, s1) and torch.equal(ec, e0) and torch.equal(sc, s0), (si, ci)
+
+
 def test_worked_blocks_on_device():
     """The hand-worked W1 / W4 / W5 blocks straight through the kernel."""
     v = torch.zeros(32, device="cuda")
