@@ -84,7 +84,8 @@ typedef struct {
                            output of dequantize); ignored by mx_gemm          */
   int32_t scale_layout; /* mx_scale_layout_t of every scale tensor in the call */
   void* stream;         /* cudaStream_t                                        */
-  int32_t check_status; /* mx_gemm: nonzero = synchronise the stream and return
+  int32_t check_status; /* mx_gemm, and the mx_quantize / mx_quantize_dual calls that run a
+                           tile kernel: nonzero = synchronise the stream and return
                            MX_ERR_TIMEOUT if a device-side wait expired        */
   int32_t pad_k128;     /* 0 or 1.  1: MX tensors are stored as those of the float
                            tensor zero-extended along the block axis to a multiple

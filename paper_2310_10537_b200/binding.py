@@ -198,9 +198,10 @@ def mx_quantize(x: torch.Tensor, axis: int, fmt: int, rounding: int = MX_RNE,
 
 
 def mx_quantize_dual(x: torch.Tensor, fmt: int, rounding: int = MX_RNE, layout: int = MX_SCALES_SWIZZLED,
-                     out=None):
+                     out=None, check_status: bool = False):
     """Both MX tensors of a contiguous 2-D CUDA tensor in one pass: returns
-    ((elems_row, scales_row), (elems_col, scales_col)) = (mx_quantize(x, 1), mx_quantize(x, 0))."""
+    ((elems_row, scales_row), (elems_col, scales_col)) = (mx_quantize(x, 1), mx_quantize(x, 0)).
+    ``check_status``: synchronise and raise if a device-side wait of the kernel gave up."""
     assert x.is_cuda and x.is_contiguous() and x.dim() == 2
     R, C = x.shape
     if out is None:
@@ -211,7 +212,7 @@ def mx_quantize_dual(x: torch.Tensor, fmt: int, rounding: int = MX_RNE, layout: 
         sc = torch.empty(mx_scales_bytes([R, C], 0, layout), **u8)
     else:
         (er, sr), (ec, sc) = out
-    o = _opts(_dtype_code(x.dtype), layout)
+    o = _opts(_dtype_code(x.dtype), layout, check=check_status)
     _check(_lib.mx_quantize_dual(x.data_ptr(), er.data_ptr(), sr.data_ptr(), ec.data_ptr(), sc.data_ptr(),
                                  R, C, fmt, rounding, ctypes.byref(o)), "mx_quantize_dual")
     return (er, sr), (ec, sc)

@@ -149,6 +149,20 @@ const char* mx_strerror(int status) {
 
 const char* mx_last_cuda_error(void) { return g_cuda_error; }
 
+// After a launch of one of the tile kernels with opts->check_status: synchronise the stream and
+// report a bounded device-side wait that gave up.
+static int tile_status_check(cudaStream_t stream) {
+  unsigned int st = 0;
+  const cudaError_t e = mx::quantize_tile_status(stream, &st);
+  if (e != cudaSuccess) return fail_cuda(e);
+  if (st != 0) {
+    std::snprintf(g_cuda_error, sizeof(g_cuda_error), "device-side wait %u of a tile kernel gave up "
+                  "(1 a tile's copy never landed, 2 a stage was never released)", st);
+    return MX_ERR_TIMEOUT;
+  }
+  return MX_OK;
+}
+
 int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int64_t* shape,
                 int ndim, int axis, mx_fmt_t fmt, mx_round_t rounding, const mx_opts_t* opts) {
   Opts o;
@@ -189,7 +203,8 @@ int mx_quantize(const void* in, void* elems_out, uint8_t* scales_out, const int6
     d.R = v.L; d.C = v.inner; d.fmt = (int)fmt; d.rounding = (int)rounding; d.dtype = o.dtype; d.layout = o.layout;
     d.sm_count = a.sm_count; d.stream = o.stream;
     e = mx::launch_quantize_tile_cols(d);
-    return e == cudaSuccess ? MX_OK : fail_cuda(e);
+    if (e != cudaSuccess) return fail_cuda(e);
+    return o.check ? tile_status_check(o.stream) : MX_OK;
   }
   e = mx::launch_quantize(a);
   return e == cudaSuccess ? MX_OK : fail_cuda(e);
@@ -233,7 +248,8 @@ int mx_quantize_dual(const void* in, void* elems_row, uint8_t* scales_row, void*
   const bool f32_tiles = o.dtype == MX_F32 && (fmt == MX_E3M2 || fmt == MX_E2M3) && C % 128 == 0;
   e = o.dtype == MX_BF16 ? mx::launch_quantize_tile(a) : f32_tiles ? mx::launch_quantize_tile_f32(a)
                                                                    : mx::launch_quantize_dual(a);
-  return e == cudaSuccess ? MX_OK : fail_cuda(e);
+  if (e != cudaSuccess) return fail_cuda(e);
+  return (o.check && (o.dtype == MX_BF16 || f32_tiles)) ? tile_status_check(o.stream) : MX_OK;
 }
 
 int mx_dequantize(const void* elems, const uint8_t* scales, void* out, const int64_t* shape,

@@ -165,7 +165,8 @@ def test_dual_axis_quantize_matches_both_single_axis_results(fmt, dtype, R, C):
     for rounding, layout in ((mx.MX_RNE, mx.MX_SCALES_SWIZZLED), (mx.MX_RHAZ, mx.MX_SCALES_LINEAR)):
         g = [Guarded(mx.mx_elems_bytes([R, C], 1, fmt)), Guarded(mx.mx_scales_bytes([R, C], 1, layout)),
              Guarded(mx.mx_elems_bytes([R, C], 0, fmt)), Guarded(mx.mx_scales_bytes([R, C], 0, layout))]
-        mx.mx_quantize_dual(x, fmt, rounding, layout, out=((g[0].view, g[1].view), (g[2].view, g[3].view)))
+        # (check_status: the call synchronises and would report a device-side wait that gave up)
+        mx.mx_quantize_dual(x, fmt, rounding, layout, out=((g[0].view, g[1].view), (g[2].view, g[3].view)), check_status=True)
         torch.cuda.synchronize()
         for gg in g:
             gg.check()
