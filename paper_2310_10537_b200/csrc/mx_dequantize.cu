@@ -143,7 +143,37 @@ dequantize_kernel(const uint8_t* __restrict__ elems, const uint8_t* __restrict__
     }
     char* dst = reinterpret_cast<char*>(out) + (size_t)unit * 64;
     uint32_t o[16];
-    if (!special) {
+    if constexpr (FMT == MX_E2M1 && DTYPE == MX_BF16) {
+      if (!special) {
+        // 4-bit codes to BF16 without touching single elements: the eight magnitudes' BF16 bytes sit
+        // in two 8-byte tables that a byte permute indexes with four code nibbles at once (the low
+        // three bits of each; its fourth selector bit would replicate a sign, so it is masked off),
+        // the signs come from a second permute in that sign-replicating mode, and X is one packed
+        // BF16 multiply per pair (exact: the values have two significant bits and X is a power of
+        // two whose products stay normal here, sb >= 24).
+        //   magnitudes 0, 0.5, 1, 1.5, 2, 3, 4, 6 = 0x0000 3F00 3F80 3FC0 4000 4040 4080 40C0
+        const uint32_t x2 = (sb << 7) * 0x00010001u;
+#pragma unroll
+        for (int i = 0; i < kWords; ++i) {
+          const uint32_t n = w[i], mag = n & 0x77777777u, up = n << 4;
+#pragma unroll
+          for (int h = 0; h < 2; ++h) {  // codes 4 h .. 4 h + 3 of the word
+            const uint32_t sel = h ? (mag >> 16) : (mag & 0xFFFFu);
+            const uint32_t lo = __byte_perm(0xC0800000u, 0xC0804000u, sel);   // low bytes of the four values
+            uint32_t hi = __byte_perm(0x3F3F3F00u, 0x40404040u, sel);         // high bytes
+            // 0xFF where the code is negative: code 2 j + 1's sign is bit 7 of byte j of n, code 2 j's of n << 4
+            const uint32_t neg = __byte_perm(n, up, h ? 0xBFAEu : 0x9D8Cu);
+            hi |= neg & 0x80808080u;
+            const uint32_t p0 = __byte_perm(lo, hi, 0x5140), p1 = __byte_perm(lo, hi, 0x7362);
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * i + 2 * h]) : "r"(p0), "r"(x2));
+            asm("mul.rn.bf16x2 %0, %1, %2;" : "=r"(o[4 * i + 2 * h + 1]) : "r"(p1), "r"(x2));
+          }
+        }
+      }
+    }
+    if (FMT == MX_E2M1 && DTYPE == MX_BF16 && !special) {
+      // (done above)
+    } else if (!special) {
       const float fix = bias_fix<FMT>();
       uint32_t r[kElems];
 #pragma unroll
