@@ -906,6 +906,12 @@ def main_case(args):
         out = mx.mx_quantize_dual(T, fmt)
         for _ in range(reps):
             mx.mx_quantize_dual(T, fmt, out=out)
+    elif args.case == "quantize_dual_f32":   # configuration 4's X (FP32 4096 x 4096, half-away rounding)
+        T = inputs.config4("cuda")["X"]
+        fmt = mx.FORMATS[args.fmt]
+        out = mx.mx_quantize_dual(T, fmt, mx.MX_RHAZ)
+        for _ in range(reps):
+            mx.mx_quantize_dual(T, fmt, mx.MX_RHAZ, out=out)
     elif args.case == "conv":         # N 32, 56 x 56, C 256 -> 256, 3 x 3, padding 1: the operand fetched inside the GEMM
         x = torch.randn((32, 56, 56, 256), device="cuda", dtype=torch.bfloat16)
         wt = torch.randn((256, 3 * 3 * 256), device="cuda", dtype=torch.bfloat16) * 0.05
@@ -930,7 +936,7 @@ def main_case(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--case", choices=["step", "quantize", "dequantize", "quantize_strided", "gemm", "gemm_dense",
-                                       "gemm_few_rows", "quantize_dual", "im2col", "conv"],
+                                       "gemm_few_rows", "quantize_dual", "quantize_dual_f32", "im2col", "conv"],
                     default="step", help="'step' = the benchmark; the others run three launches of one "
                                          "kernel on a small case for a profiler capture")
     ap.add_argument("--fmt", choices=FMT_NAMES, default="e4m3")
