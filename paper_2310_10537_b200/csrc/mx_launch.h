@@ -30,12 +30,14 @@ struct DualArgs {
   int sm_count;
   cudaStream_t stream;
 };
+// FP32 input, register kernel (mx_quantize_dual.cu).
 cudaError_t launch_quantize_dual(const DualArgs& a);
 // The same for BF16 input through TMA tiles in shared memory (mx_quantize_tile.cu).
 cudaError_t launch_quantize_tile(const DualArgs& a);
 // FP32 input, 6-bit codes, R and C multiples of 128, through the same kind of kernel.
 cudaError_t launch_quantize_tile_f32(const DualArgs& a);
-// Its column pass alone (elems_row / scales_row unused): axis-0 quantize of a 2-D BF16 tensor, R, C % 128 == 0.
+// The BF16 kernel's column pass alone (elems_row / scales_row unused): axis-0 quantize of a 2-D BF16
+// tensor with 6- or 4-bit codes, R, C % 128 == 0.
 cudaError_t launch_quantize_tile_cols(const DualArgs& a);
 // Synchronises the stream, then reads and clears the tile kernels' status word (nonzero: a
 // bounded device-side wait gave up).

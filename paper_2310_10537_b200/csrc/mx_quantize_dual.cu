@@ -15,6 +15,8 @@
 //                  writes one contiguous 128/96/64 (BF16) or 64/48/32 (FP32) byte run of the
 //                  [R x C] output.
 // Only __syncwarp is needed: every warp has private shared-memory areas.
+// Used for FP32 input (8- and 4-bit codes, and 6-bit codes of tensors that are not whole 128 x 128
+// tiles); BF16 input and the other FP32 cases go through the tile kernels of mx_quantize_tile.cu.
 #include "mx_device.cuh"
 #include "mx_launch.h"
 #include "mx_quantize_common.cuh"
